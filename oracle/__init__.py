@@ -1,0 +1,263 @@
+"""ctypes front end of the CPU oracle (oracle/tc_oracle.c).
+
+TEST INFRASTRUCTURE ONLY: the tests, the smoke check and the benchmark's CPU-baseline leg use
+it; the CUDA package never imports it.  The wrappers only marshal numpy arrays; every step of
+the method is in the C file, which cites the paper passage each function follows.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "tc_oracle.c")
+_OUT_DIR = os.path.join(_HERE, "_build")
+_SO = os.path.join(_OUT_DIR, "libtc_oracle.so")
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (plain C, -O2, no fast-math) and return the library path."""
+    os.makedirs(_OUT_DIR, exist_ok=True)
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        tmp = _SO + f".{os.getpid()}.tmp"
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-ffp-contract=off",
+                               "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _SO)
+    return _SO
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        d, i64, i32, vp = C.c_double, C.c_int64, C.c_int, C.c_void_p
+        sig = {
+            "orc_round_bf16": (d, [d]),
+            "orc_mean_cov": (None, [vp, i64, i32, i64, vp, vp]),
+            "orc_eigh_jacobi": (i32, [vp, i32, vp, vp]),
+            "orc_fit_pca": (i32, [vp, i64, i32, i64, i32, i32, vp, vp, vp, vp, vp]),
+            "orc_project": (None, [vp, i64, i32, i64, vp, vp, i32, vp]),
+            "orc_quantize": (None, [vp, i64, d, d, i32, vp, vp]),
+            "orc_histogram": (None, [vp, i64, i32, i32, i32, vp]),
+            "orc_huffman_lengths": (i32, [vp, i32, i32, vp]),
+            "orc_huffman_lengths_raw": (i32, [vp, i32, i32, i32, vp]),
+            "orc_canonical_codes": (None, [vp, i32, vp]),
+            "orc_encode": (i64, [vp, i64, i32, i32, i32, vp, i32, i32, vp, i64, vp, vp]),
+            "orc_decode_symbols": (i32, [vp, i64, vp, vp, i64, i32, i32, i32, vp, i32, i32, vp]),
+            "orc_reconstruct": (None, [vp, i64, i32, i64, i32, vp, vp, d, d, i32, vp]),
+            "orc_entropy": (d, [vp, i32]),
+            "orc_mean_length": (d, [vp, vp, i32]),
+            "orc_mse": (d, [vp, vp, i64]),
+        }
+        for name, (res, args) in sig.items():
+            fn = getattr(_lib, name)
+            fn.restype, fn.argtypes = res, args
+    return _lib
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(C.c_void_p)
+
+
+def _f32(x) -> np.ndarray:
+    """NCHW tensor (numpy or torch, fp32 or bf16) -> contiguous float32 numpy array (exact)."""
+    if hasattr(x, "detach"):
+        x = x.detach().cpu().float().numpy()
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    assert x.ndim == 4
+    return x
+
+
+@dataclass
+class Model:
+    """Per-layer transform and quantiser: y = basis (x - mean); levels lo + q*step."""
+    c: int
+    k: int
+    bits: int
+    mean: np.ndarray      # [C] float64
+    basis: np.ndarray     # [C][C] float64, row j = j-th principal direction (first k rows used)
+    eig: np.ndarray       # [C] float64, descending
+    lo: float
+    step: float
+    basis_bf16: bool
+
+
+@dataclass
+class Stream:
+    words: np.ndarray          # uint32, padded stream
+    chunk_off: np.ndarray      # uint32 [n_chunks], bits relative to the tile start
+    tile_off: np.ndarray       # uint64 [n_tiles + 1], absolute bits, multiples of 128
+    total_bits: int
+    pixels: int
+    k: int
+    chunk_pixels: int
+    tile_chunks: int
+
+
+def round_bf16(v: float) -> float:
+    return lib().orc_round_bf16(float(v))
+
+
+def mean_cov(x):
+    x = _f32(x)
+    n, c, h, w = x.shape
+    mean = np.zeros(c)
+    cov = np.zeros((c, c))
+    lib().orc_mean_cov(_p(x), n, c, h * w, _p(mean), _p(cov))
+    return mean, cov
+
+
+def eigh_jacobi(a: np.ndarray):
+    a = np.array(a, dtype=np.float64, order="C")
+    n = a.shape[0]
+    ev = np.zeros(n)
+    vt = np.zeros((n, n))
+    sweeps = lib().orc_eigh_jacobi(_p(a), n, _p(ev), _p(vt))
+    return ev, vt, sweeps
+
+
+def fit_pca(x, bits: int, *, k: int | None = None, basis_bf16: bool = False) -> Model:
+    x = _f32(x)
+    n, c, h, w = x.shape
+    mean = np.zeros(c)
+    basis = np.zeros((c, c))
+    eig = np.zeros(c)
+    lo = C.c_double()
+    step = C.c_double()
+    rc = lib().orc_fit_pca(_p(x), n, c, h * w, bits, int(basis_bf16), _p(mean), _p(basis),
+                           _p(eig), C.byref(lo), C.byref(step))
+    if rc != 0:
+        raise RuntimeError("oracle eigensolver did not converge")
+    return Model(c, c if k is None else k, bits, mean, basis, eig, lo.value, step.value,
+                 basis_bf16)
+
+
+def project(model: Model, x) -> np.ndarray:
+    """[P][K] coefficients, P = N*H*W in pixel order p = n*HW + s."""
+    x = _f32(x)
+    n, c, h, w = x.shape
+    y = np.zeros((n * h * w, model.k))
+    lib().orc_project(_p(x), n, c, h * w, _p(model.mean), _p(model.basis), model.k, _p(y))
+    return y
+
+
+def quantize(model: Model, y: np.ndarray, *, with_units: bool = False):
+    y = np.ascontiguousarray(y, dtype=np.float64)
+    q = np.zeros(y.shape, dtype=np.uint8)
+    units = np.zeros(y.shape) if with_units else None
+    lib().orc_quantize(_p(y), y.size, model.lo, model.step, model.bits, _p(q),
+                       _p(units) if with_units else None)
+    return (q, units) if with_units else q
+
+
+def histogram(q: np.ndarray, bits: int, per_channel: bool) -> np.ndarray:
+    q = np.ascontiguousarray(q, dtype=np.uint8)
+    pixels, k = q.shape
+    groups = k if per_channel else 1
+    hist = np.zeros((groups, 1 << bits), dtype=np.uint64)
+    lib().orc_histogram(_p(q), pixels, k, groups, bits, _p(hist))
+    return hist
+
+
+def huffman_lengths(hist: np.ndarray, lmax: int = 12) -> np.ndarray:
+    """Code lengths [groups][2^bits] from counts [groups][2^bits] (weights = count + 1)."""
+    hist = np.ascontiguousarray(hist, dtype=np.uint64)
+    if hist.ndim == 1:
+        hist = hist[None, :]
+    out = np.zeros(hist.shape, dtype=np.uint8)
+    for g in range(hist.shape[0]):
+        row = np.ascontiguousarray(hist[g])
+        ln = np.zeros(hist.shape[1], dtype=np.uint8)
+        if lib().orc_huffman_lengths(_p(row), hist.shape[1], lmax, _p(ln)) != 0:
+            raise ValueError("bad alphabet size / length limit")
+        out[g] = ln
+    return out
+
+
+def huffman_lengths_raw(weights, lmax: int = 31, force_limited: bool = False) -> np.ndarray:
+    w = np.ascontiguousarray(weights, dtype=np.uint64)
+    ln = np.zeros(w.shape[0], dtype=np.uint8)
+    if lib().orc_huffman_lengths_raw(_p(w), w.shape[0], lmax, int(force_limited), _p(ln)) != 0:
+        raise ValueError("bad alphabet size / length limit")
+    return ln
+
+
+def canonical_codes(lengths: np.ndarray) -> np.ndarray:
+    ln = np.ascontiguousarray(lengths, dtype=np.uint8)
+    code = np.zeros(ln.shape[0], dtype=np.uint32)
+    lib().orc_canonical_codes(_p(ln), ln.shape[0], _p(code))
+    return code
+
+
+def encode(q: np.ndarray, lengths: np.ndarray, bits: int, *, chunk_pixels: int,
+           tile_chunks: int) -> Stream:
+    q = np.ascontiguousarray(q, dtype=np.uint8)
+    pixels, k = q.shape
+    lengths = np.ascontiguousarray(lengths, dtype=np.uint8)
+    if lengths.ndim == 1:
+        lengths = lengths[None, :]
+    groups = lengths.shape[0]
+    tile_pixels = chunk_pixels * tile_chunks
+    n_tiles = max(1, -(-pixels // tile_pixels)) if pixels else 0
+    n_chunks = -(-pixels // chunk_pixels)
+    cap_bits = pixels * k * int(lengths.max()) + 128 * (n_tiles + 1)
+    cap_words = cap_bits // 32 + 4
+    words = np.zeros(cap_words, dtype=np.uint32)
+    chunk_off = np.zeros(max(n_chunks, 1), dtype=np.uint32)
+    tile_off = np.zeros(n_tiles + 1, dtype=np.uint64)
+    total = lib().orc_encode(_p(q), pixels, k, groups, bits, _p(lengths), chunk_pixels,
+                             tile_chunks, _p(words), cap_words, _p(chunk_off), _p(tile_off))
+    if total < 0:
+        raise RuntimeError("oracle stream capacity too small")
+    return Stream(words[: total // 32].copy(), chunk_off[:n_chunks].copy(), tile_off, int(total),
+                  pixels, k, chunk_pixels, tile_chunks)
+
+
+def decode_symbols(s: Stream, lengths: np.ndarray, bits: int) -> np.ndarray:
+    lengths = np.ascontiguousarray(lengths, dtype=np.uint8)
+    if lengths.ndim == 1:
+        lengths = lengths[None, :]
+    q = np.zeros((s.pixels, s.k), dtype=np.uint8)
+    words = np.ascontiguousarray(s.words, dtype=np.uint32)
+    chunk_off = np.ascontiguousarray(s.chunk_off, dtype=np.uint32)
+    tile_off = np.ascontiguousarray(s.tile_off, dtype=np.uint64)
+    rc = lib().orc_decode_symbols(_p(words), words.shape[0], _p(chunk_off), _p(tile_off),
+                                  s.pixels, s.k, lengths.shape[0], bits, _p(lengths),
+                                  s.chunk_pixels, s.tile_chunks, _p(q))
+    if rc != 0:
+        raise ValueError("corrupt stream")
+    return q
+
+
+def reconstruct(model: Model, q: np.ndarray, shape, *, out_bf16: bool) -> np.ndarray:
+    """x_hat (NCHW float32 array holding fp32 or bf16-rounded values) from symbols [P][K]."""
+    n, c, h, w = shape
+    q = np.ascontiguousarray(q, dtype=np.uint8)
+    xhat = np.zeros((n, c, h, w), dtype=np.float32)
+    lib().orc_reconstruct(_p(q), n, c, h * w, model.k, _p(model.mean), _p(model.basis),
+                          model.lo, model.step, int(out_bf16), _p(xhat))
+    return xhat
+
+
+def entropy(hist_row: np.ndarray) -> float:
+    h = np.ascontiguousarray(hist_row, dtype=np.uint64)
+    return lib().orc_entropy(_p(h), h.shape[0])
+
+
+def mean_length(hist_row: np.ndarray, lengths_row: np.ndarray) -> float:
+    h = np.ascontiguousarray(hist_row, dtype=np.uint64)
+    ln = np.ascontiguousarray(lengths_row, dtype=np.uint8)
+    return lib().orc_mean_length(_p(h), _p(ln), h.shape[0])
+
+
+def mse(x, xhat) -> float:
+    a = _f32(x).ravel()
+    b = np.ascontiguousarray(xhat, dtype=np.float32).ravel()
+    return lib().orc_mse(_p(a), _p(b), a.shape[0])
