@@ -1,0 +1,227 @@
+/*
+ * tc.h -- C ABI of the B200 feature-map transform codec.
+ *
+ * The library encodes a dense NCHW activation tensor into a Huffman-coded bit stream and
+ * decodes it back, following the transform-coding chain of the paper (Section 3):
+ *
+ *     x -> y = T (x - mu) -> Q_Delta -> VLC -> [memory] -> VLD -> Q_Delta^-1 -> T^T -> x_hat
+ *
+ * with 1 x 1 x C blocks (Section 3.1, "Linear transform"): every pixel's C-channel vector is
+ * transformed on its own, so the transform is a dense (N*H*W) x C x C contraction.
+ *
+ * Conventions
+ *   - Every pointer says whether it is HOST or DEVICE memory.  Device pointers must belong to
+ *     the device the context was created on.  The caller owns every buffer it passes in; the
+ *     library owns only the opaque handles it returns and a small scratch arena per context.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls that
+ *     take one are asynchronous on it unless stated otherwise.
+ *   - Errors are return codes.  Argument errors are found on the host before any launch.
+ *     Conditions only the device can see (corrupt stream, output capacity exceeded at run
+ *     time, a bounded wait that ran out) are recorded in a per-context status word and
+ *     reported by tc_get_status(); the kernels never read or write out of bounds because of
+ *     them and never trap.
+ *   - There is no CPU fallback: without a CUDA device tc_create() fails.
+ *   - P = N*H*W pixels, pixel index p = (n*H + h)*W + w; K = number of coefficients kept
+ *     (K <= C); V = P*C values; b = quantiser bit width.
+ */
+#ifndef TC_H_
+#define TC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    TC_OK = 0,
+    TC_ERR_INVALID_ARG = 1,      /* null pointer, bad shape, mismatched model/codebook        */
+    TC_ERR_UNSUPPORTED = 2,      /* b outside 1..8, C > 1024, code longer than 12 bits, ...   */
+    TC_ERR_BUFFER_TOO_SMALL = 3, /* stream capacity exceeded (host check or device status)    */
+    TC_ERR_CUDA = 4,             /* a CUDA runtime call failed                                */
+    TC_ERR_CORRUPT_STREAM = 5,   /* decode found offsets or codes that cannot be valid        */
+    TC_ERR_TIMEOUT = 6,          /* a bounded device-side wait ran out                        */
+    TC_ERR_NOT_CONVERGED = 7     /* eigensolver did not converge                              */
+} tc_status;
+
+typedef enum { TC_F32 = 0, TC_BF16 = 1 } tc_dtype;
+
+/* Dense NCHW tensor in DEVICE memory. `data` must be aligned to its element size. */
+typedef struct {
+    void *data;
+    int32_t n, c, h, w;
+    int32_t dtype; /* tc_dtype */
+} tc_tensor;
+
+typedef struct tc_ctx tc_ctx;
+typedef struct tc_model tc_model;
+typedef struct tc_codebook tc_codebook;
+
+/* Context: binds a device, owns the scratch arena and the device status word. */
+tc_status tc_create(tc_ctx **out, int device);
+void tc_destroy(tc_ctx *ctx);
+const char *tc_status_string(tc_status s);
+
+/* Synchronises `cuda_stream`, returns the first device-side error recorded since the last
+ * call (TC_OK if none) and clears it. */
+tc_status tc_get_status(tc_ctx *ctx, void *cuda_stream);
+
+/* ---------------------------------------------------------------------------------------
+ * Model = per-layer transform and quantiser (Section 3; Section 3.1 "Linear transform" and
+ * "Quantization"): mean mu[C]; basis T[C][C] whose row j is the j-th principal direction of
+ * the calibration covariance (descending eigenvalue, orthonormal, T^-1 = T^T); the common
+ * quantiser step Delta and lowest level lo, taken from the range of coefficient 0 (the
+ * highest-variance channel) on the calibration maps: step = (hi - lo) / (2^b - 1).
+ * ------------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t bits;        /* b, 1..8                                                        */
+    int32_t k;           /* coefficients kept, 1..C; 0 means C                             */
+    int32_t basis_dtype; /* tc_dtype: the basis is rounded to this type at fit time and
+                            the rounded matrix is the transform from then on.  TC_BF16 is
+                            required for bf16 tensors, TC_F32 for fp32 tensors.            */
+} tc_fit_params;
+
+/* Fit on calibration maps (`calib->n` maps).  Mean and covariance (1/(M-1), M = n*h*w pixel
+ * vectors) are accumulated on the device in fp64, the eigendecomposition runs on the host,
+ * then the range of coefficient 0 is taken on the device.  Synchronous: returns after the
+ * model is complete.  Errors: INVALID_ARG, UNSUPPORTED (C > 1024 or C % 8 != 0 ... see
+ * tc_encode), NOT_CONVERGED, CUDA. */
+tc_status tc_fit_pca(tc_ctx *ctx, const tc_tensor *calib, const tc_fit_params *params,
+                     tc_model **out, void *cuda_stream);
+
+/* Plain HOST description of a model, for import/export (checkpointing, and the injection
+ * point for externally computed models).  `basis` is [C][C] row-major, rows = directions;
+ * entries must already be exactly representable in `basis_dtype` (import rejects others). */
+typedef struct {
+    int32_t c, k, bits, basis_dtype;
+    double lo, step;
+    double *basis; /* HOST [c*c] */
+    double *mean;  /* HOST [c]   */
+    double *eig;   /* HOST [c], may be NULL on import */
+} tc_model_desc;
+
+tc_status tc_model_import(tc_ctx *ctx, const tc_model_desc *desc, tc_model **out);
+/* Fills the scalar fields and, where the caller set the array pointers, the arrays. */
+tc_status tc_model_export(const tc_model *model, tc_model_desc *desc);
+void tc_model_free(tc_model *model);
+
+/* ---------------------------------------------------------------------------------------
+ * Codebook = canonical Huffman code for the quantiser output (Section 3.1, "Variable
+ * length coding").  `groups` is 1 (one table per layer) or K (one table per coefficient
+ * channel).  Lengths come from counts + 1 (every symbol has a code) by Huffman's algorithm
+ * with deterministic tie-breaking -- leaves sorted by (weight, symbol), a leaf before an
+ * internal node of equal weight -- and, if the longest code would exceed `max_length`, by the
+ * length-limited optimum (package-merge).  Codes are canonical: ordered by (length, symbol).
+ * ------------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t groups;     /* 1 or K                                  */
+    int32_t max_length; /* b..12; 0 means 12                       */
+} tc_codebook_params;
+
+/* `hist` is [groups][2^b] counts, HOST memory if hist_on_device == 0 else DEVICE memory.
+ * Synchronous. */
+tc_status tc_build_codebook(tc_ctx *ctx, const tc_model *model, const uint64_t *hist,
+                            int hist_on_device, const tc_codebook_params *params,
+                            tc_codebook **out);
+/* `lengths` is HOST [groups][2^bits]; must satisfy Kraft's equality per group and be <= 12. */
+tc_status tc_codebook_import(tc_ctx *ctx, int32_t bits, int32_t groups, const uint8_t *lengths,
+                             tc_codebook **out);
+/* `lengths` may be NULL to query bits/groups only. */
+tc_status tc_codebook_export(const tc_codebook *cb, int32_t *bits, int32_t *groups,
+                             uint8_t *lengths);
+void tc_codebook_free(tc_codebook *cb);
+
+/* Host utility behind tc_build_codebook: code lengths for one alphabet of `nsym` symbols
+ * from `counts` (weights counts + 1).  HOST pointers.  No device needed. */
+tc_status tc_host_huffman_lengths(const uint64_t *counts, int32_t nsym, int32_t max_length,
+                                  uint8_t *lengths);
+/* Host utility behind tc_fit_pca: eigendecomposition of a symmetric n x n matrix `a`
+ * (HOST, row-major, destroyed).  On return evals[] is descending and row j of `evecs`
+ * ([n][n]) is the unit eigenvector of evals[j], signed so that its largest-magnitude entry
+ * is positive.  No device needed. */
+tc_status tc_host_eigh(double *a, int32_t n, double *evals, double *evecs);
+
+/* ---------------------------------------------------------------------------------------
+ * Bit stream (the paper leaves the layout open; Section 3.1 only says the stream is
+ * accumulated in external memory).
+ *   - Symbols are emitted pixel-major: p ascending, coefficient j ascending inside a pixel,
+ *     each with the code of table j (groups == K) or table 0.
+ *   - Code bits most-significant first; stream bit i is bit 31 - (i mod 32) of the
+ *     little-endian 32-bit word i / 32.
+ *   - A chunk is `chunk_pixels` consecutive pixels (a power of two, 1..128); a tile is
+ *     128 pixels.  Tile t starts at absolute bit tile_off[t], a multiple of 128, with zero
+ *     padding before it; tile_off[n_tiles] is the padded end of the stream.  chunk_off[i]
+ *     is the start of chunk i in bits relative to the start of its tile.
+ * ------------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t chunk_pixels; /* power of two in 1..128; 0 = library default for this shape */
+} tc_encode_params;
+
+typedef struct {
+    int64_t n_tiles, n_chunks;
+    size_t stream_bytes;    /* worst case: every symbol at the longest code + padding  */
+    size_t chunk_off_bytes; /* n_chunks * 4                                            */
+    size_t tile_off_bytes;  /* (n_tiles + 1) * 8                                       */
+    int32_t chunk_pixels;   /* the value that will be used                             */
+} tc_stream_layout;
+
+/* Worst-case buffer sizes for encoding `x`. Host only. */
+tc_status tc_encode_bound(const tc_model *model, const tc_codebook *cb, const tc_tensor *x,
+                          const tc_encode_params *params, tc_stream_layout *out);
+
+/* Optional debug outputs of tc_encode (DEVICE): the projected coefficients and the symbols,
+ * which the normal path never writes to memory.  Either pointer may be NULL. */
+typedef struct {
+    float *coefficients; /* [P][K] fp32: y = T (x - mu) */
+    uint8_t *symbols;    /* [P][K]                      */
+} tc_debug_out;
+
+/* Encode (Section 3: transform, quantiser, VLC).  One pass: stage, project, quantise, look up
+ * codes, scan bit offsets, pack and store.
+ *   stream_out  DEVICE, 16-byte aligned, `capacity` bytes; any capacity is accepted -- if
+ *               the coded tensor does not fit, nothing is written past it and the status
+ *               word records TC_ERR_BUFFER_TOO_SMALL.  tc_encode_bound() never fails.
+ *   chunk_off   DEVICE uint32[n_chunks];  tile_off  DEVICE uint64[n_tiles + 1]
+ *               (tile_off[n_tiles] = total stream length in bits).
+ * Errors: INVALID_ARG, UNSUPPORTED (C > 1024, K != C with the tensor-core path, dtype /
+ * basis_dtype mismatch), CUDA. */
+tc_status tc_encode(tc_ctx *ctx, const tc_model *model, const tc_codebook *cb,
+                    const tc_tensor *x, const tc_encode_params *params, void *stream_out,
+                    size_t capacity, uint32_t *chunk_off, uint64_t *tile_off,
+                    const tc_debug_out *debug, void *cuda_stream);
+
+/* Decode (Section 3: VLD, inverse quantiser, inverse transform; no non-linearity is applied).
+ *   stream       DEVICE, 16-byte aligned, `stream_bytes` readable bytes
+ *   x_hat        caller-allocated tensor of the shape and dtype that was encoded
+ * Offsets are validated against `stream_bytes` on the device; a stream that cannot be valid
+ * sets TC_ERR_CORRUPT_STREAM in the status word and leaves the affected tile's output
+ * unspecified (but in bounds). */
+tc_status tc_decode(tc_ctx *ctx, const tc_model *model, const tc_codebook *cb, const void *stream,
+                    size_t stream_bytes, const uint32_t *chunk_off, const uint64_t *tile_off,
+                    const tc_encode_params *params, const tc_tensor *x_hat, void *cuda_stream);
+
+/* ---------------------------------------------------------------------------------------
+ * Statistics (Section 3: rate and MSE distortion D = |x - x_hat|^2 / n; Section 3.1: entropy
+ * H = -sum p log2 p as the theoretical rate; Appendix G: eigenvalue energy ratio).
+ * Synchronous.  `hist` (DEVICE, uint64 [groups][2^b], may be NULL) receives the symbol
+ * counts of `x` -- the input of tc_build_codebook.
+ * ------------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t groups;        /* in: 1 or K -- granularity of `hist`                          */
+    uint64_t *hist;        /* in: DEVICE [groups][2^b] or NULL; overwritten                */
+    double entropy;        /* out: bits/value, mean over groups of the group entropies     */
+    double mean_length;    /* out: Huffman bits/value with `cb` (0 if cb == NULL)          */
+    double mse;            /* out: mean squared error of the round trip (stored dtype)     */
+    double clamped_fraction; /* out: fraction of coefficients outside the quantiser range  */
+    double zero_fraction;  /* out: fraction of input values equal to zero                  */
+    double energy_ratio_90;/* out: fraction of eigenvalues holding 90 % of the energy      */
+} tc_stats_out;
+
+tc_status tc_stats(tc_ctx *ctx, const tc_model *model, const tc_codebook *cb, const tc_tensor *x,
+                   tc_stats_out *out, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TC_H_ */

@@ -42,7 +42,7 @@ def lib() -> C.CDLL:
             "orc_round_bf16": (d, [d]),
             "orc_mean_cov": (None, [vp, i64, i32, i64, vp, vp]),
             "orc_eigh_jacobi": (i32, [vp, i32, vp, vp]),
-            "orc_fit_pca": (i32, [vp, i64, i32, i64, i32, i32, vp, vp, vp, vp, vp]),
+            "orc_fit_pca": (i32, [vp, i64, i32, i64, i32, i32, vp, vp, vp, vp, vp, vp, vp]),
             "orc_project": (None, [vp, i64, i32, i64, vp, vp, i32, vp]),
             "orc_quantize": (None, [vp, i64, d, d, i32, vp, vp]),
             "orc_histogram": (None, [vp, i64, i32, i32, i32, vp]),
@@ -86,7 +86,7 @@ class Model:
     eig: np.ndarray       # [C] float64, descending
     lo: float
     step: float
-    basis_bf16: bool
+    basis_round: str = "f64"   # "f64", "bf16" or "f32": how the basis was rounded at fit time
 
 
 @dataclass
@@ -123,20 +123,50 @@ def eigh_jacobi(a: np.ndarray):
     return ev, vt, sweeps
 
 
-def fit_pca(x, bits: int, *, k: int | None = None, basis_bf16: bool = False) -> Model:
+JACOBI_MAX_C = 128
+
+
+def fit_pca(x, bits: int, *, k: int | None = None, basis_bf16: bool = False,
+            basis_round: str | None = None, eigensolver: str = "auto") -> Model:
+    """Fit mean, basis and quantiser range on calibration maps.
+
+    basis_round: "f64" (keep), "bf16" or "f32".  eigensolver: "jacobi" (the in-file solver),
+    "lapack" (numpy.linalg.eigh, a library primitive used as one step) or "auto" = Jacobi up
+    to JACOBI_MAX_C channels, LAPACK beyond (Jacobi needs minutes there).
+    """
     x = _f32(x)
     n, c, h, w = x.shape
+    if basis_round is None:
+        basis_round = "bf16" if basis_bf16 else "f64"
+    mode = {"f64": 0, "bf16": 1, "f32": 2}[basis_round]
+    if eigensolver == "auto":
+        eigensolver = "jacobi" if c <= JACOBI_MAX_C else "lapack"
+    pre_ev = pre_vt = None
+    if eigensolver == "lapack":
+        _, cov = mean_cov(x)
+        ev, vec = np.linalg.eigh(cov)
+        pre_ev = np.ascontiguousarray(ev)
+        pre_vt = np.ascontiguousarray(vec.T)
     mean = np.zeros(c)
     basis = np.zeros((c, c))
     eig = np.zeros(c)
     lo = C.c_double()
     step = C.c_double()
-    rc = lib().orc_fit_pca(_p(x), n, c, h * w, bits, int(basis_bf16), _p(mean), _p(basis),
-                           _p(eig), C.byref(lo), C.byref(step))
+    rc = lib().orc_fit_pca(_p(x), n, c, h * w, bits, mode,
+                           _p(pre_ev) if pre_ev is not None else None,
+                           _p(pre_vt) if pre_vt is not None else None,
+                           _p(mean), _p(basis), _p(eig), C.byref(lo), C.byref(step))
     if rc != 0:
         raise RuntimeError("oracle eigensolver did not converge")
     return Model(c, c if k is None else k, bits, mean, basis, eig, lo.value, step.value,
-                 basis_bf16)
+                 basis_round)
+
+
+def with_bits(m: Model, bits: int) -> Model:
+    """The same transform with the calibration range divided into 2^bits - 1 steps."""
+    hi = m.lo + m.step * ((1 << m.bits) - 1)
+    return Model(m.c, m.k, bits, m.mean, m.basis, m.eig, m.lo, (hi - m.lo) / ((1 << bits) - 1),
+                 m.basis_round)
 
 
 def project(model: Model, x) -> np.ndarray:

@@ -136,10 +136,14 @@ int orc_eigh_jacobi(double *a, int n, double *evals, double *vt)
  * entry of largest magnitude -- the first such on ties -- is positive); eig[c]; and the
  * quantiser range [lo, hi] = min/max over the calibration pixels of coefficient 0, the
  * highest-variance channel, with step = (hi - lo) / (2^bits - 1).
- * If basis_bf16 != 0 every entry of the basis is rounded to bfloat16 before the range pass,
- * and that rounded matrix is the transform from then on.
+ * basis_round: 0 keeps fp64; 1 rounds every entry of the basis to bfloat16, 2 to fp32 (ties to
+ * even) before the range pass, and that rounded matrix is the transform from then on.
+ * The eigendecomposition is the in-file Jacobi solver, unless the caller passes one it
+ * obtained from a library routine (pre_evals[c], pre_vt[c][c] with unit eigenvectors as rows,
+ * any order): Jacobi takes minutes beyond a few hundred channels.
  * Returns 0, or -1 if the eigensolver did not converge. */
-int orc_fit_pca(const float *x, int64_t n, int c, int64_t hw, int bits, int basis_bf16,
+int orc_fit_pca(const float *x, int64_t n, int c, int64_t hw, int bits, int basis_round,
+                const double *pre_evals, const double *pre_vt,
                 double *mean, double *basis, double *eig, double *lo, double *step)
 {
     double *cov = (double *)malloc(sizeof(double) * (size_t)c * c);
@@ -147,7 +151,13 @@ int orc_fit_pca(const float *x, int64_t n, int c, int64_t hw, int bits, int basi
     double *vt = (double *)malloc(sizeof(double) * (size_t)c * c);
     int *order = (int *)malloc(sizeof(int) * (size_t)c);
     orc_mean_cov(x, n, c, hw, mean, cov);
-    int rc = orc_eigh_jacobi(cov, c, ev, vt);
+    int rc = 0;
+    if (pre_evals && pre_vt) {
+        memcpy(ev, pre_evals, sizeof(double) * (size_t)c);
+        memcpy(vt, pre_vt, sizeof(double) * (size_t)c * c);
+    } else {
+        rc = orc_eigh_jacobi(cov, c, ev, vt);
+    }
     /* stable insertion sort of indices by descending eigenvalue */
     for (int i = 0; i < c; ++i) order[i] = i;
     for (int i = 1; i < c; ++i) {
@@ -162,7 +172,9 @@ int orc_fit_pca(const float *x, int64_t n, int c, int64_t hw, int bits, int basi
         const double sgn = (src[big] < 0.0) ? -1.0 : 1.0;
         for (int k = 0; k < c; ++k) {
             double v = sgn * src[k];
-            basis[(int64_t)j * c + k] = basis_bf16 ? orc_round_bf16(v) : v;
+            if (basis_round == 1) v = orc_round_bf16(v);
+            else if (basis_round == 2) v = (double)(float)v;
+            basis[(int64_t)j * c + k] = v;
         }
         eig[j] = ev[order[j]];
     }

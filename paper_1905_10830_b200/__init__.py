@@ -1,0 +1,10 @@
+"""B200-native feature-map transform codec (arXiv 1905.10830): thin Python binding of the
+C-ABI library in `csrc/` (declared in `include/tc.h`).  The binding only marshals arguments;
+every step of the coding path runs in the library's CUDA kernels.  torch is used for device
+memory and streams only."""
+from .binding import (  # noqa: F401
+    TcError, Context, Model, Codebook, EncodedStream, StreamLayout, Stats,
+    tc_create, tc_fit_pca, tc_model_import, tc_model_export, tc_build_codebook,
+    tc_codebook_import, tc_codebook_export, tc_encode_bound, tc_encode, tc_decode, tc_stats,
+    tc_get_status, tc_host_huffman_lengths, tc_host_eigh, library_path, load_library,
+)

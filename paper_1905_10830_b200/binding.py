@@ -1,0 +1,363 @@
+"""ctypes binding of libtc_b200.so.  Function names match the C ABI (include/tc.h)."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import numpy as np
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG, "libtc_b200.so")
+
+TC_F32, TC_BF16 = 0, 1
+_STATUS = ["ok", "invalid argument", "unsupported configuration", "output buffer too small",
+           "CUDA error", "corrupt stream", "device-side wait timed out",
+           "eigensolver did not converge"]
+
+
+class TcError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        name = _STATUS[code] if 0 <= code < len(_STATUS) else f"status {code}"
+        super().__init__(f"{where}: {name}")
+
+
+class _Tensor(C.Structure):
+    _fields_ = [("data", C.c_void_p), ("n", C.c_int32), ("c", C.c_int32), ("h", C.c_int32),
+                ("w", C.c_int32), ("dtype", C.c_int32)]
+
+
+class _FitParams(C.Structure):
+    _fields_ = [("bits", C.c_int32), ("k", C.c_int32), ("basis_dtype", C.c_int32)]
+
+
+class _ModelDesc(C.Structure):
+    _fields_ = [("c", C.c_int32), ("k", C.c_int32), ("bits", C.c_int32), ("basis_dtype", C.c_int32),
+                ("lo", C.c_double), ("step", C.c_double), ("basis", C.c_void_p),
+                ("mean", C.c_void_p), ("eig", C.c_void_p)]
+
+
+class _CodebookParams(C.Structure):
+    _fields_ = [("groups", C.c_int32), ("max_length", C.c_int32)]
+
+
+class _EncodeParams(C.Structure):
+    _fields_ = [("chunk_pixels", C.c_int32)]
+
+
+class _StreamLayout(C.Structure):
+    _fields_ = [("n_tiles", C.c_int64), ("n_chunks", C.c_int64), ("stream_bytes", C.c_size_t),
+                ("chunk_off_bytes", C.c_size_t), ("tile_off_bytes", C.c_size_t),
+                ("chunk_pixels", C.c_int32)]
+
+
+class _DebugOut(C.Structure):
+    _fields_ = [("coefficients", C.c_void_p), ("symbols", C.c_void_p)]
+
+
+class _StatsOut(C.Structure):
+    _fields_ = [("groups", C.c_int32), ("hist", C.c_void_p), ("entropy", C.c_double),
+                ("mean_length", C.c_double), ("mse", C.c_double), ("clamped_fraction", C.c_double),
+                ("zero_fraction", C.c_double), ("energy_ratio_90", C.c_double)]
+
+
+EXPORTS = ["tc_create", "tc_destroy", "tc_status_string", "tc_get_status", "tc_fit_pca",
+           "tc_model_import", "tc_model_export", "tc_model_free", "tc_build_codebook",
+           "tc_codebook_import", "tc_codebook_export", "tc_codebook_free",
+           "tc_host_huffman_lengths", "tc_host_eigh", "tc_encode_bound", "tc_encode", "tc_decode",
+           "tc_stats"]
+
+_lib = None
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library() -> C.CDLL:
+    """Load the CUDA library.  There is no fallback: a missing build is an error."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ImportError(f"{_LIB_PATH} is missing: run `python -m paper_1905_10830_b200.build` "
+                              "(there is no CPU fallback)")
+        lib = C.CDLL(_LIB_PATH)
+        vp, i32 = C.c_void_p, C.c_int32
+        P = C.POINTER
+        lib.tc_create.argtypes = [P(vp), C.c_int]
+        lib.tc_destroy.argtypes = [vp]
+        lib.tc_destroy.restype = None
+        lib.tc_status_string.argtypes = [C.c_int]
+        lib.tc_status_string.restype = C.c_char_p
+        lib.tc_get_status.argtypes = [vp, vp]
+        lib.tc_fit_pca.argtypes = [vp, P(_Tensor), P(_FitParams), P(vp), vp]
+        lib.tc_model_import.argtypes = [vp, P(_ModelDesc), P(vp)]
+        lib.tc_model_export.argtypes = [vp, P(_ModelDesc)]
+        lib.tc_model_free.argtypes = [vp]
+        lib.tc_model_free.restype = None
+        lib.tc_build_codebook.argtypes = [vp, vp, vp, C.c_int, P(_CodebookParams), P(vp)]
+        lib.tc_codebook_import.argtypes = [vp, i32, i32, vp, P(vp)]
+        lib.tc_codebook_export.argtypes = [vp, P(i32), P(i32), vp]
+        lib.tc_codebook_free.argtypes = [vp]
+        lib.tc_codebook_free.restype = None
+        lib.tc_host_huffman_lengths.argtypes = [vp, i32, i32, vp]
+        lib.tc_host_eigh.argtypes = [vp, i32, vp, vp]
+        lib.tc_encode_bound.argtypes = [vp, vp, P(_Tensor), P(_EncodeParams), P(_StreamLayout)]
+        lib.tc_encode.argtypes = [vp, vp, vp, P(_Tensor), P(_EncodeParams), vp, C.c_size_t, vp, vp,
+                                  P(_DebugOut), vp]
+        lib.tc_decode.argtypes = [vp, vp, vp, vp, C.c_size_t, vp, vp, P(_EncodeParams), P(_Tensor), vp]
+        lib.tc_stats.argtypes = [vp, vp, vp, P(_Tensor), P(_StatsOut), vp]
+        _lib = lib
+    return _lib
+
+
+def _check(code: int, where: str):
+    if code != 0:
+        raise TcError(code, where)
+
+
+def _tensor(x: torch.Tensor) -> _Tensor:
+    if not x.is_cuda or not x.is_contiguous() or x.dim() != 4:
+        raise ValueError("expected a contiguous 4-d CUDA tensor (NCHW)")
+    if x.dtype == torch.float32:
+        dt = TC_F32
+    elif x.dtype == torch.bfloat16:
+        dt = TC_BF16
+    else:
+        raise ValueError("dtype must be float32 or bfloat16")
+    n, c, h, w = x.shape
+    return _Tensor(x.data_ptr(), n, c, h, w, dt)
+
+
+def _stream_ptr(device) -> int:
+    return torch.cuda.current_stream(device).cuda_stream
+
+
+class _Handle:
+    _free = None
+
+    def __init__(self, ptr: int):
+        self.ptr = C.c_void_p(ptr)
+
+    def close(self):
+        if self.ptr:
+            getattr(load_library(), self._free)(self.ptr)
+            self.ptr = C.c_void_p(None)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Context(_Handle):
+    _free = "tc_destroy"
+
+    def __init__(self, ptr: int, device: int):
+        super().__init__(ptr)
+        self.device = device
+
+
+class Model(_Handle):
+    _free = "tc_model_free"
+
+
+class Codebook(_Handle):
+    _free = "tc_codebook_free"
+
+
+@dataclass
+class StreamLayout:
+    n_tiles: int
+    n_chunks: int
+    stream_bytes: int
+    chunk_off_bytes: int
+    tile_off_bytes: int
+    chunk_pixels: int
+
+
+@dataclass
+class EncodedStream:
+    """Device buffers written by tc_encode."""
+    words: torch.Tensor        # uint8 buffer holding the little-endian 32-bit stream words
+    chunk_off: torch.Tensor    # int32 (bit pattern of uint32) [n_chunks]
+    tile_off: torch.Tensor     # int64 (bit pattern of uint64) [n_tiles + 1]
+    layout: StreamLayout
+    coefficients: torch.Tensor | None = None
+    symbols: torch.Tensor | None = None
+
+    def total_bits(self) -> int:
+        return int(self.tile_off[-1].item())
+
+
+@dataclass
+class Stats:
+    entropy: float
+    mean_length: float
+    mse: float
+    clamped_fraction: float
+    zero_fraction: float
+    energy_ratio_90: float
+    hist: torch.Tensor | None
+
+
+def tc_create(device: int = 0) -> Context:
+    out = C.c_void_p()
+    _check(load_library().tc_create(C.byref(out), device), "tc_create")
+    return Context(out.value, device)
+
+
+def tc_get_status(ctx: Context) -> int:
+    return load_library().tc_get_status(ctx.ptr, _stream_ptr(ctx.device))
+
+
+def tc_fit_pca(ctx: Context, calib: torch.Tensor, bits: int, k: int = 0, basis_dtype: int | None = None) -> Model:
+    t = _tensor(calib)
+    params = _FitParams(bits, k, t.dtype if basis_dtype is None else basis_dtype)
+    out = C.c_void_p()
+    _check(load_library().tc_fit_pca(ctx.ptr, C.byref(t), C.byref(params), C.byref(out),
+                                     _stream_ptr(ctx.device)), "tc_fit_pca")
+    return Model(out.value)
+
+
+def tc_model_import(ctx: Context, *, basis: np.ndarray, mean: np.ndarray, lo: float, step: float, bits: int,
+                    basis_dtype: int, k: int | None = None, eig: np.ndarray | None = None) -> Model:
+    basis = np.ascontiguousarray(basis, dtype=np.float64)
+    mean = np.ascontiguousarray(mean, dtype=np.float64)
+    c = basis.shape[0]
+    eig_arr = None if eig is None else np.ascontiguousarray(eig, dtype=np.float64)
+    d = _ModelDesc(c, c if k is None else k, bits, basis_dtype, lo, step, basis.ctypes.data, mean.ctypes.data,
+                   None if eig_arr is None else eig_arr.ctypes.data)
+    out = C.c_void_p()
+    _check(load_library().tc_model_import(ctx.ptr, C.byref(d), C.byref(out)), "tc_model_import")
+    return Model(out.value)
+
+
+def tc_model_export(model: Model) -> dict:
+    d = _ModelDesc()
+    _check(load_library().tc_model_export(model.ptr, C.byref(d)), "tc_model_export")
+    basis = np.zeros((d.c, d.c))
+    mean = np.zeros(d.c)
+    eig = np.zeros(d.c)
+    d.basis, d.mean, d.eig = basis.ctypes.data, mean.ctypes.data, eig.ctypes.data
+    _check(load_library().tc_model_export(model.ptr, C.byref(d)), "tc_model_export")
+    return dict(c=d.c, k=d.k, bits=d.bits, basis_dtype=d.basis_dtype, lo=d.lo, step=d.step, basis=basis,
+                mean=mean, eig=eig)
+
+
+def tc_build_codebook(ctx: Context, model: Model, hist, *, groups: int = 1, max_length: int = 0) -> Codebook:
+    params = _CodebookParams(groups, max_length)
+    out = C.c_void_p()
+    if isinstance(hist, torch.Tensor) and hist.is_cuda:
+        if hist.dtype != torch.int64 or not hist.is_contiguous():
+            raise ValueError("device histogram must be contiguous int64 (uint64 bit pattern)")
+        ptr, on_dev = hist.data_ptr(), 1
+        keep = hist
+    else:
+        keep = np.ascontiguousarray(hist.cpu().numpy() if isinstance(hist, torch.Tensor) else hist, dtype=np.uint64)
+        ptr, on_dev = keep.ctypes.data, 0
+    _check(load_library().tc_build_codebook(ctx.ptr, model.ptr, ptr, on_dev, C.byref(params), C.byref(out)),
+           "tc_build_codebook")
+    del keep
+    return Codebook(out.value)
+
+
+def tc_codebook_import(ctx: Context, lengths: np.ndarray, bits: int) -> Codebook:
+    lengths = np.ascontiguousarray(lengths, dtype=np.uint8)
+    if lengths.ndim == 1:
+        lengths = lengths[None, :]
+    out = C.c_void_p()
+    _check(load_library().tc_codebook_import(ctx.ptr, bits, lengths.shape[0], lengths.ctypes.data, C.byref(out)),
+           "tc_codebook_import")
+    return Codebook(out.value)
+
+
+def tc_codebook_export(cb: Codebook) -> np.ndarray:
+    bits, groups = C.c_int32(), C.c_int32()
+    _check(load_library().tc_codebook_export(cb.ptr, C.byref(bits), C.byref(groups), None), "tc_codebook_export")
+    out = np.zeros((groups.value, 1 << bits.value), dtype=np.uint8)
+    _check(load_library().tc_codebook_export(cb.ptr, C.byref(bits), C.byref(groups), out.ctypes.data),
+           "tc_codebook_export")
+    return out
+
+
+def tc_host_huffman_lengths(counts: np.ndarray, max_length: int = 12) -> np.ndarray:
+    counts = np.ascontiguousarray(counts, dtype=np.uint64)
+    out = np.zeros(counts.shape[0], dtype=np.uint8)
+    _check(load_library().tc_host_huffman_lengths(counts.ctypes.data, counts.shape[0], max_length, out.ctypes.data),
+           "tc_host_huffman_lengths")
+    return out
+
+
+def tc_host_eigh(a: np.ndarray):
+    a = np.array(a, dtype=np.float64, order="C")
+    n = a.shape[0]
+    evals = np.zeros(n)
+    evecs = np.zeros((n, n))
+    _check(load_library().tc_host_eigh(a.ctypes.data, n, evals.ctypes.data, evecs.ctypes.data), "tc_host_eigh")
+    return evals, evecs
+
+
+def tc_encode_bound(model: Model, cb: Codebook, x: torch.Tensor, chunk_pixels: int = 0) -> StreamLayout:
+    t = _tensor(x)
+    p = _EncodeParams(chunk_pixels)
+    lay = _StreamLayout()
+    _check(load_library().tc_encode_bound(model.ptr, cb.ptr, C.byref(t), C.byref(p), C.byref(lay)), "tc_encode_bound")
+    return StreamLayout(lay.n_tiles, lay.n_chunks, lay.stream_bytes, lay.chunk_off_bytes, lay.tile_off_bytes,
+                        lay.chunk_pixels)
+
+
+def tc_encode(ctx: Context, model: Model, cb: Codebook, x: torch.Tensor, *, chunk_pixels: int = 0,
+              out: EncodedStream | None = None, capacity: int | None = None, debug: bool = False,
+              k: int | None = None) -> EncodedStream:
+    """Encode `x`.  Buffers are allocated with torch (worst-case size) unless `out` is given."""
+    t = _tensor(x)
+    lay = tc_encode_bound(model, cb, x, chunk_pixels)
+    dev = x.device
+    if out is None:
+        nbytes = lay.stream_bytes if capacity is None else capacity
+        out = EncodedStream(torch.empty(max(nbytes, 16), dtype=torch.uint8, device=dev),
+                            torch.empty(max(lay.n_chunks, 1), dtype=torch.int32, device=dev),
+                            torch.empty(lay.n_tiles + 1, dtype=torch.int64, device=dev), lay)
+    dbg = None
+    if debug:
+        pixels = t.n * t.h * t.w
+        kk = t.c if k is None else k
+        out.coefficients = torch.empty(pixels, kk, dtype=torch.float32, device=dev)
+        out.symbols = torch.empty(pixels, kk, dtype=torch.uint8, device=dev)
+        dbg = _DebugOut(out.coefficients.data_ptr(), out.symbols.data_ptr())
+    p = _EncodeParams(chunk_pixels)
+    cap = out.words.numel() if capacity is None else min(capacity, out.words.numel())
+    _check(load_library().tc_encode(ctx.ptr, model.ptr, cb.ptr, C.byref(t), C.byref(p), out.words.data_ptr(), cap,
+                                    out.chunk_off.data_ptr(), out.tile_off.data_ptr(),
+                                    C.byref(dbg) if dbg is not None else None, _stream_ptr(ctx.device)), "tc_encode")
+    return out
+
+
+def tc_decode(ctx: Context, model: Model, cb: Codebook, enc: EncodedStream, shape, dtype, *,
+              out: torch.Tensor | None = None, stream_bytes: int | None = None) -> torch.Tensor:
+    if out is None:
+        out = torch.empty(shape, dtype=dtype, device=enc.words.device)
+    t = _tensor(out)
+    p = _EncodeParams(enc.layout.chunk_pixels)
+    nbytes = enc.words.numel() if stream_bytes is None else stream_bytes
+    _check(load_library().tc_decode(ctx.ptr, model.ptr, cb.ptr, enc.words.data_ptr(), nbytes,
+                                    enc.chunk_off.data_ptr(), enc.tile_off.data_ptr(), C.byref(p), C.byref(t),
+                                    _stream_ptr(ctx.device)), "tc_decode")
+    return out
+
+
+def tc_stats(ctx: Context, model: Model, cb: Codebook | None, x: torch.Tensor, *, groups: int = 1,
+             want_hist: bool = True) -> Stats:
+    t = _tensor(x)
+    exp = tc_model_export(model)
+    hist = None
+    if want_hist:
+        hist = torch.zeros(groups, 1 << exp["bits"], dtype=torch.int64, device=x.device)
+    s = _StatsOut(groups, hist.data_ptr() if hist is not None else None, 0, 0, 0, 0, 0, 0)
+    _check(load_library().tc_stats(ctx.ptr, model.ptr, cb.ptr if cb is not None else None, C.byref(t), C.byref(s),
+                                   _stream_ptr(ctx.device)), "tc_stats")
+    return Stats(s.entropy, s.mean_length, s.mse, s.clamped_fraction, s.zero_fraction, s.energy_ratio_90, hist)

@@ -1,0 +1,311 @@
+// Exact (fp64) encode and decode kernels: one thread per pixel, plain FMA-free double
+// arithmetic in the order the definition states, so that fp32 tensors -- whose products do not
+// fit the bf16 tensor-core path -- are coded without any rounding of their own.  They are
+// also the path for shapes the tensor-core kernels do not take, and for the statistics mode.
+//
+// Encode (Section 3: transform, quantiser, VLC): y_j = sum_c T[j][c] (x_c - mu_c),
+// q = clamp(rint((y - lo)/step)), code lookup, bit offsets by scan + tile look-back, pack.
+// Decode (Section 3: VLD, inverse quantiser, inverse transform): table-driven canonical
+// Huffman decode per chunk, y_hat = lo + q*step, x_hat_c = sum_j T[j][c] y_hat_j + mu_c.
+#include "device_utils.cuh"
+
+namespace {
+
+constexpr int kThreads = TC_TILE_PIXELS;
+constexpr int kRowBlock = 8;           // basis rows (encode) / columns (decode) per pass
+constexpr int kEncSmemEntries = 2048;  // code tables up to this many entries are staged
+
+using namespace tcdev;
+
+template <typename TIn>
+__global__ void __launch_bounds__(kThreads) encode_simt_kernel(EncodeArgs a)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    double *s_mean = reinterpret_cast<double *>(smem_raw);            // [C]
+    double *s_panel = s_mean + a.c;                                    // [kRowBlock][C]
+    uint32_t *s_enc = reinterpret_cast<uint32_t *>(s_panel + kRowBlock * a.c);
+    const int nsym = 1 << a.bits;
+    const int enc_entries = a.groups * nsym;
+    const bool enc_in_smem = enc_entries <= kEncSmemEntries;
+    uint8_t *s_q = reinterpret_cast<uint8_t *>(s_enc + (enc_in_smem ? enc_entries : 0));  // [K][128]
+
+    __shared__ long long s_tile;
+    __shared__ unsigned int s_warp_sums[4];
+    __shared__ unsigned long long s_base;
+    __shared__ int s_write_ok;
+
+    const int t = threadIdx.x;
+    if (t == 0) s_tile = a.emit ? (long long)atomicAdd(a.ticket, 1u) : (long long)blockIdx.x;
+    for (int i = t; i < a.c; i += kThreads) s_mean[i] = a.mean64[i];
+    if (enc_in_smem)
+        for (int i = t; i < enc_entries; i += kThreads) s_enc[i] = a.enc[i];
+    __syncthreads();
+    const long long tile = s_tile;
+    const uint32_t *enc = enc_in_smem ? s_enc : a.enc;
+
+    const long long p = tile * TC_TILE_PIXELS + t;
+    const bool valid = p < a.pixels;
+    const TIn *xin = reinterpret_cast<const TIn *>(a.x);
+    long long xbase = 0;
+    if (valid) {
+        const long long img = p / a.hw;
+        const long long s = p - img * a.hw;
+        xbase = img * a.c * (long long)a.hw + s;
+    }
+    const double top = (double)(nsym - 1);
+    unsigned int clamped = 0;
+
+    for (int j0 = 0; j0 < a.k; j0 += kRowBlock) {
+        __syncthreads();
+        for (int i = t; i < kRowBlock * a.c; i += kThreads) {
+            const int jj = i / a.c, cc = i - jj * a.c;
+            s_panel[i] = (j0 + jj < a.k) ? a.basis64[(long long)(j0 + jj) * a.c + cc] : 0.0;
+        }
+        __syncthreads();
+        if (valid) {
+            double acc[kRowBlock];
+#pragma unroll
+            for (int jj = 0; jj < kRowBlock; ++jj) acc[jj] = 0.0;
+            for (int cc = 0; cc < a.c; ++cc) {
+                const double d = __dsub_rn(load_as_double(xin + xbase + (long long)cc * a.hw), s_mean[cc]);
+#pragma unroll
+                for (int jj = 0; jj < kRowBlock; ++jj)
+                    acc[jj] = __dadd_rn(acc[jj], __dmul_rn(s_panel[jj * a.c + cc], d));
+            }
+#pragma unroll
+            for (int jj = 0; jj < kRowBlock; ++jj) {
+                const int j = j0 + jj;
+                if (j < a.k) {
+                    const double y = acc[jj];
+                    const double u = __ddiv_rn(__dsub_rn(y, a.lo), a.step);
+                    double r = rint(u);
+                    if (u < 0.0 || u > top) ++clamped;
+                    r = fmin(fmax(r, 0.0), top);
+                    const unsigned int q = (unsigned int)r;
+                    s_q[j * kThreads + t] = (uint8_t)q;
+                    if (a.dbg_coef) a.dbg_coef[p * a.k + j] = (float)y;
+                    if (a.dbg_sym) a.dbg_sym[p * a.k + j] = (uint8_t)q;
+                }
+            }
+        }
+    }
+    if (a.clamped) {
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) clamped += __shfl_xor_sync(0xffffffffu, clamped, d);
+        if ((t & 31) == 0 && clamped) atomicAdd(a.clamped, (unsigned long long)clamped);
+    }
+    if (!a.emit) return;
+
+    // ---- bit lengths, offsets --------------------------------------------------------
+    unsigned int my_bits = 0;
+    if (valid)
+        for (int j = 0; j < a.k; ++j) {
+            const int g = (a.groups == 1) ? 0 : j;
+            my_bits += enc[g * nsym + s_q[j * kThreads + t]] & 0xffu;
+        }
+    unsigned int tile_bits;
+    const unsigned int my_off = group_exclusive_scan_128(my_bits, s_warp_sums, t, 1, tile_bits);
+    const unsigned long long padded = ((unsigned long long)tile_bits + 127ull) & ~127ull;
+    if (t < 32) {
+        bool ok;
+        const unsigned long long base = tile_lookback(a.tile_state, tile, padded, a.status, ok);
+        if (t == 0) {
+            bool fits = base + padded <= a.capacity_bits;
+            if (ok && !fits) tc_dev_set_status(a.status, TC_ERR_BUFFER_TOO_SMALL);
+            s_base = base;
+            s_write_ok = (ok && fits) ? 1 : 0;
+            a.tile_off[tile] = base;
+            if (tile == a.n_tiles - 1) a.tile_off[a.n_tiles] = base + padded;
+        }
+    }
+    __syncthreads();
+    const unsigned long long base = s_base;
+    if (valid && (p % a.chunk_pixels) == 0) a.chunk_off[p / a.chunk_pixels] = my_off;
+    if (!s_write_ok) return;
+
+    // ---- zero the tile's words, then pack --------------------------------------------
+    {
+        uint4 *dst = reinterpret_cast<uint4 *>(a.stream + (base >> 5));
+        const unsigned int n16 = (unsigned int)(padded >> 7);
+        for (unsigned int i = t; i < n16; i += kThreads) dst[i] = make_uint4(0u, 0u, 0u, 0u);
+    }
+    __syncthreads();
+    if (valid) {
+        BitWriter w;
+        w.init(a.stream, base + my_off);
+        for (int j = 0; j < a.k; ++j) {
+            const int g = (a.groups == 1) ? 0 : j;
+            const uint32_t e = enc[g * nsym + s_q[j * kThreads + t]];
+            w.put(e >> 8, (int)(e & 0xffu));
+        }
+        w.finish();
+    }
+}
+
+// Sequential reader of an MSB-first bit stream with a 64-bit window; words past `end_word`
+// read as zero so that a corrupt offset can never cause an out-of-bounds load.
+struct BitReader {
+    const uint32_t *words;
+    unsigned long long window;   // upcoming bits, left-aligned
+    int avail;
+    unsigned long long next_word, end_word;
+
+    __device__ __forceinline__ uint32_t fetch()
+    {
+        const uint32_t v = (next_word < end_word) ? __ldg(words + next_word) : 0u;
+        ++next_word;
+        return v;
+    }
+    __device__ __forceinline__ void init(const uint32_t *base, unsigned long long bitpos, unsigned long long end_bits)
+    {
+        words = base;
+        next_word = bitpos >> 5;
+        end_word = end_bits >> 5;
+        const unsigned long long hi = fetch();
+        const unsigned long long lo = fetch();
+        const int sh = (int)(bitpos & 31);
+        window = ((hi << 32) | lo) << sh;
+        avail = 64 - sh;
+    }
+    __device__ __forceinline__ uint32_t peek(int nbits) const { return (uint32_t)(window >> (64 - nbits)); }
+    __device__ __forceinline__ void skip(int nbits)
+    {
+        window <<= nbits;
+        avail -= nbits;
+        if (avail <= 32) {
+            window |= (unsigned long long)fetch() << (32 - avail);
+            avail += 32;
+        }
+    }
+};
+
+template <typename TOut>
+__global__ void __launch_bounds__(kThreads) decode_simt_kernel(DecodeArgs a)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    double *s_mean = reinterpret_cast<double *>(smem_raw);        // [C]
+    double *s_panel = s_mean + a.c;                                // [K][kRowBlock]
+    uint8_t *s_q = reinterpret_cast<uint8_t *>(s_panel + (size_t)a.k * kRowBlock);   // [K][128]
+    __shared__ int s_bad;
+
+    const int t = threadIdx.x;
+    const long long tile = blockIdx.x;
+    const long long p = tile * TC_TILE_PIXELS + t;
+    const bool valid = p < a.pixels;
+    for (int i = t; i < a.c; i += kThreads) s_mean[i] = a.mean64[i];
+    if (t == 0) s_bad = 0;
+    __syncthreads();
+
+    if (a.symbols) {
+        if (valid)
+            for (int j = 0; j < a.k; ++j) s_q[j * kThreads + t] = a.symbols[p * a.k + j];
+    } else {
+        const unsigned long long base = a.tile_off[tile], end = a.tile_off[tile + 1];
+        const bool tile_ok = (base & 127ull) == 0 && (end & 127ull) == 0 && base <= end && end <= a.stream_bits;
+        if (!tile_ok) {
+            if (t == 0) tc_dev_set_status(a.status, TC_ERR_CORRUPT_STREAM);
+            return;
+        }
+        const int chunks_per_tile = TC_TILE_PIXELS / a.chunk_pixels;
+        const long long ch = tile * chunks_per_tile + t;
+        if (t < chunks_per_tile && ch < a.n_chunks) {
+            const unsigned long long off = a.chunk_off[ch];
+            bool bad = base + off > end;
+            if (!bad) {
+                BitReader r;
+                r.init(a.stream, base + off, end);
+                unsigned long long used = base + off;
+                const int lut_size = 1 << a.lut_bits;
+                const int first_pixel = t * a.chunk_pixels;
+                for (int pp = 0; pp < a.chunk_pixels; ++pp) {
+                    if (tile * TC_TILE_PIXELS + first_pixel + pp >= a.pixels) break;
+                    for (int j = 0; j < a.k; ++j) {
+                        const int g = (a.groups == 1) ? 0 : j;
+                        const uint32_t e = __ldg(a.lut + (size_t)g * lut_size + r.peek(a.lut_bits));
+                        const int len = (int)(e & 0xffu);
+                        s_q[j * kThreads + first_pixel + pp] = (uint8_t)(e >> 8);
+                        r.skip(len);
+                        used += len;
+                        if (len == 0) bad = true;
+                    }
+                }
+                if (used > end) bad = true;
+            }
+            if (bad) s_bad = 1;
+        }
+        __syncthreads();
+        if (s_bad) {
+            if (t == 0) tc_dev_set_status(a.status, TC_ERR_CORRUPT_STREAM);
+            return;
+        }
+    }
+
+    TOut *out = reinterpret_cast<TOut *>(a.xhat);
+    long long obase = 0;
+    if (valid) {
+        const long long img = p / a.hw;
+        const long long s = p - img * a.hw;
+        obase = img * a.c * (long long)a.hw + s;
+    }
+    for (int c0 = 0; c0 < a.c; c0 += kRowBlock) {
+        __syncthreads();
+        for (int i = t; i < a.k * kRowBlock; i += kThreads) {
+            const int j = i / kRowBlock, cc = i - j * kRowBlock;
+            s_panel[i] = (c0 + cc < a.c) ? a.basis64[(long long)j * a.c + c0 + cc] : 0.0;
+        }
+        __syncthreads();
+        if (valid) {
+            double acc[kRowBlock];
+#pragma unroll
+            for (int cc = 0; cc < kRowBlock; ++cc) acc[cc] = 0.0;
+            for (int j = 0; j < a.k; ++j) {
+                const double yh = __dadd_rn(a.lo, __dmul_rn((double)s_q[j * kThreads + t], a.step));
+#pragma unroll
+                for (int cc = 0; cc < kRowBlock; ++cc)
+                    acc[cc] = __dadd_rn(acc[cc], __dmul_rn(s_panel[j * kRowBlock + cc], yh));
+            }
+#pragma unroll
+            for (int cc = 0; cc < kRowBlock; ++cc)
+                if (c0 + cc < a.c)
+                    store_rounded(out + obase + (long long)(c0 + cc) * a.hw, __dadd_rn(acc[cc], s_mean[c0 + cc]));
+        }
+    }
+}
+
+size_t encode_smem_bytes(const EncodeArgs &a)
+{
+    const int entries = a.groups << a.bits;
+    return sizeof(double) * (size_t)a.c * (1 + kRowBlock) + (entries <= kEncSmemEntries ? entries * 4u : 0u) +
+           (size_t)a.k * kThreads;
+}
+size_t decode_smem_bytes(const DecodeArgs &a)
+{
+    return sizeof(double) * ((size_t)a.c + (size_t)a.k * kRowBlock) + (size_t)a.k * kThreads;
+}
+
+template <typename K, typename A>
+tc_status launch(K kernel, const A &a, size_t smem, const tc_ctx *ctx, cudaStream_t s)
+{
+    if (a.n_tiles <= 0) return TC_OK;
+    if (smem > (size_t)ctx->max_smem_optin) return TC_ERR_UNSUPPORTED;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return TC_ERR_CUDA;
+    kernel<<<(unsigned int)a.n_tiles, kThreads, smem, s>>>(a);
+    return cudaGetLastError() == cudaSuccess ? TC_OK : TC_ERR_CUDA;
+}
+
+}  // namespace
+
+tc_status tc_launch_encode_simt(const tc_ctx *ctx, const EncodeArgs &a, int dtype, cudaStream_t s)
+{
+    const size_t smem = encode_smem_bytes(a);
+    if (dtype == TC_F32) return launch(encode_simt_kernel<float>, a, smem, ctx, s);
+    return launch(encode_simt_kernel<__nv_bfloat16>, a, smem, ctx, s);
+}
+
+tc_status tc_launch_decode_simt(const tc_ctx *ctx, const DecodeArgs &a, int dtype, cudaStream_t s)
+{
+    const size_t smem = decode_smem_bytes(a);
+    if (dtype == TC_F32) return launch(decode_simt_kernel<float>, a, smem, ctx, s);
+    return launch(decode_simt_kernel<__nv_bfloat16>, a, smem, ctx, s);
+}

@@ -1,0 +1,605 @@
+// Host side of the C ABI declared in include/tc.h: handles, argument checks, table building
+// and kernel launches.  No step of the coding path runs on the host.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "tc_internal.h"
+
+#define TC_CUDA(call)                                   \
+    do {                                                \
+        if ((call) != cudaSuccess) { cudaGetLastError(); return TC_ERR_CUDA; } \
+    } while (0)
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+double round_to_dtype(double v, int dtype)
+{
+    if (dtype == TC_F32) return (double)(float)v;
+    if (v == 0.0 || !std::isfinite(v)) return v;
+    int e;
+    const double f = std::frexp(v, &e);                 // |f| in [0.5, 1)
+    int shift = 8;                                      // 8 significant bits
+    if (e - 8 < -133) shift = e + 133;                  // bfloat16 subnormals
+    return std::ldexp(std::nearbyint(std::ldexp(f, shift)), e - shift);
+}
+
+template <typename T>
+tc_status upload(T **dst, const std::vector<T> &src)
+{
+    *dst = nullptr;
+    if (src.empty()) return TC_OK;
+    TC_CUDA(cudaMalloc((void **)dst, src.size() * sizeof(T)));
+    TC_CUDA(cudaMemcpy(*dst, src.data(), src.size() * sizeof(T), cudaMemcpyHostToDevice));
+    return TC_OK;
+}
+
+bool valid_tensor(const tc_tensor *t)
+{
+    return t && t->n >= 0 && t->c > 0 && t->h > 0 && t->w > 0 && (t->dtype == TC_F32 || t->dtype == TC_BF16) &&
+           (t->data != nullptr || t->n == 0);
+}
+
+int default_chunk_pixels(int k)
+{
+    int cp = 1;
+    while (cp < TC_TILE_PIXELS && cp * k < 256) cp <<= 1;
+    return cp;
+}
+
+bool resolve_chunk_pixels(const tc_encode_params *p, int k, int *out)
+{
+    int cp = (p && p->chunk_pixels) ? p->chunk_pixels : default_chunk_pixels(k);
+    if (cp < 1 || cp > TC_TILE_PIXELS || (cp & (cp - 1)) != 0) return false;
+    *out = cp;
+    return true;
+}
+
+tc_status ensure_scratch(tc_ctx *ctx, size_t bytes)
+{
+    if (bytes <= ctx->scratch_bytes) return TC_OK;
+    if (ctx->scratch) { TC_CUDA(cudaDeviceSynchronize()); cudaFree(ctx->scratch); ctx->scratch = nullptr; ctx->scratch_bytes = 0; }
+    size_t want = std::max<size_t>(bytes, 1 << 20);
+    TC_CUDA(cudaMalloc(&ctx->scratch, want));
+    ctx->scratch_bytes = want;
+    return TC_OK;
+}
+
+tc_status finish_model(tc_model *m)
+{
+    const int c = m->c, k = m->k;
+    std::vector<double> tmu(k, 0.0), colsum(c, 0.0);
+    for (int j = 0; j < k; ++j) {
+        double s = 0.0;
+        for (int a = 0; a < c; ++a) s += m->basis[(size_t)j * c + a] * m->mean[a];
+        tmu[j] = s;
+        for (int a = 0; a < c; ++a) colsum[a] += m->basis[(size_t)j * c + a];
+    }
+    std::vector<float> enc_bias(k), dec_bias(c);
+    for (int j = 0; j < k; ++j) enc_bias[j] = (float)(-(tmu[j] + m->lo) / m->step);
+    for (int a = 0; a < c; ++a) dec_bias[a] = (float)(m->mean[a] + m->lo * colsum[a]);
+    tc_status st;
+    if ((st = upload(&m->d_basis64, m->basis)) != TC_OK) return st;
+    if ((st = upload(&m->d_mean64, m->mean)) != TC_OK) return st;
+    if ((st = upload(&m->d_enc_bias, enc_bias)) != TC_OK) return st;
+    if ((st = upload(&m->d_dec_bias, dec_bias)) != TC_OK) return st;
+    if (m->basis_dtype == TC_BF16) {
+        std::vector<__nv_bfloat16> b((size_t)k * c), bt((size_t)c * k);
+        for (int j = 0; j < k; ++j)
+            for (int a = 0; a < c; ++a) {
+                const __nv_bfloat16 v = __float2bfloat16((float)m->basis[(size_t)j * c + a]);
+                b[(size_t)j * c + a] = v;
+                bt[(size_t)a * k + j] = v;
+            }
+        if ((st = upload(&m->d_basis_bf16, b)) != TC_OK) return st;
+        if ((st = upload(&m->d_basis_t_bf16, bt)) != TC_OK) return st;
+    }
+    return TC_OK;
+}
+
+tc_status finish_codebook(tc_codebook *cb)
+{
+    const int nsym = 1 << cb->bits;
+    int mx = 0;
+    for (uint8_t l : cb->lengths) mx = std::max<int>(mx, l);
+    cb->max_len = mx;
+    cb->lut_bits = mx;
+    std::vector<uint32_t> enc((size_t)cb->groups * nsym);
+    std::vector<uint16_t> lut((size_t)cb->groups << cb->lut_bits);
+    std::vector<uint32_t> code(nsym);
+    for (int g = 0; g < cb->groups; ++g) {
+        const uint8_t *len = cb->lengths.data() + (size_t)g * nsym;
+        tc_canonical_codes_host(len, nsym, code.data());
+        for (int s = 0; s < nsym; ++s) {
+            enc[(size_t)g * nsym + s] = (code[s] << 8) | len[s];
+            // every table index whose leading bits equal the code decodes to this symbol
+            const uint32_t first = code[s] << (cb->lut_bits - len[s]);
+            const uint32_t span = 1u << (cb->lut_bits - len[s]);
+            for (uint32_t i = 0; i < span; ++i)
+                lut[((size_t)g << cb->lut_bits) + first + i] = (uint16_t)((s << 8) | len[s]);
+        }
+    }
+    tc_status st;
+    if ((st = upload(&cb->d_enc, enc)) != TC_OK) return st;
+    return upload(&cb->d_lut, lut);
+}
+
+bool kraft_complete(const uint8_t *len, int nsym, int lmax)
+{
+    unsigned long long sum = 0;
+    for (int s = 0; s < nsym; ++s) {
+        if (len[s] < 1 || len[s] > lmax) return false;
+        sum += 1ull << (lmax - len[s]);
+    }
+    return sum == (1ull << lmax);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *tc_status_string(tc_status s)
+{
+    switch (s) {
+        case TC_OK: return "ok";
+        case TC_ERR_INVALID_ARG: return "invalid argument";
+        case TC_ERR_UNSUPPORTED: return "unsupported configuration";
+        case TC_ERR_BUFFER_TOO_SMALL: return "output buffer too small";
+        case TC_ERR_CUDA: return "CUDA error";
+        case TC_ERR_CORRUPT_STREAM: return "corrupt stream";
+        case TC_ERR_TIMEOUT: return "device-side wait timed out";
+        case TC_ERR_NOT_CONVERGED: return "eigensolver did not converge";
+    }
+    return "unknown status";
+}
+
+tc_status tc_create(tc_ctx **out, int device)
+{
+    if (!out) return TC_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) {
+        cudaGetLastError();
+        return TC_ERR_CUDA;
+    }
+    DeviceGuard guard(device);
+    if (!guard.ok) return TC_ERR_CUDA;
+    tc_ctx *ctx = new (std::nothrow) tc_ctx();
+    if (!ctx) return TC_ERR_CUDA;
+    ctx->device = device;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return TC_ERR_CUDA; }
+    ctx->sm_count = prop.multiProcessorCount;
+    ctx->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
+    if (cudaMalloc((void **)&ctx->d_status, 64) != cudaSuccess || cudaMemset(ctx->d_status, 0, 64) != cudaSuccess) {
+        cudaGetLastError();
+        delete ctx;
+        return TC_ERR_CUDA;
+    }
+    *out = ctx;
+    return TC_OK;
+}
+
+void tc_destroy(tc_ctx *ctx)
+{
+    if (!ctx) return;
+    DeviceGuard guard(ctx->device);
+    cudaDeviceSynchronize();
+    if (ctx->scratch) cudaFree(ctx->scratch);
+    if (ctx->d_status) cudaFree(ctx->d_status);
+    delete ctx;
+}
+
+tc_status tc_get_status(tc_ctx *ctx, void *cuda_stream)
+{
+    if (!ctx) return TC_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    unsigned int word = 0;
+    TC_CUDA(cudaMemcpyAsync(&word, ctx->d_status, sizeof(word), cudaMemcpyDeviceToHost, s));
+    TC_CUDA(cudaStreamSynchronize(s));
+    if (word != 0) {
+        TC_CUDA(cudaMemsetAsync(ctx->d_status, 0, sizeof(word), s));
+        TC_CUDA(cudaStreamSynchronize(s));
+    }
+    return (tc_status)word;
+}
+
+// ---- model ------------------------------------------------------------------------------
+
+tc_status tc_model_import(tc_ctx *ctx, const tc_model_desc *d, tc_model **out)
+{
+    if (!ctx || !d || !out || !d->basis || !d->mean) return TC_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (d->c < 1 || d->k < 1 || d->k > d->c || !(d->step > 0.0) || !std::isfinite(d->lo)) return TC_ERR_INVALID_ARG;
+    if (d->bits < 1 || d->bits > 8 || d->c > TC_MAX_C) return TC_ERR_UNSUPPORTED;
+    if (d->basis_dtype != TC_F32 && d->basis_dtype != TC_BF16) return TC_ERR_INVALID_ARG;
+    for (size_t i = 0; i < (size_t)d->c * d->c; ++i)
+        if (round_to_dtype(d->basis[i], d->basis_dtype) != d->basis[i]) return TC_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    tc_model *m = new (std::nothrow) tc_model();
+    if (!m) return TC_ERR_CUDA;
+    m->c = d->c; m->k = d->k; m->bits = d->bits; m->basis_dtype = d->basis_dtype;
+    m->lo = d->lo; m->step = d->step; m->device = ctx->device;
+    m->basis.assign(d->basis, d->basis + (size_t)d->c * d->c);
+    m->mean.assign(d->mean, d->mean + d->c);
+    if (d->eig) m->eig.assign(d->eig, d->eig + d->c); else m->eig.assign(d->c, 0.0);
+    tc_status st = finish_model(m);
+    if (st != TC_OK) { tc_model_free(m); return st; }
+    *out = m;
+    return TC_OK;
+}
+
+tc_status tc_model_export(const tc_model *m, tc_model_desc *d)
+{
+    if (!m || !d) return TC_ERR_INVALID_ARG;
+    d->c = m->c; d->k = m->k; d->bits = m->bits; d->basis_dtype = m->basis_dtype;
+    d->lo = m->lo; d->step = m->step;
+    if (d->basis) std::copy(m->basis.begin(), m->basis.end(), d->basis);
+    if (d->mean) std::copy(m->mean.begin(), m->mean.end(), d->mean);
+    if (d->eig) std::copy(m->eig.begin(), m->eig.end(), d->eig);
+    return TC_OK;
+}
+
+void tc_model_free(tc_model *m)
+{
+    if (!m) return;
+    DeviceGuard guard(m->device);
+    cudaFree(m->d_basis64); cudaFree(m->d_mean64); cudaFree(m->d_basis_bf16);
+    cudaFree(m->d_basis_t_bf16); cudaFree(m->d_enc_bias); cudaFree(m->d_dec_bias);
+    delete m;
+}
+
+tc_status tc_fit_pca(tc_ctx *ctx, const tc_tensor *calib, const tc_fit_params *params, tc_model **out, void *cuda_stream)
+{
+    if (!ctx || !out || !params || !valid_tensor(calib)) return TC_ERR_INVALID_ARG;
+    *out = nullptr;
+    const int c = calib->c, hw = calib->h * calib->w, n = calib->n;
+    const long long m_samples = (long long)n * hw;
+    if (m_samples < 2) return TC_ERR_INVALID_ARG;
+    if (params->bits < 1 || params->bits > 8 || c > TC_MAX_C) return TC_ERR_UNSUPPORTED;
+    const int k = params->k ? params->k : c;
+    if (k < 1 || k > c) return TC_ERR_INVALID_ARG;
+    if (params->basis_dtype != TC_F32 && params->basis_dtype != TC_BF16) return TC_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+
+    const int range_blocks = tc_range0_max_blocks(m_samples);
+    const size_t n_doubles = (size_t)c + (size_t)c * c + (size_t)c + 2 * (size_t)range_blocks;
+    double *d_buf = nullptr;
+    TC_CUDA(cudaMalloc((void **)&d_buf, n_doubles * sizeof(double)));
+    double *d_mean = d_buf, *d_cov = d_buf + c, *d_row0 = d_cov + (size_t)c * c, *d_minmax = d_row0 + c;
+    struct Free { double *p; ~Free() { cudaFree(p); } } freer{d_buf};
+    TC_CUDA(cudaMemsetAsync(d_buf, 0, n_doubles * sizeof(double), s));
+
+    tc_status st = tc_launch_channel_sums(calib->data, calib->dtype, n, c, hw, d_mean, s);
+    if (st != TC_OK) return st;
+    std::vector<double> mean(c);
+    TC_CUDA(cudaMemcpyAsync(mean.data(), d_mean, sizeof(double) * c, cudaMemcpyDeviceToHost, s));
+    TC_CUDA(cudaStreamSynchronize(s));
+    for (double &v : mean) v /= (double)m_samples;
+    TC_CUDA(cudaMemcpyAsync(d_mean, mean.data(), sizeof(double) * c, cudaMemcpyHostToDevice, s));
+    st = tc_launch_covariance(calib->data, calib->dtype, n, c, hw, d_mean, d_cov, s);
+    if (st != TC_OK) return st;
+    std::vector<double> cov((size_t)c * c);
+    TC_CUDA(cudaMemcpyAsync(cov.data(), d_cov, sizeof(double) * cov.size(), cudaMemcpyDeviceToHost, s));
+    TC_CUDA(cudaStreamSynchronize(s));
+    const double denom = (double)(m_samples - 1);
+    for (int a = 0; a < c; ++a)
+        for (int b = a; b < c; ++b) {
+            const double v = cov[(size_t)a * c + b] / denom;
+            cov[(size_t)a * c + b] = cov[(size_t)b * c + a] = v;
+        }
+    std::vector<double> eig(c), basis((size_t)c * c);
+    if (tc_eigh_host(cov.data(), c, eig.data(), basis.data()) != 0) return TC_ERR_NOT_CONVERGED;
+    for (double &v : basis) v = round_to_dtype(v, params->basis_dtype);
+
+    TC_CUDA(cudaMemcpyAsync(d_row0, basis.data(), sizeof(double) * c, cudaMemcpyHostToDevice, s));
+    int blocks = 0;
+    st = tc_launch_range0(calib->data, calib->dtype, n, c, hw, d_mean, d_row0, d_minmax, &blocks, s);
+    if (st != TC_OK) return st;
+    std::vector<double> mm(2 * (size_t)blocks);
+    TC_CUDA(cudaMemcpyAsync(mm.data(), d_minmax, sizeof(double) * mm.size(), cudaMemcpyDeviceToHost, s));
+    TC_CUDA(cudaStreamSynchronize(s));
+    double lo = INFINITY, hi = -INFINITY;
+    for (int i = 0; i < blocks; ++i) { lo = std::min(lo, mm[2 * i]); hi = std::max(hi, mm[2 * i + 1]); }
+    if (!(hi > lo)) return TC_ERR_INVALID_ARG;    // constant calibration data: no range to quantise
+
+    tc_model_desc d;
+    d.c = c; d.k = k; d.bits = params->bits; d.basis_dtype = params->basis_dtype;
+    d.lo = lo; d.step = (hi - lo) / (double)((1 << params->bits) - 1);
+    d.basis = basis.data(); d.mean = mean.data(); d.eig = eig.data();
+    return tc_model_import(ctx, &d, out);
+}
+
+// ---- codebook ---------------------------------------------------------------------------
+
+tc_status tc_host_huffman_lengths(const uint64_t *counts, int32_t nsym, int32_t max_length, uint8_t *lengths)
+{
+    return tc_huffman_lengths_host(counts, nsym, max_length, lengths) == 0 ? TC_OK : TC_ERR_INVALID_ARG;
+}
+
+tc_status tc_host_eigh(double *a, int32_t n, double *evals, double *evecs)
+{
+    if (!a || !evals || !evecs || n < 1) return TC_ERR_INVALID_ARG;
+    return tc_eigh_host(a, n, evals, evecs) == 0 ? TC_OK : TC_ERR_NOT_CONVERGED;
+}
+
+tc_status tc_codebook_import(tc_ctx *ctx, int32_t bits, int32_t groups, const uint8_t *lengths, tc_codebook **out)
+{
+    if (!ctx || !lengths || !out || groups < 1) return TC_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (bits < 1 || bits > 8 || groups > TC_MAX_C) return TC_ERR_UNSUPPORTED;
+    const int nsym = 1 << bits;
+    for (int g = 0; g < groups; ++g) {
+        const uint8_t *len = lengths + (size_t)g * nsym;
+        for (int s = 0; s < nsym; ++s)
+            if (len[s] > TC_MAX_CODE_LEN) return TC_ERR_UNSUPPORTED;
+        if (!kraft_complete(len, nsym, TC_MAX_CODE_LEN)) return TC_ERR_INVALID_ARG;
+    }
+    DeviceGuard guard(ctx->device);
+    tc_codebook *cb = new (std::nothrow) tc_codebook();
+    if (!cb) return TC_ERR_CUDA;
+    cb->bits = bits; cb->groups = groups; cb->device = ctx->device;
+    cb->lengths.assign(lengths, lengths + (size_t)groups * nsym);
+    tc_status st = finish_codebook(cb);
+    if (st != TC_OK) { tc_codebook_free(cb); return st; }
+    *out = cb;
+    return TC_OK;
+}
+
+tc_status tc_build_codebook(tc_ctx *ctx, const tc_model *model, const uint64_t *hist, int hist_on_device,
+                            const tc_codebook_params *params, tc_codebook **out)
+{
+    if (!ctx || !model || !hist || !params || !out) return TC_ERR_INVALID_ARG;
+    *out = nullptr;
+    const int groups = params->groups;
+    if (groups != 1 && groups != model->k) return TC_ERR_INVALID_ARG;
+    const int lmax = params->max_length ? params->max_length : TC_MAX_CODE_LEN;
+    if (lmax < model->bits) return TC_ERR_INVALID_ARG;
+    if (lmax > TC_MAX_CODE_LEN) return TC_ERR_UNSUPPORTED;
+    const int nsym = 1 << model->bits;
+    std::vector<uint64_t> h((size_t)groups * nsym);
+    if (hist_on_device) {
+        DeviceGuard guard(ctx->device);
+        TC_CUDA(cudaMemcpy(h.data(), hist, h.size() * sizeof(uint64_t), cudaMemcpyDeviceToHost));
+    } else {
+        std::copy(hist, hist + h.size(), h.begin());
+    }
+    std::vector<uint8_t> lengths((size_t)groups * nsym);
+    for (int g = 0; g < groups; ++g)
+        if (tc_huffman_lengths_host(h.data() + (size_t)g * nsym, nsym, lmax, lengths.data() + (size_t)g * nsym) != 0)
+            return TC_ERR_INVALID_ARG;
+    return tc_codebook_import(ctx, model->bits, groups, lengths.data(), out);
+}
+
+tc_status tc_codebook_export(const tc_codebook *cb, int32_t *bits, int32_t *groups, uint8_t *lengths)
+{
+    if (!cb) return TC_ERR_INVALID_ARG;
+    if (bits) *bits = cb->bits;
+    if (groups) *groups = cb->groups;
+    if (lengths) std::copy(cb->lengths.begin(), cb->lengths.end(), lengths);
+    return TC_OK;
+}
+
+void tc_codebook_free(tc_codebook *cb)
+{
+    if (!cb) return;
+    DeviceGuard guard(cb->device);
+    cudaFree(cb->d_enc);
+    cudaFree(cb->d_lut);
+    delete cb;
+}
+
+// ---- encode / decode ----------------------------------------------------------------------
+
+static tc_status check_codec_args(const tc_model *m, const tc_codebook *cb, const tc_tensor *x)
+{
+    if (!m || !cb || !valid_tensor(x)) return TC_ERR_INVALID_ARG;
+    if (x->c != m->c || cb->bits != m->bits) return TC_ERR_INVALID_ARG;
+    if (cb->groups != 1 && cb->groups != m->k) return TC_ERR_INVALID_ARG;
+    if (x->dtype != m->basis_dtype) return TC_ERR_UNSUPPORTED;
+    if ((long long)x->n * x->h * x->w > (1ll << 40)) return TC_ERR_UNSUPPORTED;
+    return TC_OK;
+}
+
+tc_status tc_encode_bound(const tc_model *m, const tc_codebook *cb, const tc_tensor *x, const tc_encode_params *params,
+                          tc_stream_layout *out)
+{
+    if (!out) return TC_ERR_INVALID_ARG;
+    tc_status st = check_codec_args(m, cb, x);
+    if (st != TC_OK) return st;
+    int cp;
+    if (!resolve_chunk_pixels(params, m->k, &cp)) return TC_ERR_INVALID_ARG;
+    const long long pixels = (long long)x->n * x->h * x->w;
+    out->n_tiles = (pixels + TC_TILE_PIXELS - 1) / TC_TILE_PIXELS;
+    out->n_chunks = (pixels + cp - 1) / cp;
+    const unsigned long long tile_bits = (unsigned long long)TC_TILE_PIXELS * m->k * cb->max_len;   // multiple of 128
+    out->stream_bytes = (size_t)((unsigned long long)out->n_tiles * tile_bits / 8);
+    out->chunk_off_bytes = (size_t)out->n_chunks * 4;
+    out->tile_off_bytes = (size_t)(out->n_tiles + 1) * 8;
+    out->chunk_pixels = cp;
+    return TC_OK;
+}
+
+tc_status tc_encode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const tc_tensor *x,
+                    const tc_encode_params *params, void *stream_out, size_t capacity, uint32_t *chunk_off,
+                    uint64_t *tile_off, const tc_debug_out *debug, void *cuda_stream)
+{
+    if (!ctx || !tile_off) return TC_ERR_INVALID_ARG;
+    tc_status st = check_codec_args(m, cb, x);
+    if (st != TC_OK) return st;
+    int cp;
+    if (!resolve_chunk_pixels(params, m->k, &cp)) return TC_ERR_INVALID_ARG;
+    const long long pixels = (long long)x->n * x->h * x->w;
+    if (pixels > 0 && (!stream_out || !chunk_off)) return TC_ERR_INVALID_ARG;
+    if (((uintptr_t)stream_out & 15u) != 0) return TC_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const long long n_tiles = (pixels + TC_TILE_PIXELS - 1) / TC_TILE_PIXELS;
+    if (n_tiles == 0) {
+        TC_CUDA(cudaMemsetAsync(tile_off, 0, sizeof(uint64_t), s));
+        return TC_OK;
+    }
+    const size_t scratch = 64 + (size_t)n_tiles * sizeof(unsigned long long);
+    if ((st = ensure_scratch(ctx, scratch)) != TC_OK) return st;
+    TC_CUDA(cudaMemsetAsync(ctx->scratch, 0, scratch, s));
+
+    EncodeArgs a{};
+    a.x = x->data; a.n = x->n; a.c = x->c; a.hw = x->h * x->w; a.k = m->k; a.bits = m->bits; a.groups = cb->groups;
+    a.pixels = pixels; a.n_tiles = n_tiles; a.chunk_pixels = cp;
+    a.basis64 = m->d_basis64; a.mean64 = m->d_mean64; a.lo = m->lo; a.step = m->step;
+    a.enc = cb->d_enc; a.stream = (uint32_t *)stream_out;
+    a.capacity_bits = (unsigned long long)(capacity & ~(size_t)15) * 8ull;
+    a.chunk_off = chunk_off; a.tile_off = (unsigned long long *)tile_off;
+    a.dbg_coef = debug ? debug->coefficients : nullptr;
+    a.dbg_sym = debug ? debug->symbols : nullptr;
+    a.ticket = (unsigned int *)ctx->scratch;
+    a.tile_state = (unsigned long long *)((char *)ctx->scratch + 64);
+    a.status = ctx->d_status; a.clamped = nullptr; a.emit = 1;
+    return tc_launch_encode_simt(ctx, a, x->dtype, s);
+}
+
+tc_status tc_decode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const void *stream, size_t stream_bytes,
+                    const uint32_t *chunk_off, const uint64_t *tile_off, const tc_encode_params *params,
+                    const tc_tensor *x_hat, void *cuda_stream)
+{
+    if (!ctx) return TC_ERR_INVALID_ARG;
+    tc_status st = check_codec_args(m, cb, x_hat);
+    if (st != TC_OK) return st;
+    int cp;
+    if (!resolve_chunk_pixels(params, m->k, &cp)) return TC_ERR_INVALID_ARG;
+    const long long pixels = (long long)x_hat->n * x_hat->h * x_hat->w;
+    if (pixels == 0) return TC_OK;
+    if (!stream || !chunk_off || !tile_off || ((uintptr_t)stream & 15u) != 0) return TC_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    DecodeArgs a{};
+    a.stream = (const uint32_t *)stream; a.stream_bits = (unsigned long long)(stream_bytes & ~(size_t)3) * 8ull;
+    a.chunk_off = chunk_off; a.tile_off = (const unsigned long long *)tile_off; a.symbols = nullptr;
+    a.n = x_hat->n; a.c = x_hat->c; a.hw = x_hat->h * x_hat->w; a.k = m->k; a.bits = m->bits; a.groups = cb->groups;
+    a.pixels = pixels; a.n_tiles = (pixels + TC_TILE_PIXELS - 1) / TC_TILE_PIXELS; a.n_chunks = (pixels + cp - 1) / cp;
+    a.chunk_pixels = cp; a.lut_bits = cb->lut_bits; a.lut = cb->d_lut;
+    a.basis64 = m->d_basis64; a.mean64 = m->d_mean64; a.lo = m->lo; a.step = m->step;
+    a.xhat = x_hat->data; a.status = ctx->d_status;
+    return tc_launch_decode_simt(ctx, a, x_hat->dtype, (cudaStream_t)cuda_stream);
+}
+
+// ---- statistics ---------------------------------------------------------------------------
+
+tc_status tc_stats(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const tc_tensor *x, tc_stats_out *out,
+                   void *cuda_stream)
+{
+    if (!ctx || !m || !out || !valid_tensor(x)) return TC_ERR_INVALID_ARG;
+    if (x->c != m->c) return TC_ERR_INVALID_ARG;
+    if (x->dtype != m->basis_dtype) return TC_ERR_UNSUPPORTED;
+    if (out->groups != 1 && out->groups != m->k) return TC_ERR_INVALID_ARG;
+    if (cb && (cb->bits != m->bits || (cb->groups != 1 && cb->groups != m->k))) return TC_ERR_INVALID_ARG;
+    const long long pixels = (long long)x->n * x->h * x->w;
+    if (pixels == 0) return TC_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const int nsym = 1 << m->bits, groups = out->groups;
+    const size_t elem = (x->dtype == TC_F32) ? 4 : 2;
+    const size_t values = (size_t)pixels * m->c, symbols = (size_t)pixels * m->k;
+    const size_t hist_bytes = (size_t)m->k * nsym * sizeof(unsigned long long);
+
+    char *buf = nullptr;
+    const size_t off_xhat = (symbols + 255) & ~(size_t)255;
+    const size_t off_hist = off_xhat + ((values * elem + 255) & ~(size_t)255);
+    const size_t off_small = off_hist + hist_bytes;
+    TC_CUDA(cudaMalloc((void **)&buf, off_small + 64));
+    struct Free { char *p; ~Free() { cudaFree(p); } } freer{buf};
+    uint8_t *d_sym = (uint8_t *)buf;
+    void *d_xhat = buf + off_xhat;
+    unsigned long long *d_hist = (unsigned long long *)(buf + off_hist);   // always per channel
+    double *d_sq = (double *)(buf + off_small);
+    unsigned long long *d_zeros = (unsigned long long *)(buf + off_small + 8);
+    unsigned long long *d_clamped = (unsigned long long *)(buf + off_small + 16);
+    TC_CUDA(cudaMemsetAsync(buf + off_hist, 0, hist_bytes + 64, s));
+
+    EncodeArgs e{};
+    e.x = x->data; e.n = x->n; e.c = x->c; e.hw = x->h * x->w; e.k = m->k; e.bits = m->bits; e.groups = 1;
+    e.pixels = pixels; e.n_tiles = (pixels + TC_TILE_PIXELS - 1) / TC_TILE_PIXELS; e.chunk_pixels = 1;
+    e.basis64 = m->d_basis64; e.mean64 = m->d_mean64; e.lo = m->lo; e.step = m->step;
+    e.enc = nullptr; e.dbg_sym = d_sym; e.status = ctx->d_status; e.clamped = d_clamped; e.emit = 0;
+    e.bits = m->bits;
+    // statistics mode stages no code table: give it an empty one
+    e.groups = 0;
+    tc_status st = tc_launch_encode_simt(ctx, e, x->dtype, s);
+    if (st != TC_OK) return st;
+    if ((st = tc_launch_histogram(d_sym, pixels, m->k, m->k, m->bits, d_hist, s)) != TC_OK) return st;
+
+    DecodeArgs d{};
+    d.symbols = d_sym; d.n = x->n; d.c = x->c; d.hw = x->h * x->w; d.k = m->k; d.bits = m->bits; d.groups = 1;
+    d.pixels = pixels; d.n_tiles = e.n_tiles; d.n_chunks = pixels; d.chunk_pixels = 1;
+    d.basis64 = m->d_basis64; d.mean64 = m->d_mean64; d.lo = m->lo; d.step = m->step;
+    d.xhat = d_xhat; d.status = ctx->d_status;
+    if ((st = tc_launch_decode_simt(ctx, d, x->dtype, s)) != TC_OK) return st;
+    if ((st = tc_launch_sqerr(x->data, d_xhat, x->dtype, (long long)values, d_sq, d_zeros, s)) != TC_OK) return st;
+
+    std::vector<unsigned long long> hist((size_t)m->k * nsym);
+    double sq = 0.0;
+    unsigned long long zeros = 0, clamped = 0;
+    TC_CUDA(cudaMemcpyAsync(hist.data(), d_hist, hist_bytes, cudaMemcpyDeviceToHost, s));
+    TC_CUDA(cudaMemcpyAsync(&sq, d_sq, 8, cudaMemcpyDeviceToHost, s));
+    TC_CUDA(cudaMemcpyAsync(&zeros, d_zeros, 8, cudaMemcpyDeviceToHost, s));
+    TC_CUDA(cudaMemcpyAsync(&clamped, d_clamped, 8, cudaMemcpyDeviceToHost, s));
+    TC_CUDA(cudaStreamSynchronize(s));
+
+    // fold the per-channel counts to the requested granularity
+    std::vector<unsigned long long> folded((size_t)groups * nsym, 0ull);
+    for (int j = 0; j < m->k; ++j)
+        for (int v = 0; v < nsym; ++v) folded[(size_t)(groups == 1 ? 0 : j) * nsym + v] += hist[(size_t)j * nsym + v];
+    if (out->hist)
+        TC_CUDA(cudaMemcpy(out->hist, folded.data(), folded.size() * sizeof(unsigned long long), cudaMemcpyHostToDevice));
+    double entropy = 0.0, mean_len = 0.0;
+    for (int g = 0; g < groups; ++g) {
+        double tot = 0.0, h = 0.0;
+        for (int v = 0; v < nsym; ++v) tot += (double)folded[(size_t)g * nsym + v];
+        for (int v = 0; v < nsym; ++v) {
+            const double cnt = (double)folded[(size_t)g * nsym + v];
+            if (cnt > 0) h -= cnt / tot * std::log2(cnt / tot);
+        }
+        entropy += h / groups;
+    }
+    if (cb) {
+        double tot = 0.0, acc = 0.0;
+        for (int j = 0; j < m->k; ++j)
+            for (int v = 0; v < nsym; ++v) {
+                const double cnt = (double)hist[(size_t)j * nsym + v];
+                tot += cnt;
+                acc += cnt * cb->lengths[(size_t)(cb->groups == 1 ? 0 : j) * nsym + v];
+            }
+        mean_len = acc / tot;
+    }
+    out->entropy = entropy;
+    out->mean_length = mean_len;
+    out->mse = sq / (double)values;
+    out->clamped_fraction = (double)clamped / (double)symbols;
+    out->zero_fraction = (double)zeros / (double)values;
+    double total_energy = 0.0, run = 0.0;
+    for (double v : m->eig) total_energy += v;
+    int need = m->c;
+    for (int j = 0; j < m->c && total_energy > 0.0; ++j) {
+        run += m->eig[j];
+        if (run >= 0.9 * total_energy) { need = j + 1; break; }
+    }
+    out->energy_ratio_90 = (double)need / (double)m->c;
+    return TC_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,118 @@
+// Internal declarations shared by the host API and the kernels of the codec library.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "tc.h"
+
+constexpr int TC_TILE_PIXELS = 128;   // pixels per tile = threads per epilogue group
+constexpr int TC_MAX_C = 1024;
+constexpr int TC_MAX_CODE_LEN = 12;   // longest code the decode lookup table covers
+
+// Device status word: first error wins.
+__device__ __forceinline__ void tc_dev_set_status(unsigned int *status, unsigned int code)
+{
+    atomicCAS(status, 0u, code);
+}
+
+struct tc_ctx {
+    int device = 0;
+    int sm_count = 0;
+    int max_smem_optin = 0;
+    unsigned int *d_status = nullptr;     // device status word
+    void *scratch = nullptr;              // look-back state, ticket counter
+    size_t scratch_bytes = 0;
+    cudaEvent_t ev = nullptr;
+};
+
+struct tc_model {
+    int c = 0, k = 0, bits = 0, basis_dtype = 0;
+    double lo = 0, step = 0;
+    std::vector<double> basis, mean, eig;   // host copies (basis [c][c])
+    int device = 0;
+    // device copies
+    double *d_basis64 = nullptr;            // [c][c] exact values of the (rounded) basis
+    double *d_mean64 = nullptr;             // [c]
+    __nv_bfloat16 *d_basis_bf16 = nullptr;  // [k][c]   (bf16 models only)
+    __nv_bfloat16 *d_basis_t_bf16 = nullptr;// [c][k]   transpose, for the inverse projection
+    float *d_enc_bias = nullptr;            // [k]  -(T mu + lo)_j / step
+    float *d_dec_bias = nullptr;            // [c]  mu_c + lo * sum_j T[j][c]
+};
+
+struct tc_codebook {
+    int bits = 0, groups = 0, max_len = 0, lut_bits = 0;
+    std::vector<uint8_t> lengths;           // host [groups][2^bits]
+    int device = 0;
+    uint32_t *d_enc = nullptr;              // [groups][2^bits]  (code << 8) | length
+    uint16_t *d_lut = nullptr;              // [groups][2^lut_bits]  (symbol << 8) | length
+};
+
+// ---- kernel argument blocks -------------------------------------------------------------
+
+struct EncodeArgs {
+    const void *x;
+    int n, c, hw, k, bits, groups;
+    long long pixels;
+    long long n_tiles;
+    int chunk_pixels;
+    const double *basis64;      // [c][c]
+    const double *mean64;       // [c]
+    double lo, step;
+    const uint32_t *enc;        // [groups][2^bits]
+    uint32_t *stream;           // output words
+    unsigned long long capacity_bits;
+    uint32_t *chunk_off;
+    unsigned long long *tile_off;
+    float *dbg_coef;            // nullable
+    uint8_t *dbg_sym;           // nullable
+    unsigned long long *tile_state;   // look-back state, zeroed before launch
+    unsigned int *ticket;             // zeroed before launch
+    unsigned int *status;
+    unsigned long long *clamped;      // nullable: counts coefficients outside the range
+    int emit;                         // 0: symbols only (statistics mode)
+};
+
+struct DecodeArgs {
+    const uint32_t *stream;
+    unsigned long long stream_bits;
+    const uint32_t *chunk_off;
+    const unsigned long long *tile_off;
+    const uint8_t *symbols;     // non-null: take symbols from here instead of the stream
+    int n, c, hw, k, bits, groups;
+    long long pixels;
+    long long n_tiles, n_chunks;
+    int chunk_pixels;
+    int lut_bits;
+    const uint16_t *lut;
+    const double *basis64;
+    const double *mean64;
+    double lo, step;
+    void *xhat;
+    unsigned int *status;
+};
+
+// ---- launchers (defined in the .cu files) ----------------------------------------------
+tc_status tc_launch_encode_simt(const tc_ctx *ctx, const EncodeArgs &a, int dtype, cudaStream_t s);
+tc_status tc_launch_decode_simt(const tc_ctx *ctx, const DecodeArgs &a, int dtype, cudaStream_t s);
+
+tc_status tc_launch_channel_sums(const void *x, int dtype, int n, int c, int hw, double *sums,
+                                 cudaStream_t s);
+tc_status tc_launch_covariance(const void *x, int dtype, int n, int c, int hw, const double *mean,
+                               double *cov, cudaStream_t s);
+tc_status tc_launch_range0(const void *x, int dtype, int n, int c, int hw, const double *mean,
+                           const double *row0, double *block_minmax, int *n_blocks_out,
+                           cudaStream_t s);
+int tc_range0_max_blocks(long long pixels);
+tc_status tc_launch_histogram(const uint8_t *sym, long long pixels, int k, int groups, int bits,
+                              unsigned long long *hist, cudaStream_t s);
+tc_status tc_launch_sqerr(const void *x, const void *xhat, int dtype, long long count,
+                          double *sum_sq, unsigned long long *zeros, cudaStream_t s);
+
+// ---- host algorithms (host_algos.cpp) ---------------------------------------------------
+int tc_huffman_lengths_host(const uint64_t *counts, int nsym, int lmax, uint8_t *len);
+void tc_canonical_codes_host(const uint8_t *len, int nsym, uint32_t *code);
+int tc_eigh_host(double *a, int n, double *evals, double *evecs);

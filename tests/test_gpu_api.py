@@ -1,0 +1,204 @@
+"""GPU tests of the library's other entry points and of its error behaviour: fit, statistics,
+codebook building, capacity overflow and corrupt streams (all made on the host; nothing here
+traps or hangs the device)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_1905_10830_b200 as tc
+from synth import featuremaps as fm
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = tc.tc_create(0)
+    yield c
+    c.close()
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_fit_pca_invariants_and_agreement_with_oracle(ctx, dtype):
+    spec = fm.LayerSpec(48, 14, 14, 0.85, None, 501)
+    p = fm.layer_params(spec)
+    cal = fm.make_maps(p, 16, calib=True, dtype=dtype)
+    m = tc.tc_fit_pca(ctx, cal.cuda(), bits=6)
+    e = tc.tc_model_export(m)
+    ref = oracle.fit_pca(cal, 6, basis_round=H.basis_round_for(dtype))
+    t = e["basis"]
+    rt = 2.0 ** -8 if dtype == torch.bfloat16 else 2.0 ** -23
+    assert np.abs(t @ t.T - np.eye(48)).max() < 48 * rt
+    _, cov = oracle.mean_cov(cal)
+    d = t @ cov @ t.T
+    assert np.abs(d - np.diag(np.diag(d))).max() < 10 * rt * np.abs(cov).max()
+    assert np.allclose(e["eig"], ref.eig, rtol=1e-9, atol=1e-12 * ref.eig[0])
+    assert np.allclose(e["mean"], ref.mean, rtol=1e-12, atol=1e-14)
+    lead = ref.eig > 1e-3 * ref.eig[0]
+    gaps_ok = np.abs(np.diff(ref.eig))[: lead.sum() - 1] > 1e-3 * ref.eig[0]
+    for j in np.nonzero(lead)[0][:-1]:
+        if gaps_ok[max(j - 1, 0)] and gaps_ok[j]:
+            assert abs(t[j] @ ref.basis[j]) > 1 - 1e-4
+    assert e["lo"] == pytest.approx(ref.lo, rel=2e-2, abs=1e-3)
+    assert e["step"] == pytest.approx(ref.step, rel=2e-2)
+    # end to end: rate and distortion within 1 % of the oracle's fit
+    x = fm.make_maps(p, 4, dtype=dtype)
+    st = tc.tc_stats(ctx, m, None, x.cuda())
+    q_ref = oracle.quantize(ref, oracle.project(ref, x))
+    h_ref = oracle.entropy(oracle.histogram(q_ref, 6, False)[0])
+    mse_ref = oracle.mse(x, oracle.reconstruct(ref, q_ref, x.shape, out_bf16=(dtype == torch.bfloat16)))
+    assert st.entropy == pytest.approx(h_ref, rel=0.01)
+    assert st.mse == pytest.approx(mse_ref, rel=0.02)
+    m.close()
+
+
+@pytest.mark.parametrize("per_channel", [False, True])
+def test_stats_and_build_codebook_match_oracle(ctx, per_channel):
+    spec = fm.LayerSpec(32, 14, 14, 0.85, None, 502)
+    o = H.oracle_side(spec, 5, 8, 4, torch.float32, per_channel)
+    m = H.import_model(tc, ctx, o["model"], torch.float32)
+    groups = 32 if per_channel else 1
+    st = tc.tc_stats(ctx, m, None, o["cal"].cuda(), groups=groups)
+    hist_ref = oracle.histogram(o["q_cal"], 5, per_channel)
+    assert np.array_equal(st.hist.cpu().numpy().view(np.uint64), hist_ref)
+    want_h = np.mean([oracle.entropy(hist_ref[g]) for g in range(groups)])
+    assert st.entropy == pytest.approx(want_h, rel=1e-12)
+    cb = tc.tc_build_codebook(ctx, m, st.hist, groups=groups)
+    assert np.array_equal(tc.tc_codebook_export(cb), o["lengths"])
+    cb_host = tc.tc_build_codebook(ctx, m, hist_ref, groups=groups)
+    assert np.array_equal(tc.tc_codebook_export(cb_host), o["lengths"])
+    st2 = tc.tc_stats(ctx, m, cb, o["x"].cuda(), groups=groups)
+    q = o["q"]
+    lens = np.stack([o["lengths"][j if per_channel else 0][q[:, j]] for j in range(32)], axis=1)
+    assert st2.mean_length == pytest.approx(lens.mean(), rel=1e-12)
+    xhat = oracle.reconstruct(o["model"], q, o["x"].shape, out_bf16=False)
+    assert st2.mse == pytest.approx(oracle.mse(o["x"], xhat), rel=1e-9)
+    assert st2.zero_fraction == pytest.approx(float((o["x"] == 0).float().mean()), abs=1e-12)
+    top = (1 << 5) - 1
+    assert st2.clamped_fraction == pytest.approx(float(((o["units"] < 0) | (o["units"] > top)).mean()), abs=1e-12)
+    for h in (m, cb, cb_host):
+        h.close()
+
+
+def test_model_export_round_trip_and_rejects_unrepresentable_basis(ctx):
+    spec = fm.LayerSpec(16, 8, 8, 0.85, None, 503)
+    o = H.oracle_side(spec, 4, 4, 1, torch.bfloat16, False)
+    m = H.import_model(tc, ctx, o["model"], torch.bfloat16)
+    e = tc.tc_model_export(m)
+    assert np.array_equal(e["basis"], o["model"].basis) and np.array_equal(e["mean"], o["model"].mean)
+    assert e["lo"] == o["model"].lo and e["step"] == o["model"].step and e["bits"] == 4
+    m.close()
+    full = oracle.fit_pca(o["cal"], 4)                      # fp64 basis: not bf16-exact
+    with pytest.raises(tc.TcError) as err:
+        H.import_model(tc, ctx, full, torch.bfloat16)
+    assert err.value.code == 1
+
+
+def test_argument_errors(ctx):
+    spec = fm.LayerSpec(16, 8, 8, 0.85, None, 504)
+    o = H.oracle_side(spec, 4, 4, 1, torch.float32, False)
+    m = H.import_model(tc, ctx, o["model"], torch.float32)
+    cb = tc.tc_codebook_import(ctx, o["lengths"], 4)
+    x = o["x"].cuda()
+    with pytest.raises(tc.TcError) as err:                   # wrong channel count
+        tc.tc_encode(ctx, m, cb, torch.zeros(1, 8, 8, 8, device="cuda"))
+    assert err.value.code == 1
+    with pytest.raises(tc.TcError) as err:                   # dtype does not match the basis
+        tc.tc_encode(ctx, m, cb, x.bfloat16())
+    assert err.value.code == 2
+    with pytest.raises(tc.TcError):                          # chunk size not a power of two
+        tc.tc_encode(ctx, m, cb, x, chunk_pixels=3)
+    bad = o["lengths"].copy()
+    bad[0, 0] += 1                                           # breaks Kraft's equality
+    with pytest.raises(tc.TcError):
+        tc.tc_codebook_import(ctx, bad, 4)
+    # empty batch
+    enc = tc.tc_encode(ctx, m, cb, torch.zeros(0, 16, 8, 8, device="cuda"))
+    assert enc.total_bits() == 0
+    m.close(); cb.close()
+
+
+def test_capacity_overflow_is_reported_and_in_bounds(ctx):
+    spec = fm.LayerSpec(32, 16, 16, 0.85, None, 505)
+    o = H.oracle_side(spec, 6, 4, 2, torch.float32, False)
+    m = H.import_model(tc, ctx, o["model"], torch.float32)
+    cb = tc.tc_codebook_import(ctx, o["lengths"], 6)
+    x = o["x"].cuda()
+    full = tc.tc_encode(ctx, m, cb, x)
+    assert tc.tc_get_status(ctx) == 0
+    need = full.total_bits() // 8
+    lay = full.layout
+    guard = 4096
+    buf = torch.full((need + guard,), 0xAB, dtype=torch.uint8, device="cuda")
+    small = tc.EncodedStream(buf, torch.empty(lay.n_chunks, dtype=torch.int32, device="cuda"),
+                             torch.empty(lay.n_tiles + 1, dtype=torch.int64, device="cuda"), lay)
+    cap = (need // 2) & ~15
+    tc.tc_encode(ctx, m, cb, x, out=small, capacity=cap)
+    assert tc.tc_get_status(ctx) == 3                          # TC_ERR_BUFFER_TOO_SMALL
+    assert tc.tc_get_status(ctx) == 0                          # cleared
+    assert bool((buf[cap:] == 0xAB).all())                     # nothing written past the capacity
+    # exact capacity works
+    tc.tc_encode(ctx, m, cb, x, out=small, capacity=need)
+    assert tc.tc_get_status(ctx) == 0
+    assert torch.equal(buf[:need], full.words[:need])
+    assert bool((buf[need:] == 0xAB).all())
+    m.close(); cb.close()
+
+
+def test_corrupt_streams_are_reported_without_faults(ctx):
+    spec = fm.LayerSpec(32, 16, 16, 0.85, None, 506)
+    o = H.oracle_side(spec, 6, 4, 2, torch.float32, False)
+    m = H.import_model(tc, ctx, o["model"], torch.float32)
+    cb = tc.tc_codebook_import(ctx, o["lengths"], 6)
+    x = o["x"].cuda()
+    enc = tc.tc_encode(ctx, m, cb, x)
+    assert tc.tc_get_status(ctx) == 0
+    nbytes = enc.total_bits() // 8
+    # (a) truncated stream
+    tc.tc_decode(ctx, m, cb, enc, x.shape, x.dtype, stream_bytes=(nbytes // 2) & ~15)
+    assert tc.tc_get_status(ctx) == 5
+    # (b) tile offset beyond the stream / not aligned / decreasing
+    for bad_value in (nbytes * 8 + 128, 64, -128):
+        broken = tc.EncodedStream(enc.words, enc.chunk_off, enc.tile_off.clone(), enc.layout)
+        broken.tile_off[1] = broken.tile_off[1] + bad_value if bad_value != 64 else 64
+        tc.tc_decode(ctx, m, cb, broken, x.shape, x.dtype, stream_bytes=nbytes)
+        assert tc.tc_get_status(ctx) == 5
+    # (c) chunk offset pointing past its tile
+    broken = tc.EncodedStream(enc.words, enc.chunk_off.clone(), enc.tile_off, enc.layout)
+    broken.chunk_off[3] = 0x7FFFFFF0
+    tc.tc_decode(ctx, m, cb, broken, x.shape, x.dtype, stream_bytes=nbytes)
+    assert tc.tc_get_status(ctx) == 5
+    # (d) flipped payload bits: must stay in bounds; either decodes to other symbols or reports
+    noisy = tc.EncodedStream(enc.words.clone(), enc.chunk_off, enc.tile_off, enc.layout)
+    g = torch.Generator(device="cuda").manual_seed(1)
+    idx = torch.randint(0, nbytes, (64,), generator=g, device="cuda")
+    noisy.words[idx] ^= 0x5A
+    out = tc.tc_decode(ctx, m, cb, noisy, x.shape, x.dtype, stream_bytes=nbytes)
+    assert tc.tc_get_status(ctx) in (0, 5)
+    assert out.shape == x.shape
+    # the intact stream still decodes afterwards
+    good = tc.tc_decode(ctx, m, cb, enc, x.shape, x.dtype, stream_bytes=nbytes)
+    assert tc.tc_get_status(ctx) == 0
+    want = oracle.reconstruct(o["model"], o["q"], x.shape, out_bf16=False)
+    assert np.array_equal(good.cpu().numpy(), want)
+    m.close(); cb.close()
+
+
+def test_repeated_encodes_are_bit_identical(ctx):
+    # the look-back makes the layout deterministic: every run writes the same bytes
+    spec = fm.LayerSpec(64, 28, 28, 0.9, None, 507)
+    o = H.oracle_side(spec, 4, 4, 8, torch.bfloat16, False)
+    m = H.import_model(tc, ctx, o["model"], torch.bfloat16)
+    cb = tc.tc_codebook_import(ctx, o["lengths"], 4)
+    x = o["x"].cuda()
+    first = tc.tc_encode(ctx, m, cb, x)
+    n = first.total_bits() // 8
+    for _ in range(3):
+        again = tc.tc_encode(ctx, m, cb, x)
+        assert tc.tc_get_status(ctx) == 0
+        assert again.total_bits() == first.total_bits()
+        assert torch.equal(again.words[:n], first.words[:n])
+        assert torch.equal(again.tile_off, first.tile_off)
+    m.close(); cb.close()

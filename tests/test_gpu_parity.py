@@ -1,0 +1,120 @@
+"""GPU parity: the CUDA library against the CPU oracle on identical seeded inputs, with the
+oracle's model and codebook imported into the library (identical T, mu, lo, step, lengths).
+
+Bars: the entropy-coded stream is bit-exact given identical symbols and decode round-trips
+exactly; projected coefficients agree within 1e-3 * max(|y|, step); at most 1e-4 of the
+symbols differ, only by +-1 and only where the oracle's position (y - lo)/step lies within
+1e-3 of a half-integer; x_hat agrees within 1e-3 * max(|x_hat|, step)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_1905_10830_b200 as tc
+from synth import featuremaps as fm
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = tc.tc_create(0)
+    yield c
+    c.close()
+
+
+def check_symbols(q_gpu, o, *, exact: bool):
+    q, units = o["q"], o["units"]
+    diff = q_gpu.astype(np.int32) - q.astype(np.int32)
+    bad = diff != 0
+    if exact:
+        assert not bad.any(), f"{bad.sum()} symbols differ on the exact path"
+        return 0.0
+    rate = bad.mean()
+    assert rate <= 1e-4, f"symbol mismatch rate {rate}"
+    if bad.any():
+        assert np.all(np.abs(diff[bad]) == 1)
+        frac = np.abs(units[bad] - np.floor(units[bad]) - 0.5)
+        assert np.all(frac <= 1e-3), f"mismatch away from a rounding tie: {frac.max()}"
+    return rate
+
+
+def check_stream_against_oracle(enc, q_gpu, lengths, bits, cp):
+    """Entropy-coding stage: bit-exact given identical symbol arrays."""
+    ref = oracle.encode(q_gpu, lengths, bits, chunk_pixels=cp, tile_chunks=128 // cp)
+    assert enc.total_bits() == ref.total_bits
+    assert np.array_equal(H.tile_off(enc), ref.tile_off)
+    assert np.array_equal(H.chunk_off(enc), ref.chunk_off)
+    assert np.array_equal(H.stream_words(enc), ref.words)
+    return ref
+
+
+def run_case(ctx, spec, bits, n_cal, n_test, dtype, per_channel, *, exact, chunk_pixels=0, model=None):
+    o = H.oracle_side(spec, bits, n_cal, n_test, dtype, per_channel, model=model)
+    m, lengths = o["model"], o["lengths"]
+    model_h = H.import_model(tc, ctx, m, dtype)
+    cb = tc.tc_codebook_import(ctx, lengths, bits)
+    x = o["x"].cuda()
+    enc = tc.tc_encode(ctx, model_h, cb, x, chunk_pixels=chunk_pixels, debug=True)
+    assert tc.tc_get_status(ctx) == 0
+    cp = enc.layout.chunk_pixels
+    # coefficients
+    y_gpu = enc.coefficients.cpu().numpy().astype(np.float64)
+    tol = 1e-3 * np.maximum(np.abs(o["y"]), m.step)
+    assert np.all(np.abs(y_gpu - o["y"]) <= tol)
+    # symbols
+    q_gpu = enc.symbols.cpu().numpy()
+    check_symbols(q_gpu, o, exact=exact)
+    # stream: bit-exact against the oracle's coder on the GPU's own symbols
+    ref = check_stream_against_oracle(enc, q_gpu, lengths, bits, cp)
+    assert np.array_equal(oracle.decode_symbols(ref, lengths, bits), q_gpu)
+    # decode: reconstruct what the stream holds
+    xhat = tc.tc_decode(ctx, model_h, cb, enc, x.shape, dtype)
+    assert tc.tc_get_status(ctx) == 0
+    want = oracle.reconstruct(m, q_gpu, x.shape, out_bf16=(dtype == torch.bfloat16))
+    got = xhat.float().cpu().numpy()
+    if exact:
+        assert np.array_equal(got, want)
+    else:
+        assert np.all(np.abs(got - want) <= 1e-3 * np.maximum(np.abs(want), m.step))
+        ulp = np.abs(want) * (2.0 ** -8 if dtype == torch.bfloat16 else 2.0 ** -23) + 1e-30
+        assert (np.abs(got - want) <= ulp).mean() >= 0.999
+    model_h.close()
+    cb.close()
+    return o, enc
+
+
+def test_cfg1_single_map_f32(ctx):
+    w = fm.workload(1)
+    run_case(ctx, w.layers[0], 8, w.calib_maps, 1, torch.float32, False, exact=True)
+
+
+@pytest.mark.parametrize("layer", [0, 1, 2, 3])
+def test_cfg2_resnet18_layers_all_bit_widths_per_channel(ctx, layer):
+    w = fm.workload(2)
+    spec = w.layers[layer]
+    base = None
+    for bits in w.bits:
+        o, _ = run_case(ctx, spec, bits, w.calib_maps, 1, torch.float32, True, exact=True, model=base)
+        base = o["model"]
+
+
+@pytest.mark.parametrize("c,s,n", [(64, 56, 1), (128, 28, 2), (256, 14, 3), (512, 7, 5)])
+def test_cfg3_shapes_bf16_exact_path(ctx, c, s, n):
+    spec = fm.LayerSpec(c, s, s, 0.9, None, 3000 + c)
+    run_case(ctx, spec, 4, 4, n, torch.bfloat16, False, exact=True)
+
+
+@pytest.mark.parametrize("c,s,n", [(96, 28, 2), (144, 14, 3), (960, 7, 3)])
+def test_cfg4_like_shapes_bf16(ctx, c, s, n):
+    spec = fm.LayerSpec(c, s, s, 0.95, 0.6, 4000 + c)
+    run_case(ctx, spec, 5, max(4, (2 * c) // (s * s) + 1), n, torch.bfloat16, False, exact=True)
+
+
+@pytest.mark.parametrize("cp", [1, 2, 8, 128])
+def test_chunk_sizes_and_ragged_tail(ctx, cp):
+    # 3 maps of 9x9 = 243 pixels: one full tile and a ragged second one
+    spec = fm.LayerSpec(32, 9, 9, 0.85, None, 77)
+    run_case(ctx, spec, 6, 8, 3, torch.float32, False, exact=True, chunk_pixels=cp)
+    run_case(ctx, spec, 3, 8, 3, torch.bfloat16, True, exact=True, chunk_pixels=cp)

@@ -20,7 +20,7 @@ def _chain(spec, bits, n_cal=8, n_test=2, per_channel=False, identity=False, dty
         y_cal = cal.float().numpy().transpose(0, 2, 3, 1).reshape(-1, spec.c).astype(np.float64)
         lo, hi = y_cal.min(), y_cal.max()
         m = oracle.Model(spec.c, spec.c, bits, np.zeros(spec.c), np.eye(spec.c), m.eig, lo,
-                         (hi - lo) / ((1 << bits) - 1), False)
+                         (hi - lo) / ((1 << bits) - 1), "f64")
     q_cal = oracle.quantize(m, oracle.project(m, cal))
     hist = oracle.histogram(q_cal, bits, per_channel)
     ln = oracle.huffman_lengths(hist, 12)

@@ -179,3 +179,21 @@ def test_reconstruct_rounds_to_bf16():
     half = oracle.reconstruct(m, q, x.shape, out_bf16=True)
     assert np.array_equal(torch.tensor(half).to(torch.bfloat16).float().numpy(), half)
     assert np.all(np.abs(half - full) <= np.abs(full) * 2.0 ** -8 + 1e-30)
+
+
+def test_lapack_step_agrees_with_jacobi_and_f32_rounding():
+    # Above oracle.JACOBI_MAX_C channels the fit takes its eigendecomposition from LAPACK; on a
+    # layer small enough for both, the two routes give the same transform.
+    p = fm.layer_params(fm.LayerSpec(24, 9, 9, 0.8, None, 17))
+    x = fm.make_maps(p, 12, calib=True)
+    a = oracle.fit_pca(x, bits=6, eigensolver="jacobi")
+    b = oracle.fit_pca(x, bits=6, eigensolver="lapack")
+    assert np.allclose(a.eig, b.eig, rtol=1e-10, atol=1e-14)
+    lead = a.eig > 1e-6 * a.eig[0]
+    assert np.allclose(a.basis[lead], b.basis[lead], atol=1e-7)
+    assert a.lo == pytest.approx(b.lo, rel=1e-9) and a.step == pytest.approx(b.step, rel=1e-9)
+    f = oracle.fit_pca(x, bits=6, basis_round="f32")
+    assert np.array_equal(f.basis.astype(np.float32).astype(np.float64), f.basis)
+    assert np.abs(f.basis - a.basis).max() <= 2.0 ** -24
+    m4 = oracle.with_bits(a, 4)
+    assert m4.lo == a.lo and m4.step == pytest.approx(a.step * 63 / 15, rel=1e-14)

@@ -11,7 +11,7 @@ import oracle
 
 
 def _model(lo, step, bits):
-    return oracle.Model(1, 1, bits, np.zeros(1), np.eye(1), np.ones(1), lo, step, False)
+    return oracle.Model(1, 1, bits, np.zeros(1), np.eye(1), np.ones(1), lo, step, "f64")
 
 
 def test_quantizer_hand_values_ties_and_clamps():
