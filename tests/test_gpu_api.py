@@ -40,7 +40,8 @@ def test_fit_pca_invariants_and_agreement_with_oracle(ctx, dtype):
     gaps_ok = np.abs(np.diff(ref.eig))[: lead.sum() - 1] > 1e-3 * ref.eig[0]
     for j in np.nonzero(lead)[0][:-1]:
         if gaps_ok[max(j - 1, 0)] and gaps_ok[j]:
-            assert abs(t[j] @ ref.basis[j]) > 1 - 1e-4
+            cos = abs(t[j] @ ref.basis[j]) / (np.linalg.norm(t[j]) * np.linalg.norm(ref.basis[j]))
+            assert cos > 1 - 1e-4
     assert e["lo"] == pytest.approx(ref.lo, rel=2e-2, abs=1e-3)
     assert e["step"] == pytest.approx(ref.step, rel=2e-2)
     # end to end: rate and distortion within 1 % of the oracle's fit
@@ -75,7 +76,7 @@ def test_stats_and_build_codebook_match_oracle(ctx, per_channel):
     assert st2.mean_length == pytest.approx(lens.mean(), rel=1e-12)
     xhat = oracle.reconstruct(o["model"], q, o["x"].shape, out_bf16=False)
     assert st2.mse == pytest.approx(oracle.mse(o["x"], xhat), rel=1e-9)
-    assert st2.zero_fraction == pytest.approx(float((o["x"] == 0).float().mean()), abs=1e-12)
+    assert st2.zero_fraction == pytest.approx(float((o["x"] == 0).double().mean()), abs=1e-12)
     top = (1 << 5) - 1
     assert st2.clamped_fraction == pytest.approx(float(((o["units"] < 0) | (o["units"] > top)).mean()), abs=1e-12)
     for h in (m, cb, cb_host):
