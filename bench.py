@@ -1,0 +1,341 @@
+#!/usr/bin/env python
+"""Throughput benchmark of the feature-map transform codec on B200.
+
+One step = one pass of the whole hot path (encode, then decode) over the throughput workload:
+a 256 x 14 x 14 bf16 layer at batch 4096 (about 205 M values, 411 MB -- larger than the
+126 MB L2, so no flush is needed between iterations), synthetic correlated maps.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--bits B] [--impl ours|reference]
+
+Prints one JSON line (rank 0).  `value` is raw-activation GB/s of encode + decode with the
+input resident in HBM; `e2e` is the same metric with host buffers and the host<->device copies
+inside the timed region; `roofline` describes the slower of the two kernels; `cpu_baseline` is
+the CPU oracle timed on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from synth import featuremaps as fm
+
+METRIC = "raw_activation_GBps_encode_plus_decode"
+UNIT = "GB/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (earlier pool measurement)"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.device_index = device_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.device_index)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    sm.append(float(parts[1]))
+                    mx.append(float(parts[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                     parts[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.remove(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def oracle_setup(spec, bits, calib_maps, sample_images, dtype):
+    """Untimed: the oracle's own model and codebook, and the sample it will code."""
+    import oracle
+    params = fm.layer_params(spec)
+    cal = fm.make_maps(params, calib_maps, calib=True, dtype=dtype)
+    x = fm.make_maps(params, sample_images, dtype=dtype)
+    m = oracle.fit_pca(cal, bits, basis_round="bf16" if dtype == torch.bfloat16 else "f32")
+    q_cal = oracle.quantize(m, oracle.project(m, cal))
+    lengths = oracle.huffman_lengths(oracle.histogram(q_cal, bits, False), 12)
+    return dict(model=m, lengths=lengths, x=x, bits=bits, dtype=dtype,
+                chunk_pixels=max(1, 256 // spec.c))
+
+
+def oracle_timed_pass(o):
+    """Time the CPU oracle's encode + decode over the prepared sample (one pass)."""
+    import oracle
+    m, lengths, x, bits, cp = o["model"], o["lengths"], o["x"], o["bits"], o["chunk_pixels"]
+    t0 = time.perf_counter()
+    q = oracle.quantize(m, oracle.project(m, x))
+    s = oracle.encode(q, lengths, bits, chunk_pixels=cp, tile_chunks=128 // cp)
+    t1 = time.perf_counter()
+    q2 = oracle.decode_symbols(s, lengths, bits)
+    oracle.reconstruct(m, q2, x.shape, out_bf16=(o["dtype"] == torch.bfloat16))
+    t2 = time.perf_counter()
+    raw_bytes = x.numel() * x.element_size()
+    return dict(seconds=t2 - t0, encode_s=t1 - t0, decode_s=t2 - t1, raw_bytes=raw_bytes,
+                gbs=raw_bytes / (t2 - t0) / 1e9, bits_per_value=s.total_bits / q.size)
+
+
+def run_reference(args, rank):
+    """Reference arm: the CPU oracle, as it stands, on a bounded sample per step."""
+    if rank != 0:
+        return
+    w = fm.workload(5)
+    spec = w.layers[0]
+    sample = args.sample_images
+    times = []
+    res = None
+    o = oracle_setup(spec, args.bits, 32, sample, w.dtype)
+    for i in range(args.warmup + args.steps):
+        res = oracle_timed_pass(o)
+        if i >= args.warmup:
+            times.append(res["seconds"])
+    total = sum(times)
+    value = res["raw_bytes"] * len(times) / total / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "bits": args.bits, "sample": f"{sample} of {w.batch} images per step"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "sample": f"{sample} images of {spec.name} ({res['raw_bytes'] / 1e6:.1f} MB raw) per step"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "bits_per_value": res["bits_per_value"],
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--bits", type=int, default=4)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=0, help="override the batch size (smaller captures)")
+    ap.add_argument("--sample-images", type=int, default=0, help="images per oracle timing sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.sample_images <= 0:      # about 15 s of oracle work in our arm; short steps in the reference arm
+        args.sample_images = 512 if args.impl == "ours" else 128
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import paper_1905_10830_b200 as tc
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the codec has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    w = fm.workload(5)
+    spec = w.layers[0]
+    batch = args.batch or w.batch
+    bits = args.bits
+    params = fm.layer_params(spec)
+
+    # ---- set-up (untimed): fit, statistics, codebook -- all through the library ---------
+    ctx = tc.tc_create(local_rank)
+    cal = fm.make_maps(params, w.calib_maps, calib=True, dtype=w.dtype, device=dev)
+    model = tc.tc_fit_pca(ctx, cal, bits=bits)
+    st = tc.tc_stats(ctx, model, None, cal, groups=1)
+    cb = tc.tc_build_codebook(ctx, model, st.hist, groups=1)
+    x = fm.make_maps(params, batch, dtype=w.dtype, device=dev, offset=rank)   # each rank its own maps
+    raw_bytes = x.numel() * x.element_size()
+    lay = tc.tc_encode_bound(model, cb, x)
+    enc = tc.tc_encode(ctx, model, cb, x)
+    xhat = torch.empty_like(x)
+    tc.tc_decode(ctx, model, cb, enc, x.shape, x.dtype, out=xhat)
+    status = tc.tc_get_status(ctx)
+    if status != 0:
+        raise SystemExit(f"codec reported status {status}")
+    total_bits = enc.total_bits()
+    stream_bytes = total_bits // 8
+    side_bytes = lay.chunk_off_bytes + lay.tile_off_bytes
+    test_stats = tc.tc_stats(ctx, model, cb, x[: min(batch, 256)], groups=1, want_hist=False)
+
+    def step():
+        tc.tc_encode(ctx, model, cb, x, out=enc)
+        tc.tc_decode(ctx, model, cb, enc, x.shape, x.dtype, out=xhat, stream_bytes=stream_bytes)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+
+    # ---- timed region: K steps, CUDA events on the launching stream ----------------------
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    sampler = ClockSampler(local_rank)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    t_begin = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_begin.record()
+    for i in range(args.steps):
+        ev[i][0].record()
+        tc.tc_encode(ctx, model, cb, x, out=enc)
+        ev[i][1].record()
+        tc.tc_decode(ctx, model, cb, enc, x.shape, x.dtype, out=xhat, stream_bytes=stream_bytes)
+        ev[i][2].record()
+    t_end.record()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    clocks = sampler.stop()
+    total_ms = t_begin.elapsed_time(t_end)
+    enc_ms = [ev[i][0].elapsed_time(ev[i][1]) for i in range(args.steps)]
+    dec_ms = [ev[i][1].elapsed_time(ev[i][2]) for i in range(args.steps)]
+    if tc.tc_get_status(ctx) != 0:
+        raise SystemExit("codec reported an error during the timed region")
+    if dist is not None:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+
+    # ---- end to end: host buffers, copies inside the timed region -------------------------
+    e2e = None
+    if not args.no_e2e:
+        hx = torch.empty(x.shape, dtype=x.dtype, pin_memory=True)
+        hx.copy_(x)
+        hout = torch.empty(x.shape, dtype=x.dtype, pin_memory=True)
+        dx = torch.empty_like(x)
+        e2e_steps = max(2, min(args.steps, 5))
+
+        def e2e_step():
+            dx.copy_(hx, non_blocking=True)
+            tc.tc_encode(ctx, model, cb, dx, out=enc)
+            tc.tc_decode(ctx, model, cb, enc, x.shape, x.dtype, out=xhat, stream_bytes=stream_bytes)
+            hout.copy_(xhat, non_blocking=True)
+
+        e2e_step()
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        b.record()
+        torch.cuda.synchronize()
+        e2e_ms = a.elapsed_time(b)
+        if dist is not None:
+            t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        e2e = {"value": raw_bytes * world * e2e_steps / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": raw_bytes, "d2h_bytes_per_step": raw_bytes, "steps": e2e_steps}
+        assert torch.equal(hout.to(dev), xhat)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_src = measured_peaks()
+    enc_avg, dec_avg = statistics.mean(enc_ms), statistics.mean(dec_ms)
+    algo_bytes = raw_bytes + stream_bytes + side_bytes          # per launch, either direction
+    dominant = "encode" if enc_avg >= dec_avg else "decode"
+    dom_ms = max(enc_avg, dec_avg)
+    achieved = algo_bytes / (dom_ms * 1e-3) / 1e9
+    values = x.numel()
+    line = {
+        "metric": METRIC,
+        "value": raw_bytes * world * args.steps / (total_ms * 1e-3) / 1e9,
+        "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "layer": spec.name, "batch_per_gpu": batch, "bits": bits,
+                   "chunk_pixels": lay.chunk_pixels, "codebook": "per-layer", "calib_maps": w.calib_maps,
+                   "l2": "inputs larger than L2 (411 MB per pass), no flush", "parallelism": f"batch-sharded x{world}"},
+        "encode_gbs": raw_bytes / (enc_avg * 1e-3) / 1e9, "decode_gbs": raw_bytes / (dec_avg * 1e-3) / 1e9,
+        "encode_ms": enc_avg, "decode_ms": dec_avg,
+        "bits_per_value": {"entropy_calib": st.entropy, "huffman_payload_sample": test_stats.mean_length,
+                           "stream_with_padding": total_bits / values,
+                           "stream_plus_offsets": (total_bits + 8 * side_bytes) / values},
+        "mse_sample": test_stats.mse,
+        "roofline": {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "frac_of_nominal_8TBps": achieved / 8000.0, "peak_source": peak_src,
+                     "algorithmic_bytes_per_launch": algo_bytes, "traffic": None,
+                     "encode_frac": algo_bytes / (enc_avg * 1e-3) / 1e9 / peak,
+                     "decode_frac": algo_bytes / (dec_avg * 1e-3) / 1e9 / peak},
+        "gpu_launches": 2 * args.steps,
+        "clocks": clocks,
+    }
+    if e2e is not None:
+        line["e2e"] = e2e
+    if not args.no_cpu_baseline and world == 1:
+        res = oracle_timed_pass(oracle_setup(spec, bits, 32, args.sample_images, w.dtype))
+        line["cpu_baseline"] = {"value": res["gbs"], "unit": UNIT, "cores": 1, "kind": "oracle",
+                                "sample": f"{args.sample_images} of {batch} images ({res['raw_bytes'] / 1e6:.1f} MB raw), "
+                                          f"{res['seconds']:.1f} s, oracle model fitted on 32 calibration maps",
+                                "bits_per_value": res["bits_per_value"]}
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
