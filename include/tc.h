@@ -67,6 +67,14 @@ const char *tc_status_string(tc_status s);
  * call (TC_OK if none) and clears it. */
 tc_status tc_get_status(tc_ctx *ctx, void *cuda_stream);
 
+/* Validation switch.  bf16 tensors normally take the tensor-core kernels (bf16 products, fp32
+ * accumulation); fp32 tensors, and shapes those kernels do not take, run on kernels that
+ * evaluate the definition in fp64.  With `on` != 0 every tensor takes the fp64 kernels. */
+void tc_force_exact_path(tc_ctx *ctx, int on);
+/* Which kernels the last tc_encode (decode == 0) or tc_decode (decode != 0) of this context
+ * launched: 0 = fp64 kernels, 1 = tensor-core kernels; -1 for a NULL context. */
+int tc_last_path(const tc_ctx *ctx, int decode);
+
 /* ---------------------------------------------------------------------------------------
  * Model = per-layer transform and quantiser (Section 3; Section 3.1 "Linear transform" and
  * "Quantization"): mean mu[C]; basis T[C][C] whose row j is the j-th principal direction of

@@ -63,7 +63,7 @@ class _StatsOut(C.Structure):
                 ("zero_fraction", C.c_double), ("energy_ratio_90", C.c_double)]
 
 
-EXPORTS = ["tc_create", "tc_destroy", "tc_status_string", "tc_get_status", "tc_fit_pca",
+EXPORTS = ["tc_create", "tc_destroy", "tc_status_string", "tc_get_status", "tc_force_exact_path", "tc_last_path", "tc_fit_pca",
            "tc_model_import", "tc_model_export", "tc_model_free", "tc_build_codebook",
            "tc_codebook_import", "tc_codebook_export", "tc_codebook_free",
            "tc_host_huffman_lengths", "tc_host_eigh", "tc_encode_bound", "tc_encode", "tc_decode",
@@ -92,6 +92,9 @@ def load_library() -> C.CDLL:
         lib.tc_status_string.argtypes = [C.c_int]
         lib.tc_status_string.restype = C.c_char_p
         lib.tc_get_status.argtypes = [vp, vp]
+        lib.tc_force_exact_path.argtypes = [vp, C.c_int]
+        lib.tc_force_exact_path.restype = None
+        lib.tc_last_path.argtypes = [vp, C.c_int]
         lib.tc_fit_pca.argtypes = [vp, P(_Tensor), P(_FitParams), P(vp), vp]
         lib.tc_model_import.argtypes = [vp, P(_ModelDesc), P(vp)]
         lib.tc_model_export.argtypes = [vp, P(_ModelDesc)]
@@ -208,6 +211,14 @@ def tc_create(device: int = 0) -> Context:
     out = C.c_void_p()
     _check(load_library().tc_create(C.byref(out), device), "tc_create")
     return Context(out.value, device)
+
+
+def tc_force_exact_path(ctx: Context, on: bool) -> None:
+    load_library().tc_force_exact_path(ctx.ptr, int(on))
+
+
+def tc_last_path(ctx: Context, decode: bool = False) -> int:
+    return load_library().tc_last_path(ctx.ptr, int(decode))
 
 
 def tc_get_status(ctx: Context) -> int:

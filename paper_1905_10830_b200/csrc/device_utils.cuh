@@ -74,21 +74,23 @@ __device__ __forceinline__ unsigned int group_exclusive_scan_128(unsigned int v,
     return before + inc - v;
 }
 
-// Decoupled look-back over per-tile sizes (called by one full warp).  `own` is this tile's
-// padded size; returns the sum of the sizes of all earlier tiles.  Tile indices come from an
-// atomic ticket, so every earlier tile has been started by a resident block and the waits end;
-// they are bounded all the same, and a wait that runs out clears `ok` and records a timeout.
-__device__ __forceinline__ unsigned long long tile_lookback(unsigned long long *state, long long tile,
-                                                            unsigned long long own, unsigned int *status,
-                                                            bool &ok)
+// Decoupled look-back over per-tile sizes.  A tile first publishes its own padded size
+// (lookback_publish, one thread), later one full warp resolves the sum of the sizes of all
+// earlier tiles (lookback_resolve) and publishes the inclusive prefix.  Every earlier tile is
+// owned by a block that is resident (tickets or a co-resident persistent grid), so the waits
+// end; they are bounded all the same, and a wait that runs out clears `ok` and records a
+// timeout in the status word.
+__device__ __forceinline__ void lookback_publish(unsigned long long *state, long long tile, unsigned long long own)
+{
+    st_volatile_u64(state + tile, (tile == 0 ? kFlagPrefix : kFlagAggregate) | own);
+}
+
+__device__ __forceinline__ unsigned long long lookback_resolve(unsigned long long *state, long long tile,
+                                                               unsigned long long own, unsigned int *status, bool &ok)
 {
     const int lane = threadIdx.x & 31;
     ok = true;
-    if (tile == 0) {
-        if (lane == 0) st_volatile_u64(state, kFlagPrefix | own);
-        return 0;
-    }
-    if (lane == 0) st_volatile_u64(state + tile, kFlagAggregate | own);
+    if (tile == 0) return 0;
     unsigned long long exclusive = 0;
     long long idx = tile - 1;
     const unsigned long long t0 = global_timer_ns();
@@ -120,20 +122,28 @@ __device__ __forceinline__ unsigned long long tile_lookback(unsigned long long *
     return exclusive;
 }
 
+__device__ __forceinline__ unsigned long long tile_lookback(unsigned long long *state, long long tile,
+                                                            unsigned long long own, unsigned int *status, bool &ok)
+{
+    if ((threadIdx.x & 31) == 0) lookback_publish(state, tile, own);
+    __syncwarp();
+    return lookback_resolve(state, tile, own, status, ok);
+}
+
 // MSB-first bit writer into a zero-initialised word array.  The first and the last word a
 // writer touches may be shared with its neighbours and are merged with atomicOr; words in
 // between belong to this writer alone.
 struct BitWriter {
-    uint32_t *words;           // base of the (shared or global) word array
+    uint32_t *words;           // the (shared or global) word holding the writer's first bit
     unsigned long long acc;    // pending bits, right-aligned
     int pending;               // number of pending bits incl. the lead-in of the first word
-    unsigned int word;         // index of the word being filled
+    unsigned int word;         // index of the word being filled, relative to `words`
     bool first;
 
     __device__ __forceinline__ void init(uint32_t *base, unsigned long long bitpos)
     {
-        words = base;
-        word = (unsigned int)(bitpos >> 5);
+        words = base + (bitpos >> 5);
+        word = 0;
         pending = (int)(bitpos & 31);
         acc = 0;
         first = true;

@@ -89,14 +89,15 @@ tc_status finish_model(tc_model *m)
         tmu[j] = s;
         for (int a = 0; a < c; ++a) colsum[a] += m->basis[(size_t)j * c + a];
     }
-    std::vector<float> enc_bias(k), dec_bias(c);
-    for (int j = 0; j < k; ++j) enc_bias[j] = (float)(-(tmu[j] + m->lo) / m->step);
+    std::vector<float> enc_bias(k), dec_bias(c), tmu32(k);
+    for (int j = 0; j < k; ++j) { enc_bias[j] = (float)(-(tmu[j] + m->lo) / m->step); tmu32[j] = (float)tmu[j]; }
     for (int a = 0; a < c; ++a) dec_bias[a] = (float)(m->mean[a] + m->lo * colsum[a]);
     tc_status st;
     if ((st = upload(&m->d_basis64, m->basis)) != TC_OK) return st;
     if ((st = upload(&m->d_mean64, m->mean)) != TC_OK) return st;
     if ((st = upload(&m->d_enc_bias, enc_bias)) != TC_OK) return st;
     if ((st = upload(&m->d_dec_bias, dec_bias)) != TC_OK) return st;
+    if ((st = upload(&m->d_tmu32, tmu32)) != TC_OK) return st;
     if (m->basis_dtype == TC_BF16) {
         std::vector<__nv_bfloat16> b((size_t)k * c), bt((size_t)c * k);
         for (int j = 0; j < k; ++j)
@@ -204,6 +205,17 @@ void tc_destroy(tc_ctx *ctx)
     delete ctx;
 }
 
+void tc_force_exact_path(tc_ctx *ctx, int on)
+{
+    if (ctx) ctx->force_exact = on ? 1 : 0;
+}
+
+int tc_last_path(const tc_ctx *ctx, int decode)
+{
+    if (!ctx) return -1;
+    return decode ? ctx->last_decode_path : ctx->last_encode_path;
+}
+
 tc_status tc_get_status(tc_ctx *ctx, void *cuda_stream)
 {
     if (!ctx) return TC_ERR_INVALID_ARG;
@@ -260,7 +272,7 @@ void tc_model_free(tc_model *m)
     if (!m) return;
     DeviceGuard guard(m->device);
     cudaFree(m->d_basis64); cudaFree(m->d_mean64); cudaFree(m->d_basis_bf16);
-    cudaFree(m->d_basis_t_bf16); cudaFree(m->d_enc_bias); cudaFree(m->d_dec_bias);
+    cudaFree(m->d_basis_t_bf16); cudaFree(m->d_enc_bias); cudaFree(m->d_dec_bias); cudaFree(m->d_tmu32);
     delete m;
 }
 
@@ -471,6 +483,12 @@ tc_status tc_encode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
     a.ticket = (unsigned int *)ctx->scratch;
     a.tile_state = (unsigned long long *)((char *)ctx->scratch + 64);
     a.status = ctx->d_status; a.clamped = nullptr; a.emit = 1;
+    a.basis_bf16 = m->d_basis_bf16; a.enc_bias = m->d_enc_bias; a.tmu32 = m->d_tmu32;
+    if (!ctx->force_exact && x->dtype == TC_BF16 && tc_encode_tc_supported(ctx, a)) {
+        ctx->last_encode_path = 1;
+        return tc_launch_encode_tc(ctx, a, s);
+    }
+    ctx->last_encode_path = 0;
     return tc_launch_encode_simt(ctx, a, x->dtype, s);
 }
 

@@ -26,7 +26,9 @@ struct tc_ctx {
     unsigned int *d_status = nullptr;     // device status word
     void *scratch = nullptr;              // look-back state, ticket counter
     size_t scratch_bytes = 0;
-    cudaEvent_t ev = nullptr;
+    int force_exact = 0;                  // route every tensor through the fp64 kernels
+    int last_encode_path = 0;             // 0 = fp64 kernels, 1 = tensor-core kernels
+    int last_decode_path = 0;
 };
 
 struct tc_model {
@@ -41,6 +43,7 @@ struct tc_model {
     __nv_bfloat16 *d_basis_t_bf16 = nullptr;// [c][k]   transpose, for the inverse projection
     float *d_enc_bias = nullptr;            // [k]  -(T mu + lo)_j / step
     float *d_dec_bias = nullptr;            // [c]  mu_c + lo * sum_j T[j][c]
+    float *d_tmu32 = nullptr;               // [k]  (T mu)_j
 };
 
 struct tc_codebook {
@@ -61,6 +64,9 @@ struct EncodeArgs {
     int chunk_pixels;
     const double *basis64;      // [c][c]
     const double *mean64;       // [c]
+    const __nv_bfloat16 *basis_bf16;   // [k][c]  (tensor-core path)
+    const float *enc_bias;      // [k]  -(T mu + lo)_j / step
+    const float *tmu32;         // [k]  (T mu)_j
     double lo, step;
     const uint32_t *enc;        // [groups][2^bits]
     uint32_t *stream;           // output words
@@ -98,6 +104,8 @@ struct DecodeArgs {
 // ---- launchers (defined in the .cu files) ----------------------------------------------
 tc_status tc_launch_encode_simt(const tc_ctx *ctx, const EncodeArgs &a, int dtype, cudaStream_t s);
 tc_status tc_launch_decode_simt(const tc_ctx *ctx, const DecodeArgs &a, int dtype, cudaStream_t s);
+bool tc_encode_tc_supported(const tc_ctx *ctx, const EncodeArgs &a);
+tc_status tc_launch_encode_tc(const tc_ctx *ctx, const EncodeArgs &a, cudaStream_t s);
 
 tc_status tc_launch_channel_sums(const void *x, int dtype, int n, int c, int hw, double *sums,
                                  cudaStream_t s);

@@ -19,6 +19,16 @@ pytestmark = pytest.mark.gpu
 
 @pytest.fixture(scope="module")
 def ctx():
+    """Context pinned to the fp64 kernels: results must be identical to the oracle's."""
+    c = tc.tc_create(0)
+    tc.tc_force_exact_path(c, True)
+    yield c
+    c.close()
+
+
+@pytest.fixture(scope="module")
+def ctx_tc():
+    """Context on the default route: bf16 tensors take the tensor-core kernels."""
     c = tc.tc_create(0)
     yield c
     c.close()
@@ -58,6 +68,7 @@ def run_case(ctx, spec, bits, n_cal, n_test, dtype, per_channel, *, exact, chunk
     x = o["x"].cuda()
     enc = tc.tc_encode(ctx, model_h, cb, x, chunk_pixels=chunk_pixels, debug=True)
     assert tc.tc_get_status(ctx) == 0
+    assert tc.tc_last_path(ctx) == (0 if exact else 1), "unexpected kernel route"
     cp = enc.layout.chunk_pixels
     # coefficients
     y_gpu = enc.coefficients.cpu().numpy().astype(np.float64)
@@ -118,3 +129,31 @@ def test_chunk_sizes_and_ragged_tail(ctx, cp):
     spec = fm.LayerSpec(32, 9, 9, 0.85, None, 77)
     run_case(ctx, spec, 6, 8, 3, torch.float32, False, exact=True, chunk_pixels=cp)
     run_case(ctx, spec, 3, 8, 3, torch.bfloat16, True, exact=True, chunk_pixels=cp)
+
+
+# ---- tensor-core path (bf16 products, fp32 accumulation) -------------------------------------
+
+@pytest.mark.parametrize("c,s,n,bits", [(64, 56, 2, 4), (128, 28, 3, 4), (256, 14, 5, 4), (96, 28, 2, 5),
+                                        (144, 14, 5, 5), (192, 28, 2, 5), (16, 8, 9, 3), (256, 14, 3, 8)])
+def test_tensor_core_path_shapes(ctx_tc, c, s, n, bits):
+    spec = fm.LayerSpec(c, s, s, 0.9, None, 5000 + c + s)
+    run_case(ctx_tc, spec, bits, 6, n, torch.bfloat16, False, exact=False)
+
+
+@pytest.mark.parametrize("bits", [2, 3, 5, 6, 7])
+def test_tensor_core_path_bit_width_sweep(ctx_tc, bits):
+    spec = fm.workload(5).layers[0]
+    run_case(ctx_tc, spec, bits, 8, 7, torch.bfloat16, False, exact=False)
+
+
+def test_tensor_core_path_per_channel_codebook_and_chunks(ctx_tc):
+    spec = fm.LayerSpec(64, 14, 14, 0.9, None, 5100)
+    for cp in (1, 4, 32):
+        run_case(ctx_tc, spec, 4, 6, 3, torch.bfloat16, True, exact=False, chunk_pixels=cp)
+
+
+def test_tensor_core_path_high_rate_tile_overflows_staging(ctx_tc):
+    # nearly uniform symbols at 8 bits: a 128-pixel tile of 256 channels packs to more than the
+    # staging buffer holds, which exercises the direct-to-global packing route
+    spec = fm.LayerSpec(256, 14, 14, 0.999, None, 5200)
+    run_case(ctx_tc, spec, 8, 6, 3, torch.bfloat16, False, exact=False)
