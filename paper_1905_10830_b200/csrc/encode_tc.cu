@@ -41,6 +41,54 @@ __host__ __device__ inline SmemLayout smem_layout(int c, int k, int enc_entries)
     return l;
 }
 
+// Quantiser in fp32: v = acc/step - (T mu + lo)/step, rounded to the nearest integer (ties to
+// even) by adding 1.5 * 2^23 -- the integer then sits in the low mantissa bits -- and clamped to
+// [0, 2^b - 1] while still a float.  (A float -> int conversion instruction would do the same
+// but issues at a quarter of the rate.)
+constexpr float kMagic = 12582912.0f;
+__device__ __forceinline__ uint32_t quantise(float acc, float inv_step, float bias, float vmax)
+{
+    const float v = fminf(fmaxf(fmaf(acc, inv_step, bias) + kMagic, kMagic), vmax);
+    return __float_as_uint(v) & 0xffu;
+}
+
+// Bit writer into the shared-memory staging buffer.  A word is stored (plain, predicated
+// store) by the writer that supplies its last bit; bits that other writers own in that word
+// are zero in the stored value.  What is left after the last full word -- a writer's tail --
+// is merged afterwards with one shared-memory OR per writer (finish()), behind a barrier, so
+// that it cannot be overwritten by the store of the word's last writer.  A put adds fewer
+// than 32 bits (the pending count stays below 32 between puts).
+struct SmemBitWriter {
+    uint32_t addr;             // shared address of the word being filled
+    uint32_t lo, hi;           // pending bits, right-aligned in hi:lo (bits above `pending` are stale)
+    int pending;
+    __device__ __forceinline__ void init(uint32_t base_addr, unsigned int bitpos)
+    {
+        addr = base_addr + (bitpos >> 5) * 4u;
+        pending = (int)(bitpos & 31u);
+        lo = hi = 0;
+    }
+    __device__ __forceinline__ void put(uint32_t code, int len)
+    {
+        hi = __funnelshift_l(lo, hi, len);
+        lo = (lo << len) | code;
+        pending += len;
+        const uint32_t flush = pending >= 32 ? 1u : 0u;
+        const uint32_t out = __funnelshift_r(lo, hi, pending - 32);
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.shared.u32 [%0], %1;\n\t}"
+                     ::"r"(addr), "r"(out), "r"(flush));
+        addr += flush * 4u;
+        pending -= (int)(flush * 32u);
+    }
+    // call after a barrier that follows every writer's puts
+    __device__ __forceinline__ void finish()
+    {
+        const uint32_t out = pending > 0 ? (lo << (32 - pending)) : 0u;
+        if (out) asm volatile("red.shared.or.b32 [%0], %1;" ::"r"(addr), "r"(out) : "memory");
+    }
+};
+
+template <bool kPerChannel, bool kDebug>
 __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -52,7 +100,7 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nsym = 1 << a.bits;
-    const bool enc_in_smem = a.groups == 1;
+    constexpr bool enc_in_smem = !kPerChannel;
     const SmemLayout L = smem_layout(a.c, a.k, enc_in_smem ? nsym : 0);
     unsigned char *s_basis = smem + L.basis;
     uint32_t *s_enc = reinterpret_cast<uint32_t *>(smem + L.enc);
@@ -171,12 +219,35 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
         const int grp = warp >> 2;                 // 0 or 1
         const int t = tid & 127;                   // pixel within the tile = TMEM lane
         const int wq = warp & 3;
-        uint32_t *stg = reinterpret_cast<uint32_t *>(smem + L.staging + grp * kStagingBytes);
-        const uint32_t *enc = enc_in_smem ? s_enc : a.enc;
+        const uint32_t stg_addr = smem_u32(smem + L.staging + grp * kStagingBytes);
+        const uint32_t enc_addr = smem_u32(s_enc);
         const float inv_step = (float)(1.0 / a.step);
-        const int top = nsym - 1;
+        const float vmax = kMagic + (float)(nsym - 1);
         const int bar_id = 1 + grp;
         bool alive = true;
+
+        // code table entry of symbol q of coefficient j: (code << 8) | length
+        auto lookup = [&](int j, uint32_t q) -> uint32_t {
+            if constexpr (kPerChannel) return __ldg(a.enc + j * nsym + q);
+            else {
+                uint32_t e;
+                asm("ld.shared.u32 %0, [%1];" : "=r"(e) : "r"(enc_addr + q * 4u));
+                return e;
+            }
+        };
+        auto resolve_base = [&](long long tile, unsigned long long padded) {
+            if (wq == 0) {
+                bool ok;
+                const unsigned long long base = lookback_resolve(a.tile_state, tile, padded, a.status, ok);
+                if (lane == 0) {
+                    const bool fits = base + padded <= a.capacity_bits;
+                    if (ok && !fits) tc_dev_set_status(a.status, TC_ERR_BUFFER_TOO_SMALL);
+                    s_base[grp] = base;
+                    s_write_ok[grp] = (ok && fits) ? 1 : 0;
+                }
+            }
+        };
+
         for (long long tl = grp; tl < my_tiles && alive; tl += 2) {
             const long long tile = blockIdx.x + tl * gridDim.x;
             const long long p = tile * TC_TILE_PIXELS + t;
@@ -188,24 +259,20 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
             // pass 1: code lengths
             unsigned int my_bits = 0;
             for (int c0 = 0; c0 < a.k; c0 += 32) {
-                uint32_t r[32];
-                const int n = min(32, a.k - c0);
-                if (n == 32) tmem_ld_32x32b_x32(trow + c0, r);
-                else {
+                if (a.k - c0 >= 32) {
+                    uint32_t r[32];
+                    tmem_ld_32x32b_x32(trow + c0, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        my_bits += lookup(c0 + i, quantise(__uint_as_float(r[i]), inv_step, s_bias[c0 + i], vmax)) & 0xffu;
+                } else {
                     uint32_t r16[16];
                     tmem_ld_32x32b_x16(trow + c0, r16);
+                    tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) r[i] = r16[i];
-                }
-                tmem_ld_wait();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    if (i < n) {
-                        const int j = c0 + i;
-                        int q = __float2int_rn(fmaf(__uint_as_float(r[i]), inv_step, s_bias[j]));
-                        q = max(0, min(q, top));
-                        my_bits += enc[(a.groups == 1 ? 0 : j * nsym) + q] & 0xffu;
-                    }
+                    for (int i = 0; i < 16; ++i)
+                        my_bits += lookup(c0 + i, quantise(__uint_as_float(r16[i]), inv_step, s_bias[c0 + i], vmax)) & 0xffu;
                 }
             }
             if (!valid) my_bits = 0;
@@ -215,86 +282,90 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
             if (t == 0) lookback_publish(a.tile_state, tile, padded);
             const bool staged = padded <= (unsigned long long)kStagingBytes * 8ull;
 
-            uint32_t *out_words = stg;
-            unsigned long long out_bit = my_off;
             if (staged) {
-                uint4 *z = reinterpret_cast<uint4 *>(stg);
-                for (unsigned int i = t; i < (unsigned int)(padded >> 7); i += 128) z[i] = make_uint4(0u, 0u, 0u, 0u);
+                // every word below tile_bits / 32 is stored by the writer of its last bit; the last
+                // partial word and the padding up to the 128-bit boundary start as zero
+                const unsigned int first_open = tile_bits >> 5, end_word = (unsigned int)(padded >> 5);
+                if (t < end_word - first_open)
+                    asm volatile("st.shared.u32 [%0], %1;" ::"r"(stg_addr + (first_open + t) * 4u), "r"(0u) : "memory");
             } else {
                 // rare: the tile does not fit the staging buffer -> resolve its position first and
                 // pack straight into (zeroed) global memory
-                if (wq == 0) {
-                    bool ok;
-                    const unsigned long long base = lookback_resolve(a.tile_state, tile, padded, a.status, ok);
-                    if (lane == 0) {
-                        const bool fits = base + padded <= a.capacity_bits;
-                        if (ok && !fits) tc_dev_set_status(a.status, TC_ERR_BUFFER_TOO_SMALL);
-                        s_base[grp] = base;
-                        s_write_ok[grp] = (ok && fits) ? 1 : 0;
-                    }
-                }
+                resolve_base(tile, padded);
                 named_bar_sync(bar_id, 128);
                 if (s_write_ok[grp]) {
                     uint4 *z = reinterpret_cast<uint4 *>(a.stream + (s_base[grp] >> 5));
                     for (unsigned int i = t; i < (unsigned int)(padded >> 7); i += 128) z[i] = make_uint4(0u, 0u, 0u, 0u);
                 }
-                out_words = a.stream;
-                out_bit = s_base[grp] + my_off;
             }
             named_bar_sync(bar_id, 128);
 
-            // pass 2: quantise again, look up codes, pack
+            // pass 2: quantise again, look up codes, pack (two symbols are joined in registers and
+            // appended as one piece of at most 24 bits)
             const bool do_pack = valid && (staged || s_write_ok[grp]);
-            BitWriter w;
-            w.init(out_words, out_bit);
-            for (int c0 = 0; c0 < a.k; c0 += 32) {
-                uint32_t r[32];
-                const int n = min(32, a.k - c0);
-                if (n == 32) tmem_ld_32x32b_x32(trow + c0, r);
-                else {
-                    uint32_t r16[16];
-                    tmem_ld_32x32b_x16(trow + c0, r16);
+            auto pack_tile = [&](auto &w) {
+                for (int c0 = 0; c0 < a.k; c0 += 32) {
+                    uint32_t r[32];
+                    const bool full = a.k - c0 >= 32;
+                    if (full) tmem_ld_32x32b_x32(trow + c0, r);
+                    else {
+                        uint32_t r16[16];
+                        tmem_ld_32x32b_x16(trow + c0, r16);
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) r[i] = r16[i];
-                }
-                tmem_ld_wait();
-                if (do_pack) {
+                        for (int i = 0; i < 16; ++i) r[i] = r16[i];
+                    }
+                    tmem_ld_wait();
+                    if (do_pack) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        if (i < n) {
-                            const int j = c0 + i;
-                            const float accv = __uint_as_float(r[i]);
-                            int q = __float2int_rn(fmaf(accv, inv_step, s_bias[j]));
-                            q = max(0, min(q, top));
-                            const uint32_t e = enc[(a.groups == 1 ? 0 : j * nsym) + q];
-                            w.put(e >> 8, (int)(e & 0xffu));
-                            if (a.dbg_coef) a.dbg_coef[p * a.k + j] = accv - a.tmu32[j];
-                            if (a.dbg_sym) a.dbg_sym[p * a.k + j] = (uint8_t)q;
+                        for (int i = 0; i < 32; i += 2) {
+                            if (i < 16 || full) {
+                                const uint32_t q0 = quantise(__uint_as_float(r[i]), inv_step, s_bias[c0 + i], vmax);
+                                const uint32_t q1 = quantise(__uint_as_float(r[i + 1]), inv_step, s_bias[c0 + i + 1], vmax);
+                                const uint32_t e0 = lookup(c0 + i, q0), e1 = lookup(c0 + i + 1, q1);
+                                const uint32_t l1 = e1 & 0xffu;
+                                w.put(((e0 >> 8) << l1) | (e1 >> 8), (int)((e0 & 0xffu) + l1));
+                                if constexpr (kDebug) {
+                                    if (a.dbg_coef) {
+                                        a.dbg_coef[p * a.k + c0 + i] = __uint_as_float(r[i]) - a.tmu32[c0 + i];
+                                        a.dbg_coef[p * a.k + c0 + i + 1] = __uint_as_float(r[i + 1]) - a.tmu32[c0 + i + 1];
+                                    }
+                                    if (a.dbg_sym) {
+                                        a.dbg_sym[p * a.k + c0 + i] = (uint8_t)q0;
+                                        a.dbg_sym[p * a.k + c0 + i + 1] = (uint8_t)q1;
+                                    }
+                                }
+                            }
                         }
                     }
                 }
+            };
+            if (staged) {
+                SmemBitWriter ws;
+                ws.init(stg_addr, my_off);
+                pack_tile(ws);
+                named_bar_sync(bar_id, 128);      // all full words stored
+                if (do_pack) ws.finish();
+            } else {
+                BitWriter wg;
+                wg.init(a.stream, s_base[grp] + my_off);
+                pack_tile(wg);
+                if (do_pack) wg.finish();
             }
-            if (do_pack) w.finish();
             // the accumulator buffer is free for the tile after next
             tc_fence_before_sync();
             mbar_arrive(smem_u32(&s_tempty[grp]));
 
             if (staged) {
-                if (wq == 0) {
-                    bool ok;
-                    const unsigned long long base = lookback_resolve(a.tile_state, tile, padded, a.status, ok);
-                    if (lane == 0) {
-                        const bool fits = base + padded <= a.capacity_bits;
-                        if (ok && !fits) tc_dev_set_status(a.status, TC_ERR_BUFFER_TOO_SMALL);
-                        s_base[grp] = base;
-                        s_write_ok[grp] = (ok && fits) ? 1 : 0;
-                    }
-                }
+                resolve_base(tile, padded);
                 named_bar_sync(bar_id, 128);      // staging complete, base known
                 if (s_write_ok[grp]) {
                     uint4 *dst = reinterpret_cast<uint4 *>(a.stream + (s_base[grp] >> 5));
-                    const uint4 *srcv = reinterpret_cast<const uint4 *>(stg);
-                    for (unsigned int i = t; i < (unsigned int)(padded >> 7); i += 128) dst[i] = srcv[i];
+                    for (unsigned int i = t; i < (unsigned int)(padded >> 7); i += 128) {
+                        uint4 v;
+                        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                                     : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(stg_addr + i * 16u));
+                        dst[i] = v;
+                    }
                 }
             }
             const unsigned long long base = s_base[grp];
@@ -331,13 +402,16 @@ tc_status tc_launch_encode_tc(const tc_ctx *ctx, const EncodeArgs &a, cudaStream
 {
     if (a.n_tiles <= 0) return TC_OK;
     const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.bits) : 0);
-    if (cudaFuncSetAttribute(encode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.total) != cudaSuccess)
+    const bool per_channel = a.groups != 1, debug = a.dbg_coef || a.dbg_sym;
+    void (*kernel)(EncodeArgs) = per_channel ? (debug ? encode_tc_kernel<true, true> : encode_tc_kernel<true, false>)
+                                             : (debug ? encode_tc_kernel<false, true> : encode_tc_kernel<false, false>);
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.total) != cudaSuccess)
         return TC_ERR_CUDA;
     const unsigned int grid = (unsigned int)((a.n_tiles < ctx->sm_count) ? a.n_tiles : ctx->sm_count);
     EncodeArgs args = a;
     void *params[] = {&args};
     // cooperative launch: the grid must be co-resident, which is what makes the look-back safe
-    if (cudaLaunchCooperativeKernel((void *)encode_tc_kernel, dim3(grid), dim3(kThreads), params, l.total, s) != cudaSuccess) {
+    if (cudaLaunchCooperativeKernel((void *)kernel, dim3(grid), dim3(kThreads), params, l.total, s) != cudaSuccess) {
         cudaGetLastError();
         return TC_ERR_CUDA;
     }

@@ -91,7 +91,12 @@ tc_status finish_model(tc_model *m)
     }
     std::vector<float> enc_bias(k), dec_bias(c), tmu32(k);
     for (int j = 0; j < k; ++j) { enc_bias[j] = (float)(-(tmu[j] + m->lo) / m->step); tmu32[j] = (float)tmu[j]; }
-    for (int a = 0; a < c; ++a) dec_bias[a] = (float)(m->mean[a] + m->lo * colsum[a]);
+    // The inverse projection runs on symbols centred on the level nearest to y = 0, so that the
+    // accumulators stay small and no large terms cancel in fp32:
+    // x_hat = step * sum_j T[j][c] (q_j - center) + mu_c + (lo + center*step) * sum_j T[j][c]
+    const double top = (double)((1 << m->bits) - 1);
+    m->center = (int)std::min(top, std::max(0.0, std::nearbyint(-m->lo / m->step)));
+    for (int a = 0; a < c; ++a) dec_bias[a] = (float)(m->mean[a] + (m->lo + m->center * m->step) * colsum[a]);
     tc_status st;
     if ((st = upload(&m->d_basis64, m->basis)) != TC_OK) return st;
     if ((st = upload(&m->d_mean64, m->mean)) != TC_OK) return st;
@@ -121,6 +126,7 @@ tc_status finish_codebook(tc_codebook *cb)
     cb->lut_bits = mx;
     std::vector<uint32_t> enc((size_t)cb->groups * nsym);
     std::vector<uint16_t> lut((size_t)cb->groups << cb->lut_bits);
+    std::vector<uint32_t> lut32((size_t)cb->groups << cb->lut_bits);
     std::vector<uint32_t> code(nsym);
     for (int g = 0; g < cb->groups; ++g) {
         const uint8_t *len = cb->lengths.data() + (size_t)g * nsym;
@@ -130,12 +136,18 @@ tc_status finish_codebook(tc_codebook *cb)
             // every table index whose leading bits equal the code decodes to this symbol
             const uint32_t first = code[s] << (cb->lut_bits - len[s]);
             const uint32_t span = 1u << (cb->lut_bits - len[s]);
-            for (uint32_t i = 0; i < span; ++i)
+            const float as_float = (float)s;
+            uint32_t fbits;
+            std::memcpy(&fbits, &as_float, 4);               // small integers are exact in bf16
+            for (uint32_t i = 0; i < span; ++i) {
                 lut[((size_t)g << cb->lut_bits) + first + i] = (uint16_t)((s << 8) | len[s]);
+                lut32[((size_t)g << cb->lut_bits) + first + i] = (fbits & 0xffff0000u) | ((uint32_t)s << 8) | len[s];
+            }
         }
     }
     tc_status st;
     if ((st = upload(&cb->d_enc, enc)) != TC_OK) return st;
+    if ((st = upload(&cb->d_lut32, lut32)) != TC_OK) return st;
     return upload(&cb->d_lut, lut);
 }
 
@@ -414,6 +426,7 @@ void tc_codebook_free(tc_codebook *cb)
     DeviceGuard guard(cb->device);
     cudaFree(cb->d_enc);
     cudaFree(cb->d_lut);
+    cudaFree(cb->d_lut32);
     delete cb;
 }
 
@@ -513,6 +526,12 @@ tc_status tc_decode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
     a.chunk_pixels = cp; a.lut_bits = cb->lut_bits; a.lut = cb->d_lut;
     a.basis64 = m->d_basis64; a.mean64 = m->d_mean64; a.lo = m->lo; a.step = m->step;
     a.xhat = x_hat->data; a.status = ctx->d_status;
+    a.lut32 = cb->d_lut32; a.basis_t_bf16 = m->d_basis_t_bf16; a.dec_bias = m->d_dec_bias; a.center = m->center;
+    if (!ctx->force_exact && x_hat->dtype == TC_BF16 && tc_decode_tc_supported(ctx, a)) {
+        ctx->last_decode_path = 1;
+        return tc_launch_decode_tc(ctx, a, (cudaStream_t)cuda_stream);
+    }
+    ctx->last_decode_path = 0;
     return tc_launch_decode_simt(ctx, a, x_hat->dtype, (cudaStream_t)cuda_stream);
 }
 

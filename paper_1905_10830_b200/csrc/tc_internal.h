@@ -34,6 +34,7 @@ struct tc_ctx {
 struct tc_model {
     int c = 0, k = 0, bits = 0, basis_dtype = 0;
     double lo = 0, step = 0;
+    int center = 0;                         // symbol whose level is nearest to y = 0
     std::vector<double> basis, mean, eig;   // host copies (basis [c][c])
     int device = 0;
     // device copies
@@ -42,7 +43,7 @@ struct tc_model {
     __nv_bfloat16 *d_basis_bf16 = nullptr;  // [k][c]   (bf16 models only)
     __nv_bfloat16 *d_basis_t_bf16 = nullptr;// [c][k]   transpose, for the inverse projection
     float *d_enc_bias = nullptr;            // [k]  -(T mu + lo)_j / step
-    float *d_dec_bias = nullptr;            // [c]  mu_c + lo * sum_j T[j][c]
+    float *d_dec_bias = nullptr;            // [c]  mu_c + (lo + center*step) * sum_j T[j][c]
     float *d_tmu32 = nullptr;               // [k]  (T mu)_j
 };
 
@@ -52,6 +53,7 @@ struct tc_codebook {
     int device = 0;
     uint32_t *d_enc = nullptr;              // [groups][2^bits]  (code << 8) | length
     uint16_t *d_lut = nullptr;              // [groups][2^lut_bits]  (symbol << 8) | length
+    uint32_t *d_lut32 = nullptr;            // [groups][2^lut_bits]  bf16(symbol) << 16 | symbol << 8 | length
 };
 
 // ---- kernel argument blocks -------------------------------------------------------------
@@ -94,6 +96,10 @@ struct DecodeArgs {
     int chunk_pixels;
     int lut_bits;
     const uint16_t *lut;
+    const uint32_t *lut32;              // tensor-core path
+    const __nv_bfloat16 *basis_t_bf16;  // [c][k]
+    const float *dec_bias;              // [c]
+    int center;                         // subtracted from every symbol before the MMA
     const double *basis64;
     const double *mean64;
     double lo, step;
@@ -106,6 +112,8 @@ tc_status tc_launch_encode_simt(const tc_ctx *ctx, const EncodeArgs &a, int dtyp
 tc_status tc_launch_decode_simt(const tc_ctx *ctx, const DecodeArgs &a, int dtype, cudaStream_t s);
 bool tc_encode_tc_supported(const tc_ctx *ctx, const EncodeArgs &a);
 tc_status tc_launch_encode_tc(const tc_ctx *ctx, const EncodeArgs &a, cudaStream_t s);
+bool tc_decode_tc_supported(const tc_ctx *ctx, const DecodeArgs &a);
+tc_status tc_launch_decode_tc(const tc_ctx *ctx, const DecodeArgs &a, cudaStream_t s);
 
 tc_status tc_launch_channel_sums(const void *x, int dtype, int n, int c, int hw, double *sums,
                                  cudaStream_t s);

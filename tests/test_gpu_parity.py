@@ -4,7 +4,8 @@ oracle's model and codebook imported into the library (identical T, mu, lo, step
 Bars: the entropy-coded stream is bit-exact given identical symbols and decode round-trips
 exactly; projected coefficients agree within 1e-3 * max(|y|, step); at most 1e-4 of the
 symbols differ, only by +-1 and only where the oracle's position (y - lo)/step lies within
-1e-3 of a half-integer; x_hat agrees within 1e-3 * max(|x_hat|, step)."""
+1e-3 of a half-integer; x_hat agrees within max(1e-3 * max(|x_hat|, step), one output ulp)
+and is bit-identical for at least 99.9 % of the values."""
 import numpy as np
 import pytest
 import torch
@@ -83,14 +84,18 @@ def run_case(ctx, spec, bits, n_cal, n_test, dtype, per_channel, *, exact, chunk
     # decode: reconstruct what the stream holds
     xhat = tc.tc_decode(ctx, model_h, cb, enc, x.shape, dtype)
     assert tc.tc_get_status(ctx) == 0
+    assert tc.tc_last_path(ctx, True) == (0 if exact else 1), "unexpected kernel route"
     want = oracle.reconstruct(m, q_gpu, x.shape, out_bf16=(dtype == torch.bfloat16))
     got = xhat.float().cpu().numpy()
     if exact:
         assert np.array_equal(got, want)
     else:
-        assert np.all(np.abs(got - want) <= 1e-3 * np.maximum(np.abs(want), m.step))
-        ulp = np.abs(want) * (2.0 ** -8 if dtype == torch.bfloat16 else 2.0 ** -23) + 1e-30
-        assert (np.abs(got - want) <= ulp).mean() >= 0.999
+        # fp32 accumulation may land on the other side of an output rounding boundary: allow one
+        # unit in the last place of the output type there, and demand bit equality for 99.9 %
+        mant = 7 if dtype == torch.bfloat16 else 23
+        ulp = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(want), 1e-30))) - mant)
+        assert np.all(np.abs(got - want) <= np.maximum(1e-3 * np.maximum(np.abs(want), m.step), ulp))
+        assert (got == want).mean() >= 0.999
     model_h.close()
     cb.close()
     return o, enc
