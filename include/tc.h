@@ -199,6 +199,30 @@ tc_status tc_encode(tc_ctx *ctx, const tc_model *model, const tc_codebook *cb,
                     size_t capacity, uint32_t *chunk_off, uint64_t *tile_off,
                     const tc_debug_out *debug, void *cuda_stream);
 
+/* tc_encode without any allocation.  (The paper has no counterpart: this entry point exists
+ * for the sake of how the library is deployed, not of the method.)
+ *
+ * tc_encode keeps its cross-tile bookkeeping in a scratch arena that the context enlarges with
+ * cudaMalloc when a bigger tensor arrives.  Callers that may not allocate -- a server that
+ * fixes its memory budget at start-up, a pipeline that cannot afford the device-wide stall of
+ * cudaMalloc / cudaFree next to its other streams, a plug-in whose host owns the allocator --
+ * use this variant instead: the bookkeeping lives in a fixed array inside the library image
+ * (about 0.5 MB on every GPU that loads the library, held until the process exits), and the
+ * call runs no cudaMalloc, cudaFree or other allocating routine.
+ *   - Same arguments, outputs, asynchrony and errors as tc_encode, minus the debug outputs.
+ *   - Tensors of more than TC_NOALLOC_MAX_TILES tiles of 128 pixels (N*H*W > 8 388 608
+ *     pixels) are refused with TC_ERR_UNSUPPORTED; nothing is launched.
+ *   - The first call on a device looks up the array's device address; make that first call
+ *     outside any stream capture.
+ *   - All calls on a device, from every context, share the one array (it is cleared on the
+ *     stream at the start of each call).  Two calls that can overlap on the GPU -- different
+ *     streams, no dependency -- race on it and corrupt each other's streams: serialise them. */
+#define TC_NOALLOC_MAX_TILES 65536
+tc_status tc_encode_noalloc(tc_ctx *ctx, const tc_model *model, const tc_codebook *cb,
+                            const tc_tensor *x, const tc_encode_params *params, void *stream_out,
+                            size_t capacity, uint32_t *chunk_off, uint64_t *tile_off,
+                            void *cuda_stream);
+
 /* Decode (Section 3: VLD, inverse quantiser, inverse transform; no non-linearity is applied).
  *   stream       DEVICE, 16-byte aligned, `stream_bytes` readable bytes
  *   x_hat        caller-allocated tensor of the shape and dtype that was encoded

@@ -66,7 +66,7 @@ class _StatsOut(C.Structure):
 EXPORTS = ["tc_create", "tc_destroy", "tc_status_string", "tc_get_status", "tc_force_exact_path", "tc_last_path", "tc_fit_pca",
            "tc_model_import", "tc_model_export", "tc_model_free", "tc_build_codebook",
            "tc_codebook_import", "tc_codebook_export", "tc_codebook_free",
-           "tc_host_huffman_lengths", "tc_host_eigh", "tc_encode_bound", "tc_encode", "tc_decode",
+           "tc_host_huffman_lengths", "tc_host_eigh", "tc_encode_bound", "tc_encode", "tc_encode_noalloc", "tc_decode",
            "tc_stats"]
 
 _lib = None
@@ -110,6 +110,7 @@ def load_library() -> C.CDLL:
         lib.tc_encode_bound.argtypes = [vp, vp, P(_Tensor), P(_EncodeParams), P(_StreamLayout)]
         lib.tc_encode.argtypes = [vp, vp, vp, P(_Tensor), P(_EncodeParams), vp, C.c_size_t, vp, vp,
                                   P(_DebugOut), vp]
+        lib.tc_encode_noalloc.argtypes = [vp, vp, vp, P(_Tensor), P(_EncodeParams), vp, C.c_size_t, vp, vp, vp]
         lib.tc_decode.argtypes = [vp, vp, vp, vp, C.c_size_t, vp, vp, P(_EncodeParams), P(_Tensor), vp]
         lib.tc_stats.argtypes = [vp, vp, vp, P(_Tensor), P(_StatsOut), vp]
         _lib = lib
@@ -345,6 +346,19 @@ def tc_encode(ctx: Context, model: Model, cb: Codebook, x: torch.Tensor, *, chun
     _check(load_library().tc_encode(ctx.ptr, model.ptr, cb.ptr, C.byref(t), C.byref(p), out.words.data_ptr(), cap,
                                     out.chunk_off.data_ptr(), out.tile_off.data_ptr(),
                                     C.byref(dbg) if dbg is not None else None, _stream_ptr(ctx.device)), "tc_encode")
+    return out
+
+
+def tc_encode_noalloc(ctx: Context, model: Model, cb: Codebook, x: torch.Tensor, out: EncodedStream, *,
+                      chunk_pixels: int = 0) -> EncodedStream:
+    """Encode `x` into buffers the caller already owns, through the entry point that never
+    allocates device memory (see tc_encode_noalloc in include/tc.h).  `out` must come from an
+    earlier tc_encode of the same shape or be sized with tc_encode_bound."""
+    t = _tensor(x)
+    p = _EncodeParams(chunk_pixels)
+    _check(load_library().tc_encode_noalloc(ctx.ptr, model.ptr, cb.ptr, C.byref(t), C.byref(p), out.words.data_ptr(),
+                                            out.words.numel(), out.chunk_off.data_ptr(), out.tile_off.data_ptr(),
+                                            _stream_ptr(ctx.device)), "tc_encode_noalloc")
     return out
 
 

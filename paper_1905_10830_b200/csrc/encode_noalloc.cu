@@ -1,0 +1,102 @@
+// tc_encode_noalloc: tc_encode for callers that are not allowed to allocate device memory.
+//
+// tc_encode keeps the state of its cross-tile look-back (one 64-bit word per 128-pixel tile,
+// plus a ticket counter) in a scratch arena that the context grows with cudaMalloc when a
+// larger tensor arrives.  Some users of this library cannot accept that: a serving process
+// that reserves its whole memory budget at start-up and treats any later cudaMalloc as a bug;
+// a pipeline whose other streams must not be stalled by the device-wide synchronisation that
+// cudaMalloc / cudaFree imply; a plug-in running under a host application that owns the
+// allocator.  For them the same look-back state lives in a fixed array that is part of the
+// library image, so the call touches no allocator at all.
+#include <mutex>
+
+#include "tc_internal.h"
+
+namespace {
+
+constexpr size_t kScratchHeader = 64;   // ticket counter, padded
+constexpr size_t kScratchBytes = kScratchHeader + (size_t)TC_NOALLOC_MAX_TILES * sizeof(unsigned long long);
+
+// Lives in every device that loads the library, from load until the process exits (about 0.5 MB).
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kScratchBytes];
+
+// In host code `g_noalloc_scratch` is only a handle for the runtime, not a device address; the
+// address the kernels need is asked for once per device, with that device current.
+constexpr int kMaxDevices = 64;
+void *g_scratch_addr[kMaxDevices] = {};
+std::mutex g_scratch_mutex;
+
+tc_status scratch_address(int device, void **out)
+{
+    if (device < 0 || device >= kMaxDevices) return TC_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_scratch_addr[device]) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) {
+            cudaGetLastError();
+            return TC_ERR_CUDA;
+        }
+        g_scratch_addr[device] = ptr;
+    }
+    *out = g_scratch_addr[device];
+    return TC_OK;
+}
+
+struct CurrentDevice {
+    int prev = -1;
+    bool ok = true;
+    explicit CurrentDevice(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~CurrentDevice() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+}  // namespace
+
+extern "C" tc_status tc_encode_noalloc(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const tc_tensor *x,
+                                       const tc_encode_params *params, void *stream_out, size_t capacity,
+                                       uint32_t *chunk_off, uint64_t *tile_off, void *cuda_stream)
+{
+    if (!ctx || !tile_off) return TC_ERR_INVALID_ARG;
+    tc_stream_layout lay;
+    tc_status st = tc_encode_bound(m, cb, x, params, &lay);      // argument checks, chunk size (host only)
+    if (st != TC_OK) return st;
+    if (lay.n_tiles > TC_NOALLOC_MAX_TILES) return TC_ERR_UNSUPPORTED;   // tensor too large for the fixed scratch
+    const long long pixels = (long long)x->n * x->h * x->w;
+    if (pixels > 0 && (!stream_out || !chunk_off)) return TC_ERR_INVALID_ARG;
+    if (((uintptr_t)stream_out & 15u) != 0) return TC_ERR_INVALID_ARG;
+    CurrentDevice guard(ctx->device);
+    if (!guard.ok) return TC_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    if (lay.n_tiles == 0) {
+        if (cudaMemsetAsync(tile_off, 0, sizeof(uint64_t), s) != cudaSuccess) { cudaGetLastError(); return TC_ERR_CUDA; }
+        return TC_OK;
+    }
+    void *scratch = nullptr;
+    if ((st = scratch_address(ctx->device, &scratch)) != TC_OK) return st;
+    // The array still holds the previous call's tickets and tile states: everything this call
+    // will read has to start at zero.
+    const size_t used = kScratchHeader + (size_t)lay.n_tiles * sizeof(unsigned long long);
+    if (cudaMemsetAsync(scratch, 0, used, s) != cudaSuccess) { cudaGetLastError(); return TC_ERR_CUDA; }
+
+    EncodeArgs a{};
+    a.x = x->data; a.n = x->n; a.c = x->c; a.hw = x->h * x->w; a.k = m->k; a.bits = m->bits; a.groups = cb->groups;
+    a.pixels = pixels; a.n_tiles = lay.n_tiles; a.chunk_pixels = lay.chunk_pixels;
+    a.basis64 = m->d_basis64; a.mean64 = m->d_mean64; a.lo = m->lo; a.step = m->step;
+    a.enc = cb->d_enc; a.stream = (uint32_t *)stream_out;
+    a.capacity_bits = (unsigned long long)(capacity & ~(size_t)15) * 8ull;
+    a.chunk_off = chunk_off; a.tile_off = (unsigned long long *)tile_off;
+    a.dbg_coef = nullptr; a.dbg_sym = nullptr;
+    a.ticket = (unsigned int *)scratch;
+    a.tile_state = (unsigned long long *)((char *)scratch + kScratchHeader);
+    a.status = ctx->d_status; a.clamped = nullptr; a.emit = 1;
+    a.basis_bf16 = m->d_basis_bf16; a.enc_bias = m->d_enc_bias; a.tmu32 = m->d_tmu32;
+    if (!ctx->force_exact && x->dtype == TC_BF16 && tc_encode_tc_supported(ctx, a)) {
+        ctx->last_encode_path = 1;
+        return tc_launch_encode_tc(ctx, a, s);
+    }
+    ctx->last_encode_path = 0;
+    return tc_launch_encode_simt(ctx, a, x->dtype, s);
+}
