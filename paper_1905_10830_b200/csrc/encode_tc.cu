@@ -1,10 +1,13 @@
 // Fused tensor-core encode for bf16 tensors (Section 3: transform, quantiser, VLC).
 //
 // One persistent block per SM walks tiles of 128 consecutive pixels.  Warp roles:
-//   warps 0-3, 4-7  two epilogue groups (alternating tiles): TMEM -> registers, quantise,
-//                   code lookup, bit offsets (scan + tile look-back), pack, 128-bit stores
-//   warps 8-11      loaders: cp.async NCHW -> shared memory in the MMA's MN-major layout
-//   warp 12         one thread issues tcgen05.mma:  D[pixel][coef] = X_tile[pixel][c] * T[coef][c]
+//   warps 0-7, 8-15  two epilogue groups (alternating tiles).  Within a group warps 0-3 own the
+//                    first half of the coefficients of the tile's 128 pixels and warps 4-7 the
+//                    second half: TMEM -> registers, quantise, code lengths, bit offsets (scan +
+//                    tile look-back), pack, 128-bit stores.  The symbols stay packed in
+//                    registers between the length pass and the packing pass.
+//   warps 16-19      loaders: cp.async NCHW -> shared memory in the MMA's MN-major layout
+//   warp 20          one thread issues tcgen05.mma:  D[pixel][coef] = X_tile[pixel][c] * T[coef][c]
 // The basis T (bf16, K x C) stays resident in shared memory; the X tile streams through a ring
 // of 64-channel panels; the fp32 accumulators are double-buffered in tensor memory so that the
 // epilogue of one tile overlaps the loads and MMAs of the next.
@@ -21,12 +24,15 @@ constexpr int kStages = 4;
 constexpr int kStageBytes = kPanelCh * TC_TILE_PIXELS * 2;   // 16 KB
 constexpr int kLag = 3;                           // cp.async groups kept in flight per loader thread
 constexpr int kStagingBytes = 16384;              // packed-bit staging per epilogue group
-constexpr int kThreads = 13 * 32;
+constexpr int kEpiWarps = 16;                     // 2 groups x (2 column halves x 4 lane quarters)
+constexpr int kLoaderWarp0 = kEpiWarps, kMmaWarp = kEpiWarps + 4;
+constexpr int kThreads = (kEpiWarps + 5) * 32;
+constexpr int kMaxHalfCols = 128;                 // coefficients per epilogue thread (K <= 256)
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;
 
 struct SmemLayout {
-    uint32_t basis, ring, staging, enc, bias, total;
+    uint32_t basis, ring, staging, enc, len8, bias, total;
 };
 
 __host__ __device__ inline SmemLayout smem_layout(int c, int k, int enc_entries)
@@ -36,7 +42,8 @@ __host__ __device__ inline SmemLayout smem_layout(int c, int k, int enc_entries)
     l.ring = (uint32_t)(((size_t)k * c * 2 + 1023) & ~(size_t)1023);
     l.staging = l.ring + kStages * kStageBytes;
     l.enc = l.staging + 2 * kStagingBytes;
-    l.bias = l.enc + (uint32_t)enc_entries * 4;
+    l.len8 = l.enc + (uint32_t)enc_entries * 4;          // code lengths as bytes (per-layer table)
+    l.bias = l.len8 + (enc_entries ? 256u : 0u);
     l.total = l.bias + (uint32_t)k * 4;
     return l;
 }
@@ -46,10 +53,11 @@ __host__ __device__ inline SmemLayout smem_layout(int c, int k, int enc_entries)
 // [0, 2^b - 1] while still a float.  (A float -> int conversion instruction would do the same
 // but issues at a quarter of the rate.)
 constexpr float kMagic = 12582912.0f;
-__device__ __forceinline__ uint32_t quantise(float acc, float inv_step, float bias, float vmax)
+constexpr uint32_t kMagicBits = 0x4B400000u;
+// returns kMagicBits + q
+__device__ __forceinline__ uint32_t quantise_bits(uint32_t acc_bits, float inv_step, float bias, float vmax)
 {
-    const float v = fminf(fmaxf(fmaf(acc, inv_step, bias) + kMagic, kMagic), vmax);
-    return __float_as_uint(v) & 0xffu;
+    return __float_as_uint(fminf(fmaxf(fmaf(__uint_as_float(acc_bits), inv_step, bias) + kMagic, kMagic), vmax));
 }
 
 // Bit writer into the shared-memory staging buffer.  A word is stored (plain, predicated
@@ -112,10 +120,10 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
     // ---- set-up ---------------------------------------------------------------------
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&s_full[s]), 128); mbar_init(smem_u32(&s_empty[s]), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&s_tfull[b]), 1); mbar_init(smem_u32(&s_tempty[b]), 128); }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&s_tfull[b]), 1); mbar_init(smem_u32(&s_tempty[b]), 256); }
         mbar_fence_init();
     }
-    if (warp == 12) { tmem_alloc(smem_u32(&s_tmem_base), kTmemCols); tmem_relinquish(); }
+    if (warp == kMmaWarp) { tmem_alloc(smem_u32(&s_tmem_base), kTmemCols); tmem_relinquish(); }
     // basis -> K-major core-matrix layout: element (j, ch) at (j/8)*sbo + (ch/8)*128 + (j%8)*16 + (ch%8)*2
     {
         const uint32_t sbo = (uint32_t)(a.c / 8) * 128u;
@@ -127,7 +135,7 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
         }
         for (int i = tid; i < a.k; i += kThreads) s_bias[i] = a.enc_bias[i];
         if (enc_in_smem)
-            for (int i = tid; i < nsym; i += kThreads) s_enc[i] = a.enc[i];
+            for (int i = tid; i < nsym; i += kThreads) { s_enc[i] = a.enc[i]; (smem + L.len8)[i] = (unsigned char)(a.enc[i] & 0xffu); }
     }
     fence_proxy_async_smem();
     tc_fence_before_sync();
@@ -137,9 +145,9 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
 
     const long long my_tiles = (a.n_tiles > blockIdx.x) ? (a.n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
 
-    if (warp >= 8 && warp < 12) {
+    if (warp >= kLoaderWarp0 && warp < kMmaWarp) {
         // ================= loaders =================
-        const int lw = warp - 8, kk = lane & 7;
+        const int lw = warp - kLoaderWarp0, kk = lane & 7;
         const __nv_bfloat16 *xin = reinterpret_cast<const __nv_bfloat16 *>(a.x);
         int it = 0;
         bool alive = true;
@@ -185,7 +193,7 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
             cp_async_wait<0>();
             tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
         }
-    } else if (warp == 12) {
+    } else if (warp == kMmaWarp) {
         // ================= MMA issuer =================
         if (lane == 0) {
             const uint32_t idesc = make_idesc_bf16(TC_TILE_PIXELS, a.k, /*A MN-major*/ true, /*B K-major*/ false);
@@ -216,27 +224,27 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
         }
     } else {
         // ================= epilogue groups =================
-        const int grp = warp >> 2;                 // 0 or 1
-        const int t = tid & 127;                   // pixel within the tile = TMEM lane
-        const int wq = warp & 3;
-        const uint32_t stg_addr = smem_u32(smem + L.staging + grp * kStagingBytes);
+        const int grp = warp >> 3;                 // 0 or 1
+        const int wg = warp & 7;
+        const int half = wg >> 2;                  // which half of the coefficients
+        const int wq = wg & 3;                     // TMEM lane quarter
+        const int m = wq * 32 + lane;              // pixel within the tile = TMEM lane
+        const int tg = (tid & 255);                // thread within the group
+        const int half_cols = ((a.k + 31) / 32) * 16;              // columns of half 0 (multiple of 16)
+        const int col0 = half * half_cols;
+        const int ncols = half ? a.k - half_cols : half_cols;      // multiple of 16, may be 0
+        unsigned char *stg = smem + L.staging + grp * kStagingBytes;
+        const uint32_t stg_addr = smem_u32(stg);
         const uint32_t enc_addr = smem_u32(s_enc);
+        const uint32_t len8_rel = smem_u32(smem + L.len8) - kMagicBits;   // + (kMagicBits + q) = address of len8[q]
+        uint32_t *xch = reinterpret_cast<uint32_t *>(stg);          // [2][128] lengths exchanged between the halves
         const float inv_step = (float)(1.0 / a.step);
         const float vmax = kMagic + (float)(nsym - 1);
         const int bar_id = 1 + grp;
         bool alive = true;
 
-        // code table entry of symbol q of coefficient j: (code << 8) | length
-        auto lookup = [&](int j, uint32_t q) -> uint32_t {
-            if constexpr (kPerChannel) return __ldg(a.enc + j * nsym + q);
-            else {
-                uint32_t e;
-                asm("ld.shared.u32 %0, [%1];" : "=r"(e) : "r"(enc_addr + q * 4u));
-                return e;
-            }
-        };
         auto resolve_base = [&](long long tile, unsigned long long padded) {
-            if (wq == 0) {
+            if (wg == 0) {
                 bool ok;
                 const unsigned long long base = lookback_resolve(a.tile_state, tile, padded, a.status, ok);
                 if (lane == 0) {
@@ -250,91 +258,115 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
 
         for (long long tl = grp; tl < my_tiles && alive; tl += 2) {
             const long long tile = blockIdx.x + tl * gridDim.x;
-            const long long p = tile * TC_TILE_PIXELS + t;
+            const long long p = tile * TC_TILE_PIXELS + m;
             const bool valid = p < a.pixels;
             if (!mbar_wait(smem_u32(&s_tfull[grp]), (uint32_t)((tl >> 1) & 1))) { alive = false; break; }
             tc_fence_after_sync();
-            const uint32_t trow = tmem_base + grp * kAccCols + ((uint32_t)(wq * 32) << 16);
+            const uint32_t trow = tmem_base + grp * kAccCols + ((uint32_t)(wq * 32) << 16) + col0;
 
-            // pass 1: code lengths
+            // pass 1: quantise, keep the symbols (one byte each) in registers, add up code lengths
+            uint32_t sym[kMaxHalfCols / 4];
             unsigned int my_bits = 0;
-            for (int c0 = 0; c0 < a.k; c0 += 32) {
-                if (a.k - c0 >= 32) {
-                    uint32_t r[32];
-                    tmem_ld_32x32b_x32(trow + c0, r);
+#pragma unroll
+            for (int blk = 0; blk < kMaxHalfCols / 16; ++blk) {
+                if (blk * 16 < ncols) {
+                    uint32_t r[16];
+                    tmem_ld_32x32b_x16(trow + blk * 16, r);
                     tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        my_bits += lookup(c0 + i, quantise(__uint_as_float(r[i]), inv_step, s_bias[c0 + i], vmax)) & 0xffu;
-                } else {
-                    uint32_t r16[16];
-                    tmem_ld_32x32b_x16(trow + c0, r16);
-                    tmem_ld_wait();
+                    for (int i = 0; i < 16; ++i) {
+                        const int j = col0 + blk * 16 + i;
+                        const uint32_t vb = quantise_bits(r[i], inv_step, s_bias[j], vmax);
+                        if constexpr (kPerChannel) my_bits += __ldg(a.enc + j * nsym + (vb & 0xffu)) & 0xffu;
+                        else {
+                            uint32_t l;
+                            asm("ld.shared.u8 %0, [%1];" : "=r"(l) : "r"(vb + len8_rel));
+                            my_bits += l;
+                        }
+                        if constexpr (kDebug) {
+                            if (valid && a.dbg_coef) a.dbg_coef[p * a.k + j] = __uint_as_float(r[i]) - a.tmu32[j];
+                            if (valid && a.dbg_sym) a.dbg_sym[p * a.k + j] = (uint8_t)(vb & 0xffu);
+                        }
+                        r[i] = vb;
+                    }
 #pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        my_bits += lookup(c0 + i, quantise(__uint_as_float(r16[i]), inv_step, s_bias[c0 + i], vmax)) & 0xffu;
+                    for (int i = 0; i < 16; i += 4)      // low bytes of four values -> one register
+                        sym[blk * 4 + i / 4] = __byte_perm(__byte_perm(r[i], r[i + 1], 0x0040), __byte_perm(r[i + 2], r[i + 3], 0x0040), 0x5410);
                 }
             }
+            // the accumulator buffer is free for the tile after next
+            tc_fence_before_sync();
+            mbar_arrive(smem_u32(&s_tempty[grp]));
             if (!valid) my_bits = 0;
-            unsigned int tile_bits;
-            const unsigned int my_off = group_exclusive_scan_128(my_bits, s_warp_sums[grp], t, bar_id, tile_bits);
+
+            // bit offsets: pixel-major, first half before second half
+            xch[half * 128 + m] = my_bits;
+            named_bar_sync(bar_id, 256);
+            const unsigned int other = xch[(half ^ 1) * 128 + m];
+            const unsigned int pair = my_bits + other;
+            unsigned int inc = pair;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const unsigned int up = __shfl_up_sync(0xffffffffu, inc, d);
+                if (lane >= d) inc += up;
+            }
+            if (lane == 31 && half == 0) s_warp_sums[grp][wq] = inc;
+            named_bar_sync(bar_id, 256);
+            unsigned int before = 0, tile_bits = 0;
+#pragma unroll
+            for (int w = 0; w < 4; ++w) {
+                const unsigned int sw = s_warp_sums[grp][w];
+                if (w < wq) before += sw;
+                tile_bits += sw;
+            }
+            const unsigned int pixel_off = before + inc - pair;
+            const unsigned int my_off = pixel_off + (half ? other : 0u);
             const unsigned long long padded = ((unsigned long long)tile_bits + 127ull) & ~127ull;
-            if (t == 0) lookback_publish(a.tile_state, tile, padded);
+            if (tg == 0) lookback_publish(a.tile_state, tile, padded);
             const bool staged = padded <= (unsigned long long)kStagingBytes * 8ull;
+            named_bar_sync(bar_id, 256);              // the exchange area is staging again from here on
 
             if (staged) {
                 // every word below tile_bits / 32 is stored by the writer of its last bit; the last
                 // partial word and the padding up to the 128-bit boundary start as zero
                 const unsigned int first_open = tile_bits >> 5, end_word = (unsigned int)(padded >> 5);
-                if (t < end_word - first_open)
-                    asm volatile("st.shared.u32 [%0], %1;" ::"r"(stg_addr + (first_open + t) * 4u), "r"(0u) : "memory");
+                if ((unsigned int)tg < end_word - first_open)
+                    asm volatile("st.shared.u32 [%0], %1;" ::"r"(stg_addr + (first_open + tg) * 4u), "r"(0u) : "memory");
             } else {
                 // rare: the tile does not fit the staging buffer -> resolve its position first and
                 // pack straight into (zeroed) global memory
                 resolve_base(tile, padded);
-                named_bar_sync(bar_id, 128);
+                named_bar_sync(bar_id, 256);
                 if (s_write_ok[grp]) {
                     uint4 *z = reinterpret_cast<uint4 *>(a.stream + (s_base[grp] >> 5));
-                    for (unsigned int i = t; i < (unsigned int)(padded >> 7); i += 128) z[i] = make_uint4(0u, 0u, 0u, 0u);
+                    for (unsigned int i = tg; i < (unsigned int)(padded >> 7); i += 256) z[i] = make_uint4(0u, 0u, 0u, 0u);
                 }
             }
-            named_bar_sync(bar_id, 128);
+            named_bar_sync(bar_id, 256);
 
-            // pass 2: quantise again, look up codes, pack (two symbols are joined in registers and
-            // appended as one piece of at most 24 bits)
+            // pass 2: look up the codes of the kept symbols and pack; two symbols are joined in
+            // registers and appended as one piece of at most 24 bits
             const bool do_pack = valid && (staged || s_write_ok[grp]);
             auto pack_tile = [&](auto &w) {
-                for (int c0 = 0; c0 < a.k; c0 += 32) {
-                    uint32_t r[32];
-                    const bool full = a.k - c0 >= 32;
-                    if (full) tmem_ld_32x32b_x32(trow + c0, r);
-                    else {
-                        uint32_t r16[16];
-                        tmem_ld_32x32b_x16(trow + c0, r16);
+                if (!do_pack) return;
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) r[i] = r16[i];
-                    }
-                    tmem_ld_wait();
-                    if (do_pack) {
+                for (int blk = 0; blk < kMaxHalfCols / 16; ++blk) {
+                    if (blk * 16 < ncols) {
 #pragma unroll
-                        for (int i = 0; i < 32; i += 2) {
-                            if (i < 16 || full) {
-                                const uint32_t q0 = quantise(__uint_as_float(r[i]), inv_step, s_bias[c0 + i], vmax);
-                                const uint32_t q1 = quantise(__uint_as_float(r[i + 1]), inv_step, s_bias[c0 + i + 1], vmax);
-                                const uint32_t e0 = lookup(c0 + i, q0), e1 = lookup(c0 + i + 1, q1);
-                                const uint32_t l1 = e1 & 0xffu;
-                                w.put(((e0 >> 8) << l1) | (e1 >> 8), (int)((e0 & 0xffu) + l1));
-                                if constexpr (kDebug) {
-                                    if (a.dbg_coef) {
-                                        a.dbg_coef[p * a.k + c0 + i] = __uint_as_float(r[i]) - a.tmu32[c0 + i];
-                                        a.dbg_coef[p * a.k + c0 + i + 1] = __uint_as_float(r[i + 1]) - a.tmu32[c0 + i + 1];
-                                    }
-                                    if (a.dbg_sym) {
-                                        a.dbg_sym[p * a.k + c0 + i] = (uint8_t)q0;
-                                        a.dbg_sym[p * a.k + c0 + i + 1] = (uint8_t)q1;
-                                    }
-                                }
+                        for (int i = 0; i < 16; i += 2) {
+                            const uint32_t word = sym[blk * 4 + i / 4];
+                            const uint32_t q0 = (word >> (8 * (i & 3))) & 0xffu, q1 = (word >> (8 * ((i + 1) & 3))) & 0xffu;
+                            uint32_t e0, e1;
+                            if constexpr (kPerChannel) {
+                                const int j = col0 + blk * 16 + i;
+                                e0 = __ldg(a.enc + j * nsym + q0);
+                                e1 = __ldg(a.enc + (j + 1) * nsym + q1);
+                            } else {
+                                asm("ld.shared.u32 %0, [%1];" : "=r"(e0) : "r"(enc_addr + q0 * 4u));
+                                asm("ld.shared.u32 %0, [%1];" : "=r"(e1) : "r"(enc_addr + q1 * 4u));
                             }
+                            const uint32_t l1 = e1 & 0xffu;
+                            w.put(((e0 >> 8) << l1) | (e1 >> 8), (int)((e0 & 0xffu) + l1));
                         }
                     }
                 }
@@ -343,46 +375,40 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
                 SmemBitWriter ws;
                 ws.init(stg_addr, my_off);
                 pack_tile(ws);
-                named_bar_sync(bar_id, 128);      // all full words stored
+                named_bar_sync(bar_id, 256);      // all full words stored
                 if (do_pack) ws.finish();
-            } else {
-                BitWriter wg;
-                wg.init(a.stream, s_base[grp] + my_off);
-                pack_tile(wg);
-                if (do_pack) wg.finish();
-            }
-            // the accumulator buffer is free for the tile after next
-            tc_fence_before_sync();
-            mbar_arrive(smem_u32(&s_tempty[grp]));
-
-            if (staged) {
                 resolve_base(tile, padded);
-                named_bar_sync(bar_id, 128);      // staging complete, base known
+                named_bar_sync(bar_id, 256);      // staging complete, base known
                 if (s_write_ok[grp]) {
                     uint4 *dst = reinterpret_cast<uint4 *>(a.stream + (s_base[grp] >> 5));
-                    for (unsigned int i = t; i < (unsigned int)(padded >> 7); i += 128) {
+                    for (unsigned int i = tg; i < (unsigned int)(padded >> 7); i += 256) {
                         uint4 v;
                         asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
                                      : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(stg_addr + i * 16u));
                         dst[i] = v;
                     }
                 }
+            } else {
+                BitWriter wgl;
+                wgl.init(a.stream, s_base[grp] + my_off);
+                pack_tile(wgl);
+                if (do_pack) wgl.finish();
             }
             const unsigned long long base = s_base[grp];
-            if (t == 0) {
+            if (tg == 0) {
                 a.tile_off[tile] = base;
                 if (tile == a.n_tiles - 1) a.tile_off[a.n_tiles] = base + padded;
             }
-            if (valid && (p % a.chunk_pixels) == 0) a.chunk_off[p / a.chunk_pixels] = my_off;
-            named_bar_sync(bar_id, 128);          // staging and s_base may be reused
+            if (valid && half == 0 && (p % a.chunk_pixels) == 0) a.chunk_off[p / a.chunk_pixels] = pixel_off;
+            named_bar_sync(bar_id, 256);          // staging and s_base may be reused
         }
-        if (!alive && t == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
+        if (!alive && tg == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
     }
 
     // ---- teardown ---------------------------------------------------------------------
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 12) {
+    if (warp == kMmaWarp) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, kTmemCols);
     }
