@@ -9,6 +9,9 @@
 //                      round to bf16, NCHW stores
 //   warps 16, 17       one thread each issues the tcgen05.mma of its group:
 //                      D[pixel][c] = (Q[pixel][j] - center) * T[j][c]
+// Each VLD group copies the bit-stream segment of its next tile into shared memory (cp.async,
+// double-buffered) while it decodes the current one, so that the decoder's refills are
+// shared-memory reads; a segment too long for the buffer is read from global memory instead.
 // The transposed basis (bf16, C x K, K-major) stays resident in shared memory; dequantisation
 // is folded into the epilogue so that the MMA consumes integers exactly: the symbols minus the
 // symbol `center` whose level is nearest to y = 0 (most coefficients sit there, so the
@@ -22,16 +25,21 @@ namespace {
 using namespace tcdev;
 using namespace sm100;
 
-constexpr int kPanelK = 64;                                   // coefficients per ring stage
-constexpr int kStageBytes = kPanelK * TC_TILE_PIXELS * 2;     // 16 KB
+constexpr int kPanelK = 32;                                   // coefficients per ring stage
+constexpr int kStageBytes = kPanelK * TC_TILE_PIXELS * 2;     // 8 KB
 constexpr int kThreads = 18 * 32;
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;
-constexpr int kMaxStages = 4;                                 // per group
+constexpr int kMaxStages = 8;                                 // per group
+// A chunk that starts inside a staged segment is read for at most chunk_pixels * K codes of 12
+// bits, whatever the bits say; the slack after each buffer keeps those reads inside the block's
+// shared memory even for a corrupt stream.  Chunks longer than the slack allows are not staged.
+constexpr int kStreamSlack = 1024;
 
 struct SmemLayout {
-    uint32_t basis, ring, lut, bias, total;
+    uint32_t basis, ring, lut, bias, sbuf, total;
     int stages;                                               // ring stages per group
+    uint32_t stream_buf;                                      // bytes per staged stream buffer (4 buffers), 0 = none
 };
 
 __host__ __device__ inline SmemLayout smem_layout(int c, int k, int lut_entries, int chunk_pixels, int budget)
@@ -48,7 +56,11 @@ __host__ __device__ inline SmemLayout smem_layout(int c, int k, int lut_entries,
     int want = chunk_pixels > 1 ? n_panels : 2;
     if (want < 2) want = 2;
     l.stages = want;
-    l.total = l.ring + 2u * (uint32_t)want * kStageBytes;
+    l.sbuf = l.ring + 2u * (uint32_t)want * kStageBytes;
+    l.stream_buf = 0;
+    for (uint32_t kb = 12; kb >= 4; kb -= 4)
+        if ((long long)l.sbuf + 4ll * (kb * 1024 + kStreamSlack) <= (long long)budget) { l.stream_buf = kb * 1024; break; }
+    l.total = l.sbuf + (l.stream_buf ? 4u * (l.stream_buf + kStreamSlack) : 0u);
     if ((int)l.total > budget || want > kMaxStages) l.stages = 0;
     return l;
 }
@@ -99,6 +111,64 @@ struct WindowReader {
     }
 };
 
+// The same reader over a segment staged in shared memory.  The word after the window is kept
+// in a register, so that the shared-memory load of a refill is off the critical path, and the
+// refill is predicated rather than branched.
+struct SmemWindowReader {
+    uint32_t next_addr;               // shared address of the word after `ahead`
+    uint32_t hi, lo, ahead;
+    int avail;
+
+    __device__ __forceinline__ static uint32_t lds(uint32_t addr)
+    {
+        uint32_t v;
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+        return v;
+    }
+    // `bitpos` is relative to the start of the staged segment at shared address `seg_addr`
+    __device__ __forceinline__ void init(uint32_t seg_addr, uint32_t bitpos)
+    {
+        const uint32_t a0 = seg_addr + (bitpos >> 5) * 4u;
+        const uint32_t w0 = lds(a0), w1 = lds(a0 + 4);
+        ahead = lds(a0 + 8);
+        next_addr = a0 + 12;
+        const int sh = (int)(bitpos & 31u);
+        hi = __funnelshift_l(w1, w0, sh);
+        lo = w1 << sh;
+        avail = 64 - sh;
+    }
+    __device__ __forceinline__ uint32_t peek(int nbits) const { return hi >> (32 - nbits); }
+    // the shift takes its amount modulo 32: a table entry with the length in its low 5 bits
+    // can be passed as it is
+    __device__ __forceinline__ void skip_entry(uint32_t e)
+    {
+        hi = __funnelshift_l(lo, hi, e);
+        lo = __funnelshift_l(0u, lo, e);
+        avail -= (int)(e & 31u);
+    }
+    __device__ __forceinline__ void refill()
+    {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b32 s, t;\n\t"
+            "setp.le.s32 p, %3, 32;\n\t"
+            "sub.s32 s, 32, %3;\n\t"
+            "shf.l.wrap.b32 t, %2, 0, s;\n\t"
+            "@p or.b32 %0, %0, t;\n\t"
+            "shl.b32 t, %2, s;\n\t"
+            "@p or.b32 %1, %1, t;\n\t"
+            "@p add.s32 %3, %3, 32;\n\t"
+            "@p ld.shared.u32 %2, [%4];\n\t"
+            "@p add.s32 %4, %4, 4;\n\t}"
+            : "+r"(hi), "+r"(lo), "+r"(ahead), "+r"(avail), "+r"(next_addr));
+    }
+    // bits consumed since init(seg_addr, bitpos)
+    __device__ __forceinline__ uint32_t consumed(uint32_t seg_addr, uint32_t bitpos) const
+    {
+        const uint32_t a0 = seg_addr + (bitpos >> 5) * 4u;
+        return (next_addr - 4u - a0) * 8u - (bitpos & 31u) - (uint32_t)avail;
+    }
+};
+
 template <bool kPerChannel>
 __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
 {
@@ -108,7 +178,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int lut_size = 1 << a.lut_bits;
-    const SmemLayout L = smem_layout(a.c, a.k, kPerChannel ? 0 : lut_size, a.chunk_pixels, 1 << 30);
+    const SmemLayout L = smem_layout(a.c, a.k, kPerChannel ? 0 : lut_size, a.chunk_pixels, a.smem_budget);
     const int stages = L.stages;
     unsigned char *s_basis = smem + L.basis;
     uint32_t *s_lut = reinterpret_cast<uint32_t *>(smem + L.lut);
@@ -161,67 +231,132 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
         const int cp = a.chunk_pixels;
         const int chunks_per_tile = TC_TILE_PIXELS / cp;
         const uint32_t ring_g = ring_addr + (uint32_t)grp * stages * kStageBytes;
+        const uint32_t sbuf_bytes = L.stream_buf;
+        const uint32_t sbuf_g = smem_u32(smem + L.sbuf) + (uint32_t)grp * 2u * (sbuf_bytes + kStreamSlack);
+        const int bar_id = 1 + grp;
         long long it = 0;                       // panels produced by this group so far
         bool alive = true;
-        for (long long tl = grp; tl < my_tiles && alive; tl += 2) {
+
+        // offsets of a tile, validated; a tile that cannot be valid decodes nothing
+        struct TileInfo { unsigned long long base, bits; bool ok, staged; unsigned int chunk_off; };
+        auto tile_info = [&](long long tl) {
+            TileInfo ti{0, 0, false, false, 0};
+            if (tl >= my_tiles) return ti;
             const long long tile = blockIdx.x + tl * gridDim.x;
             const unsigned long long base = a.tile_off[tile], end = a.tile_off[tile + 1];
-            const bool tile_ok = (base & 127ull) == 0 && (end & 127ull) == 0 && base <= end && end <= a.stream_bits;
+            ti.ok = (base & 127ull) == 0 && (end & 127ull) == 0 && base <= end && end <= a.stream_bits;
+            if (!ti.ok) return ti;
+            ti.base = base;
+            ti.bits = end - base;
+            ti.staged = sbuf_bytes != 0 && ti.bits <= (unsigned long long)sbuf_bytes * 8ull &&
+                        (cp * a.k * TC_MAX_CODE_LEN) / 8 + 16 <= kStreamSlack;
             const long long ch = tile * chunks_per_tile + t;
-            bool active = tile_ok && t < chunks_per_tile && ch < a.n_chunks;
-            bool bad = !tile_ok;
-            WindowReader r;
-            unsigned long long used = 0;
-            if (active) {
-                const unsigned long long off = a.chunk_off[ch];
-                if (base + off > end) { bad = true; active = false; }
-                else { r.init(a.stream, base + off, end); used = base + off; }
+            if (t < chunks_per_tile && ch < a.n_chunks) ti.chunk_off = a.chunk_off[ch];
+            return ti;
+        };
+        // start the copy of a tile's segment into stream buffer `which` (16 bytes per cp.async)
+        auto stage_tile = [&](const TileInfo &ti, int which) {
+            if (ti.ok && ti.staged) {
+                const uint32_t dst = sbuf_g + (uint32_t)which * (sbuf_bytes + kStreamSlack);
+                const unsigned char *src = reinterpret_cast<const unsigned char *>(a.stream) + (ti.base >> 3);
+                const uint32_t n16 = (uint32_t)(ti.bits >> 7);
+                for (uint32_t i = t; i < n16; i += 128) cp_async_16(dst + i * 16u, src + (size_t)i * 16u, 16u);
             }
+            cp_async_commit();
+        };
+
+        TileInfo cur = tile_info(grp), nxt = tile_info(grp + 2);
+        stage_tile(cur, 0);
+        int li = 0;
+        for (long long tl = grp; tl < my_tiles && alive; tl += 2, ++li) {
+            const long long tile = blockIdx.x + tl * gridDim.x;
+            stage_tile(nxt, (li + 1) & 1);           // its buffer was released by the barrier that ended tile li - 1
+            cp_async_wait<1>();
+            named_bar_sync(bar_id, 128);             // every thread's part of this tile's segment has landed
+            const TileInfo after = tile_info(tl + 4); // offsets two tiles ahead: their latency hides behind the decode
+
+            const long long ch = tile * chunks_per_tile + t;
+            bool active = cur.ok && t < chunks_per_tile && ch < a.n_chunks;
+            bool bad = !cur.ok;
+            if (active && (unsigned long long)cur.chunk_off > cur.bits) { bad = true; active = false; }
             const int n_pix = active ? (int)min((long long)cp, a.pixels - (tile * TC_TILE_PIXELS + (long long)t * cp)) : 0;
-            for (int pp = 0; pp < cp && alive; ++pp) {
-                const bool decode = pp < n_pix;
-                const int row = t * cp + pp;       // only meaningful while t < chunks_per_tile
-                for (int kp = 0; kp < n_panels; ++kp) {
-                    const long long pit = it + kp;
-                    const int s = (int)(pit % stages);
-                    if (pp == 0 && !mbar_wait(smem_u32(&s_empty[grp][s]), (uint32_t)(((pit / stages) & 1) ^ 1))) { alive = false; break; }
-                    if (decode) {
-                        const int k0 = kp * kPanelK;
-                        const int nk8 = min(kPanelK, a.k - k0) >> 3;
-                        const uint32_t dst = ring_g + s * kStageBytes + (row >> 3) * 128 + (row & 7) * 16;
-                        for (int k8 = 0; k8 < nk8; ++k8) {
-                            uint32_t pk[4];
+            const uint32_t seg_addr = sbuf_g + (uint32_t)(li & 1) * (sbuf_bytes + kStreamSlack);
+
+            // decodes this thread's chunk with the given reader; `next8` returns eight table entries
+            auto decode_chunk = [&](auto &&next_pair) {
+                for (int pp = 0; pp < cp && alive; ++pp) {
+                    const bool decode = pp < n_pix;
+                    const int row = t * cp + pp;       // only meaningful while t < chunks_per_tile
+                    for (int kp = 0; kp < n_panels; ++kp) {
+                        const long long pit = it + kp;
+                        const int s = (int)(pit % stages);
+                        if (pp == 0 && !mbar_wait(smem_u32(&s_empty[grp][s]), (uint32_t)(((pit / stages) & 1) ^ 1))) { alive = false; break; }
+                        if (decode) {
+                            const int k0 = kp * kPanelK;
+                            const int nk8 = min(kPanelK, a.k - k0) >> 3;
+                            const uint32_t dst = ring_g + s * kStageBytes + (row >> 3) * 128 + (row & 7) * 16;
+                            for (int k8 = 0; k8 < nk8; ++k8) {
+                                uint32_t pk[4];
 #pragma unroll
-                            for (int i = 0; i < 8; i += 2) {
-                                r.refill();
-                                uint32_t e0, e1;
-                                if constexpr (kPerChannel) e0 = __ldg(a.lut32 + (size_t)(k0 + k8 * 8 + i) * lut_size + r.peek(a.lut_bits));
-                                else asm("ld.shared.u32 %0, [%1];" : "=r"(e0) : "r"(lut_addr + r.peek(a.lut_bits) * 4u));
-                                r.skip((int)(e0 & 0xffu));
-                                if constexpr (kPerChannel) e1 = __ldg(a.lut32 + (size_t)(k0 + k8 * 8 + i + 1) * lut_size + r.peek(a.lut_bits));
-                                else asm("ld.shared.u32 %0, [%1];" : "=r"(e1) : "r"(lut_addr + r.peek(a.lut_bits) * 4u));
-                                r.skip((int)(e1 & 0xffu));
-                                used += (e0 & 0xffu) + (e1 & 0xffu);
-                                if constexpr (kPerChannel) {   // tables in global memory hold the plain symbol
-                                    e0 = __float_as_uint((float)((int)((e0 >> 8) & 0xffu) - a.center));
-                                    e1 = __float_as_uint((float)((int)((e1 >> 8) & 0xffu) - a.center));
-                                }
-                                pk[i >> 1] = __byte_perm(e0, e1, 0x7632);     // bf16(sym0) | bf16(sym1) << 16
+                                for (int i = 0; i < 8; i += 2) pk[i >> 1] = next_pair(k0 + k8 * 8 + i);
+                                asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + k8 * 2048), "r"(pk[0]),
+                                             "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
                             }
-                            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + k8 * 2048), "r"(pk[0]),
-                                         "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
+                        }
+                        if (pp == cp - 1) {
+                            fence_proxy_async_smem();
+                            mbar_arrive(smem_u32(&s_full[grp][s]));
                         }
                     }
-                    if (pp == cp - 1) {
-                        fence_proxy_async_smem();
-                        mbar_arrive(smem_u32(&s_full[grp][s]));
-                    }
                 }
+            };
+            // table entry: bf16(symbol - center) << 16 | symbol << 8 | length; returns two bf16 values
+            auto centre = [&](uint32_t e) { return __float_as_uint((float)((int)((e >> 8) & 0xffu) - a.center)); };
+
+            if (cur.ok && cur.staged) {
+                SmemWindowReader r;
+                if (active) r.init(seg_addr, cur.chunk_off);
+                else { r.hi = r.lo = r.ahead = 0; r.avail = 64; r.next_addr = seg_addr; }
+                decode_chunk([&](int j) -> uint32_t {
+                    r.refill();
+                    uint32_t e0, e1;
+                    if constexpr (kPerChannel) e0 = __ldg(a.lut32 + (size_t)j * lut_size + r.peek(a.lut_bits));
+                    else asm("ld.shared.u32 %0, [%1];" : "=r"(e0) : "r"(lut_addr + r.peek(a.lut_bits) * 4u));
+                    r.skip_entry(e0);
+                    if constexpr (kPerChannel) e1 = __ldg(a.lut32 + (size_t)(j + 1) * lut_size + r.peek(a.lut_bits));
+                    else asm("ld.shared.u32 %0, [%1];" : "=r"(e1) : "r"(lut_addr + r.peek(a.lut_bits) * 4u));
+                    r.skip_entry(e1);
+                    if constexpr (kPerChannel) { e0 = centre(e0); e1 = centre(e1); }
+                    return __byte_perm(e0, e1, 0x7632);
+                });
+                if (active && (unsigned long long)cur.chunk_off + r.consumed(seg_addr, cur.chunk_off) > cur.bits) bad = true;
+            } else {
+                WindowReader r;
+                unsigned long long used = cur.base + cur.chunk_off;
+                if (active) r.init(a.stream, used, cur.base + cur.bits);
+                else { r.words = a.stream; r.next = r.end = 0; r.hi = r.lo = 0; r.avail = 64; }
+                decode_chunk([&](int j) -> uint32_t {
+                    r.refill();
+                    uint32_t e0, e1;
+                    if constexpr (kPerChannel) e0 = __ldg(a.lut32 + (size_t)j * lut_size + r.peek(a.lut_bits));
+                    else asm("ld.shared.u32 %0, [%1];" : "=r"(e0) : "r"(lut_addr + r.peek(a.lut_bits) * 4u));
+                    r.skip((int)(e0 & 0xffu));
+                    if constexpr (kPerChannel) e1 = __ldg(a.lut32 + (size_t)(j + 1) * lut_size + r.peek(a.lut_bits));
+                    else asm("ld.shared.u32 %0, [%1];" : "=r"(e1) : "r"(lut_addr + r.peek(a.lut_bits) * 4u));
+                    r.skip((int)(e1 & 0xffu));
+                    used += (e0 & 0xffu) + (e1 & 0xffu);
+                    if constexpr (kPerChannel) { e0 = centre(e0); e1 = centre(e1); }
+                    return __byte_perm(e0, e1, 0x7632);
+                });
+                if (active && used > cur.base + cur.bits) bad = true;
             }
             it += n_panels;
-            if (active && used > end) bad = true;
             if (bad) tc_dev_set_status(a.status, TC_ERR_CORRUPT_STREAM);
+            named_bar_sync(bar_id, 128);             // this tile's stream buffer may be refilled
+            cur = nxt;
+            nxt = after;
         }
+        cp_async_wait<0>();
         if (!alive && t == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
     } else if (warp < 16) {
         // ================= epilogue groups =================
@@ -328,9 +463,11 @@ tc_status tc_launch_decode_tc(const tc_ctx *ctx, const DecodeArgs &a, cudaStream
                                      ctx->max_smem_optin - 512);
     if (l.stages == 0) return TC_ERR_UNSUPPORTED;
     void (*kernel)(DecodeArgs) = a.groups != 1 ? decode_tc_kernel<true> : decode_tc_kernel<false>;
+    DecodeArgs args = a;
+    args.smem_budget = ctx->max_smem_optin - 512;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.total) != cudaSuccess)
         return TC_ERR_CUDA;
     const unsigned int grid = (unsigned int)((a.n_tiles < ctx->sm_count) ? a.n_tiles : ctx->sm_count);
-    kernel<<<grid, kThreads, l.total, s>>>(a);
+    kernel<<<grid, kThreads, l.total, s>>>(args);
     return cudaGetLastError() == cudaSuccess ? TC_OK : TC_ERR_CUDA;
 }

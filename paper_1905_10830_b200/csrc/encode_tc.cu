@@ -11,6 +11,9 @@
 // The basis T (bf16, K x C) stays resident in shared memory; the X tile streams through a ring
 // of 64-channel panels; the fp32 accumulators are double-buffered in tensor memory so that the
 // epilogue of one tile overlaps the loads and MMAs of the next.
+#include <cstdio>
+#include <cstdlib>
+
 #include "device_utils.cuh"
 #include "sm100_ptx.cuh"
 
@@ -43,7 +46,7 @@ __host__ __device__ inline SmemLayout smem_layout(int c, int k, int enc_entries)
     l.staging = l.ring + kStages * kStageBytes;
     l.enc = l.staging + 2 * kStagingBytes;
     l.len8 = l.enc + (uint32_t)enc_entries * 4;          // code lengths as bytes (per-layer table)
-    l.bias = l.len8 + (enc_entries ? 256u : 0u);
+    l.bias = (l.len8 + (enc_entries ? 256u : 0u) + 15u) & ~15u;
     l.total = l.bias + (uint32_t)k * 4;
     return l;
 }
@@ -78,15 +81,22 @@ struct SmemBitWriter {
     }
     __device__ __forceinline__ void put(uint32_t code, int len)
     {
-        hi = __funnelshift_l(lo, hi, len);
-        lo = (lo << len) | code;
-        pending += len;
-        const uint32_t flush = pending >= 32 ? 1u : 0u;
-        const uint32_t out = __funnelshift_r(lo, hi, pending - 32);
-        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.shared.u32 [%0], %1;\n\t}"
-                     ::"r"(addr), "r"(out), "r"(flush));
-        addr += flush * 4u;
-        pending -= (int)(flush * 32u);
+        // hi:lo <<= len; lo |= code; pending += len; if (pending >= 32) { store bits
+        // [pending-32, pending) of hi:lo; addr += 4; pending -= 32; }  (the funnel shift takes
+        // its amount modulo 32, so `pending` itself serves as pending - 32)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b32 t, o;\n\t"
+            "shf.l.wrap.b32 %1, %0, %1, %5;\n\t"
+            "shl.b32 t, %0, %5;\n\t"
+            "or.b32 %0, t, %4;\n\t"
+            "add.s32 %2, %2, %5;\n\t"
+            "setp.ge.s32 p, %2, 32;\n\t"
+            "shf.r.wrap.b32 o, %0, %1, %2;\n\t"
+            "@p st.shared.u32 [%3], o;\n\t"
+            "@p add.s32 %3, %3, 4;\n\t"
+            "@p add.s32 %2, %2, -32;\n\t}"
+            : "+r"(lo), "+r"(hi), "+r"(pending), "+r"(addr)
+            : "r"(code), "r"(len));
     }
     // call after a barrier that follows every writer's puts
     __device__ __forceinline__ void finish()
@@ -272,11 +282,15 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
                 if (blk * 16 < ncols) {
                     uint32_t r[16];
                     tmem_ld_32x32b_x16(trow + blk * 16, r);
+                    float4 bias4[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) bias4[i] = *reinterpret_cast<const float4 *>(s_bias + col0 + blk * 16 + 4 * i);
+                    const float *biasv = reinterpret_cast<const float *>(bias4);
                     tmem_ld_wait();
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
                         const int j = col0 + blk * 16 + i;
-                        const uint32_t vb = quantise_bits(r[i], inv_step, s_bias[j], vmax);
+                        const uint32_t vb = quantise_bits(r[i], inv_step, biasv[i], vmax);
                         if constexpr (kPerChannel) my_bits += __ldg(a.enc + j * nsym + (vb & 0xffu)) & 0xffu;
                         else {
                             uint32_t l;
@@ -437,7 +451,9 @@ tc_status tc_launch_encode_tc(const tc_ctx *ctx, const EncodeArgs &a, cudaStream
     EncodeArgs args = a;
     void *params[] = {&args};
     // cooperative launch: the grid must be co-resident, which is what makes the look-back safe
-    if (cudaLaunchCooperativeKernel((void *)kernel, dim3(grid), dim3(kThreads), params, l.total, s) != cudaSuccess) {
+    const cudaError_t err = cudaLaunchCooperativeKernel((void *)kernel, dim3(grid), dim3(kThreads), params, l.total, s);
+    if (err != cudaSuccess) {
+        if (getenv("TC_VERBOSE")) fprintf(stderr, "tc: encode launch failed: %s\n", cudaGetErrorString(err));
         cudaGetLastError();
         return TC_ERR_CUDA;
     }
