@@ -5,8 +5,8 @@
 //   warps 0-3, 4-7     two VLD groups (alternating tiles): one thread per chunk walks its part
 //                      of the bit stream with a table-driven canonical Huffman decoder and
 //                      writes the symbols, as exact bf16 integers, into the K-major A operand
-//   warps 8-11, 12-15  two epilogue groups: TMEM -> registers, x_hat = step * acc + bias,
-//                      round to bf16, NCHW stores
+//   warps 8-15         epilogue, all eight warps on every tile (two channel halves):
+//                      TMEM -> registers, x_hat = step * acc + bias, round to bf16, NCHW stores
 //   warps 16, 17       one thread each issues the tcgen05.mma of its group:
 //                      D[pixel][c] = (Q[pixel][j] - center) * T[j][c]
 // Each VLD group copies the bit-stream segment of its next tile into shared memory (cp.async,
@@ -193,7 +193,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
         for (int g = 0; g < 2; ++g) {
             for (int s = 0; s < kMaxStages; ++s) { mbar_init(smem_u32(&s_full[g][s]), 128); mbar_init(smem_u32(&s_empty[g][s]), 1); }
             mbar_init(smem_u32(&s_tfull[g]), 1);
-            mbar_init(smem_u32(&s_tempty[g]), 128);
+            mbar_init(smem_u32(&s_tempty[g]), 256);
         }
         mbar_fence_init();
     }
@@ -359,50 +359,47 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
         cp_async_wait<0>();
         if (!alive && t == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
     } else if (warp < 16) {
-        // ================= epilogue groups =================
-        const int grp = (warp - 8) >> 2;
-        const int t = tid & 127;
+        // ================= epilogue: all eight warps work on every tile =================
+        // warps 8-11 store the first half of the channels, warps 12-15 the second half, so that an
+        // accumulator is released after half the store time and the VLD group behind it stalls less
+        const int half = (warp - 8) >> 2;
         const int wq = warp & 3;
+        const int m = wq * 32 + lane;                       // pixel within the tile = TMEM lane
+        const int half_cols = ((a.c + 31) / 32) * 16;
+        const int col0 = half * half_cols;
+        const int ncols = half ? a.c - half_cols : half_cols;   // multiple of 16
         const float step = (float)a.step;
         __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(a.xhat);
         bool alive = true;
-        for (long long tl = grp; tl < my_tiles && alive; tl += 2) {
+        for (long long tl = 0; tl < my_tiles && alive; ++tl) {
+            const int grp = (int)(tl & 1);
             const long long tile = blockIdx.x + tl * gridDim.x;
-            const long long p = tile * TC_TILE_PIXELS + t;
+            const long long p = tile * TC_TILE_PIXELS + m;
             const bool valid = p < a.pixels;
             const long long img = valid ? p / a.hw : 0;
-            __nv_bfloat16 *dst = out + img * a.c * (long long)a.hw + (valid ? p - img * a.hw : 0);
+            __nv_bfloat16 *dst = out + img * a.c * (long long)a.hw + (valid ? p - img * a.hw : 0) + (long long)col0 * a.hw;
             if (!mbar_wait(smem_u32(&s_tfull[grp]), (uint32_t)((tl >> 1) & 1))) { alive = false; break; }
             tc_fence_after_sync();
-            const uint32_t trow = tmem_base + grp * kAccCols + ((uint32_t)(wq * 32) << 16);
-            for (int c0 = 0; c0 < a.c; c0 += 32) {
-                uint32_t r[32];
-                const bool full = a.c - c0 >= 32;
-                if (full) tmem_ld_32x32b_x32(trow + c0, r);
-                else {
-                    uint32_t r16[16];
-                    tmem_ld_32x32b_x16(trow + c0, r16);
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) r[i] = r16[i];
-                }
+            const uint32_t trow = tmem_base + grp * kAccCols + ((uint32_t)(wq * 32) << 16) + col0;
+            for (int c0 = 0; c0 < ncols; c0 += 16) {
+                uint32_t r[16];
+                tmem_ld_32x32b_x16(trow + c0, r);
                 tmem_ld_wait();
                 if (valid) {
 #pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        if (i < 16 || full) {
-                            const float v0 = fmaf(__uint_as_float(r[i]), step, s_bias[c0 + i]);
-                            const float v1 = fmaf(__uint_as_float(r[i + 1]), step, s_bias[c0 + i + 1]);
-                            const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
-                            dst[(long long)(c0 + i) * a.hw] = h.x;
-                            dst[(long long)(c0 + i + 1) * a.hw] = h.y;
-                        }
+                    for (int i = 0; i < 16; i += 2) {
+                        const float v0 = fmaf(__uint_as_float(r[i]), step, s_bias[col0 + c0 + i]);
+                        const float v1 = fmaf(__uint_as_float(r[i + 1]), step, s_bias[col0 + c0 + i + 1]);
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
+                        dst[(long long)(c0 + i) * a.hw] = h.x;
+                        dst[(long long)(c0 + i + 1) * a.hw] = h.y;
                     }
                 }
             }
             tc_fence_before_sync();
             mbar_arrive(smem_u32(&s_tempty[grp]));
         }
-        if (!alive && t == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
+        if (!alive && lane == 0 && wq == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
     } else {
         // ================= MMA issuers (one per group) =================
         const int grp = warp - 16;
