@@ -31,13 +31,15 @@ constexpr int kThreads = 18 * 32;
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;
 constexpr int kMaxStages = 8;                                 // per group
+constexpr int kTransposeBytes = 32 * TC_TILE_PIXELS * 2;      // 32 channels x 128 pixels of bf16
 // A chunk that starts inside a staged segment is read for at most chunk_pixels * K codes of 12
 // bits, whatever the bits say; the slack after each buffer keeps those reads inside the block's
-// shared memory even for a corrupt stream.  Chunks longer than the slack allows are not staged.
+// shared memory even for a corrupt stream (the buffers lie back to back, the slack follows the
+// last one).  Chunks longer than the slack allows are not staged.
 constexpr int kStreamSlack = 1024;
 
 struct SmemLayout {
-    uint32_t basis, ring, lut, bias, sbuf, total;
+    uint32_t basis, ring, lut, bias, sbuf, tbuf, total;
     int stages;                                               // ring stages per group
     uint32_t stream_buf;                                      // bytes per staged stream buffer (4 buffers), 0 = none
 };
@@ -56,11 +58,13 @@ __host__ __device__ inline SmemLayout smem_layout(int c, int k, int lut_entries,
     int want = chunk_pixels > 1 ? n_panels : 2;
     if (want < 2) want = 2;
     l.stages = want;
-    l.sbuf = l.ring + 2u * (uint32_t)want * kStageBytes;
+    l.tbuf = l.ring + 2u * (uint32_t)want * kStageBytes;          // two 8 KB transpose buffers (epilogue)
+    l.sbuf = l.tbuf + 2u * kTransposeBytes;
     l.stream_buf = 0;
-    for (uint32_t kb = 12; kb >= 4; kb -= 4)
-        if ((long long)l.sbuf + 4ll * (kb * 1024 + kStreamSlack) <= (long long)budget) { l.stream_buf = kb * 1024; break; }
-    l.total = l.sbuf + (l.stream_buf ? 4u * (l.stream_buf + kStreamSlack) : 0u);
+    // four stream buffers back to back (an overrun of one lands in the next), one slack area at the end
+    for (uint32_t kb = 12; kb >= 3; --kb)
+        if ((long long)l.sbuf + 4ll * kb * 1024 + kStreamSlack <= (long long)budget) { l.stream_buf = kb * 1024; break; }
+    l.total = l.sbuf + (l.stream_buf ? 4u * l.stream_buf + kStreamSlack : 0u);
     if ((int)l.total > budget || want > kMaxStages) l.stages = 0;
     return l;
 }
@@ -145,6 +149,13 @@ struct SmemWindowReader {
         hi = __funnelshift_l(lo, hi, e);
         lo = __funnelshift_l(0u, lo, e);
         avail -= (int)(e & 31u);
+    }
+    // nbits < 32
+    __device__ __forceinline__ void skip_bits(int nbits)
+    {
+        hi = __funnelshift_l(lo, hi, nbits);
+        lo <<= nbits;
+        avail -= nbits;
     }
     __device__ __forceinline__ void refill()
     {
@@ -232,7 +243,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
         const int chunks_per_tile = TC_TILE_PIXELS / cp;
         const uint32_t ring_g = ring_addr + (uint32_t)grp * stages * kStageBytes;
         const uint32_t sbuf_bytes = L.stream_buf;
-        const uint32_t sbuf_g = smem_u32(smem + L.sbuf) + (uint32_t)grp * 2u * (sbuf_bytes + kStreamSlack);
+        const uint32_t sbuf_g = smem_u32(smem + L.sbuf) + (uint32_t)grp * 2u * sbuf_bytes;
         const int bar_id = 1 + grp;
         long long it = 0;                       // panels produced by this group so far
         bool alive = true;
@@ -257,7 +268,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
         // start the copy of a tile's segment into stream buffer `which` (16 bytes per cp.async)
         auto stage_tile = [&](const TileInfo &ti, int which) {
             if (ti.ok && ti.staged) {
-                const uint32_t dst = sbuf_g + (uint32_t)which * (sbuf_bytes + kStreamSlack);
+                const uint32_t dst = sbuf_g + (uint32_t)which * sbuf_bytes;
                 const unsigned char *src = reinterpret_cast<const unsigned char *>(a.stream) + (ti.base >> 3);
                 const uint32_t n16 = (uint32_t)(ti.bits >> 7);
                 for (uint32_t i = t; i < n16; i += 128) cp_async_16(dst + i * 16u, src + (size_t)i * 16u, 16u);
@@ -280,10 +291,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
             bool bad = !cur.ok;
             if (active && (unsigned long long)cur.chunk_off > cur.bits) { bad = true; active = false; }
             const int n_pix = active ? (int)min((long long)cp, a.pixels - (tile * TC_TILE_PIXELS + (long long)t * cp)) : 0;
-            const uint32_t seg_addr = sbuf_g + (uint32_t)(li & 1) * (sbuf_bytes + kStreamSlack);
+            const uint32_t seg_addr = sbuf_g + (uint32_t)(li & 1) * sbuf_bytes;
 
-            // decodes this thread's chunk with the given reader; `next8` returns eight table entries
-            auto decode_chunk = [&](auto &&next_pair) {
+            // walks this thread's chunk; `fill_panel(dst, k0, nk8)` decodes the next 8 * nk8 symbols
+            // (coefficients k0 ...) into the operand row at shared address `dst`
+            auto decode_chunk = [&](auto &&fill_panel) {
                 for (int pp = 0; pp < cp && alive; ++pp) {
                     const bool decode = pp < n_pix;
                     const int row = t * cp + pp;       // only meaningful while t < chunks_per_tile
@@ -295,13 +307,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
                             const int k0 = kp * kPanelK;
                             const int nk8 = min(kPanelK, a.k - k0) >> 3;
                             const uint32_t dst = ring_g + s * kStageBytes + (row >> 3) * 128 + (row & 7) * 16;
-                            for (int k8 = 0; k8 < nk8; ++k8) {
-                                uint32_t pk[4];
-#pragma unroll
-                                for (int i = 0; i < 8; i += 2) pk[i >> 1] = next_pair(k0 + k8 * 8 + i);
-                                asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + k8 * 2048), "r"(pk[0]),
-                                             "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
-                            }
+                            fill_panel(dst, k0, nk8);
                         }
                         if (pp == cp - 1) {
                             fence_proxy_async_smem();
@@ -310,6 +316,18 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
                     }
                 }
             };
+            // symbol by symbol: eight symbols -> one 16-byte store
+            auto by_pairs = [&](auto &&next_pair) {
+                return [&, next_pair](uint32_t dst, int k0, int nk8) mutable {
+                    for (int k8 = 0; k8 < nk8; ++k8) {
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int i = 0; i < 8; i += 2) pk[i >> 1] = next_pair(k0 + k8 * 8 + i);
+                        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + k8 * 2048), "r"(pk[0]),
+                                     "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
+                    }
+                };
+            };
             // table entry: bf16(symbol - center) << 16 | symbol << 8 | length; returns two bf16 values
             auto centre = [&](uint32_t e) { return __float_as_uint((float)((int)((e >> 8) & 0xffu) - a.center)); };
 
@@ -317,7 +335,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
                 SmemWindowReader r;
                 if (active) r.init(seg_addr, cur.chunk_off);
                 else { r.hi = r.lo = r.ahead = 0; r.avail = 64; r.next_addr = seg_addr; }
-                decode_chunk([&](int j) -> uint32_t {
+                auto next_pair = [&](int j) -> uint32_t {
                     r.refill();
                     uint32_t e0, e1;
                     if constexpr (kPerChannel) e0 = __ldg(a.lut32 + (size_t)j * lut_size + r.peek(a.lut_bits));
@@ -328,14 +346,38 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
                     r.skip_entry(e1);
                     if constexpr (kPerChannel) { e0 = centre(e0); e1 = centre(e1); }
                     return __byte_perm(e0, e1, 0x7632);
-                });
+                };
+                if (!kPerChannel && a.run_shift >= 0) {
+                    // The shortest code is all zeros (canonical order), and at low rates it belongs to
+                    // the symbol that nearly every coefficient of the trailing channels takes.  Eight
+                    // such symbols in a row are 8 (or 16) zero bits: one test replaces eight lookups.
+                    const uint32_t fill = a.run_fill;              // bf16(that symbol - center) twice
+                    const int bits8 = 8 << a.run_shift;            // bits of eight shortest codes
+                    decode_chunk([&](uint32_t dst, int k0, int nk8) {
+                        for (int k8 = 0; k8 < nk8; ++k8) {
+                            uint32_t pk[4];
+                            r.refill();
+                            if ((r.hi >> (32 - bits8)) == 0u) {
+                                r.skip_bits(bits8);
+                                pk[0] = pk[1] = pk[2] = pk[3] = fill;
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 8; i += 2) pk[i >> 1] = next_pair(k0 + k8 * 8 + i);
+                            }
+                            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + k8 * 2048), "r"(pk[0]),
+                                         "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
+                        }
+                    });
+                } else {
+                    decode_chunk(by_pairs(next_pair));
+                }
                 if (active && (unsigned long long)cur.chunk_off + r.consumed(seg_addr, cur.chunk_off) > cur.bits) bad = true;
             } else {
                 WindowReader r;
                 unsigned long long used = cur.base + cur.chunk_off;
                 if (active) r.init(a.stream, used, cur.base + cur.bits);
                 else { r.words = a.stream; r.next = r.end = 0; r.hi = r.lo = 0; r.avail = 64; }
-                decode_chunk([&](int j) -> uint32_t {
+                decode_chunk(by_pairs([&](int j) -> uint32_t {
                     r.refill();
                     uint32_t e0, e1;
                     if constexpr (kPerChannel) e0 = __ldg(a.lut32 + (size_t)j * lut_size + r.peek(a.lut_bits));
@@ -347,7 +389,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
                     used += (e0 & 0xffu) + (e1 & 0xffu);
                     if constexpr (kPerChannel) { e0 = centre(e0); e1 = centre(e1); }
                     return __byte_perm(e0, e1, 0x7632);
-                });
+                }));
                 if (active && used > cur.base + cur.bits) bad = true;
             }
             it += n_panels;
@@ -370,6 +412,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
         const int ncols = half ? a.c - half_cols : half_cols;   // multiple of 16
         const float step = (float)a.step;
         __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(a.xhat);
+        // With H*W a multiple of 4 every aligned group of four pixels lies inside one image and is
+        // 8-byte aligned: 32 channels x 128 pixels are transposed through shared memory and leave
+        // as one 256-byte row per warp store.  Otherwise each lane stores its own 2-byte values.
+        const bool vec = (a.hw & 3) == 0;
+        const uint32_t tb_addr = smem_u32(smem + L.tbuf) + (uint32_t)half * kTransposeBytes;
+        const int ebar = 3 + half;
         bool alive = true;
         for (long long tl = 0; tl < my_tiles && alive; ++tl) {
             const int grp = (int)(tl & 1);
@@ -378,21 +426,58 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
             const bool valid = p < a.pixels;
             const long long img = valid ? p / a.hw : 0;
             __nv_bfloat16 *dst = out + img * a.c * (long long)a.hw + (valid ? p - img * a.hw : 0) + (long long)col0 * a.hw;
+            // the four pixels this lane stores in the transposed phase
+            const long long p4 = tile * TC_TILE_PIXELS + 4 * lane;
+            const bool valid4 = p4 < a.pixels;
+            const long long img4 = valid4 ? p4 / a.hw : 0;
+            __nv_bfloat16 *dst4 = out + img4 * a.c * (long long)a.hw + (valid4 ? p4 - img4 * a.hw : 0) + (long long)col0 * a.hw;
             if (!mbar_wait(smem_u32(&s_tfull[grp]), (uint32_t)((tl >> 1) & 1))) { alive = false; break; }
             tc_fence_after_sync();
             const uint32_t trow = tmem_base + grp * kAccCols + ((uint32_t)(wq * 32) << 16) + col0;
-            for (int c0 = 0; c0 < ncols; c0 += 16) {
-                uint32_t r[16];
-                tmem_ld_32x32b_x16(trow + c0, r);
-                tmem_ld_wait();
-                if (valid) {
+            for (int c0 = 0; c0 < ncols; c0 += 32) {
+                const int nc = min(32, ncols - c0);            // 32 or 16
+                uint32_t r[32];
+                {
+                    uint32_t r16[16];
+                    tmem_ld_32x32b_x16(trow + c0, r16);
 #pragma unroll
-                    for (int i = 0; i < 16; i += 2) {
-                        const float v0 = fmaf(__uint_as_float(r[i]), step, s_bias[col0 + c0 + i]);
-                        const float v1 = fmaf(__uint_as_float(r[i + 1]), step, s_bias[col0 + c0 + i + 1]);
-                        const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
-                        dst[(long long)(c0 + i) * a.hw] = h.x;
-                        dst[(long long)(c0 + i + 1) * a.hw] = h.y;
+                    for (int i = 0; i < 16; ++i) r[i] = r16[i];
+                    if (nc == 32) {
+                        tmem_ld_32x32b_x16(trow + c0 + 16, r16);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) r[16 + i] = r16[i];
+                    }
+                }
+                tmem_ld_wait();
+                if (vec) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        if (i < nc) {
+                            const float v0 = fmaf(__uint_as_float(r[i]), step, s_bias[col0 + c0 + i]);
+                            const float v1 = fmaf(__uint_as_float(r[i + 1]), step, s_bias[col0 + c0 + i + 1]);
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
+                            const uint32_t hb = *reinterpret_cast<const uint32_t *>(&h);
+                            asm volatile("st.shared.u16 [%0], %1;" ::"r"(tb_addr + i * 256 + m * 2), "h"((unsigned short)(hb & 0xffffu)) : "memory");
+                            asm volatile("st.shared.u16 [%0], %1;" ::"r"(tb_addr + (i + 1) * 256 + m * 2), "h"((unsigned short)(hb >> 16)) : "memory");
+                        }
+                    }
+                    named_bar_sync(ebar, 128);                 // the block is in shared memory
+                    for (int ch = wq; ch < nc; ch += 4) {      // one channel row of 128 pixels per warp store
+                        uint32_t lo2, hi2;
+                        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(lo2), "=r"(hi2) : "r"(tb_addr + ch * 256 + lane * 8));
+                        if (valid4) *reinterpret_cast<uint2 *>(dst4 + (long long)(c0 + ch) * a.hw) = make_uint2(lo2, hi2);
+                    }
+                    named_bar_sync(ebar, 128);                 // the buffer may be overwritten
+                } else if (valid) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        if (i < nc) {
+                            const float v0 = fmaf(__uint_as_float(r[i]), step, s_bias[col0 + c0 + i]);
+                            const float v1 = fmaf(__uint_as_float(r[i + 1]), step, s_bias[col0 + c0 + i + 1]);
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
+                            dst[(long long)(c0 + i) * a.hw] = h.x;
+                            dst[(long long)(c0 + i + 1) * a.hw] = h.y;
+                        }
                     }
                 }
             }

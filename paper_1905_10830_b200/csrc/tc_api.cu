@@ -124,6 +124,9 @@ tc_status finish_codebook(tc_codebook *cb)
     for (uint8_t l : cb->lengths) mx = std::max<int>(mx, l);
     cb->max_len = mx;
     cb->lut_bits = mx;
+    cb->min_len = 255;
+    for (int v = 0; v < nsym; ++v)
+        if (cb->lengths[v] < cb->min_len) { cb->min_len = cb->lengths[v]; cb->min_len_symbol = v; }
     std::vector<uint32_t> enc((size_t)cb->groups * nsym);
     std::vector<uint16_t> lut((size_t)cb->groups << cb->lut_bits);
     std::vector<uint32_t> lut32((size_t)cb->groups << cb->lut_bits);
@@ -527,6 +530,13 @@ tc_status tc_decode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
     a.basis64 = m->d_basis64; a.mean64 = m->d_mean64; a.lo = m->lo; a.step = m->step;
     a.xhat = x_hat->data; a.status = ctx->d_status;
     a.lut32 = cb->d_lut32; a.basis_t_bf16 = m->d_basis_t_bf16; a.dec_bias = m->d_dec_bias; a.center = m->center;
+    a.run_shift = (cb->groups == 1 && cb->min_len <= 2) ? cb->min_len - 1 : -1;
+    {
+        const __nv_bfloat16 f = __float2bfloat16((float)(cb->min_len_symbol - m->center));
+        unsigned short raw;
+        std::memcpy(&raw, &f, 2);
+        a.run_fill = ((unsigned int)raw << 16) | raw;
+    }
     if (!ctx->force_exact && x_hat->dtype == TC_BF16 && tc_decode_tc_supported(ctx, a)) {
         ctx->last_decode_path = 1;
         return tc_launch_decode_tc(ctx, a, (cudaStream_t)cuda_stream);

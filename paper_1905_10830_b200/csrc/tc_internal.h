@@ -49,6 +49,7 @@ struct tc_model {
 
 struct tc_codebook {
     int bits = 0, groups = 0, max_len = 0, lut_bits = 0;
+    int min_len = 0, min_len_symbol = 0;    // shortest code of table 0 and its (lowest) symbol: the all-zero code
     std::vector<uint8_t> lengths;           // host [groups][2^bits]
     int device = 0;
     uint32_t *d_enc = nullptr;              // [groups][2^bits]  (code << 8) | length
@@ -101,6 +102,8 @@ struct DecodeArgs {
     const float *dec_bias;              // [c]
     int center;                         // subtracted from every symbol before the MMA
     int smem_budget;                    // shared memory the tensor-core kernel may lay out (set by its launcher)
+    int run_shift;                      // per-layer table whose shortest code has 1 or 2 bits: that length - 1; else -1
+    unsigned int run_fill;              // bf16(symbol of the shortest code - center), twice
     const double *basis64;
     const double *mean64;
     double lo, step;
