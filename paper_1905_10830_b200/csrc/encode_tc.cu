@@ -6,6 +6,9 @@
 //                    second half: TMEM -> registers, quantise, code lengths, bit offsets (scan +
 //                    tile look-back), pack, 128-bit stores.  The symbols stay packed in
 //                    registers between the length pass and the packing pass.
+//   warps 21, 22     one store warp per epilogue group: resolves the tile's stream offset by
+//                    look-back and copies the group's staging buffer out, while the group
+//                    already works on its next tile
 //   warps 16-19      loaders: cp.async NCHW -> shared memory in the MMA's MN-major layout
 //   warp 20          one thread issues tcgen05.mma:  D[pixel][coef] = X_tile[pixel][c] * T[coef][c]
 // The basis T (bf16, K x C) stays resident in shared memory; the X tile streams through a ring
@@ -25,17 +28,19 @@ using namespace sm100;
 constexpr int kPanelCh = 64;                      // channels per ring stage
 constexpr int kStages = 4;
 constexpr int kStageBytes = kPanelCh * TC_TILE_PIXELS * 2;   // 16 KB
-constexpr int kLag = 3;                           // cp.async groups kept in flight per loader thread
-constexpr int kStagingBytes = 16384;              // packed-bit staging per epilogue group
+constexpr int kLag = 2;                           // cp.async groups kept in flight per loader thread; the
+                                                  // remaining ring stage absorbs the MMA's latency
+constexpr int kStagingBytes = 15360;              // packed-bit staging per epilogue group (15 KB)
 constexpr int kEpiWarps = 16;                     // 2 groups x (2 column halves x 4 lane quarters)
 constexpr int kLoaderWarp0 = kEpiWarps, kMmaWarp = kEpiWarps + 4;
-constexpr int kThreads = (kEpiWarps + 5) * 32;
+constexpr int kStoreWarp0 = kMmaWarp + 1;         // two store warps follow
+constexpr int kThreads = (kEpiWarps + 7) * 32;
 constexpr int kMaxHalfCols = 128;                 // coefficients per epilogue thread (K <= 256)
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;
 
 struct SmemLayout {
-    uint32_t basis, ring, staging, enc, len8, bias, total;
+    uint32_t basis, ring, staging, enc, len8, bias, xch, total;
 };
 
 __host__ __device__ inline SmemLayout smem_layout(int c, int k, int enc_entries)
@@ -45,9 +50,10 @@ __host__ __device__ inline SmemLayout smem_layout(int c, int k, int enc_entries)
     l.ring = (uint32_t)(((size_t)k * c * 2 + 1023) & ~(size_t)1023);
     l.staging = l.ring + kStages * kStageBytes;
     l.enc = l.staging + 2 * kStagingBytes;
-    l.len8 = l.enc + (uint32_t)enc_entries * 4;          // code lengths as bytes (per-layer table)
+    l.len8 = l.enc + (uint32_t)enc_entries * 8;          // code lengths as bytes (per-layer table)
     l.bias = (l.len8 + (enc_entries ? 256u : 0u) + 15u) & ~15u;
-    l.total = l.bias + (uint32_t)k * 4;
+    l.xch = l.bias + (uint32_t)k * 4;                   // code lengths exchanged between the halves: [2 groups][2][128] u16
+    l.total = l.xch + 2u * 2u * 128u * 2u;
     return l;
 }
 
@@ -115,6 +121,9 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
     __shared__ unsigned int s_warp_sums[2][4];
     __shared__ unsigned long long s_base[2];
     __shared__ int s_write_ok[2];
+    __shared__ __align__(8) unsigned long long s_stg_full[2], s_stg_free[2];   // staging hand-over to the store warp
+    __shared__ unsigned long long s_padded[2];
+    __shared__ int s_store_cmd[2];             // 1: copy the staged tile out, 2: nothing to copy, 3: stop
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nsym = 1 << a.bits;
@@ -130,7 +139,12 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
     // ---- set-up ---------------------------------------------------------------------
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&s_full[s]), 128); mbar_init(smem_u32(&s_empty[s]), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&s_tfull[b]), 1); mbar_init(smem_u32(&s_tempty[b]), 256); }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&s_tfull[b]), 1);
+            mbar_init(smem_u32(&s_tempty[b]), 256);
+            mbar_init(smem_u32(&s_stg_full[b]), 256);
+            mbar_init(smem_u32(&s_stg_free[b]), 1);
+        }
         mbar_fence_init();
     }
     if (warp == kMmaWarp) { tmem_alloc(smem_u32(&s_tmem_base), kTmemCols); tmem_relinquish(); }
@@ -145,7 +159,14 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
         }
         for (int i = tid; i < a.k; i += kThreads) s_bias[i] = a.enc_bias[i];
         if (enc_in_smem)
-            for (int i = tid; i < nsym; i += kThreads) { s_enc[i] = a.enc[i]; (smem + L.len8)[i] = (unsigned char)(a.enc[i] & 0xffu); }
+            for (int i = tid; i < nsym; i += kThreads) {
+                // per-layer table: (1 << length, code) pairs, so that appending a code to a register is
+                // one multiply-add, and the lengths once more as bytes
+                const uint32_t e = a.enc[i];
+                s_enc[2 * i] = 1u << (e & 0xffu);
+                s_enc[2 * i + 1] = e >> 8;
+                (smem + L.len8)[i] = (unsigned char)(e & 0xffu);
+            }
     }
     fence_proxy_async_smem();
     tc_fence_before_sync();
@@ -196,7 +217,6 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
             }
         }
         if (alive) {
-            if (it >= 3) { cp_async_wait<2>(); fence_proxy_async_smem(); mbar_arrive(smem_u32(&s_full[(it - 3) % kStages])); }
             if (it >= 2) { cp_async_wait<1>(); fence_proxy_async_smem(); mbar_arrive(smem_u32(&s_full[(it - 2) % kStages])); }
             if (it >= 1) { cp_async_wait<0>(); fence_proxy_async_smem(); mbar_arrive(smem_u32(&s_full[(it - 1) % kStages])); }
         } else {
@@ -232,6 +252,39 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
             }
             if (!alive) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
         }
+    } else if (warp >= kStoreWarp0) {
+        // ================= store warps =================
+        const int grp = warp - kStoreWarp0;
+        const uint32_t stg_addr = smem_u32(smem + L.staging + grp * kStagingBytes);
+        long long n = 0;
+        for (long long tl = grp; tl < my_tiles; tl += 2, ++n) {
+            const long long tile = blockIdx.x + tl * gridDim.x;
+            if (!mbar_wait(smem_u32(&s_stg_full[grp]), (uint32_t)(n & 1))) { if (lane == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT); break; }
+            const int cmd = s_store_cmd[grp];
+            if (cmd == 3) break;
+            if (cmd == 1) {
+                const unsigned long long padded = s_padded[grp];
+                bool ok;
+                const unsigned long long base = lookback_resolve(a.tile_state, tile, padded, a.status, ok);
+                const bool fits = base + padded <= a.capacity_bits;
+                if (ok && !fits && lane == 0) tc_dev_set_status(a.status, TC_ERR_BUFFER_TOO_SMALL);
+                if (ok && fits) {
+                    uint4 *dst = reinterpret_cast<uint4 *>(a.stream + (base >> 5));
+                    for (unsigned int i = lane; i < (unsigned int)(padded >> 7); i += 32) {
+                        uint4 v;
+                        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                                     : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(stg_addr + i * 16u));
+                        dst[i] = v;
+                    }
+                }
+                if (lane == 0) {
+                    a.tile_off[tile] = base;
+                    if (tile == a.n_tiles - 1) a.tile_off[a.n_tiles] = base + padded;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&s_stg_free[grp]));
+        }
     } else {
         // ================= epilogue groups =================
         const int grp = warp >> 3;                 // 0 or 1
@@ -247,7 +300,8 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
         const uint32_t stg_addr = smem_u32(stg);
         const uint32_t enc_addr = smem_u32(s_enc);
         const uint32_t len8_rel = smem_u32(smem + L.len8) - kMagicBits;   // + (kMagicBits + q) = address of len8[q]
-        uint32_t *xch = reinterpret_cast<uint32_t *>(stg);          // [2][128] lengths exchanged between the halves
+        unsigned short *xch = reinterpret_cast<unsigned short *>(smem + L.xch) + grp * 256;   // [2][128] lengths exchanged between the halves
+        long long n_done = 0;                      // tiles this group has handed to its store warp
         const float inv_step = (float)(1.0 / a.step);
         const float vmax = kMagic + (float)(nsym - 1);
         const int bar_id = 1 + grp;
@@ -276,10 +330,12 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
 
             // pass 1: quantise, keep the symbols (one byte each) in registers, add up code lengths
             uint32_t sym[kMaxHalfCols / 4];
+            uint32_t blk_bits[kMaxHalfCols / 64] = {};          // code bits of each block of 16 symbols, one byte each
             unsigned int my_bits = 0;
 #pragma unroll
             for (int blk = 0; blk < kMaxHalfCols / 16; ++blk) {
                 if (blk * 16 < ncols) {
+                    const unsigned int bits_before = my_bits;
                     uint32_t r[16];
                     tmem_ld_32x32b_x16(trow + blk * 16, r);
                     float4 bias4[4];
@@ -306,6 +362,7 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
 #pragma unroll
                     for (int i = 0; i < 16; i += 4)      // low bytes of four values -> one register
                         sym[blk * 4 + i / 4] = __byte_perm(__byte_perm(r[i], r[i + 1], 0x0040), __byte_perm(r[i + 2], r[i + 3], 0x0040), 0x5410);
+                    blk_bits[blk >> 2] |= (my_bits - bits_before) << (8 * (blk & 3));      // at most 16 * 12 = 192
                 }
             }
             // the accumulator buffer is free for the tile after next
@@ -314,7 +371,7 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
             if (!valid) my_bits = 0;
 
             // bit offsets: pixel-major, first half before second half
-            xch[half * 128 + m] = my_bits;
+            xch[half * 128 + m] = (unsigned short)my_bits;     // at most 128 * 12 bits
             named_bar_sync(bar_id, 256);
             const unsigned int other = xch[(half ^ 1) * 128 + m];
             const unsigned int pair = my_bits + other;
@@ -338,7 +395,8 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
             const unsigned long long padded = ((unsigned long long)tile_bits + 127ull) & ~127ull;
             if (tg == 0) lookback_publish(a.tile_state, tile, padded);
             const bool staged = padded <= (unsigned long long)kStagingBytes * 8ull;
-            named_bar_sync(bar_id, 256);              // the exchange area is staging again from here on
+            // the store warp must be done with the previous tile before staging is written again
+            if (n_done > 0 && !mbar_wait(smem_u32(&s_stg_free[grp]), (uint32_t)((n_done - 1) & 1))) { alive = false; break; }
 
             if (staged) {
                 // every word below tile_bits / 32 is stored by the writer of its last bit; the last
@@ -367,20 +425,36 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
                 for (int blk = 0; blk < kMaxHalfCols / 16; ++blk) {
                     if (blk * 16 < ncols) {
 #pragma unroll
-                        for (int i = 0; i < 16; i += 2) {
-                            const uint32_t word = sym[blk * 4 + i / 4];
-                            const uint32_t q0 = (word >> (8 * (i & 3))) & 0xffu, q1 = (word >> (8 * ((i + 1) & 3))) & 0xffu;
-                            uint32_t e0, e1;
-                            if constexpr (kPerChannel) {
-                                const int j = col0 + blk * 16 + i;
-                                e0 = __ldg(a.enc + j * nsym + q0);
-                                e1 = __ldg(a.enc + (j + 1) * nsym + q1);
-                            } else {
-                                asm("ld.shared.u32 %0, [%1];" : "=r"(e0) : "r"(enc_addr + q0 * 4u));
-                                asm("ld.shared.u32 %0, [%1];" : "=r"(e1) : "r"(enc_addr + q1 * 4u));
+                        const int nbits = (int)((blk_bits[blk >> 2] >> (8 * (blk & 3))) & 0xffu);
+                        if (!kPerChannel && nbits < 32) {
+                            // the whole block fits one register: acc = acc * 2^len + code per symbol
+                            uint32_t acc = 0;
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                const uint32_t q = (sym[blk * 4 + i / 4] >> (8 * (i & 3))) & 0xffu;
+                                uint32_t mul, code;
+                                asm("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(mul), "=r"(code) : "r"(enc_addr + q * 8u));
+                                acc = acc * mul + code;
                             }
-                            const uint32_t l1 = e1 & 0xffu;
-                            w.put(((e0 >> 8) << l1) | (e1 >> 8), (int)((e0 & 0xffu) + l1));
+                            w.put(acc, nbits);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 16; i += 2) {
+                                const uint32_t word = sym[blk * 4 + i / 4];
+                                const uint32_t q0 = (word >> (8 * (i & 3))) & 0xffu, q1 = (word >> (8 * ((i + 1) & 3))) & 0xffu;
+                                uint32_t c0, c1, l0, l1;
+                                if constexpr (kPerChannel) {
+                                    const int j = col0 + blk * 16 + i;
+                                    const uint32_t e0 = __ldg(a.enc + j * nsym + q0), e1 = __ldg(a.enc + (j + 1) * nsym + q1);
+                                    c0 = e0 >> 8; l0 = e0 & 0xffu; c1 = e1 >> 8; l1 = e1 & 0xffu;
+                                } else {
+                                    asm("ld.shared.u32 %0, [%1];" : "=r"(c0) : "r"(enc_addr + q0 * 8u + 4u));
+                                    asm("ld.shared.u32 %0, [%1];" : "=r"(c1) : "r"(enc_addr + q1 * 8u + 4u));
+                                    asm("ld.shared.u8 %0, [%1];" : "=r"(l0) : "r"(len8_rel + kMagicBits + q0));
+                                    asm("ld.shared.u8 %0, [%1];" : "=r"(l1) : "r"(len8_rel + kMagicBits + q1));
+                                }
+                                w.put((c0 << l1) | c1, (int)(l0 + l1));
+                            }
                         }
                     }
                 }
@@ -391,32 +465,28 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
                 pack_tile(ws);
                 named_bar_sync(bar_id, 256);      // all full words stored
                 if (do_pack) ws.finish();
-                resolve_base(tile, padded);
-                named_bar_sync(bar_id, 256);      // staging complete, base known
-                if (s_write_ok[grp]) {
-                    uint4 *dst = reinterpret_cast<uint4 *>(a.stream + (s_base[grp] >> 5));
-                    for (unsigned int i = tg; i < (unsigned int)(padded >> 7); i += 256) {
-                        uint4 v;
-                        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                                     : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(stg_addr + i * 16u));
-                        dst[i] = v;
-                    }
-                }
+                if (tg == 0) { s_padded[grp] = padded; s_store_cmd[grp] = 1; }
             } else {
                 BitWriter wgl;
                 wgl.init(a.stream, s_base[grp] + my_off);
                 pack_tile(wgl);
                 if (do_pack) wgl.finish();
+                if (tg == 0) {
+                    const unsigned long long base = s_base[grp];
+                    a.tile_off[tile] = base;
+                    if (tile == a.n_tiles - 1) a.tile_off[a.n_tiles] = base + padded;
+                    s_store_cmd[grp] = 2;
+                }
             }
-            const unsigned long long base = s_base[grp];
-            if (tg == 0) {
-                a.tile_off[tile] = base;
-                if (tile == a.n_tiles - 1) a.tile_off[a.n_tiles] = base + padded;
-            }
+            // hand the tile to the store warp (each thread's arrival releases its own writes)
+            mbar_arrive(smem_u32(&s_stg_full[grp]));
+            ++n_done;
             if (valid && half == 0 && (p % a.chunk_pixels) == 0) a.chunk_off[p / a.chunk_pixels] = pixel_off;
-            named_bar_sync(bar_id, 256);          // staging and s_base may be reused
         }
-        if (!alive && tg == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
+        if (!alive) {
+            if (tg == 0) { tc_dev_set_status(a.status, TC_ERR_TIMEOUT); s_store_cmd[grp] = 3; }
+            mbar_arrive(smem_u32(&s_stg_full[grp]));   // lets the store warp leave
+        }
     }
 
     // ---- teardown ---------------------------------------------------------------------
