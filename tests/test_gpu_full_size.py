@@ -1,0 +1,111 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times.
+
+The tensors are too large for the bit-serial oracle to code whole, so a few tiles (first, ragged
+last, some in the middle) are checked element by element: the tile's slice of the GPU stream
+must be bit-identical to the oracle's coding of the symbols it holds, those symbols must equal
+the oracle's own quantisation of the same pixels up to the allowed rounding ties, and the
+decoded pixels must match the oracle's reconstruction.  Whole-tensor properties (offsets
+monotone and aligned, total size, round trip through the fp64 kernels on a sample) cover the
+rest."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_1905_10830_b200 as tc
+from synth import featuremaps as fm
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _check_tiles(ctx, model_desc, lengths, bits, x, enc, xhat, tiles):
+    n, c, h, w = x.shape
+    hw = h * w
+    pixels = n * hw
+    cp = enc.layout.chunk_pixels
+    cpt = 128 // cp
+    tile_off = H.tile_off(enc)
+    chunk_off = H.chunk_off(enc)
+    words_all = enc.words[: int(tile_off[-1]) // 8].cpu().numpy().view(np.uint32)
+    m = oracle.Model(c, c, bits, model_desc["mean"], model_desc["basis"], model_desc["eig"],
+                     model_desc["lo"], model_desc["step"], "bf16")
+    total_bad = 0
+    total = 0
+    for t in tiles:
+        p0, p1 = t * 128, min(pixels, (t + 1) * 128)
+        # the tile's slice of the stream, as a stream of its own
+        sub = oracle.Stream(words_all[int(tile_off[t]) // 32: int(tile_off[t + 1]) // 32].copy(),
+                            chunk_off[t * cpt: t * cpt + -(-(p1 - p0) // cp)].copy(),
+                            np.array([0, tile_off[t + 1] - tile_off[t]], dtype=np.uint64),
+                            int(tile_off[t + 1] - tile_off[t]), p1 - p0, c, cp, cpt)
+        q_stream = oracle.decode_symbols(sub, lengths, bits)
+        # entropy coding is bit-exact given the symbols
+        ref = oracle.encode(q_stream, lengths, bits, chunk_pixels=cp, tile_chunks=cpt)
+        assert np.array_equal(ref.words, sub.words)
+        assert np.array_equal(ref.chunk_off, sub.chunk_off)
+        # the symbols are the oracle's, up to +-1 at rounding ties
+        i0, i1 = p0 // hw, (p1 - 1) // hw + 1
+        xs = x[i0:i1].cpu()
+        y = oracle.project(m, xs)[p0 - i0 * hw: p1 - i0 * hw]
+        q, units = oracle.quantize(m, y, with_units=True)
+        bad = q_stream != q
+        if bad.any():
+            assert np.all(np.abs(q_stream[bad].astype(int) - q[bad].astype(int)) == 1)
+            assert np.all(np.abs(units[bad] - np.floor(units[bad]) - 0.5) <= 1e-3)
+        total_bad += int(bad.sum())
+        total += q.size
+        # decode: the reconstruction of what the stream holds
+        img_pixels = np.zeros(((i1 - i0) * hw, c), dtype=np.uint8)
+        img_pixels[p0 - i0 * hw: p1 - i0 * hw] = q_stream
+        want = oracle.reconstruct(m, img_pixels, (i1 - i0, c, h, w), out_bf16=True)
+        want = want.transpose(0, 2, 3, 1).reshape(-1, c)[p0 - i0 * hw: p1 - i0 * hw]
+        got = xhat[i0:i1].float().cpu().numpy().transpose(0, 2, 3, 1).reshape(-1, c)[p0 - i0 * hw: p1 - i0 * hw]
+        ulp = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(want), 1e-30))) - 7)
+        assert np.all(np.abs(got - want) <= np.maximum(1e-3 * np.maximum(np.abs(want), m.step), ulp))
+        assert (got == want).mean() >= 0.999
+    assert total_bad <= max(1, int(1e-4 * total))
+
+
+@pytest.mark.parametrize("cfg,layer,bits", [(5, 0, 4), (5, 0, 8), (3, 0, 4), (4, 0, 5)])
+def test_full_size_layer_sampled_against_oracle(cfg, layer, bits):
+    w = fm.workload(cfg)
+    spec = w.layers[layer]
+    params = fm.layer_params(spec)
+    ctx = tc.tc_create(0)
+    cal = fm.make_maps(params, min(w.calib_maps, 64), calib=True, dtype=w.dtype, device="cuda")
+    model = tc.tc_fit_pca(ctx, cal, bits=bits)
+    st = tc.tc_stats(ctx, model, None, cal)
+    cb = tc.tc_build_codebook(ctx, model, st.hist)
+    x = fm.make_maps(params, w.batch, dtype=w.dtype, device="cuda")
+    enc = tc.tc_encode(ctx, model, cb, x)
+    xhat = tc.tc_decode(ctx, model, cb, enc, x.shape, x.dtype)
+    assert tc.tc_get_status(ctx) == 0
+    assert tc.tc_last_path(ctx, False) == 1 and tc.tc_last_path(ctx, True) == 1
+    # whole-tensor properties
+    toff = H.tile_off(enc).astype(np.int64)
+    assert toff[0] == 0 and np.all(toff % 128 == 0) and np.all(np.diff(toff) > 0)
+    lay = enc.layout
+    assert len(toff) == lay.n_tiles + 1
+    coff = H.chunk_off(enc).astype(np.int64).reshape(lay.n_tiles if lay.n_chunks % lay.n_tiles == 0 else -1, -1) \
+        if lay.n_chunks % lay.n_tiles == 0 else None
+    if coff is not None:
+        assert np.all(coff[:, 0] == 0) and np.all(np.diff(coff, axis=1) > 0)
+        assert np.all(coff[:, -1] < np.diff(toff)[:, None][:, 0])
+    # the fp64 kernels decode the same stream to the same symbols: compare outputs on a slice
+    exact = tc.tc_create(0)
+    tc.tc_force_exact_path(exact, True)
+    n_s = 2
+    enc_s = tc.tc_encode(ctx, model, cb, x[:n_s].contiguous())
+    a = tc.tc_decode(ctx, model, cb, enc_s, x[:n_s].shape, x.dtype)
+    b = tc.tc_decode(exact, model, cb, enc_s, x[:n_s].shape, x.dtype)
+    assert tc.tc_get_status(ctx) == 0 and tc.tc_get_status(exact) == 0
+    assert (a == b).double().mean().item() >= 0.999
+    # sampled tiles against the oracle
+    desc = tc.tc_model_export(model)
+    lengths = tc.tc_codebook_export(cb)
+    rng = np.random.default_rng(cfg * 10 + bits)
+    tiles = sorted(set([0, lay.n_tiles - 1] + rng.integers(0, lay.n_tiles, 4).tolist()))
+    _check_tiles(ctx, desc, lengths, bits, x, enc, xhat, tiles)
+    for hnd in (model, cb, ctx, exact):
+        hnd.close()
