@@ -181,6 +181,7 @@ def main():
         return
 
     import paper_1905_10830_b200 as tc
+    from paper_1905_10830_b200 import sharding
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the codec has no CPU fallback")
     torch.cuda.set_device(local_rank)
@@ -250,10 +251,8 @@ def main():
     dec_ms = [ev[i][1].elapsed_time(ev[i][2]) for i in range(args.steps)]
     if tc.tc_get_status(ctx) != 0:
         raise SystemExit("codec reported an error during the timed region")
-    if dist is not None:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    # whole job: bytes summed over ranks, device time as the max over ranks
+    job_bytes, total_ms = sharding.aggregate(raw_bytes * args.steps, total_ms, dev)
 
     # ---- end to end: host buffers, copies inside the timed region -------------------------
     e2e = None
@@ -281,11 +280,8 @@ def main():
         b.record()
         torch.cuda.synchronize()
         e2e_ms = a.elapsed_time(b)
-        if dist is not None:
-            t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
-        e2e = {"value": raw_bytes * world * e2e_steps / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
+        e2e_bytes, e2e_ms = sharding.aggregate(raw_bytes * e2e_steps, e2e_ms, dev)
+        e2e = {"value": e2e_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
                "h2d_bytes_per_step": raw_bytes, "d2h_bytes_per_step": raw_bytes, "steps": e2e_steps}
         assert torch.equal(hout.to(dev), xhat)
 
@@ -303,7 +299,7 @@ def main():
     values = x.numel()
     line = {
         "metric": METRIC,
-        "value": raw_bytes * world * args.steps / (total_ms * 1e-3) / 1e9,
+        "value": job_bytes / (total_ms * 1e-3) / 1e9,
         "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
