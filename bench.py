@@ -260,14 +260,11 @@ def main():
         hx = torch.empty(x.shape, dtype=x.dtype, pin_memory=True)
         hx.copy_(x)
         hout = torch.empty(x.shape, dtype=x.dtype, pin_memory=True)
-        dx = torch.empty_like(x)
         e2e_steps = max(2, min(args.steps, 5))
 
         def e2e_step():
-            dx.copy_(hx, non_blocking=True)
-            tc.tc_encode(ctx, model, cb, dx, out=enc)
-            tc.tc_decode(ctx, model, cb, enc, x.shape, x.dtype, out=xhat, stream_bytes=stream_bytes)
-            hout.copy_(xhat, non_blocking=True)
+            # one C-ABI call with host buffers: H2D copy, encode, decode, D2H copy
+            tc.tc_roundtrip_host(ctx, model, cb, hx, hout)
 
         e2e_step()
         torch.cuda.synchronize()

@@ -233,6 +233,17 @@ tc_status tc_decode(tc_ctx *ctx, const tc_model *model, const tc_codebook *cb, c
                     size_t stream_bytes, const uint32_t *chunk_off, const uint64_t *tile_off,
                     const tc_encode_params *params, const tc_tensor *x_hat, void *cuda_stream);
 
+/* Whole chain on HOST tensors (Section 3: encoder, memory, decoder): copies `x_host` (dense
+ * NCHW, `dtype`, pinned memory recommended) to the device, encodes, decodes and copies the
+ * reconstruction to `x_hat_host`, all on `cuda_stream`, then synchronises it.  The device
+ * buffers (tensor, reconstruction, worst-case stream, offsets) live in a context-owned arena
+ * that grows with cudaMalloc when a larger tensor arrives.  `stream_bits` (HOST, may be NULL)
+ * receives the length of the coded stream.  Returns the first host- or device-side error. */
+tc_status tc_roundtrip_host(tc_ctx *ctx, const tc_model *model, const tc_codebook *cb,
+                            const void *x_host, void *x_hat_host, int32_t n, int32_t c, int32_t h,
+                            int32_t w, int32_t dtype, const tc_encode_params *params,
+                            uint64_t *stream_bits, void *cuda_stream);
+
 /* ---------------------------------------------------------------------------------------
  * Statistics (Section 3: rate and MSE distortion D = |x - x_hat|^2 / n; Section 3.1: entropy
  * H = -sum p log2 p as the theoretical rate; Appendix G: eigenvalue energy ratio).

@@ -5,6 +5,6 @@ memory and streams only."""
 from .binding import (  # noqa: F401
     TcError, Context, Model, Codebook, EncodedStream, StreamLayout, Stats,
     tc_create, tc_fit_pca, tc_model_import, tc_model_export, tc_build_codebook,
-    tc_codebook_import, tc_codebook_export, tc_encode_bound, tc_encode, tc_encode_noalloc, tc_decode, tc_stats,
+    tc_codebook_import, tc_codebook_export, tc_encode_bound, tc_encode, tc_encode_noalloc, tc_roundtrip_host, tc_decode, tc_stats,
     tc_get_status, tc_force_exact_path, tc_last_path, tc_host_huffman_lengths, tc_host_eigh, library_path, load_library,
 )

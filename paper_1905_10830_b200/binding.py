@@ -66,7 +66,7 @@ class _StatsOut(C.Structure):
 EXPORTS = ["tc_create", "tc_destroy", "tc_status_string", "tc_get_status", "tc_force_exact_path", "tc_last_path", "tc_fit_pca",
            "tc_model_import", "tc_model_export", "tc_model_free", "tc_build_codebook",
            "tc_codebook_import", "tc_codebook_export", "tc_codebook_free",
-           "tc_host_huffman_lengths", "tc_host_eigh", "tc_encode_bound", "tc_encode", "tc_encode_noalloc", "tc_decode",
+           "tc_host_huffman_lengths", "tc_host_eigh", "tc_encode_bound", "tc_encode", "tc_encode_noalloc", "tc_decode", "tc_roundtrip_host",
            "tc_stats"]
 
 _lib = None
@@ -112,6 +112,7 @@ def load_library() -> C.CDLL:
                                   P(_DebugOut), vp]
         lib.tc_encode_noalloc.argtypes = [vp, vp, vp, P(_Tensor), P(_EncodeParams), vp, C.c_size_t, vp, vp, vp]
         lib.tc_decode.argtypes = [vp, vp, vp, vp, C.c_size_t, vp, vp, P(_EncodeParams), P(_Tensor), vp]
+        lib.tc_roundtrip_host.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, P(_EncodeParams), P(C.c_uint64), vp]
         lib.tc_stats.argtypes = [vp, vp, vp, P(_Tensor), P(_StatsOut), vp]
         _lib = lib
     return _lib
@@ -373,6 +374,23 @@ def tc_decode(ctx: Context, model: Model, cb: Codebook, enc: EncodedStream, shap
                                     enc.chunk_off.data_ptr(), enc.tile_off.data_ptr(), C.byref(p), C.byref(t),
                                     _stream_ptr(ctx.device)), "tc_decode")
     return out
+
+
+def tc_roundtrip_host(ctx: Context, model: Model, cb: Codebook, x_host: torch.Tensor, out_host: torch.Tensor, *,
+                      chunk_pixels: int = 0) -> int:
+    """Encode + decode a HOST tensor (dense NCHW, ideally pinned) into `out_host`; returns the
+    coded length in bits.  The copies and both kernels run inside the C call."""
+    if x_host.is_cuda or out_host.is_cuda or not x_host.is_contiguous() or not out_host.is_contiguous():
+        raise ValueError("expected contiguous host tensors")
+    if x_host.shape != out_host.shape or x_host.dtype != out_host.dtype:
+        raise ValueError("input and output must have the same shape and dtype")
+    n, c, h, w = x_host.shape
+    dt = TC_F32 if x_host.dtype == torch.float32 else TC_BF16
+    p = _EncodeParams(chunk_pixels)
+    bits = C.c_uint64(0)
+    _check(load_library().tc_roundtrip_host(ctx.ptr, model.ptr, cb.ptr, x_host.data_ptr(), out_host.data_ptr(), n, c, h, w,
+                                            dt, C.byref(p), C.byref(bits), _stream_ptr(ctx.device)), "tc_roundtrip_host")
+    return bits.value
 
 
 def tc_stats(ctx: Context, model: Model, cb: Codebook | None, x: torch.Tensor, *, groups: int = 1,

@@ -216,6 +216,7 @@ void tc_destroy(tc_ctx *ctx)
     DeviceGuard guard(ctx->device);
     cudaDeviceSynchronize();
     if (ctx->scratch) cudaFree(ctx->scratch);
+    if (ctx->host_arena) cudaFree(ctx->host_arena);
     if (ctx->d_status) cudaFree(ctx->d_status);
     delete ctx;
 }
@@ -543,6 +544,46 @@ tc_status tc_decode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
     }
     ctx->last_decode_path = 0;
     return tc_launch_decode_simt(ctx, a, x_hat->dtype, (cudaStream_t)cuda_stream);
+}
+
+tc_status tc_roundtrip_host(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const void *x_host, void *x_hat_host,
+                            int32_t n, int32_t c, int32_t h, int32_t w, int32_t dtype, const tc_encode_params *params,
+                            uint64_t *stream_bits, void *cuda_stream)
+{
+    if (!ctx || !x_host || !x_hat_host) return TC_ERR_INVALID_ARG;
+    tc_tensor x{nullptr, n, c, h, w, dtype};
+    x.data = (void *)x_host;                      // only for the shape checks of tc_encode_bound
+    tc_stream_layout lay;
+    tc_status st = tc_encode_bound(m, cb, &x, params, &lay);
+    if (st != TC_OK) return st;
+    if (lay.n_tiles == 0) { if (stream_bits) *stream_bits = 0; return TC_OK; }
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const size_t elem = dtype == TC_F32 ? 4 : 2;
+    const size_t bytes = (size_t)n * c * h * w * elem;
+    auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+    const size_t off_xhat = up(bytes), off_stream = off_xhat + up(bytes), off_chunk = off_stream + up(lay.stream_bytes),
+                 off_tile = off_chunk + up(lay.chunk_off_bytes), total = off_tile + up(lay.tile_off_bytes);
+    if (total > ctx->host_arena_bytes) {
+        if (ctx->host_arena) { TC_CUDA(cudaDeviceSynchronize()); cudaFree(ctx->host_arena); ctx->host_arena = nullptr; ctx->host_arena_bytes = 0; }
+        TC_CUDA(cudaMalloc(&ctx->host_arena, total));
+        ctx->host_arena_bytes = total;
+    }
+    char *base = (char *)ctx->host_arena;
+    tc_tensor xd{base, n, c, h, w, dtype}, xh{base + off_xhat, n, c, h, w, dtype};
+    TC_CUDA(cudaMemcpyAsync(xd.data, x_host, bytes, cudaMemcpyHostToDevice, s));
+    st = tc_encode(ctx, m, cb, &xd, params, base + off_stream, lay.stream_bytes, (uint32_t *)(base + off_chunk),
+                   (uint64_t *)(base + off_tile), nullptr, s);
+    if (st != TC_OK) return st;
+    st = tc_decode(ctx, m, cb, base + off_stream, lay.stream_bytes, (const uint32_t *)(base + off_chunk),
+                   (const uint64_t *)(base + off_tile), params, &xh, s);
+    if (st != TC_OK) return st;
+    TC_CUDA(cudaMemcpyAsync(x_hat_host, xh.data, bytes, cudaMemcpyDeviceToHost, s));
+    uint64_t bits = 0;
+    TC_CUDA(cudaMemcpyAsync(&bits, base + off_tile + (size_t)lay.n_tiles * 8, 8, cudaMemcpyDeviceToHost, s));
+    TC_CUDA(cudaStreamSynchronize(s));
+    if (stream_bits) *stream_bits = bits;
+    return tc_get_status(ctx, s);
 }
 
 // ---- statistics ---------------------------------------------------------------------------

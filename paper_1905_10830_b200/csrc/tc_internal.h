@@ -26,6 +26,8 @@ struct tc_ctx {
     unsigned int *d_status = nullptr;     // device status word
     void *scratch = nullptr;              // look-back state, ticket counter
     size_t scratch_bytes = 0;
+    void *host_arena = nullptr;           // device staging of tc_roundtrip_host (grown on demand)
+    size_t host_arena_bytes = 0;
     int force_exact = 0;                  // route every tensor through the fp64 kernels
     int last_encode_path = 0;             // 0 = fp64 kernels, 1 = tensor-core kernels
     int last_decode_path = 0;

@@ -203,3 +203,21 @@ def test_repeated_encodes_are_bit_identical(ctx):
         assert torch.equal(again.words[:n], first.words[:n])
         assert torch.equal(again.tile_off, first.tile_off)
     m.close(); cb.close()
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_roundtrip_host_matches_the_device_path(ctx, dtype):
+    spec = fm.LayerSpec(64, 14, 14, 0.9, None, 508)
+    o = H.oracle_side(spec, 4, 6, 5, dtype, False)
+    m = H.import_model(tc, ctx, o["model"], dtype)
+    cb = tc.tc_codebook_import(ctx, o["lengths"], 4)
+    x = o["x"]
+    host_in = x.clone().pin_memory()
+    host_out = torch.empty_like(host_in).pin_memory()
+    bits = tc.tc_roundtrip_host(ctx, m, cb, host_in, host_out)
+    enc = tc.tc_encode(ctx, m, cb, x.cuda())
+    dev = tc.tc_decode(ctx, m, cb, enc, x.shape, dtype)
+    assert tc.tc_get_status(ctx) == 0
+    assert bits == enc.total_bits()
+    assert torch.equal(host_out, dev.cpu())
+    m.close(); cb.close()
