@@ -189,7 +189,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int lut_size = 1 << a.lut_bits;
-    const SmemLayout L = smem_layout(a.c, a.k, kPerChannel ? 0 : lut_size, a.chunk_pixels, a.smem_budget);
+    constexpr int pair_size = 1 << TC_PAIR_LUT_BITS;
+    const SmemLayout L = smem_layout(a.c, a.k, kPerChannel ? 0 : 2 * pair_size, a.chunk_pixels, a.smem_budget);
     const int stages = L.stages;
     unsigned char *s_basis = smem + L.basis;
     uint32_t *s_lut = reinterpret_cast<uint32_t *>(smem + L.lut);
@@ -220,11 +221,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
         }
         for (int i = tid; i < a.c; i += kThreads) s_bias[i] = a.dec_bias[i];
         if (!kPerChannel)
-            for (int i = tid; i < lut_size; i += kThreads) {
-                // table entry: bf16(symbol - center) << 16 | symbol << 8 | length
-                const uint32_t e = a.lut32[i];
-                const float centred = (float)((int)((e >> 8) & 0xffu) - a.center);
-                s_lut[i] = (__float_as_uint(centred) & 0xffff0000u) | (e & 0xffffu);
+            for (int i = tid; i < pair_size; i += kThreads) {
+                // pair table entry: x = bf16(symbol0 - center) | bf16(symbol1 - center) << 16,
+                //                   y = bits consumed | symbols decoded << 8 | length of the first code << 16
+                const uint2 e = a.lut_pair[i];
+                const float f0 = (float)((int)(e.x & 0xffu) - a.center), f1 = (float)((int)((e.x >> 8) & 0xffu) - a.center);
+                s_lut[2 * i] = (__float_as_uint(f0) >> 16) | (__float_as_uint(f1) & 0xffff0000u);
+                s_lut[2 * i + 1] = e.y;
             }
     }
     fence_proxy_async_smem();
@@ -338,14 +341,36 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
                 auto next_pair = [&](int j) -> uint32_t {
                     r.refill();
                     uint32_t e0, e1;
-                    if constexpr (kPerChannel) e0 = __ldg(a.lut32 + (size_t)j * lut_size + r.peek(a.lut_bits));
-                    else asm("ld.shared.u32 %0, [%1];" : "=r"(e0) : "r"(lut_addr + r.peek(a.lut_bits) * 4u));
-                    r.skip_entry(e0);
-                    if constexpr (kPerChannel) e1 = __ldg(a.lut32 + (size_t)(j + 1) * lut_size + r.peek(a.lut_bits));
-                    else asm("ld.shared.u32 %0, [%1];" : "=r"(e1) : "r"(lut_addr + r.peek(a.lut_bits) * 4u));
-                    r.skip_entry(e1);
-                    if constexpr (kPerChannel) { e0 = centre(e0); e1 = centre(e1); }
-                    return __byte_perm(e0, e1, 0x7632);
+                    if constexpr (!kPerChannel) {
+                        // both symbols from one lookup when their codes fit a 10-bit window
+                        uint32_t v, meta;
+                        asm("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v), "=r"(meta) : "r"(lut_addr + r.peek(TC_PAIR_LUT_BITS) * 8u));
+                        if (((meta >> 8) & 3u) == 2u) {
+                            r.skip_entry(meta);
+                            return v;
+                        }
+                        // one symbol at a time: the first symbol of a pair entry, or, for the rare
+                        // code longer than the window, the full table in global memory
+                        auto one = [&](uint32_t vv, uint32_t mm) -> uint32_t {
+                            if (((mm >> 8) & 3u) != 0u) {
+                                r.skip_entry(mm >> 16);
+                                return vv << 16;                      // bf16 bits in the upper half, as in lut32
+                            }
+                            const uint32_t e = __ldg(a.lut32 + r.peek(a.lut_bits));
+                            r.skip_entry(e);
+                            return centre(e);
+                        };
+                        const uint32_t h0 = one(v, meta);
+                        asm("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v), "=r"(meta) : "r"(lut_addr + r.peek(TC_PAIR_LUT_BITS) * 8u));
+                        const uint32_t h1 = one(v, meta);
+                        return __byte_perm(h0, h1, 0x7632);
+                    } else {
+                        e0 = __ldg(a.lut32 + (size_t)j * lut_size + r.peek(a.lut_bits));
+                        r.skip_entry(e0);
+                        e1 = __ldg(a.lut32 + (size_t)(j + 1) * lut_size + r.peek(a.lut_bits));
+                        r.skip_entry(e1);
+                    }
+                    return __byte_perm(centre(e0), centre(e1), 0x7632);
                 };
                 if (!kPerChannel && a.run_shift >= 0) {
                     // The shortest code is all zeros (canonical order), and at low rates it belongs to
@@ -379,16 +404,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
                 else { r.words = a.stream; r.next = r.end = 0; r.hi = r.lo = 0; r.avail = 64; }
                 decode_chunk(by_pairs([&](int j) -> uint32_t {
                     r.refill();
-                    uint32_t e0, e1;
-                    if constexpr (kPerChannel) e0 = __ldg(a.lut32 + (size_t)j * lut_size + r.peek(a.lut_bits));
-                    else asm("ld.shared.u32 %0, [%1];" : "=r"(e0) : "r"(lut_addr + r.peek(a.lut_bits) * 4u));
+                    const size_t tbl = kPerChannel ? (size_t)j * lut_size : 0, tbl1 = kPerChannel ? (size_t)(j + 1) * lut_size : 0;
+                    const uint32_t e0 = __ldg(a.lut32 + tbl + r.peek(a.lut_bits));
                     r.skip((int)(e0 & 0xffu));
-                    if constexpr (kPerChannel) e1 = __ldg(a.lut32 + (size_t)(j + 1) * lut_size + r.peek(a.lut_bits));
-                    else asm("ld.shared.u32 %0, [%1];" : "=r"(e1) : "r"(lut_addr + r.peek(a.lut_bits) * 4u));
+                    const uint32_t e1 = __ldg(a.lut32 + tbl1 + r.peek(a.lut_bits));
                     r.skip((int)(e1 & 0xffu));
                     used += (e0 & 0xffu) + (e1 & 0xffu);
-                    if constexpr (kPerChannel) { e0 = centre(e0); e1 = centre(e1); }
-                    return __byte_perm(e0, e1, 0x7632);
+                    return __byte_perm(centre(e0), centre(e1), 0x7632);
                 }));
                 if (active && used > cur.base + cur.bits) bad = true;
             }
@@ -533,7 +555,7 @@ bool tc_decode_tc_supported(const tc_ctx *ctx, const DecodeArgs &a)
     if (a.c % 16 != 0 || a.k != a.c || a.c > 256) return false;
     if (a.groups != 1 && a.groups != a.k) return false;
     if (a.lut_bits > TC_MAX_CODE_LEN) return false;
-    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, a.chunk_pixels,
+    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (2 << TC_PAIR_LUT_BITS) : 0, a.chunk_pixels,
                                      ctx->max_smem_optin - 512);
     return l.stages > 0;
 }
@@ -541,7 +563,7 @@ bool tc_decode_tc_supported(const tc_ctx *ctx, const DecodeArgs &a)
 tc_status tc_launch_decode_tc(const tc_ctx *ctx, const DecodeArgs &a, cudaStream_t s)
 {
     if (a.n_tiles <= 0) return TC_OK;
-    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, a.chunk_pixels,
+    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (2 << TC_PAIR_LUT_BITS) : 0, a.chunk_pixels,
                                      ctx->max_smem_optin - 512);
     if (l.stages == 0) return TC_ERR_UNSUPPORTED;
     void (*kernel)(DecodeArgs) = a.groups != 1 ? decode_tc_kernel<true> : decode_tc_kernel<false>;

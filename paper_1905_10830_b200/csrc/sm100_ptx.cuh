@@ -25,29 +25,34 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+// One wait attempt.  The thread may be suspended by the hardware for up to `suspend_ns`
+// nanoseconds and is woken when the phase completes: a waiting warp issues no instructions
+// meanwhile, which matters because the roles of a block share the SM's issue slots.
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity, uint32_t suspend_ns)
 {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(suspend_ns)
         : "memory");
     return ok != 0;
 }
 // Wait for the phase with the given parity; gives up after about two seconds and returns
-// false, so that no kernel can spin forever on a barrier that nothing completes.
+// false, so that no kernel can spin forever on a barrier that nothing completes.  Between
+// attempts the warp sleeps, so that warps that wait do not compete with warps that work.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 {
-    for (int i = 0; i < 4096; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait(bar, parity, 0u)) return true;
     unsigned long long t0, t1;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
     while (true) {
-        for (int i = 0; i < 256; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
+        for (int i = 0; i < 64; ++i) {
+            if (mbar_try_wait(bar, parity, 100000u)) return true;
+            __nanosleep(100);
+        }
         asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
         if (t1 - t0 > 2000000000ull) return false;
     }

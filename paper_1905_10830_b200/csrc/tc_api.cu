@@ -151,6 +151,31 @@ tc_status finish_codebook(tc_codebook *cb)
     tc_status st;
     if ((st = upload(&cb->d_enc, enc)) != TC_OK) return st;
     if ((st = upload(&cb->d_lut32, lut32)) != TC_OK) return st;
+    if (cb->groups == 1) {
+        // Two symbols per lookup: for every 10-bit window, x = symbol0 | symbol1 << 8 and
+        // y = bits consumed | count << 8 | length of the first code << 16, count = 2 if both codes
+        // lie inside the window, 1 if only the first does, 0 if not even the first.
+        const int wb = TC_PAIR_LUT_BITS;
+        auto first_symbol = [&](uint32_t window) -> uint32_t {       // window: wb bits, left-aligned codes
+            const uint32_t idx = cb->lut_bits >= wb ? window << (cb->lut_bits - wb) : window >> (wb - cb->lut_bits);
+            return lut32[idx];
+        };
+        std::vector<uint2> pair((size_t)1 << wb);
+        for (uint32_t win = 0; win < (1u << wb); ++win) {
+            const uint32_t e0 = first_symbol(win);
+            const uint32_t l0 = e0 & 0xffu, s0 = (e0 >> 8) & 0xffu;
+            uint2 v = make_uint2(0u, 0u);
+            if (l0 <= (uint32_t)wb) {
+                const uint32_t rest = (win << l0) & ((1u << wb) - 1u);
+                const uint32_t e1 = first_symbol(rest);
+                const uint32_t l1 = e1 & 0xffu, s1 = (e1 >> 8) & 0xffu;
+                if (l0 + l1 <= (uint32_t)wb) v = make_uint2(s0 | (s1 << 8), (l0 + l1) | (2u << 8) | (l0 << 16));
+                else v = make_uint2(s0, l0 | (1u << 8) | (l0 << 16));
+            }
+            pair[win] = v;
+        }
+        if ((st = upload(&cb->d_lut_pair, pair)) != TC_OK) return st;
+    }
     return upload(&cb->d_lut, lut);
 }
 
@@ -431,6 +456,7 @@ void tc_codebook_free(tc_codebook *cb)
     cudaFree(cb->d_enc);
     cudaFree(cb->d_lut);
     cudaFree(cb->d_lut32);
+    cudaFree(cb->d_lut_pair);
     delete cb;
 }
 
@@ -530,7 +556,7 @@ tc_status tc_decode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
     a.chunk_pixels = cp; a.lut_bits = cb->lut_bits; a.lut = cb->d_lut;
     a.basis64 = m->d_basis64; a.mean64 = m->d_mean64; a.lo = m->lo; a.step = m->step;
     a.xhat = x_hat->data; a.status = ctx->d_status;
-    a.lut32 = cb->d_lut32; a.basis_t_bf16 = m->d_basis_t_bf16; a.dec_bias = m->d_dec_bias; a.center = m->center;
+    a.lut32 = cb->d_lut32; a.lut_pair = cb->d_lut_pair; a.basis_t_bf16 = m->d_basis_t_bf16; a.dec_bias = m->d_dec_bias; a.center = m->center;
     a.run_shift = (cb->groups == 1 && cb->min_len <= 2) ? cb->min_len - 1 : -1;
     {
         const __nv_bfloat16 f = __float2bfloat16((float)(cb->min_len_symbol - m->center));

@@ -12,6 +12,7 @@
 constexpr int TC_TILE_PIXELS = 128;   // pixels per tile = threads per epilogue group
 constexpr int TC_MAX_C = 1024;
 constexpr int TC_MAX_CODE_LEN = 12;   // longest code the decode lookup table covers
+constexpr int TC_PAIR_LUT_BITS = 10;  // window of the two-symbol decode table
 
 // Device status word: first error wins.
 __device__ __forceinline__ void tc_dev_set_status(unsigned int *status, unsigned int code)
@@ -57,6 +58,7 @@ struct tc_codebook {
     uint32_t *d_enc = nullptr;              // [groups][2^bits]  (code << 8) | length
     uint16_t *d_lut = nullptr;              // [groups][2^lut_bits]  (symbol << 8) | length
     uint32_t *d_lut32 = nullptr;            // [groups][2^lut_bits]  bf16(symbol) << 16 | symbol << 8 | length
+    uint2 *d_lut_pair = nullptr;            // per-layer tables: [1024] two symbols per 10-bit window (see tc_api.cu)
 };
 
 // ---- kernel argument blocks -------------------------------------------------------------
@@ -100,6 +102,7 @@ struct DecodeArgs {
     int lut_bits;
     const uint16_t *lut;
     const uint32_t *lut32;              // tensor-core path
+    const uint2 *lut_pair;              // tensor-core path, per-layer tables: two symbols per lookup
     const __nv_bfloat16 *basis_t_bf16;  // [c][k]
     const float *dec_bias;              // [c]
     int center;                         // subtracted from every symbol before the MMA
