@@ -1,0 +1,153 @@
+"""Runs the five workload configurations through the library on one GPU and prints a Markdown
+table: bits/value, encode / decode / round-trip GB/s of raw activations, fraction of the HBM
+roofline, which kernels ran, and parity against the CPU oracle on a sample of each layer.
+
+    python -m paper_1905_10830_b200.report [--cfg 1 2 3 4 5] [--reps 5] [--out FILE]
+
+The oracle (test infrastructure) is imported only for the parity columns; with --no-oracle the
+table has the throughput columns alone."""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import paper_1905_10830_b200 as tc
+from synth import featuremaps as fm
+
+
+def _peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        return float(json.load(open(path))["hbm_gbs"])
+    return 6650.0
+
+
+def _time(fn, reps):
+    fn()
+    torch.cuda.synchronize()
+    best = 1e30
+    for _ in range(reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        torch.cuda.synchronize()
+        best = min(best, a.elapsed_time(b))
+    return best
+
+
+def _parity(ctx, model, cb, x_sample, bits, per_channel):
+    import oracle
+    d = tc.tc_model_export(model)
+    dtype = x_sample.dtype
+    m = oracle.Model(d["c"], d["k"], bits, d["mean"], d["basis"], d["eig"], d["lo"], d["step"],
+                     "bf16" if dtype == torch.bfloat16 else "f32")
+    lengths = tc.tc_codebook_export(cb)
+    enc = tc.tc_encode(ctx, model, cb, x_sample, debug=True)
+    xhat = tc.tc_decode(ctx, model, cb, enc, x_sample.shape, dtype)
+    assert tc.tc_get_status(ctx) == 0
+    q_gpu = enc.symbols.cpu().numpy()
+    y = oracle.project(m, x_sample.cpu())
+    q, units = oracle.quantize(m, y, with_units=True)
+    y_gpu = enc.coefficients.cpu().numpy().astype(np.float64)
+    coef_err = float(np.max(np.abs(y_gpu - y) / np.maximum(np.abs(y), m.step)))
+    bad = q_gpu != q
+    ties_only = bool(np.all(np.abs(units[bad] - np.floor(units[bad]) - 0.5) <= 1e-3)) if bad.any() else True
+    cp = enc.layout.chunk_pixels
+    ref = oracle.encode(q_gpu, lengths, bits, chunk_pixels=cp, tile_chunks=128 // cp)
+    words = enc.words[: enc.total_bits() // 8].cpu().numpy().view(np.uint32)
+    stream_exact = bool(np.array_equal(words, ref.words))
+    want = oracle.reconstruct(m, q_gpu, x_sample.shape, out_bf16=(dtype == torch.bfloat16))
+    got = xhat.float().cpu().numpy()
+    return dict(stream_exact=stream_exact, coef_err=coef_err, mismatch=float(bad.mean()), ties_only=ties_only,
+                xhat_equal=float((got == want).mean()))
+
+
+def run(cfgs, reps, with_oracle, max_batch):
+    peak = _peak()
+    ctx = tc.tc_create(0)
+    rows = []
+    for cfg in cfgs:
+        w = fm.workload(cfg)
+        for spec, repeat in zip(w.layers, w.repeats):
+            params = fm.layer_params(spec)
+            batch = min(w.batch, max_batch)
+            cal = fm.make_maps(params, w.calib_maps, calib=True, dtype=w.dtype, device="cuda")
+            x = fm.make_maps(params, batch, dtype=w.dtype, device="cuda")
+            values = x.numel()
+            raw = values * x.element_size()
+            groups = spec.c if w.per_channel_codebook else 1
+            for bits in w.bits:
+                model = tc.tc_fit_pca(ctx, cal, bits=bits)
+                st = tc.tc_stats(ctx, model, None, cal, groups=groups)
+                cb = tc.tc_build_codebook(ctx, model, st.hist, groups=groups)
+                enc = tc.tc_encode(ctx, model, cb, x)
+                xhat = torch.empty_like(x)
+                nbytes = enc.total_bits() // 8
+                t_enc = _time(lambda: tc.tc_encode(ctx, model, cb, x, out=enc), reps)
+                t_dec = _time(lambda: tc.tc_decode(ctx, model, cb, enc, x.shape, x.dtype, out=xhat, stream_bytes=nbytes), reps)
+                assert tc.tc_get_status(ctx) == 0
+                side = enc.layout.chunk_off_bytes + enc.layout.tile_off_bytes
+                algo = raw + nbytes + side
+                tst = tc.tc_stats(ctx, model, cb, x[: min(batch, 64)], groups=groups, want_hist=False)
+                row = dict(cfg=cfg, layer=spec.name + (f" x{repeat}" if repeat > 1 else ""), batch=batch, dtype=str(w.dtype).split(".")[-1],
+                           b=bits, entropy=tst.entropy, huffman=tst.mean_length, stream=8 * nbytes / values,
+                           total=8 * (nbytes + side) / values, mse=tst.mse,
+                           enc_gbs=raw / t_enc / 1e6, dec_gbs=raw / t_dec / 1e6, rt_gbs=raw / (t_enc + t_dec) / 1e6,
+                           enc_ms=t_enc, dec_ms=t_dec, enc_frac=algo / t_enc / 1e6 / peak, dec_frac=algo / t_dec / 1e6 / peak,
+                           enc_frac8=algo / t_enc / 1e6 / 8000, dec_frac8=algo / t_dec / 1e6 / 8000,
+                           kernels=("tcgen05" if tc.tc_last_path(ctx, False) else "fp64") + "/" + ("tcgen05" if tc.tc_last_path(ctx, True) else "fp64"))
+                if with_oracle:
+                    row.update(_parity(ctx, model, cb, x[: max(1, min(batch, 2))].contiguous(), bits, w.per_channel_codebook))
+                rows.append(row)
+                model.close()
+                cb.close()
+            del x, cal
+            torch.cuda.empty_cache()
+    return rows, peak
+
+
+def to_markdown(rows, peak, with_oracle):
+    head = ["cfg", "layer", "N", "dtype", "b", "entropy", "Huffman", "stream+pad", "+offsets", "MSE", "enc ms", "dec ms", "enc GB/s", "dec GB/s",
+            "round trip GB/s", f"HBM frac enc/dec (of {peak:.0f} GB/s measured)", "(of 8000 GB/s)", "kernels enc/dec"]
+    if with_oracle:
+        head += ["stream bit-exact", "coef max rel err", "symbol mismatch", "only at ties", "x_hat bit-equal"]
+    out = ["| " + " | ".join(head) + " |", "|" + "---|" * len(head)]
+    for r in rows:
+        cells = [r["cfg"], r["layer"], r["batch"], r["dtype"], r["b"], f"{r['entropy']:.3f}", f"{r['huffman']:.3f}", f"{r['stream']:.3f}",
+                 f"{r['total']:.3f}", f"{r['mse']:.3g}", f"{r['enc_ms']:.3f}", f"{r['dec_ms']:.3f}", f"{r['enc_gbs']:.1f}", f"{r['dec_gbs']:.1f}",
+                 f"{r['rt_gbs']:.1f}", f"{r['enc_frac']:.3f} / {r['dec_frac']:.3f}", f"{r['enc_frac8']:.3f} / {r['dec_frac8']:.3f}", r["kernels"]]
+        if with_oracle:
+            cells += ["yes" if r["stream_exact"] else "NO", f"{r['coef_err']:.1e}", f"{r['mismatch']:.1e}", "yes" if r["ties_only"] else "NO",
+                      f"{r['xhat_equal']:.5f}"]
+        out.append("| " + " | ".join(str(c) for c in cells) + " |")
+    return "\n".join(out)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--cfg", type=int, nargs="*", default=[1, 2, 3, 4, 5])
+    ap.add_argument("--reps", type=int, default=5)
+    ap.add_argument("--max-batch", type=int, default=1 << 30)
+    ap.add_argument("--no-oracle", action="store_true")
+    ap.add_argument("--out", default="")
+    args = ap.parse_args()
+    rows, peak = run(args.cfg, args.reps, not args.no_oracle, args.max_batch)
+    md = to_markdown(rows, peak, not args.no_oracle)
+    print(md)
+    if args.out:
+        with open(args.out, "w") as f:
+            f.write(md + "\n")
+
+
+if __name__ == "__main__":
+    main()
