@@ -49,8 +49,8 @@ def lib() -> C.CDLL:
             "orc_huffman_lengths": (i32, [vp, i32, i32, vp]),
             "orc_huffman_lengths_raw": (i32, [vp, i32, i32, i32, vp]),
             "orc_canonical_codes": (None, [vp, i32, vp]),
-            "orc_encode": (i64, [vp, i64, i32, i32, i32, vp, i32, i32, vp, i64, vp, vp]),
-            "orc_decode_symbols": (i32, [vp, i64, vp, vp, i64, i32, i32, i32, vp, i32, i32, vp]),
+            "orc_encode": (i64, [vp, i64, i32, i32, i32, vp, i64, i64, vp, i64, vp, vp]),
+            "orc_decode_symbols": (i32, [vp, i64, vp, vp, i64, i32, i32, i32, vp, i64, i64, vp]),
             "orc_reconstruct": (None, [vp, i64, i32, i64, i32, vp, vp, d, d, i32, vp]),
             "orc_entropy": (d, [vp, i32]),
             "orc_mean_length": (d, [vp, vp, i32]),
@@ -92,13 +92,27 @@ class Model:
 @dataclass
 class Stream:
     words: np.ndarray          # uint32, padded stream
-    chunk_off: np.ndarray      # uint32 [n_chunks], bits relative to the tile start
+    chunk_len: np.ndarray      # uint16 [n_chunks], bits of every chunk
     tile_off: np.ndarray       # uint64 [n_tiles + 1], absolute bits, multiples of 128
     total_bits: int
     pixels: int
     k: int
-    chunk_pixels: int
-    tile_chunks: int
+    chunk_pixels: int          # pixels per chunk (1 when pixel_splits > 1)
+    pixel_splits: int          # chunks per pixel
+    tile_pixels: int
+
+    @property
+    def chunk_symbols(self) -> int:
+        return self.chunk_pixels * self.k // self.pixel_splits
+
+    def chunk_starts(self) -> np.ndarray:
+        """Absolute start bit of every chunk (tile start plus the lengths before it)."""
+        cpt = self.tile_pixels * self.k // self.chunk_symbols
+        out = np.zeros(self.chunk_len.shape[0], dtype=np.uint64)
+        for t in range(self.tile_off.shape[0] - 1):
+            ln = self.chunk_len[t * cpt:(t + 1) * cpt].astype(np.uint64)
+            out[t * cpt:t * cpt + ln.shape[0]] = self.tile_off[t] + np.concatenate(([0], np.cumsum(ln)[:-1])).astype(np.uint64)
+        return out
 
 
 def round_bf16(v: float) -> float:
@@ -226,28 +240,34 @@ def canonical_codes(lengths: np.ndarray) -> np.ndarray:
     return code
 
 
-def encode(q: np.ndarray, lengths: np.ndarray, bits: int, *, chunk_pixels: int,
-           tile_chunks: int) -> Stream:
+def encode(q: np.ndarray, lengths: np.ndarray, bits: int, *, chunk_pixels: int = 1,
+           pixel_splits: int = 1, tile_pixels: int = 128) -> Stream:
     q = np.ascontiguousarray(q, dtype=np.uint8)
     pixels, k = q.shape
     lengths = np.ascontiguousarray(lengths, dtype=np.uint8)
     if lengths.ndim == 1:
         lengths = lengths[None, :]
     groups = lengths.shape[0]
-    tile_pixels = chunk_pixels * tile_chunks
-    n_tiles = max(1, -(-pixels // tile_pixels)) if pixels else 0
-    n_chunks = -(-pixels // chunk_pixels)
+    if pixel_splits > 1 and chunk_pixels != 1:
+        raise ValueError("a pixel is split only when a chunk is one pixel")
+    if (chunk_pixels * k) % pixel_splits or (tile_pixels * k) % (chunk_pixels * k // pixel_splits):
+        raise ValueError("tiles must hold a whole number of chunks")
+    chunk_symbols = chunk_pixels * k // pixel_splits
+    n_tiles = -(-pixels // tile_pixels) if pixels else 0
+    n_chunks = -(-(pixels * k) // chunk_symbols)
     cap_bits = pixels * k * int(lengths.max()) + 128 * (n_tiles + 1)
     cap_words = cap_bits // 32 + 4
     words = np.zeros(cap_words, dtype=np.uint32)
-    chunk_off = np.zeros(max(n_chunks, 1), dtype=np.uint32)
+    chunk_len = np.zeros(max(n_chunks, 1), dtype=np.uint16)
     tile_off = np.zeros(n_tiles + 1, dtype=np.uint64)
-    total = lib().orc_encode(_p(q), pixels, k, groups, bits, _p(lengths), chunk_pixels,
-                             tile_chunks, _p(words), cap_words, _p(chunk_off), _p(tile_off))
+    total = lib().orc_encode(_p(q), pixels, k, groups, bits, _p(lengths), chunk_symbols,
+                             tile_pixels, _p(words), cap_words, _p(chunk_len), _p(tile_off))
+    if total == -2:
+        raise ValueError("a chunk is longer than 65535 bits")
     if total < 0:
         raise RuntimeError("oracle stream capacity too small")
-    return Stream(words[: total // 32].copy(), chunk_off[:n_chunks].copy(), tile_off, int(total),
-                  pixels, k, chunk_pixels, tile_chunks)
+    return Stream(words[: total // 32].copy(), chunk_len[:n_chunks].copy(), tile_off, int(total),
+                  pixels, k, chunk_pixels, pixel_splits, tile_pixels)
 
 
 def decode_symbols(s: Stream, lengths: np.ndarray, bits: int) -> np.ndarray:
@@ -256,11 +276,11 @@ def decode_symbols(s: Stream, lengths: np.ndarray, bits: int) -> np.ndarray:
         lengths = lengths[None, :]
     q = np.zeros((s.pixels, s.k), dtype=np.uint8)
     words = np.ascontiguousarray(s.words, dtype=np.uint32)
-    chunk_off = np.ascontiguousarray(s.chunk_off, dtype=np.uint32)
+    chunk_len = np.ascontiguousarray(s.chunk_len, dtype=np.uint16)
     tile_off = np.ascontiguousarray(s.tile_off, dtype=np.uint64)
-    rc = lib().orc_decode_symbols(_p(words), words.shape[0], _p(chunk_off), _p(tile_off),
+    rc = lib().orc_decode_symbols(_p(words), words.shape[0], _p(chunk_len), _p(tile_off),
                                   s.pixels, s.k, lengths.shape[0], bits, _p(lengths),
-                                  s.chunk_pixels, s.tile_chunks, _p(q))
+                                  s.chunk_symbols, s.tile_pixels, _p(q))
     if rc != 0:
         raise ValueError("corrupt stream")
     return q

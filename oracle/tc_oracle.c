@@ -378,11 +378,15 @@ void orc_canonical_codes(const uint8_t *len, int nsym, uint32_t *code)
  * O6 / O7. Bit stream.  Symbols are emitted pixel by pixel (p ascending), coefficient j
  * ascending inside a pixel, each with the code of its group's table, most significant code
  * bit first.  Stream bit i lives in 32-bit word i/32 at bit position 31 - (i mod 32).
- * A chunk is chunk_pixels consecutive pixels; a tile is tile_chunks consecutive chunks.
+ * A tile is tile_pixels consecutive pixels; a chunk is chunk_symbols consecutive symbols of
+ * that order (several pixels, one pixel, or a fraction of a pixel's coefficients), with
+ * tile_pixels * K a multiple of chunk_symbols, so that every tile starts a chunk.
  * Tile t starts at absolute bit tile_off[t], always a multiple of 128 (zero padding before
- * it); tile_off[n_tiles] is the padded end of the stream.  chunk_off[i] is the start of
- * chunk i in bits, relative to the start of its tile.  (The paper leaves the layout open:
- * Section 3.1 only says the bit stream is accumulated in external memory.)
+ * it); tile_off[n_tiles] is the padded end of the stream.  chunk_len[i] is the length of
+ * chunk i in bits (16 bits each); inside a tile the chunks follow one another without gaps,
+ * so a chunk starts at its tile's start plus the lengths of the tile's earlier chunks.
+ * (The paper leaves the layout open: Section 3.1 only says the bit stream is accumulated in
+ * external memory.)
  * ---------------------------------------------------------------------------------------- */
 static void put_bit(uint32_t *stream, uint64_t pos, int bit)
 {
@@ -393,48 +397,64 @@ static int get_bit(const uint32_t *stream, uint64_t pos)
     return (int)((stream[pos >> 5] >> (31 - (pos & 31))) & 1u);
 }
 
-/* Encode.  len is [groups][2^bits].  Returns the total padded length in bits, or -1 if
- * cap_words is too small.  stream[0 .. cap_words) is zeroed first. */
+/* Encode.  len is [groups][2^bits].  Returns the total padded length in bits, -1 if
+ * cap_words is too small, -2 if a chunk is longer than 65535 bits.  stream[0 .. cap_words) is
+ * zeroed first. */
 int64_t orc_encode(const uint8_t *q, int64_t pixels, int k, int groups, int bits,
-                   const uint8_t *len, int chunk_pixels, int tile_chunks,
-                   uint32_t *stream, int64_t cap_words, uint32_t *chunk_off, uint64_t *tile_off)
+                   const uint8_t *len, int64_t chunk_symbols, int64_t tile_pixels,
+                   uint32_t *stream, int64_t cap_words, uint16_t *chunk_len, uint64_t *tile_off)
 {
     const int nsym = 1 << bits;
     uint32_t *code = (uint32_t *)malloc(sizeof(uint32_t) * (size_t)groups * nsym);
     for (int g = 0; g < groups; ++g) orc_canonical_codes(len + (int64_t)g * nsym, nsym, code + (int64_t)g * nsym);
     memset(stream, 0, sizeof(uint32_t) * (size_t)cap_words);
-    const int64_t tile_pixels = (int64_t)chunk_pixels * tile_chunks;
     const uint64_t cap_bits = (uint64_t)cap_words * 32u;
-    uint64_t pos = 0, tile_start = 0;
-    int64_t tile = 0, chunk = 0;
-    for (int64_t p = 0; p < pixels; ++p) {
+    uint64_t pos = 0, chunk_start = 0;
+    int64_t tile = 0, chunk = -1, rc = 0;
+    for (int64_t p = 0; p < pixels && rc == 0; ++p) {
         if (p % tile_pixels == 0) {
+            if (chunk >= 0) {
+                if (pos - chunk_start > 65535u) { rc = -2; break; }
+                chunk_len[chunk] = (uint16_t)(pos - chunk_start);   /* last chunk of the tile before */
+            }
             pos = (pos + 127u) & ~(uint64_t)127u;
-            tile_start = pos;
             tile_off[tile++] = pos;
+            chunk_start = pos;
+            ++chunk;
         }
-        if (p % chunk_pixels == 0) chunk_off[chunk++] = (uint32_t)(pos - tile_start);
         for (int j = 0; j < k; ++j) {
+            const int64_t in_tile = (p % tile_pixels) * k + j;       /* symbol index inside the tile */
+            if (in_tile > 0 && in_tile % chunk_symbols == 0) {
+                if (pos - chunk_start > 65535u) { rc = -2; break; }
+                chunk_len[chunk++] = (uint16_t)(pos - chunk_start);
+                chunk_start = pos;
+            }
             const int g = (groups == 1) ? 0 : j;
             const int s = q[p * k + j];
             const int l = len[(int64_t)g * nsym + s];
             const uint32_t cw = code[(int64_t)g * nsym + s];
-            if (pos + (uint64_t)l > cap_bits) { free(code); return -1; }
+            if (pos + (uint64_t)l > cap_bits) { rc = -1; break; }
             for (int b = l - 1; b >= 0; --b) put_bit(stream, pos++, (int)((cw >> b) & 1u));
         }
+    }
+    if (rc == 0 && chunk >= 0) {
+        if (pos - chunk_start > 65535u) rc = -2;
+        else chunk_len[chunk] = (uint16_t)(pos - chunk_start);
     }
     pos = (pos + 127u) & ~(uint64_t)127u;
     tile_off[tile] = pos;
     free(code);
+    if (rc != 0) return rc;
     return (pos <= cap_bits) ? (int64_t)pos : -1;
 }
 
 /* Decode symbols by walking the canonical code one bit at a time: at length l the codes are
  * first[l] .. first[l] + count[l] - 1 and map to the symbols of that length in symbol
- * order.  Returns 0, or -1 if a chunk holds no valid code (corrupt stream). */
-int orc_decode_symbols(const uint32_t *stream, int64_t stream_words, const uint32_t *chunk_off,
+ * order.  Every chunk is decoded from its own start (tile start plus the lengths before it)
+ * and must end exactly after chunk_len bits.  Returns 0, or -1 for a corrupt stream. */
+int orc_decode_symbols(const uint32_t *stream, int64_t stream_words, const uint16_t *chunk_len,
                        const uint64_t *tile_off, int64_t pixels, int k, int groups, int bits,
-                       const uint8_t *len, int chunk_pixels, int tile_chunks, uint8_t *q)
+                       const uint8_t *len, int64_t chunk_symbols, int64_t tile_pixels, uint8_t *q)
 {
     const int nsym = 1 << bits;
     const uint64_t total_bits = (uint64_t)stream_words * 32u;
@@ -460,13 +480,20 @@ int orc_decode_symbols(const uint32_t *stream, int64_t stream_words, const uint3
                 }
         }
     }
-    const int64_t n_chunks = (pixels + chunk_pixels - 1) / chunk_pixels;
-    for (int64_t ch = 0; ch < n_chunks && rc == 0; ++ch) {
-        uint64_t pos = tile_off[ch / tile_chunks] + chunk_off[ch];
-        const int64_t p0 = ch * chunk_pixels;
-        const int64_t p1 = (p0 + chunk_pixels < pixels) ? p0 + chunk_pixels : pixels;
-        for (int64_t p = p0; p < p1 && rc == 0; ++p)
-            for (int j = 0; j < k; ++j) {
+    const int64_t tile_symbols = tile_pixels * k;
+    const int64_t chunks_per_tile = tile_symbols / chunk_symbols;
+    const int64_t total_symbols = pixels * k;
+    const int64_t n_tiles = (pixels + tile_pixels - 1) / tile_pixels;
+    for (int64_t t = 0; t < n_tiles && rc == 0; ++t) {
+        uint64_t chunk_start = tile_off[t];
+        for (int64_t c = 0; c < chunks_per_tile && rc == 0; ++c) {
+            const int64_t n0 = t * tile_symbols + c * chunk_symbols;       /* first symbol of the chunk */
+            if (n0 >= total_symbols) break;
+            const int64_t n1 = (n0 + chunk_symbols < total_symbols) ? n0 + chunk_symbols : total_symbols;
+            const int64_t ch = t * chunks_per_tile + c;
+            uint64_t pos = chunk_start;
+            for (int64_t n = n0; n < n1 && rc == 0; ++n) {
+                const int j = (int)(n % k);
                 const int g = (groups == 1) ? 0 : j;
                 uint32_t cw = 0;
                 int l = 0, found = 0;
@@ -475,13 +502,16 @@ int orc_decode_symbols(const uint32_t *stream, int64_t stream_words, const uint3
                     ++l;
                     if (count[g * 33 + l] > 0 && cw >= first[g * 33 + l] &&
                         cw - first[g * 33 + l] < (uint32_t)count[g * 33 + l]) {
-                        q[p * k + j] = (uint8_t)sorted[(int64_t)g * nsym + start[g * 33 + l] + (int)(cw - first[g * 33 + l])];
+                        q[n] = (uint8_t)sorted[(int64_t)g * nsym + start[g * 33 + l] + (int)(cw - first[g * 33 + l])];
                         found = 1;
                         break;
                     }
                 }
-                if (!found) { rc = -1; break; }
+                if (!found) rc = -1;
             }
+            if (rc == 0 && pos - chunk_start != (uint64_t)chunk_len[ch]) rc = -1;
+            chunk_start += chunk_len[ch];
+        }
     }
     free(first); free(count); free(start); free(sorted); free(code);
     return rc;

@@ -25,7 +25,7 @@ def _chain(spec, bits, n_cal=8, n_test=2, per_channel=False, identity=False, dty
     hist = oracle.histogram(q_cal, bits, per_channel)
     ln = oracle.huffman_lengths(hist, 12)
     q = oracle.quantize(m, oracle.project(m, x))
-    s = oracle.encode(q, ln, bits, chunk_pixels=1, tile_chunks=128)
+    s = oracle.encode(q, ln, bits, chunk_pixels=1, tile_pixels=128)
     assert np.array_equal(oracle.decode_symbols(s, ln, bits), q)
     xhat = oracle.reconstruct(m, q, x.shape, out_bf16=(dtype == torch.bfloat16))
     return dict(model=m, q=q, q_cal=q_cal, hist=hist, lengths=ln, stream=s, x=x, xhat=xhat,
@@ -62,7 +62,7 @@ def test_tail_channels_collapse_to_one_symbol():
     assert oracle.entropy(hist[-1]) == 0.0
     assert ln[-1][q[0, -1]] == 1
     assert oracle.entropy(hist[0]) > 2.0         # while the leading channel carries the bits
-    s = oracle.encode(q, ln, 4, chunk_pixels=1, tile_chunks=128)
+    s = oracle.encode(q, ln, 4, chunk_pixels=1, tile_pixels=128)
     assert np.array_equal(oracle.decode_symbols(s, ln, 4), q)
 
 
