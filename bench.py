@@ -109,16 +109,16 @@ def oracle_setup(spec, bits, calib_maps, sample_images, dtype):
     q_cal = oracle.quantize(m, oracle.project(m, cal))
     lengths = oracle.huffman_lengths(oracle.histogram(q_cal, bits, False), 12)
     return dict(model=m, lengths=lengths, x=x, bits=bits, dtype=dtype,
-                chunk_pixels=max(1, 256 // spec.c))
+                chunk_pixels=1 << max(0, (127 // spec.c).bit_length()), pixel_splits=2 if spec.c >= 256 and spec.c % 32 == 0 else 1)
 
 
 def oracle_timed_pass(o):
     """Time the CPU oracle's encode + decode over the prepared sample (one pass)."""
     import oracle
-    m, lengths, x, bits, cp = o["model"], o["lengths"], o["x"], o["bits"], o["chunk_pixels"]
+    m, lengths, x, bits, cp, splits = o["model"], o["lengths"], o["x"], o["bits"], o["chunk_pixels"], o["pixel_splits"]
     t0 = time.perf_counter()
     q = oracle.quantize(m, oracle.project(m, x))
-    s = oracle.encode(q, lengths, bits, chunk_pixels=cp, tile_chunks=128 // cp)
+    s = oracle.encode(q, lengths, bits, chunk_pixels=cp, pixel_splits=splits, tile_pixels=128)
     t1 = time.perf_counter()
     q2 = oracle.decode_symbols(s, lengths, bits)
     oracle.reconstruct(m, q2, x.shape, out_bf16=(o["dtype"] == torch.bfloat16))
@@ -214,7 +214,7 @@ def main():
         raise SystemExit(f"codec reported status {status}")
     total_bits = enc.total_bits()
     stream_bytes = total_bits // 8
-    side_bytes = lay.chunk_off_bytes + lay.tile_off_bytes
+    side_bytes = lay.chunk_len_bytes + lay.tile_off_bytes
     test_stats = tc.tc_stats(ctx, model, cb, x[: min(batch, 256)], groups=1, want_hist=False)
 
     def step():
@@ -301,7 +301,7 @@ def main():
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "layer": spec.name, "batch_per_gpu": batch, "bits": bits,
-                   "chunk_pixels": lay.chunk_pixels, "codebook": "per-layer", "calib_maps": w.calib_maps,
+                   "chunk_pixels": lay.chunk_pixels, "pixel_splits": lay.pixel_splits, "codebook": "per-layer", "calib_maps": w.calib_maps,
                    "l2": "inputs larger than L2 (411 MB per pass), no flush", "parallelism": f"batch-sharded x{world}"},
         "encode_gbs": raw_bytes / (enc_avg * 1e-3) / 1e9, "decode_gbs": raw_bytes / (dec_avg * 1e-3) / 1e9,
         "encode_ms": enc_avg, "decode_ms": dec_avg,

@@ -157,24 +157,32 @@ tc_status tc_host_eigh(double *a, int32_t n, double *evals, double *evecs);
  *     each with the code of table j (groups == K) or table 0.
  *   - Code bits most-significant first; stream bit i is bit 31 - (i mod 32) of the
  *     little-endian 32-bit word i / 32.
- *   - A chunk is `chunk_pixels` consecutive pixels (a power of two, 1..128); a tile is
- *     128 pixels.  Tile t starts at absolute bit tile_off[t], a multiple of 128, with zero
- *     padding before it; tile_off[n_tiles] is the padded end of the stream.  chunk_off[i]
- *     is the start of chunk i in bits relative to the start of its tile.
+ *   - A tile is 128 pixels.  Tile t starts at absolute bit tile_off[t], a multiple of 128,
+ *     with zero padding before it; tile_off[n_tiles] is the padded end of the stream.
+ *   - A chunk is the unit a decoder thread starts from: `chunk_pixels` consecutive pixels (a
+ *     power of two, 1..128), or, with chunk_pixels == 1, one of `pixel_splits` equal runs of
+ *     a pixel's K coefficients (pixel_splits 1, 2 or 4; K a multiple of 8 * pixel_splits).
+ *     Chunks are numbered in stream order; chunk_len[i] is the length of chunk i in bits, and
+ *     inside a tile the chunks follow one another without gaps, so a chunk starts at its
+ *     tile's start plus the lengths of the tile's earlier chunks.  A chunk may not exceed
+ *     65535 bits: chunk_pixels * K / pixel_splits * (longest code) must stay below that.
  * ------------------------------------------------------------------------------------- */
 typedef struct {
-    int32_t chunk_pixels; /* power of two in 1..128; 0 = library default for this shape */
+    int32_t chunk_pixels; /* power of two in 1..128; 0 = library default for this shape   */
+    int32_t pixel_splits; /* 1, 2 or 4 (needs chunk_pixels == 1); 0 = library default      */
 } tc_encode_params;
 
 typedef struct {
     int64_t n_tiles, n_chunks;
     size_t stream_bytes;    /* worst case: every symbol at the longest code + padding  */
-    size_t chunk_off_bytes; /* n_chunks * 4                                            */
+    size_t chunk_len_bytes; /* n_chunks * 2                                            */
     size_t tile_off_bytes;  /* (n_tiles + 1) * 8                                       */
-    int32_t chunk_pixels;   /* the value that will be used                             */
+    int32_t chunk_pixels;   /* the values that will be used                            */
+    int32_t pixel_splits;
 } tc_stream_layout;
 
-/* Worst-case buffer sizes for encoding `x`. Host only. */
+/* Worst-case buffer sizes for encoding `x`. Host only.  INVALID_ARG for a chunk shape the
+ * format cannot hold (see above). */
 tc_status tc_encode_bound(const tc_model *model, const tc_codebook *cb, const tc_tensor *x,
                           const tc_encode_params *params, tc_stream_layout *out);
 
@@ -190,13 +198,13 @@ typedef struct {
  *   stream_out  DEVICE, 16-byte aligned, `capacity` bytes; any capacity is accepted -- if
  *               the coded tensor does not fit, nothing is written past it and the status
  *               word records TC_ERR_BUFFER_TOO_SMALL.  tc_encode_bound() never fails.
- *   chunk_off   DEVICE uint32[n_chunks];  tile_off  DEVICE uint64[n_tiles + 1]
+ *   chunk_len   DEVICE uint16[n_chunks], 4-byte aligned;  tile_off  DEVICE uint64[n_tiles + 1]
  *               (tile_off[n_tiles] = total stream length in bits).
  * Errors: INVALID_ARG, UNSUPPORTED (C > 1024, K != C with the tensor-core path, dtype /
  * basis_dtype mismatch), CUDA. */
 tc_status tc_encode(tc_ctx *ctx, const tc_model *model, const tc_codebook *cb,
                     const tc_tensor *x, const tc_encode_params *params, void *stream_out,
-                    size_t capacity, uint32_t *chunk_off, uint64_t *tile_off,
+                    size_t capacity, uint16_t *chunk_len, uint64_t *tile_off,
                     const tc_debug_out *debug, void *cuda_stream);
 
 /* tc_encode without any allocation.  (The paper has no counterpart: this entry point exists
@@ -220,17 +228,18 @@ tc_status tc_encode(tc_ctx *ctx, const tc_model *model, const tc_codebook *cb,
 #define TC_NOALLOC_MAX_TILES 65536
 tc_status tc_encode_noalloc(tc_ctx *ctx, const tc_model *model, const tc_codebook *cb,
                             const tc_tensor *x, const tc_encode_params *params, void *stream_out,
-                            size_t capacity, uint32_t *chunk_off, uint64_t *tile_off,
+                            size_t capacity, uint16_t *chunk_len, uint64_t *tile_off,
                             void *cuda_stream);
 
 /* Decode (Section 3: VLD, inverse quantiser, inverse transform; no non-linearity is applied).
  *   stream       DEVICE, 16-byte aligned, `stream_bytes` readable bytes
  *   x_hat        caller-allocated tensor of the shape and dtype that was encoded
- * Offsets are validated against `stream_bytes` on the device; a stream that cannot be valid
- * sets TC_ERR_CORRUPT_STREAM in the status word and leaves the affected tile's output
- * unspecified (but in bounds). */
+ * Offsets and lengths are validated on the device (tile offsets against `stream_bytes`, the
+ * chunk lengths of a tile against the tile's size, and every chunk must decode to exactly
+ * its recorded length); a stream that fails sets TC_ERR_CORRUPT_STREAM in the status word and
+ * leaves the affected tile's output unspecified (but in bounds). */
 tc_status tc_decode(tc_ctx *ctx, const tc_model *model, const tc_codebook *cb, const void *stream,
-                    size_t stream_bytes, const uint32_t *chunk_off, const uint64_t *tile_off,
+                    size_t stream_bytes, const uint16_t *chunk_len, const uint64_t *tile_off,
                     const tc_encode_params *params, const tc_tensor *x_hat, void *cuda_stream);
 
 /* Whole chain on HOST tensors (Section 3: encoder, memory, decoder): copies `x_host` (dense

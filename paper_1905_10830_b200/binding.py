@@ -44,13 +44,13 @@ class _CodebookParams(C.Structure):
 
 
 class _EncodeParams(C.Structure):
-    _fields_ = [("chunk_pixels", C.c_int32)]
+    _fields_ = [("chunk_pixels", C.c_int32), ("pixel_splits", C.c_int32)]
 
 
 class _StreamLayout(C.Structure):
     _fields_ = [("n_tiles", C.c_int64), ("n_chunks", C.c_int64), ("stream_bytes", C.c_size_t),
-                ("chunk_off_bytes", C.c_size_t), ("tile_off_bytes", C.c_size_t),
-                ("chunk_pixels", C.c_int32)]
+                ("chunk_len_bytes", C.c_size_t), ("tile_off_bytes", C.c_size_t),
+                ("chunk_pixels", C.c_int32), ("pixel_splits", C.c_int32)]
 
 
 class _DebugOut(C.Structure):
@@ -179,16 +179,17 @@ class StreamLayout:
     n_tiles: int
     n_chunks: int
     stream_bytes: int
-    chunk_off_bytes: int
+    chunk_len_bytes: int
     tile_off_bytes: int
     chunk_pixels: int
+    pixel_splits: int
 
 
 @dataclass
 class EncodedStream:
     """Device buffers written by tc_encode."""
     words: torch.Tensor        # uint8 buffer holding the little-endian 32-bit stream words
-    chunk_off: torch.Tensor    # int32 (bit pattern of uint32) [n_chunks]
+    chunk_len: torch.Tensor    # int16 (bit pattern of uint16) [n_chunks, rounded up to even]
     tile_off: torch.Tensor     # int64 (bit pattern of uint64) [n_tiles + 1]
     layout: StreamLayout
     coefficients: torch.Tensor | None = None
@@ -314,26 +315,27 @@ def tc_host_eigh(a: np.ndarray):
     return evals, evecs
 
 
-def tc_encode_bound(model: Model, cb: Codebook, x: torch.Tensor, chunk_pixels: int = 0) -> StreamLayout:
+def tc_encode_bound(model: Model, cb: Codebook, x: torch.Tensor, chunk_pixels: int = 0,
+                    pixel_splits: int = 0) -> StreamLayout:
     t = _tensor(x)
-    p = _EncodeParams(chunk_pixels)
+    p = _EncodeParams(chunk_pixels, pixel_splits)
     lay = _StreamLayout()
     _check(load_library().tc_encode_bound(model.ptr, cb.ptr, C.byref(t), C.byref(p), C.byref(lay)), "tc_encode_bound")
-    return StreamLayout(lay.n_tiles, lay.n_chunks, lay.stream_bytes, lay.chunk_off_bytes, lay.tile_off_bytes,
-                        lay.chunk_pixels)
+    return StreamLayout(lay.n_tiles, lay.n_chunks, lay.stream_bytes, lay.chunk_len_bytes, lay.tile_off_bytes,
+                        lay.chunk_pixels, lay.pixel_splits)
 
 
 def tc_encode(ctx: Context, model: Model, cb: Codebook, x: torch.Tensor, *, chunk_pixels: int = 0,
-              out: EncodedStream | None = None, capacity: int | None = None, debug: bool = False,
+              pixel_splits: int = 0, out: EncodedStream | None = None, capacity: int | None = None, debug: bool = False,
               k: int | None = None) -> EncodedStream:
     """Encode `x`.  Buffers are allocated with torch (worst-case size) unless `out` is given."""
     t = _tensor(x)
-    lay = tc_encode_bound(model, cb, x, chunk_pixels)
+    lay = tc_encode_bound(model, cb, x, chunk_pixels, pixel_splits)
     dev = x.device
     if out is None:
         nbytes = lay.stream_bytes if capacity is None else capacity
         out = EncodedStream(torch.empty(max(nbytes, 16), dtype=torch.uint8, device=dev),
-                            torch.empty(max(lay.n_chunks, 1), dtype=torch.int32, device=dev),
+                            torch.empty(max(lay.n_chunks + (lay.n_chunks & 1), 2), dtype=torch.int16, device=dev),
                             torch.empty(lay.n_tiles + 1, dtype=torch.int64, device=dev), lay)
     dbg = None
     if debug:
@@ -342,23 +344,23 @@ def tc_encode(ctx: Context, model: Model, cb: Codebook, x: torch.Tensor, *, chun
         out.coefficients = torch.empty(pixels, kk, dtype=torch.float32, device=dev)
         out.symbols = torch.empty(pixels, kk, dtype=torch.uint8, device=dev)
         dbg = _DebugOut(out.coefficients.data_ptr(), out.symbols.data_ptr())
-    p = _EncodeParams(chunk_pixels)
+    p = _EncodeParams(lay.chunk_pixels, lay.pixel_splits)
     cap = out.words.numel() if capacity is None else min(capacity, out.words.numel())
     _check(load_library().tc_encode(ctx.ptr, model.ptr, cb.ptr, C.byref(t), C.byref(p), out.words.data_ptr(), cap,
-                                    out.chunk_off.data_ptr(), out.tile_off.data_ptr(),
+                                    out.chunk_len.data_ptr(), out.tile_off.data_ptr(),
                                     C.byref(dbg) if dbg is not None else None, _stream_ptr(ctx.device)), "tc_encode")
     return out
 
 
 def tc_encode_noalloc(ctx: Context, model: Model, cb: Codebook, x: torch.Tensor, out: EncodedStream, *,
-                      chunk_pixels: int = 0) -> EncodedStream:
+                      chunk_pixels: int = 0, pixel_splits: int = 0) -> EncodedStream:
     """Encode `x` into buffers the caller already owns, through the entry point that never
     allocates device memory (see tc_encode_noalloc in include/tc.h).  `out` must come from an
     earlier tc_encode of the same shape or be sized with tc_encode_bound."""
     t = _tensor(x)
-    p = _EncodeParams(chunk_pixels)
+    p = _EncodeParams(chunk_pixels, pixel_splits)
     _check(load_library().tc_encode_noalloc(ctx.ptr, model.ptr, cb.ptr, C.byref(t), C.byref(p), out.words.data_ptr(),
-                                            out.words.numel(), out.chunk_off.data_ptr(), out.tile_off.data_ptr(),
+                                            out.words.numel(), out.chunk_len.data_ptr(), out.tile_off.data_ptr(),
                                             _stream_ptr(ctx.device)), "tc_encode_noalloc")
     return out
 
@@ -368,16 +370,16 @@ def tc_decode(ctx: Context, model: Model, cb: Codebook, enc: EncodedStream, shap
     if out is None:
         out = torch.empty(shape, dtype=dtype, device=enc.words.device)
     t = _tensor(out)
-    p = _EncodeParams(enc.layout.chunk_pixels)
+    p = _EncodeParams(enc.layout.chunk_pixels, enc.layout.pixel_splits)
     nbytes = enc.words.numel() if stream_bytes is None else stream_bytes
     _check(load_library().tc_decode(ctx.ptr, model.ptr, cb.ptr, enc.words.data_ptr(), nbytes,
-                                    enc.chunk_off.data_ptr(), enc.tile_off.data_ptr(), C.byref(p), C.byref(t),
+                                    enc.chunk_len.data_ptr(), enc.tile_off.data_ptr(), C.byref(p), C.byref(t),
                                     _stream_ptr(ctx.device)), "tc_decode")
     return out
 
 
 def tc_roundtrip_host(ctx: Context, model: Model, cb: Codebook, x_host: torch.Tensor, out_host: torch.Tensor, *,
-                      chunk_pixels: int = 0) -> int:
+                      chunk_pixels: int = 0, pixel_splits: int = 0) -> int:
     """Encode + decode a HOST tensor (dense NCHW, ideally pinned) into `out_host`; returns the
     coded length in bits.  The copies and both kernels run inside the C call."""
     if x_host.is_cuda or out_host.is_cuda or not x_host.is_contiguous() or not out_host.is_contiguous():
@@ -386,7 +388,7 @@ def tc_roundtrip_host(ctx: Context, model: Model, cb: Codebook, x_host: torch.Te
         raise ValueError("input and output must have the same shape and dtype")
     n, c, h, w = x_host.shape
     dt = TC_F32 if x_host.dtype == torch.float32 else TC_BF16
-    p = _EncodeParams(chunk_pixels)
+    p = _EncodeParams(chunk_pixels, pixel_splits)
     bits = C.c_uint64(0)
     _check(load_library().tc_roundtrip_host(ctx.ptr, model.ptr, cb.ptr, x_host.data_ptr(), out_host.data_ptr(), n, c, h, w,
                                             dt, C.byref(p), C.byref(bits), _stream_ptr(ctx.device)), "tc_roundtrip_host")

@@ -33,6 +33,7 @@ __global__ void __launch_bounds__(kThreads) encode_simt_kernel(EncodeArgs a)
     __shared__ unsigned int s_warp_sums[4];
     __shared__ unsigned long long s_base;
     __shared__ int s_write_ok;
+    __shared__ unsigned int s_pixel_off[TC_TILE_PIXELS + 1];   // bit offset of every pixel in the tile, then the tile's bits
 
     const int t = threadIdx.x;
     if (t == 0) s_tile = a.emit ? (long long)atomicAdd(a.ticket, 1u) : (long long)blockIdx.x;
@@ -98,10 +99,14 @@ __global__ void __launch_bounds__(kThreads) encode_simt_kernel(EncodeArgs a)
 
     // ---- bit lengths, offsets --------------------------------------------------------
     unsigned int my_bits = 0;
+    unsigned int part_bits[4] = {0u, 0u, 0u, 0u};             // per run of K / splits coefficients
+    const int k_part = a.k / a.splits;
     if (valid)
         for (int j = 0; j < a.k; ++j) {
             const int g = (a.groups == 1) ? 0 : j;
-            my_bits += enc[g * nsym + s_q[j * kThreads + t]] & 0xffu;
+            const unsigned int l = enc[g * nsym + s_q[j * kThreads + t]] & 0xffu;
+            my_bits += l;
+            part_bits[j / k_part] += l;
         }
     unsigned int tile_bits;
     const unsigned int my_off = group_exclusive_scan_128(my_bits, s_warp_sums, t, 1, tile_bits);
@@ -120,7 +125,18 @@ __global__ void __launch_bounds__(kThreads) encode_simt_kernel(EncodeArgs a)
     }
     __syncthreads();
     const unsigned long long base = s_base;
-    if (valid && (p % a.chunk_pixels) == 0) a.chunk_off[p / a.chunk_pixels] = my_off;
+    // chunk lengths: a chunk is chunk_pixels pixels, or one of `splits` runs of one pixel
+    s_pixel_off[t] = my_off;
+    if (t == 0) s_pixel_off[TC_TILE_PIXELS] = tile_bits;
+    __syncthreads();
+    if (valid) {
+        if (a.splits > 1) {
+            for (int sp = 0; sp < a.splits; ++sp) a.chunk_len[p * a.splits + sp] = (uint16_t)part_bits[sp];
+        } else if ((p % a.chunk_pixels) == 0) {
+            const int last = min(t + a.chunk_pixels, TC_TILE_PIXELS);
+            a.chunk_len[p / a.chunk_pixels] = (uint16_t)(s_pixel_off[last] - my_off);
+        }
+    }
     if (!s_write_ok) return;
 
     // ---- zero the tile's words, then pack --------------------------------------------
@@ -187,6 +203,7 @@ __global__ void __launch_bounds__(kThreads) decode_simt_kernel(DecodeArgs a)
     double *s_panel = s_mean + a.c;                                // [K][kRowBlock]
     uint8_t *s_q = reinterpret_cast<uint8_t *>(s_panel + (size_t)a.k * kRowBlock);   // [K][128]
     __shared__ int s_bad;
+    __shared__ uint16_t s_len[4 * TC_TILE_PIXELS];                 // chunk lengths of the tile
 
     const int t = threadIdx.x;
     const long long tile = blockIdx.x;
@@ -206,30 +223,38 @@ __global__ void __launch_bounds__(kThreads) decode_simt_kernel(DecodeArgs a)
             if (t == 0) tc_dev_set_status(a.status, TC_ERR_CORRUPT_STREAM);
             return;
         }
-        const int chunks_per_tile = TC_TILE_PIXELS / a.chunk_pixels;
-        const long long ch = tile * chunks_per_tile + t;
-        if (t < chunks_per_tile && ch < a.n_chunks) {
-            const unsigned long long off = a.chunk_off[ch];
-            bool bad = base + off > end;
+        const int chunks_per_tile = a.splits * TC_TILE_PIXELS / a.chunk_pixels;      // at most 512
+        const int chunk_symbols = a.chunk_pixels * a.k / a.splits;
+        for (int ci = t; ci < chunks_per_tile; ci += kThreads) {
+            const long long ch = tile * chunks_per_tile + ci;
+            s_len[ci] = ch < a.n_chunks ? a.chunk_len[ch] : (uint16_t)0;
+        }
+        __syncthreads();
+        const int lut_size = 1 << a.lut_bits;
+        for (int ci = t; ci < chunks_per_tile; ci += kThreads) {
+            if (tile * chunks_per_tile + ci >= a.n_chunks) break;
+            // the chunk starts after the tile's earlier chunks and must end after its own length
+            unsigned long long off = 0;
+            for (int i = 0; i < ci; ++i) off += s_len[i];
+            const unsigned int want = s_len[ci];
+            bool bad = base + off + want > end;
             if (!bad) {
                 BitReader r;
                 r.init(a.stream, base + off, end);
-                unsigned long long used = base + off;
-                const int lut_size = 1 << a.lut_bits;
-                const int first_pixel = t * a.chunk_pixels;
-                for (int pp = 0; pp < a.chunk_pixels; ++pp) {
-                    if (tile * TC_TILE_PIXELS + first_pixel + pp >= a.pixels) break;
-                    for (int j = 0; j < a.k; ++j) {
-                        const int g = (a.groups == 1) ? 0 : j;
-                        const uint32_t e = __ldg(a.lut + (size_t)g * lut_size + r.peek(a.lut_bits));
-                        const int len = (int)(e & 0xffu);
-                        s_q[j * kThreads + first_pixel + pp] = (uint8_t)(e >> 8);
-                        r.skip(len);
-                        used += len;
-                        if (len == 0) bad = true;
-                    }
+                unsigned int used = 0;
+                const int first = ci * chunk_symbols;                 // first symbol, counted inside the tile
+                for (int n = first; n < first + chunk_symbols; ++n) {
+                    const int lp = n / a.k, j = n - lp * a.k;           // pixel inside the tile, coefficient
+                    if (tile * TC_TILE_PIXELS + lp >= a.pixels) break;
+                    const int g = (a.groups == 1) ? 0 : j;
+                    const uint32_t e = __ldg(a.lut + (size_t)g * lut_size + r.peek(a.lut_bits));
+                    const int len = (int)(e & 0xffu);
+                    s_q[j * kThreads + lp] = (uint8_t)(e >> 8);
+                    r.skip(len);
+                    used += len;
+                    if (len == 0) bad = true;
                 }
-                if (used > end) bad = true;
+                if (used != want) bad = true;
             }
             if (bad) s_bad = 1;
         }

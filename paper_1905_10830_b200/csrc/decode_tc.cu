@@ -2,13 +2,22 @@
 // transform).
 //
 // One persistent block per SM; two tiles of 128 pixels are in flight at a time.  Warp roles:
-//   warps 0-3, 4-7     two VLD groups (alternating tiles): one thread per chunk walks its part
+//   warps 0-7, 8-15    two VLD groups (alternating tiles): one thread per chunk walks its part
 //                      of the bit stream with a table-driven canonical Huffman decoder and
-//                      writes the symbols, as exact bf16 integers, into the K-major A operand
-//   warps 8-15         epilogue, all eight warps on every tile (two channel halves):
-//                      TMEM -> registers, x_hat = step * acc + bias, round to bf16, NCHW stores
-//   warps 16, 17       one thread each issues the tcgen05.mma of its group:
-//                      D[pixel][c] = (Q[pixel][j] - center) * T[j][c]
+//                      writes the symbols, as exact bf16 integers, into the K-major A operand.
+//                      With two chunks per pixel (pixel_splits = 2) warps 0-3 of a group decode
+//                      the first half of the coefficients and warps 4-7 the second half, each
+//                      half feeding its own two-slot ring of 16-coefficient panels; otherwise
+//                      only warps 0-3 of a group work.
+//   warps 16-23        epilogue, all eight warps on every tile: TMEM -> registers,
+//                      x_hat = step * acc + bias, round to bf16, NCHW stores.  The accumulator is
+//                      held transposed (TMEM lane = channel, column = pixel): a thread owns one
+//                      channel and gets 16 consecutive pixels per TMEM load; each warp turns its
+//                      32 channels x 32 pixels through a private shared-memory block (16-byte
+//                      writes, no block barrier) so that every channel row leaves as 64
+//                      contiguous bytes.
+//   warps 24, 25       one thread each issues the tcgen05.mma of its group, one per block of 128
+//                      channels:  D[c][pixel] = T[j][c] * (Q[pixel][j] - center)
 // Each VLD group copies the bit-stream segment of its next tile into shared memory (cp.async,
 // double-buffered) while it decodes the current one, so that the decoder's refills are
 // shared-memory reads; a segment too long for the buffer is read from global memory instead.
@@ -25,47 +34,54 @@ namespace {
 using namespace tcdev;
 using namespace sm100;
 
-constexpr int kPanelK = 32;                                   // coefficients per ring stage
-constexpr int kStageBytes = kPanelK * TC_TILE_PIXELS * 2;     // 8 KB
-constexpr int kThreads = 18 * 32;
+constexpr int kVldWarps = 16, kEpiWarp0 = 16, kMmaWarp0 = 24;
+constexpr int kThreads = 26 * 32;
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;
-constexpr int kMaxStages = 8;                                 // per group
-constexpr int kTransposeBytes = 32 * TC_TILE_PIXELS * 2;      // 32 channels x 128 pixels of bf16
+constexpr int kMaxSlots = 8;                                  // ring slots per group
 // A chunk that starts inside a staged segment is read for at most chunk_pixels * K codes of 12
 // bits, whatever the bits say; the slack after each buffer keeps those reads inside the block's
 // shared memory even for a corrupt stream (the buffers lie back to back, the slack follows the
 // last one).  Chunks longer than the slack allows are not staged.
 constexpr int kStreamSlack = 1024;
+// Epilogue transpose block of one warp: 32 channel rows of 32 pixels (64 bytes) with 16 bytes
+// of padding, which keeps both the 16-byte row writes and the 8-byte reads spread over the banks.
+constexpr int kTrRowBytes = 80;
+constexpr int kTrWarpBytes = 32 * kTrRowBytes;
 
 struct SmemLayout {
-    uint32_t basis, ring, lut, bias, sbuf, tbuf, total;
-    int stages;                                               // ring stages per group
+    uint32_t basis, ring, lut, tbuf, sbuf, total;
+    int slots;                                                // ring slots per group (0: does not fit)
+    int panel_k;                                              // coefficients per ring slot
+    uint32_t slot_bytes;
     uint32_t stream_buf;                                      // bytes per staged stream buffer (4 buffers), 0 = none
 };
 
-__host__ __device__ inline SmemLayout smem_layout(int c, int k, int lut_entries, int chunk_pixels, int budget)
+__host__ __device__ inline SmemLayout smem_layout(int c, int k, int lut_entries, int chunk_pixels, int splits, int budget)
 {
     SmemLayout l;
     l.basis = 0;
-    l.lut = (uint32_t)(((size_t)c * k * 2 + 1023) & ~(size_t)1023);
-    l.bias = l.lut + (uint32_t)lut_entries * 4;
-    l.ring = (l.bias + (uint32_t)c * 4 + 1023) & ~1023u;
-    const int n_panels = (k + kPanelK - 1) / kPanelK;
-    // a chunk of several pixels is decoded pixel by pixel, so every panel of the tile has to
-    // stay resident until the chunk's last pixel is done; single-pixel chunks stream through
-    // two stages
-    int want = chunk_pixels > 1 ? n_panels : 2;
+    const int c_pad = ((c + 127) / 128) * 128;                // the MMA takes 128 channels at a time
+    l.lut = (uint32_t)(((size_t)c_pad * k * 2 + 1023) & ~(size_t)1023);
+    l.ring = (l.lut + (uint32_t)lut_entries * 4 + 1023) & ~1023u;
+    // Two chunks per pixel: each half of the coefficients streams through its own two slots of
+    // 16 coefficients.  One chunk per pixel: two slots of 32 coefficients.  A chunk of several
+    // pixels is decoded pixel by pixel, so every panel of the tile has to stay resident until
+    // the chunk's last pixel is done.
+    l.panel_k = splits == 2 ? 16 : 32;
+    l.slot_bytes = (uint32_t)l.panel_k * TC_TILE_PIXELS * 2;
+    const int n_panels = (k + l.panel_k - 1) / l.panel_k;
+    int want = splits == 2 ? 4 : (chunk_pixels > 1 ? n_panels : 2);
     if (want < 2) want = 2;
-    l.stages = want;
-    l.tbuf = l.ring + 2u * (uint32_t)want * kStageBytes;          // two 8 KB transpose buffers (epilogue)
-    l.sbuf = l.tbuf + 2u * kTransposeBytes;
+    l.slots = want;
+    l.tbuf = l.ring + 2u * (uint32_t)want * l.slot_bytes;         // eight warp-private transpose blocks (epilogue)
+    l.sbuf = l.tbuf + 8u * kTrWarpBytes;
     l.stream_buf = 0;
     // four stream buffers back to back (an overrun of one lands in the next), one slack area at the end
-    for (uint32_t kb = 12; kb >= 3; --kb)
+    for (uint32_t kb = 16; kb >= 3; --kb)
         if ((long long)l.sbuf + 4ll * kb * 1024 + kStreamSlack <= (long long)budget) { l.stream_buf = kb * 1024; break; }
     l.total = l.sbuf + (l.stream_buf ? 4u * l.stream_buf + kStreamSlack : 0u);
-    if ((int)l.total > budget || want > kMaxStages) l.stages = 0;
+    if ((int)l.total > budget || want > kMaxSlots) l.slots = 0;
     return l;
 }
 
@@ -180,54 +196,120 @@ struct SmemWindowReader {
     }
 };
 
+// Branch-free reader for per-layer tables held in shared memory.  The window hi:lo holds the
+// next 64 - c stream bits left-aligned, where c (the low bits of `used`) counts the bits taken
+// since the last refill; a table entry carries its code length in bits 0-7, zeros in bits 8-15
+// and the decoded value in bits 16-31, so that `used += entry` counts bits without a mask and
+// the funnel shifts (which take their amount modulo 32) can be fed the entry as it is.
+// refill() runs once per two symbols: codes are at most 12 bits, so that after it c < 32, the
+// first symbol sees at least 33 valid bits and the second at least 21.
+struct SmemSymbolReader {
+    uint32_t next_addr;               // shared address of the word after `ahead`
+    uint32_t hi, lo, ahead;
+    uint32_t used;                    // low 8 bits: c
+
+    __device__ __forceinline__ static uint32_t lds(uint32_t addr)
+    {
+        uint32_t v;
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+        return v;
+    }
+    __device__ __forceinline__ void init(uint32_t seg_addr, uint32_t bitpos)
+    {
+        const uint32_t a0 = seg_addr + (bitpos >> 5) * 4u;
+        const uint32_t w0 = lds(a0), w1 = lds(a0 + 4);
+        ahead = lds(a0 + 8);
+        next_addr = a0 + 12;
+        const int sh = (int)(bitpos & 31u);
+        hi = __funnelshift_l(w1, w0, sh);
+        lo = w1 << sh;
+        used = (uint32_t)sh;
+    }
+    __device__ __forceinline__ void idle(uint32_t seg_addr)
+    {
+        hi = lo = ahead = 0;
+        used = 0;
+        next_addr = seg_addr;
+    }
+    __device__ __forceinline__ uint32_t peek(int nbits) const { return hi >> (32 - nbits); }
+    __device__ __forceinline__ void take(uint32_t entry)
+    {
+        hi = __funnelshift_l(lo, hi, entry);
+        lo = __funnelshift_l(0u, lo, entry);
+        used += entry;
+    }
+    __device__ __forceinline__ void refill()
+    {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b32 t, u;\n\t"
+            "and.b32 t, %3, 32;\n\t"
+            "setp.ne.u32 p, t, 0;\n\t"
+            "shf.l.wrap.b32 t, %2, 0, %3;\n\t"     // ahead >> (32 - (c - 32)); the shifts take c modulo 32
+            "shf.l.wrap.b32 u, 0, %2, %3;\n\t"     // ahead << (c - 32)
+            "@p or.b32 %0, %0, t;\n\t"
+            "@p or.b32 %1, %1, u;\n\t"
+            "@p add.u32 %3, %3, -32;\n\t"
+            "@p ld.shared.u32 %2, [%4];\n\t"
+            "@p add.u32 %4, %4, 4;\n\t}"
+            : "+r"(hi), "+r"(lo), "+r"(ahead), "+r"(used), "+r"(next_addr));
+    }
+    // bits consumed since init(seg_addr, bitpos)
+    __device__ __forceinline__ uint32_t consumed(uint32_t seg_addr, uint32_t bitpos) const
+    {
+        const uint32_t a0 = seg_addr + (bitpos >> 5) * 4u;
+        return (next_addr - 12u - a0) * 8u + (used & 0xffu) - (bitpos & 31u);
+    }
+};
+
 template <bool kPerChannel>
 __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem[];
-    __shared__ __align__(8) unsigned long long s_full[2][kMaxStages], s_empty[2][kMaxStages], s_tfull[2], s_tempty[2];
+    __shared__ __align__(8) unsigned long long s_full[2][kMaxSlots], s_empty[2][kMaxSlots], s_tfull[2], s_tempty[2];
     __shared__ uint32_t s_tmem_base;
+    __shared__ unsigned int s_wsum[2][2][4];   // [group][half][warp]: chunk bits per warp, for the start positions
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int lut_size = 1 << a.lut_bits;
-    constexpr int pair_size = 1 << TC_PAIR_LUT_BITS;
-    const SmemLayout L = smem_layout(a.c, a.k, kPerChannel ? 0 : 2 * pair_size, a.chunk_pixels, a.smem_budget);
-    const int stages = L.stages;
+    const int S = a.splits;                      // chunks per pixel: 1 or 2
+    const SmemLayout L = smem_layout(a.c, a.k, kPerChannel ? 0 : lut_size, a.chunk_pixels, S, a.smem_budget);
+    const int slots = L.slots, panel_k = L.panel_k;
+    const uint32_t slot_bytes = L.slot_bytes;
     unsigned char *s_basis = smem + L.basis;
     uint32_t *s_lut = reinterpret_cast<uint32_t *>(smem + L.lut);
-    float *s_bias = reinterpret_cast<float *>(smem + L.bias);
     const uint32_t ring_addr = smem_u32(smem + L.ring);
     const uint32_t basis_addr = smem_u32(s_basis);
     const uint32_t lut_addr = smem_u32(s_lut);
-    const int n_panels = (a.k + kPanelK - 1) / kPanelK;
+    const int k_sub = a.k / S;                   // coefficients per chunk of one pixel
+    const int n_panels = (k_sub + panel_k - 1) / panel_k;       // panels per half (S = 2) or per pixel
 
     // ---- set-up ---------------------------------------------------------------------
     if (tid == 0) {
         for (int g = 0; g < 2; ++g) {
-            for (int s = 0; s < kMaxStages; ++s) { mbar_init(smem_u32(&s_full[g][s]), 128); mbar_init(smem_u32(&s_empty[g][s]), 1); }
+            for (int s = 0; s < kMaxSlots; ++s) { mbar_init(smem_u32(&s_full[g][s]), 128); mbar_init(smem_u32(&s_empty[g][s]), 1); }
             mbar_init(smem_u32(&s_tfull[g]), 1);
             mbar_init(smem_u32(&s_tempty[g]), 256);
         }
         mbar_fence_init();
     }
-    if (warp == 16) { tmem_alloc(smem_u32(&s_tmem_base), kTmemCols); tmem_relinquish(); }
+    if (warp == kMmaWarp0) { tmem_alloc(smem_u32(&s_tmem_base), kTmemCols); tmem_relinquish(); }
     {
         // transposed basis [c][j] -> K-major core matrices: (c/8)*sbo + (j/8)*128 + (c%8)*16 + (j%8)*2
         const uint32_t sbo = (uint32_t)(a.k / 8) * 128u;
         const int chunks_per_row = a.k / 8;
         const uint4 *src = reinterpret_cast<const uint4 *>(a.basis_t_bf16);
-        for (int i = tid; i < a.c * chunks_per_row; i += kThreads) {
+        const int c_pad = ((a.c + 127) / 128) * 128;         // rows past C are zero: their outputs are never stored
+        for (int i = tid; i < c_pad * chunks_per_row; i += kThreads) {
             const int ch = i / chunks_per_row, j8 = i - ch * chunks_per_row;
-            *reinterpret_cast<uint4 *>(s_basis + (ch >> 3) * sbo + j8 * 128 + (ch & 7) * 16) = __ldg(src + i);
+            *reinterpret_cast<uint4 *>(s_basis + (ch >> 3) * sbo + j8 * 128 + (ch & 7) * 16) =
+                ch < a.c ? __ldg(src + i) : make_uint4(0u, 0u, 0u, 0u);
         }
-        for (int i = tid; i < a.c; i += kThreads) s_bias[i] = a.dec_bias[i];
         if (!kPerChannel)
-            for (int i = tid; i < pair_size; i += kThreads) {
-                // pair table entry: x = bf16(symbol0 - center) | bf16(symbol1 - center) << 16,
-                //                   y = bits consumed | symbols decoded << 8 | length of the first code << 16
-                const uint2 e = a.lut_pair[i];
-                const float f0 = (float)((int)(e.x & 0xffu) - a.center), f1 = (float)((int)((e.x >> 8) & 0xffu) - a.center);
-                s_lut[2 * i] = (__float_as_uint(f0) >> 16) | (__float_as_uint(f1) & 0xffff0000u);
-                s_lut[2 * i + 1] = e.y;
+            for (int i = tid; i < lut_size; i += kThreads) {
+                // per-layer table: bf16(symbol - center) << 16 | code length
+                const uint32_t e = a.lut32[i];
+                const float f = (float)((int)((e >> 8) & 0xffu) - a.center);
+                s_lut[i] = (__float_as_uint(f) & 0xffff0000u) | (e & 0xffu);
             }
     }
     fence_proxy_async_smem();
@@ -238,21 +320,31 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
 
     const long long my_tiles = (a.n_tiles > blockIdx.x) ? (a.n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
 
-    if (warp < 8) {
+    if (warp < kVldWarps) {
         // ================= VLD groups =================
-        const int grp = warp >> 2;
-        const int t = tid & 127;
+        const int grp = warp >> 3;
+        const int tg = tid & 255;                // thread within the group
+        const int sub = S == 2 ? (tg >> 7) : 0;  // which half of the coefficients (warp-uniform)
+        const int t = tg & 127;                  // S = 2: pixel within the tile; S = 1: chunk within the tile
+        const int wq = t >> 5;
         const int cp = a.chunk_pixels;
-        const int chunks_per_tile = TC_TILE_PIXELS / cp;
-        const uint32_t ring_g = ring_addr + (uint32_t)grp * stages * kStageBytes;
+        const int chunks_per_tile = S * TC_TILE_PIXELS / cp;
+        const int n_thr = 128 * S;               // working threads of the group
+        const bool working = tg < n_thr;
+        const uint32_t ring_g = ring_addr + (uint32_t)grp * slots * slot_bytes;
         const uint32_t sbuf_bytes = L.stream_buf;
         const uint32_t sbuf_g = smem_u32(smem + L.sbuf) + (uint32_t)grp * 2u * sbuf_bytes;
         const int bar_id = 1 + grp;
-        long long it = 0;                       // panels produced by this group so far
+        const int sub_slots = S == 2 ? 2 : slots; // ring slots of this thread's half
+        // ring position of this thread's half at the start of a tile: slot and phase parity of
+        // the next panel (kept incrementally: a division per panel would cost more than the decode)
+        int slot0 = 0;
+        uint32_t phase0 = 0;
         bool alive = true;
 
-        // offsets of a tile, validated; a tile that cannot be valid decodes nothing
-        struct TileInfo { unsigned long long base, bits; bool ok, staged; unsigned int chunk_off; };
+        // offsets of a tile, validated; a tile that cannot be valid decodes nothing.  `lens` holds
+        // the chunk length(s) of this thread's pixel: both halves (S = 2) or the one chunk.
+        struct TileInfo { unsigned long long base, bits; bool ok, staged; unsigned int lens; };
         auto tile_info = [&](long long tl) {
             TileInfo ti{0, 0, false, false, 0};
             if (tl >= my_tiles) return ti;
@@ -263,9 +355,14 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
             ti.base = base;
             ti.bits = end - base;
             ti.staged = sbuf_bytes != 0 && ti.bits <= (unsigned long long)sbuf_bytes * 8ull &&
-                        (cp * a.k * TC_MAX_CODE_LEN) / 8 + 16 <= kStreamSlack;
-            const long long ch = tile * chunks_per_tile + t;
-            if (t < chunks_per_tile && ch < a.n_chunks) ti.chunk_off = a.chunk_off[ch];
+                        (cp * k_sub * TC_MAX_CODE_LEN) / 8 + 16 <= kStreamSlack;
+            if (S == 2) {
+                const long long ch = tile * chunks_per_tile + 2 * t;     // even: both lengths in one aligned word
+                if (ch < a.n_chunks) ti.lens = *reinterpret_cast<const unsigned int *>(a.chunk_len + ch);
+            } else {
+                const long long ch = tile * chunks_per_tile + t;
+                if (t < chunks_per_tile && ch < a.n_chunks) ti.lens = a.chunk_len[ch];
+            }
             return ti;
         };
         // start the copy of a tile's segment into stream buffer `which` (16 bytes per cp.async)
@@ -274,54 +371,82 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
                 const uint32_t dst = sbuf_g + (uint32_t)which * sbuf_bytes;
                 const unsigned char *src = reinterpret_cast<const unsigned char *>(a.stream) + (ti.base >> 3);
                 const uint32_t n16 = (uint32_t)(ti.bits >> 7);
-                for (uint32_t i = t; i < n16; i += 128) cp_async_16(dst + i * 16u, src + (size_t)i * 16u, 16u);
+                for (uint32_t i = tg; i < n16; i += n_thr) cp_async_16(dst + i * 16u, src + (size_t)i * 16u, 16u);
             }
             cp_async_commit();
         };
 
-        TileInfo cur = tile_info(grp), nxt = tile_info(grp + 2);
-        stage_tile(cur, 0);
+        // (with one chunk per pixel or fewer, warps 4-7 of a group have nothing to do)
+        TileInfo cur{0, 0, false, false, 0}, nxt = cur;
+        if (working) {
+            cur = tile_info(grp);
+            nxt = tile_info(grp + 2);
+            stage_tile(cur, 0);
+        }
         int li = 0;
-        for (long long tl = grp; tl < my_tiles && alive; tl += 2, ++li) {
+        for (long long tl = grp; tl < my_tiles && alive && working; tl += 2, ++li) {
             const long long tile = blockIdx.x + tl * gridDim.x;
             stage_tile(nxt, (li + 1) & 1);           // its buffer was released by the barrier that ended tile li - 1
             cp_async_wait<1>();
-            named_bar_sync(bar_id, 128);             // every thread's part of this tile's segment has landed
+            // start of every chunk = sum of the lengths before it in the tile (chunk order: pixel,
+            // then half): scan over the pixels' totals; both halves of a group compute the same scan
+            const unsigned int len0 = S == 2 ? (cur.lens & 0xffffu) : cur.lens, len1 = S == 2 ? (cur.lens >> 16) : 0u;
+            const unsigned int tot = len0 + len1;
+            unsigned int inc = tot;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const unsigned int up = __shfl_up_sync(0xffffffffu, inc, d);
+                if (lane >= d) inc += up;
+            }
+            if (lane == 31) s_wsum[grp][sub][wq] = inc;
+            named_bar_sync(bar_id, n_thr);           // every thread's part of this tile's segment has landed
             const TileInfo after = tile_info(tl + 4); // offsets two tiles ahead: their latency hides behind the decode
+            unsigned int before = 0, tile_total = 0;
+#pragma unroll
+            for (int w = 0; w < 4; ++w) {
+                const unsigned int sw = s_wsum[grp][sub][w];
+                if (w < wq) before += sw;
+                tile_total += sw;
+            }
+            const unsigned int chunk_start = before + inc - tot + (sub ? len0 : 0u);
+            const unsigned int chunk_bits = sub ? len1 : len0;
 
-            const long long ch = tile * chunks_per_tile + t;
-            bool active = cur.ok && t < chunks_per_tile && ch < a.n_chunks;
-            bool bad = !cur.ok;
-            if (active && (unsigned long long)cur.chunk_off > cur.bits) { bad = true; active = false; }
-            const int n_pix = active ? (int)min((long long)cp, a.pixels - (tile * TC_TILE_PIXELS + (long long)t * cp)) : 0;
+            const long long ch = tile * chunks_per_tile + (S == 2 ? 2 * t + sub : t);
+            bool active = cur.ok && (S == 2 || t < chunks_per_tile) && ch < a.n_chunks;
+            bool bad = !cur.ok || (unsigned long long)tile_total > cur.bits;
+            if (bad) active = false;
+            const int n_pix = active ? (int)min((long long)cp, a.pixels - (tile * TC_TILE_PIXELS + (S == 2 ? (long long)t : (long long)t * cp))) : 0;
             const uint32_t seg_addr = sbuf_g + (uint32_t)(li & 1) * sbuf_bytes;
+            const int k_first = sub * k_sub, k_end = k_first + k_sub;
 
             // walks this thread's chunk; `fill_panel(dst, k0, nk8)` decodes the next 8 * nk8 symbols
             // (coefficients k0 ...) into the operand row at shared address `dst`
-            auto decode_chunk = [&](auto &&fill_panel) {
+            // (`every_lane`: the filler is called by all 32 lanes of the warp, with `store` telling
+            // whether the lane has a pixel to decode -- needed when the filler votes across the warp)
+            auto decode_chunk = [&](auto &&fill_panel, bool every_lane) {
                 for (int pp = 0; pp < cp && alive; ++pp) {
                     const bool decode = pp < n_pix;
-                    const int row = t * cp + pp;       // only meaningful while t < chunks_per_tile
+                    const int row = t * cp + pp;       // only meaningful while the chunk exists
+                    int slot = slot0;
+                    uint32_t phase = phase0;
                     for (int kp = 0; kp < n_panels; ++kp) {
-                        const long long pit = it + kp;
-                        const int s = (int)(pit % stages);
-                        if (pp == 0 && !mbar_wait(smem_u32(&s_empty[grp][s]), (uint32_t)(((pit / stages) & 1) ^ 1))) { alive = false; break; }
-                        if (decode) {
-                            const int k0 = kp * kPanelK;
-                            const int nk8 = min(kPanelK, a.k - k0) >> 3;
-                            const uint32_t dst = ring_g + s * kStageBytes + (row >> 3) * 128 + (row & 7) * 16;
-                            fill_panel(dst, k0, nk8);
+                        const int s = sub * 2 + slot;
+                        if (pp == 0 && !mbar_wait(smem_u32(&s_empty[grp][s]), phase ^ 1u, 200u)) { alive = false; break; }
+                        if (++slot == sub_slots) { slot = 0; phase ^= 1u; }
+                        if (decode || every_lane) {
+                            const int k0 = k_first + kp * panel_k;
+                            const int nk8 = min(panel_k, k_end - k0) >> 3;
+                            const uint32_t dst = ring_g + s * slot_bytes + ((row & 127) >> 3) * 128 + (row & 7) * 16;
+                            fill_panel(dst, k0, nk8, decode);
                         }
-                        if (pp == cp - 1) {
-                            fence_proxy_async_smem();
-                            mbar_arrive(smem_u32(&s_full[grp][s]));
-                        }
+                        // (the issuing thread makes the panel visible to the tensor core's proxy)
+                        if (pp == cp - 1) mbar_arrive(smem_u32(&s_full[grp][s]));
                     }
                 }
             };
             // symbol by symbol: eight symbols -> one 16-byte store
             auto by_pairs = [&](auto &&next_pair) {
-                return [&, next_pair](uint32_t dst, int k0, int nk8) mutable {
+                return [&, next_pair](uint32_t dst, int k0, int nk8, bool) mutable {
                     for (int k8 = 0; k8 < nk8; ++k8) {
                         uint32_t pk[4];
 #pragma unroll
@@ -334,73 +459,49 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
             // table entry: bf16(symbol - center) << 16 | symbol << 8 | length; returns two bf16 values
             auto centre = [&](uint32_t e) { return __float_as_uint((float)((int)((e >> 8) & 0xffu) - a.center)); };
 
-            if (cur.ok && cur.staged) {
-                SmemWindowReader r;
-                if (active) r.init(seg_addr, cur.chunk_off);
-                else { r.hi = r.lo = r.ahead = 0; r.avail = 64; r.next_addr = seg_addr; }
-                auto next_pair = [&](int j) -> uint32_t {
-                    r.refill();
-                    uint32_t e0, e1;
-                    if constexpr (!kPerChannel) {
-                        // both symbols from one lookup when their codes fit a 10-bit window
-                        uint32_t v, meta;
-                        asm("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v), "=r"(meta) : "r"(lut_addr + r.peek(TC_PAIR_LUT_BITS) * 8u));
-                        if (((meta >> 8) & 3u) == 2u) {
-                            r.skip_entry(meta);
-                            return v;
-                        }
-                        // one symbol at a time: the first symbol of a pair entry, or, for the rare
-                        // code longer than the window, the full table in global memory
-                        auto one = [&](uint32_t vv, uint32_t mm) -> uint32_t {
-                            if (((mm >> 8) & 3u) != 0u) {
-                                r.skip_entry(mm >> 16);
-                                return vv << 16;                      // bf16 bits in the upper half, as in lut32
-                            }
-                            const uint32_t e = __ldg(a.lut32 + r.peek(a.lut_bits));
-                            r.skip_entry(e);
-                            return centre(e);
-                        };
-                        const uint32_t h0 = one(v, meta);
-                        asm("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v), "=r"(meta) : "r"(lut_addr + r.peek(TC_PAIR_LUT_BITS) * 8u));
-                        const uint32_t h1 = one(v, meta);
-                        return __byte_perm(h0, h1, 0x7632);
-                    } else {
-                        e0 = __ldg(a.lut32 + (size_t)j * lut_size + r.peek(a.lut_bits));
-                        r.skip_entry(e0);
-                        e1 = __ldg(a.lut32 + (size_t)(j + 1) * lut_size + r.peek(a.lut_bits));
-                        r.skip_entry(e1);
-                    }
-                    return __byte_perm(centre(e0), centre(e1), 0x7632);
-                };
-                if (!kPerChannel && a.run_shift >= 0) {
-                    // The shortest code is all zeros (canonical order), and at low rates it belongs to
-                    // the symbol that nearly every coefficient of the trailing channels takes.  Eight
-                    // such symbols in a row are 8 (or 16) zero bits: one test replaces eight lookups.
-                    const uint32_t fill = a.run_fill;              // bf16(that symbol - center) twice
-                    const int bits8 = 8 << a.run_shift;            // bits of eight shortest codes
-                    decode_chunk([&](uint32_t dst, int k0, int nk8) {
-                        for (int k8 = 0; k8 < nk8; ++k8) {
-                            uint32_t pk[4];
-                            r.refill();
-                            if ((r.hi >> (32 - bits8)) == 0u) {
-                                r.skip_bits(bits8);
-                                pk[0] = pk[1] = pk[2] = pk[3] = fill;
-                            } else {
+            if (!kPerChannel && cur.ok && cur.staged) {
+                // per-layer table in shared memory: one lookup per symbol and no branch, so that the
+                // 32 lanes of a warp stay in step whatever their bits are
+                SmemSymbolReader r;
+                if (active) r.init(seg_addr, chunk_start);
+                else r.idle(seg_addr);
+                const int lb = a.lut_bits;
+                decode_chunk([&](uint32_t dst, int k0, int nk8, bool) {
+                    for (int k8 = 0; k8 < nk8; ++k8) {
+                        uint32_t pk[4];
 #pragma unroll
-                                for (int i = 0; i < 8; i += 2) pk[i >> 1] = next_pair(k0 + k8 * 8 + i);
-                            }
-                            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + k8 * 2048), "r"(pk[0]),
-                                         "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
+                        for (int i = 0; i < 4; ++i) {
+                            r.refill();
+                            const uint32_t e0 = SmemSymbolReader::lds(lut_addr + (r.peek(lb) << 2));
+                            r.take(e0);
+                            const uint32_t e1 = SmemSymbolReader::lds(lut_addr + (r.peek(lb) << 2));
+                            r.take(e1);
+                            pk[i] = __byte_perm(e0, e1, 0x7632);
                         }
-                    });
-                } else {
-                    decode_chunk(by_pairs(next_pair));
-                }
-                if (active && (unsigned long long)cur.chunk_off + r.consumed(seg_addr, cur.chunk_off) > cur.bits) bad = true;
+                        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + k8 * 2048), "r"(pk[0]),
+                                     "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
+                    }
+                }, false);
+                // a chunk must end exactly where its recorded length says
+                if (active && r.consumed(seg_addr, chunk_start) != chunk_bits) bad = true;
+            } else if (cur.ok && cur.staged) {
+                // per-channel tables (global memory), stream from shared memory
+                SmemWindowReader r;
+                if (active) r.init(seg_addr, chunk_start);
+                else { r.hi = r.lo = r.ahead = 0; r.avail = 64; r.next_addr = seg_addr; }
+                decode_chunk(by_pairs([&](int j) -> uint32_t {
+                    r.refill();
+                    const uint32_t e0 = __ldg(a.lut32 + (size_t)j * lut_size + r.peek(a.lut_bits));
+                    r.skip_entry(e0);
+                    const uint32_t e1 = __ldg(a.lut32 + (size_t)(j + 1) * lut_size + r.peek(a.lut_bits));
+                    r.skip_entry(e1);
+                    return __byte_perm(centre(e0), centre(e1), 0x7632);
+                }), false);
+                if (active && r.consumed(seg_addr, chunk_start) != chunk_bits) bad = true;
             } else {
                 WindowReader r;
-                unsigned long long used = cur.base + cur.chunk_off;
-                if (active) r.init(a.stream, used, cur.base + cur.bits);
+                unsigned int used = 0;
+                if (active) r.init(a.stream, cur.base + chunk_start, cur.base + cur.bits);
                 else { r.words = a.stream; r.next = r.end = 0; r.hi = r.lo = 0; r.avail = 64; }
                 decode_chunk(by_pairs([&](int j) -> uint32_t {
                     r.refill();
@@ -411,95 +512,113 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
                     r.skip((int)(e1 & 0xffu));
                     used += (e0 & 0xffu) + (e1 & 0xffu);
                     return __byte_perm(centre(e0), centre(e1), 0x7632);
-                }));
-                if (active && used > cur.base + cur.bits) bad = true;
+                }), false);
+                if (active && used != chunk_bits) bad = true;
             }
-            it += n_panels;
+            for (int kp = 0; kp < n_panels; ++kp)
+                if (++slot0 == sub_slots) { slot0 = 0; phase0 ^= 1u; }
             if (bad) tc_dev_set_status(a.status, TC_ERR_CORRUPT_STREAM);
-            named_bar_sync(bar_id, 128);             // this tile's stream buffer may be refilled
+            named_bar_sync(bar_id, n_thr);           // this tile's stream buffer may be refilled
             cur = nxt;
             nxt = after;
         }
         cp_async_wait<0>();
         if (!alive && t == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
-    } else if (warp < 16) {
+    } else if (warp < kMmaWarp0) {
         // ================= epilogue: all eight warps work on every tile =================
-        // warps 8-11 store the first half of the channels, warps 12-15 the second half, so that an
-        // accumulator is released after half the store time and the VLD group behind it stalls less
-        const int half = (warp - 8) >> 2;
-        const int wq = warp & 3;
-        const int m = wq * 32 + lane;                       // pixel within the tile = TMEM lane
-        const int half_cols = ((a.c + 31) / 32) * 16;
-        const int col0 = half * half_cols;
-        const int ncols = half ? a.c - half_cols : half_cols;   // multiple of 16
+        // A thread owns one channel (its TMEM lane) of one block of 128 channels.  With two
+        // channel blocks warps 16-19 take the first and warps 20-23 the second; with one block
+        // the two warp sets split the tile's pixels (TMEM columns) in halves.
+        const int set = (warp - kEpiWarp0) >> 2;
+        const int wq = warp & 3;                            // TMEM lane quarter of this warp
+        const int n_blocks = (a.c + 127) / 128;
+        const int blk = n_blocks == 2 ? set : 0;
+        const int col_first = n_blocks == 2 ? 0 : 64 * set, col_count = n_blocks == 2 ? 128 : 64;
+        const int ch = blk * 128 + wq * 32 + lane;
+        const bool ch_ok = ch < a.c;
         const float step = (float)a.step;
+        const float bias = ch_ok ? a.dec_bias[ch] : 0.f;
         __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(a.xhat);
         // With H*W a multiple of 4 every aligned group of four pixels lies inside one image and is
-        // 8-byte aligned: 32 channels x 128 pixels are transposed through shared memory and leave
-        // as one 256-byte row per warp store.  Otherwise each lane stores its own 2-byte values.
+        // 8-byte aligned; otherwise pixels are stored one by one.
         const bool vec = (a.hw & 3) == 0;
-        const uint32_t tb_addr = smem_u32(smem + L.tbuf) + (uint32_t)half * kTransposeBytes;
-        const int ebar = 3 + half;
+        const long long img_stride = (long long)a.c * a.hw;
+        const int ch_base = blk * 128 + wq * 32;            // first channel of this warp
+        const int pgrp = lane & 7, r_sub = lane >> 3;
+        const uint32_t tb = smem_u32(smem + L.tbuf) + (uint32_t)(warp - kEpiWarp0) * kTrWarpBytes;
+        const uint32_t tb_wr = tb + (uint32_t)lane * kTrRowBytes;                   // this thread's channel row
+        const uint32_t tb_rd = tb + (uint32_t)r_sub * kTrRowBytes + (uint32_t)pgrp * 8u;
         bool alive = true;
         for (long long tl = 0; tl < my_tiles && alive; ++tl) {
             const int grp = (int)(tl & 1);
             const long long tile = blockIdx.x + tl * gridDim.x;
-            const long long p = tile * TC_TILE_PIXELS + m;
-            const bool valid = p < a.pixels;
-            const long long img = valid ? p / a.hw : 0;
-            __nv_bfloat16 *dst = out + img * a.c * (long long)a.hw + (valid ? p - img * a.hw : 0) + (long long)col0 * a.hw;
-            // the four pixels this lane stores in the transposed phase
-            const long long p4 = tile * TC_TILE_PIXELS + 4 * lane;
-            const bool valid4 = p4 < a.pixels;
-            const long long img4 = valid4 ? p4 / a.hw : 0;
-            __nv_bfloat16 *dst4 = out + img4 * a.c * (long long)a.hw + (valid4 ? p4 - img4 * a.hw : 0) + (long long)col0 * a.hw;
-            if (!mbar_wait(smem_u32(&s_tfull[grp]), (uint32_t)((tl >> 1) & 1))) { alive = false; break; }
+            const long long p_first = tile * TC_TILE_PIXELS + col_first;
+            const long long left = a.pixels - p_first;                       // pixels from this thread's first column on
+            const int n_valid = (int)(left < (long long)col_count ? (left < 0 ? 0 : left) : (long long)col_count);
+            // position of the first pixel; from there on it moves incrementally
+            const long long img0 = left > 0 ? p_first / a.hw : 0;
+            int s = left > 0 ? (int)(p_first - img0 * a.hw) : 0;
+            __nv_bfloat16 *dst = out + img0 * img_stride + (long long)(ch_ok ? ch : 0) * a.hw + s;
+            if (!mbar_wait(smem_u32(&s_tfull[grp]), (uint32_t)((tl >> 1) & 1), 1000u)) { alive = false; break; }
             tc_fence_after_sync();
-            const uint32_t trow = tmem_base + grp * kAccCols + ((uint32_t)(wq * 32) << 16) + col0;
-            for (int c0 = 0; c0 < ncols; c0 += 32) {
-                const int nc = min(32, ncols - c0);            // 32 or 16
-                uint32_t r[32];
-                {
-                    uint32_t r16[16];
-                    tmem_ld_32x32b_x16(trow + c0, r16);
+            const uint32_t trow = tmem_base + grp * kAccCols + blk * 128 + ((uint32_t)(wq * 32) << 16) + col_first;
+            if (vec) {
+                // position of this lane's pixel group (4 pixels) in the first pass
+                const long long pg = p_first + 4 * pgrp;
+                long long img = pg < a.pixels ? pg / a.hw : 0;
+                int sp = pg < a.pixels ? (int)(pg - img * a.hw) : 0;
+                for (int c0 = 0; c0 < col_count; c0 += 32) {
+                    uint32_t r[32];
+                    {
+                        uint32_t r16[16];
+                        tmem_ld_32x32b_x16(trow + c0, r16);
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) r[i] = r16[i];
-                    if (nc == 32) {
+                        for (int i = 0; i < 16; ++i) r[i] = r16[i];
                         tmem_ld_32x32b_x16(trow + c0 + 16, r16);
 #pragma unroll
                         for (int i = 0; i < 16; ++i) r[16 + i] = r16[i];
                     }
-                }
-                tmem_ld_wait();
-                if (vec) {
+                    tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        if (i < nc) {
-                            const float v0 = fmaf(__uint_as_float(r[i]), step, s_bias[col0 + c0 + i]);
-                            const float v1 = fmaf(__uint_as_float(r[i + 1]), step, s_bias[col0 + c0 + i + 1]);
-                            const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
-                            const uint32_t hb = *reinterpret_cast<const uint32_t *>(&h);
-                            asm volatile("st.shared.u16 [%0], %1;" ::"r"(tb_addr + i * 256 + m * 2), "h"((unsigned short)(hb & 0xffffu)) : "memory");
-                            asm volatile("st.shared.u16 [%0], %1;" ::"r"(tb_addr + (i + 1) * 256 + m * 2), "h"((unsigned short)(hb >> 16)) : "memory");
+                    for (int q = 0; q < 4; ++q) {
+                        uint32_t h2[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(fmaf(__uint_as_float(r[8 * q + 2 * i]), step, bias),
+                                                                           fmaf(__uint_as_float(r[8 * q + 2 * i + 1]), step, bias));
+                            h2[i] = *reinterpret_cast<const uint32_t *>(&h);
                         }
+                        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(tb_wr + q * 16), "r"(h2[0]), "r"(h2[1]),
+                                     "r"(h2[2]), "r"(h2[3]) : "memory");
                     }
-                    named_bar_sync(ebar, 128);                 // the block is in shared memory
-                    for (int ch = wq; ch < nc; ch += 4) {      // one channel row of 128 pixels per warp store
+                    __syncwarp();
+                    // read phase: lane -> (row r_sub of every group of four channel rows, pixel group pgrp)
+                    const bool px_ok = c0 + 4 * pgrp < n_valid;
+                    __nv_bfloat16 *row_ptr = out + img * img_stride + (long long)(ch_base + r_sub) * a.hw + sp;
+#pragma unroll
+                    for (int it = 0; it < 8; ++it) {
                         uint32_t lo2, hi2;
-                        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(lo2), "=r"(hi2) : "r"(tb_addr + ch * 256 + lane * 8));
-                        if (valid4) *reinterpret_cast<uint2 *>(dst4 + (long long)(c0 + ch) * a.hw) = make_uint2(lo2, hi2);
+                        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(lo2), "=r"(hi2) : "r"(tb_rd + it * 4 * kTrRowBytes));
+                        if (px_ok && ch_base + 4 * it + r_sub < a.c)
+                            *reinterpret_cast<uint2 *>(row_ptr + (long long)(4 * it) * a.hw) = make_uint2(lo2, hi2);
                     }
-                    named_bar_sync(ebar, 128);                 // the buffer may be overwritten
-                } else if (valid) {
+                    sp += 32;
+                    while (sp >= a.hw) { sp -= a.hw; ++img; }
+                    __syncwarp();                                   // the block may be overwritten
+                }
+            } else {
+                for (int c0 = 0; c0 < col_count; c0 += 16) {
+                    uint32_t r[16];
+                    tmem_ld_32x32b_x16(trow + c0, r);
+                    tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        if (i < nc) {
-                            const float v0 = fmaf(__uint_as_float(r[i]), step, s_bias[col0 + c0 + i]);
-                            const float v1 = fmaf(__uint_as_float(r[i + 1]), step, s_bias[col0 + c0 + i + 1]);
-                            const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
-                            dst[(long long)(c0 + i) * a.hw] = h.x;
-                            dst[(long long)(c0 + i + 1) * a.hw] = h.y;
-                        }
+                    for (int i = 0; i < 16; ++i) {
+                        const __nv_bfloat16 h = __float2bfloat16_rn(fmaf(__uint_as_float(r[i]), step, bias));
+                        if (ch_ok && c0 + i < n_valid) *dst = h;
+                        s += 1;
+                        const bool wrap = s == a.hw;            // the next pixel starts the next image
+                        dst += wrap ? 1 + img_stride - a.hw : 1;
+                        s = wrap ? 0 : s;
                     }
                 }
             }
@@ -509,29 +628,44 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
         if (!alive && lane == 0 && wq == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
     } else {
         // ================= MMA issuers (one per group) =================
-        const int grp = warp - 16;
+        const int grp = warp - kMmaWarp0;
         if (lane == 0) {
-            const uint32_t idesc = make_idesc_bf16(TC_TILE_PIXELS, a.c, /*A K-major*/ false, /*B K-major*/ false);
-            const uint32_t b_sbo = (uint32_t)(a.k / 8) * 128u;
-            const uint32_t ring_g = ring_addr + (uint32_t)grp * stages * kStageBytes;
-            long long it = 0;
+            // A = transposed basis (128 channels per instruction), B = the decoded symbols of 128 pixels
+            const uint32_t idesc = make_idesc_bf16(128, TC_TILE_PIXELS, /*A K-major*/ false, /*B K-major*/ false);
+            const uint32_t a_sbo = (uint32_t)(a.k / 8) * 128u;
+            const int n_blocks = (a.c + 127) / 128;
+            const uint32_t ring_g = ring_addr + (uint32_t)grp * slots * slot_bytes;
+            const int sub_slots = S == 2 ? 2 : slots;
+            int slot = 0;                           // ring position (same for both halves) and its phase parity
+            uint32_t phase = 0;
             bool alive = true;
             for (long long tl = grp; tl < my_tiles && alive; tl += 2) {
-                if (!mbar_wait(smem_u32(&s_tempty[grp]), (uint32_t)(((tl >> 1) & 1) ^ 1))) { alive = false; break; }
+                if (!mbar_wait(smem_u32(&s_tempty[grp]), (uint32_t)(((tl >> 1) & 1) ^ 1), 500u)) { alive = false; break; }
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + grp * kAccCols;
-                for (int kp = 0; kp < n_panels; ++kp, ++it) {
-                    const int s = (int)(it % stages);
-                    if (!mbar_wait(smem_u32(&s_full[grp][s]), (uint32_t)((it / stages) & 1))) { alive = false; break; }
-                    tc_fence_after_sync();
-                    const int k0 = kp * kPanelK;
-                    const int nk16 = min(kPanelK, a.k - k0) >> 4;
-                    for (int q = 0; q < nk16; ++q) {
-                        const uint64_t adesc = make_smem_desc(ring_g + s * kStageBytes + q * 4096, 2048, 128);
-                        const uint64_t bdesc = make_smem_desc(basis_addr + ((k0 + 16 * q) >> 3) * 128, 128, b_sbo);
-                        mma_bf16_ss(d_tmem, adesc, bdesc, idesc, (kp | q) != 0 ? 1u : 0u);
+                uint32_t accumulate = 0;
+                for (int kp = 0; kp < n_panels && alive; ++kp) {
+                    for (int sub = 0; sub < S; ++sub) {
+                        const int s = sub * 2 + slot;
+                        if (!mbar_wait(smem_u32(&s_full[grp][s]), phase, 200u)) { alive = false; break; }
+                        // the panel was written with ordinary stores by threads that have arrived on the
+                        // barrier: one proxy fence here, between that synchronisation and the MMA's
+                        // operand reads, orders them for all 128 writers
+                        fence_proxy_async_smem();
+                        tc_fence_after_sync();
+                        const int k0 = sub * k_sub + kp * panel_k;
+                        const int nk16 = min(panel_k, (sub + 1) * k_sub - k0) >> 4;
+                        for (int q = 0; q < nk16; ++q) {
+                            const uint64_t bdesc = make_smem_desc(ring_g + s * slot_bytes + q * 4096, 2048, 128);
+                            for (int blk = 0; blk < n_blocks; ++blk) {
+                                const uint64_t adesc = make_smem_desc(basis_addr + blk * 16 * a_sbo + ((k0 + 16 * q) >> 3) * 128, 128, a_sbo);
+                                mma_bf16_ss(d_tmem + blk * 128, adesc, bdesc, idesc, accumulate);
+                            }
+                            accumulate = 1u;
+                        }
+                        mma_commit(smem_u32(&s_empty[grp][s]));
                     }
-                    mma_commit(smem_u32(&s_empty[grp][s]));
+                    if (++slot == sub_slots) { slot = 0; phase ^= 1u; }
                 }
                 if (alive) mma_commit(smem_u32(&s_tfull[grp]));
             }
@@ -542,7 +676,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
     // ---- teardown ---------------------------------------------------------------------
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 16) {
+    if (warp == kMmaWarp0) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, kTmemCols);
     }
@@ -553,19 +687,20 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
 bool tc_decode_tc_supported(const tc_ctx *ctx, const DecodeArgs &a)
 {
     if (a.c % 16 != 0 || a.k != a.c || a.c > 256) return false;
+    if (a.splits != 1 && !(a.splits == 2 && a.chunk_pixels == 1 && a.k % 32 == 0)) return false;
     if (a.groups != 1 && a.groups != a.k) return false;
     if (a.lut_bits > TC_MAX_CODE_LEN) return false;
-    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (2 << TC_PAIR_LUT_BITS) : 0, a.chunk_pixels,
-                                     ctx->max_smem_optin - 512);
-    return l.stages > 0;
+    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, a.chunk_pixels,
+                                     a.splits, ctx->max_smem_optin - 512);
+    return l.slots > 0;
 }
 
 tc_status tc_launch_decode_tc(const tc_ctx *ctx, const DecodeArgs &a, cudaStream_t s)
 {
     if (a.n_tiles <= 0) return TC_OK;
-    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (2 << TC_PAIR_LUT_BITS) : 0, a.chunk_pixels,
-                                     ctx->max_smem_optin - 512);
-    if (l.stages == 0) return TC_ERR_UNSUPPORTED;
+    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, a.chunk_pixels,
+                                     a.splits, ctx->max_smem_optin - 512);
+    if (l.slots == 0) return TC_ERR_UNSUPPORTED;
     void (*kernel)(DecodeArgs) = a.groups != 1 ? decode_tc_kernel<true> : decode_tc_kernel<false>;
     DecodeArgs args = a;
     args.smem_budget = ctx->max_smem_optin - 512;

@@ -57,7 +57,7 @@ struct CurrentDevice {
 
 extern "C" tc_status tc_encode_noalloc(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const tc_tensor *x,
                                        const tc_encode_params *params, void *stream_out, size_t capacity,
-                                       uint32_t *chunk_off, uint64_t *tile_off, void *cuda_stream)
+                                       uint16_t *chunk_len, uint64_t *tile_off, void *cuda_stream)
 {
     if (!ctx || !tile_off) return TC_ERR_INVALID_ARG;
     tc_stream_layout lay;
@@ -65,8 +65,8 @@ extern "C" tc_status tc_encode_noalloc(tc_ctx *ctx, const tc_model *m, const tc_
     if (st != TC_OK) return st;
     if (lay.n_tiles > TC_NOALLOC_MAX_TILES) return TC_ERR_UNSUPPORTED;   // tensor too large for the fixed scratch
     const long long pixels = (long long)x->n * x->h * x->w;
-    if (pixels > 0 && (!stream_out || !chunk_off)) return TC_ERR_INVALID_ARG;
-    if (((uintptr_t)stream_out & 15u) != 0) return TC_ERR_INVALID_ARG;
+    if (pixels > 0 && (!stream_out || !chunk_len)) return TC_ERR_INVALID_ARG;
+    if (((uintptr_t)stream_out & 15u) != 0 || ((uintptr_t)chunk_len & 3u) != 0) return TC_ERR_INVALID_ARG;
     CurrentDevice guard(ctx->device);
     if (!guard.ok) return TC_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)cuda_stream;
@@ -83,11 +83,11 @@ extern "C" tc_status tc_encode_noalloc(tc_ctx *ctx, const tc_model *m, const tc_
 
     EncodeArgs a{};
     a.x = x->data; a.n = x->n; a.c = x->c; a.hw = x->h * x->w; a.k = m->k; a.bits = m->bits; a.groups = cb->groups;
-    a.pixels = pixels; a.n_tiles = lay.n_tiles; a.chunk_pixels = lay.chunk_pixels;
+    a.pixels = pixels; a.n_tiles = lay.n_tiles; a.chunk_pixels = lay.chunk_pixels; a.splits = lay.pixel_splits;
     a.basis64 = m->d_basis64; a.mean64 = m->d_mean64; a.lo = m->lo; a.step = m->step;
     a.enc = cb->d_enc; a.stream = (uint32_t *)stream_out;
     a.capacity_bits = (unsigned long long)(capacity & ~(size_t)15) * 8ull;
-    a.chunk_off = chunk_off; a.tile_off = (unsigned long long *)tile_off;
+    a.chunk_len = chunk_len; a.tile_off = (unsigned long long *)tile_off;
     a.dbg_coef = nullptr; a.dbg_sym = nullptr;
     a.ticket = (unsigned int *)scratch;
     a.tile_state = (unsigned long long *)((char *)scratch + kScratchHeader);

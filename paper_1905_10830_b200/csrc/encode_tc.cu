@@ -392,6 +392,20 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
             }
             const unsigned int pixel_off = before + inc - pair;
             const unsigned int my_off = pixel_off + (half ? other : 0u);
+            // end of the chunk that starts at this pixel (chunks of several pixels): the offset of
+            // the pixel chunk_pixels further on, which sits in this warp, or is a sum of warp totals
+            unsigned int chunk_end = 0;
+            if (a.chunk_pixels > 1) {
+                const int cpx = a.chunk_pixels;
+                if (cpx < 32) {
+                    const unsigned int further = __shfl_down_sync(0xffffffffu, pixel_off, cpx);
+                    chunk_end = (lane + cpx < 32) ? further : before + s_warp_sums[grp][wq];
+                } else {
+#pragma unroll
+                    for (int w = 0; w < 4; ++w)
+                        if (w < wq + (cpx >> 5)) chunk_end += s_warp_sums[grp][w];
+                }
+            }
             const unsigned long long padded = ((unsigned long long)tile_bits + 127ull) & ~127ull;
             if (tg == 0) lookback_publish(a.tile_state, tile, padded);
             const bool staged = padded <= (unsigned long long)kStagingBytes * 8ull;
@@ -481,7 +495,15 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
             // hand the tile to the store warp (each thread's arrival releases its own writes)
             mbar_arrive(smem_u32(&s_stg_full[grp]));
             ++n_done;
-            if (valid && half == 0 && (p % a.chunk_pixels) == 0) a.chunk_off[p / a.chunk_pixels] = pixel_off;
+            // chunk lengths (the first half's thread of a pixel writes them)
+            if (valid && half == 0) {
+                if (a.splits == 2)                        // one chunk per half: both lengths in one aligned word
+                    *reinterpret_cast<uint32_t *>(a.chunk_len + 2 * p) = my_bits | (other << 16);
+                else if (a.chunk_pixels == 1)
+                    a.chunk_len[p] = (uint16_t)pair;
+                else if ((p % a.chunk_pixels) == 0)
+                    a.chunk_len[p / a.chunk_pixels] = (uint16_t)(chunk_end - pixel_off);
+            }
         }
         if (!alive) {
             if (tg == 0) { tc_dev_set_status(a.status, TC_ERR_TIMEOUT); s_store_cmd[grp] = 3; }
@@ -503,9 +525,11 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
 bool tc_encode_tc_supported(const tc_ctx *ctx, const EncodeArgs &a)
 {
     if (a.c % 16 != 0 || a.k != a.c || a.c > 256 || a.hw % 4 != 0) return false;
+    // two chunks per pixel must coincide with the two halves the epilogue threads work on
+    if (a.splits != 1 && !(a.splits == 2 && a.k % 32 == 0)) return false;
     if (a.groups != 1 && a.groups != a.k) return false;
     const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.bits) : 0);
-    return (int)l.total + 512 <= ctx->max_smem_optin;
+    return (int)l.total + 512 <= ctx->max_smem_optin;       // leaves room for the static shared variables
 }
 
 tc_status tc_launch_encode_tc(const tc_ctx *ctx, const EncodeArgs &a, cudaStream_t s)

@@ -42,16 +42,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity, uin
 }
 // Wait for the phase with the given parity; gives up after about two seconds and returns
 // false, so that no kernel can spin forever on a barrier that nothing completes.  Between
-// attempts the warp sleeps, so that warps that wait do not compete with warps that work.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+// attempts the warp sleeps for about `sleep_ns`: a polling warp takes issue slots and integer
+// pipe cycles from the warps that work, so a waiter that can afford the extra latency should
+// ask for a long sleep.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t sleep_ns = 100u)
 {
     if (mbar_try_wait(bar, parity, 0u)) return true;
     unsigned long long t0, t1;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
     while (true) {
         for (int i = 0; i < 64; ++i) {
+            __nanosleep(sleep_ns);
             if (mbar_try_wait(bar, parity, 100000u)) return true;
-            __nanosleep(100);
         }
         asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
         if (t1 - t0 > 2000000000ull) return false;

@@ -54,18 +54,25 @@ bool valid_tensor(const tc_tensor *t)
            (t->data != nullptr || t->n == 0);
 }
 
-int default_chunk_pixels(int k)
+// Chunk shape: `cp` pixels per chunk, or `splits` chunks per pixel when cp == 1.  Defaults
+// keep the side information at 16 bits per 128 to 255 symbols (about 0.1 bit per value).
+struct ChunkShape {
+    int cp, splits;
+    long long chunks(long long pixels) const { return splits > 1 ? pixels * splits : (pixels + cp - 1) / cp; }
+};
+
+bool resolve_chunks(const tc_encode_params *p, int k, int max_len, ChunkShape *out)
 {
     int cp = 1;
-    while (cp < TC_TILE_PIXELS && cp * k < 256) cp <<= 1;
-    return cp;
-}
-
-bool resolve_chunk_pixels(const tc_encode_params *p, int k, int *out)
-{
-    int cp = (p && p->chunk_pixels) ? p->chunk_pixels : default_chunk_pixels(k);
+    if (p && p->chunk_pixels) cp = p->chunk_pixels;
+    else while (cp < TC_TILE_PIXELS && cp * k < 128) cp <<= 1;
     if (cp < 1 || cp > TC_TILE_PIXELS || (cp & (cp - 1)) != 0) return false;
-    *out = cp;
+    int splits = (p && p->pixel_splits) ? p->pixel_splits : ((cp == 1 && k >= 256 && k % 32 == 0) ? 2 : 1);
+    if (splits != 1 && splits != 2 && splits != 4) return false;
+    if (splits > 1 && (cp != 1 || k % (8 * splits) != 0)) return false;
+    if ((long long)cp * k / splits * max_len > 65535) return false;     // a chunk length has 16 bits
+    out->cp = cp;
+    out->splits = splits;
     return true;
 }
 
@@ -124,9 +131,6 @@ tc_status finish_codebook(tc_codebook *cb)
     for (uint8_t l : cb->lengths) mx = std::max<int>(mx, l);
     cb->max_len = mx;
     cb->lut_bits = mx;
-    cb->min_len = 255;
-    for (int v = 0; v < nsym; ++v)
-        if (cb->lengths[v] < cb->min_len) { cb->min_len = cb->lengths[v]; cb->min_len_symbol = v; }
     std::vector<uint32_t> enc((size_t)cb->groups * nsym);
     std::vector<uint16_t> lut((size_t)cb->groups << cb->lut_bits);
     std::vector<uint32_t> lut32((size_t)cb->groups << cb->lut_bits);
@@ -151,31 +155,6 @@ tc_status finish_codebook(tc_codebook *cb)
     tc_status st;
     if ((st = upload(&cb->d_enc, enc)) != TC_OK) return st;
     if ((st = upload(&cb->d_lut32, lut32)) != TC_OK) return st;
-    if (cb->groups == 1) {
-        // Two symbols per lookup: for every 10-bit window, x = symbol0 | symbol1 << 8 and
-        // y = bits consumed | count << 8 | length of the first code << 16, count = 2 if both codes
-        // lie inside the window, 1 if only the first does, 0 if not even the first.
-        const int wb = TC_PAIR_LUT_BITS;
-        auto first_symbol = [&](uint32_t window) -> uint32_t {       // window: wb bits, left-aligned codes
-            const uint32_t idx = cb->lut_bits >= wb ? window << (cb->lut_bits - wb) : window >> (wb - cb->lut_bits);
-            return lut32[idx];
-        };
-        std::vector<uint2> pair((size_t)1 << wb);
-        for (uint32_t win = 0; win < (1u << wb); ++win) {
-            const uint32_t e0 = first_symbol(win);
-            const uint32_t l0 = e0 & 0xffu, s0 = (e0 >> 8) & 0xffu;
-            uint2 v = make_uint2(0u, 0u);
-            if (l0 <= (uint32_t)wb) {
-                const uint32_t rest = (win << l0) & ((1u << wb) - 1u);
-                const uint32_t e1 = first_symbol(rest);
-                const uint32_t l1 = e1 & 0xffu, s1 = (e1 >> 8) & 0xffu;
-                if (l0 + l1 <= (uint32_t)wb) v = make_uint2(s0 | (s1 << 8), (l0 + l1) | (2u << 8) | (l0 << 16));
-                else v = make_uint2(s0, l0 | (1u << 8) | (l0 << 16));
-            }
-            pair[win] = v;
-        }
-        if ((st = upload(&cb->d_lut_pair, pair)) != TC_OK) return st;
-    }
     return upload(&cb->d_lut, lut);
 }
 
@@ -456,7 +435,6 @@ void tc_codebook_free(tc_codebook *cb)
     cudaFree(cb->d_enc);
     cudaFree(cb->d_lut);
     cudaFree(cb->d_lut32);
-    cudaFree(cb->d_lut_pair);
     delete cb;
 }
 
@@ -478,31 +456,32 @@ tc_status tc_encode_bound(const tc_model *m, const tc_codebook *cb, const tc_ten
     if (!out) return TC_ERR_INVALID_ARG;
     tc_status st = check_codec_args(m, cb, x);
     if (st != TC_OK) return st;
-    int cp;
-    if (!resolve_chunk_pixels(params, m->k, &cp)) return TC_ERR_INVALID_ARG;
+    ChunkShape cs;
+    if (!resolve_chunks(params, m->k, cb->max_len, &cs)) return TC_ERR_INVALID_ARG;
     const long long pixels = (long long)x->n * x->h * x->w;
     out->n_tiles = (pixels + TC_TILE_PIXELS - 1) / TC_TILE_PIXELS;
-    out->n_chunks = (pixels + cp - 1) / cp;
+    out->n_chunks = cs.chunks(pixels);
     const unsigned long long tile_bits = (unsigned long long)TC_TILE_PIXELS * m->k * cb->max_len;   // multiple of 128
     out->stream_bytes = (size_t)((unsigned long long)out->n_tiles * tile_bits / 8);
-    out->chunk_off_bytes = (size_t)out->n_chunks * 4;
+    out->chunk_len_bytes = (size_t)out->n_chunks * 2;
     out->tile_off_bytes = (size_t)(out->n_tiles + 1) * 8;
-    out->chunk_pixels = cp;
+    out->chunk_pixels = cs.cp;
+    out->pixel_splits = cs.splits;
     return TC_OK;
 }
 
 tc_status tc_encode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const tc_tensor *x,
-                    const tc_encode_params *params, void *stream_out, size_t capacity, uint32_t *chunk_off,
+                    const tc_encode_params *params, void *stream_out, size_t capacity, uint16_t *chunk_len,
                     uint64_t *tile_off, const tc_debug_out *debug, void *cuda_stream)
 {
     if (!ctx || !tile_off) return TC_ERR_INVALID_ARG;
     tc_status st = check_codec_args(m, cb, x);
     if (st != TC_OK) return st;
-    int cp;
-    if (!resolve_chunk_pixels(params, m->k, &cp)) return TC_ERR_INVALID_ARG;
+    ChunkShape cs;
+    if (!resolve_chunks(params, m->k, cb->max_len, &cs)) return TC_ERR_INVALID_ARG;
     const long long pixels = (long long)x->n * x->h * x->w;
-    if (pixels > 0 && (!stream_out || !chunk_off)) return TC_ERR_INVALID_ARG;
-    if (((uintptr_t)stream_out & 15u) != 0) return TC_ERR_INVALID_ARG;
+    if (pixels > 0 && (!stream_out || !chunk_len)) return TC_ERR_INVALID_ARG;
+    if (((uintptr_t)stream_out & 15u) != 0 || ((uintptr_t)chunk_len & 3u) != 0) return TC_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     cudaStream_t s = (cudaStream_t)cuda_stream;
     const long long n_tiles = (pixels + TC_TILE_PIXELS - 1) / TC_TILE_PIXELS;
@@ -516,11 +495,11 @@ tc_status tc_encode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
 
     EncodeArgs a{};
     a.x = x->data; a.n = x->n; a.c = x->c; a.hw = x->h * x->w; a.k = m->k; a.bits = m->bits; a.groups = cb->groups;
-    a.pixels = pixels; a.n_tiles = n_tiles; a.chunk_pixels = cp;
+    a.pixels = pixels; a.n_tiles = n_tiles; a.chunk_pixels = cs.cp; a.splits = cs.splits;
     a.basis64 = m->d_basis64; a.mean64 = m->d_mean64; a.lo = m->lo; a.step = m->step;
     a.enc = cb->d_enc; a.stream = (uint32_t *)stream_out;
     a.capacity_bits = (unsigned long long)(capacity & ~(size_t)15) * 8ull;
-    a.chunk_off = chunk_off; a.tile_off = (unsigned long long *)tile_off;
+    a.chunk_len = chunk_len; a.tile_off = (unsigned long long *)tile_off;
     a.dbg_coef = debug ? debug->coefficients : nullptr;
     a.dbg_sym = debug ? debug->symbols : nullptr;
     a.ticket = (unsigned int *)ctx->scratch;
@@ -536,34 +515,28 @@ tc_status tc_encode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
 }
 
 tc_status tc_decode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const void *stream, size_t stream_bytes,
-                    const uint32_t *chunk_off, const uint64_t *tile_off, const tc_encode_params *params,
+                    const uint16_t *chunk_len, const uint64_t *tile_off, const tc_encode_params *params,
                     const tc_tensor *x_hat, void *cuda_stream)
 {
     if (!ctx) return TC_ERR_INVALID_ARG;
     tc_status st = check_codec_args(m, cb, x_hat);
     if (st != TC_OK) return st;
-    int cp;
-    if (!resolve_chunk_pixels(params, m->k, &cp)) return TC_ERR_INVALID_ARG;
+    ChunkShape cs;
+    if (!resolve_chunks(params, m->k, cb->max_len, &cs)) return TC_ERR_INVALID_ARG;
     const long long pixels = (long long)x_hat->n * x_hat->h * x_hat->w;
     if (pixels == 0) return TC_OK;
-    if (!stream || !chunk_off || !tile_off || ((uintptr_t)stream & 15u) != 0) return TC_ERR_INVALID_ARG;
+    if (!stream || !chunk_len || !tile_off || ((uintptr_t)stream & 15u) != 0 || ((uintptr_t)chunk_len & 3u) != 0)
+        return TC_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     DecodeArgs a{};
     a.stream = (const uint32_t *)stream; a.stream_bits = (unsigned long long)(stream_bytes & ~(size_t)3) * 8ull;
-    a.chunk_off = chunk_off; a.tile_off = (const unsigned long long *)tile_off; a.symbols = nullptr;
+    a.chunk_len = chunk_len; a.splits = cs.splits; a.tile_off = (const unsigned long long *)tile_off; a.symbols = nullptr;
     a.n = x_hat->n; a.c = x_hat->c; a.hw = x_hat->h * x_hat->w; a.k = m->k; a.bits = m->bits; a.groups = cb->groups;
-    a.pixels = pixels; a.n_tiles = (pixels + TC_TILE_PIXELS - 1) / TC_TILE_PIXELS; a.n_chunks = (pixels + cp - 1) / cp;
-    a.chunk_pixels = cp; a.lut_bits = cb->lut_bits; a.lut = cb->d_lut;
+    a.pixels = pixels; a.n_tiles = (pixels + TC_TILE_PIXELS - 1) / TC_TILE_PIXELS; a.n_chunks = cs.chunks(pixels);
+    a.chunk_pixels = cs.cp; a.lut_bits = cb->lut_bits; a.lut = cb->d_lut;
     a.basis64 = m->d_basis64; a.mean64 = m->d_mean64; a.lo = m->lo; a.step = m->step;
     a.xhat = x_hat->data; a.status = ctx->d_status;
-    a.lut32 = cb->d_lut32; a.lut_pair = cb->d_lut_pair; a.basis_t_bf16 = m->d_basis_t_bf16; a.dec_bias = m->d_dec_bias; a.center = m->center;
-    a.run_shift = (cb->groups == 1 && cb->min_len <= 2) ? cb->min_len - 1 : -1;
-    {
-        const __nv_bfloat16 f = __float2bfloat16((float)(cb->min_len_symbol - m->center));
-        unsigned short raw;
-        std::memcpy(&raw, &f, 2);
-        a.run_fill = ((unsigned int)raw << 16) | raw;
-    }
+    a.lut32 = cb->d_lut32; a.basis_t_bf16 = m->d_basis_t_bf16; a.dec_bias = m->d_dec_bias; a.center = m->center;
     if (!ctx->force_exact && x_hat->dtype == TC_BF16 && tc_decode_tc_supported(ctx, a)) {
         ctx->last_decode_path = 1;
         return tc_launch_decode_tc(ctx, a, (cudaStream_t)cuda_stream);
@@ -589,7 +562,7 @@ tc_status tc_roundtrip_host(tc_ctx *ctx, const tc_model *m, const tc_codebook *c
     const size_t bytes = (size_t)n * c * h * w * elem;
     auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
     const size_t off_xhat = up(bytes), off_stream = off_xhat + up(bytes), off_chunk = off_stream + up(lay.stream_bytes),
-                 off_tile = off_chunk + up(lay.chunk_off_bytes), total = off_tile + up(lay.tile_off_bytes);
+                 off_tile = off_chunk + up(lay.chunk_len_bytes), total = off_tile + up(lay.tile_off_bytes);
     if (total > ctx->host_arena_bytes) {
         if (ctx->host_arena) { TC_CUDA(cudaDeviceSynchronize()); cudaFree(ctx->host_arena); ctx->host_arena = nullptr; ctx->host_arena_bytes = 0; }
         TC_CUDA(cudaMalloc(&ctx->host_arena, total));
@@ -598,10 +571,10 @@ tc_status tc_roundtrip_host(tc_ctx *ctx, const tc_model *m, const tc_codebook *c
     char *base = (char *)ctx->host_arena;
     tc_tensor xd{base, n, c, h, w, dtype}, xh{base + off_xhat, n, c, h, w, dtype};
     TC_CUDA(cudaMemcpyAsync(xd.data, x_host, bytes, cudaMemcpyHostToDevice, s));
-    st = tc_encode(ctx, m, cb, &xd, params, base + off_stream, lay.stream_bytes, (uint32_t *)(base + off_chunk),
+    st = tc_encode(ctx, m, cb, &xd, params, base + off_stream, lay.stream_bytes, (uint16_t *)(base + off_chunk),
                    (uint64_t *)(base + off_tile), nullptr, s);
     if (st != TC_OK) return st;
-    st = tc_decode(ctx, m, cb, base + off_stream, lay.stream_bytes, (const uint32_t *)(base + off_chunk),
+    st = tc_decode(ctx, m, cb, base + off_stream, lay.stream_bytes, (const uint16_t *)(base + off_chunk),
                    (const uint64_t *)(base + off_tile), params, &xh, s);
     if (st != TC_OK) return st;
     TC_CUDA(cudaMemcpyAsync(x_hat_host, xh.data, bytes, cudaMemcpyDeviceToHost, s));
@@ -647,7 +620,7 @@ tc_status tc_stats(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const 
 
     EncodeArgs e{};
     e.x = x->data; e.n = x->n; e.c = x->c; e.hw = x->h * x->w; e.k = m->k; e.bits = m->bits; e.groups = 1;
-    e.pixels = pixels; e.n_tiles = (pixels + TC_TILE_PIXELS - 1) / TC_TILE_PIXELS; e.chunk_pixels = 1;
+    e.pixels = pixels; e.n_tiles = (pixels + TC_TILE_PIXELS - 1) / TC_TILE_PIXELS; e.chunk_pixels = 1; e.splits = 1;
     e.basis64 = m->d_basis64; e.mean64 = m->d_mean64; e.lo = m->lo; e.step = m->step;
     e.enc = nullptr; e.dbg_sym = d_sym; e.status = ctx->d_status; e.clamped = d_clamped; e.emit = 0;
     e.bits = m->bits;
@@ -659,7 +632,7 @@ tc_status tc_stats(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const 
 
     DecodeArgs d{};
     d.symbols = d_sym; d.n = x->n; d.c = x->c; d.hw = x->h * x->w; d.k = m->k; d.bits = m->bits; d.groups = 1;
-    d.pixels = pixels; d.n_tiles = e.n_tiles; d.n_chunks = pixels; d.chunk_pixels = 1;
+    d.pixels = pixels; d.n_tiles = e.n_tiles; d.n_chunks = pixels; d.chunk_pixels = 1; d.splits = 1;
     d.basis64 = m->d_basis64; d.mean64 = m->d_mean64; d.lo = m->lo; d.step = m->step;
     d.xhat = d_xhat; d.status = ctx->d_status;
     if ((st = tc_launch_decode_simt(ctx, d, x->dtype, s)) != TC_OK) return st;

@@ -12,7 +12,6 @@
 constexpr int TC_TILE_PIXELS = 128;   // pixels per tile = threads per epilogue group
 constexpr int TC_MAX_C = 1024;
 constexpr int TC_MAX_CODE_LEN = 12;   // longest code the decode lookup table covers
-constexpr int TC_PAIR_LUT_BITS = 10;  // window of the two-symbol decode table
 
 // Device status word: first error wins.
 __device__ __forceinline__ void tc_dev_set_status(unsigned int *status, unsigned int code)
@@ -52,13 +51,11 @@ struct tc_model {
 
 struct tc_codebook {
     int bits = 0, groups = 0, max_len = 0, lut_bits = 0;
-    int min_len = 0, min_len_symbol = 0;    // shortest code of table 0 and its (lowest) symbol: the all-zero code
     std::vector<uint8_t> lengths;           // host [groups][2^bits]
     int device = 0;
     uint32_t *d_enc = nullptr;              // [groups][2^bits]  (code << 8) | length
     uint16_t *d_lut = nullptr;              // [groups][2^lut_bits]  (symbol << 8) | length
     uint32_t *d_lut32 = nullptr;            // [groups][2^lut_bits]  bf16(symbol) << 16 | symbol << 8 | length
-    uint2 *d_lut_pair = nullptr;            // per-layer tables: [1024] two symbols per 10-bit window (see tc_api.cu)
 };
 
 // ---- kernel argument blocks -------------------------------------------------------------
@@ -69,6 +66,7 @@ struct EncodeArgs {
     long long pixels;
     long long n_tiles;
     int chunk_pixels;
+    int splits;                 // chunks per pixel (1, 2 or 4; more than 1 only with chunk_pixels == 1)
     const double *basis64;      // [c][c]
     const double *mean64;       // [c]
     const __nv_bfloat16 *basis_bf16;   // [k][c]  (tensor-core path)
@@ -78,7 +76,7 @@ struct EncodeArgs {
     const uint32_t *enc;        // [groups][2^bits]
     uint32_t *stream;           // output words
     unsigned long long capacity_bits;
-    uint32_t *chunk_off;
+    uint16_t *chunk_len;        // bits of every chunk
     unsigned long long *tile_off;
     float *dbg_coef;            // nullable
     uint8_t *dbg_sym;           // nullable
@@ -92,7 +90,8 @@ struct EncodeArgs {
 struct DecodeArgs {
     const uint32_t *stream;
     unsigned long long stream_bits;
-    const uint32_t *chunk_off;
+    const uint16_t *chunk_len;          // bits of every chunk
+    int splits;                         // chunks per pixel (1, 2 or 4)
     const unsigned long long *tile_off;
     const uint8_t *symbols;     // non-null: take symbols from here instead of the stream
     int n, c, hw, k, bits, groups;
@@ -102,13 +101,10 @@ struct DecodeArgs {
     int lut_bits;
     const uint16_t *lut;
     const uint32_t *lut32;              // tensor-core path
-    const uint2 *lut_pair;              // tensor-core path, per-layer tables: two symbols per lookup
     const __nv_bfloat16 *basis_t_bf16;  // [c][k]
     const float *dec_bias;              // [c]
     int center;                         // subtracted from every symbol before the MMA
     int smem_budget;                    // shared memory the tensor-core kernel may lay out (set by its launcher)
-    int run_shift;                      // per-layer table whose shortest code has 1 or 2 bits: that length - 1; else -1
-    unsigned int run_fill;              // bf16(symbol of the shortest code - center), twice
     const double *basis64;
     const double *mean64;
     double lo, step;

@@ -62,10 +62,11 @@ def _parity(ctx, model, cb, x_sample, bits, per_channel):
     coef_err = float(np.max(np.abs(y_gpu - y) / np.maximum(np.abs(y), m.step)))
     bad = q_gpu != q
     ties_only = bool(np.all(np.abs(units[bad] - np.floor(units[bad]) - 0.5) <= 1e-3)) if bad.any() else True
-    cp = enc.layout.chunk_pixels
-    ref = oracle.encode(q_gpu, lengths, bits, chunk_pixels=cp, tile_chunks=128 // cp)
+    ref = oracle.encode(q_gpu, lengths, bits, chunk_pixels=enc.layout.chunk_pixels,
+                        pixel_splits=enc.layout.pixel_splits, tile_pixels=128)
     words = enc.words[: enc.total_bits() // 8].cpu().numpy().view(np.uint32)
-    stream_exact = bool(np.array_equal(words, ref.words))
+    lens = enc.chunk_len[: enc.layout.n_chunks].cpu().numpy().view(np.uint16)
+    stream_exact = bool(np.array_equal(words, ref.words) and np.array_equal(lens, ref.chunk_len))
     want = oracle.reconstruct(m, q_gpu, x_sample.shape, out_bf16=(dtype == torch.bfloat16))
     got = xhat.float().cpu().numpy()
     return dict(stream_exact=stream_exact, coef_err=coef_err, mismatch=float(bad.mean()), ties_only=ties_only,
@@ -96,7 +97,7 @@ def run(cfgs, reps, with_oracle, max_batch):
                 t_enc = _time(lambda: tc.tc_encode(ctx, model, cb, x, out=enc), reps)
                 t_dec = _time(lambda: tc.tc_decode(ctx, model, cb, enc, x.shape, x.dtype, out=xhat, stream_bytes=nbytes), reps)
                 assert tc.tc_get_status(ctx) == 0
-                side = enc.layout.chunk_off_bytes + enc.layout.tile_off_bytes
+                side = enc.layout.chunk_len_bytes + enc.layout.tile_off_bytes
                 algo = raw + nbytes + side
                 tst = tc.tc_stats(ctx, model, cb, x[: min(batch, 64)], groups=groups, want_hist=False)
                 row = dict(cfg=cfg, layer=spec.name + (f" x{repeat}" if repeat > 1 else ""), batch=batch, dtype=str(w.dtype).split(".")[-1],

@@ -42,8 +42,8 @@ def stream_words(enc) -> np.ndarray:
     return enc.words[: total // 8].cpu().numpy().view(np.uint32)
 
 
-def chunk_off(enc) -> np.ndarray:
-    return enc.chunk_off[: enc.layout.n_chunks].cpu().numpy().view(np.uint32)
+def chunk_len(enc) -> np.ndarray:
+    return enc.chunk_len[: enc.layout.n_chunks].cpu().numpy().view(np.uint16)
 
 
 def tile_off(enc) -> np.ndarray:

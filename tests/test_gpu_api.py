@@ -111,6 +111,12 @@ def test_argument_errors(ctx):
     assert err.value.code == 2
     with pytest.raises(tc.TcError):                          # chunk size not a power of two
         tc.tc_encode(ctx, m, cb, x, chunk_pixels=3)
+    with pytest.raises(tc.TcError):                          # a pixel is split only when a chunk is one pixel
+        tc.tc_encode(ctx, m, cb, x, chunk_pixels=2, pixel_splits=2)
+    with pytest.raises(tc.TcError):                          # 16 coefficients do not split in four runs of 8
+        tc.tc_encode(ctx, m, cb, x, chunk_pixels=1, pixel_splits=4)
+    with pytest.raises(tc.TcError):                          # three splits
+        tc.tc_encode(ctx, m, cb, x, chunk_pixels=1, pixel_splits=3)
     bad = o["lengths"].copy()
     bad[0, 0] += 1                                           # breaks Kraft's equality
     with pytest.raises(tc.TcError):
@@ -162,17 +168,18 @@ def test_corrupt_streams_are_reported_without_faults(ctx):
     assert tc.tc_get_status(ctx) == 5
     # (b) tile offset beyond the stream / not aligned / decreasing
     for bad_value in (nbytes * 8 + 128, 64, -128):
-        broken = tc.EncodedStream(enc.words, enc.chunk_off, enc.tile_off.clone(), enc.layout)
+        broken = tc.EncodedStream(enc.words, enc.chunk_len, enc.tile_off.clone(), enc.layout)
         broken.tile_off[1] = broken.tile_off[1] + bad_value if bad_value != 64 else 64
         tc.tc_decode(ctx, m, cb, broken, x.shape, x.dtype, stream_bytes=nbytes)
         assert tc.tc_get_status(ctx) == 5
-    # (c) chunk offset pointing past its tile
-    broken = tc.EncodedStream(enc.words, enc.chunk_off.clone(), enc.tile_off, enc.layout)
-    broken.chunk_off[3] = 0x7FFFFFF0
-    tc.tc_decode(ctx, m, cb, broken, x.shape, x.dtype, stream_bytes=nbytes)
-    assert tc.tc_get_status(ctx) == 5
+    # (c) a chunk length that runs past its tile, and one that is off by a single bit
+    for delta in (30000, 1, -1):
+        broken = tc.EncodedStream(enc.words, enc.chunk_len.clone(), enc.tile_off, enc.layout)
+        broken.chunk_len[3] += delta
+        tc.tc_decode(ctx, m, cb, broken, x.shape, x.dtype, stream_bytes=nbytes)
+        assert tc.tc_get_status(ctx) == 5
     # (d) flipped payload bits: must stay in bounds; either decodes to other symbols or reports
-    noisy = tc.EncodedStream(enc.words.clone(), enc.chunk_off, enc.tile_off, enc.layout)
+    noisy = tc.EncodedStream(enc.words.clone(), enc.chunk_len, enc.tile_off, enc.layout)
     g = torch.Generator(device="cuda").manual_seed(1)
     idx = torch.randint(0, nbytes, (64,), generator=g, device="cuda")
     noisy.words[idx] ^= 0x5A

@@ -23,10 +23,11 @@ def _check_tiles(ctx, model_desc, lengths, bits, x, enc, xhat, tiles):
     n, c, h, w = x.shape
     hw = h * w
     pixels = n * hw
-    cp = enc.layout.chunk_pixels
-    cpt = 128 // cp
+    cp, splits = enc.layout.chunk_pixels, enc.layout.pixel_splits
+    cpt = 128 * splits // cp                       # chunks per tile
+    chunk_symbols = cp * c // splits
     tile_off = H.tile_off(enc)
-    chunk_off = H.chunk_off(enc)
+    chunk_len = H.chunk_len(enc)
     words_all = enc.words[: int(tile_off[-1]) // 8].cpu().numpy().view(np.uint32)
     m = oracle.Model(c, c, bits, model_desc["mean"], model_desc["basis"], model_desc["eig"],
                      model_desc["lo"], model_desc["step"], "bf16")
@@ -36,14 +37,14 @@ def _check_tiles(ctx, model_desc, lengths, bits, x, enc, xhat, tiles):
         p0, p1 = t * 128, min(pixels, (t + 1) * 128)
         # the tile's slice of the stream, as a stream of its own
         sub = oracle.Stream(words_all[int(tile_off[t]) // 32: int(tile_off[t + 1]) // 32].copy(),
-                            chunk_off[t * cpt: t * cpt + -(-(p1 - p0) // cp)].copy(),
+                            chunk_len[t * cpt: t * cpt + -(-((p1 - p0) * c) // chunk_symbols)].copy(),
                             np.array([0, tile_off[t + 1] - tile_off[t]], dtype=np.uint64),
-                            int(tile_off[t + 1] - tile_off[t]), p1 - p0, c, cp, cpt)
+                            int(tile_off[t + 1] - tile_off[t]), p1 - p0, c, cp, splits, 128)
         q_stream = oracle.decode_symbols(sub, lengths, bits)
         # entropy coding is bit-exact given the symbols
-        ref = oracle.encode(q_stream, lengths, bits, chunk_pixels=cp, tile_chunks=cpt)
+        ref = oracle.encode(q_stream, lengths, bits, chunk_pixels=cp, pixel_splits=splits, tile_pixels=128)
         assert np.array_equal(ref.words, sub.words)
-        assert np.array_equal(ref.chunk_off, sub.chunk_off)
+        assert np.array_equal(ref.chunk_len, sub.chunk_len)
         # the symbols are the oracle's, up to +-1 at rounding ties
         i0, i1 = p0 // hw, (p1 - 1) // hw + 1
         xs = x[i0:i1].cpu()
@@ -87,11 +88,13 @@ def test_full_size_layer_sampled_against_oracle(cfg, layer, bits):
     assert toff[0] == 0 and np.all(toff % 128 == 0) and np.all(np.diff(toff) > 0)
     lay = enc.layout
     assert len(toff) == lay.n_tiles + 1
-    coff = H.chunk_off(enc).astype(np.int64).reshape(lay.n_tiles if lay.n_chunks % lay.n_tiles == 0 else -1, -1) \
-        if lay.n_chunks % lay.n_tiles == 0 else None
-    if coff is not None:
-        assert np.all(coff[:, 0] == 0) and np.all(np.diff(coff, axis=1) > 0)
-        assert np.all(coff[:, -1] < np.diff(toff)[:, None][:, 0])
+    # the chunk lengths of every tile add up to the tile's size less its padding (under 128 bits)
+    clen = H.chunk_len(enc).astype(np.int64)
+    assert len(clen) == lay.n_chunks and np.all(clen > 0)
+    cpt = 128 * lay.pixel_splits // lay.chunk_pixels
+    per_tile = np.add.reduceat(clen, np.arange(0, lay.n_chunks, cpt))
+    pad = np.diff(toff) - per_tile
+    assert np.all(pad >= 0) and np.all(pad < 128)
     # the fp64 kernels decode the same stream to the same symbols: compare outputs on a slice
     exact = tc.tc_create(0)
     tc.tc_force_exact_path(exact, True)

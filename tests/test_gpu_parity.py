@@ -51,26 +51,27 @@ def check_symbols(q_gpu, o, *, exact: bool):
     return rate
 
 
-def check_stream_against_oracle(enc, q_gpu, lengths, bits, cp):
+def check_stream_against_oracle(enc, q_gpu, lengths, bits):
     """Entropy-coding stage: bit-exact given identical symbol arrays."""
-    ref = oracle.encode(q_gpu, lengths, bits, chunk_pixels=cp, tile_chunks=128 // cp)
+    ref = oracle.encode(q_gpu, lengths, bits, chunk_pixels=enc.layout.chunk_pixels,
+                        pixel_splits=enc.layout.pixel_splits, tile_pixels=128)
     assert enc.total_bits() == ref.total_bits
     assert np.array_equal(H.tile_off(enc), ref.tile_off)
-    assert np.array_equal(H.chunk_off(enc), ref.chunk_off)
+    assert enc.layout.n_chunks == ref.chunk_len.shape[0]
+    assert np.array_equal(H.chunk_len(enc), ref.chunk_len)
     assert np.array_equal(H.stream_words(enc), ref.words)
     return ref
 
 
-def run_case(ctx, spec, bits, n_cal, n_test, dtype, per_channel, *, exact, chunk_pixels=0, model=None):
+def run_case(ctx, spec, bits, n_cal, n_test, dtype, per_channel, *, exact, chunk_pixels=0, pixel_splits=0, model=None):
     o = H.oracle_side(spec, bits, n_cal, n_test, dtype, per_channel, model=model)
     m, lengths = o["model"], o["lengths"]
     model_h = H.import_model(tc, ctx, m, dtype)
     cb = tc.tc_codebook_import(ctx, lengths, bits)
     x = o["x"].cuda()
-    enc = tc.tc_encode(ctx, model_h, cb, x, chunk_pixels=chunk_pixels, debug=True)
+    enc = tc.tc_encode(ctx, model_h, cb, x, chunk_pixels=chunk_pixels, pixel_splits=pixel_splits, debug=True)
     assert tc.tc_get_status(ctx) == 0
     assert tc.tc_last_path(ctx) == (0 if exact else 1), "unexpected kernel route"
-    cp = enc.layout.chunk_pixels
     # coefficients
     y_gpu = enc.coefficients.cpu().numpy().astype(np.float64)
     tol = 1e-3 * np.maximum(np.abs(o["y"]), m.step)
@@ -79,7 +80,7 @@ def run_case(ctx, spec, bits, n_cal, n_test, dtype, per_channel, *, exact, chunk
     q_gpu = enc.symbols.cpu().numpy()
     check_symbols(q_gpu, o, exact=exact)
     # stream: bit-exact against the oracle's coder on the GPU's own symbols
-    ref = check_stream_against_oracle(enc, q_gpu, lengths, bits, cp)
+    ref = check_stream_against_oracle(enc, q_gpu, lengths, bits)
     assert np.array_equal(oracle.decode_symbols(ref, lengths, bits), q_gpu)
     # decode: reconstruct what the stream holds
     xhat = tc.tc_decode(ctx, model_h, cb, enc, x.shape, dtype)
@@ -136,6 +137,30 @@ def test_chunk_sizes_and_ragged_tail(ctx, cp):
     run_case(ctx, spec, 3, 8, 3, torch.bfloat16, True, exact=True, chunk_pixels=cp)
 
 
+@pytest.mark.parametrize("splits", [1, 2, 4])
+def test_pixel_splits_exact_path(ctx, splits):
+    # chunks of a half or a quarter of a pixel's coefficients, one full tile and a ragged one
+    spec = fm.LayerSpec(32, 9, 9, 0.85, None, 78)
+    _, enc = run_case(ctx, spec, 6, 8, 3, torch.float32, False, exact=True, chunk_pixels=1, pixel_splits=splits)
+    assert enc.layout.pixel_splits == splits and enc.layout.n_chunks == 243 * splits
+    run_case(ctx, spec, 3, 8, 3, torch.bfloat16, True, exact=True, chunk_pixels=1, pixel_splits=splits)
+
+
+def test_default_chunk_shapes(ctx):
+    # side information stays at 16 bits per 128..255 symbols: K = 16 -> 8 pixels per chunk,
+    # K = 64 -> 2, K = 128 -> 1, K = 256 -> two chunks per pixel
+    for c, want in ((16, (8, 1)), (64, (2, 1)), (128, (1, 1)), (256, (1, 2)), (512, (1, 2))):
+        spec = fm.LayerSpec(c, 4, 4, 0.9, None, 90 + c)
+        o = H.oracle_side(spec, 4, 4, 1, torch.bfloat16, False)
+        model_h = H.import_model(tc, ctx, o["model"], torch.bfloat16)
+        cb = tc.tc_codebook_import(ctx, o["lengths"], 4)
+        lay = tc.tc_encode_bound(model_h, cb, o["x"].cuda())
+        assert (lay.chunk_pixels, lay.pixel_splits) == want
+        assert lay.chunk_len_bytes == 2 * lay.n_chunks
+        model_h.close()
+        cb.close()
+
+
 # ---- tensor-core path (bf16 products, fp32 accumulation) -------------------------------------
 
 @pytest.mark.parametrize("c,s,n,bits", [(64, 56, 2, 4), (128, 28, 3, 4), (256, 14, 5, 4), (96, 28, 2, 5),
@@ -155,6 +180,19 @@ def test_tensor_core_path_per_channel_codebook_and_chunks(ctx_tc):
     spec = fm.LayerSpec(64, 14, 14, 0.9, None, 5100)
     for cp in (1, 4, 32):
         run_case(ctx_tc, spec, 4, 6, 3, torch.bfloat16, True, exact=False, chunk_pixels=cp)
+    run_case(ctx_tc, spec, 4, 6, 3, torch.bfloat16, True, exact=False, chunk_pixels=1, pixel_splits=2)
+
+
+@pytest.mark.parametrize("c,splits", [(256, 1), (256, 2), (64, 2), (128, 2), (192, 2)])
+def test_tensor_core_path_pixel_splits(ctx_tc, c, splits):
+    spec = fm.LayerSpec(c, 14, 14, 0.9, None, 5300 + c)
+    _, enc = run_case(ctx_tc, spec, 5, 6, 5, torch.bfloat16, False, exact=False, chunk_pixels=1, pixel_splits=splits)
+    assert enc.layout.pixel_splits == splits
+
+
+def test_four_splits_fall_back_to_the_exact_kernels(ctx_tc):
+    spec = fm.LayerSpec(64, 14, 14, 0.9, None, 5400)
+    run_case(ctx_tc, spec, 4, 6, 3, torch.bfloat16, False, exact=True, chunk_pixels=1, pixel_splits=4)
 
 
 def test_tensor_core_path_high_rate_tile_overflows_staging(ctx_tc):

@@ -19,7 +19,7 @@ pytestmark = pytest.mark.gpu
 
 def _fresh_buffers(ref: tc.EncodedStream) -> tc.EncodedStream:
     # same sizes as the reference run, pre-filled with a pattern so that stale bytes show
-    return tc.EncodedStream(torch.full_like(ref.words, 0x5A), torch.full_like(ref.chunk_off, -1),
+    return tc.EncodedStream(torch.full_like(ref.words, 0x5A), torch.full_like(ref.chunk_len, -1),
                             torch.full_like(ref.tile_off, -1), ref.layout)
 
 
@@ -41,7 +41,7 @@ def test_noalloc_encode_matches_tc_encode_twice_in_a_row(dtype, c, s, n, bits):
         out = tc.tc_encode_noalloc(ctx, model, cb, x, _fresh_buffers(ref))
         assert tc.tc_get_status(ctx) == 0
         assert torch.equal(out.tile_off, ref.tile_off), f"tile offsets differ on call {attempt + 1}"
-        assert torch.equal(out.chunk_off[: ref.layout.n_chunks], ref.chunk_off[: ref.layout.n_chunks])
+        assert torch.equal(out.chunk_len[: ref.layout.n_chunks], ref.chunk_len[: ref.layout.n_chunks])
         assert torch.equal(out.words[:nbytes], ref.words[:nbytes]), f"stream differs on call {attempt + 1}"
         if attempt == 0:
             tc.tc_encode_noalloc(ctx, model, cb, other, _fresh_buffers(ref))
