@@ -299,11 +299,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
         const int chunks_per_row = a.k / 8;
         const uint4 *src = reinterpret_cast<const uint4 *>(a.basis_t_bf16);
         const int c_pad = ((a.c + 127) / 128) * 128;         // rows past C are zero: their outputs are never stored
+        // (asynchronous copies: all of a thread's pieces are in flight at once; a copy of zero
+        // source bytes fills its 16 bytes with zeros)
         for (int i = tid; i < c_pad * chunks_per_row; i += kThreads) {
             const int ch = i / chunks_per_row, j8 = i - ch * chunks_per_row;
-            *reinterpret_cast<uint4 *>(s_basis + (ch >> 3) * sbo + j8 * 128 + (ch & 7) * 16) =
-                ch < a.c ? __ldg(src + i) : make_uint4(0u, 0u, 0u, 0u);
+            cp_async_16(basis_addr + (ch >> 3) * sbo + j8 * 128 + (ch & 7) * 16, ch < a.c ? src + i : src, ch < a.c ? 16u : 0u);
         }
+        cp_async_commit();
         if (!kPerChannel)
             for (int i = tid; i < lut_size; i += kThreads) {
                 // per-layer table: bf16(symbol - center) << 16 | code length
@@ -312,6 +314,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
                 s_lut[i] = (__float_as_uint(f) & 0xffff0000u) | (e & 0xffu);
             }
     }
+    cp_async_wait<0>();
     fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();

@@ -38,6 +38,7 @@ constexpr int kThreads = (kEpiWarps + 7) * 32;
 constexpr int kMaxHalfCols = 128;                 // coefficients per epilogue thread (K <= 256)
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;
+constexpr int kPairMaxBits = 4;                   // symbols of up to 4 bits are coded two at a time (256-entry tables)
 
 struct SmemLayout {
     uint32_t basis, ring, staging, enc, len8, bias, xch, total;
@@ -112,7 +113,9 @@ struct SmemBitWriter {
     }
 };
 
-template <bool kPerChannel, bool kDebug>
+// kPair (per-layer tables, b <= 4): the code tables are indexed by two neighbouring symbols at
+// once (q0 | q1 << b, at most 256 entries), which halves the lookups of both passes.
+template <bool kPerChannel, bool kDebug, bool kPair>
 __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -128,7 +131,8 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nsym = 1 << a.bits;
     constexpr bool enc_in_smem = !kPerChannel;
-    const SmemLayout L = smem_layout(a.c, a.k, enc_in_smem ? nsym : 0);
+    const int enc_entries = enc_in_smem ? (kPair ? nsym * nsym : nsym) : 0;
+    const SmemLayout L = smem_layout(a.c, a.k, enc_entries);
     unsigned char *s_basis = smem + L.basis;
     uint32_t *s_enc = reinterpret_cast<uint32_t *>(smem + L.enc);
     float *s_bias = reinterpret_cast<float *>(smem + L.bias);
@@ -153,21 +157,34 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
         const uint32_t sbo = (uint32_t)(a.c / 8) * 128u;
         const int chunks_per_row = a.c / 8;
         const uint4 *src = reinterpret_cast<const uint4 *>(a.basis_bf16);
+        // (asynchronous copies: all of a thread's pieces are in flight at once)
         for (int i = tid; i < a.k * chunks_per_row; i += kThreads) {
             const int j = i / chunks_per_row, c8 = i - j * chunks_per_row;
-            *reinterpret_cast<uint4 *>(s_basis + (j >> 3) * sbo + c8 * 128 + (j & 7) * 16) = __ldg(src + i);
+            cp_async_16(basis_addr + (j >> 3) * sbo + c8 * 128 + (j & 7) * 16, src + i, 16u);
         }
+        cp_async_commit();
         for (int i = tid; i < a.k; i += kThreads) s_bias[i] = a.enc_bias[i];
         if (enc_in_smem)
-            for (int i = tid; i < nsym; i += kThreads) {
+            for (int i = tid; i < enc_entries; i += kThreads) {
                 // per-layer table: (1 << length, code) pairs, so that appending a code to a register is
-                // one multiply-add, and the lengths once more as bytes
-                const uint32_t e = a.enc[i];
-                s_enc[2 * i] = 1u << (e & 0xffu);
-                s_enc[2 * i + 1] = e >> 8;
-                (smem + L.len8)[i] = (unsigned char)(e & 0xffu);
+                // one multiply-add, and the lengths once more as bytes.  In pair mode entry
+                // q0 | q1 << b holds the two codes joined (q0's first), at most 24 bits.
+                uint32_t len, code;
+                if constexpr (kPair) {
+                    const uint32_t e0 = a.enc[i & (nsym - 1)], e1 = a.enc[i >> a.bits];
+                    len = (e0 & 0xffu) + (e1 & 0xffu);
+                    code = ((e0 >> 8) << (e1 & 0xffu)) | (e1 >> 8);
+                } else {
+                    const uint32_t e = a.enc[i];
+                    len = e & 0xffu;
+                    code = e >> 8;
+                }
+                s_enc[2 * i] = 1u << len;
+                s_enc[2 * i + 1] = code;
+                (smem + L.len8)[i] = (unsigned char)len;
             }
     }
+    cp_async_wait<0>();
     fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();
@@ -300,6 +317,7 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
         const uint32_t stg_addr = smem_u32(stg);
         const uint32_t enc_addr = smem_u32(s_enc);
         const uint32_t len8_rel = smem_u32(smem + L.len8) - kMagicBits;   // + (kMagicBits + q) = address of len8[q]
+        const uint32_t pair_len_rel = smem_u32(smem + L.len8) - kMagicBits * (1u + (1u << a.bits));   // same for a pair sum
         unsigned short *xch = reinterpret_cast<unsigned short *>(smem + L.xch) + grp * 256;   // [2][128] lengths exchanged between the halves
         long long n_done = 0;                      // tiles this group has handed to its store warp
         const float inv_step = (float)(1.0 / a.step);
@@ -329,7 +347,7 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
             const uint32_t trow = tmem_base + grp * kAccCols + ((uint32_t)(wq * 32) << 16) + col0;
 
             // pass 1: quantise, keep the symbols (one byte each) in registers, add up code lengths
-            uint32_t sym[kMaxHalfCols / 4];
+            uint32_t sym[kPair ? kMaxHalfCols / 8 : kMaxHalfCols / 4];   // one byte per symbol, or per pair of symbols
             uint32_t blk_bits[kMaxHalfCols / 64] = {};          // code bits of each block of 16 symbols, one byte each
             unsigned int my_bits = 0;
 #pragma unroll
@@ -348,7 +366,7 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
                         const int j = col0 + blk * 16 + i;
                         const uint32_t vb = quantise_bits(r[i], inv_step, biasv[i], vmax);
                         if constexpr (kPerChannel) my_bits += __ldg(a.enc + j * nsym + (vb & 0xffu)) & 0xffu;
-                        else {
+                        else if constexpr (!kPair) {
                             uint32_t l;
                             asm("ld.shared.u8 %0, [%1];" : "=r"(l) : "r"(vb + len8_rel));
                             my_bits += l;
@@ -359,9 +377,24 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
                         }
                         r[i] = vb;
                     }
+                    if constexpr (kPair) {
+                        // pair index in the low byte of vb0 + (vb1 << b) (the magic constants have a zero
+                        // low byte); the same sum, rebased, addresses the pair-length table
 #pragma unroll
-                    for (int i = 0; i < 16; i += 4)      // low bytes of four values -> one register
-                        sym[blk * 4 + i / 4] = __byte_perm(__byte_perm(r[i], r[i + 1], 0x0040), __byte_perm(r[i + 2], r[i + 3], 0x0040), 0x5410);
+                        for (int i = 0; i < 16; i += 2) {
+                            r[i] = r[i] + (r[i + 1] << a.bits);
+                            uint32_t l;
+                            asm("ld.shared.u8 %0, [%1];" : "=r"(l) : "r"(r[i] + pair_len_rel));
+                            my_bits += l;
+                        }
+#pragma unroll
+                        for (int i = 0; i < 16; i += 8)      // low bytes of four pairs -> one register
+                            sym[blk * 2 + i / 8] = __byte_perm(__byte_perm(r[i], r[i + 2], 0x0040), __byte_perm(r[i + 4], r[i + 6], 0x0040), 0x5410);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; i += 4)      // low bytes of four values -> one register
+                            sym[blk * 4 + i / 4] = __byte_perm(__byte_perm(r[i], r[i + 1], 0x0040), __byte_perm(r[i + 2], r[i + 3], 0x0040), 0x5410);
+                    }
                     blk_bits[blk >> 2] |= (my_bits - bits_before) << (8 * (blk & 3));      // at most 16 * 12 = 192
                 }
             }
@@ -441,16 +474,35 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
 #pragma unroll
                         const int nbits = (int)((blk_bits[blk >> 2] >> (8 * (blk & 3))) & 0xffu);
                         if (!kPerChannel && nbits < 32) {
-                            // the whole block fits one register: acc = acc * 2^len + code per symbol
+                            // the whole block fits one register: acc = acc * 2^len + code per symbol (or pair)
                             uint32_t acc = 0;
+                            if constexpr (kPair) {
 #pragma unroll
-                            for (int i = 0; i < 16; ++i) {
-                                const uint32_t q = (sym[blk * 4 + i / 4] >> (8 * (i & 3))) & 0xffu;
-                                uint32_t mul, code;
-                                asm("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(mul), "=r"(code) : "r"(enc_addr + q * 8u));
-                                acc = acc * mul + code;
+                                for (int i = 0; i < 8; ++i) {
+                                    const uint32_t q = (sym[blk * 2 + i / 4] >> (8 * (i & 3))) & 0xffu;
+                                    uint32_t mul, code;
+                                    asm("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(mul), "=r"(code) : "r"(enc_addr + q * 8u));
+                                    acc = acc * mul + code;
+                                }
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 16; ++i) {
+                                    const uint32_t q = (sym[blk * 4 + i / 4] >> (8 * (i & 3))) & 0xffu;
+                                    uint32_t mul, code;
+                                    asm("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(mul), "=r"(code) : "r"(enc_addr + q * 8u));
+                                    acc = acc * mul + code;
+                                }
                             }
                             w.put(acc, nbits);
+                        } else if constexpr (kPair) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {         // pair by pair: at most 24 bits each
+                                const uint32_t q = (sym[blk * 2 + i / 4] >> (8 * (i & 3))) & 0xffu;
+                                uint32_t code, l;
+                                asm("ld.shared.u32 %0, [%1];" : "=r"(code) : "r"(enc_addr + q * 8u + 4u));
+                                asm("ld.shared.u8 %0, [%1];" : "=r"(l) : "r"(len8_rel + kMagicBits + q));
+                                w.put(code, (int)l);
+                            }
                         } else {
 #pragma unroll
                             for (int i = 0; i < 16; i += 2) {
@@ -522,23 +574,33 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
 
 }  // namespace
 
+// entries of the code table held in shared memory: none (per-channel tables stay in global
+// memory), one per symbol, or one per pair of symbols
+static int enc_table_entries(const EncodeArgs &a)
+{
+    if (a.groups != 1) return 0;
+    return a.bits <= kPairMaxBits ? (1 << (2 * a.bits)) : (1 << a.bits);
+}
+
 bool tc_encode_tc_supported(const tc_ctx *ctx, const EncodeArgs &a)
 {
     if (a.c % 16 != 0 || a.k != a.c || a.c > 256 || a.hw % 4 != 0) return false;
     // two chunks per pixel must coincide with the two halves the epilogue threads work on
     if (a.splits != 1 && !(a.splits == 2 && a.k % 32 == 0)) return false;
     if (a.groups != 1 && a.groups != a.k) return false;
-    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.bits) : 0);
+    const SmemLayout l = smem_layout(a.c, a.k, enc_table_entries(a));
     return (int)l.total + 512 <= ctx->max_smem_optin;       // leaves room for the static shared variables
 }
 
 tc_status tc_launch_encode_tc(const tc_ctx *ctx, const EncodeArgs &a, cudaStream_t s)
 {
     if (a.n_tiles <= 0) return TC_OK;
-    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.bits) : 0);
-    const bool per_channel = a.groups != 1, debug = a.dbg_coef || a.dbg_sym;
-    void (*kernel)(EncodeArgs) = per_channel ? (debug ? encode_tc_kernel<true, true> : encode_tc_kernel<true, false>)
-                                             : (debug ? encode_tc_kernel<false, true> : encode_tc_kernel<false, false>);
+    const SmemLayout l = smem_layout(a.c, a.k, enc_table_entries(a));
+    const bool per_channel = a.groups != 1, debug = a.dbg_coef || a.dbg_sym, pair = !per_channel && a.bits <= kPairMaxBits;
+    void (*kernel)(EncodeArgs) =
+        per_channel ? (debug ? encode_tc_kernel<true, true, false> : encode_tc_kernel<true, false, false>)
+        : pair      ? (debug ? encode_tc_kernel<false, true, true> : encode_tc_kernel<false, false, true>)
+                    : (debug ? encode_tc_kernel<false, true, false> : encode_tc_kernel<false, false, false>);
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.total) != cudaSuccess)
         return TC_ERR_CUDA;
     const unsigned int grid = (unsigned int)((a.n_tiles < ctx->sm_count) ? a.n_tiles : ctx->sm_count);
