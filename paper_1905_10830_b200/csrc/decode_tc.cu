@@ -347,9 +347,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
 
         // offsets of a tile, validated; a tile that cannot be valid decodes nothing.  `lens` holds
         // the chunk length(s) of this thread's pixel: both halves (S = 2) or the one chunk.
-        struct TileInfo { unsigned long long base, bits; bool ok, staged; unsigned int lens; };
+        // A segment of up to one stream buffer is copied while the tile before it is decoded; a
+        // `big` one (up to two buffers) takes both buffers of the group and is copied when its own
+        // turn comes; anything larger is read from global memory.
+        struct TileInfo { unsigned long long base, bits; bool ok, staged, big; unsigned int lens; };
         auto tile_info = [&](long long tl) {
-            TileInfo ti{0, 0, false, false, 0};
+            TileInfo ti{0, 0, false, false, false, 0};
             if (tl >= my_tiles) return ti;
             const long long tile = blockIdx.x + tl * gridDim.x;
             const unsigned long long base = a.tile_off[tile], end = a.tile_off[tile + 1];
@@ -357,8 +360,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
             if (!ti.ok) return ti;
             ti.base = base;
             ti.bits = end - base;
-            ti.staged = sbuf_bytes != 0 && ti.bits <= (unsigned long long)sbuf_bytes * 8ull &&
+            ti.staged = sbuf_bytes != 0 && ti.bits <= (unsigned long long)sbuf_bytes * 16ull &&
                         (cp * k_sub * TC_MAX_CODE_LEN) / 8 + 16 <= kStreamSlack;
+            ti.big = ti.staged && ti.bits > (unsigned long long)sbuf_bytes * 8ull;
             if (S == 2) {
                 const long long ch = tile * chunks_per_tile + 2 * t;     // even: both lengths in one aligned word
                 if (ch < a.n_chunks) ti.lens = *reinterpret_cast<const unsigned int *>(a.chunk_len + ch);
@@ -380,17 +384,26 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
         };
 
         // (with one chunk per pixel or fewer, warps 4-7 of a group have nothing to do)
-        TileInfo cur{0, 0, false, false, 0}, nxt = cur;
+        TileInfo cur{0, 0, false, false, false, 0}, nxt = cur;
         if (working) {
             cur = tile_info(grp);
             nxt = tile_info(grp + 2);
-            stage_tile(cur, 0);
         }
         int li = 0;
+        bool cur_copied = false;                     // the copy of `cur` was started one tile earlier
         for (long long tl = grp; tl < my_tiles && alive && working; tl += 2, ++li) {
             const long long tile = blockIdx.x + tl * gridDim.x;
-            stage_tile(nxt, (li + 1) & 1);           // its buffer was released by the barrier that ended tile li - 1
-            cp_async_wait<1>();
+            const int cur_buf = cur.big ? 0 : (li & 1);
+            if (!cur_copied) stage_tile(cur, cur_buf);
+            // the next tile's buffer was released by the barrier that ended tile li - 1; no copy
+            // ahead while this tile or the next needs both buffers
+            const bool ahead = !cur.big && !nxt.big;
+            if (ahead) {
+                stage_tile(nxt, (li + 1) & 1);
+                cp_async_wait<1>();
+            } else {
+                cp_async_wait<0>();
+            }
             // start of every chunk = sum of the lengths before it in the tile (chunk order: pixel,
             // then half): scan over the pixels' totals; both halves of a group compute the same scan
             const unsigned int len0 = S == 2 ? (cur.lens & 0xffffu) : cur.lens, len1 = S == 2 ? (cur.lens >> 16) : 0u;
@@ -419,7 +432,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
             bool bad = !cur.ok || (unsigned long long)tile_total > cur.bits;
             if (bad) active = false;
             const int n_pix = active ? (int)min((long long)cp, a.pixels - (tile * TC_TILE_PIXELS + (S == 2 ? (long long)t : (long long)t * cp))) : 0;
-            const uint32_t seg_addr = sbuf_g + (uint32_t)(li & 1) * sbuf_bytes;
+            const uint32_t seg_addr = sbuf_g + (uint32_t)cur_buf * sbuf_bytes;
             const int k_first = sub * k_sub, k_end = k_first + k_sub;
 
             // walks this thread's chunk; `fill_panel(dst, k0, nk8)` decodes the next 8 * nk8 symbols
@@ -524,6 +537,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
             named_bar_sync(bar_id, n_thr);           // this tile's stream buffer may be refilled
             cur = nxt;
             nxt = after;
+            cur_copied = ahead;
         }
         cp_async_wait<0>();
         if (!alive && t == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
