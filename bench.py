@@ -315,8 +315,8 @@ def main():
                      "encode_frac": algo_bytes / (enc_avg * 1e-3) / 1e9 / peak,
                      "decode_frac": algo_bytes / (dec_avg * 1e-3) / 1e9 / peak},
         "gpu_launches": 2 * args.steps,
-        "kernels": {"encode": ["fp64", "tcgen05"][tc.tc_last_path(ctx, False)],
-                    "decode": ["fp64", "tcgen05"][tc.tc_last_path(ctx, True)]},
+        "kernels": {"encode": ["fp64", "tcgen05", "fp32"][tc.tc_last_path(ctx, False)],
+                    "decode": ["fp64", "tcgen05", "fp32"][tc.tc_last_path(ctx, True)]},
         "clocks": clocks,
     }
     if e2e is not None:

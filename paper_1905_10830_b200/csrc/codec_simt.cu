@@ -1,7 +1,13 @@
 // Exact (fp64) encode and decode kernels: one thread per pixel, plain FMA-free double
 // arithmetic in the order the definition states, so that fp32 tensors -- whose products do not
 // fit the bf16 tensor-core path -- are coded without any rounding of their own.  They are
-// also the path for shapes the tensor-core kernels do not take, and for the statistics mode.
+// also the validation path and the statistics mode.
+//
+// The same kernels have an fp32 mode (kFp32) for bf16 tensors whose shape the tensor-core
+// kernels do not take (more than 256 channels, odd map sizes): bf16 x bf16 products are exact
+// in fp32, accumulation is fp32 with fused multiply-adds, and the quantiser / dequantiser use
+// the same folded constants as the tensor-core kernels (acc / step + bias, step * acc + bias
+// around the centre symbol), so that the two bf16 routes take their decisions alike.
 //
 // Encode (Section 3: transform, quantiser, VLC): y_j = sum_c T[j][c] (x_c - mu_c),
 // q = clamp(rint((y - lo)/step)), code lookup, bit offsets by scan + tile look-back, pack.
@@ -12,18 +18,21 @@
 namespace {
 
 constexpr int kThreads = TC_TILE_PIXELS;
-constexpr int kRowBlock = 8;           // basis rows (encode) / columns (decode) per pass
+constexpr int kRowBlock = 8;           // basis rows (encode) / columns (decode) per pass, fp64 mode
+constexpr int kRowBlock32 = 16;        // the same in fp32 mode
 constexpr int kEncSmemEntries = 2048;  // code tables up to this many entries are staged
 
 using namespace tcdev;
 
-template <typename TIn>
+template <typename TIn, bool kFp32>
 __global__ void __launch_bounds__(kThreads) encode_simt_kernel(EncodeArgs a)
 {
+    constexpr int RB = kFp32 ? kRowBlock32 : kRowBlock;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    double *s_mean = reinterpret_cast<double *>(smem_raw);            // [C]
-    double *s_panel = s_mean + a.c;                                    // [kRowBlock][C]
-    uint32_t *s_enc = reinterpret_cast<uint32_t *>(s_panel + kRowBlock * a.c);
+    double *s_mean = reinterpret_cast<double *>(smem_raw);            // [C]  (fp64 mode)
+    double *s_panel = s_mean + a.c;                                    // [RB][C] doubles, or [C][RB] floats in fp32 mode
+    float *s_panel32 = reinterpret_cast<float *>(s_panel);
+    uint32_t *s_enc = reinterpret_cast<uint32_t *>(s_panel + kRowBlock * a.c);      // 8 doubles = 16 floats per channel
     const int nsym = 1 << a.bits;
     const int enc_entries = a.groups * nsym;
     const bool enc_in_smem = enc_entries <= kEncSmemEntries;
@@ -56,14 +65,54 @@ __global__ void __launch_bounds__(kThreads) encode_simt_kernel(EncodeArgs a)
     const double top = (double)(nsym - 1);
     unsigned int clamped = 0;
 
-    for (int j0 = 0; j0 < a.k; j0 += kRowBlock) {
+    for (int j0 = 0; j0 < a.k; j0 += RB) {
         __syncthreads();
-        for (int i = t; i < kRowBlock * a.c; i += kThreads) {
-            const int jj = i / a.c, cc = i - jj * a.c;
-            s_panel[i] = (j0 + jj < a.k) ? a.basis64[(long long)(j0 + jj) * a.c + cc] : 0.0;
+        if constexpr (kFp32) {
+            // [C][RB] floats: the RB coefficients of one channel are one 64-byte row
+            for (int i = t; i < RB * a.c; i += kThreads) {
+                const int jj = i / a.c, cc = i - jj * a.c;
+                s_panel32[cc * RB + jj] = (j0 + jj < a.k) ? __bfloat162float(a.basis_bf16[(long long)(j0 + jj) * a.c + cc]) : 0.f;
+            }
+        } else {
+            for (int i = t; i < kRowBlock * a.c; i += kThreads) {
+                const int jj = i / a.c, cc = i - jj * a.c;
+                s_panel[i] = (j0 + jj < a.k) ? a.basis64[(long long)(j0 + jj) * a.c + cc] : 0.0;
+            }
         }
         __syncthreads();
-        if (valid) {
+        if constexpr (kFp32) {
+            if (valid) {
+                float acc[RB];
+#pragma unroll
+                for (int jj = 0; jj < RB; ++jj) acc[jj] = 0.f;
+                for (int cc = 0; cc < a.c; ++cc) {
+                    const float xv = (float)load_as_double(xin + xbase + (long long)cc * a.hw);
+                    const float4 *row = reinterpret_cast<const float4 *>(s_panel32 + cc * RB);
+#pragma unroll
+                    for (int q4 = 0; q4 < RB / 4; ++q4) {
+                        const float4 w = row[q4];
+                        acc[4 * q4 + 0] = fmaf(w.x, xv, acc[4 * q4 + 0]);
+                        acc[4 * q4 + 1] = fmaf(w.y, xv, acc[4 * q4 + 1]);
+                        acc[4 * q4 + 2] = fmaf(w.z, xv, acc[4 * q4 + 2]);
+                        acc[4 * q4 + 3] = fmaf(w.w, xv, acc[4 * q4 + 3]);
+                    }
+                }
+                const float inv_step = (float)(1.0 / a.step);
+#pragma unroll
+                for (int jj = 0; jj < RB; ++jj) {
+                    const int j = j0 + jj;
+                    if (j < a.k) {
+                        const float u = fmaf(acc[jj], inv_step, a.enc_bias[j]);      // (y - lo) / step
+                        if (u < 0.f || u > (float)top) ++clamped;
+                        const float r = fminf(fmaxf(rintf(u), 0.f), (float)top);
+                        const unsigned int q = (unsigned int)r;
+                        s_q[j * kThreads + t] = (uint8_t)q;
+                        if (a.dbg_coef) a.dbg_coef[p * a.k + j] = acc[jj] - a.tmu32[j];
+                        if (a.dbg_sym) a.dbg_sym[p * a.k + j] = (uint8_t)q;
+                    }
+                }
+            }
+        } else if (valid) {
             double acc[kRowBlock];
 #pragma unroll
             for (int jj = 0; jj < kRowBlock; ++jj) acc[jj] = 0.0;
@@ -195,12 +244,14 @@ struct BitReader {
     }
 };
 
-template <typename TOut>
+template <typename TOut, bool kFp32>
 __global__ void __launch_bounds__(kThreads) decode_simt_kernel(DecodeArgs a)
 {
+    constexpr int RB = kFp32 ? kRowBlock32 : kRowBlock;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    double *s_mean = reinterpret_cast<double *>(smem_raw);        // [C]
-    double *s_panel = s_mean + a.c;                                // [K][kRowBlock]
+    double *s_mean = reinterpret_cast<double *>(smem_raw);        // [C]  (fp64 mode)
+    double *s_panel = s_mean + a.c;                                // [K][RB] doubles (fp64) or floats (fp32: same bytes)
+    float *s_panel32 = reinterpret_cast<float *>(s_panel);
     uint8_t *s_q = reinterpret_cast<uint8_t *>(s_panel + (size_t)a.k * kRowBlock);   // [K][128]
     __shared__ int s_bad;
     __shared__ uint16_t s_len[4 * TC_TILE_PIXELS];                 // chunk lengths of the tile
@@ -272,14 +323,44 @@ __global__ void __launch_bounds__(kThreads) decode_simt_kernel(DecodeArgs a)
         const long long s = p - img * a.hw;
         obase = img * a.c * (long long)a.hw + s;
     }
-    for (int c0 = 0; c0 < a.c; c0 += kRowBlock) {
+    for (int c0 = 0; c0 < a.c; c0 += RB) {
         __syncthreads();
-        for (int i = t; i < a.k * kRowBlock; i += kThreads) {
-            const int j = i / kRowBlock, cc = i - j * kRowBlock;
-            s_panel[i] = (c0 + cc < a.c) ? a.basis64[(long long)j * a.c + c0 + cc] : 0.0;
+        if constexpr (kFp32) {
+            for (int i = t; i < a.k * RB; i += kThreads) {
+                const int cc = i / a.k, j = i - cc * a.k;             // consecutive threads read consecutive j of one channel row
+                s_panel32[j * RB + cc] = (c0 + cc < a.c) ? __bfloat162float(a.basis_t_bf16[(long long)(c0 + cc) * a.k + j]) : 0.f;
+            }
+        } else {
+            for (int i = t; i < a.k * kRowBlock; i += kThreads) {
+                const int j = i / kRowBlock, cc = i - j * kRowBlock;
+                s_panel[i] = (c0 + cc < a.c) ? a.basis64[(long long)j * a.c + c0 + cc] : 0.0;
+            }
         }
         __syncthreads();
-        if (valid) {
+        if constexpr (kFp32) {
+            if (valid) {
+                float acc[RB];
+#pragma unroll
+                for (int cc = 0; cc < RB; ++cc) acc[cc] = 0.f;
+                for (int j = 0; j < a.k; ++j) {
+                    const float qv = (float)((int)s_q[j * kThreads + t] - a.center);
+                    const float4 *row = reinterpret_cast<const float4 *>(s_panel32 + j * RB);
+#pragma unroll
+                    for (int q4 = 0; q4 < RB / 4; ++q4) {
+                        const float4 w = row[q4];
+                        acc[4 * q4 + 0] = fmaf(w.x, qv, acc[4 * q4 + 0]);
+                        acc[4 * q4 + 1] = fmaf(w.y, qv, acc[4 * q4 + 1]);
+                        acc[4 * q4 + 2] = fmaf(w.z, qv, acc[4 * q4 + 2]);
+                        acc[4 * q4 + 3] = fmaf(w.w, qv, acc[4 * q4 + 3]);
+                    }
+                }
+                const float step = (float)a.step;
+#pragma unroll
+                for (int cc = 0; cc < RB; ++cc)
+                    if (c0 + cc < a.c)
+                        store_rounded(out + obase + (long long)(c0 + cc) * a.hw, (double)fmaf(acc[cc], step, a.dec_bias[c0 + cc]));
+            }
+        } else if (valid) {
             double acc[kRowBlock];
 #pragma unroll
             for (int cc = 0; cc < kRowBlock; ++cc) acc[cc] = 0.0;
@@ -324,13 +405,27 @@ tc_status launch(K kernel, const A &a, size_t smem, const tc_ctx *ctx, cudaStrea
 tc_status tc_launch_encode_simt(const tc_ctx *ctx, const EncodeArgs &a, int dtype, cudaStream_t s)
 {
     const size_t smem = encode_smem_bytes(a);
-    if (dtype == TC_F32) return launch(encode_simt_kernel<float>, a, smem, ctx, s);
-    return launch(encode_simt_kernel<__nv_bfloat16>, a, smem, ctx, s);
+    if (dtype == TC_F32) return launch(encode_simt_kernel<float, false>, a, smem, ctx, s);
+    return launch(encode_simt_kernel<__nv_bfloat16, false>, a, smem, ctx, s);
 }
 
 tc_status tc_launch_decode_simt(const tc_ctx *ctx, const DecodeArgs &a, int dtype, cudaStream_t s)
 {
     const size_t smem = decode_smem_bytes(a);
-    if (dtype == TC_F32) return launch(decode_simt_kernel<float>, a, smem, ctx, s);
-    return launch(decode_simt_kernel<__nv_bfloat16>, a, smem, ctx, s);
+    if (dtype == TC_F32) return launch(decode_simt_kernel<float, false>, a, smem, ctx, s);
+    return launch(decode_simt_kernel<__nv_bfloat16, false>, a, smem, ctx, s);
+}
+
+// fp32 mode, bf16 tensors only (the shared-memory carve-up is the fp64 mode's: 16 floats take
+// the room of 8 doubles)
+tc_status tc_launch_encode_simt_fp32(const tc_ctx *ctx, const EncodeArgs &a, cudaStream_t s)
+{
+    if (!a.basis_bf16 || !a.enc_bias || !a.tmu32) return TC_ERR_UNSUPPORTED;
+    return launch(encode_simt_kernel<__nv_bfloat16, true>, a, encode_smem_bytes(a), ctx, s);
+}
+
+tc_status tc_launch_decode_simt_fp32(const tc_ctx *ctx, const DecodeArgs &a, cudaStream_t s)
+{
+    if (!a.basis_t_bf16 || !a.dec_bias) return TC_ERR_UNSUPPORTED;
+    return launch(decode_simt_kernel<__nv_bfloat16, true>, a, decode_smem_bytes(a), ctx, s);
 }

@@ -97,6 +97,10 @@ extern "C" tc_status tc_encode_noalloc(tc_ctx *ctx, const tc_model *m, const tc_
         ctx->last_encode_path = 1;
         return tc_launch_encode_tc(ctx, a, s);
     }
+    if (!ctx->force_exact && x->dtype == TC_BF16 && x->c % 2 == 0) {      // shapes the tensor-core kernel does not take
+        ctx->last_encode_path = 2;
+        return tc_launch_encode_simt_fp32(ctx, a, s);
+    }
     ctx->last_encode_path = 0;
     return tc_launch_encode_simt(ctx, a, x->dtype, s);
 }

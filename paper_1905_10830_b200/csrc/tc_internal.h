@@ -29,7 +29,7 @@ struct tc_ctx {
     void *host_arena = nullptr;           // device staging of tc_roundtrip_host (grown on demand)
     size_t host_arena_bytes = 0;
     int force_exact = 0;                  // route every tensor through the fp64 kernels
-    int last_encode_path = 0;             // 0 = fp64 kernels, 1 = tensor-core kernels
+    int last_encode_path = 0;             // 0 = fp64 kernels, 1 = tensor-core kernels, 2 = fp32 kernels
     int last_decode_path = 0;
 };
 
@@ -115,6 +115,8 @@ struct DecodeArgs {
 // ---- launchers (defined in the .cu files) ----------------------------------------------
 tc_status tc_launch_encode_simt(const tc_ctx *ctx, const EncodeArgs &a, int dtype, cudaStream_t s);
 tc_status tc_launch_decode_simt(const tc_ctx *ctx, const DecodeArgs &a, int dtype, cudaStream_t s);
+tc_status tc_launch_encode_simt_fp32(const tc_ctx *ctx, const EncodeArgs &a, cudaStream_t s);
+tc_status tc_launch_decode_simt_fp32(const tc_ctx *ctx, const DecodeArgs &a, cudaStream_t s);
 bool tc_encode_tc_supported(const tc_ctx *ctx, const EncodeArgs &a);
 tc_status tc_launch_encode_tc(const tc_ctx *ctx, const EncodeArgs &a, cudaStream_t s);
 bool tc_decode_tc_supported(const tc_ctx *ctx, const DecodeArgs &a);

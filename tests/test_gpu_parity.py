@@ -63,7 +63,11 @@ def check_stream_against_oracle(enc, q_gpu, lengths, bits):
     return ref
 
 
-def run_case(ctx, spec, bits, n_cal, n_test, dtype, per_channel, *, exact, chunk_pixels=0, pixel_splits=0, model=None):
+def run_case(ctx, spec, bits, n_cal, n_test, dtype, per_channel, *, exact, chunk_pixels=0, pixel_splits=0, model=None,
+             routes=None):
+    """`routes`: the kernels expected for (encode, decode): 0 fp64, 1 tensor core, 2 fp32."""
+    if routes is None:
+        routes = (0, 0) if exact else (1, 1)
     o = H.oracle_side(spec, bits, n_cal, n_test, dtype, per_channel, model=model)
     m, lengths = o["model"], o["lengths"]
     model_h = H.import_model(tc, ctx, m, dtype)
@@ -71,7 +75,7 @@ def run_case(ctx, spec, bits, n_cal, n_test, dtype, per_channel, *, exact, chunk
     x = o["x"].cuda()
     enc = tc.tc_encode(ctx, model_h, cb, x, chunk_pixels=chunk_pixels, pixel_splits=pixel_splits, debug=True)
     assert tc.tc_get_status(ctx) == 0
-    assert tc.tc_last_path(ctx) == (0 if exact else 1), "unexpected kernel route"
+    assert tc.tc_last_path(ctx) == routes[0], "unexpected kernel route"
     # coefficients
     y_gpu = enc.coefficients.cpu().numpy().astype(np.float64)
     tol = 1e-3 * np.maximum(np.abs(o["y"]), m.step)
@@ -85,7 +89,7 @@ def run_case(ctx, spec, bits, n_cal, n_test, dtype, per_channel, *, exact, chunk
     # decode: reconstruct what the stream holds
     xhat = tc.tc_decode(ctx, model_h, cb, enc, x.shape, dtype)
     assert tc.tc_get_status(ctx) == 0
-    assert tc.tc_last_path(ctx, True) == (0 if exact else 1), "unexpected kernel route"
+    assert tc.tc_last_path(ctx, True) == routes[1], "unexpected kernel route"
     want = oracle.reconstruct(m, q_gpu, x.shape, out_bf16=(dtype == torch.bfloat16))
     got = xhat.float().cpu().numpy()
     if exact:
@@ -190,9 +194,27 @@ def test_tensor_core_path_pixel_splits(ctx_tc, c, splits):
     assert enc.layout.pixel_splits == splits
 
 
-def test_four_splits_fall_back_to_the_exact_kernels(ctx_tc):
+def test_four_splits_take_the_fp32_kernels(ctx_tc):
     spec = fm.LayerSpec(64, 14, 14, 0.9, None, 5400)
-    run_case(ctx_tc, spec, 4, 6, 3, torch.bfloat16, False, exact=True, chunk_pixels=1, pixel_splits=4)
+    run_case(ctx_tc, spec, 4, 6, 3, torch.bfloat16, False, exact=False, chunk_pixels=1, pixel_splits=4, routes=(2, 2))
+
+
+# ---- fp32 kernels: bf16 tensors of shapes the tensor-core kernels do not take -----------------
+
+@pytest.mark.parametrize("c,s,n,bits", [(512, 7, 5, 4), (384, 14, 2, 5), (576, 14, 1, 5), (960, 7, 3, 5), (1024, 4, 9, 3)])
+def test_fp32_route_wide_layers(ctx_tc, c, s, n, bits):
+    spec = fm.LayerSpec(c, s, s, 0.95, 0.6 if c != 512 else None, 5500 + c)
+    run_case(ctx_tc, spec, bits, max(4, (2 * c) // (s * s) + 1), n, torch.bfloat16, False, exact=False, routes=(2, 2))
+
+
+def test_fp32_route_odd_map_size_and_per_channel_codebook(ctx_tc):
+    # 5x5 maps: the tensor-core encoder needs H*W % 4 == 0, its decoder does not
+    spec = fm.LayerSpec(64, 5, 5, 0.9, None, 5600)
+    run_case(ctx_tc, spec, 6, 8, 7, torch.bfloat16, False, exact=False, routes=(2, 1))
+    run_case(ctx_tc, spec, 4, 8, 7, torch.bfloat16, True, exact=False, routes=(2, 1))
+    # 24 channels: neither tensor-core kernel (C % 16 != 0)
+    spec = fm.LayerSpec(24, 9, 9, 0.9, None, 5601)
+    run_case(ctx_tc, spec, 5, 8, 3, torch.bfloat16, False, exact=False, chunk_pixels=4, routes=(2, 2))
 
 
 def test_tensor_core_path_high_rate_tile_overflows_staging(ctx_tc):
