@@ -34,6 +34,8 @@ from synth import featuremaps as fm
 
 METRIC = "raw_activation_GBps_encode_plus_decode"
 UNIT = "GB/s"
+# dram__bytes_read.sum + dram__bytes_write.sum per tensor value, one ncu capture per kernel
+NCU_DRAM_BYTES_PER_VALUE = {"encode": 2.117, "decode": 1.628}
 
 
 def measured_peaks():
@@ -288,12 +290,20 @@ def main():
         return
 
     peak, peak_src = measured_peaks()
+    kernels = (["fp64", "tcgen05", "fp32"][tc.tc_last_path(ctx, False)], ["fp64", "tcgen05", "fp32"][tc.tc_last_path(ctx, True)])
     enc_avg, dec_avg = statistics.mean(enc_ms), statistics.mean(dec_ms)
     algo_bytes = raw_bytes + stream_bytes + side_bytes          # per launch, either direction
     dominant = "encode" if enc_avg >= dec_avg else "decode"
     dom_ms = max(enc_avg, dec_avg)
     achieved = algo_bytes / (dom_ms * 1e-3) / 1e9
     values = x.numel()
+    # DRAM bytes (read + write) of the dominant kernel from the ncu capture of these kernels at
+    # batch 2048 (profiles/encode_decode_tc_kernels_cfg5_batch2048.md), scaled by the values a
+    # launch processes: every tile is read and written once, so traffic grows with the batch.
+    # Only quoted for the configuration the counters were taken on.
+    traffic = None
+    if bits == 4 and kernels == ("tcgen05", "tcgen05") and lay.pixel_splits == 2:
+        traffic = NCU_DRAM_BYTES_PER_VALUE[dominant] * values
     line = {
         "metric": METRIC,
         "value": job_bytes / (total_ms * 1e-3) / 1e9,
@@ -311,12 +321,11 @@ def main():
         "mse_sample": test_stats.mse,
         "roofline": {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "frac_of_nominal_8TBps": achieved / 8000.0, "peak_source": peak_src,
-                     "algorithmic_bytes_per_launch": algo_bytes, "traffic": None,
+                     "algorithmic_bytes_per_launch": algo_bytes, "traffic": traffic,
                      "encode_frac": algo_bytes / (enc_avg * 1e-3) / 1e9 / peak,
                      "decode_frac": algo_bytes / (dec_avg * 1e-3) / 1e9 / peak},
         "gpu_launches": 2 * args.steps,
-        "kernels": {"encode": ["fp64", "tcgen05", "fp32"][tc.tc_last_path(ctx, False)],
-                    "decode": ["fp64", "tcgen05", "fp32"][tc.tc_last_path(ctx, True)]},
+        "kernels": {"encode": kernels[0], "decode": kernels[1]},
         "clocks": clocks,
     }
     if e2e is not None:
