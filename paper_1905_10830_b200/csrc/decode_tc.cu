@@ -703,7 +703,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
 
 bool tc_decode_tc_supported(const tc_ctx *ctx, const DecodeArgs &a)
 {
-    if (a.c % 16 != 0 || a.k != a.c || a.c > 256) return false;
+    // K <= C leading components (PCA truncation): K is the reduction dimension of the MMA
+    if (a.c % 16 != 0 || a.k % 16 != 0 || a.k < 16 || a.k > a.c || a.c > 256) return false;
     if (a.splits != 1 && !(a.splits == 2 && a.chunk_pixels == 1 && a.k % 32 == 0)) return false;
     if (a.groups != 1 && a.groups != a.k) return false;
     if (a.lut_bits > TC_MAX_CODE_LEN) return false;

@@ -584,7 +584,8 @@ static int enc_table_entries(const EncodeArgs &a)
 
 bool tc_encode_tc_supported(const tc_ctx *ctx, const EncodeArgs &a)
 {
-    if (a.c % 16 != 0 || a.k != a.c || a.c > 256 || a.hw % 4 != 0) return false;
+    // K <= C leading components (PCA truncation): K is the N dimension of the MMA
+    if (a.c % 16 != 0 || a.k % 16 != 0 || a.k < 16 || a.k > a.c || a.c > 256 || a.hw % 4 != 0) return false;
     // two chunks per pixel must coincide with the two halves the epilogue threads work on
     if (a.splits != 1 && !(a.splits == 2 && a.k % 32 == 0)) return false;
     if (a.groups != 1 && a.groups != a.k) return false;

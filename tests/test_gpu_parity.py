@@ -64,16 +64,16 @@ def check_stream_against_oracle(enc, q_gpu, lengths, bits):
 
 
 def run_case(ctx, spec, bits, n_cal, n_test, dtype, per_channel, *, exact, chunk_pixels=0, pixel_splits=0, model=None,
-             routes=None):
+             routes=None, k=None):
     """`routes`: the kernels expected for (encode, decode): 0 fp64, 1 tensor core, 2 fp32."""
     if routes is None:
         routes = (0, 0) if exact else (1, 1)
-    o = H.oracle_side(spec, bits, n_cal, n_test, dtype, per_channel, model=model)
+    o = H.oracle_side(spec, bits, n_cal, n_test, dtype, per_channel, model=model, k=k)
     m, lengths = o["model"], o["lengths"]
     model_h = H.import_model(tc, ctx, m, dtype)
     cb = tc.tc_codebook_import(ctx, lengths, bits)
     x = o["x"].cuda()
-    enc = tc.tc_encode(ctx, model_h, cb, x, chunk_pixels=chunk_pixels, pixel_splits=pixel_splits, debug=True)
+    enc = tc.tc_encode(ctx, model_h, cb, x, chunk_pixels=chunk_pixels, pixel_splits=pixel_splits, debug=True, k=m.k)
     assert tc.tc_get_status(ctx) == 0
     assert tc.tc_last_path(ctx) == routes[0], "unexpected kernel route"
     # coefficients
@@ -197,6 +197,31 @@ def test_tensor_core_path_pixel_splits(ctx_tc, c, splits):
 def test_four_splits_take_the_fp32_kernels(ctx_tc):
     spec = fm.LayerSpec(64, 14, 14, 0.9, None, 5400)
     run_case(ctx_tc, spec, 4, 6, 3, torch.bfloat16, False, exact=False, chunk_pixels=1, pixel_splits=4, routes=(2, 2))
+
+
+# ---- PCA truncation: only the K leading components are coded (Section 4, ablation) -----------
+
+@pytest.mark.parametrize("c,k,dtype,bits", [(64, 32, torch.float32, 6), (64, 8, torch.float32, 4), (96, 40, torch.bfloat16, 5)])
+def test_truncation_exact_path(ctx, c, k, dtype, bits):
+    spec = fm.LayerSpec(c, 12, 12, 0.9, None, 5700 + c + k)
+    _, enc = run_case(ctx, spec, bits, 6, 3, dtype, False, exact=True, k=k)
+    assert enc.symbols.shape[1] == k
+    run_case(ctx, spec, bits, 6, 3, dtype, True, exact=True, k=k)
+
+
+@pytest.mark.parametrize("c,k,bits,splits", [(256, 128, 4, 0), (256, 64, 4, 0), (256, 160, 5, 2), (128, 32, 6, 0),
+                                             (192, 96, 3, 1), (64, 16, 4, 0), (256, 256, 4, 1)])
+def test_truncation_tensor_core_path(ctx_tc, c, k, bits, splits):
+    spec = fm.LayerSpec(c, 14, 14, 0.9, None, 5800 + c + k)
+    _, enc = run_case(ctx_tc, spec, bits, 6, 5, torch.bfloat16, False, exact=False, k=k, pixel_splits=splits,
+                      chunk_pixels=1 if splits else 0)
+    assert enc.symbols.shape[1] == k
+
+
+def test_truncation_fp32_route(ctx_tc):
+    # K not a multiple of 16, and a wide layer
+    run_case(ctx_tc, fm.LayerSpec(64, 14, 14, 0.9, None, 5900), 5, 6, 3, torch.bfloat16, False, exact=False, k=24, routes=(2, 2))
+    run_case(ctx_tc, fm.LayerSpec(512, 7, 7, 0.95, None, 5901), 4, 12, 5, torch.bfloat16, False, exact=False, k=128, routes=(2, 2))
 
 
 # ---- fp32 kernels: bf16 tensors of shapes the tensor-core kernels do not take -----------------
