@@ -166,13 +166,6 @@ struct SmemWindowReader {
         lo = __funnelshift_l(0u, lo, e);
         avail -= (int)(e & 31u);
     }
-    // nbits < 32
-    __device__ __forceinline__ void skip_bits(int nbits)
-    {
-        hi = __funnelshift_l(lo, hi, nbits);
-        lo <<= nbits;
-        avail -= nbits;
-    }
     __device__ __forceinline__ void refill()
     {
         asm volatile(
@@ -437,9 +430,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
 
             // walks this thread's chunk; `fill_panel(dst, k0, nk8)` decodes the next 8 * nk8 symbols
             // (coefficients k0 ...) into the operand row at shared address `dst`
-            // (`every_lane`: the filler is called by all 32 lanes of the warp, with `store` telling
-            // whether the lane has a pixel to decode -- needed when the filler votes across the warp)
-            auto decode_chunk = [&](auto &&fill_panel, bool every_lane) {
+            auto decode_chunk = [&](auto &&fill_panel) {
                 for (int pp = 0; pp < cp && alive; ++pp) {
                     const bool decode = pp < n_pix;
                     const int row = t * cp + pp;       // only meaningful while the chunk exists
@@ -449,11 +440,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
                         const int s = sub * 2 + slot;
                         if (pp == 0 && !mbar_wait(smem_u32(&s_empty[grp][s]), phase ^ 1u, 200u)) { alive = false; break; }
                         if (++slot == sub_slots) { slot = 0; phase ^= 1u; }
-                        if (decode || every_lane) {
+                        if (decode) {
                             const int k0 = k_first + kp * panel_k;
                             const int nk8 = min(panel_k, k_end - k0) >> 3;
-                            const uint32_t dst = ring_g + s * slot_bytes + ((row & 127) >> 3) * 128 + (row & 7) * 16;
-                            fill_panel(dst, k0, nk8, decode);
+                            const uint32_t dst = ring_g + s * slot_bytes + (row >> 3) * 128 + (row & 7) * 16;
+                            fill_panel(dst, k0, nk8);
                         }
                         // (the issuing thread makes the panel visible to the tensor core's proxy)
                         if (pp == cp - 1) mbar_arrive(smem_u32(&s_full[grp][s]));
@@ -462,7 +453,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
             };
             // symbol by symbol: eight symbols -> one 16-byte store
             auto by_pairs = [&](auto &&next_pair) {
-                return [&, next_pair](uint32_t dst, int k0, int nk8, bool) mutable {
+                return [&, next_pair](uint32_t dst, int k0, int nk8) mutable {
                     for (int k8 = 0; k8 < nk8; ++k8) {
                         uint32_t pk[4];
 #pragma unroll
@@ -482,7 +473,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
                 if (active) r.init(seg_addr, chunk_start);
                 else r.idle(seg_addr);
                 const int lb = a.lut_bits;
-                decode_chunk([&](uint32_t dst, int k0, int nk8, bool) {
+                decode_chunk([&](uint32_t dst, int k0, int nk8) {
                     for (int k8 = 0; k8 < nk8; ++k8) {
                         uint32_t pk[4];
 #pragma unroll
@@ -497,7 +488,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
                         asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + k8 * 2048), "r"(pk[0]),
                                      "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
                     }
-                }, false);
+                });
                 // a chunk must end exactly where its recorded length says
                 if (active && r.consumed(seg_addr, chunk_start) != chunk_bits) bad = true;
             } else if (cur.ok && cur.staged) {
@@ -512,7 +503,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
                     const uint32_t e1 = __ldg(a.lut32 + (size_t)(j + 1) * lut_size + r.peek(a.lut_bits));
                     r.skip_entry(e1);
                     return __byte_perm(centre(e0), centre(e1), 0x7632);
-                }), false);
+                }));
                 if (active && r.consumed(seg_addr, chunk_start) != chunk_bits) bad = true;
             } else {
                 WindowReader r;
@@ -528,7 +519,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
                     r.skip((int)(e1 & 0xffu));
                     used += (e0 & 0xffu) + (e1 & 0xffu);
                     return __byte_perm(centre(e0), centre(e1), 0x7632);
-                }), false);
+                }));
                 if (active && used != chunk_bits) bad = true;
             }
             for (int kp = 0; kp < n_panels; ++kp)
