@@ -42,7 +42,7 @@ def lib() -> C.CDLL:
             "orc_round_bf16": (d, [d]),
             "orc_mean_cov": (None, [vp, i64, i32, i64, vp, vp]),
             "orc_eigh_jacobi": (i32, [vp, i32, vp, vp]),
-            "orc_fit_pca": (i32, [vp, i64, i32, i64, i32, i32, vp, vp, vp, vp, vp, vp, vp]),
+            "orc_fit_pca": (i32, [vp, i64, i32, i64, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]),
             "orc_project": (None, [vp, i64, i32, i64, vp, vp, i32, vp]),
             "orc_quantize": (None, [vp, i64, d, d, i32, vp, vp]),
             "orc_histogram": (None, [vp, i64, i32, i32, i32, vp]),
@@ -86,7 +86,8 @@ class Model:
     eig: np.ndarray       # [C] float64, descending
     lo: float
     step: float
-    basis_round: str = "f64"   # "f64", "bf16" or "f32": how the basis was rounded at fit time
+    basis_round: str = "f64"   # "f64", "bf16", "f32" or "int8": how the basis was rounded at fit time
+    basis_scale: float = 1.0   # "int8": every basis entry is an integer in [-127, 127] times this
 
 
 @dataclass
@@ -144,7 +145,7 @@ def fit_pca(x, bits: int, *, k: int | None = None, basis_bf16: bool = False,
             basis_round: str | None = None, eigensolver: str = "auto") -> Model:
     """Fit mean, basis and quantiser range on calibration maps.
 
-    basis_round: "f64" (keep), "bf16" or "f32".  eigensolver: "jacobi" (the in-file solver),
+    basis_round: "f64" (keep), "bf16", "f32" or "int8" (8-bit matrix with one scale).  eigensolver: "jacobi" (the in-file solver),
     "lapack" (numpy.linalg.eigh, a library primitive used as one step) or "auto" = Jacobi up
     to JACOBI_MAX_C channels, LAPACK beyond (Jacobi needs minutes there).
     """
@@ -152,7 +153,7 @@ def fit_pca(x, bits: int, *, k: int | None = None, basis_bf16: bool = False,
     n, c, h, w = x.shape
     if basis_round is None:
         basis_round = "bf16" if basis_bf16 else "f64"
-    mode = {"f64": 0, "bf16": 1, "f32": 2}[basis_round]
+    mode = {"f64": 0, "bf16": 1, "f32": 2, "int8": 3}[basis_round]
     if eigensolver == "auto":
         eigensolver = "jacobi" if c <= JACOBI_MAX_C else "lapack"
     pre_ev = pre_vt = None
@@ -166,21 +167,22 @@ def fit_pca(x, bits: int, *, k: int | None = None, basis_bf16: bool = False,
     eig = np.zeros(c)
     lo = C.c_double()
     step = C.c_double()
+    scale = C.c_double()
     rc = lib().orc_fit_pca(_p(x), n, c, h * w, bits, mode,
                            _p(pre_ev) if pre_ev is not None else None,
                            _p(pre_vt) if pre_vt is not None else None,
-                           _p(mean), _p(basis), _p(eig), C.byref(lo), C.byref(step))
+                           _p(mean), _p(basis), _p(eig), C.byref(lo), C.byref(step), C.byref(scale))
     if rc != 0:
         raise RuntimeError("oracle eigensolver did not converge")
     return Model(c, c if k is None else k, bits, mean, basis, eig, lo.value, step.value,
-                 basis_round)
+                 basis_round, scale.value)
 
 
 def with_bits(m: Model, bits: int) -> Model:
     """The same transform with the calibration range divided into 2^bits - 1 steps."""
     hi = m.lo + m.step * ((1 << m.bits) - 1)
     return Model(m.c, m.k, bits, m.mean, m.basis, m.eig, m.lo, (hi - m.lo) / ((1 << bits) - 1),
-                 m.basis_round)
+                 m.basis_round, m.basis_scale)
 
 
 def project(model: Model, x) -> np.ndarray:

@@ -138,13 +138,17 @@ int orc_eigh_jacobi(double *a, int n, double *evals, double *vt)
  * highest-variance channel, with step = (hi - lo) / (2^bits - 1).
  * basis_round: 0 keeps fp64; 1 rounds every entry of the basis to bfloat16, 2 to fp32 (ties to
  * even) before the range pass, and that rounded matrix is the transform from then on.
+ * 3 quantises the matrix to 8 bits (Section 3.1 says the PCA matrix is stored in 8 bits; the
+ * quantiser is this reading: one scale s = max|T| / 127 for the whole matrix, every entry
+ * becomes s * rint(T / s), an integer in [-127, 127] times s); *basis_scale receives s (1.0 in
+ * the other modes).  The decoder uses the transpose of the same quantised matrix.
  * The eigendecomposition is the in-file Jacobi solver, unless the caller passes one it
  * obtained from a library routine (pre_evals[c], pre_vt[c][c] with unit eigenvectors as rows,
  * any order): Jacobi takes minutes beyond a few hundred channels.
  * Returns 0, or -1 if the eigensolver did not converge. */
 int orc_fit_pca(const float *x, int64_t n, int c, int64_t hw, int bits, int basis_round,
                 const double *pre_evals, const double *pre_vt,
-                double *mean, double *basis, double *eig, double *lo, double *step)
+                double *mean, double *basis, double *eig, double *lo, double *step, double *basis_scale)
 {
     double *cov = (double *)malloc(sizeof(double) * (size_t)c * c);
     double *ev = (double *)malloc(sizeof(double) * (size_t)c);
@@ -178,6 +182,14 @@ int orc_fit_pca(const float *x, int64_t n, int c, int64_t hw, int bits, int basi
         }
         eig[j] = ev[order[j]];
     }
+    double scale = 1.0;
+    if (basis_round == 3) {
+        double biggest = 0.0;
+        for (int64_t i = 0; i < (int64_t)c * c; ++i) if (fabs(basis[i]) > biggest) biggest = fabs(basis[i]);
+        scale = biggest / 127.0;
+        for (int64_t i = 0; i < (int64_t)c * c; ++i) basis[i] = scale * rint(basis[i] / scale);
+    }
+    if (basis_scale) *basis_scale = scale;
     double mn = INFINITY, mx = -INFINITY;
     for (int64_t i = 0; i < n; ++i)
         for (int64_t t = 0; t < hw; ++t) {
