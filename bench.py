@@ -166,6 +166,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--bits", type=int, default=4)
     ap.add_argument("--k", type=int, default=0, help="code only the K leading components (0 = all C)")
+    ap.add_argument("--basis", default="bf16", choices=["bf16", "int8"], help="precision the fitted basis is stored in")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (smaller captures)")
     ap.add_argument("--sample-images", type=int, default=0, help="images per oracle timing sample")
@@ -203,7 +204,8 @@ def main():
     # ---- set-up (untimed): fit, statistics, codebook -- all through the library ---------
     ctx = tc.tc_create(local_rank)
     cal = fm.make_maps(params, w.calib_maps, calib=True, dtype=w.dtype, device=dev)
-    model = tc.tc_fit_pca(ctx, cal, bits=bits, k=args.k)
+    model = tc.tc_fit_pca(ctx, cal, bits=bits, k=args.k,
+                          basis_dtype=tc.binding.TC_INT8 if args.basis == "int8" else None)
     st = tc.tc_stats(ctx, model, None, cal, groups=1)
     cb = tc.tc_build_codebook(ctx, model, st.hist, groups=1)
     x = fm.make_maps(params, batch, dtype=w.dtype, device=dev, offset=rank)   # each rank its own maps
@@ -303,7 +305,7 @@ def main():
     # launch processes: every tile is read and written once, so traffic grows with the batch.
     # Only quoted for the configuration the counters were taken on.
     traffic = None
-    if bits == 4 and args.k == 0 and kernels == ("tcgen05", "tcgen05") and lay.pixel_splits == 2:
+    if bits == 4 and args.k == 0 and args.basis == "bf16" and kernels == ("tcgen05", "tcgen05") and lay.pixel_splits == 2:
         traffic = NCU_DRAM_BYTES_PER_VALUE[dominant] * values
     line = {
         "metric": METRIC,
@@ -311,7 +313,7 @@ def main():
         "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": w.name, "layer": spec.name, "batch_per_gpu": batch, "bits": bits, "k": args.k or spec.c,
+        "config": {"workload": w.name, "layer": spec.name, "batch_per_gpu": batch, "bits": bits, "k": args.k or spec.c, "basis": args.basis,
                    "chunk_pixels": lay.chunk_pixels, "pixel_splits": lay.pixel_splits, "codebook": "per-layer", "calib_maps": w.calib_maps,
                    "l2": "inputs larger than L2 (411 MB per pass), no flush", "parallelism": f"batch-sharded x{world}"},
         "encode_gbs": raw_bytes / (enc_avg * 1e-3) / 1e9, "decode_gbs": raw_bytes / (dec_avg * 1e-3) / 1e9,

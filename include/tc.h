@@ -45,7 +45,8 @@ typedef enum {
     TC_ERR_NOT_CONVERGED = 7     /* eigensolver did not converge                              */
 } tc_status;
 
-typedef enum { TC_F32 = 0, TC_BF16 = 1 } tc_dtype;
+/* Element types.  TC_INT8 is not a tensor type: it only names the 8-bit basis of a model. */
+typedef enum { TC_F32 = 0, TC_BF16 = 1, TC_INT8 = 2 } tc_dtype;
 
 /* Dense NCHW tensor in DEVICE memory. `data` must be aligned to its element size. */
 typedef struct {
@@ -89,7 +90,11 @@ typedef struct {
     int32_t k;           /* coefficients kept, 1..C; 0 means C                             */
     int32_t basis_dtype; /* tc_dtype: the basis is rounded to this type at fit time and
                             the rounded matrix is the transform from then on.  TC_BF16 is
-                            required for bf16 tensors, TC_F32 for fp32 tensors.            */
+                            required for bf16 tensors, TC_F32 for fp32 tensors.  TC_INT8
+                            (Section 3.1: the PCA matrix is stored in 8 bits) serves both:
+                            one scale s = max|T| / 127 for the matrix, every entry becomes
+                            s * n with n an integer in [-127, 127]; the decoder uses the
+                            transpose of the same matrix.                                   */
 } tc_fit_params;
 
 /* Fit on calibration maps (`calib->n` maps).  Mean and covariance (1/(M-1), M = n*h*w pixel
@@ -109,6 +114,9 @@ typedef struct {
     double *basis; /* HOST [c*c] */
     double *mean;  /* HOST [c]   */
     double *eig;   /* HOST [c], may be NULL on import */
+    double basis_scale; /* TC_INT8 basis: the scale s (every basis entry is an integer in
+                           [-127, 127] times s, checked on import); otherwise ignored on
+                           import and 1.0 on export */
 } tc_model_desc;
 
 tc_status tc_model_import(tc_ctx *ctx, const tc_model_desc *desc, tc_model **out);

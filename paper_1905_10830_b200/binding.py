@@ -11,7 +11,7 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_PKG, "libtc_b200.so")
 
-TC_F32, TC_BF16 = 0, 1
+TC_F32, TC_BF16, TC_INT8 = 0, 1, 2       # TC_INT8 only names the 8-bit basis of a model
 _STATUS = ["ok", "invalid argument", "unsupported configuration", "output buffer too small",
            "CUDA error", "corrupt stream", "device-side wait timed out",
            "eigensolver did not converge"]
@@ -36,7 +36,7 @@ class _FitParams(C.Structure):
 class _ModelDesc(C.Structure):
     _fields_ = [("c", C.c_int32), ("k", C.c_int32), ("bits", C.c_int32), ("basis_dtype", C.c_int32),
                 ("lo", C.c_double), ("step", C.c_double), ("basis", C.c_void_p),
-                ("mean", C.c_void_p), ("eig", C.c_void_p)]
+                ("mean", C.c_void_p), ("eig", C.c_void_p), ("basis_scale", C.c_double)]
 
 
 class _CodebookParams(C.Structure):
@@ -238,13 +238,14 @@ def tc_fit_pca(ctx: Context, calib: torch.Tensor, bits: int, k: int = 0, basis_d
 
 
 def tc_model_import(ctx: Context, *, basis: np.ndarray, mean: np.ndarray, lo: float, step: float, bits: int,
-                    basis_dtype: int, k: int | None = None, eig: np.ndarray | None = None) -> Model:
+                    basis_dtype: int, k: int | None = None, eig: np.ndarray | None = None,
+                    basis_scale: float = 1.0) -> Model:
     basis = np.ascontiguousarray(basis, dtype=np.float64)
     mean = np.ascontiguousarray(mean, dtype=np.float64)
     c = basis.shape[0]
     eig_arr = None if eig is None else np.ascontiguousarray(eig, dtype=np.float64)
     d = _ModelDesc(c, c if k is None else k, bits, basis_dtype, lo, step, basis.ctypes.data, mean.ctypes.data,
-                   None if eig_arr is None else eig_arr.ctypes.data)
+                   None if eig_arr is None else eig_arr.ctypes.data, basis_scale)
     out = C.c_void_p()
     _check(load_library().tc_model_import(ctx.ptr, C.byref(d), C.byref(out)), "tc_model_import")
     return Model(out.value)
@@ -259,7 +260,7 @@ def tc_model_export(model: Model) -> dict:
     d.basis, d.mean, d.eig = basis.ctypes.data, mean.ctypes.data, eig.ctypes.data
     _check(load_library().tc_model_export(model.ptr, C.byref(d)), "tc_model_export")
     return dict(c=d.c, k=d.k, bits=d.bits, basis_dtype=d.basis_dtype, lo=d.lo, step=d.step, basis=basis,
-                mean=mean, eig=eig)
+                mean=mean, eig=eig, basis_scale=d.basis_scale)
 
 
 def tc_build_codebook(ctx: Context, model: Model, hist, *, groups: int = 1, max_length: int = 0) -> Codebook:

@@ -97,7 +97,7 @@ __global__ void __launch_bounds__(kThreads) encode_simt_kernel(EncodeArgs a)
                         acc[4 * q4 + 3] = fmaf(w.w, xv, acc[4 * q4 + 3]);
                     }
                 }
-                const float inv_step = (float)(1.0 / a.step);
+                const float inv_step = (float)(a.basis_scale / a.step);     // the operand holds basis / basis_scale
 #pragma unroll
                 for (int jj = 0; jj < RB; ++jj) {
                     const int j = j0 + jj;
@@ -107,7 +107,7 @@ __global__ void __launch_bounds__(kThreads) encode_simt_kernel(EncodeArgs a)
                         const float r = fminf(fmaxf(rintf(u), 0.f), (float)top);
                         const unsigned int q = (unsigned int)r;
                         s_q[j * kThreads + t] = (uint8_t)q;
-                        if (a.dbg_coef) a.dbg_coef[p * a.k + j] = acc[jj] - a.tmu32[j];
+                        if (a.dbg_coef) a.dbg_coef[p * a.k + j] = fmaf(acc[jj], (float)a.basis_scale, -a.tmu32[j]);
                         if (a.dbg_sym) a.dbg_sym[p * a.k + j] = (uint8_t)q;
                     }
                 }
@@ -354,7 +354,7 @@ __global__ void __launch_bounds__(kThreads) decode_simt_kernel(DecodeArgs a)
                         acc[4 * q4 + 3] = fmaf(w.w, qv, acc[4 * q4 + 3]);
                     }
                 }
-                const float step = (float)a.step;
+                const float step = (float)(a.step * a.basis_scale);        // the operand holds basis / basis_scale
 #pragma unroll
                 for (int cc = 0; cc < RB; ++cc)
                     if (c0 + cc < a.c)

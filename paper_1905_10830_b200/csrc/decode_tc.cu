@@ -544,7 +544,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
         const int col_first = n_blocks == 2 ? 0 : 64 * set, col_count = n_blocks == 2 ? 128 : 64;
         const int ch = blk * 128 + wq * 32 + lane;
         const bool ch_ok = ch < a.c;
-        const float step = (float)a.step;
+        const float step = (float)(a.step * a.basis_scale);        // the operand holds basis / basis_scale
         const float bias = ch_ok ? a.dec_bias[ch] : 0.f;
         __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(a.xhat);
         // With H*W a multiple of 4 every aligned group of four pixels lies inside one image and is

@@ -87,7 +87,7 @@ extern "C" tc_status tc_encode_noalloc(tc_ctx *ctx, const tc_model *m, const tc_
     a.basis64 = m->d_basis64; a.mean64 = m->d_mean64; a.lo = m->lo; a.step = m->step;
     a.enc = cb->d_enc; a.stream = (uint32_t *)stream_out;
     a.capacity_bits = (unsigned long long)(capacity & ~(size_t)15) * 8ull;
-    a.chunk_len = chunk_len; a.tile_off = (unsigned long long *)tile_off;
+    a.chunk_len = chunk_len; a.tile_off = (unsigned long long *)tile_off; a.basis_scale = m->basis_scale;
     a.dbg_coef = nullptr; a.dbg_sym = nullptr;
     a.ticket = (unsigned int *)scratch;
     a.tile_state = (unsigned long long *)((char *)scratch + kScratchHeader);

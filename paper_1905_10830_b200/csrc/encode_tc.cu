@@ -320,7 +320,8 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
         const uint32_t pair_len_rel = smem_u32(smem + L.len8) - kMagicBits * (1u + (1u << a.bits));   // same for a pair sum
         unsigned short *xch = reinterpret_cast<unsigned short *>(smem + L.xch) + grp * 256;   // [2][128] lengths exchanged between the halves
         long long n_done = 0;                      // tiles this group has handed to its store warp
-        const float inv_step = (float)(1.0 / a.step);
+        const float inv_step = (float)(a.basis_scale / a.step);   // the operand holds basis / basis_scale
+        const float coef_scale = (float)a.basis_scale;
         const float vmax = kMagic + (float)(nsym - 1);
         const int bar_id = 1 + grp;
         bool alive = true;
@@ -372,7 +373,7 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
                             my_bits += l;
                         }
                         if constexpr (kDebug) {
-                            if (valid && a.dbg_coef) a.dbg_coef[p * a.k + j] = __uint_as_float(r[i]) - a.tmu32[j];
+                            if (valid && a.dbg_coef) a.dbg_coef[p * a.k + j] = fmaf(__uint_as_float(r[i]), coef_scale, -a.tmu32[j]);
                             if (valid && a.dbg_sym) a.dbg_sym[p * a.k + j] = (uint8_t)(vb & 0xffu);
                         }
                         r[i] = vb;

@@ -110,11 +110,14 @@ tc_status finish_model(tc_model *m)
     if ((st = upload(&m->d_enc_bias, enc_bias)) != TC_OK) return st;
     if ((st = upload(&m->d_dec_bias, dec_bias)) != TC_OK) return st;
     if ((st = upload(&m->d_tmu32, tmu32)) != TC_OK) return st;
-    if (m->basis_dtype == TC_BF16) {
+    if (m->basis_dtype == TC_BF16 || m->basis_dtype == TC_INT8) {
+        // an 8-bit basis goes to the bf16 kernels as its integers (exact in bf16); the scale is
+        // folded into their quantiser and dequantiser constants
         std::vector<__nv_bfloat16> b((size_t)k * c), bt((size_t)c * k);
         for (int j = 0; j < k; ++j)
             for (int a = 0; a < c; ++a) {
-                const __nv_bfloat16 v = __float2bfloat16((float)m->basis[(size_t)j * c + a]);
+                const __nv_bfloat16 v = __float2bfloat16((float)(m->basis_dtype == TC_INT8 ? std::nearbyint(m->basis[(size_t)j * c + a] / m->basis_scale)
+                                                                                          : m->basis[(size_t)j * c + a]));
                 b[(size_t)j * c + a] = v;
                 bt[(size_t)a * k + j] = v;
             }
@@ -259,14 +262,24 @@ tc_status tc_model_import(tc_ctx *ctx, const tc_model_desc *d, tc_model **out)
     *out = nullptr;
     if (d->c < 1 || d->k < 1 || d->k > d->c || !(d->step > 0.0) || !std::isfinite(d->lo)) return TC_ERR_INVALID_ARG;
     if (d->bits < 1 || d->bits > 8 || d->c > TC_MAX_C) return TC_ERR_UNSUPPORTED;
-    if (d->basis_dtype != TC_F32 && d->basis_dtype != TC_BF16) return TC_ERR_INVALID_ARG;
-    for (size_t i = 0; i < (size_t)d->c * d->c; ++i)
-        if (round_to_dtype(d->basis[i], d->basis_dtype) != d->basis[i]) return TC_ERR_INVALID_ARG;
+    if (d->basis_dtype != TC_F32 && d->basis_dtype != TC_BF16 && d->basis_dtype != TC_INT8) return TC_ERR_INVALID_ARG;
+    if (d->basis_dtype == TC_INT8) {
+        // every entry must be an integer in [-127, 127] times the scale
+        if (!(d->basis_scale > 0.0) || !std::isfinite(d->basis_scale)) return TC_ERR_INVALID_ARG;
+        for (size_t i = 0; i < (size_t)d->c * d->c; ++i) {
+            const double n = d->basis[i] / d->basis_scale;
+            if (std::fabs(n - std::nearbyint(n)) > 1e-9 || std::fabs(n) > 127.0 + 1e-9) return TC_ERR_INVALID_ARG;
+        }
+    } else {
+        for (size_t i = 0; i < (size_t)d->c * d->c; ++i)
+            if (round_to_dtype(d->basis[i], d->basis_dtype) != d->basis[i]) return TC_ERR_INVALID_ARG;
+    }
     DeviceGuard guard(ctx->device);
     tc_model *m = new (std::nothrow) tc_model();
     if (!m) return TC_ERR_CUDA;
     m->c = d->c; m->k = d->k; m->bits = d->bits; m->basis_dtype = d->basis_dtype;
     m->lo = d->lo; m->step = d->step; m->device = ctx->device;
+    m->basis_scale = d->basis_dtype == TC_INT8 ? d->basis_scale : 1.0;
     m->basis.assign(d->basis, d->basis + (size_t)d->c * d->c);
     m->mean.assign(d->mean, d->mean + d->c);
     if (d->eig) m->eig.assign(d->eig, d->eig + d->c); else m->eig.assign(d->c, 0.0);
@@ -280,7 +293,7 @@ tc_status tc_model_export(const tc_model *m, tc_model_desc *d)
 {
     if (!m || !d) return TC_ERR_INVALID_ARG;
     d->c = m->c; d->k = m->k; d->bits = m->bits; d->basis_dtype = m->basis_dtype;
-    d->lo = m->lo; d->step = m->step;
+    d->lo = m->lo; d->step = m->step; d->basis_scale = m->basis_scale;
     if (d->basis) std::copy(m->basis.begin(), m->basis.end(), d->basis);
     if (d->mean) std::copy(m->mean.begin(), m->mean.end(), d->mean);
     if (d->eig) std::copy(m->eig.begin(), m->eig.end(), d->eig);
@@ -306,7 +319,7 @@ tc_status tc_fit_pca(tc_ctx *ctx, const tc_tensor *calib, const tc_fit_params *p
     if (params->bits < 1 || params->bits > 8 || c > TC_MAX_C) return TC_ERR_UNSUPPORTED;
     const int k = params->k ? params->k : c;
     if (k < 1 || k > c) return TC_ERR_INVALID_ARG;
-    if (params->basis_dtype != TC_F32 && params->basis_dtype != TC_BF16) return TC_ERR_INVALID_ARG;
+    if (params->basis_dtype != TC_F32 && params->basis_dtype != TC_BF16 && params->basis_dtype != TC_INT8) return TC_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     cudaStream_t s = (cudaStream_t)cuda_stream;
 
@@ -338,7 +351,15 @@ tc_status tc_fit_pca(tc_ctx *ctx, const tc_tensor *calib, const tc_fit_params *p
         }
     std::vector<double> eig(c), basis((size_t)c * c);
     if (tc_eigh_host(cov.data(), c, eig.data(), basis.data()) != 0) return TC_ERR_NOT_CONVERGED;
-    for (double &v : basis) v = round_to_dtype(v, params->basis_dtype);
+    double basis_scale = 1.0;
+    if (params->basis_dtype == TC_INT8) {
+        double biggest = 0.0;
+        for (double v : basis) biggest = std::max(biggest, std::fabs(v));
+        basis_scale = biggest / 127.0;
+        for (double &v : basis) v = basis_scale * std::nearbyint(v / basis_scale);
+    } else {
+        for (double &v : basis) v = round_to_dtype(v, params->basis_dtype);
+    }
 
     TC_CUDA(cudaMemcpyAsync(d_row0, basis.data(), sizeof(double) * c, cudaMemcpyHostToDevice, s));
     int blocks = 0;
@@ -354,7 +375,7 @@ tc_status tc_fit_pca(tc_ctx *ctx, const tc_tensor *calib, const tc_fit_params *p
     tc_model_desc d;
     d.c = c; d.k = k; d.bits = params->bits; d.basis_dtype = params->basis_dtype;
     d.lo = lo; d.step = (hi - lo) / (double)((1 << params->bits) - 1);
-    d.basis = basis.data(); d.mean = mean.data(); d.eig = eig.data();
+    d.basis = basis.data(); d.mean = mean.data(); d.eig = eig.data(); d.basis_scale = basis_scale;
     return tc_model_import(ctx, &d, out);
 }
 
@@ -445,7 +466,7 @@ static tc_status check_codec_args(const tc_model *m, const tc_codebook *cb, cons
     if (!m || !cb || !valid_tensor(x)) return TC_ERR_INVALID_ARG;
     if (x->c != m->c || cb->bits != m->bits) return TC_ERR_INVALID_ARG;
     if (cb->groups != 1 && cb->groups != m->k) return TC_ERR_INVALID_ARG;
-    if (x->dtype != m->basis_dtype) return TC_ERR_UNSUPPORTED;
+    if (x->dtype != m->basis_dtype && m->basis_dtype != TC_INT8) return TC_ERR_UNSUPPORTED;   // an 8-bit basis serves both tensor types
     if ((long long)x->n * x->h * x->w > (1ll << 40)) return TC_ERR_UNSUPPORTED;
     return TC_OK;
 }
@@ -499,7 +520,7 @@ tc_status tc_encode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
     a.basis64 = m->d_basis64; a.mean64 = m->d_mean64; a.lo = m->lo; a.step = m->step;
     a.enc = cb->d_enc; a.stream = (uint32_t *)stream_out;
     a.capacity_bits = (unsigned long long)(capacity & ~(size_t)15) * 8ull;
-    a.chunk_len = chunk_len; a.tile_off = (unsigned long long *)tile_off;
+    a.chunk_len = chunk_len; a.tile_off = (unsigned long long *)tile_off; a.basis_scale = m->basis_scale;
     a.dbg_coef = debug ? debug->coefficients : nullptr;
     a.dbg_sym = debug ? debug->symbols : nullptr;
     a.ticket = (unsigned int *)ctx->scratch;
@@ -538,7 +559,7 @@ tc_status tc_decode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
     a.n = x_hat->n; a.c = x_hat->c; a.hw = x_hat->h * x_hat->w; a.k = m->k; a.bits = m->bits; a.groups = cb->groups;
     a.pixels = pixels; a.n_tiles = (pixels + TC_TILE_PIXELS - 1) / TC_TILE_PIXELS; a.n_chunks = cs.chunks(pixels);
     a.chunk_pixels = cs.cp; a.lut_bits = cb->lut_bits; a.lut = cb->d_lut;
-    a.basis64 = m->d_basis64; a.mean64 = m->d_mean64; a.lo = m->lo; a.step = m->step;
+    a.basis64 = m->d_basis64; a.mean64 = m->d_mean64; a.lo = m->lo; a.step = m->step; a.basis_scale = m->basis_scale;
     a.xhat = x_hat->data; a.status = ctx->d_status;
     a.lut32 = cb->d_lut32; a.basis_t_bf16 = m->d_basis_t_bf16; a.dec_bias = m->d_dec_bias; a.center = m->center;
     if (!ctx->force_exact && x_hat->dtype == TC_BF16 && tc_decode_tc_supported(ctx, a)) {
@@ -600,7 +621,7 @@ tc_status tc_stats(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const 
 {
     if (!ctx || !m || !out || !valid_tensor(x)) return TC_ERR_INVALID_ARG;
     if (x->c != m->c) return TC_ERR_INVALID_ARG;
-    if (x->dtype != m->basis_dtype) return TC_ERR_UNSUPPORTED;
+    if (x->dtype != m->basis_dtype && m->basis_dtype != TC_INT8) return TC_ERR_UNSUPPORTED;   // an 8-bit basis serves both tensor types
     if (out->groups != 1 && out->groups != m->k) return TC_ERR_INVALID_ARG;
     if (cb && (cb->bits != m->bits || (cb->groups != 1 && cb->groups != m->k))) return TC_ERR_INVALID_ARG;
     const long long pixels = (long long)x->n * x->h * x->w;
@@ -629,7 +650,7 @@ tc_status tc_stats(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const 
     EncodeArgs e{};
     e.x = x->data; e.n = x->n; e.c = x->c; e.hw = x->h * x->w; e.k = m->k; e.bits = m->bits; e.groups = 1;
     e.pixels = pixels; e.n_tiles = (pixels + TC_TILE_PIXELS - 1) / TC_TILE_PIXELS; e.chunk_pixels = 1; e.splits = 1;
-    e.basis64 = m->d_basis64; e.mean64 = m->d_mean64; e.lo = m->lo; e.step = m->step;
+    e.basis64 = m->d_basis64; e.mean64 = m->d_mean64; e.lo = m->lo; e.step = m->step; e.basis_scale = m->basis_scale;
     e.enc = nullptr; e.dbg_sym = d_sym; e.status = ctx->d_status; e.clamped = d_clamped; e.emit = 0;
     e.bits = m->bits;
     // statistics mode stages no code table: give it an empty one
@@ -641,7 +662,7 @@ tc_status tc_stats(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const 
     DecodeArgs d{};
     d.symbols = d_sym; d.n = x->n; d.c = x->c; d.hw = x->h * x->w; d.k = m->k; d.bits = m->bits; d.groups = 1;
     d.pixels = pixels; d.n_tiles = e.n_tiles; d.n_chunks = pixels; d.chunk_pixels = 1; d.splits = 1;
-    d.basis64 = m->d_basis64; d.mean64 = m->d_mean64; d.lo = m->lo; d.step = m->step;
+    d.basis64 = m->d_basis64; d.mean64 = m->d_mean64; d.lo = m->lo; d.step = m->step; d.basis_scale = m->basis_scale;
     d.xhat = d_xhat; d.status = ctx->d_status;
     if ((st = tc_launch_decode_simt(ctx, d, x->dtype, s)) != TC_OK) return st;
     if ((st = tc_launch_sqerr(x->data, d_xhat, x->dtype, (long long)values, d_sq, d_zeros, s)) != TC_OK) return st;

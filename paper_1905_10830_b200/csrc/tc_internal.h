@@ -36,13 +36,14 @@ struct tc_ctx {
 struct tc_model {
     int c = 0, k = 0, bits = 0, basis_dtype = 0;
     double lo = 0, step = 0;
+    double basis_scale = 1.0;               // 8-bit basis: entries are integers times this; 1 otherwise
     int center = 0;                         // symbol whose level is nearest to y = 0
     std::vector<double> basis, mean, eig;   // host copies (basis [c][c])
     int device = 0;
     // device copies
     double *d_basis64 = nullptr;            // [c][c] exact values of the (rounded) basis
     double *d_mean64 = nullptr;             // [c]
-    __nv_bfloat16 *d_basis_bf16 = nullptr;  // [k][c]   (bf16 models only)
+    __nv_bfloat16 *d_basis_bf16 = nullptr;  // [k][c]   bf16 basis, or the integers of an 8-bit basis (exact in bf16)
     __nv_bfloat16 *d_basis_t_bf16 = nullptr;// [c][k]   transpose, for the inverse projection
     float *d_enc_bias = nullptr;            // [k]  -(T mu + lo)_j / step
     float *d_dec_bias = nullptr;            // [c]  mu_c + (lo + center*step) * sum_j T[j][c]
@@ -73,6 +74,7 @@ struct EncodeArgs {
     const float *enc_bias;      // [k]  -(T mu + lo)_j / step
     const float *tmu32;         // [k]  (T mu)_j
     double lo, step;
+    double basis_scale;         // basis_bf16 holds basis / basis_scale (8-bit basis: integers); 1 otherwise
     const uint32_t *enc;        // [groups][2^bits]
     uint32_t *stream;           // output words
     unsigned long long capacity_bits;
@@ -108,6 +110,7 @@ struct DecodeArgs {
     const double *basis64;
     const double *mean64;
     double lo, step;
+    double basis_scale;                 // basis_t_bf16 holds basis / basis_scale
     void *xhat;
     unsigned int *status;
 };

@@ -15,13 +15,14 @@ def basis_round_for(dtype) -> str:
 
 
 def oracle_side(spec: fm.LayerSpec, bits: int, n_cal: int, n_test: int, dtype, per_channel: bool,
-                lmax: int = 12, model: oracle.Model | None = None, k: int | None = None):
+                lmax: int = 12, model: oracle.Model | None = None, k: int | None = None,
+                basis_round: str | None = None):
     """Returns dict(model, lengths, cal, x, y, q, units) computed by the oracle on CPU maps."""
     params = fm.layer_params(spec)
     cal = fm.make_maps(params, n_cal, calib=True, dtype=dtype)
     x = fm.make_maps(params, n_test, dtype=dtype)
     if model is None:
-        model = oracle.fit_pca(cal, bits, basis_round=basis_round_for(dtype), k=k)
+        model = oracle.fit_pca(cal, bits, basis_round=basis_round or basis_round_for(dtype), k=k)
     elif model.bits != bits:
         model = oracle.with_bits(model, bits)
     q_cal = oracle.quantize(model, oracle.project(model, cal))
@@ -32,9 +33,12 @@ def oracle_side(spec: fm.LayerSpec, bits: int, n_cal: int, n_test: int, dtype, p
 
 
 def import_model(tc, ctx, m: oracle.Model, dtype):
+    if m.basis_round == "int8":
+        basis_dtype = tc.binding.TC_INT8
+    else:
+        basis_dtype = tc.binding.TC_BF16 if dtype == torch.bfloat16 else tc.binding.TC_F32
     return tc.tc_model_import(ctx, basis=m.basis, mean=m.mean, lo=m.lo, step=m.step, bits=m.bits,
-                              basis_dtype=tc.binding.TC_BF16 if dtype == torch.bfloat16 else tc.binding.TC_F32,
-                              k=m.k, eig=m.eig)
+                              basis_dtype=basis_dtype, k=m.k, eig=m.eig, basis_scale=m.basis_scale)
 
 
 def stream_words(enc) -> np.ndarray:

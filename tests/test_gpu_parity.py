@@ -64,11 +64,11 @@ def check_stream_against_oracle(enc, q_gpu, lengths, bits):
 
 
 def run_case(ctx, spec, bits, n_cal, n_test, dtype, per_channel, *, exact, chunk_pixels=0, pixel_splits=0, model=None,
-             routes=None, k=None):
+             routes=None, k=None, basis_round=None):
     """`routes`: the kernels expected for (encode, decode): 0 fp64, 1 tensor core, 2 fp32."""
     if routes is None:
         routes = (0, 0) if exact else (1, 1)
-    o = H.oracle_side(spec, bits, n_cal, n_test, dtype, per_channel, model=model, k=k)
+    o = H.oracle_side(spec, bits, n_cal, n_test, dtype, per_channel, model=model, k=k, basis_round=basis_round)
     m, lengths = o["model"], o["lengths"]
     model_h = H.import_model(tc, ctx, m, dtype)
     cb = tc.tc_codebook_import(ctx, lengths, bits)
@@ -222,6 +222,59 @@ def test_truncation_fp32_route(ctx_tc):
     # K not a multiple of 16, and a wide layer
     run_case(ctx_tc, fm.LayerSpec(64, 14, 14, 0.9, None, 5900), 5, 6, 3, torch.bfloat16, False, exact=False, k=24, routes=(2, 2))
     run_case(ctx_tc, fm.LayerSpec(512, 7, 7, 0.95, None, 5901), 4, 12, 5, torch.bfloat16, False, exact=False, k=128, routes=(2, 2))
+
+
+# ---- 8-bit basis (Section 3.1: the PCA matrix is stored in 8 bits) -------------------------------
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_int8_basis_exact_path(ctx, dtype):
+    spec = fm.LayerSpec(48, 12, 12, 0.9, None, 6000)
+    o, _ = run_case(ctx, spec, 6, 6, 3, dtype, False, exact=True, basis_round="int8")
+    assert o["model"].basis_round == "int8"
+    run_case(ctx, spec, 4, 6, 3, dtype, True, exact=True, basis_round="int8", k=16)
+
+
+@pytest.mark.parametrize("c,s,bits,k", [(256, 14, 4, None), (128, 28, 6, None), (64, 28, 8, None), (256, 14, 5, 96)])
+def test_int8_basis_tensor_core_path(ctx_tc, c, s, bits, k):
+    spec = fm.LayerSpec(c, s, s, 0.9, None, 6100 + c)
+    run_case(ctx_tc, spec, bits, 6, 4, torch.bfloat16, False, exact=False, basis_round="int8", k=k)
+
+
+def test_int8_basis_fp32_route(ctx_tc):
+    run_case(ctx_tc, fm.LayerSpec(384, 7, 7, 0.95, None, 6200), 5, 16, 4, torch.bfloat16, False, exact=False,
+             basis_round="int8", routes=(2, 2))
+
+
+def test_library_fit_with_int8_basis_matches_the_oracle(ctx_tc):
+    spec = fm.LayerSpec(64, 14, 14, 0.9, None, 6300)
+    params = fm.layer_params(spec)
+    cal = fm.make_maps(params, 8, calib=True, dtype=torch.bfloat16)
+    want = oracle.fit_pca(cal, 5, basis_round="int8")
+    model = tc.tc_fit_pca(ctx_tc, cal.cuda(), 5, basis_dtype=tc.binding.TC_INT8)
+    got = tc.tc_model_export(model)
+    assert got["basis_dtype"] == tc.binding.TC_INT8
+    n_got, n_want = got["basis"] / got["basis_scale"], want.basis / want.basis_scale
+    assert np.abs(n_got - np.rint(n_got)).max() <= 1e-9 and np.abs(n_got).max() == 127
+    assert np.isclose(got["basis_scale"], want.basis_scale, rtol=1e-9)
+    # the two eigensolvers agree to rounding: an entry may land on the neighbouring integer at a tie
+    assert np.abs(np.rint(n_got) - np.rint(n_want)).max() <= 1
+    assert (np.rint(n_got) == np.rint(n_want)).mean() >= 0.999
+    assert np.isclose(got["lo"], want.lo, rtol=1e-6, atol=1e-6) and np.isclose(got["step"], want.step, rtol=1e-6)
+    # the fitted model codes a bf16 tensor on the tensor-core kernels and an fp32 one on the fp64 kernels
+    x = fm.make_maps(params, 3, dtype=torch.bfloat16).cuda()
+    st = tc.tc_stats(ctx_tc, model, None, cal.cuda())
+    cb = tc.tc_build_codebook(ctx_tc, model, st.hist)
+    enc = tc.tc_encode(ctx_tc, model, cb, x)
+    assert tc.tc_last_path(ctx_tc) == 1
+    a = tc.tc_decode(ctx_tc, model, cb, enc, x.shape, torch.bfloat16)
+    enc32 = tc.tc_encode(ctx_tc, model, cb, x.float())
+    assert tc.tc_last_path(ctx_tc) == 0
+    b = tc.tc_decode(ctx_tc, model, cb, enc32, x.shape, torch.float32)
+    assert tc.tc_get_status(ctx_tc) == 0
+    assert torch.equal(enc.words[: enc.total_bits() // 8], enc32.words[: enc32.total_bits() // 8]) or \
+        (enc.total_bits() - enc32.total_bits()) ** 2 < 1e-6 * enc.total_bits() ** 2
+    assert (a.float() - b).abs().max().item() <= 0.02 * b.abs().max().item()
+    model.close(); cb.close()
 
 
 # ---- fp32 kernels: bf16 tensors of shapes the tensor-core kernels do not take -----------------
