@@ -293,7 +293,7 @@ def main():
         return
 
     peak, peak_src = measured_peaks()
-    kernels = (["fp64", "tcgen05", "fp32"][tc.tc_last_path(ctx, False)], ["fp64", "tcgen05", "fp32"][tc.tc_last_path(ctx, True)])
+    kernels = (["fp64", "tcgen05", "fp32", "tcgen05-stream"][tc.tc_last_path(ctx, False)], ["fp64", "tcgen05", "fp32", "tcgen05-stream"][tc.tc_last_path(ctx, True)])
     enc_avg, dec_avg = statistics.mean(enc_ms), statistics.mean(dec_ms)
     algo_bytes = raw_bytes + stream_bytes + side_bytes          # per launch, either direction
     dominant = "encode" if enc_avg >= dec_avg else "decode"

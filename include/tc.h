@@ -69,12 +69,16 @@ const char *tc_status_string(tc_status s);
 tc_status tc_get_status(tc_ctx *ctx, void *cuda_stream);
 
 /* Validation switch.  bf16 tensors normally take the tensor-core kernels (bf16 products, fp32
- * accumulation) or, for shapes those do not take (more than 256 channels, odd map sizes), plain
- * fp32 kernels with the same arithmetic; fp32 tensors run on kernels that evaluate the
- * definition in fp64.  With `on` != 0 every tensor takes the fp64 kernels. */
+ * accumulation): up to 256 channels with rows of H*W % 4 == 0 elements the kernels that keep
+ * the basis in shared memory, wider layers (up to 1024 channels) and other map sizes the
+ * kernels that stream it; shapes neither takes (channel or coefficient counts that are not
+ * multiples of 16) run on plain fp32 kernels with the same arithmetic.  fp32 tensors run on
+ * kernels that evaluate the definition in fp64.  With `on` != 0 every tensor takes the fp64
+ * kernels. */
 void tc_force_exact_path(tc_ctx *ctx, int on);
 /* Which kernels the last tc_encode (decode == 0) or tc_decode (decode != 0) of this context
- * launched: 0 = fp64 kernels, 1 = tensor-core kernels, 2 = fp32 kernels; -1 for a NULL
+ * launched: 0 = fp64 kernels, 1 = tensor-core kernels with the basis resident in shared
+ * memory, 2 = fp32 kernels, 3 = tensor-core kernels that stream the basis; -1 for a NULL
  * context. */
 int tc_last_path(const tc_ctx *ctx, int decode);
 

@@ -85,52 +85,6 @@ __host__ __device__ inline SmemLayout smem_layout(int c, int k, int lut_entries,
     return l;
 }
 
-// MSB-first reader over 32-bit words with a 64-bit window held in two registers.  Words at or
-// past `end` read as zero, so a corrupt offset can never cause an out-of-bounds load.
-struct WindowReader {
-    const uint32_t *words;
-    unsigned long long next, end;     // word indices
-    uint32_t hi, lo;                  // upcoming bits, left-aligned in hi:lo
-    int avail;                        // valid bits in the window
-
-    __device__ __forceinline__ uint32_t fetch()
-    {
-        const uint32_t w = (next < end) ? __ldg(words + next) : 0u;
-        ++next;
-        return w;
-    }
-    __device__ __forceinline__ void init(const uint32_t *base, unsigned long long bitpos, unsigned long long end_bits)
-    {
-        words = base;
-        next = bitpos >> 5;
-        end = end_bits >> 5;
-        const uint32_t w0 = fetch(), w1 = fetch();
-        const int sh = (int)(bitpos & 31);
-        hi = __funnelshift_l(w1, w0, sh);
-        lo = w1 << sh;
-        avail = 64 - sh;
-    }
-    __device__ __forceinline__ uint32_t peek(int nbits) const { return hi >> (32 - nbits); }
-    // nbits < 32
-    __device__ __forceinline__ void skip(int nbits)
-    {
-        hi = __funnelshift_l(lo, hi, nbits);
-        lo <<= nbits;
-        avail -= nbits;
-    }
-    // keeps more than 32 valid bits in the window
-    __device__ __forceinline__ void refill()
-    {
-        if (avail <= 32) {
-            const uint32_t w = fetch();
-            const int s = 32 - avail;                 // 0..31
-            hi |= __funnelshift_l(w, 0u, s);
-            lo |= w << s;
-            avail += 32;
-        }
-    }
-};
-
 // The same reader over a segment staged in shared memory.  The word after the window is kept
 // in a register, so that the shared-memory load of a refill is off the critical path, and the
 // refill is predicated rather than branched.

@@ -1,0 +1,379 @@
+// Tensor-core decode for bf16 tensors of more than 256 channels (Section 3: VLD, inverse
+// quantiser, inverse transform), where neither the transposed basis nor a double-buffered
+// accumulator for every channel fits on chip.
+//
+// One persistent block per SM walks work items of NP pixels: a whole tile of 128 pixels up to
+// 512 channels, half a tile beyond (the accumulators of all channels, NP columns per block of
+// 128 channels, fill tensor memory exactly).  Per item:
+//   warps 0-7     VLD: one thread per chunk walks the bit stream (global memory, table-driven
+//                 canonical Huffman) and writes the symbols minus the centre symbol, as exact
+//                 bf16 integers, into the K-major B operand, which holds all K coefficients of
+//                 the item's pixels (2 K NP bytes)
+//   warps 16-19   loaders: the transposed basis streams from L2 through a ring of
+//                 128-channel x 64-coefficient panels (cp.async, K-major core matrices)
+//   warp 20       one thread issues tcgen05.mma:  D[c][pixel] += T[j][c] * (Q[pixel][j] - center)
+//   warps 8-15    epilogue: TMEM -> registers (lane = channel), x_hat = step * acc + bias_c,
+//                 round to bf16, NCHW stores; runs while the VLD warps decode the next item
+// Dequantisation is folded as in the resident-basis kernel:
+// bias_c = mu_c + (lo + center * step) * sum_j T[j][c].
+#include "device_utils.cuh"
+#include "sm100_ptx.cuh"
+
+namespace {
+
+using namespace tcdev;
+using namespace sm100;
+
+constexpr int kVldThreads = 256;
+constexpr int kEpiWarp0 = 8, kLoaderWarp0 = 16, kMmaWarp = 20;
+constexpr int kThreads = 21 * 32;
+constexpr int kTmemCols = 512;
+constexpr int kPanelK = 64;                                   // coefficients per ring stage
+constexpr int kStageBytes = 128 * kPanelK * 2;                // 16 KB: 128 channels x 64 coefficients
+constexpr int kMaxStages = 6;
+constexpr int kLag = 2;
+constexpr int kVldBar = 1;
+constexpr int kMaxTileChunks = 512;
+
+struct SmemLayout {
+    uint32_t ring, bop, lut, start, total;
+    int stages, np;
+};
+
+__host__ __device__ inline SmemLayout smem_layout(int c, int k, int lut_entries, int budget)
+{
+    SmemLayout l;
+    l.np = ((c + 127) / 128 <= 4) ? 128 : 64;
+    const uint32_t bop_bytes = 2u * (uint32_t)k * (uint32_t)l.np;
+    const uint32_t fixed = bop_bytes + (uint32_t)lut_entries * 4u + (kMaxTileChunks + 8) * 4u;
+    int stages = ((long long)budget - (long long)fixed) / kStageBytes;
+    if (stages > kMaxStages) stages = kMaxStages;
+    l.stages = stages < 2 ? 0 : stages;
+    l.ring = 0;
+    l.bop = (uint32_t)(l.stages * kStageBytes);
+    l.lut = l.bop + bop_bytes;
+    l.start = l.lut + (uint32_t)lut_entries * 4u;
+    l.total = l.start + (kMaxTileChunks + 8) * 4u;
+    return l;
+}
+
+template <bool kPerChannel>
+__global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ __align__(8) unsigned long long s_full[kMaxStages], s_empty[kMaxStages];
+    __shared__ __align__(8) unsigned long long s_bfull, s_bfree, s_tfull, s_tempty;
+    __shared__ uint32_t s_tmem_base;
+    __shared__ unsigned int s_wsum[8];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int lut_size = 1 << a.lut_bits;
+    const SmemLayout L = smem_layout(a.c, a.k, kPerChannel ? 0 : lut_size, a.smem_budget);
+    const int stages = L.stages, NP = L.np;
+    const uint32_t ring_addr = smem_u32(smem + L.ring);
+    const uint32_t bop_addr = smem_u32(smem + L.bop);
+    uint32_t *s_lut = reinterpret_cast<uint32_t *>(smem + L.lut);
+    unsigned int *s_start = reinterpret_cast<unsigned int *>(smem + L.start);     // start of every chunk of the tile, then the tile's bits
+    const int n_cblocks = (a.c + 127) / 128;                  // blocks of 128 channels
+    const int n_kpanels = (a.k + kPanelK - 1) / kPanelK;
+    const int items_per_tile = TC_TILE_PIXELS / NP;
+    const long long n_items = a.n_tiles * items_per_tile;
+    const long long my_items = (n_items > blockIdx.x) ? (n_items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+
+    // ---- set-up ---------------------------------------------------------------------
+    if (tid == 0) {
+        for (int s = 0; s < kMaxStages; ++s) { mbar_init(smem_u32(&s_full[s]), 128); mbar_init(smem_u32(&s_empty[s]), 1); }
+        mbar_init(smem_u32(&s_bfull), kVldThreads);
+        mbar_init(smem_u32(&s_bfree), 1);
+        mbar_init(smem_u32(&s_tfull), 1);
+        mbar_init(smem_u32(&s_tempty), 256);
+        mbar_fence_init();
+    }
+    if (warp == kMmaWarp) { tmem_alloc(smem_u32(&s_tmem_base), kTmemCols); tmem_relinquish(); }
+    if (!kPerChannel)
+        for (int i = tid; i < lut_size; i += kThreads) {
+            // per-layer table: bf16(symbol - center) << 16 | code length
+            const uint32_t e = a.lut32[i];
+            const float f = (float)((int)((e >> 8) & 0xffu) - a.center);
+            s_lut[i] = (__float_as_uint(f) & 0xffff0000u) | (e & 0xffu);
+        }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = s_tmem_base;
+
+    if (warp < kEpiWarp0) {
+        // ================= VLD =================
+        const int t = tid;                                    // 0..255
+        const int S = a.splits, cp = a.chunk_pixels;
+        const int chunks_per_tile = S * TC_TILE_PIXELS / cp;  // at most 512
+        const int k_sub = a.k / S;
+        const int item_chunks = S * NP / cp;
+        const int pix_chunks = NP / cp;                       // chunks of one run of coefficients in an item
+        const uint32_t row_bytes = (uint32_t)NP * 16u;        // one group of 8 coefficients of all the item's pixels
+        bool alive = true;
+        for (long long n = 0; n < my_items && alive; ++n) {
+            const long long item = blockIdx.x + n * gridDim.x;
+            const long long tile = item / items_per_tile;
+            const int h = (int)(item - tile * items_per_tile);
+            // chunk lengths of the tile -> start positions (exclusive scan over 2 x 256 values)
+            const unsigned long long base = a.tile_off[tile], end = a.tile_off[tile + 1];
+            const bool tile_ok = (base & 127ull) == 0 && (end & 127ull) == 0 && base <= end && end <= a.stream_bits;
+            unsigned int l0 = 0, l1 = 0;
+            {
+                const long long ch = tile * chunks_per_tile + 2 * t;
+                if (2 * t < chunks_per_tile && ch < a.n_chunks) l0 = a.chunk_len[ch];
+                if (2 * t + 1 < chunks_per_tile && ch + 1 < a.n_chunks) l1 = a.chunk_len[ch + 1];
+            }
+            unsigned int inc = l0 + l1;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const unsigned int up = __shfl_up_sync(0xffffffffu, inc, d);
+                if (lane >= d) inc += up;
+            }
+            // the B operand and the start positions are free once the previous item's MMAs are done
+            if (!mbar_wait(smem_u32(&s_bfree), (uint32_t)((n & 1) ^ 1))) { alive = false; break; }
+            if (lane == 31) s_wsum[warp] = inc;
+            named_bar_sync(kVldBar, kVldThreads);
+            unsigned int before = 0, tile_total = 0;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) {
+                const unsigned int sw = s_wsum[w];
+                if (w < warp) before += sw;
+                tile_total += sw;
+            }
+            const unsigned int excl = before + inc - (l0 + l1);
+            if (2 * t < kMaxTileChunks) { s_start[2 * t] = excl; s_start[2 * t + 1] = excl + l0; }
+            named_bar_sync(kVldBar, kVldThreads);
+            bool bad = !tile_ok || (unsigned long long)tile_total > end - base;
+
+            for (int u = t; u < item_chunks && !bad; u += kVldThreads) {
+                // chunk u of the item: run `sub` of the coefficients of pixel(s) r0 ...
+                const int sub = u / pix_chunks, cidx = u - sub * pix_chunks;
+                const int r0 = cidx * cp;                                     // first pixel inside the item
+                const int ci = (h * NP + r0) / cp * S + sub;                  // chunk inside the tile (S > 1 only with cp = 1)
+                const long long p0 = tile * TC_TILE_PIXELS + h * NP + r0;
+                if (p0 >= a.pixels) continue;
+                const int n_pix = (int)min((long long)cp, a.pixels - p0);
+                const unsigned int start = s_start[ci], want = (ci + 1 < chunks_per_tile ? s_start[ci + 1] : tile_total) - start;
+                WindowReader r;
+                r.init(a.stream, base + start, end);
+                unsigned int used = 0;
+                const int k_first = sub * k_sub;
+                for (int pp = 0; pp < n_pix; ++pp) {
+                    const uint32_t dst = bop_addr + (uint32_t)(k_first >> 3) * row_bytes + (uint32_t)(r0 + pp) * 16u;
+                    for (int k8 = 0; k8 < (k_sub >> 3); ++k8) {
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            r.refill();
+                            uint32_t v0, v1, len0, len1;
+                            if constexpr (kPerChannel) {
+                                const int j = k_first + k8 * 8 + 2 * i;
+                                const uint32_t e0 = __ldg(a.lut32 + (size_t)j * lut_size + r.peek(a.lut_bits));
+                                len0 = e0 & 0xffu;
+                                r.skip((int)len0);
+                                const uint32_t e1 = __ldg(a.lut32 + (size_t)(j + 1) * lut_size + r.peek(a.lut_bits));
+                                len1 = e1 & 0xffu;
+                                r.skip((int)len1);
+                                v0 = __float_as_uint((float)((int)((e0 >> 8) & 0xffu) - a.center));
+                                v1 = __float_as_uint((float)((int)((e1 >> 8) & 0xffu) - a.center));
+                            } else {
+                                v0 = s_lut[r.peek(a.lut_bits)];
+                                len0 = v0 & 0xffu;
+                                r.skip((int)len0);
+                                v1 = s_lut[r.peek(a.lut_bits)];
+                                len1 = v1 & 0xffu;
+                                r.skip((int)len1);
+                            }
+                            used += len0 + len1;
+                            pk[i] = __byte_perm(v0, v1, 0x7632);
+                        }
+                        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (uint32_t)k8 * row_bytes), "r"(pk[0]),
+                                     "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
+                    }
+                }
+                // a chunk must end exactly where its recorded length says
+                if (used != want) bad = true;
+            }
+            if (bad) tc_dev_set_status(a.status, TC_ERR_CORRUPT_STREAM);
+            // the writes become visible to the tensor core's proxy, then the operand is handed over
+            fence_proxy_async_smem();
+            mbar_arrive(smem_u32(&s_bfull));
+        }
+        if (!alive && t == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
+    } else if (warp < kLoaderWarp0) {
+        // ================= epilogue =================
+        const int ew = warp - kEpiWarp0;
+        const int set = ew >> 2, wq = ew & 3;                // two sets of four warps take alternate channel blocks
+        const float step = (float)(a.step * a.basis_scale);  // the operand holds basis / basis_scale
+        __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(a.xhat);
+        const bool vec = (a.hw & 3) == 0;                    // four aligned pixels lie inside one image, 8-byte aligned
+        const long long img_stride = (long long)a.c * a.hw;
+        bool alive = true;
+        for (long long n = 0; n < my_items && alive; ++n) {
+            const long long item = blockIdx.x + n * gridDim.x;
+            const long long p_first = item * NP;
+            const long long left = a.pixels - p_first;
+            const int n_valid = (int)(left < (long long)NP ? (left < 0 ? 0 : left) : (long long)NP);
+            const long long img0 = left > 0 ? p_first / a.hw : 0;
+            const int s0 = left > 0 ? (int)(p_first - img0 * a.hw) : 0;
+            if (!mbar_wait(smem_u32(&s_tfull), (uint32_t)(n & 1))) { alive = false; break; }
+            tc_fence_after_sync();
+            for (int blk = set; blk < n_cblocks; blk += 2) {
+                const int ch = blk * 128 + wq * 32 + lane;
+                const bool ch_ok = ch < a.c;
+                const float bias = ch_ok ? __ldg(a.dec_bias + ch) : 0.f;
+                const uint32_t trow = tmem_base + (uint32_t)(blk * NP) + ((uint32_t)(wq * 32) << 16);
+                int s = s0;
+                __nv_bfloat16 *dst = out + img0 * img_stride + (long long)(ch_ok ? ch : 0) * a.hw + s;
+                for (int c0 = 0; c0 < NP; c0 += 16) {
+                    uint32_t r[16];
+                    tmem_ld_32x32b_x16(trow + c0, r);
+                    tmem_ld_wait();
+                    if (vec) {
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) {
+                            const __nv_bfloat162 h0 = __floats2bfloat162_rn(fmaf(__uint_as_float(r[4 * g]), step, bias),
+                                                                            fmaf(__uint_as_float(r[4 * g + 1]), step, bias));
+                            const __nv_bfloat162 h1 = __floats2bfloat162_rn(fmaf(__uint_as_float(r[4 * g + 2]), step, bias),
+                                                                            fmaf(__uint_as_float(r[4 * g + 3]), step, bias));
+                            if (ch_ok && c0 + 4 * g < n_valid)
+                                *reinterpret_cast<uint2 *>(dst) = make_uint2(*reinterpret_cast<const uint32_t *>(&h0),
+                                                                             *reinterpret_cast<const uint32_t *>(&h1));
+                            s += 4;
+                            const bool wrap = s >= a.hw;          // the next group starts the next image
+                            dst += wrap ? 4 + img_stride - a.hw : 4;
+                            s = wrap ? s - a.hw : s;
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const __nv_bfloat16 hv = __float2bfloat16_rn(fmaf(__uint_as_float(r[i]), step, bias));
+                            if (ch_ok && c0 + i < n_valid) *dst = hv;
+                            s += 1;
+                            const bool wrap = s == a.hw;
+                            dst += wrap ? 1 + img_stride - a.hw : 1;
+                            s = wrap ? 0 : s;
+                        }
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            mbar_arrive(smem_u32(&s_tempty));
+        }
+        if (!alive && lane == 0 && ew == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
+    } else if (warp < kMmaWarp) {
+        // ================= loaders =================
+        const int lt = tid - kLoaderWarp0 * 32;               // 0..127
+        int it = 0;
+        bool alive = true;
+        for (long long n = 0; n < my_items && alive; ++n) {
+            for (int jp = 0; jp < n_kpanels && alive; ++jp) {
+                const int j0 = jp * kPanelK;
+                const int nk8 = min(kPanelK, a.k - j0) >> 3;
+                for (int blk = 0; blk < n_cblocks; ++blk, ++it) {
+                    const int s = it % stages;
+                    if (!mbar_wait(smem_u32(&s_empty[s]), ((it / stages) & 1) ^ 1)) { alive = false; break; }
+                    const uint32_t stage = ring_addr + s * kStageBytes;
+                    // transposed basis rows (channels) blk * 128 ..., coefficients j0 ...: K-major core
+                    // matrices (row / 8) * 1024 + (j / 8) * 128 + (row % 8) * 16; rows past C are zero
+                    for (int i = lt; i < 128 * 8; i += 128) {
+                        const int row = i >> 3, j8 = i & 7;
+                        const int ch = blk * 128 + row;
+                        const bool ok = ch < a.c && j8 < nk8;
+                        cp_async_16(stage + (row >> 3) * 1024 + j8 * 128 + (row & 7) * 16,
+                                    a.basis_t_bf16 + (ok ? (long long)ch * a.k + j0 + j8 * 8 : 0), ok ? 16u : 0u);
+                    }
+                    cp_async_commit();
+                    if (it >= kLag) {
+                        cp_async_wait<kLag>();
+                        fence_proxy_async_smem();
+                        mbar_arrive(smem_u32(&s_full[(it - kLag) % stages]));
+                    }
+                }
+            }
+        }
+        if (alive) {
+            if (it >= 2) { cp_async_wait<1>(); fence_proxy_async_smem(); mbar_arrive(smem_u32(&s_full[(it - 2) % stages])); }
+            if (it >= 1) { cp_async_wait<0>(); fence_proxy_async_smem(); mbar_arrive(smem_u32(&s_full[(it - 1) % stages])); }
+        } else {
+            cp_async_wait<0>();
+            tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
+        }
+    } else {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            // A = transposed basis (128 channels per instruction), B = the decoded symbols of NP pixels
+            const uint32_t idesc = make_idesc_bf16(128, NP, /*A K-major*/ false, /*B K-major*/ false);
+            const uint32_t b_lbo = (uint32_t)NP * 16u;
+            int it = 0;
+            bool alive = true;
+            for (long long n = 0; n < my_items && alive; ++n) {
+                if (!mbar_wait(smem_u32(&s_bfull), (uint32_t)(n & 1))) { alive = false; break; }
+                if (!mbar_wait(smem_u32(&s_tempty), (uint32_t)((n & 1) ^ 1))) { alive = false; break; }
+                fence_proxy_async_smem();
+                tc_fence_after_sync();
+                for (int jp = 0; jp < n_kpanels && alive; ++jp) {
+                    const int j0 = jp * kPanelK;
+                    const int nk16 = min(kPanelK, a.k - j0) >> 4;
+                    for (int blk = 0; blk < n_cblocks; ++blk, ++it) {
+                        const int s = it % stages;
+                        if (!mbar_wait(smem_u32(&s_full[s]), (it / stages) & 1)) { alive = false; break; }
+                        tc_fence_after_sync();
+                        const uint32_t stage = ring_addr + s * kStageBytes;
+                        for (int q = 0; q < nk16; ++q) {
+                            const uint64_t adesc = make_smem_desc(stage + q * 256, 128, 1024);
+                            const uint64_t bdesc = make_smem_desc(bop_addr + (uint32_t)((j0 + 16 * q) >> 3) * b_lbo, b_lbo, 128);
+                            mma_bf16_ss(tmem_base + (uint32_t)(blk * NP), adesc, bdesc, idesc, (jp | q) != 0 ? 1u : 0u);
+                        }
+                        mma_commit(smem_u32(&s_empty[s]));
+                    }
+                }
+                if (alive) {
+                    mma_commit(smem_u32(&s_tfull));
+                    mma_commit(smem_u32(&s_bfree));
+                }
+            }
+            if (!alive) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
+        }
+    }
+
+    // ---- teardown ---------------------------------------------------------------------
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == kMmaWarp) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+}  // namespace
+
+bool tc_decode_wide_supported(const tc_ctx *ctx, const DecodeArgs &a)
+{
+    if (a.c % 16 != 0 || a.k % 16 != 0 || a.k < 16 || a.k > a.c || a.c > TC_MAX_C) return false;
+    if (a.splits != 1 && a.splits != 2 && a.splits != 4) return false;
+    if (a.splits > 1 && (a.chunk_pixels != 1 || a.k % a.splits != 0 || (a.k / a.splits) % 8 != 0)) return false;
+    if (a.groups != 1 && a.groups != a.k) return false;
+    if (a.lut_bits > TC_MAX_CODE_LEN) return false;
+    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, ctx->max_smem_optin - 1024);
+    if (l.stages < 2) return false;
+    return a.chunk_pixels <= l.np;                            // a chunk lies inside one work item
+}
+
+tc_status tc_launch_decode_wide(const tc_ctx *ctx, const DecodeArgs &a, cudaStream_t s)
+{
+    if (a.n_tiles <= 0) return TC_OK;
+    DecodeArgs args = a;
+    args.smem_budget = ctx->max_smem_optin - 1024;            // leaves room for the static shared variables
+    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, args.smem_budget);
+    if (l.stages < 2) return TC_ERR_UNSUPPORTED;
+    void (*kernel)(DecodeArgs) = a.groups != 1 ? decode_wide_kernel<true> : decode_wide_kernel<false>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.total) != cudaSuccess)
+        return TC_ERR_CUDA;
+    const long long n_items = a.n_tiles * (TC_TILE_PIXELS / l.np);
+    const unsigned int grid = (unsigned int)((n_items < ctx->sm_count) ? n_items : ctx->sm_count);
+    kernel<<<grid, kThreads, l.total, s>>>(args);
+    return cudaGetLastError() == cudaSuccess ? TC_OK : TC_ERR_CUDA;
+}

@@ -1,0 +1,446 @@
+// Tensor-core encode for bf16 tensors the resident-basis kernel does not take: up to 1024
+// channels (the basis no longer fits shared memory) and map sizes whose rows are not 8-byte
+// aligned (7 x 7).  Section 3: transform, quantiser, VLC.
+//
+// One persistent block per SM walks tiles of 128 consecutive pixels.  The coefficients of a
+// tile are produced in blocks of up to 256 (one accumulator of tensor memory each, two
+// accumulators in flight); for every block the pixels' channels stream through a ring of
+// 32-channel panels together with the matching 256 x 32 piece of the basis, both read from L2.
+//   warps 0-7     epilogue: warps 0-3 take the first half of a block's coefficients, warps 4-7
+//                 the second half.  Pass 1 (per block): TMEM -> registers, quantise, code length,
+//                 symbols parked in shared memory (one byte each, K x 128 per tile), bits added up
+//                 per run of coefficients.  Then: bit offsets (scan over the pixels, tile
+//                 look-back), chunk lengths.  Pass 2: codes of the parked symbols packed straight
+//                 into the (zeroed) stream words.
+//   warps 8-11    loaders: cp.async (or, for unaligned rows, plain 2-byte loads) into the MMA's
+//                 shared-memory layouts
+//   warp 12       one thread issues tcgen05.mma:  D[pixel][coef] = X[pixel][c] * T[coef][c]
+#include <cstdio>
+#include <cstdlib>
+
+#include "device_utils.cuh"
+#include "sm100_ptx.cuh"
+
+namespace {
+
+using namespace tcdev;
+using namespace sm100;
+
+constexpr int kPanelCh = 32;                                  // channels per ring stage
+constexpr int kBlockCoef = 256;                               // coefficients per accumulator
+constexpr int kStageA = kPanelCh * TC_TILE_PIXELS * 2;        // 8 KB: pixels x channels
+constexpr int kStageB = kBlockCoef * kPanelCh * 2;            // 16 KB: coefficients x channels
+constexpr int kStageBytes = kStageA + kStageB;
+constexpr int kMaxStages = 4;
+constexpr int kLag = 2;                                       // cp.async groups in flight per loader thread
+constexpr int kLoaderWarp0 = 8, kMmaWarp = 12;          // warps 0-7 are the epilogue
+constexpr int kThreads = 13 * 32;
+constexpr int kTmemCols = 512;
+constexpr int kEpiBar = 1;                                    // named barrier of the 256 epilogue threads
+
+struct SmemLayout {
+    uint32_t ring, symq, part, bias, enc, len8, total;
+    int stages;
+};
+
+__host__ __device__ inline SmemLayout smem_layout(int k, int enc_entries, int budget)
+{
+    SmemLayout l;
+    const uint32_t fixed = (uint32_t)k * TC_TILE_PIXELS + 4u * TC_TILE_PIXELS * 4u + (uint32_t)k * 4u +
+                           (uint32_t)enc_entries * 4u + (((uint32_t)enc_entries + 15u) & ~15u);
+    int stages = ((long long)budget - (long long)fixed) / kStageBytes;
+    if (stages > kMaxStages) stages = kMaxStages;
+    l.stages = stages < 2 ? 0 : stages;
+    l.ring = 0;
+    l.symq = (uint32_t)(l.stages * kStageBytes);              // [K / 4][128] words: four symbols of one pixel
+    l.part = l.symq + (uint32_t)k * TC_TILE_PIXELS;           // [4][128] bits of each run of coefficients
+    l.bias = l.part + 4u * TC_TILE_PIXELS * 4u;
+    l.enc = l.bias + (uint32_t)k * 4u;                        // per-layer table: code << 8 | length
+    l.len8 = l.enc + (uint32_t)enc_entries * 4u;              // and the lengths once more as bytes
+    l.total = l.len8 + (((uint32_t)enc_entries + 15u) & ~15u);
+    return l;
+}
+
+// Quantiser in fp32 (the same arithmetic as the resident-basis kernel): v = acc/step + bias,
+// rounded to the nearest integer (ties to even) by adding 1.5 * 2^23, clamped while a float.
+constexpr float kMagic = 12582912.0f;
+constexpr uint32_t kMagicBits = 0x4B400000u;
+__device__ __forceinline__ uint32_t quantise_bits(uint32_t acc_bits, float inv_step, float bias, float vmax)
+{
+    return __float_as_uint(fminf(fmaxf(fmaf(__uint_as_float(acc_bits), inv_step, bias) + kMagic, kMagic), vmax));
+}
+
+template <bool kPerChannel, bool kDebug>
+__global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, int smem_budget)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ __align__(8) unsigned long long s_full[kMaxStages], s_empty[kMaxStages], s_tfull[2], s_tempty[2];
+    __shared__ uint32_t s_tmem_base;
+    __shared__ unsigned int s_warp_sums[2][4];
+    __shared__ unsigned long long s_base;
+    __shared__ int s_write_ok;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int nsym = 1 << a.bits;
+    const int enc_entries = kPerChannel ? 0 : nsym;
+    const SmemLayout L = smem_layout(a.k, enc_entries, smem_budget);
+    const int stages = L.stages;
+    const uint32_t ring_addr = smem_u32(smem + L.ring);
+    uint32_t *s_symq = reinterpret_cast<uint32_t *>(smem + L.symq);
+    unsigned int *s_part = reinterpret_cast<unsigned int *>(smem + L.part);
+    float *s_bias = reinterpret_cast<float *>(smem + L.bias);
+    uint32_t *s_enc = reinterpret_cast<uint32_t *>(smem + L.enc);
+    unsigned char *s_len8 = smem + L.len8;
+    const int n_panels = (a.c + kPanelCh - 1) / kPanelCh;
+    const int n_blocks = (a.k + kBlockCoef - 1) / kBlockCoef;
+
+    // ---- set-up ---------------------------------------------------------------------
+    if (tid == 0) {
+        for (int s = 0; s < kMaxStages; ++s) { mbar_init(smem_u32(&s_full[s]), 128); mbar_init(smem_u32(&s_empty[s]), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&s_tfull[b]), 1); mbar_init(smem_u32(&s_tempty[b]), 256); }
+        mbar_fence_init();
+    }
+    if (warp == kMmaWarp) { tmem_alloc(smem_u32(&s_tmem_base), kTmemCols); tmem_relinquish(); }
+    for (int i = tid; i < a.k; i += kThreads) s_bias[i] = a.enc_bias[i];
+    for (int i = tid; i < enc_entries; i += kThreads) {
+        const uint32_t e = a.enc[i];
+        s_enc[i] = e;
+        s_len8[i] = (unsigned char)(e & 0xffu);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = s_tmem_base;
+
+    const long long my_tiles = (a.n_tiles > blockIdx.x) ? (a.n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+
+    if (warp >= kLoaderWarp0 && warp < kMmaWarp) {
+        // ================= loaders =================
+        const int lt = tid - kLoaderWarp0 * 32;               // 0..127
+        const int lw = lt >> 5, kk = lane & 7;
+        const __nv_bfloat16 *xin = reinterpret_cast<const __nv_bfloat16 *>(a.x);
+        const bool aligned = (a.hw & 3) == 0;                 // groups of four pixels are 8-byte aligned and inside one image
+        int it = 0;
+        bool alive = true;
+        for (long long tl = 0; tl < my_tiles && alive; ++tl) {
+            const long long tile = blockIdx.x + tl * gridDim.x;
+            // aligned rows: this thread copies two groups of four pixels of every channel kk (mod 8)
+            const __nv_bfloat16 *src[2];
+            uint32_t dst_off[2], nbytes[2];
+#pragma unroll
+            for (int g = 0; g < 2; ++g) {
+                const int mg = 8 * lw + (lane >> 3) + 4 * g;
+                const long long p0 = tile * TC_TILE_PIXELS + 4 * mg;
+                const bool valid = p0 < a.pixels;
+                const long long img = valid ? p0 / a.hw : 0;
+                const long long s = valid ? p0 - img * a.hw : 0;
+                src[g] = xin + img * a.c * (long long)a.hw + s;
+                nbytes[g] = valid ? 8u : 0u;
+                dst_off[g] = (uint32_t)((mg >> 1) * 128 + kk * 16 + (mg & 1) * 8);
+            }
+            // unaligned rows: this thread loads pixel lt of every channel
+            const long long p1 = tile * TC_TILE_PIXELS + lt;
+            const bool valid1 = p1 < a.pixels;
+            const long long img1 = valid1 ? p1 / a.hw : 0;
+            const unsigned short *src1 = reinterpret_cast<const unsigned short *>(xin) + img1 * a.c * (long long)a.hw +
+                                         (valid1 ? p1 - img1 * a.hw : 0);
+            const uint32_t dst1 = (uint32_t)((lt >> 3) * 128 + (lt & 7) * 2);
+            for (int nb = 0; nb < n_blocks && alive; ++nb) {
+                const int j0 = nb * kBlockCoef;
+                const int ncols = min(kBlockCoef, a.k - j0);
+                for (int kp = 0; kp < n_panels; ++kp, ++it) {
+                    const int s = it % stages;
+                    if (!mbar_wait(smem_u32(&s_empty[s]), ((it / stages) & 1) ^ 1)) { alive = false; break; }
+                    const int k0 = kp * kPanelCh;
+                    const int nk8 = min(kPanelCh, a.c - k0) >> 3;
+                    const uint32_t stage_a = ring_addr + s * kStageBytes, stage_b = stage_a + kStageA;
+                    // basis piece: coefficient rows j0 .. j0 + ncols, channels k0 .. k0 + 8 nk8, K-major
+                    // core matrices: (j / 8) * 512 + (ch / 8) * 128 + (j % 8) * 16 + (ch % 8) * 2
+                    for (int i = lt; i < ncols * 4; i += 128) {
+                        const int j = i >> 2, c8 = i & 3;
+                        const bool ok = c8 < nk8;
+                        cp_async_16(stage_b + (j >> 3) * 512 + c8 * 128 + (j & 7) * 16,
+                                    a.basis_bf16 + (long long)(j0 + j) * a.c + (ok ? k0 + c8 * 8 : 0), ok ? 16u : 0u);
+                    }
+                    if (aligned) {
+                        for (int k8 = 0; k8 < nk8; ++k8) {
+                            const long long ch_off = (long long)(k0 + 8 * k8 + kk) * a.hw;
+#pragma unroll
+                            for (int g = 0; g < 2; ++g) cp_async_8(stage_a + k8 * 2048 + dst_off[g], src[g] + ch_off, nbytes[g]);
+                        }
+                    } else {
+                        for (int c4 = 0; c4 < nk8 * 8; c4 += 8) {
+                            unsigned short v[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) v[i] = valid1 ? __ldg(src1 + (long long)(k0 + c4 + i) * a.hw) : (unsigned short)0;
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                asm volatile("st.shared.u16 [%0], %1;" ::"r"(stage_a + (c4 >> 3) * 2048 + dst1 + i * 16), "h"(v[i]) : "memory");
+                        }
+                    }
+                    cp_async_commit();
+                    if (it >= kLag) {
+                        cp_async_wait<kLag>();
+                        fence_proxy_async_smem();
+                        mbar_arrive(smem_u32(&s_full[(it - kLag) % stages]));
+                    }
+                }
+            }
+        }
+        if (alive) {
+            if (it >= 2) { cp_async_wait<1>(); fence_proxy_async_smem(); mbar_arrive(smem_u32(&s_full[(it - 2) % stages])); }
+            if (it >= 1) { cp_async_wait<0>(); fence_proxy_async_smem(); mbar_arrive(smem_u32(&s_full[(it - 1) % stages])); }
+        } else {
+            cp_async_wait<0>();
+            tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
+        }
+    } else if (warp == kMmaWarp) {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            int it = 0;
+            long long work = 0;                                // (tile, block) pairs issued so far
+            bool alive = true;
+            for (long long tl = 0; tl < my_tiles && alive; ++tl) {
+                for (int nb = 0; nb < n_blocks && alive; ++nb, ++work) {
+                    const int acc = (int)(work & 1);
+                    if (!mbar_wait(smem_u32(&s_tempty[acc]), (uint32_t)(((work >> 1) & 1) ^ 1))) { alive = false; break; }
+                    tc_fence_after_sync();
+                    const int ncols = min(kBlockCoef, a.k - nb * kBlockCoef);
+                    const uint32_t idesc = make_idesc_bf16(TC_TILE_PIXELS, ncols, /*A MN-major*/ true, /*B K-major*/ false);
+                    const uint32_t d_tmem = tmem_base + acc * kBlockCoef;
+                    for (int kp = 0; kp < n_panels; ++kp, ++it) {
+                        const int s = it % stages;
+                        if (!mbar_wait(smem_u32(&s_full[s]), (it / stages) & 1)) { alive = false; break; }
+                        tc_fence_after_sync();
+                        const int nk16 = min(kPanelCh, a.c - kp * kPanelCh) >> 4;
+                        const uint32_t stage_a = ring_addr + s * kStageBytes, stage_b = stage_a + kStageA;
+                        for (int q = 0; q < nk16; ++q) {
+                            const uint64_t adesc = make_smem_desc(stage_a + q * 4096, 2048, 128);
+                            const uint64_t bdesc = make_smem_desc(stage_b + q * 256, 128, 512);
+                            mma_bf16_ss(d_tmem, adesc, bdesc, idesc, (kp | q) != 0 ? 1u : 0u);
+                        }
+                        mma_commit(smem_u32(&s_empty[s]));
+                    }
+                    if (alive) mma_commit(smem_u32(&s_tfull[acc]));
+                }
+            }
+            if (!alive) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
+        }
+    } else {
+        // ================= epilogue =================
+        const int half = warp >> 2;                // which half of a block's coefficients
+        const int wq = warp & 3;                   // TMEM lane quarter
+        const int m = wq * 32 + lane;              // pixel within the tile = TMEM lane
+        const float inv_step = (float)(a.basis_scale / a.step);   // the operand holds basis / basis_scale
+        const float coef_scale = (float)a.basis_scale;
+        const float vmax = kMagic + (float)(nsym - 1);
+        const uint32_t len8_rel = smem_u32(s_len8) - kMagicBits;  // + (kMagicBits + q) = address of len8[q]
+        // runs of coefficients whose bits are added up separately: the chunks of a pixel, or --
+        // with one chunk per pixel or fewer -- two halves, so that the two threads of a pixel can
+        // pack side by side.  The bounds are multiples of 16.
+        const int n_runs = a.splits > 2 ? 4 : 2;
+        int bnd[5];
+        if (a.splits == 1) { bnd[0] = 0; bnd[1] = ((a.k + 31) / 32) * 16; bnd[2] = a.k; bnd[3] = bnd[4] = a.k; }
+        else
+            for (int v = 0; v <= 4; ++v) bnd[v] = min(v, a.splits) * (a.k / a.splits);
+        const int run_lo = half * (n_runs / 2), run_hi = run_lo + n_runs / 2;      // this thread packs runs [run_lo, run_hi)
+        long long work = 0;
+        bool alive = true;
+
+        for (long long tl = 0; tl < my_tiles && alive; ++tl) {
+            const long long tile = blockIdx.x + tl * gridDim.x;
+            const long long p = tile * TC_TILE_PIXELS + m;
+            const bool valid = p < a.pixels;
+            s_part[(2 * half) * TC_TILE_PIXELS + m] = 0u;
+            s_part[(2 * half + 1) * TC_TILE_PIXELS + m] = 0u;
+            named_bar_sync(kEpiBar, 256);          // the previous tile's symbols have been packed; the sums are zero
+
+            // pass 1: quantise block by block, park the symbols, add up the code lengths
+            for (int nb = 0; nb < n_blocks && alive; ++nb, ++work) {
+                const int acc = (int)(work & 1);
+                if (!mbar_wait(smem_u32(&s_tfull[acc]), (uint32_t)((work >> 1) & 1))) { alive = false; break; }
+                tc_fence_after_sync();
+                const int ncols = min(kBlockCoef, a.k - nb * kBlockCoef);
+                const int half_cols = ((ncols + 31) / 32) * 16;
+                const int col0 = half * half_cols;
+                const int my_n = half ? ncols - half_cols : half_cols;
+                const uint32_t trow = tmem_base + acc * kBlockCoef + ((uint32_t)(wq * 32) << 16) + col0;
+#pragma unroll 1
+                for (int blk = 0; blk * 16 < my_n; ++blk) {
+                    const int j0 = nb * kBlockCoef + col0 + blk * 16;
+                    uint32_t r[16];
+                    tmem_ld_32x32b_x16(trow + blk * 16, r);
+                    float4 bias4[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) bias4[i] = *reinterpret_cast<const float4 *>(s_bias + j0 + 4 * i);
+                    const float *biasv = reinterpret_cast<const float *>(bias4);
+                    tmem_ld_wait();
+                    unsigned int bits16 = 0;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const uint32_t vb = quantise_bits(r[i], inv_step, biasv[i], vmax);
+                        if constexpr (kPerChannel) bits16 += __ldg(a.enc + (j0 + i) * nsym + (vb & 0xffu)) & 0xffu;
+                        else {
+                            uint32_t l;
+                            asm("ld.shared.u8 %0, [%1];" : "=r"(l) : "r"(vb + len8_rel));
+                            bits16 += l;
+                        }
+                        if constexpr (kDebug) {
+                            if (valid && a.dbg_coef) a.dbg_coef[p * a.k + j0 + i] = fmaf(__uint_as_float(r[i]), coef_scale, -a.tmu32[j0 + i]);
+                            if (valid && a.dbg_sym) a.dbg_sym[p * a.k + j0 + i] = (uint8_t)(vb & 0xffu);
+                        }
+                        r[i] = vb;
+                    }
+#pragma unroll
+                    for (int i = 0; i < 16; i += 4)          // low bytes of four values -> one word
+                        s_symq[((j0 + i) >> 2) * TC_TILE_PIXELS + m] =
+                            __byte_perm(__byte_perm(r[i], r[i + 1], 0x0040), __byte_perm(r[i + 2], r[i + 3], 0x0040), 0x5410);
+                    const int run = (j0 >= bnd[1] ? 1 : 0) + (j0 >= bnd[2] ? 1 : 0) + (j0 >= bnd[3] ? 1 : 0);
+                    if (valid) atomicAdd(&s_part[run * TC_TILE_PIXELS + m], bits16);
+                }
+                // the accumulator is free for the block after next
+                tc_fence_before_sync();
+                mbar_arrive(smem_u32(&s_tempty[acc]));
+            }
+            if (!alive) break;
+            named_bar_sync(kEpiBar, 256);          // every run's sum is complete
+
+            // bit offsets: pixel-major, runs in order inside a pixel
+            unsigned int run_bits[4], pixel_bits = 0, before_mine = 0, my_bits = 0;
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                run_bits[v] = v < n_runs ? s_part[v * TC_TILE_PIXELS + m] : 0u;
+                if (v < run_lo) before_mine += run_bits[v];
+                if (v >= run_lo && v < run_hi) my_bits += run_bits[v];
+                pixel_bits += run_bits[v];
+            }
+            unsigned int inc = pixel_bits;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const unsigned int up = __shfl_up_sync(0xffffffffu, inc, d);
+                if (lane >= d) inc += up;
+            }
+            if (lane == 31) s_warp_sums[half][wq] = inc;
+            named_bar_sync(kEpiBar, 256);
+            unsigned int before = 0, tile_bits = 0;
+#pragma unroll
+            for (int w = 0; w < 4; ++w) {
+                const unsigned int sw = s_warp_sums[half][w];
+                if (w < wq) before += sw;
+                tile_bits += sw;
+            }
+            const unsigned int pixel_off = before + inc - pixel_bits;
+            const unsigned int my_off = pixel_off + before_mine;
+            unsigned int chunk_end = 0;            // end of the chunk of several pixels that starts at this pixel
+            if (a.chunk_pixels > 1) {
+                const int cpx = a.chunk_pixels;
+                if (cpx < 32) {
+                    const unsigned int further = __shfl_down_sync(0xffffffffu, pixel_off, cpx);
+                    chunk_end = (lane + cpx < 32) ? further : before + s_warp_sums[half][wq];
+                } else {
+#pragma unroll
+                    for (int w = 0; w < 4; ++w)
+                        if (w < wq + (cpx >> 5)) chunk_end += s_warp_sums[half][w];
+                }
+            }
+            const unsigned long long padded = ((unsigned long long)tile_bits + 127ull) & ~127ull;
+            if (warp == 0) {
+                if (lane == 0) lookback_publish(a.tile_state, tile, padded);
+                __syncwarp();
+                bool ok;
+                const unsigned long long base = lookback_resolve(a.tile_state, tile, padded, a.status, ok);
+                if (lane == 0) {
+                    const bool fits = base + padded <= a.capacity_bits;
+                    if (ok && !fits) tc_dev_set_status(a.status, TC_ERR_BUFFER_TOO_SMALL);
+                    s_base = base;
+                    s_write_ok = (ok && fits) ? 1 : 0;
+                    a.tile_off[tile] = base;
+                    if (tile == a.n_tiles - 1) a.tile_off[a.n_tiles] = base + padded;
+                }
+            }
+            // chunk lengths
+            if (valid) {
+                if (a.splits > 1) {
+                    for (int v = run_lo; v < run_hi; ++v)
+                        if (v < a.splits) a.chunk_len[p * a.splits + v] = (uint16_t)run_bits[v];
+                } else if (half == 0) {
+                    if (a.chunk_pixels == 1) a.chunk_len[p] = (uint16_t)pixel_bits;
+                    else if ((p % a.chunk_pixels) == 0) a.chunk_len[p / a.chunk_pixels] = (uint16_t)(chunk_end - pixel_off);
+                }
+            }
+            named_bar_sync(kEpiBar, 256);          // the tile's position is known
+            const unsigned long long base = s_base;
+            const bool write_ok = s_write_ok != 0;
+            if (write_ok) {
+                uint4 *z = reinterpret_cast<uint4 *>(a.stream + (base >> 5));
+                for (unsigned int i = tid; i < (unsigned int)(padded >> 7); i += 256) z[i] = make_uint4(0u, 0u, 0u, 0u);
+            }
+            named_bar_sync(kEpiBar, 256);          // the tile's words are zero
+
+            // pass 2: codes of the parked symbols, packed into the stream
+            if (valid && write_ok && my_bits > 0) {
+                BitWriter w;
+                w.init(a.stream, base + my_off);
+                for (int j = bnd[run_lo]; j < bnd[run_hi]; j += 4) {
+                    const uint32_t word = s_symq[(j >> 2) * TC_TILE_PIXELS + m];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const uint32_t q = (word >> (8 * i)) & 0xffu;
+                        uint32_t e;
+                        if constexpr (kPerChannel) e = __ldg(a.enc + (j + i) * nsym + q);
+                        else e = s_enc[q];
+                        w.put(e >> 8, (int)(e & 0xffu));
+                    }
+                }
+                w.finish();
+            }
+        }
+        if (!alive && (tid & 255) == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
+    }
+
+    // ---- teardown ---------------------------------------------------------------------
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == kMmaWarp) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+}  // namespace
+
+bool tc_encode_wide_supported(const tc_ctx *ctx, const EncodeArgs &a)
+{
+    if (a.c % 16 != 0 || a.k % 16 != 0 || a.k < 16 || a.k > a.c || a.c > TC_MAX_C) return false;
+    if (a.splits != 1 && a.splits != 2 && a.splits != 4) return false;
+    if (a.splits > 1 && (a.chunk_pixels != 1 || (a.k / a.splits) % 16 != 0 || a.k % a.splits != 0)) return false;
+    if (a.groups != 1 && a.groups != a.k) return false;
+    const SmemLayout l = smem_layout(a.k, a.groups == 1 ? (1 << a.bits) : 0, ctx->max_smem_optin - 1024);
+    return l.stages >= 2;
+}
+
+tc_status tc_launch_encode_wide(const tc_ctx *ctx, const EncodeArgs &a, cudaStream_t s)
+{
+    if (a.n_tiles <= 0) return TC_OK;
+    const int budget = ctx->max_smem_optin - 1024;            // leaves room for the static shared variables
+    const SmemLayout l = smem_layout(a.k, a.groups == 1 ? (1 << a.bits) : 0, budget);
+    if (l.stages < 2) return TC_ERR_UNSUPPORTED;
+    const bool per_channel = a.groups != 1, debug = a.dbg_coef || a.dbg_sym;
+    void (*kernel)(EncodeArgs, int) =
+        per_channel ? (debug ? encode_wide_kernel<true, true> : encode_wide_kernel<true, false>)
+                    : (debug ? encode_wide_kernel<false, true> : encode_wide_kernel<false, false>);
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.total) != cudaSuccess)
+        return TC_ERR_CUDA;
+    const unsigned int grid = (unsigned int)((a.n_tiles < ctx->sm_count) ? a.n_tiles : ctx->sm_count);
+    EncodeArgs args = a;
+    int budget_arg = budget;
+    void *params[] = {&args, &budget_arg};
+    // cooperative launch: the grid must be co-resident, which is what makes the look-back safe
+    const cudaError_t err = cudaLaunchCooperativeKernel((void *)kernel, dim3(grid), dim3(kThreads), params, l.total, s);
+    if (err != cudaSuccess) {
+        if (getenv("TC_VERBOSE")) fprintf(stderr, "tc: wide encode launch failed: %s\n", cudaGetErrorString(err));
+        cudaGetLastError();
+        return TC_ERR_CUDA;
+    }
+    return TC_OK;
+}

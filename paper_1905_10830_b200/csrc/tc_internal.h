@@ -29,7 +29,7 @@ struct tc_ctx {
     void *host_arena = nullptr;           // device staging of tc_roundtrip_host (grown on demand)
     size_t host_arena_bytes = 0;
     int force_exact = 0;                  // route every tensor through the fp64 kernels
-    int last_encode_path = 0;             // 0 = fp64 kernels, 1 = tensor-core kernels, 2 = fp32 kernels
+    int last_encode_path = 0;             // 0 = fp64 kernels, 1 = tensor-core kernels (resident basis), 2 = fp32 kernels, 3 = tensor-core kernels (streamed basis)
     int last_decode_path = 0;
 };
 
@@ -124,6 +124,10 @@ bool tc_encode_tc_supported(const tc_ctx *ctx, const EncodeArgs &a);
 tc_status tc_launch_encode_tc(const tc_ctx *ctx, const EncodeArgs &a, cudaStream_t s);
 bool tc_decode_tc_supported(const tc_ctx *ctx, const DecodeArgs &a);
 tc_status tc_launch_decode_tc(const tc_ctx *ctx, const DecodeArgs &a, cudaStream_t s);
+bool tc_encode_wide_supported(const tc_ctx *ctx, const EncodeArgs &a);
+tc_status tc_launch_encode_wide(const tc_ctx *ctx, const EncodeArgs &a, cudaStream_t s);
+bool tc_decode_wide_supported(const tc_ctx *ctx, const DecodeArgs &a);
+tc_status tc_launch_decode_wide(const tc_ctx *ctx, const DecodeArgs &a, cudaStream_t s);
 
 tc_status tc_launch_channel_sums(const void *x, int dtype, int n, int c, int hw, double *sums,
                                  cudaStream_t s);

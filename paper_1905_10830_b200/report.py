@@ -106,7 +106,7 @@ def run(cfgs, reps, with_oracle, max_batch):
                            enc_gbs=raw / t_enc / 1e6, dec_gbs=raw / t_dec / 1e6, rt_gbs=raw / (t_enc + t_dec) / 1e6,
                            enc_ms=t_enc, dec_ms=t_dec, enc_frac=algo / t_enc / 1e6 / peak, dec_frac=algo / t_dec / 1e6 / peak,
                            enc_frac8=algo / t_enc / 1e6 / 8000, dec_frac8=algo / t_dec / 1e6 / 8000,
-                           kernels=["fp64", "tcgen05", "fp32"][tc.tc_last_path(ctx, False)] + "/" + ["fp64", "tcgen05", "fp32"][tc.tc_last_path(ctx, True)])
+                           kernels=["fp64", "tcgen05", "fp32", "tcgen05-stream"][tc.tc_last_path(ctx, False)] + "/" + ["fp64", "tcgen05", "fp32", "tcgen05-stream"][tc.tc_last_path(ctx, True)])
                 if with_oracle:
                     row.update(_parity(ctx, model, cb, x[: max(1, min(batch, 2))].contiguous(), bits, w.per_channel_codebook))
                 rows.append(row)

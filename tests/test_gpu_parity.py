@@ -65,7 +65,8 @@ def check_stream_against_oracle(enc, q_gpu, lengths, bits):
 
 def run_case(ctx, spec, bits, n_cal, n_test, dtype, per_channel, *, exact, chunk_pixels=0, pixel_splits=0, model=None,
              routes=None, k=None, basis_round=None):
-    """`routes`: the kernels expected for (encode, decode): 0 fp64, 1 tensor core, 2 fp32."""
+    """`routes`: the kernels expected for (encode, decode): 0 fp64, 1 tensor core (basis resident
+    in shared memory), 2 fp32, 3 tensor core (basis streamed: wide layers, unaligned rows)."""
     if routes is None:
         routes = (0, 0) if exact else (1, 1)
     o = H.oracle_side(spec, bits, n_cal, n_test, dtype, per_channel, model=model, k=k, basis_round=basis_round)
@@ -194,9 +195,9 @@ def test_tensor_core_path_pixel_splits(ctx_tc, c, splits):
     assert enc.layout.pixel_splits == splits
 
 
-def test_four_splits_take_the_fp32_kernels(ctx_tc):
+def test_four_splits_take_the_streaming_kernels(ctx_tc):
     spec = fm.LayerSpec(64, 14, 14, 0.9, None, 5400)
-    run_case(ctx_tc, spec, 4, 6, 3, torch.bfloat16, False, exact=False, chunk_pixels=1, pixel_splits=4, routes=(2, 2))
+    run_case(ctx_tc, spec, 4, 6, 3, torch.bfloat16, False, exact=False, chunk_pixels=1, pixel_splits=4, routes=(3, 3))
 
 
 # ---- PCA truncation: only the K leading components are coded (Section 4, ablation) -----------
@@ -218,10 +219,12 @@ def test_truncation_tensor_core_path(ctx_tc, c, k, bits, splits):
     assert enc.symbols.shape[1] == k
 
 
-def test_truncation_fp32_route(ctx_tc):
-    # K not a multiple of 16, and a wide layer
+def test_truncation_fp32_and_streaming_routes(ctx_tc):
+    # K not a multiple of 16 (fp32 kernels), and wide layers (tensor-core kernels that stream the basis)
     run_case(ctx_tc, fm.LayerSpec(64, 14, 14, 0.9, None, 5900), 5, 6, 3, torch.bfloat16, False, exact=False, k=24, routes=(2, 2))
-    run_case(ctx_tc, fm.LayerSpec(512, 7, 7, 0.95, None, 5901), 4, 12, 5, torch.bfloat16, False, exact=False, k=128, routes=(2, 2))
+    run_case(ctx_tc, fm.LayerSpec(512, 7, 7, 0.95, None, 5901), 4, 12, 5, torch.bfloat16, False, exact=False, k=128, routes=(3, 3))
+    run_case(ctx_tc, fm.LayerSpec(384, 14, 14, 0.95, None, 5902), 5, 4, 2, torch.bfloat16, False, exact=False, k=32, routes=(3, 3))
+    run_case(ctx_tc, fm.LayerSpec(576, 14, 14, 0.95, None, 5903), 5, 4, 2, torch.bfloat16, False, exact=False, k=304, routes=(3, 3))
 
 
 # ---- 8-bit basis (Section 3.1: the PCA matrix is stored in 8 bits) -------------------------------
@@ -240,9 +243,9 @@ def test_int8_basis_tensor_core_path(ctx_tc, c, s, bits, k):
     run_case(ctx_tc, spec, bits, 6, 4, torch.bfloat16, False, exact=False, basis_round="int8", k=k)
 
 
-def test_int8_basis_fp32_route(ctx_tc):
+def test_int8_basis_streaming_route(ctx_tc):
     run_case(ctx_tc, fm.LayerSpec(384, 7, 7, 0.95, None, 6200), 5, 16, 4, torch.bfloat16, False, exact=False,
-             basis_round="int8", routes=(2, 2))
+             basis_round="int8", routes=(3, 3))
 
 
 def test_library_fit_with_int8_basis_matches_the_oracle(ctx_tc):
@@ -277,20 +280,42 @@ def test_library_fit_with_int8_basis_matches_the_oracle(ctx_tc):
     model.close(); cb.close()
 
 
-# ---- fp32 kernels: bf16 tensors of shapes the tensor-core kernels do not take -----------------
+# ---- tensor-core kernels that stream the basis: wide layers, unaligned rows ---------------------
 
-@pytest.mark.parametrize("c,s,n,bits", [(512, 7, 5, 4), (384, 14, 2, 5), (576, 14, 1, 5), (960, 7, 3, 5), (1024, 4, 9, 3)])
-def test_fp32_route_wide_layers(ctx_tc, c, s, n, bits):
+@pytest.mark.parametrize("c,s,n,bits", [(512, 7, 5, 4), (384, 14, 2, 5), (576, 14, 1, 5), (960, 7, 3, 5), (1024, 4, 9, 3),
+                                        (272, 6, 8, 6), (960, 7, 6, 8)])
+def test_streaming_route_wide_layers(ctx_tc, c, s, n, bits):
     spec = fm.LayerSpec(c, s, s, 0.95, 0.6 if c != 512 else None, 5500 + c)
-    run_case(ctx_tc, spec, bits, max(4, (2 * c) // (s * s) + 1), n, torch.bfloat16, False, exact=False, routes=(2, 2))
+    run_case(ctx_tc, spec, bits, max(4, (2 * c) // (s * s) + 1), n, torch.bfloat16, False, exact=False, routes=(3, 3))
 
 
-def test_fp32_route_odd_map_size_and_per_channel_codebook(ctx_tc):
-    # 5x5 maps: the tensor-core encoder needs H*W % 4 == 0, its decoder does not
+@pytest.mark.parametrize("splits", [1, 2, 4])
+def test_streaming_route_pixel_splits_and_per_channel_codebook(ctx_tc, splits):
+    # 640 channels: five blocks of 128 channels, half-tile work items in the decoder
+    spec = fm.LayerSpec(640, 7, 7, 0.95, None, 5650)
+    _, enc = run_case(ctx_tc, spec, 5, 28, 6, torch.bfloat16, False, exact=False, chunk_pixels=1, pixel_splits=splits,
+                      routes=(3, 3))
+    assert enc.layout.pixel_splits == splits
+    spec = fm.LayerSpec(320, 10, 10, 0.95, None, 5651)
+    run_case(ctx_tc, spec, 4, 8, 3, torch.bfloat16, True, exact=False, chunk_pixels=1, pixel_splits=splits, routes=(3, 3))
+
+
+@pytest.mark.parametrize("cp", [2, 16, 64])
+def test_streaming_route_chunks_of_several_pixels(ctx_tc, cp):
+    # few coefficients of a wide layer: a chunk holds several pixels; 245 pixels leave a ragged tile
+    spec = fm.LayerSpec(576, 7, 7, 0.95, None, 5660)
+    run_case(ctx_tc, spec, 5, 24, 5, torch.bfloat16, False, exact=False, k=48, chunk_pixels=cp, routes=(3, 3))
+    spec = fm.LayerSpec(288, 7, 7, 0.95, None, 5661)
+    run_case(ctx_tc, spec, 5, 12, 5, torch.bfloat16, True, exact=False, k=32, chunk_pixels=cp, routes=(3, 3))
+
+
+def test_odd_map_sizes_and_shapes_left_to_the_fp32_kernels(ctx_tc):
+    # 5x5 maps: the resident-basis encoder needs H*W % 4 == 0 (its decoder does not); the
+    # streaming encoder loads such rows element by element
     spec = fm.LayerSpec(64, 5, 5, 0.9, None, 5600)
-    run_case(ctx_tc, spec, 6, 8, 7, torch.bfloat16, False, exact=False, routes=(2, 1))
-    run_case(ctx_tc, spec, 4, 8, 7, torch.bfloat16, True, exact=False, routes=(2, 1))
-    # 24 channels: neither tensor-core kernel (C % 16 != 0)
+    run_case(ctx_tc, spec, 6, 8, 7, torch.bfloat16, False, exact=False, routes=(3, 1))
+    run_case(ctx_tc, spec, 4, 8, 7, torch.bfloat16, True, exact=False, routes=(3, 1))
+    # 24 channels: no tensor-core kernel (C % 16 != 0)
     spec = fm.LayerSpec(24, 9, 9, 0.9, None, 5601)
     run_case(ctx_tc, spec, 5, 8, 3, torch.bfloat16, False, exact=False, chunk_pixels=4, routes=(2, 2))
 
