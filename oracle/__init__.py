@@ -51,7 +51,12 @@ def lib() -> C.CDLL:
             "orc_canonical_codes": (None, [vp, i32, vp]),
             "orc_encode": (i64, [vp, i64, i32, i32, i32, vp, i64, i64, vp, i64, vp, vp]),
             "orc_decode_symbols": (i32, [vp, i64, vp, vp, i64, i32, i32, i32, vp, i64, i64, vp]),
-            "orc_reconstruct": (None, [vp, i64, i32, i64, i32, vp, vp, d, d, i32, vp]),
+            "orc_reconstruct": (None, [vp, i64, i32, i64, i32, vp, vp, d, d, i32, i32, vp]),
+            "orc_moments_update": (None, [vp, i64, i32, i64, vp, vp, vp]),
+            "orc_moments_mean_cov": (None, [i64, vp, vp, i32, vp, vp]),
+            "orc_fit_pca_moments": (i32, [i64, vp, vp, vp, i64, i32, i64, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]),
+            "orc_fold_forward": (None, [vp, vp, i32, i32, vp, vp, vp, vp, i64, vp, vp]),
+            "orc_fold_inverse": (None, [vp, vp, i32, i32, vp, vp, i32, i32, vp, vp]),
             "orc_entropy": (d, [vp, i32]),
             "orc_mean_length": (d, [vp, vp, i32]),
             "orc_mse": (d, [vp, vp, i64]),
@@ -288,14 +293,98 @@ def decode_symbols(s: Stream, lengths: np.ndarray, bits: int) -> np.ndarray:
     return q
 
 
-def reconstruct(model: Model, q: np.ndarray, shape, *, out_bf16: bool) -> np.ndarray:
-    """x_hat (NCHW float32 array holding fp32 or bf16-rounded values) from symbols [P][K]."""
+def reconstruct(model: Model, q: np.ndarray, shape, *, out_bf16: bool, relu: bool = False) -> np.ndarray:
+    """x_hat (NCHW float32 array holding fp32 or bf16-rounded values) from symbols [P][K];
+    `relu` applies the layer's non-linearity after the inverse transform."""
     n, c, h, w = shape
     q = np.ascontiguousarray(q, dtype=np.uint8)
     xhat = np.zeros((n, c, h, w), dtype=np.float32)
     lib().orc_reconstruct(_p(q), n, c, h * w, model.k, _p(model.mean), _p(model.basis),
-                          model.lo, model.step, int(out_bf16), _p(xhat))
+                          model.lo, model.step, int(out_bf16), int(relu), _p(xhat))
     return xhat
+
+
+class Moments:
+    """Running state of the online estimate: count, sum of pixel vectors, sum of outer products."""
+
+    def __init__(self, c: int):
+        self.c = c
+        self.count = 0
+        self.sum = np.zeros(c)
+        self.outer = np.zeros((c, c))
+
+    def update(self, x) -> "Moments":
+        x = _f32(x)
+        n, c, h, w = x.shape
+        cnt = C.c_int64(self.count)
+        lib().orc_moments_update(_p(x), n, c, h * w, C.byref(cnt), _p(self.sum), _p(self.outer))
+        self.count = cnt.value
+        return self
+
+    def merge(self, other: "Moments") -> "Moments":
+        self.count += other.count
+        self.sum += other.sum
+        self.outer += other.outer
+        return self
+
+    def mean_cov(self):
+        mean = np.zeros(self.c)
+        cov = np.zeros((self.c, self.c))
+        lib().orc_moments_mean_cov(self.count, _p(self.sum), _p(self.outer), self.c, _p(mean), _p(cov))
+        return mean, cov
+
+
+def fit_pca_moments(state: Moments, x_range, bits: int, *, k: int | None = None, basis_round: str = "f64",
+                    eigensolver: str = "auto") -> Model:
+    """fit_pca with mean and covariance from a running state; the range of coefficient 0 is
+    measured on `x_range`."""
+    x = _f32(x_range)
+    n, c, h, w = x.shape
+    mode = {"f64": 0, "bf16": 1, "f32": 2, "int8": 3}[basis_round]
+    if eigensolver == "auto":
+        eigensolver = "jacobi" if c <= JACOBI_MAX_C else "lapack"
+    pre_ev = pre_vt = None
+    if eigensolver == "lapack":
+        _, cov = state.mean_cov()
+        ev, vec = np.linalg.eigh(cov)
+        pre_ev = np.ascontiguousarray(ev)
+        pre_vt = np.ascontiguousarray(vec.T)
+    mean = np.zeros(c)
+    basis = np.zeros((c, c))
+    eig = np.zeros(c)
+    lo, step, scale = C.c_double(), C.c_double(), C.c_double()
+    rc = lib().orc_fit_pca_moments(state.count, _p(state.sum), _p(state.outer), _p(x), n, c, h * w, bits, mode,
+                                   _p(pre_ev) if pre_ev is not None else None,
+                                   _p(pre_vt) if pre_vt is not None else None,
+                                   _p(mean), _p(basis), _p(eig), C.byref(lo), C.byref(step), C.byref(scale))
+    if rc != 0:
+        raise RuntimeError("oracle eigensolver did not converge")
+    return Model(c, c if k is None else k, bits, mean, basis, eig, lo.value, step.value, basis_round, scale.value)
+
+
+def fold_forward(model: Model, w: np.ndarray, bias: np.ndarray, scale: np.ndarray, shift: np.ndarray):
+    """Producer-side folding: conv weights w[C][fan], bias[C], batch-norm affine (scale, shift)
+    -> weights [K][fan] and bias [K] of the convolution that outputs the coefficients y."""
+    w = np.ascontiguousarray(w, dtype=np.float64).reshape(model.c, -1)
+    fan = w.shape[1]
+    bias, scale, shift = (np.ascontiguousarray(v, dtype=np.float64) for v in (bias, scale, shift))
+    wf = np.zeros((model.k, fan))
+    bf = np.zeros(model.k)
+    lib().orc_fold_forward(_p(model.basis), _p(model.mean), model.c, model.k, _p(w), _p(bias), _p(scale), _p(shift),
+                           fan, _p(wf), _p(bf))
+    return wf, bf
+
+
+def fold_inverse(model: Model, wn: np.ndarray, bias: np.ndarray):
+    """Consumer-side folding: next-layer weights wn[Cout][C][taps], bias[Cout] -> weights
+    [Cout][K][taps] and bias [Cout] of the convolution that consumes the dequantised y_hat."""
+    wn = np.ascontiguousarray(wn, dtype=np.float64)
+    cout, c, taps = wn.shape
+    bias = np.ascontiguousarray(bias, dtype=np.float64)
+    wi = np.zeros((cout, model.k, taps))
+    bi = np.zeros(cout)
+    lib().orc_fold_inverse(_p(model.basis), _p(model.mean), c, model.k, _p(wn), _p(bias), cout, taps, _p(wi), _p(bi))
+    return wi, bi
 
 
 def entropy(hist_row: np.ndarray) -> float:

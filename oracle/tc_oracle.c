@@ -146,15 +146,13 @@ int orc_eigh_jacobi(double *a, int n, double *evals, double *vt)
  * obtained from a library routine (pre_evals[c], pre_vt[c][c] with unit eigenvectors as rows,
  * any order): Jacobi takes minutes beyond a few hundred channels.
  * Returns 0, or -1 if the eigensolver did not converge. */
-int orc_fit_pca(const float *x, int64_t n, int c, int64_t hw, int bits, int basis_round,
-                const double *pre_evals, const double *pre_vt,
-                double *mean, double *basis, double *eig, double *lo, double *step, double *basis_scale)
+static int fit_from_mean_cov(const float *x, int64_t n, int c, int64_t hw, int bits, int basis_round,
+                             const double *pre_evals, const double *pre_vt, const double *mean, double *cov,
+                             double *basis, double *eig, double *lo, double *step, double *basis_scale)
 {
-    double *cov = (double *)malloc(sizeof(double) * (size_t)c * c);
     double *ev = (double *)malloc(sizeof(double) * (size_t)c);
     double *vt = (double *)malloc(sizeof(double) * (size_t)c * c);
     int *order = (int *)malloc(sizeof(int) * (size_t)c);
-    orc_mean_cov(x, n, c, hw, mean, cov);
     int rc = 0;
     if (pre_evals && pre_vt) {
         memcpy(ev, pre_evals, sizeof(double) * (size_t)c);
@@ -200,8 +198,67 @@ int orc_fit_pca(const float *x, int64_t n, int c, int64_t hw, int bits, int basi
         }
     *lo = mn;
     *step = (mx - mn) / (double)((1 << bits) - 1);
-    free(cov); free(ev); free(vt); free(order);
+    free(ev); free(vt); free(order);
     return rc < 0 ? -1 : 0;
+}
+
+int orc_fit_pca(const float *x, int64_t n, int c, int64_t hw, int bits, int basis_round,
+                const double *pre_evals, const double *pre_vt,
+                double *mean, double *basis, double *eig, double *lo, double *step, double *basis_scale)
+{
+    double *cov = (double *)malloc(sizeof(double) * (size_t)c * c);
+    orc_mean_cov(x, n, c, hw, mean, cov);
+    const int rc = fit_from_mean_cov(x, n, c, hw, bits, basis_round, pre_evals, pre_vt, mean, cov, basis, eig, lo, step,
+                                     basis_scale);
+    free(cov);
+    return rc;
+}
+
+/* Online estimate (Section 3.1: the covariance "can be updated online").  The running state is
+ * the sample count M, the sum of the pixel vectors s[c] and the sum of their outer products
+ * S[c][c]; a further batch only adds to the three, so states of disjoint batches (later
+ * batches, other devices, an earlier run) merge by addition.  orc_moments_update adds the n*hw
+ * pixel vectors of x. */
+void orc_moments_update(const float *x, int64_t n, int c, int64_t hw, int64_t *count, double *sum, double *outer)
+{
+    double *v = (double *)malloc(sizeof(double) * (size_t)c);
+    for (int64_t i = 0; i < n; ++i)
+        for (int64_t t = 0; t < hw; ++t) {
+            for (int a = 0; a < c; ++a) v[a] = (double)x[(i * c + a) * hw + t];
+            for (int a = 0; a < c; ++a) {
+                sum[a] += v[a];
+                for (int b = 0; b < c; ++b) outer[(int64_t)a * c + b] += v[a] * v[b];
+            }
+        }
+    free(v);
+    *count += n * hw;
+}
+
+/* mean = s / M and the unbiased covariance (S - s s^T / M) / (M - 1) of the running state. */
+void orc_moments_mean_cov(int64_t count, const double *sum, const double *outer, int c, double *mean, double *cov)
+{
+    const double m = (double)count;
+    for (int a = 0; a < c; ++a) mean[a] = sum[a] / m;
+    const double denom = (count > 1) ? m - 1.0 : 1.0;
+    for (int a = 0; a < c; ++a)
+        for (int b = 0; b < c; ++b)
+            cov[(int64_t)a * c + b] = (outer[(int64_t)a * c + b] - sum[a] * sum[b] / m) / denom;
+}
+
+/* The fit of orc_fit_pca with mean and covariance taken from a running state; the quantiser
+ * range (coefficient 0) is measured on the maps x, which the caller chooses (for instance the
+ * last calibration batch): the basis is not known while the state is being accumulated. */
+int orc_fit_pca_moments(int64_t count, const double *sum, const double *outer,
+                        const float *x, int64_t n, int c, int64_t hw, int bits, int basis_round,
+                        const double *pre_evals, const double *pre_vt,
+                        double *mean, double *basis, double *eig, double *lo, double *step, double *basis_scale)
+{
+    double *cov = (double *)malloc(sizeof(double) * (size_t)c * c);
+    orc_moments_mean_cov(count, sum, outer, c, mean, cov);
+    const int rc = fit_from_mean_cov(x, n, c, hw, bits, basis_round, pre_evals, pre_vt, mean, cov, basis, eig, lo, step,
+                                     basis_scale);
+    free(cov);
+    return rc;
 }
 
 /* ------------------------------------------------------------------------------------------
@@ -531,9 +588,11 @@ int orc_decode_symbols(const uint32_t *stream, int64_t stream_words, const uint1
 
 /* O7 (second half). Inverse quantiser and inverse transform: y_hat = lo + q*step (levels
  * "scaled back to the transform domain"), x_hat = T^T y_hat + mu (T orthonormal, Section 3),
- * rounded to the tensor's type (out_bf16 != 0: bfloat16, else fp32), ties to even. */
+ * rounded to the tensor's type (out_bf16 != 0: bfloat16, else fp32), ties to even.  With
+ * relu != 0 the layer's non-linearity follows the decoder (Section 3.1: the inverse PCA is
+ * applied "before applying the non-linearity"): x_hat = max(T^T y_hat + mu, 0), then rounded. */
 void orc_reconstruct(const uint8_t *q, int64_t n, int c, int64_t hw, int k, const double *mean,
-                     const double *basis, double lo, double step, int out_bf16, float *xhat)
+                     const double *basis, double lo, double step, int out_bf16, int relu, float *xhat)
 {
     double *yh = (double *)malloc(sizeof(double) * (size_t)k);
     for (int64_t i = 0; i < n; ++i)
@@ -544,10 +603,59 @@ void orc_reconstruct(const uint8_t *q, int64_t n, int c, int64_t hw, int k, cons
                 double s = 0.0;
                 for (int j = 0; j < k; ++j) s += basis[(int64_t)j * c + a] * yh[j];
                 s += mean[a];
+                if (relu && s < 0.0) s = 0.0;
                 xhat[(i * c + a) * hw + t] = out_bf16 ? (float)orc_round_bf16(s) : (float)s;
             }
         }
     free(yh);
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Folding (Section 3.1, "Linear transform": with 1 x 1 x C blocks the PCA is a 1 x 1
+ * convolution and, like the batch normalisation, folds into the convolution that produces the
+ * feature map; the inverse transform folds into the convolution that consumes it).
+ * ---------------------------------------------------------------------------------------- */
+
+/* Producer side.  The layer computes z_c = scale_c * (sum_f W[c][f] u_f + bias_c) + shift_c
+ * (f runs over input channel x kernel position, `fan` of them; scale/shift are the batch
+ * normalisation written as an affine map) and the encoder y_j = sum_c T[j][c] (z_c - mu_c).
+ * Folded: y_j = sum_f Wf[j][f] u_f + bf[j] with
+ *   Wf[j][f] = sum_c T[j][c] scale_c W[c][f],   bf[j] = sum_c T[j][c] (scale_c bias_c + shift_c - mu_c). */
+void orc_fold_forward(const double *basis, const double *mean, int c, int k, const double *w, const double *bias,
+                      const double *scale, const double *shift, int64_t fan, double *wf, double *bf)
+{
+    for (int j = 0; j < k; ++j) {
+        for (int64_t f = 0; f < fan; ++f) {
+            double s = 0.0;
+            for (int a = 0; a < c; ++a) s += basis[(int64_t)j * c + a] * (scale[a] * w[(int64_t)a * fan + f]);
+            wf[(int64_t)j * fan + f] = s;
+        }
+        double b = 0.0;
+        for (int a = 0; a < c; ++a) b += basis[(int64_t)j * c + a] * (scale[a] * bias[a] + shift[a] - mean[a]);
+        bf[j] = b;
+    }
+}
+
+/* Consumer side, for a next layer that takes x_hat = T^T y_hat + mu with no non-linearity in
+ * between: v_o = sum_{c,s} Wn[o][c][s] x_hat_c(s) + bias_o (s runs over the `taps` kernel
+ * positions).  Folded: v_o = sum_{j,s} Wi[o][j][s] y_hat_j(s) + bi[o] with
+ *   Wi[o][j][s] = sum_c Wn[o][c][s] T[j][c],   bi[o] = bias_o + sum_{c,s} Wn[o][c][s] mu_c
+ * (the constant holds where every tap lies inside the map; zero padding breaks it at the border). */
+void orc_fold_inverse(const double *basis, const double *mean, int c, int k, const double *wn, const double *bias,
+                      int cout, int taps, double *wi, double *bi)
+{
+    for (int o = 0; o < cout; ++o) {
+        for (int j = 0; j < k; ++j)
+            for (int s = 0; s < taps; ++s) {
+                double acc = 0.0;
+                for (int a = 0; a < c; ++a) acc += wn[((int64_t)o * c + a) * taps + s] * basis[(int64_t)j * c + a];
+                wi[((int64_t)o * k + j) * taps + s] = acc;
+            }
+        double b = bias[o];
+        for (int a = 0; a < c; ++a)
+            for (int s = 0; s < taps; ++s) b += wn[((int64_t)o * c + a) * taps + s] * mean[a];
+        bi[o] = b;
+    }
 }
 
 /* ------------------------------------------------------------------------------------------
