@@ -168,6 +168,8 @@ def main():
     ap.add_argument("--k", type=int, default=0, help="code only the K leading components (0 = all C)")
     ap.add_argument("--basis", default="bf16", choices=["bf16", "int8"], help="precision the fitted basis is stored in")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--splits", type=int, default=0, choices=[0, 1, 2, 4],
+                    help="chunks per pixel in the stream (0 = the library's default: 2 at K >= 256)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (smaller captures)")
     ap.add_argument("--sample-images", type=int, default=0, help="images per oracle timing sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -199,6 +201,7 @@ def main():
     spec = w.layers[0]
     batch = args.batch or w.batch
     bits = args.bits
+    chunking = {"chunk_pixels": 1, "pixel_splits": args.splits} if args.splits else {}
     params = fm.layer_params(spec)
 
     # ---- set-up (untimed): fit, statistics, codebook -- all through the library ---------
@@ -210,8 +213,8 @@ def main():
     cb = tc.tc_build_codebook(ctx, model, st.hist, groups=1)
     x = fm.make_maps(params, batch, dtype=w.dtype, device=dev, offset=rank)   # each rank its own maps
     raw_bytes = x.numel() * x.element_size()
-    lay = tc.tc_encode_bound(model, cb, x)
-    enc = tc.tc_encode(ctx, model, cb, x)
+    lay = tc.tc_encode_bound(model, cb, x, **chunking)
+    enc = tc.tc_encode(ctx, model, cb, x, **chunking)
     xhat = torch.empty_like(x)
     tc.tc_decode(ctx, model, cb, enc, x.shape, x.dtype, out=xhat)
     status = tc.tc_get_status(ctx)
@@ -223,7 +226,7 @@ def main():
     test_stats = tc.tc_stats(ctx, model, cb, x[: min(batch, 256)], groups=1, want_hist=False)
 
     def step():
-        tc.tc_encode(ctx, model, cb, x, out=enc)
+        tc.tc_encode(ctx, model, cb, x, out=enc, **chunking)
         tc.tc_decode(ctx, model, cb, enc, x.shape, x.dtype, out=xhat, stream_bytes=stream_bytes)
 
     for _ in range(args.warmup):
@@ -242,7 +245,7 @@ def main():
     t_begin.record()
     for i in range(args.steps):
         ev[i][0].record()
-        tc.tc_encode(ctx, model, cb, x, out=enc)
+        tc.tc_encode(ctx, model, cb, x, out=enc, **chunking)
         ev[i][1].record()
         tc.tc_decode(ctx, model, cb, enc, x.shape, x.dtype, out=xhat, stream_bytes=stream_bytes)
         ev[i][2].record()
@@ -269,7 +272,7 @@ def main():
 
         def e2e_step():
             # one C-ABI call with host buffers: H2D copy, encode, decode, D2H copy
-            tc.tc_roundtrip_host(ctx, model, cb, hx, hout)
+            tc.tc_roundtrip_host(ctx, model, cb, hx, hout, **chunking)
 
         e2e_step()
         torch.cuda.synchronize()

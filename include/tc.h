@@ -109,6 +109,37 @@ typedef struct {
 tc_status tc_fit_pca(tc_ctx *ctx, const tc_tensor *calib, const tc_fit_params *params,
                      tc_model **out, void *cuda_stream);
 
+/* Online fit (Section 3.1, "Linear transform": the covariance is estimated on calibration
+ * data and "can be updated online").  The running state is the sample count M, the sum of the
+ * pixel vectors s[C] and the sum of their outer products S[C][C], held in fp64 on the device.
+ * A further batch only adds to the three, so the state can be carried across batches,
+ * checkpointed, and merged with the states of other devices by adding them (one all-reduce of
+ * count, s and S -- at most 8.4 MB at C = 1024).
+ *   tc_fit_state_create  zeroed state for C channels.
+ *   tc_fit_state_update  adds the N*H*W pixel vectors of `maps` (DEVICE tensor, fp32 or bf16,
+ *                        C channels); asynchronous on `cuda_stream`.
+ *   tc_fit_state_export  synchronises and copies the state to HOST arrays sum[C],
+ *                        outer[C][C] (full symmetric matrix) and *count.
+ *   tc_fit_state_import  replaces the state by HOST arrays (for example the sum over devices).
+ *   tc_fit_state_finish  mean = s / M, covariance = (S - s s^T / M) / (M - 1), then as
+ *                        tc_fit_pca: eigendecomposition on the host, basis rounded to
+ *                        params->basis_dtype, quantiser range from coefficient 0 over
+ *                        `range_maps` (DEVICE tensor; the basis is not known while the state
+ *                        is being accumulated, so the caller names the maps the range is
+ *                        measured on, for instance the last calibration batch).  Synchronous.
+ * Errors: INVALID_ARG (shape mismatch, fewer than two samples, constant range maps),
+ * UNSUPPORTED (C > 1024, bits outside 1..8), NOT_CONVERGED, CUDA. */
+typedef struct tc_fit_state tc_fit_state;
+tc_status tc_fit_state_create(tc_ctx *ctx, int32_t c, tc_fit_state **out);
+void tc_fit_state_free(tc_fit_state *state);
+tc_status tc_fit_state_update(tc_ctx *ctx, tc_fit_state *state, const tc_tensor *maps, void *cuda_stream);
+tc_status tc_fit_state_export(tc_ctx *ctx, const tc_fit_state *state, int64_t *count, double *sum,
+                              double *outer, void *cuda_stream);
+tc_status tc_fit_state_import(tc_ctx *ctx, tc_fit_state *state, int64_t count, const double *sum,
+                              const double *outer, void *cuda_stream);
+tc_status tc_fit_state_finish(tc_ctx *ctx, const tc_fit_state *state, const tc_tensor *range_maps,
+                              const tc_fit_params *params, tc_model **out, void *cuda_stream);
+
 /* Plain HOST description of a model, for import/export (checkpointing, and the injection
  * point for externally computed models).  `basis` is [C][C] row-major, rows = directions;
  * entries must already be exactly representable in `basis_dtype` (import rejects others). */
@@ -127,6 +158,28 @@ tc_status tc_model_import(tc_ctx *ctx, const tc_model_desc *desc, tc_model **out
 /* Fills the scalar fields and, where the caller set the array pointers, the arrays. */
 tc_status tc_model_export(const tc_model *model, tc_model_desc *desc);
 void tc_model_free(tc_model *model);
+
+/* Folding (Section 3.1, "Linear transform": with 1 x 1 x C blocks the PCA is a 1 x 1
+ * convolution and can be folded, like the batch normalisation, into the convolution that
+ * produces the feature map; the inverse transform folds into the convolution that reads it).
+ * Offline helpers on HOST arrays, fp64, no device work.
+ *
+ * tc_fold_forward: the producing layer computes z_c = scale_c (sum_f W[c][f] u_f + bias_c) +
+ * shift_c, f over the `fan` = C_in * kernel positions (`w` is [C][fan] row-major; scale/shift
+ * are the batch normalisation as an affine map; bias, scale, shift may be NULL = 0, 1, 0), and
+ * the encoder y = T (z - mu).  Out: w_folded [K][fan], bias_folded [K] with
+ * y_j = sum_f w_folded[j][f] u_f + bias_folded[j].
+ *
+ * tc_fold_inverse: a next layer that reads x_hat = T^T y_hat + mu directly (no non-linearity
+ * in between) computes v_o = sum_{c,t} w_next[o][c][t] x_hat_c(t) + bias_next[o], t over the
+ * `taps` kernel positions (`w_next` is [c_out][C][taps]).  Out: w_folded [c_out][K][taps],
+ * bias_folded [c_out] with v_o = sum_{j,t} w_folded[o][j][t] y_hat_j(t) + bias_folded[o]; the
+ * constant is exact where every tap lies inside the map (zero padding breaks it at the border).
+ * Errors: INVALID_ARG. */
+tc_status tc_fold_forward(const tc_model *model, const double *w, const double *bias, const double *scale,
+                          const double *shift, int64_t fan, double *w_folded, double *bias_folded);
+tc_status tc_fold_inverse(const tc_model *model, const double *w_next, const double *bias_next, int32_t c_out,
+                          int32_t taps, double *w_folded, double *bias_folded);
 
 /* ---------------------------------------------------------------------------------------
  * Codebook = canonical Huffman code for the quantiser output (Section 3.1, "Variable
@@ -184,6 +237,9 @@ tc_status tc_host_eigh(double *a, int32_t n, double *evals, double *evecs);
 typedef struct {
     int32_t chunk_pixels; /* power of two in 1..128; 0 = library default for this shape   */
     int32_t pixel_splits; /* 1, 2 or 4 (needs chunk_pixels == 1); 0 = library default      */
+    int32_t relu;         /* tc_decode / tc_roundtrip_host only: non-zero applies the layer's
+                             non-linearity after the inverse transform (Section 3.1),
+                             x_hat = max(T^T y_hat + mu, 0), before rounding to the tensor type */
 } tc_encode_params;
 
 typedef struct {
@@ -245,7 +301,8 @@ tc_status tc_encode_noalloc(tc_ctx *ctx, const tc_model *model, const tc_codeboo
                             size_t capacity, uint16_t *chunk_len, uint64_t *tile_off,
                             void *cuda_stream);
 
-/* Decode (Section 3: VLD, inverse quantiser, inverse transform; no non-linearity is applied).
+/* Decode (Section 3: VLD, inverse quantiser, inverse transform; params->relu adds the ReLU that
+ * follows the decoder in Section 3.1, off by default).
  *   stream       DEVICE, 16-byte aligned, `stream_bytes` readable bytes
  *   x_hat        caller-allocated tensor of the shape and dtype that was encoded
  * Offsets and lengths are validated on the device (tile offsets against `stream_bytes`, the

@@ -44,7 +44,7 @@ class _CodebookParams(C.Structure):
 
 
 class _EncodeParams(C.Structure):
-    _fields_ = [("chunk_pixels", C.c_int32), ("pixel_splits", C.c_int32)]
+    _fields_ = [("chunk_pixels", C.c_int32), ("pixel_splits", C.c_int32), ("relu", C.c_int32)]
 
 
 class _StreamLayout(C.Structure):
@@ -67,7 +67,8 @@ EXPORTS = ["tc_create", "tc_destroy", "tc_status_string", "tc_get_status", "tc_f
            "tc_model_import", "tc_model_export", "tc_model_free", "tc_build_codebook",
            "tc_codebook_import", "tc_codebook_export", "tc_codebook_free",
            "tc_host_huffman_lengths", "tc_host_eigh", "tc_encode_bound", "tc_encode", "tc_encode_noalloc", "tc_decode", "tc_roundtrip_host",
-           "tc_stats"]
+           "tc_stats", "tc_fit_state_create", "tc_fit_state_free", "tc_fit_state_update", "tc_fit_state_export",
+           "tc_fit_state_import", "tc_fit_state_finish", "tc_fold_forward", "tc_fold_inverse"]
 
 _lib = None
 
@@ -114,6 +115,15 @@ def load_library() -> C.CDLL:
         lib.tc_decode.argtypes = [vp, vp, vp, vp, C.c_size_t, vp, vp, P(_EncodeParams), P(_Tensor), vp]
         lib.tc_roundtrip_host.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, P(_EncodeParams), P(C.c_uint64), vp]
         lib.tc_stats.argtypes = [vp, vp, vp, P(_Tensor), P(_StatsOut), vp]
+        lib.tc_fit_state_create.argtypes = [vp, i32, P(vp)]
+        lib.tc_fit_state_free.argtypes = [vp]
+        lib.tc_fit_state_free.restype = None
+        lib.tc_fit_state_update.argtypes = [vp, vp, P(_Tensor), vp]
+        lib.tc_fit_state_export.argtypes = [vp, vp, P(C.c_int64), vp, vp, vp]
+        lib.tc_fit_state_import.argtypes = [vp, vp, C.c_int64, vp, vp, vp]
+        lib.tc_fit_state_finish.argtypes = [vp, vp, P(_Tensor), P(_FitParams), P(vp), vp]
+        lib.tc_fold_forward.argtypes = [vp, vp, vp, vp, vp, C.c_int64, vp, vp]
+        lib.tc_fold_inverse.argtypes = [vp, vp, vp, i32, i32, vp, vp]
         _lib = lib
     return _lib
 
@@ -172,6 +182,10 @@ class Model(_Handle):
 
 class Codebook(_Handle):
     _free = "tc_codebook_free"
+
+
+class FitState(_Handle):
+    _free = "tc_fit_state_free"
 
 
 @dataclass
@@ -235,6 +249,73 @@ def tc_fit_pca(ctx: Context, calib: torch.Tensor, bits: int, k: int = 0, basis_d
     _check(load_library().tc_fit_pca(ctx.ptr, C.byref(t), C.byref(params), C.byref(out),
                                      _stream_ptr(ctx.device)), "tc_fit_pca")
     return Model(out.value)
+
+
+def tc_fit_state_create(ctx: Context, c: int) -> FitState:
+    out = C.c_void_p()
+    _check(load_library().tc_fit_state_create(ctx.ptr, c, C.byref(out)), "tc_fit_state_create")
+    st = FitState(out.value)
+    st.c = c
+    return st
+
+
+def tc_fit_state_update(ctx: Context, state: FitState, maps: torch.Tensor) -> None:
+    t = _tensor(maps)
+    _check(load_library().tc_fit_state_update(ctx.ptr, state.ptr, C.byref(t), _stream_ptr(ctx.device)), "tc_fit_state_update")
+
+
+def tc_fit_state_export(ctx: Context, state: FitState):
+    """(count, sum[C], outer[C][C]) as host arrays."""
+    c = state.c
+    count = C.c_int64()
+    s1 = np.zeros(c)
+    s2 = np.zeros((c, c))
+    _check(load_library().tc_fit_state_export(ctx.ptr, state.ptr, C.byref(count), s1.ctypes.data, s2.ctypes.data,
+                                              _stream_ptr(ctx.device)), "tc_fit_state_export")
+    return count.value, s1, s2
+
+
+def tc_fit_state_import(ctx: Context, state: FitState, count: int, s1: np.ndarray, s2: np.ndarray) -> None:
+    s1 = np.ascontiguousarray(s1, dtype=np.float64)
+    s2 = np.ascontiguousarray(s2, dtype=np.float64)
+    if s1.shape != (state.c,) or s2.shape != (state.c, state.c):
+        raise ValueError("state arrays do not match the channel count")
+    _check(load_library().tc_fit_state_import(ctx.ptr, state.ptr, int(count), s1.ctypes.data, s2.ctypes.data,
+                                              _stream_ptr(ctx.device)), "tc_fit_state_import")
+
+
+def tc_fit_state_finish(ctx: Context, state: FitState, range_maps: torch.Tensor, bits: int, k: int = 0,
+                        basis_dtype: int | None = None) -> Model:
+    t = _tensor(range_maps)
+    params = _FitParams(bits, k, t.dtype if basis_dtype is None else basis_dtype)
+    out = C.c_void_p()
+    _check(load_library().tc_fit_state_finish(ctx.ptr, state.ptr, C.byref(t), C.byref(params), C.byref(out),
+                                              _stream_ptr(ctx.device)), "tc_fit_state_finish")
+    return Model(out.value)
+
+
+def tc_fold_forward(model: Model, k: int, w: np.ndarray, bias=None, scale=None, shift=None):
+    """Folded weights [K][fan] and bias [K] of the producing convolution (`w` is [C][fan])."""
+    w = np.ascontiguousarray(w, dtype=np.float64)
+    c, fan = w.shape
+    opt = [None if v is None else np.ascontiguousarray(v, dtype=np.float64) for v in (bias, scale, shift)]
+    wf = np.zeros((k, fan))
+    bf = np.zeros(k)
+    _check(load_library().tc_fold_forward(model.ptr, w.ctypes.data, *[None if v is None else v.ctypes.data for v in opt],
+                                          fan, wf.ctypes.data, bf.ctypes.data), "tc_fold_forward")
+    return wf, bf
+
+
+def tc_fold_inverse(model: Model, k: int, w_next: np.ndarray, bias_next=None):
+    """Folded weights [Cout][K][taps] and bias [Cout] of the consuming convolution (`w_next` is [Cout][C][taps])."""
+    w_next = np.ascontiguousarray(w_next, dtype=np.float64)
+    cout, c, taps = w_next.shape
+    b = None if bias_next is None else np.ascontiguousarray(bias_next, dtype=np.float64)
+    wi = np.zeros((cout, k, taps))
+    bi = np.zeros(cout)
+    _check(load_library().tc_fold_inverse(model.ptr, w_next.ctypes.data, None if b is None else b.ctypes.data, cout, taps,
+                                          wi.ctypes.data, bi.ctypes.data), "tc_fold_inverse")
+    return wi, bi
 
 
 def tc_model_import(ctx: Context, *, basis: np.ndarray, mean: np.ndarray, lo: float, step: float, bits: int,
@@ -367,11 +448,12 @@ def tc_encode_noalloc(ctx: Context, model: Model, cb: Codebook, x: torch.Tensor,
 
 
 def tc_decode(ctx: Context, model: Model, cb: Codebook, enc: EncodedStream, shape, dtype, *,
-              out: torch.Tensor | None = None, stream_bytes: int | None = None) -> torch.Tensor:
+              out: torch.Tensor | None = None, stream_bytes: int | None = None, relu: bool = False) -> torch.Tensor:
+    """Decode `enc`; `relu` applies the layer's non-linearity after the inverse transform."""
     if out is None:
         out = torch.empty(shape, dtype=dtype, device=enc.words.device)
     t = _tensor(out)
-    p = _EncodeParams(enc.layout.chunk_pixels, enc.layout.pixel_splits)
+    p = _EncodeParams(enc.layout.chunk_pixels, enc.layout.pixel_splits, int(relu))
     nbytes = enc.words.numel() if stream_bytes is None else stream_bytes
     _check(load_library().tc_decode(ctx.ptr, model.ptr, cb.ptr, enc.words.data_ptr(), nbytes,
                                     enc.chunk_len.data_ptr(), enc.tile_off.data_ptr(), C.byref(p), C.byref(t),

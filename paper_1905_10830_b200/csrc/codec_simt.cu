@@ -358,7 +358,11 @@ __global__ void __launch_bounds__(kThreads) decode_simt_kernel(DecodeArgs a)
 #pragma unroll
                 for (int cc = 0; cc < RB; ++cc)
                     if (c0 + cc < a.c)
-                        store_rounded(out + obase + (long long)(c0 + cc) * a.hw, (double)fmaf(acc[cc], step, a.dec_bias[c0 + cc]));
+                        {
+                        float v = fmaf(acc[cc], step, a.dec_bias[c0 + cc]);
+                        if (a.relu) v = fmaxf(v, 0.f);
+                        store_rounded(out + obase + (long long)(c0 + cc) * a.hw, (double)v);
+                    }
             }
         } else if (valid) {
             double acc[kRowBlock];
@@ -373,7 +377,11 @@ __global__ void __launch_bounds__(kThreads) decode_simt_kernel(DecodeArgs a)
 #pragma unroll
             for (int cc = 0; cc < kRowBlock; ++cc)
                 if (c0 + cc < a.c)
-                    store_rounded(out + obase + (long long)(c0 + cc) * a.hw, __dadd_rn(acc[cc], s_mean[c0 + cc]));
+                    {
+                    double v = __dadd_rn(acc[cc], s_mean[c0 + cc]);
+                    if (a.relu && v < 0.0) v = 0.0;
+                    store_rounded(out + obase + (long long)(c0 + cc) * a.hw, v);
+                }
         }
     }
 }

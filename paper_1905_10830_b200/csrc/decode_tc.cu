@@ -500,6 +500,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
         const bool ch_ok = ch < a.c;
         const float step = (float)(a.step * a.basis_scale);        // the operand holds basis / basis_scale
         const float bias = ch_ok ? a.dec_bias[ch] : 0.f;
+        const float floor_v = a.relu ? 0.f : __int_as_float((int)0xff800000u);        // the layer's non-linearity, when it follows the decoder
         __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(a.xhat);
         // With H*W a multiple of 4 every aligned group of four pixels lies inside one image and is
         // 8-byte aligned; otherwise pixels are stored one by one.
@@ -546,8 +547,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
                         uint32_t h2[4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
-                            const __nv_bfloat162 h = __floats2bfloat162_rn(fmaf(__uint_as_float(r[8 * q + 2 * i]), step, bias),
-                                                                           fmaf(__uint_as_float(r[8 * q + 2 * i + 1]), step, bias));
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(fmaxf(fmaf(__uint_as_float(r[8 * q + 2 * i]), step, bias), floor_v),
+                                                                           fmaxf(fmaf(__uint_as_float(r[8 * q + 2 * i + 1]), step, bias), floor_v));
                             h2[i] = *reinterpret_cast<const uint32_t *>(&h);
                         }
                         asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(tb_wr + q * 16), "r"(h2[0]), "r"(h2[1]),
@@ -575,7 +576,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
                     tmem_ld_wait();
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
-                        const __nv_bfloat16 h = __float2bfloat16_rn(fmaf(__uint_as_float(r[i]), step, bias));
+                        const __nv_bfloat16 h = __float2bfloat16_rn(fmaxf(fmaf(__uint_as_float(r[i]), step, bias), floor_v));
                         if (ch_ok && c0 + i < n_valid) *dst = h;
                         s += 1;
                         const bool wrap = s == a.hw;            // the next pixel starts the next image

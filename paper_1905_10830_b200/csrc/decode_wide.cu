@@ -207,6 +207,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a)
         const int ew = warp - kEpiWarp0;
         const int set = ew >> 2, wq = ew & 3;                // two sets of four warps take alternate channel blocks
         const float step = (float)(a.step * a.basis_scale);  // the operand holds basis / basis_scale
+        const float floor_v = a.relu ? 0.f : __int_as_float((int)0xff800000u);      // the layer's non-linearity, when it follows the decoder
         __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(a.xhat);
         const bool vec = (a.hw & 3) == 0;                    // four aligned pixels lie inside one image, 8-byte aligned
         const long long img_stride = (long long)a.c * a.hw;
@@ -234,10 +235,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a)
                     if (vec) {
 #pragma unroll
                         for (int g = 0; g < 4; ++g) {
-                            const __nv_bfloat162 h0 = __floats2bfloat162_rn(fmaf(__uint_as_float(r[4 * g]), step, bias),
-                                                                            fmaf(__uint_as_float(r[4 * g + 1]), step, bias));
-                            const __nv_bfloat162 h1 = __floats2bfloat162_rn(fmaf(__uint_as_float(r[4 * g + 2]), step, bias),
-                                                                            fmaf(__uint_as_float(r[4 * g + 3]), step, bias));
+                            const __nv_bfloat162 h0 = __floats2bfloat162_rn(fmaxf(fmaf(__uint_as_float(r[4 * g]), step, bias), floor_v),
+                                                                            fmaxf(fmaf(__uint_as_float(r[4 * g + 1]), step, bias), floor_v));
+                            const __nv_bfloat162 h1 = __floats2bfloat162_rn(fmaxf(fmaf(__uint_as_float(r[4 * g + 2]), step, bias), floor_v),
+                                                                            fmaxf(fmaf(__uint_as_float(r[4 * g + 3]), step, bias), floor_v));
                             if (ch_ok && c0 + 4 * g < n_valid)
                                 *reinterpret_cast<uint2 *>(dst) = make_uint2(*reinterpret_cast<const uint32_t *>(&h0),
                                                                              *reinterpret_cast<const uint32_t *>(&h1));
@@ -249,7 +250,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a)
                     } else {
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
-                            const __nv_bfloat16 hv = __float2bfloat16_rn(fmaf(__uint_as_float(r[i]), step, bias));
+                            const __nv_bfloat16 hv = __float2bfloat16_rn(fmaxf(fmaf(__uint_as_float(r[i]), step, bias), floor_v));
                             if (ch_ok && c0 + i < n_valid) *dst = hv;
                             s += 1;
                             const bool wrap = s == a.hw;

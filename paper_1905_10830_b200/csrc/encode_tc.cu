@@ -350,10 +350,11 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
             // pass 1: quantise, keep the symbols (one byte each) in registers, add up code lengths
             uint32_t sym[kPair ? kMaxHalfCols / 8 : kMaxHalfCols / 4];   // one byte per symbol, or per pair of symbols
             uint32_t blk_bits[kMaxHalfCols / 64] = {};          // code bits of each block of 16 symbols, one byte each
-            unsigned int my_bits = 0;
+            unsigned int my_bits = 0, bits_first = 0;          // bits_first: the first half of this thread's coefficients
 #pragma unroll
             for (int blk = 0; blk < kMaxHalfCols / 16; ++blk) {
                 if (blk * 16 < ncols) {
+                    if (blk * 32 == ncols) bits_first = my_bits;
                     const unsigned int bits_before = my_bits;
                     uint32_t r[16];
                     tmem_ld_32x32b_x16(trow + blk * 16, r);
@@ -548,8 +549,11 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
             // hand the tile to the store warp (each thread's arrival releases its own writes)
             mbar_arrive(smem_u32(&s_stg_full[grp]));
             ++n_done;
-            // chunk lengths (the first half's thread of a pixel writes them)
-            if (valid && half == 0) {
+            // chunk lengths: with four chunks per pixel each thread writes the two of its half
+            // (one aligned word); otherwise the first half's thread of a pixel writes them
+            if (valid && a.splits == 4)
+                *reinterpret_cast<uint32_t *>(a.chunk_len + 4 * p + 2 * half) = bits_first | ((my_bits - bits_first) << 16);
+            else if (valid && half == 0) {
                 if (a.splits == 2)                        // one chunk per half: both lengths in one aligned word
                     *reinterpret_cast<uint32_t *>(a.chunk_len + 2 * p) = my_bits | (other << 16);
                 else if (a.chunk_pixels == 1)
@@ -588,7 +592,8 @@ bool tc_encode_tc_supported(const tc_ctx *ctx, const EncodeArgs &a)
     // K <= C leading components (PCA truncation): K is the N dimension of the MMA
     if (a.c % 16 != 0 || a.k % 16 != 0 || a.k < 16 || a.k > a.c || a.c > 256 || a.hw % 4 != 0) return false;
     // two chunks per pixel must coincide with the two halves the epilogue threads work on
-    if (a.splits != 1 && !(a.splits == 2 && a.k % 32 == 0)) return false;
+    // (four chunks: each half splits once more in its middle)
+    if (a.splits != 1 && !(a.splits == 2 && a.k % 32 == 0) && !(a.splits == 4 && a.k % 64 == 0 && a.chunk_pixels == 1)) return false;
     if (a.groups != 1 && a.groups != a.k) return false;
     const SmemLayout l = smem_layout(a.c, a.k, enc_table_entries(a));
     return (int)l.total + 512 <= ctx->max_smem_optin;       // leaves room for the static shared variables

@@ -169,14 +169,14 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
                             for (int g = 0; g < 2; ++g) cp_async_8(stage_a + k8 * 2048 + dst_off[g], src[g] + ch_off, nbytes[g]);
                         }
                     } else {
-                        for (int c4 = 0; c4 < nk8 * 8; c4 += 8) {
-                            unsigned short v[8];
+                        // every load of the panel is in flight before the first store needs its value
+                        unsigned short v[kPanelCh];
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) v[i] = valid1 ? __ldg(src1 + (long long)(k0 + c4 + i) * a.hw) : (unsigned short)0;
+                        for (int i = 0; i < kPanelCh; ++i)
+                            v[i] = (valid1 && i < nk8 * 8) ? __ldg(src1 + (long long)(k0 + i) * a.hw) : (unsigned short)0;
 #pragma unroll
-                            for (int i = 0; i < 8; ++i)
-                                asm volatile("st.shared.u16 [%0], %1;" ::"r"(stage_a + (c4 >> 3) * 2048 + dst1 + i * 16), "h"(v[i]) : "memory");
-                        }
+                        for (int i = 0; i < kPanelCh; ++i)
+                            asm volatile("st.shared.u16 [%0], %1;" ::"r"(stage_a + (i >> 3) * 2048 + dst1 + (i & 7) * 16), "h"(v[i]) : "memory");
                     }
                     cp_async_commit();
                     if (it >= kLag) {

@@ -309,6 +309,9 @@ void tc_model_free(tc_model *m)
     delete m;
 }
 
+static tc_status finish_fit(tc_ctx *ctx, const tc_tensor *range_maps, const tc_fit_params *params, int k,
+                            std::vector<double> &mean, std::vector<double> &cov, tc_model **out, cudaStream_t s);
+
 tc_status tc_fit_pca(tc_ctx *ctx, const tc_tensor *calib, const tc_fit_params *params, tc_model **out, void *cuda_stream)
 {
     if (!ctx || !out || !params || !valid_tensor(calib)) return TC_ERR_INVALID_ARG;
@@ -323,11 +326,10 @@ tc_status tc_fit_pca(tc_ctx *ctx, const tc_tensor *calib, const tc_fit_params *p
     DeviceGuard guard(ctx->device);
     cudaStream_t s = (cudaStream_t)cuda_stream;
 
-    const int range_blocks = tc_range0_max_blocks(m_samples);
-    const size_t n_doubles = (size_t)c + (size_t)c * c + (size_t)c + 2 * (size_t)range_blocks;
+    const size_t n_doubles = (size_t)c + (size_t)c * c;
     double *d_buf = nullptr;
     TC_CUDA(cudaMalloc((void **)&d_buf, n_doubles * sizeof(double)));
-    double *d_mean = d_buf, *d_cov = d_buf + c, *d_row0 = d_cov + (size_t)c * c, *d_minmax = d_row0 + c;
+    double *d_mean = d_buf, *d_cov = d_buf + c;
     struct Free { double *p; ~Free() { cudaFree(p); } } freer{d_buf};
     TC_CUDA(cudaMemsetAsync(d_buf, 0, n_doubles * sizeof(double), s));
 
@@ -349,6 +351,23 @@ tc_status tc_fit_pca(tc_ctx *ctx, const tc_tensor *calib, const tc_fit_params *p
             const double v = cov[(size_t)a * c + b] / denom;
             cov[(size_t)a * c + b] = cov[(size_t)b * c + a] = v;
         }
+    return finish_fit(ctx, calib, params, k, mean, cov, out, s);
+}
+
+// Second half of a fit: eigendecomposition of the (symmetric, normalised) covariance on the
+// host, rounding of the basis, range of coefficient 0 over `range_maps` on the device.
+static tc_status finish_fit(tc_ctx *ctx, const tc_tensor *range_maps, const tc_fit_params *params, int k,
+                            std::vector<double> &mean, std::vector<double> &cov, tc_model **out, cudaStream_t s)
+{
+    const int c = range_maps->c, hw = range_maps->h * range_maps->w, n = range_maps->n;
+    const long long m_samples = (long long)n * hw;
+    const int range_blocks = tc_range0_max_blocks(m_samples);
+    double *d_buf = nullptr;
+    TC_CUDA(cudaMalloc((void **)&d_buf, (2 * (size_t)c + 2 * (size_t)range_blocks) * sizeof(double)));
+    struct Free { double *p; ~Free() { cudaFree(p); } } freer{d_buf};
+    double *d_mean = d_buf, *d_row0 = d_buf + c, *d_minmax = d_row0 + c;
+    TC_CUDA(cudaMemcpyAsync(d_mean, mean.data(), sizeof(double) * c, cudaMemcpyHostToDevice, s));
+    tc_status st;
     std::vector<double> eig(c), basis((size_t)c * c);
     if (tc_eigh_host(cov.data(), c, eig.data(), basis.data()) != 0) return TC_ERR_NOT_CONVERGED;
     double basis_scale = 1.0;
@@ -363,7 +382,7 @@ tc_status tc_fit_pca(tc_ctx *ctx, const tc_tensor *calib, const tc_fit_params *p
 
     TC_CUDA(cudaMemcpyAsync(d_row0, basis.data(), sizeof(double) * c, cudaMemcpyHostToDevice, s));
     int blocks = 0;
-    st = tc_launch_range0(calib->data, calib->dtype, n, c, hw, d_mean, d_row0, d_minmax, &blocks, s);
+    st = tc_launch_range0(range_maps->data, range_maps->dtype, n, c, hw, d_mean, d_row0, d_minmax, &blocks, s);
     if (st != TC_OK) return st;
     std::vector<double> mm(2 * (size_t)blocks);
     TC_CUDA(cudaMemcpyAsync(mm.data(), d_minmax, sizeof(double) * mm.size(), cudaMemcpyDeviceToHost, s));
@@ -377,6 +396,158 @@ tc_status tc_fit_pca(tc_ctx *ctx, const tc_tensor *calib, const tc_fit_params *p
     d.lo = lo; d.step = (hi - lo) / (double)((1 << params->bits) - 1);
     d.basis = basis.data(); d.mean = mean.data(); d.eig = eig.data(); d.basis_scale = basis_scale;
     return tc_model_import(ctx, &d, out);
+}
+
+// ---- online fit: running sums ---------------------------------------------------------------
+
+struct tc_fit_state {
+    int c = 0, device = 0;
+    long long count = 0;
+    double *d_sum = nullptr;      // [c]     sum of the pixel vectors
+    double *d_outer = nullptr;    // [c][c]  sum of their outer products (upper triangle)
+    double *d_zero = nullptr;     // [c]     zeros: the "mean" that makes the covariance kernel add raw products
+};
+
+tc_status tc_fit_state_create(tc_ctx *ctx, int32_t c, tc_fit_state **out)
+{
+    if (!ctx || !out || c < 1) return TC_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (c > TC_MAX_C) return TC_ERR_UNSUPPORTED;
+    DeviceGuard guard(ctx->device);
+    double *buf = nullptr;
+    const size_t n = 2 * (size_t)c + (size_t)c * c;
+    TC_CUDA(cudaMalloc((void **)&buf, n * sizeof(double)));
+    if (cudaMemset(buf, 0, n * sizeof(double)) != cudaSuccess) { cudaFree(buf); return TC_ERR_CUDA; }
+    tc_fit_state *st = new tc_fit_state;
+    st->c = c; st->device = ctx->device;
+    st->d_sum = buf; st->d_zero = buf + c; st->d_outer = buf + 2 * (size_t)c;
+    *out = st;
+    return TC_OK;
+}
+
+void tc_fit_state_free(tc_fit_state *st)
+{
+    if (!st) return;
+    DeviceGuard guard(st->device);
+    cudaFree(st->d_sum);          // one allocation holds all three arrays
+    delete st;
+}
+
+tc_status tc_fit_state_update(tc_ctx *ctx, tc_fit_state *st, const tc_tensor *maps, void *cuda_stream)
+{
+    if (!ctx || !st || !valid_tensor(maps) || maps->c != st->c || ctx->device != st->device) return TC_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const int hw = maps->h * maps->w;
+    if ((long long)maps->n * hw == 0) return TC_OK;
+    tc_status rc = tc_launch_channel_sums(maps->data, maps->dtype, maps->n, st->c, hw, st->d_sum, s);
+    if (rc != TC_OK) return rc;
+    rc = tc_launch_covariance(maps->data, maps->dtype, maps->n, st->c, hw, st->d_zero, st->d_outer, s);
+    if (rc != TC_OK) return rc;
+    st->count += (long long)maps->n * hw;
+    return TC_OK;
+}
+
+tc_status tc_fit_state_export(tc_ctx *ctx, const tc_fit_state *st, int64_t *count, double *sum, double *outer,
+                              void *cuda_stream)
+{
+    if (!ctx || !st || !count || !sum || !outer) return TC_ERR_INVALID_ARG;
+    DeviceGuard guard(st->device);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const int c = st->c;
+    TC_CUDA(cudaMemcpyAsync(sum, st->d_sum, sizeof(double) * c, cudaMemcpyDeviceToHost, s));
+    TC_CUDA(cudaMemcpyAsync(outer, st->d_outer, sizeof(double) * (size_t)c * c, cudaMemcpyDeviceToHost, s));
+    TC_CUDA(cudaStreamSynchronize(s));
+    for (int a = 0; a < c; ++a)                       // the device holds the upper triangle
+        for (int b = a + 1; b < c; ++b) outer[(size_t)b * c + a] = outer[(size_t)a * c + b];
+    *count = st->count;
+    return TC_OK;
+}
+
+tc_status tc_fit_state_import(tc_ctx *ctx, tc_fit_state *st, int64_t count, const double *sum, const double *outer,
+                              void *cuda_stream)
+{
+    if (!ctx || !st || count < 0 || !sum || !outer) return TC_ERR_INVALID_ARG;
+    DeviceGuard guard(st->device);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    TC_CUDA(cudaMemcpyAsync(st->d_sum, sum, sizeof(double) * st->c, cudaMemcpyHostToDevice, s));
+    TC_CUDA(cudaMemcpyAsync(st->d_outer, outer, sizeof(double) * (size_t)st->c * st->c, cudaMemcpyHostToDevice, s));
+    TC_CUDA(cudaStreamSynchronize(s));
+    st->count = count;
+    return TC_OK;
+}
+
+tc_status tc_fit_state_finish(tc_ctx *ctx, const tc_fit_state *st, const tc_tensor *range_maps,
+                              const tc_fit_params *params, tc_model **out, void *cuda_stream)
+{
+    if (!ctx || !st || !out || !params || !valid_tensor(range_maps) || range_maps->c != st->c) return TC_ERR_INVALID_ARG;
+    *out = nullptr;
+    const int c = st->c;
+    if (st->count < 2 || (long long)range_maps->n * range_maps->h * range_maps->w < 1) return TC_ERR_INVALID_ARG;
+    if (params->bits < 1 || params->bits > 8) return TC_ERR_UNSUPPORTED;
+    const int k = params->k ? params->k : c;
+    if (k < 1 || k > c) return TC_ERR_INVALID_ARG;
+    if (params->basis_dtype != TC_F32 && params->basis_dtype != TC_BF16 && params->basis_dtype != TC_INT8) return TC_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    std::vector<double> sum(c), cov((size_t)c * c);
+    int64_t count = 0;
+    tc_status rc = tc_fit_state_export(ctx, st, &count, sum.data(), cov.data(), cuda_stream);
+    if (rc != TC_OK) return rc;
+    // mean = s / M, covariance = (S - s s^T / M) / (M - 1)
+    const double m = (double)count;
+    std::vector<double> mean(c);
+    for (int a = 0; a < c; ++a) mean[a] = sum[a] / m;
+    for (int a = 0; a < c; ++a)
+        for (int b = a; b < c; ++b) {
+            const double v = (cov[(size_t)a * c + b] - sum[a] * sum[b] / m) / (m - 1.0);
+            cov[(size_t)a * c + b] = cov[(size_t)b * c + a] = v;
+        }
+    return finish_fit(ctx, range_maps, params, k, mean, cov, out, s);
+}
+
+// ---- folding into the neighbouring convolutions (host arithmetic, fp64) --------------------------
+
+tc_status tc_fold_forward(const tc_model *m, const double *w, const double *bias, const double *scale,
+                          const double *shift, int64_t fan, double *w_folded, double *bias_folded)
+{
+    if (!m || !w || !w_folded || !bias_folded || fan < 1) return TC_ERR_INVALID_ARG;
+    const int c = m->c, k = m->k;
+    for (int j = 0; j < k; ++j) {
+        const double *row = m->basis.data() + (size_t)j * c;
+        for (int64_t f = 0; f < fan; ++f) {
+            double acc = 0.0;
+            for (int a = 0; a < c; ++a) acc += row[a] * ((scale ? scale[a] : 1.0) * w[(size_t)a * fan + f]);
+            w_folded[(size_t)j * fan + f] = acc;
+        }
+        double b = 0.0;
+        for (int a = 0; a < c; ++a)
+            b += row[a] * ((scale ? scale[a] : 1.0) * (bias ? bias[a] : 0.0) + (shift ? shift[a] : 0.0) - m->mean[a]);
+        bias_folded[j] = b;
+    }
+    return TC_OK;
+}
+
+tc_status tc_fold_inverse(const tc_model *m, const double *w_next, const double *bias_next, int32_t c_out,
+                          int32_t taps, double *w_folded, double *bias_folded)
+{
+    if (!m || !w_next || !w_folded || !bias_folded || c_out < 1 || taps < 1) return TC_ERR_INVALID_ARG;
+    const int c = m->c, k = m->k;
+    for (int o = 0; o < c_out; ++o) {
+        for (int j = 0; j < k; ++j) {
+            const double *row = m->basis.data() + (size_t)j * c;
+            for (int t = 0; t < taps; ++t) {
+                double acc = 0.0;
+                for (int a = 0; a < c; ++a) acc += w_next[((size_t)o * c + a) * taps + t] * row[a];
+                w_folded[((size_t)o * k + j) * taps + t] = acc;
+            }
+        }
+        double b = bias_next ? bias_next[o] : 0.0;
+        for (int a = 0; a < c; ++a)
+            for (int t = 0; t < taps; ++t) b += w_next[((size_t)o * c + a) * taps + t] * m->mean[a];
+        bias_folded[o] = b;
+    }
+    return TC_OK;
 }
 
 // ---- codebook ---------------------------------------------------------------------------
@@ -566,6 +737,7 @@ tc_status tc_decode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
     a.basis64 = m->d_basis64; a.mean64 = m->d_mean64; a.lo = m->lo; a.step = m->step; a.basis_scale = m->basis_scale;
     a.xhat = x_hat->data; a.status = ctx->d_status;
     a.lut32 = cb->d_lut32; a.basis_t_bf16 = m->d_basis_t_bf16; a.dec_bias = m->d_dec_bias; a.center = m->center;
+    a.relu = (params && params->relu) ? 1 : 0;
     if (!ctx->force_exact && x_hat->dtype == TC_BF16 && tc_decode_tc_supported(ctx, a)) {
         ctx->last_decode_path = 1;
         return tc_launch_decode_tc(ctx, a, (cudaStream_t)cuda_stream);

@@ -106,6 +106,7 @@ struct DecodeArgs {
     const __nv_bfloat16 *basis_t_bf16;  // [c][k]
     const float *dec_bias;              // [c]
     int center;                         // subtracted from every symbol before the MMA
+    int relu;                           // x_hat = max(x_hat, 0) before it is rounded to the tensor type
     int smem_budget;                    // shared memory the tensor-core kernel may lay out (set by its launcher)
     const double *basis64;
     const double *mean64;
