@@ -35,9 +35,13 @@ constexpr int kLag = 2;
 constexpr int kVldBar = 1;
 constexpr int kMaxTileChunks = 512;
 
+constexpr int kSegBytes = 16384;                              // staged stream segment of one work item
+constexpr int kSegSlack = 32;                                 // the reader's window may look two words past the end
+
 struct SmemLayout {
-    uint32_t ring, bop, lut, start, total;
+    uint32_t ring, bop, lut, start, seg, total;
     int stages, np;
+    bool staged;                                              // room for the segment buffer beside at least three stages
 };
 
 __host__ __device__ inline SmemLayout smem_layout(int c, int k, int lut_entries, int budget)
@@ -46,14 +50,17 @@ __host__ __device__ inline SmemLayout smem_layout(int c, int k, int lut_entries,
     l.np = ((c + 127) / 128 <= 4) ? 128 : 64;
     const uint32_t bop_bytes = 2u * (uint32_t)k * (uint32_t)l.np;
     const uint32_t fixed = bop_bytes + (uint32_t)lut_entries * 4u + (kMaxTileChunks + 8) * 4u;
-    int stages = ((long long)budget - (long long)fixed) / kStageBytes;
+    int stages = ((long long)budget - (long long)fixed - (kSegBytes + kSegSlack)) / kStageBytes;
+    l.staged = stages >= 3;
+    if (!l.staged) stages = ((long long)budget - (long long)fixed) / kStageBytes;
     if (stages > kMaxStages) stages = kMaxStages;
     l.stages = stages < 2 ? 0 : stages;
     l.ring = 0;
     l.bop = (uint32_t)(l.stages * kStageBytes);
     l.lut = l.bop + bop_bytes;
     l.start = l.lut + (uint32_t)lut_entries * 4u;
-    l.total = l.start + (kMaxTileChunks + 8) * 4u;
+    l.seg = (l.start + (kMaxTileChunks + 8) * 4u + 15u) & ~15u;
+    l.total = l.seg + (l.staged ? (uint32_t)(kSegBytes + kSegSlack) : 0u);
     return l;
 }
 
@@ -147,6 +154,25 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a)
             named_bar_sync(kVldBar, kVldThreads);
             bool bad = !tile_ok || (unsigned long long)tile_total > end - base;
 
+            // the item's part of the tile's segment, staged in shared memory when it fits: the
+            // readers' refills become shared-memory loads instead of dependent global loads
+            const int ci_first = (h * NP / cp) * S, ci_end = ((h + 1) * NP / cp) * S;
+            const unsigned int seg_lo = s_start[ci_first];
+            const unsigned int seg_hi = ci_end < chunks_per_tile ? s_start[ci_end] : tile_total;
+            const unsigned int byte_lo = (seg_lo >> 3) & ~15u, byte_hi = ((seg_hi + 127u) >> 7) << 4;
+            const bool staged = L.staged && !bad && byte_hi - byte_lo <= (unsigned int)kSegBytes;
+            if (staged) {
+                const unsigned char *src = reinterpret_cast<const unsigned char *>(a.stream) + (base >> 3) + byte_lo;
+                const uint32_t dst = smem_u32(smem + L.seg);
+                for (unsigned int i = (unsigned int)t; i < ((byte_hi - byte_lo) >> 4); i += kVldThreads)
+                    cp_async_16(dst + i * 16u, src + (size_t)i * 16u, 16u);
+            }
+            cp_async_commit();
+            cp_async_wait<0>();
+            named_bar_sync(kVldBar, kVldThreads);       // every thread's part of the segment has landed
+            const uint32_t *seg_words = reinterpret_cast<const uint32_t *>(smem + L.seg);
+
+            auto decode_chunks = [&](auto &r) {
             for (int u = t; u < item_chunks && !bad; u += kVldThreads) {
                 // chunk u of the item: run `sub` of the coefficients of pixel(s) r0 ...
                 const int sub = u / pix_chunks, cidx = u - sub * pix_chunks;
@@ -156,8 +182,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a)
                 if (p0 >= a.pixels) continue;
                 const int n_pix = (int)min((long long)cp, a.pixels - p0);
                 const unsigned int start = s_start[ci], want = (ci + 1 < chunks_per_tile ? s_start[ci + 1] : tile_total) - start;
-                WindowReader r;
-                r.init(a.stream, base + start, end);
+                if (staged) r.init(seg_words, (unsigned long long)start - 8ull * byte_lo, 8ull * (byte_hi - byte_lo));
+                else r.init(a.stream, base + start, end);
                 unsigned int used = 0;
                 const int k_first = sub * k_sub;
                 for (int pp = 0; pp < n_pix; ++pp) {
@@ -196,6 +222,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a)
                 // a chunk must end exactly where its recorded length says
                 if (used != want) bad = true;
             }
+            };
+            if (staged) { WindowReaderT<true> r; decode_chunks(r); }
+            else { WindowReader r; decode_chunks(r); }
             if (bad) tc_dev_set_status(a.status, TC_ERR_CORRUPT_STREAM);
             // the writes become visible to the tensor core's proxy, then the operand is handed over
             fence_proxy_async_smem();

@@ -172,7 +172,9 @@ struct BitWriter {
 
 // MSB-first reader over 32-bit words with a 64-bit window held in two registers.  Words at or
 // past `end` read as zero, so a corrupt offset can never cause an out-of-bounds load.
-struct WindowReader {
+// kShared: the words lie in shared memory (a staged segment) instead of global memory.
+template <bool kShared>
+struct WindowReaderT {
     const uint32_t *words;
     unsigned long long next, end;     // word indices
     uint32_t hi, lo;                  // upcoming bits, left-aligned in hi:lo
@@ -180,7 +182,11 @@ struct WindowReader {
 
     __device__ __forceinline__ uint32_t fetch()
     {
-        const uint32_t w = (next < end) ? __ldg(words + next) : 0u;
+        uint32_t w = 0u;
+        if (next < end) {
+            if constexpr (kShared) w = words[next];
+            else w = __ldg(words + next);
+        }
         ++next;
         return w;
     }
@@ -215,5 +221,6 @@ struct WindowReader {
         }
     }
 };
+using WindowReader = WindowReaderT<false>;
 
 }  // namespace tcdev

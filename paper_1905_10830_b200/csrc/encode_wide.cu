@@ -6,15 +6,15 @@
 // tile are produced in blocks of up to 256 (one accumulator of tensor memory each, two
 // accumulators in flight); for every block the pixels' channels stream through a ring of
 // 32-channel panels together with the matching 256 x 32 piece of the basis, both read from L2.
-//   warps 0-7     epilogue: warps 0-3 take the first half of a block's coefficients, warps 4-7
-//                 the second half.  Pass 1 (per block): TMEM -> registers, quantise, code length,
+//   warps 0-15    epilogue: four warps per quarter of a block's coefficients (a warp reads its own
+//                 32 lanes of tensor memory).  Pass 1 (per block): TMEM -> registers, quantise, code length,
 //                 symbols parked in shared memory (one byte each, K x 128 per tile), bits added up
 //                 per run of coefficients.  Then: bit offsets (scan over the pixels, tile
 //                 look-back), chunk lengths.  Pass 2: codes of the parked symbols packed straight
 //                 into the (zeroed) stream words.
-//   warps 8-11    loaders: cp.async (or, for unaligned rows, plain 2-byte loads) into the MMA's
+//   warps 16-23   loaders: cp.async (or, for unaligned rows, plain 2-byte loads) into the MMA's
 //                 shared-memory layouts
-//   warp 12       one thread issues tcgen05.mma:  D[pixel][coef] = X[pixel][c] * T[coef][c]
+//   warp 24       one thread issues tcgen05.mma:  D[pixel][coef] = X[pixel][c] * T[coef][c]
 #include <cstdio>
 #include <cstdlib>
 
@@ -32,11 +32,11 @@ constexpr int kStageA = kPanelCh * TC_TILE_PIXELS * 2;        // 8 KB: pixels x 
 constexpr int kStageB = kBlockCoef * kPanelCh * 2;            // 16 KB: coefficients x channels
 constexpr int kStageBytes = kStageA + kStageB;
 constexpr int kMaxStages = 4;
-constexpr int kLag = 2;                                       // cp.async groups in flight per loader thread
-constexpr int kLoaderWarp0 = 8, kMmaWarp = 12;          // warps 0-7 are the epilogue
-constexpr int kThreads = 13 * 32;
+constexpr int kLoaderWarp0 = 16, kMmaWarp = 24;               // warps 0-15 are the epilogue, 16-23 the loaders
+constexpr int kThreads = 25 * 32;
+constexpr int kEpiThreads = 16 * 32;
 constexpr int kTmemCols = 512;
-constexpr int kEpiBar = 1;                                    // named barrier of the 256 epilogue threads
+constexpr int kEpiBar = 1;                                    // named barrier of the epilogue threads
 
 struct SmemLayout {
     uint32_t ring, symq, part, bias, enc, len8, total;
@@ -76,7 +76,7 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) unsigned long long s_full[kMaxStages], s_empty[kMaxStages], s_tfull[2], s_tempty[2];
     __shared__ uint32_t s_tmem_base;
-    __shared__ unsigned int s_warp_sums[2][4];
+    __shared__ unsigned int s_warp_sums[4][4];
     __shared__ unsigned long long s_base;
     __shared__ int s_write_ok;
 
@@ -96,8 +96,8 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
 
     // ---- set-up ---------------------------------------------------------------------
     if (tid == 0) {
-        for (int s = 0; s < kMaxStages; ++s) { mbar_init(smem_u32(&s_full[s]), 128); mbar_init(smem_u32(&s_empty[s]), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&s_tfull[b]), 1); mbar_init(smem_u32(&s_tempty[b]), 256); }
+        for (int s = 0; s < kMaxStages; ++s) { mbar_init(smem_u32(&s_full[s]), 256); mbar_init(smem_u32(&s_empty[s]), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&s_tfull[b]), 1); mbar_init(smem_u32(&s_tempty[b]), kEpiThreads); }
         mbar_fence_init();
     }
     if (warp == kMmaWarp) { tmem_alloc(smem_u32(&s_tmem_base), kTmemCols); tmem_relinquish(); }
@@ -116,79 +116,92 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
 
     if (warp >= kLoaderWarp0 && warp < kMmaWarp) {
         // ================= loaders =================
-        const int lt = tid - kLoaderWarp0 * 32;               // 0..127
-        const int lw = lt >> 5, kk = lane & 7;
+        // 256 threads; every address is a per-thread constant plus a per-stage offset, so that a
+        // stage costs a thread four 16-byte copies of the basis and four 8-byte copies (or sixteen
+        // element loads) of the pixels and little arithmetic besides.
+        const int lt = tid - kLoaderWarp0 * 32;               // 0..255
         const __nv_bfloat16 *xin = reinterpret_cast<const __nv_bfloat16 *>(a.x);
         const bool aligned = (a.hw & 3) == 0;                 // groups of four pixels are 8-byte aligned and inside one image
+        const int lag = stages - 1;                           // 1..3 cp.async groups pending behind the one handed over
+        // basis piece of a stage: coefficient rows j0 .. j0 + ncols, channels k0 .. k0 + 32, K-major core
+        // matrices (j / 8) * 512 + (ch / 8) * 128 + (j % 8) * 16; this thread copies 16-byte piece
+        // c8 of rows jb, jb + 64, jb + 128, jb + 192
+        const int jb = lt >> 2, c8 = lt & 3;
+        const __nv_bfloat16 *b_src0 = a.basis_bf16 + (long long)jb * a.c + c8 * 8;
+        const uint32_t b_dst0 = (uint32_t)((jb >> 3) * 512 + c8 * 128 + (jb & 7) * 16);
+        const long long b_row_step = 64ll * a.c;
+        // pixels, aligned rows: channel kk (mod 8) of one group of four pixels
+        const int lt7 = lt & 127, kk = lt7 & 7;
+        const int mg = 8 * (lt7 >> 5) + ((lt7 & 31) >> 3) + 4 * (lt >> 7);
+        const uint32_t a_dst0 = (uint32_t)((mg >> 1) * 128 + kk * 16 + (mg & 1) * 8);
+        // pixels, unaligned rows: sixteen channels of pixel lt7
+        const int ch_half = lt >> 7;
+        const uint32_t a_dst1 = (uint32_t)((lt7 >> 3) * 128 + (lt7 & 7) * 2 + ch_half * 2 * 2048);
         int it = 0;
         bool alive = true;
         for (long long tl = 0; tl < my_tiles && alive; ++tl) {
             const long long tile = blockIdx.x + tl * gridDim.x;
-            // aligned rows: this thread copies two groups of four pixels of every channel kk (mod 8)
-            const __nv_bfloat16 *src[2];
-            uint32_t dst_off[2], nbytes[2];
-#pragma unroll
-            for (int g = 0; g < 2; ++g) {
-                const int mg = 8 * lw + (lane >> 3) + 4 * g;
-                const long long p0 = tile * TC_TILE_PIXELS + 4 * mg;
-                const bool valid = p0 < a.pixels;
-                const long long img = valid ? p0 / a.hw : 0;
-                const long long s = valid ? p0 - img * a.hw : 0;
-                src[g] = xin + img * a.c * (long long)a.hw + s;
-                nbytes[g] = valid ? 8u : 0u;
-                dst_off[g] = (uint32_t)((mg >> 1) * 128 + kk * 16 + (mg & 1) * 8);
-            }
-            // unaligned rows: this thread loads pixel lt of every channel
-            const long long p1 = tile * TC_TILE_PIXELS + lt;
+            const long long p0 = tile * TC_TILE_PIXELS + 4 * mg;
+            const bool valid = p0 < a.pixels;
+            const long long img = valid ? p0 / a.hw : 0;
+            const __nv_bfloat16 *a_src0 = xin + img * a.c * (long long)a.hw + (valid ? p0 - img * a.hw : 0) + (long long)kk * a.hw;
+            const uint32_t a_bytes = valid ? 8u : 0u;
+            const long long p1 = tile * TC_TILE_PIXELS + lt7;
             const bool valid1 = p1 < a.pixels;
             const long long img1 = valid1 ? p1 / a.hw : 0;
-            const unsigned short *src1 = reinterpret_cast<const unsigned short *>(xin) + img1 * a.c * (long long)a.hw +
-                                         (valid1 ? p1 - img1 * a.hw : 0);
-            const uint32_t dst1 = (uint32_t)((lt >> 3) * 128 + (lt & 7) * 2);
+            const unsigned short *a_src1 = reinterpret_cast<const unsigned short *>(xin) + img1 * a.c * (long long)a.hw +
+                                           (valid1 ? p1 - img1 * a.hw : 0) + (long long)(16 * ch_half) * a.hw;
             for (int nb = 0; nb < n_blocks && alive; ++nb) {
                 const int j0 = nb * kBlockCoef;
                 const int ncols = min(kBlockCoef, a.k - j0);
+                const __nv_bfloat16 *b_src = b_src0 + (long long)j0 * a.c;
                 for (int kp = 0; kp < n_panels; ++kp, ++it) {
                     const int s = it % stages;
                     if (!mbar_wait(smem_u32(&s_empty[s]), ((it / stages) & 1) ^ 1)) { alive = false; break; }
                     const int k0 = kp * kPanelCh;
                     const int nk8 = min(kPanelCh, a.c - k0) >> 3;
                     const uint32_t stage_a = ring_addr + s * kStageBytes, stage_b = stage_a + kStageA;
-                    // basis piece: coefficient rows j0 .. j0 + ncols, channels k0 .. k0 + 8 nk8, K-major
-                    // core matrices: (j / 8) * 512 + (ch / 8) * 128 + (j % 8) * 16 + (ch % 8) * 2
-                    for (int i = lt; i < ncols * 4; i += 128) {
-                        const int j = i >> 2, c8 = i & 3;
+                    {
                         const bool ok = c8 < nk8;
-                        cp_async_16(stage_b + (j >> 3) * 512 + c8 * 128 + (j & 7) * 16,
-                                    a.basis_bf16 + (long long)(j0 + j) * a.c + (ok ? k0 + c8 * 8 : 0), ok ? 16u : 0u);
+                        const __nv_bfloat16 *src = ok ? b_src + k0 : a.basis_bf16;
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            if (jb + 64 * u < ncols)
+                                cp_async_16(stage_b + b_dst0 + u * 4096, ok ? src + u * b_row_step : src, ok ? 16u : 0u);
                     }
                     if (aligned) {
-                        for (int k8 = 0; k8 < nk8; ++k8) {
-                            const long long ch_off = (long long)(k0 + 8 * k8 + kk) * a.hw;
+                        const __nv_bfloat16 *src = a_src0 + (long long)k0 * a.hw;
+                        const long long step8 = 8ll * a.hw;
 #pragma unroll
-                            for (int g = 0; g < 2; ++g) cp_async_8(stage_a + k8 * 2048 + dst_off[g], src[g] + ch_off, nbytes[g]);
-                        }
+                        for (int k8 = 0; k8 < kPanelCh / 8; ++k8)
+                            if (k8 < nk8) cp_async_8(stage_a + k8 * 2048 + a_dst0, src + k8 * step8, a_bytes);
                     } else {
                         // every load of the panel is in flight before the first store needs its value
-                        unsigned short v[kPanelCh];
+                        const unsigned short *src = a_src1 + (long long)k0 * a.hw;
+                        unsigned short v[kPanelCh / 2];
 #pragma unroll
-                        for (int i = 0; i < kPanelCh; ++i)
-                            v[i] = (valid1 && i < nk8 * 8) ? __ldg(src1 + (long long)(k0 + i) * a.hw) : (unsigned short)0;
+                        for (int i = 0; i < kPanelCh / 2; ++i)
+                            v[i] = (valid1 && 16 * ch_half + i < nk8 * 8) ? __ldg(src + (long long)i * a.hw) : (unsigned short)0;
 #pragma unroll
-                        for (int i = 0; i < kPanelCh; ++i)
-                            asm volatile("st.shared.u16 [%0], %1;" ::"r"(stage_a + (i >> 3) * 2048 + dst1 + (i & 7) * 16), "h"(v[i]) : "memory");
+                        for (int i = 0; i < kPanelCh / 2; ++i)
+                            asm volatile("st.shared.u16 [%0], %1;" ::"r"(stage_a + (i >> 3) * 2048 + a_dst1 + (i & 7) * 16), "h"(v[i]) : "memory");
                     }
                     cp_async_commit();
-                    if (it >= kLag) {
-                        cp_async_wait<kLag>();
+                    // every stage of the ring is in flight: the panel issued `lag` iterations ago is
+                    // handed over once at most `lag` younger groups are still pending
+                    if (it >= lag) {
+                        if (lag == 3) cp_async_wait<3>();
+                        else if (lag == 2) cp_async_wait<2>();
+                        else cp_async_wait<1>();
                         fence_proxy_async_smem();
-                        mbar_arrive(smem_u32(&s_full[(it - kLag) % stages]));
+                        mbar_arrive(smem_u32(&s_full[(it - lag) % stages]));
                     }
                 }
             }
         }
         if (alive) {
-            if (it >= 2) { cp_async_wait<1>(); fence_proxy_async_smem(); mbar_arrive(smem_u32(&s_full[(it - 2) % stages])); }
+            if (lag >= 3 && it >= 3) { cp_async_wait<2>(); fence_proxy_async_smem(); mbar_arrive(smem_u32(&s_full[(it - 3) % stages])); }
+            if (lag >= 2 && it >= 2) { cp_async_wait<1>(); fence_proxy_async_smem(); mbar_arrive(smem_u32(&s_full[(it - 2) % stages])); }
             if (it >= 1) { cp_async_wait<0>(); fence_proxy_async_smem(); mbar_arrive(smem_u32(&s_full[(it - 1) % stages])); }
         } else {
             cp_async_wait<0>();
@@ -228,22 +241,27 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
         }
     } else {
         // ================= epilogue =================
-        const int half = warp >> 2;                // which half of a block's coefficients
+        const int part = warp >> 2;                // which quarter of a block's coefficients, and which run of a pixel
         const int wq = warp & 3;                   // TMEM lane quarter
         const int m = wq * 32 + lane;              // pixel within the tile = TMEM lane
         const float inv_step = (float)(a.basis_scale / a.step);   // the operand holds basis / basis_scale
         const float coef_scale = (float)a.basis_scale;
         const float vmax = kMagic + (float)(nsym - 1);
         const uint32_t len8_rel = smem_u32(s_len8) - kMagicBits;  // + (kMagicBits + q) = address of len8[q]
-        // runs of coefficients whose bits are added up separately: the chunks of a pixel, or --
-        // with one chunk per pixel or fewer -- two halves, so that the two threads of a pixel can
-        // pack side by side.  The bounds are multiples of 16.
-        const int n_runs = a.splits > 2 ? 4 : 2;
+        // Four runs of coefficients whose bits are added up separately, one per thread of a pixel,
+        // so that the four pack side by side: the chunks of a pixel, their halves, or quarters
+        // of the pixel.  The bounds are multiples of 16 (a chunk is a multiple of 16 coefficients).
         int bnd[5];
-        if (a.splits == 1) { bnd[0] = 0; bnd[1] = ((a.k + 31) / 32) * 16; bnd[2] = a.k; bnd[3] = bnd[4] = a.k; }
-        else
-            for (int v = 0; v <= 4; ++v) bnd[v] = min(v, a.splits) * (a.k / a.splits);
-        const int run_lo = half * (n_runs / 2), run_hi = run_lo + n_runs / 2;      // this thread packs runs [run_lo, run_hi)
+        {
+            const int n_chunk = a.k / a.splits;                          // coefficients per chunk of a pixel
+            const int per = 4 / a.splits;                                // runs per chunk: 4, 2 or 1
+            const int step = ((n_chunk + 16 * per - 1) / (16 * per)) * 16;
+            for (int v = 0; v <= 4; ++v) {
+                const int c = v / per, r = v - c * per;
+                bnd[v] = min(c * n_chunk + min(r * step, n_chunk), a.k);
+            }
+        }
+        const int run_lo = part, run_hi = part + 1;                      // this thread packs run `part`
         long long work = 0;
         bool alive = true;
 
@@ -251,9 +269,8 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
             const long long tile = blockIdx.x + tl * gridDim.x;
             const long long p = tile * TC_TILE_PIXELS + m;
             const bool valid = p < a.pixels;
-            s_part[(2 * half) * TC_TILE_PIXELS + m] = 0u;
-            s_part[(2 * half + 1) * TC_TILE_PIXELS + m] = 0u;
-            named_bar_sync(kEpiBar, 256);          // the previous tile's symbols have been packed; the sums are zero
+            s_part[part * TC_TILE_PIXELS + m] = 0u;
+            named_bar_sync(kEpiBar, kEpiThreads);  // the previous tile's symbols have been packed; the sums are zero
 
             // pass 1: quantise block by block, park the symbols, add up the code lengths
             for (int nb = 0; nb < n_blocks && alive; ++nb, ++work) {
@@ -261,9 +278,9 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
                 if (!mbar_wait(smem_u32(&s_tfull[acc]), (uint32_t)((work >> 1) & 1))) { alive = false; break; }
                 tc_fence_after_sync();
                 const int ncols = min(kBlockCoef, a.k - nb * kBlockCoef);
-                const int half_cols = ((ncols + 31) / 32) * 16;
-                const int col0 = half * half_cols;
-                const int my_n = half ? ncols - half_cols : half_cols;
+                const int part_cols = ((ncols + 63) / 64) * 16;
+                const int col0 = part * part_cols;
+                const int my_n = max(0, min(part_cols, ncols - col0));
                 const uint32_t trow = tmem_base + acc * kBlockCoef + ((uint32_t)(wq * 32) << 16) + col0;
 #pragma unroll 1
                 for (int blk = 0; blk * 16 < my_n; ++blk) {
@@ -303,13 +320,13 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
                 mbar_arrive(smem_u32(&s_tempty[acc]));
             }
             if (!alive) break;
-            named_bar_sync(kEpiBar, 256);          // every run's sum is complete
+            named_bar_sync(kEpiBar, kEpiThreads);  // every run's sum is complete
 
             // bit offsets: pixel-major, runs in order inside a pixel
             unsigned int run_bits[4], pixel_bits = 0, before_mine = 0, my_bits = 0;
 #pragma unroll
             for (int v = 0; v < 4; ++v) {
-                run_bits[v] = v < n_runs ? s_part[v * TC_TILE_PIXELS + m] : 0u;
+                run_bits[v] = s_part[v * TC_TILE_PIXELS + m];
                 if (v < run_lo) before_mine += run_bits[v];
                 if (v >= run_lo && v < run_hi) my_bits += run_bits[v];
                 pixel_bits += run_bits[v];
@@ -320,12 +337,12 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
                 const unsigned int up = __shfl_up_sync(0xffffffffu, inc, d);
                 if (lane >= d) inc += up;
             }
-            if (lane == 31) s_warp_sums[half][wq] = inc;
-            named_bar_sync(kEpiBar, 256);
+            if (lane == 31) s_warp_sums[part][wq] = inc;
+            named_bar_sync(kEpiBar, kEpiThreads);
             unsigned int before = 0, tile_bits = 0;
 #pragma unroll
             for (int w = 0; w < 4; ++w) {
-                const unsigned int sw = s_warp_sums[half][w];
+                const unsigned int sw = s_warp_sums[part][w];
                 if (w < wq) before += sw;
                 tile_bits += sw;
             }
@@ -336,11 +353,11 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
                 const int cpx = a.chunk_pixels;
                 if (cpx < 32) {
                     const unsigned int further = __shfl_down_sync(0xffffffffu, pixel_off, cpx);
-                    chunk_end = (lane + cpx < 32) ? further : before + s_warp_sums[half][wq];
+                    chunk_end = (lane + cpx < 32) ? further : before + s_warp_sums[part][wq];
                 } else {
 #pragma unroll
                     for (int w = 0; w < 4; ++w)
-                        if (w < wq + (cpx >> 5)) chunk_end += s_warp_sums[half][w];
+                        if (w < wq + (cpx >> 5)) chunk_end += s_warp_sums[part][w];
                 }
             }
             const unsigned long long padded = ((unsigned long long)tile_bits + 127ull) & ~127ull;
@@ -360,22 +377,23 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
             }
             // chunk lengths
             if (valid) {
-                if (a.splits > 1) {
-                    for (int v = run_lo; v < run_hi; ++v)
-                        if (v < a.splits) a.chunk_len[p * a.splits + v] = (uint16_t)run_bits[v];
-                } else if (half == 0) {
+                if (a.splits == 4) {
+                    a.chunk_len[p * 4 + part] = (uint16_t)run_bits[part];
+                } else if (a.splits == 2) {
+                    if ((part & 1) == 0) a.chunk_len[p * 2 + (part >> 1)] = (uint16_t)(run_bits[part] + run_bits[part + 1]);
+                } else if (part == 0) {
                     if (a.chunk_pixels == 1) a.chunk_len[p] = (uint16_t)pixel_bits;
                     else if ((p % a.chunk_pixels) == 0) a.chunk_len[p / a.chunk_pixels] = (uint16_t)(chunk_end - pixel_off);
                 }
             }
-            named_bar_sync(kEpiBar, 256);          // the tile's position is known
+            named_bar_sync(kEpiBar, kEpiThreads);  // the tile's position is known
             const unsigned long long base = s_base;
             const bool write_ok = s_write_ok != 0;
             if (write_ok) {
                 uint4 *z = reinterpret_cast<uint4 *>(a.stream + (base >> 5));
-                for (unsigned int i = tid; i < (unsigned int)(padded >> 7); i += 256) z[i] = make_uint4(0u, 0u, 0u, 0u);
+                for (unsigned int i = tid; i < (unsigned int)(padded >> 7); i += kEpiThreads) z[i] = make_uint4(0u, 0u, 0u, 0u);
             }
-            named_bar_sync(kEpiBar, 256);          // the tile's words are zero
+            named_bar_sync(kEpiBar, kEpiThreads);  // the tile's words are zero
 
             // pass 2: codes of the parked symbols, packed into the stream
             if (valid && write_ok && my_bits > 0) {
@@ -395,7 +413,7 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
                 w.finish();
             }
         }
-        if (!alive && (tid & 255) == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
+        if (!alive && tid == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
     }
 
     // ---- teardown ---------------------------------------------------------------------
