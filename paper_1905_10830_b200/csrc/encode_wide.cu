@@ -17,6 +17,7 @@
 //   warp 24       one thread issues tcgen05.mma:  D[pixel][coef] = X[pixel][c] * T[coef][c]
 #include <cstdio>
 #include <cstdlib>
+#include <cstring>
 
 #include "device_utils.cuh"
 #include "sm100_ptx.cuh"
@@ -70,10 +71,15 @@ __device__ __forceinline__ uint32_t quantise_bits(uint32_t acc_bits, float inv_s
     return __float_as_uint(fminf(fmaxf(fmaf(__uint_as_float(acc_bits), inv_step, bias) + kMagic, kMagic), vmax));
 }
 
-template <bool kPerChannel, bool kDebug>
-__global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, int smem_budget)
+// kTma: the basis pieces arrive by tiled TMA copies (one instruction per stage, 64-byte swizzle)
+// instead of 1024 cp.async copies; `bmap` is then the tensor map of the basis.
+template <bool kPerChannel, bool kDebug, bool kTma>
+__global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, int smem_budget,
+                                                                  const __grid_constant__ CUtensorMap bmap)
 {
-    extern __shared__ __align__(128) unsigned char smem[];
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    // the swizzled basis pieces want their 512-byte atoms aligned; the ring starts the buffer
+    unsigned char *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     __shared__ __align__(8) unsigned long long s_full[kMaxStages], s_empty[kMaxStages], s_tfull[2], s_tempty[2];
     __shared__ uint32_t s_tmem_base;
     __shared__ unsigned int s_warp_sums[4][4];
@@ -96,7 +102,7 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
 
     // ---- set-up ---------------------------------------------------------------------
     if (tid == 0) {
-        for (int s = 0; s < kMaxStages; ++s) { mbar_init(smem_u32(&s_full[s]), 256); mbar_init(smem_u32(&s_empty[s]), 1); }
+        for (int s = 0; s < kMaxStages; ++s) { mbar_init(smem_u32(&s_full[s]), kTma ? 257 : 256); mbar_init(smem_u32(&s_empty[s]), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&s_tfull[b]), 1); mbar_init(smem_u32(&s_tempty[b]), kEpiThreads); }
         mbar_fence_init();
     }
@@ -161,7 +167,14 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
                     const int k0 = kp * kPanelCh;
                     const int nk8 = min(kPanelCh, a.c - k0) >> 3;
                     const uint32_t stage_a = ring_addr + s * kStageBytes, stage_b = stage_a + kStageA;
-                    {
+                    if constexpr (kTma) {
+                        // one thread asks for the 256 x 32 box at (channel k0, coefficient j0); rows and
+                        // channels past the matrix arrive as zeros and count towards the bytes
+                        if (lt == 0) {
+                            mbar_arrive_expect_tx(smem_u32(&s_full[s]), (uint32_t)kStageB);
+                            tma_load_2d(stage_b, &bmap, k0, j0, smem_u32(&s_full[s]));
+                        }
+                    } else {
                         const bool ok = c8 < nk8;
                         const __nv_bfloat16 *src = ok ? b_src + k0 : a.basis_bf16;
 #pragma unroll
@@ -193,16 +206,15 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
                         if (lag == 3) cp_async_wait<3>();
                         else if (lag == 2) cp_async_wait<2>();
                         else cp_async_wait<1>();
-                        fence_proxy_async_smem();
                         mbar_arrive(smem_u32(&s_full[(it - lag) % stages]));
                     }
                 }
             }
         }
         if (alive) {
-            if (lag >= 3 && it >= 3) { cp_async_wait<2>(); fence_proxy_async_smem(); mbar_arrive(smem_u32(&s_full[(it - 3) % stages])); }
-            if (lag >= 2 && it >= 2) { cp_async_wait<1>(); fence_proxy_async_smem(); mbar_arrive(smem_u32(&s_full[(it - 2) % stages])); }
-            if (it >= 1) { cp_async_wait<0>(); fence_proxy_async_smem(); mbar_arrive(smem_u32(&s_full[(it - 1) % stages])); }
+            if (lag >= 3 && it >= 3) { cp_async_wait<2>(); mbar_arrive(smem_u32(&s_full[(it - 3) % stages])); }
+            if (lag >= 2 && it >= 2) { cp_async_wait<1>(); mbar_arrive(smem_u32(&s_full[(it - 2) % stages])); }
+            if (it >= 1) { cp_async_wait<0>(); mbar_arrive(smem_u32(&s_full[(it - 1) % stages])); }
         } else {
             cp_async_wait<0>();
             tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
@@ -224,12 +236,16 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
                     for (int kp = 0; kp < n_panels; ++kp, ++it) {
                         const int s = it % stages;
                         if (!mbar_wait(smem_u32(&s_full[s]), (it / stages) & 1)) { alive = false; break; }
+                        // the panel was written by the 256 loader threads (cp.async, plain stores), all of
+                        // which have arrived on the barrier: one proxy fence here, between that
+                        // synchronisation and the MMA's operand reads, orders the writes for all of them
+                        fence_proxy_async_smem();
                         tc_fence_after_sync();
                         const int nk16 = min(kPanelCh, a.c - kp * kPanelCh) >> 4;
                         const uint32_t stage_a = ring_addr + s * kStageBytes, stage_b = stage_a + kStageA;
                         for (int q = 0; q < nk16; ++q) {
                             const uint64_t adesc = make_smem_desc(stage_a + q * 4096, 2048, 128);
-                            const uint64_t bdesc = make_smem_desc(stage_b + q * 256, 128, 512);
+                            const uint64_t bdesc = kTma ? make_smem_desc_sw64(stage_b + q * 32, 512) : make_smem_desc(stage_b + q * 256, 128, 512);
                             mma_bf16_ss(d_tmem, adesc, bdesc, idesc, (kp | q) != 0 ? 1u : 0u);
                         }
                         mma_commit(smem_u32(&s_empty[s]));
@@ -433,28 +449,35 @@ bool tc_encode_wide_supported(const tc_ctx *ctx, const EncodeArgs &a)
     if (a.splits != 1 && a.splits != 2 && a.splits != 4) return false;
     if (a.splits > 1 && (a.chunk_pixels != 1 || (a.k / a.splits) % 16 != 0 || a.k % a.splits != 0)) return false;
     if (a.groups != 1 && a.groups != a.k) return false;
-    const SmemLayout l = smem_layout(a.k, a.groups == 1 ? (1 << a.bits) : 0, ctx->max_smem_optin - 1024);
+    const SmemLayout l = smem_layout(a.k, a.groups == 1 ? (1 << a.bits) : 0, ctx->max_smem_optin - 2048);
     return l.stages >= 2;
 }
 
 tc_status tc_launch_encode_wide(const tc_ctx *ctx, const EncodeArgs &a, cudaStream_t s)
 {
     if (a.n_tiles <= 0) return TC_OK;
-    const int budget = ctx->max_smem_optin - 1024;            // leaves room for the static shared variables
+    const int budget = ctx->max_smem_optin - 2048;            // leaves room for the static shared variables
     const SmemLayout l = smem_layout(a.k, a.groups == 1 ? (1 << a.bits) : 0, budget);
     if (l.stages < 2) return TC_ERR_UNSUPPORTED;
     const bool per_channel = a.groups != 1, debug = a.dbg_coef || a.dbg_sym;
-    void (*kernel)(EncodeArgs, int) =
-        per_channel ? (debug ? encode_wide_kernel<true, true> : encode_wide_kernel<true, false>)
-                    : (debug ? encode_wide_kernel<false, true> : encode_wide_kernel<false, false>);
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.total) != cudaSuccess)
+    const bool tma = a.basis_map != nullptr;
+    void (*kernel)(EncodeArgs, int, const CUtensorMap) =
+        tma ? (per_channel ? (debug ? encode_wide_kernel<true, true, true> : encode_wide_kernel<true, false, true>)
+                           : (debug ? encode_wide_kernel<false, true, true> : encode_wide_kernel<false, false, true>))
+            : (per_channel ? (debug ? encode_wide_kernel<true, true, false> : encode_wide_kernel<true, false, false>)
+                           : (debug ? encode_wide_kernel<false, true, false> : encode_wide_kernel<false, false, false>));
+    const size_t smem_bytes = (size_t)l.total + 1024;         // room to align the buffer to 1 KB
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
         return TC_ERR_CUDA;
     const unsigned int grid = (unsigned int)((a.n_tiles < ctx->sm_count) ? a.n_tiles : ctx->sm_count);
     EncodeArgs args = a;
     int budget_arg = budget;
-    void *params[] = {&args, &budget_arg};
+    CUtensorMap map_arg;
+    if (tma) map_arg = *a.basis_map;
+    else memset(&map_arg, 0, sizeof(map_arg));
+    void *params[] = {&args, &budget_arg, &map_arg};
     // cooperative launch: the grid must be co-resident, which is what makes the look-back safe
-    const cudaError_t err = cudaLaunchCooperativeKernel((void *)kernel, dim3(grid), dim3(kThreads), params, l.total, s);
+    const cudaError_t err = cudaLaunchCooperativeKernel((void *)kernel, dim3(grid), dim3(kThreads), params, smem_bytes, s);
     if (err != cudaSuccess) {
         if (getenv("TC_VERBOSE")) fprintf(stderr, "tc: wide encode launch failed: %s\n", cudaGetErrorString(err));
         cudaGetLastError();

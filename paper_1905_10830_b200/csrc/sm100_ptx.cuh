@@ -1,6 +1,7 @@
 // Thin wrappers over the sm_100a PTX used by the tensor-core kernels: mbarriers with bounded
 // waits, cp.async, tcgen05 (TMEM allocation, MMA, commit, loads) and the shared-memory matrix
-// descriptors.  Everything here is cta_group::1 (one CTA per tile, no clusters, no multicast).
+// descriptors, tiled TMA loads.  Everything here is cta_group::1 (one CTA per tile, no clusters,
+// no multicast).
 #pragma once
 
 #include <stdint.h>
@@ -150,6 +151,39 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t 
     d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
     d |= 1ull << 46;       // descriptor version for this architecture
     return d;              // base offset 0, layout type 0 = no swizzle
+}
+
+// The same for a K-major operand that a tiled TMA copy with 64-byte swizzling wrote: rows of 64
+// bytes (32 bf16 along K), eight rows per 512-byte swizzle atom, the 16-byte pieces of row r
+// exchanged by XOR with (r / 2) % 4.  `sbo` is the distance between 8-row groups; the leading
+// offset is not used in this mode.  A K step of 16 elements inside the row adds 32 bytes to
+// the start address.  The buffer must be aligned to the atom.
+__device__ __forceinline__ uint64_t make_smem_desc_sw64(uint32_t smem_addr, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3fffu);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
+    d |= 1ull << 46;       // descriptor version for this architecture
+    d |= 4ull << 61;       // layout type: 64-byte swizzle
+    return d;
+}
+
+// ---- TMA (tiled bulk copy global -> shared, no multicast) -------------------------------------
+// The barrier is told how many bytes the copy will deliver; it completes the phase when they
+// have landed (and every other expected arrival has come).
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Box at element coordinates (x, y) of a 2-D tensor map; x * element size must be a multiple of
+// 16 bytes.  Out-of-range parts of the box arrive as zeros and count towards the bytes.
+__device__ __forceinline__ void tma_load_2d(uint32_t smem_dst, const void *tensor_map, int x, int y, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_dst), "l"(tensor_map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
 }
 
 // Instruction descriptor for kind::f16 with bf16 operands and fp32 accumulation.

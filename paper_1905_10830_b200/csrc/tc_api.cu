@@ -123,6 +123,20 @@ tc_status finish_model(tc_model *m)
             }
         if ((st = upload(&m->d_basis_bf16, b)) != TC_OK) return st;
         if ((st = upload(&m->d_basis_t_bf16, bt)) != TC_OK) return st;
+        // Tensor map for the kernels that stream the basis: boxes of 256 coefficient rows x 32
+        // channels (64 bytes), written with the 64-byte swizzle the MMA descriptor names.  Needs
+        // rows of a multiple of 16 bytes; without a map those kernels copy the basis with cp.async.
+        m->has_basis_map = false;
+        if (c % 16 == 0) {
+            const cuuint64_t dims[2] = {(cuuint64_t)c, (cuuint64_t)k};
+            const cuuint64_t strides[1] = {(cuuint64_t)c * 2};
+            const cuuint32_t box[2] = {32u, 256u};
+            const cuuint32_t elem[2] = {1u, 1u};
+            const CUresult rc = cuTensorMapEncodeTiled(&m->basis_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, m->d_basis_bf16, dims,
+                                                       strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
+                                                       CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            m->has_basis_map = rc == CUDA_SUCCESS;
+        }
     }
     return TC_OK;
 }
@@ -698,6 +712,7 @@ tc_status tc_encode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
     a.tile_state = (unsigned long long *)((char *)ctx->scratch + 64);
     a.status = ctx->d_status; a.clamped = nullptr; a.emit = 1;
     a.basis_bf16 = m->d_basis_bf16; a.enc_bias = m->d_enc_bias; a.tmu32 = m->d_tmu32;
+    a.basis_map = m->has_basis_map ? &m->basis_map : nullptr;
     if (!ctx->force_exact && x->dtype == TC_BF16 && tc_encode_tc_supported(ctx, a)) {
         ctx->last_encode_path = 1;
         return tc_launch_encode_tc(ctx, a, s);

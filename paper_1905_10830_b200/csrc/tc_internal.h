@@ -1,6 +1,7 @@
 // Internal declarations shared by the host API and the kernels of the codec library.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -48,6 +49,8 @@ struct tc_model {
     float *d_enc_bias = nullptr;            // [k]  -(T mu + lo)_j / step
     float *d_dec_bias = nullptr;            // [c]  mu_c + (lo + center*step) * sum_j T[j][c]
     float *d_tmu32 = nullptr;               // [k]  (T mu)_j
+    CUtensorMap basis_map;                  // d_basis_bf16 as a [k][c] tensor, boxes of 256 rows x 32 channels, 64-byte swizzle
+    bool has_basis_map = false;
 };
 
 struct tc_codebook {
@@ -71,6 +74,7 @@ struct EncodeArgs {
     const double *basis64;      // [c][c]
     const double *mean64;       // [c]
     const __nv_bfloat16 *basis_bf16;   // [k][c]  (tensor-core path)
+    const CUtensorMap *basis_map;      // HOST pointer to the model's tensor map of basis_bf16, or null
     const float *enc_bias;      // [k]  -(T mu + lo)_j / step
     const float *tmu32;         // [k]  (T mu)_j
     double lo, step;
