@@ -16,6 +16,8 @@
 //                 round to bf16, NCHW stores; runs while the VLD warps decode the next item
 // Dequantisation is folded as in the resident-basis kernel:
 // bias_c = mu_c + (lo + center * step) * sum_j T[j][c].
+#include <cstring>
+
 #include "device_utils.cuh"
 #include "sm100_ptx.cuh"
 
@@ -64,10 +66,14 @@ __host__ __device__ inline SmemLayout smem_layout(int c, int k, int lut_entries,
     return l;
 }
 
-template <bool kPerChannel>
-__global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a)
+// kTma: the panels of the transposed basis arrive by tiled TMA copies (one instruction per stage,
+// 128-byte swizzle) instead of 1024 cp.async copies; `tmap` is then its tensor map.
+template <bool kPerChannel, bool kTma>
+__global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap tmap)
 {
-    extern __shared__ __align__(128) unsigned char smem[];
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    // the swizzled panels want their 1 KB atoms aligned; the ring starts the buffer
+    unsigned char *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     __shared__ __align__(8) unsigned long long s_full[kMaxStages], s_empty[kMaxStages];
     __shared__ __align__(8) unsigned long long s_bfull, s_bfree, s_tfull, s_tempty;
     __shared__ uint32_t s_tmem_base;
@@ -89,7 +95,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a)
 
     // ---- set-up ---------------------------------------------------------------------
     if (tid == 0) {
-        for (int s = 0; s < kMaxStages; ++s) { mbar_init(smem_u32(&s_full[s]), 128); mbar_init(smem_u32(&s_empty[s]), 1); }
+        for (int s = 0; s < kMaxStages; ++s) { mbar_init(smem_u32(&s_full[s]), kTma ? 1 : 128); mbar_init(smem_u32(&s_empty[s]), 1); }
         mbar_init(smem_u32(&s_bfull), kVldThreads);
         mbar_init(smem_u32(&s_bfree), 1);
         mbar_init(smem_u32(&s_tfull), 1);
@@ -299,6 +305,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a)
         int it = 0;
         bool alive = true;
         for (long long n = 0; n < my_items && alive; ++n) {
+            if (kTma && lt != 0) break;                       // one thread asks for the boxes
             for (int jp = 0; jp < n_kpanels && alive; ++jp) {
                 const int j0 = jp * kPanelK;
                 const int nk8 = min(kPanelK, a.k - j0) >> 3;
@@ -306,6 +313,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a)
                     const int s = it % stages;
                     if (!mbar_wait(smem_u32(&s_empty[s]), ((it / stages) & 1) ^ 1)) { alive = false; break; }
                     const uint32_t stage = ring_addr + s * kStageBytes;
+                    if constexpr (kTma) {
+                        // box of 128 channels x 64 coefficients at (coefficient j0, channel blk * 128); rows
+                        // and columns past the matrix arrive as zeros and count towards the bytes
+                        mbar_arrive_expect_tx(smem_u32(&s_full[s]), (uint32_t)kStageBytes);
+                        tma_load_2d(stage, &tmap, j0, blk * 128, smem_u32(&s_full[s]));
+                        continue;
+                    }
                     // transposed basis rows (channels) blk * 128 ..., coefficients j0 ...: K-major core
                     // matrices (row / 8) * 1024 + (j / 8) * 128 + (row % 8) * 16; rows past C are zero
                     for (int i = lt; i < 128 * 8; i += 128) {
@@ -324,7 +338,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a)
                 }
             }
         }
-        if (alive) {
+        if (kTma) {
+            if (!alive) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
+        } else if (alive) {
             if (it >= 2) { cp_async_wait<1>(); fence_proxy_async_smem(); mbar_arrive(smem_u32(&s_full[(it - 2) % stages])); }
             if (it >= 1) { cp_async_wait<0>(); fence_proxy_async_smem(); mbar_arrive(smem_u32(&s_full[(it - 1) % stages])); }
         } else {
@@ -353,7 +369,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a)
                         tc_fence_after_sync();
                         const uint32_t stage = ring_addr + s * kStageBytes;
                         for (int q = 0; q < nk16; ++q) {
-                            const uint64_t adesc = make_smem_desc(stage + q * 256, 128, 1024);
+                            const uint64_t adesc = kTma ? make_smem_desc_sw128(stage + q * 32, 1024) : make_smem_desc(stage + q * 256, 128, 1024);
                             const uint64_t bdesc = make_smem_desc(bop_addr + (uint32_t)((j0 + 16 * q) >> 3) * b_lbo, b_lbo, 128);
                             mma_bf16_ss(tmem_base + (uint32_t)(blk * NP), adesc, bdesc, idesc, (jp | q) != 0 ? 1u : 0u);
                         }
@@ -387,7 +403,7 @@ bool tc_decode_wide_supported(const tc_ctx *ctx, const DecodeArgs &a)
     if (a.splits > 1 && (a.chunk_pixels != 1 || a.k % a.splits != 0 || (a.k / a.splits) % 8 != 0)) return false;
     if (a.groups != 1 && a.groups != a.k) return false;
     if (a.lut_bits > TC_MAX_CODE_LEN) return false;
-    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, ctx->max_smem_optin - 1024);
+    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, ctx->max_smem_optin - 2048);
     if (l.stages < 2) return false;
     return a.chunk_pixels <= l.np;                            // a chunk lies inside one work item
 }
@@ -396,14 +412,21 @@ tc_status tc_launch_decode_wide(const tc_ctx *ctx, const DecodeArgs &a, cudaStre
 {
     if (a.n_tiles <= 0) return TC_OK;
     DecodeArgs args = a;
-    args.smem_budget = ctx->max_smem_optin - 1024;            // leaves room for the static shared variables
+    args.smem_budget = ctx->max_smem_optin - 2048;            // leaves room for the static shared variables
     const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, args.smem_budget);
     if (l.stages < 2) return TC_ERR_UNSUPPORTED;
-    void (*kernel)(DecodeArgs) = a.groups != 1 ? decode_wide_kernel<true> : decode_wide_kernel<false>;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.total) != cudaSuccess)
+    const bool tma = a.basis_t_map != nullptr;
+    void (*kernel)(DecodeArgs, const CUtensorMap) =
+        tma ? (a.groups != 1 ? decode_wide_kernel<true, true> : decode_wide_kernel<false, true>)
+            : (a.groups != 1 ? decode_wide_kernel<true, false> : decode_wide_kernel<false, false>);
+    const size_t smem_bytes = (size_t)l.total + 1024;         // room to align the buffer to 1 KB
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
         return TC_ERR_CUDA;
     const long long n_items = a.n_tiles * (TC_TILE_PIXELS / l.np);
     const unsigned int grid = (unsigned int)((n_items < ctx->sm_count) ? n_items : ctx->sm_count);
-    kernel<<<grid, kThreads, l.total, s>>>(args);
+    CUtensorMap map_arg;
+    if (tma) map_arg = *a.basis_t_map;
+    else memset(&map_arg, 0, sizeof(map_arg));
+    kernel<<<grid, kThreads, smem_bytes, s>>>(args, map_arg);
     return cudaGetLastError() == cudaSuccess ? TC_OK : TC_ERR_CUDA;
 }

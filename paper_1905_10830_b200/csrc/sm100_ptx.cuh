@@ -169,6 +169,19 @@ __device__ __forceinline__ uint64_t make_smem_desc_sw64(uint32_t smem_addr, uint
     return d;
 }
 
+// The same with 128-byte swizzling: rows of 128 bytes (64 bf16 along K), eight rows per 1 KB
+// atom, the 16-byte pieces of row r exchanged by XOR with r % 8.
+__device__ __forceinline__ uint64_t make_smem_desc_sw128(uint32_t smem_addr, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3fffu);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
+    d |= 1ull << 46;       // descriptor version for this architecture
+    d |= 2ull << 61;       // layout type: 128-byte swizzle
+    return d;
+}
+
 // ---- TMA (tiled bulk copy global -> shared, no multicast) -------------------------------------
 // The barrier is told how many bytes the copy will deliver; it completes the phase when they
 // have landed (and every other expected arrival has come).

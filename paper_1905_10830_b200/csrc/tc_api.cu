@@ -67,7 +67,10 @@ bool resolve_chunks(const tc_encode_params *p, int k, int max_len, ChunkShape *o
     if (p && p->chunk_pixels) cp = p->chunk_pixels;
     else while (cp < TC_TILE_PIXELS && cp * k < 128) cp <<= 1;
     if (cp < 1 || cp > TC_TILE_PIXELS || (cp & (cp - 1)) != 0) return false;
-    int splits = (p && p->pixel_splits) ? p->pixel_splits : ((cp == 1 && k >= 256 && k % 32 == 0) ? 2 : 1);
+    // default: a chunk of 128 .. 255 symbols where the shape allows it -- two chunks per pixel
+    // from 256 coefficients, four from 512
+    int splits = (p && p->pixel_splits) ? p->pixel_splits
+                 : (cp == 1 && k >= 512 && k % 64 == 0) ? 4 : ((cp == 1 && k >= 256 && k % 32 == 0) ? 2 : 1);
     if (splits != 1 && splits != 2 && splits != 4) return false;
     if (splits > 1 && (cp != 1 || k % (8 * splits) != 0)) return false;
     if ((long long)cp * k / splits * max_len > 65535) return false;     // a chunk length has 16 bits
@@ -136,6 +139,18 @@ tc_status finish_model(tc_model *m)
                                                        strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
                                                        CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             m->has_basis_map = rc == CUDA_SUCCESS;
+        }
+        // and for the decoder: the transposed basis in boxes of 128 channel rows x 64 coefficients
+        m->has_basis_t_map = false;
+        if (k % 16 == 0) {
+            const cuuint64_t dims[2] = {(cuuint64_t)k, (cuuint64_t)c};
+            const cuuint64_t strides[1] = {(cuuint64_t)k * 2};
+            const cuuint32_t box[2] = {64u, 128u};
+            const cuuint32_t elem[2] = {1u, 1u};
+            const CUresult rc = cuTensorMapEncodeTiled(&m->basis_t_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, m->d_basis_t_bf16, dims,
+                                                       strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                                       CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            m->has_basis_t_map = rc == CUDA_SUCCESS;
         }
     }
     return TC_OK;
@@ -753,6 +768,7 @@ tc_status tc_decode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
     a.xhat = x_hat->data; a.status = ctx->d_status;
     a.lut32 = cb->d_lut32; a.basis_t_bf16 = m->d_basis_t_bf16; a.dec_bias = m->d_dec_bias; a.center = m->center;
     a.relu = (params && params->relu) ? 1 : 0;
+    a.basis_t_map = m->has_basis_t_map ? &m->basis_t_map : nullptr;
     if (!ctx->force_exact && x_hat->dtype == TC_BF16 && tc_decode_tc_supported(ctx, a)) {
         ctx->last_decode_path = 1;
         return tc_launch_decode_tc(ctx, a, (cudaStream_t)cuda_stream);

@@ -51,6 +51,8 @@ struct tc_model {
     float *d_tmu32 = nullptr;               // [k]  (T mu)_j
     CUtensorMap basis_map;                  // d_basis_bf16 as a [k][c] tensor, boxes of 256 rows x 32 channels, 64-byte swizzle
     bool has_basis_map = false;
+    CUtensorMap basis_t_map;                // d_basis_t_bf16 as a [c][k] tensor, boxes of 128 channel rows x 64 coefficients, 128-byte swizzle
+    bool has_basis_t_map = false;
 };
 
 struct tc_codebook {
@@ -108,6 +110,7 @@ struct DecodeArgs {
     const uint16_t *lut;
     const uint32_t *lut32;              // tensor-core path
     const __nv_bfloat16 *basis_t_bf16;  // [c][k]
+    const CUtensorMap *basis_t_map;     // HOST pointer to the model's tensor map of basis_t_bf16, or null
     const float *dec_bias;              // [c]
     int center;                         // subtracted from every symbol before the MMA
     int relu;                           // x_hat = max(x_hat, 0) before it is rounded to the tensor type
