@@ -59,7 +59,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     if (not os.path.exists(LIB)) or any(os.path.getmtime(o) > os.path.getmtime(LIB) for o in objs):
         tmp = LIB + f".{os.getpid()}.tmp"
         subprocess.check_call([NVCC, "-shared", "-gencode", "arch=compute_100a,code=sm_100a",
-                               "-o", tmp, *objs, "-lcuda"])
+                               "-o", tmp, *objs])
         os.replace(tmp, LIB)
     return LIB
 

@@ -9,6 +9,27 @@
 
 #include "tc_internal.h"
 
+// cuTensorMapEncodeTiled, looked up through the runtime so that the library does not link the
+// driver library (it must load, for the host-side entry points, on machines without a driver).
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = []() -> EncodeTiledFn {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        return (EncodeTiledFn)p;
+    }();
+    return fn;
+}
+
+
 #define TC_CUDA(call)                                   \
     do {                                                \
         if ((call) != cudaSuccess) { cudaGetLastError(); return TC_ERR_CUDA; } \
@@ -130,24 +151,25 @@ tc_status finish_model(tc_model *m)
         // channels (64 bytes), written with the 64-byte swizzle the MMA descriptor names.  Needs
         // rows of a multiple of 16 bytes; without a map those kernels copy the basis with cp.async.
         m->has_basis_map = false;
-        if (c % 16 == 0) {
+        const EncodeTiledFn encode_tiled = encode_tiled_fn();
+        if (encode_tiled && c % 16 == 0) {
             const cuuint64_t dims[2] = {(cuuint64_t)c, (cuuint64_t)k};
             const cuuint64_t strides[1] = {(cuuint64_t)c * 2};
             const cuuint32_t box[2] = {32u, 256u};
             const cuuint32_t elem[2] = {1u, 1u};
-            const CUresult rc = cuTensorMapEncodeTiled(&m->basis_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, m->d_basis_bf16, dims,
+            const CUresult rc = encode_tiled(&m->basis_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, m->d_basis_bf16, dims,
                                                        strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
                                                        CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             m->has_basis_map = rc == CUDA_SUCCESS;
         }
         // and for the decoder: the transposed basis in boxes of 128 channel rows x 64 coefficients
         m->has_basis_t_map = false;
-        if (k % 16 == 0) {
+        if (encode_tiled && k % 16 == 0) {
             const cuuint64_t dims[2] = {(cuuint64_t)k, (cuuint64_t)c};
             const cuuint64_t strides[1] = {(cuuint64_t)k * 2};
             const cuuint32_t box[2] = {64u, 128u};
             const cuuint32_t elem[2] = {1u, 1u};
-            const CUresult rc = cuTensorMapEncodeTiled(&m->basis_t_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, m->d_basis_t_bf16, dims,
+            const CUresult rc = encode_tiled(&m->basis_t_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, m->d_basis_t_bf16, dims,
                                                        strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                                        CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             m->has_basis_t_map = rc == CUDA_SUCCESS;
