@@ -5,12 +5,13 @@
 // One persistent block per SM walks work items of NP pixels: a whole tile of 128 pixels up to
 // 512 channels, half a tile beyond (the accumulators of all channels, NP columns per block of
 // 128 channels, fill tensor memory exactly).  Per item:
-//   warps 0-7     VLD: one thread per chunk walks the bit stream (global memory, table-driven
-//                 canonical Huffman) and writes the symbols minus the centre symbol, as exact
+//   warps 0-7     VLD: one thread per chunk walks the bit stream (the item's segment staged in
+//                 shared memory when it fits, table-driven canonical Huffman) and writes the symbols minus the centre symbol, as exact
 //                 bf16 integers, into the K-major B operand, which holds all K coefficients of
 //                 the item's pixels (2 K NP bytes)
 //   warps 16-19   loaders: the transposed basis streams from L2 through a ring of
-//                 128-channel x 64-coefficient panels (cp.async, K-major core matrices)
+//                 128-channel x 64-coefficient panels (one tiled TMA copy with 128-byte swizzle
+//                 per panel, issued by one thread; cp.async copies without a tensor map)
 //   warp 20       one thread issues tcgen05.mma:  D[c][pixel] += T[j][c] * (Q[pixel][j] - center)
 //   warps 8-15    epilogue: TMEM -> registers (lane = channel), x_hat = step * acc + bias_c,
 //                 round to bf16, NCHW stores; runs while the VLD warps decode the next item

@@ -5,7 +5,8 @@
 // One persistent block per SM walks tiles of 128 consecutive pixels.  The coefficients of a
 // tile are produced in blocks of up to 256 (one accumulator of tensor memory each, two
 // accumulators in flight); for every block the pixels' channels stream through a ring of
-// 32-channel panels together with the matching 256 x 32 piece of the basis, both read from L2.
+// 32-channel panels together with the matching 256 x 32 piece of the basis, both read from L2
+// (the basis piece as one tiled TMA copy with 64-byte swizzle, the pixels by the loader warps).
 //   warps 0-15    epilogue: four warps per quarter of a block's coefficients (a warp reads its own
 //                 32 lanes of tensor memory).  Pass 1 (per block): TMEM -> registers, quantise, code length,
 //                 symbols parked in shared memory (one byte each, K x 128 per tile), bits added up

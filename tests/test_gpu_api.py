@@ -228,3 +228,59 @@ def test_roundtrip_host_matches_the_device_path(ctx, dtype):
     assert bits == enc.total_bits()
     assert torch.equal(host_out, dev.cpu())
     m.close(); cb.close()
+
+
+# ---- the same robustness checks on the tensor-core routes (1: basis resident, 3: basis streamed) ----
+
+@pytest.mark.parametrize("c,s,n,route", [(64, 16, 3, 1), (320, 8, 5, 3), (576, 7, 6, 3)])
+def test_tensor_core_routes_overflow_corruption_and_repeatability(ctx, c, s, n, route):
+    spec = fm.LayerSpec(c, s, s, 0.9, None, 520 + c)
+    o = H.oracle_side(spec, 5, max(4, (2 * c) // (s * s) + 1), n, torch.bfloat16, False)
+    m = H.import_model(tc, ctx, o["model"], torch.bfloat16)
+    cb = tc.tc_codebook_import(ctx, o["lengths"], 5)
+    x = o["x"].cuda()
+    enc = tc.tc_encode(ctx, m, cb, x)
+    assert tc.tc_get_status(ctx) == 0 and tc.tc_last_path(ctx) == route
+    nbytes = enc.total_bits() // 8
+    lay = enc.layout
+    ref = tc.tc_decode(ctx, m, cb, enc, x.shape, x.dtype, stream_bytes=nbytes)
+    assert tc.tc_get_status(ctx) == 0 and tc.tc_last_path(ctx, True) == route
+    # repeated encodes write the same bytes
+    again = tc.tc_encode(ctx, m, cb, x)
+    assert torch.equal(again.words[:nbytes], enc.words[:nbytes]) and torch.equal(again.tile_off, enc.tile_off)
+    assert torch.equal(again.chunk_len[:lay.n_chunks], enc.chunk_len[:lay.n_chunks])
+    # capacity overflow: reported, nothing written past the capacity; exact capacity works
+    guard = 4096
+    buf = torch.full((nbytes + guard,), 0xAB, dtype=torch.uint8, device="cuda")
+    small = tc.EncodedStream(buf, torch.empty(lay.n_chunks + (lay.n_chunks & 1), dtype=torch.int16, device="cuda"),
+                             torch.empty(lay.n_tiles + 1, dtype=torch.int64, device="cuda"), lay)
+    cap = (nbytes // 2) & ~15
+    tc.tc_encode(ctx, m, cb, x, out=small, capacity=cap)
+    assert tc.tc_get_status(ctx) == 3
+    assert bool((buf[cap:] == 0xAB).all())
+    tc.tc_encode(ctx, m, cb, x, out=small, capacity=nbytes)
+    assert tc.tc_get_status(ctx) == 0
+    assert torch.equal(buf[:nbytes], enc.words[:nbytes]) and bool((buf[nbytes:] == 0xAB).all())
+    # corrupt streams (made on the host): reported, never a fault
+    tc.tc_decode(ctx, m, cb, enc, x.shape, x.dtype, stream_bytes=(nbytes // 2) & ~15)
+    assert tc.tc_get_status(ctx) == 5
+    for bad_value in (nbytes * 8 + 128, 64, -128):
+        broken = tc.EncodedStream(enc.words, enc.chunk_len, enc.tile_off.clone(), lay)
+        broken.tile_off[1] = broken.tile_off[1] + bad_value if bad_value != 64 else 64
+        tc.tc_decode(ctx, m, cb, broken, x.shape, x.dtype, stream_bytes=nbytes)
+        assert tc.tc_get_status(ctx) == 5
+    for delta in (30000, 1, -1):
+        broken = tc.EncodedStream(enc.words, enc.chunk_len.clone(), enc.tile_off, lay)
+        broken.chunk_len[3] += delta
+        tc.tc_decode(ctx, m, cb, broken, x.shape, x.dtype, stream_bytes=nbytes)
+        assert tc.tc_get_status(ctx) == 5
+    noisy = tc.EncodedStream(enc.words.clone(), enc.chunk_len, enc.tile_off, lay)
+    g = torch.Generator(device="cuda").manual_seed(2)
+    idx = torch.randint(0, nbytes, (64,), generator=g, device="cuda")
+    noisy.words[idx] ^= 0x5A
+    out = tc.tc_decode(ctx, m, cb, noisy, x.shape, x.dtype, stream_bytes=nbytes)
+    assert tc.tc_get_status(ctx) in (0, 5) and out.shape == x.shape
+    # the intact stream still decodes to the same tensor afterwards
+    good = tc.tc_decode(ctx, m, cb, enc, x.shape, x.dtype, stream_bytes=nbytes)
+    assert tc.tc_get_status(ctx) == 0 and torch.equal(good, ref)
+    m.close(); cb.close()
