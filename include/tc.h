@@ -73,8 +73,9 @@ tc_status tc_get_status(tc_ctx *ctx, void *cuda_stream);
  * the basis in shared memory, wider layers (up to 1024 channels) and other map sizes the
  * kernels that stream it; shapes neither takes (channel or coefficient counts that are not
  * multiples of 16) run on plain fp32 kernels with the same arithmetic.  fp32 tensors run on
- * kernels that evaluate the definition in fp64.  With `on` != 0 every tensor takes the fp64
- * kernels. */
+ * kernels that evaluate the definition in fp64.  With `on` == 1 every tensor takes the fp64
+ * kernels; with `on` == 2 bf16 tensors skip the resident-basis kernels, so that the streaming
+ * kernels can be checked on the shapes both take; 0 restores the default. */
 void tc_force_exact_path(tc_ctx *ctx, int on);
 /* Which kernels the last tc_encode (decode == 0) or tc_decode (decode != 0) of this context
  * launched: 0 = fp64 kernels, 1 = tensor-core kernels with the basis resident in shared

@@ -230,7 +230,9 @@ def tc_create(device: int = 0) -> Context:
     return Context(out.value, device)
 
 
-def tc_force_exact_path(ctx: Context, on: bool) -> None:
+def tc_force_exact_path(ctx: Context, on) -> None:
+    """0 / False: default routes; 1 / True: fp64 kernels for everything; 2: bf16 tensors skip the
+    resident-basis tensor-core kernels (validation of the streaming kernels)."""
     load_library().tc_force_exact_path(ctx.ptr, int(on))
 
 

@@ -38,11 +38,15 @@ constexpr int kLag = 2;
 constexpr int kVldBar = 1;
 constexpr int kMaxTileChunks = 512;
 
+// Epilogue transpose block of one warp: 32 channel rows of 32 pixels (64 bytes) with 16 bytes
+// of padding, which keeps both the 16-byte row writes and the 8-byte reads spread over the banks.
+constexpr int kTrRowBytes = 80;
+constexpr int kTrWarpBytes = 32 * kTrRowBytes;
 constexpr int kSegBytes = 16384;                              // staged stream segment of one work item
 constexpr int kSegSlack = 32;                                 // the reader's window may look two words past the end
 
 struct SmemLayout {
-    uint32_t ring, bop, lut, start, seg, total;
+    uint32_t ring, bop, lut, start, tbuf, seg, total;
     int stages, np;
     bool staged;                                              // room for the segment buffer beside at least three stages
 };
@@ -52,7 +56,7 @@ __host__ __device__ inline SmemLayout smem_layout(int c, int k, int lut_entries,
     SmemLayout l;
     l.np = ((c + 127) / 128 <= 4) ? 128 : 64;
     const uint32_t bop_bytes = 2u * (uint32_t)k * (uint32_t)l.np;
-    const uint32_t fixed = bop_bytes + (uint32_t)lut_entries * 4u + (kMaxTileChunks + 8) * 4u;
+    const uint32_t fixed = bop_bytes + (uint32_t)lut_entries * 4u + (kMaxTileChunks + 8) * 4u + 16u + 8u * kTrWarpBytes;
     int stages = ((long long)budget - (long long)fixed - (kSegBytes + kSegSlack)) / kStageBytes;
     l.staged = stages >= 3;
     if (!l.staged) stages = ((long long)budget - (long long)fixed) / kStageBytes;
@@ -62,7 +66,8 @@ __host__ __device__ inline SmemLayout smem_layout(int c, int k, int lut_entries,
     l.bop = (uint32_t)(l.stages * kStageBytes);
     l.lut = l.bop + bop_bytes;
     l.start = l.lut + (uint32_t)lut_entries * 4u;
-    l.seg = (l.start + (kMaxTileChunks + 8) * 4u + 15u) & ~15u;
+    l.tbuf = (l.start + (kMaxTileChunks + 8) * 4u + 15u) & ~15u;      // eight warp-private transpose blocks (epilogue)
+    l.seg = l.tbuf + 8u * kTrWarpBytes;
     l.total = l.seg + (l.staged ? (uint32_t)(kSegBytes + kSegSlack) : 0u);
     return l;
 }
@@ -247,6 +252,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a, 
         __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(a.xhat);
         const bool vec = (a.hw & 3) == 0;                    // four aligned pixels lie inside one image, 8-byte aligned
         const long long img_stride = (long long)a.c * a.hw;
+        const uint32_t tb = smem_u32(smem + L.tbuf) + (uint32_t)ew * kTrWarpBytes;
+        const uint32_t tb_wr = tb + (uint32_t)lane * kTrRowBytes;                              // this thread's channel row
+        const uint32_t tb_rd = tb + (uint32_t)(lane >> 3) * kTrRowBytes + (uint32_t)(lane & 7) * 8u;
         bool alive = true;
         for (long long n = 0; n < my_items && alive; ++n) {
             const long long item = blockIdx.x + n * gridDim.x;
@@ -262,28 +270,60 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a, 
                 const bool ch_ok = ch < a.c;
                 const float bias = ch_ok ? __ldg(a.dec_bias + ch) : 0.f;
                 const uint32_t trow = tmem_base + (uint32_t)(blk * NP) + ((uint32_t)(wq * 32) << 16);
-                int s = s0;
-                __nv_bfloat16 *dst = out + img0 * img_stride + (long long)(ch_ok ? ch : 0) * a.hw + s;
-                for (int c0 = 0; c0 < NP; c0 += 16) {
-                    uint32_t r[16];
-                    tmem_ld_32x32b_x16(trow + c0, r);
-                    tmem_ld_wait();
-                    if (vec) {
+                if (vec) {
+                    // 32 pixels at a time: the thread rounds its channel's values and writes them as one
+                    // 64-byte row of the warp's block; the warp then reads the block back four rows per
+                    // instruction, so that every channel row leaves as 64 contiguous bytes
+                    const int pgrp = lane & 7, r_sub = lane >> 3;
+                    const int ch_base = blk * 128 + wq * 32;
+                    const long long pg = p_first + 4 * pgrp;
+                    long long img = pg < a.pixels ? pg / a.hw : 0;
+                    int sp = pg < a.pixels ? (int)(pg - img * a.hw) : 0;
+                    for (int c0 = 0; c0 < NP; c0 += 32) {
+                        uint32_t r[32];
+                        {
+                            uint32_t r16[16];
+                            tmem_ld_32x32b_x16(trow + c0, r16);
 #pragma unroll
-                        for (int g = 0; g < 4; ++g) {
-                            const __nv_bfloat162 h0 = __floats2bfloat162_rn(fmaxf(fmaf(__uint_as_float(r[4 * g]), step, bias), floor_v),
-                                                                            fmaxf(fmaf(__uint_as_float(r[4 * g + 1]), step, bias), floor_v));
-                            const __nv_bfloat162 h1 = __floats2bfloat162_rn(fmaxf(fmaf(__uint_as_float(r[4 * g + 2]), step, bias), floor_v),
-                                                                            fmaxf(fmaf(__uint_as_float(r[4 * g + 3]), step, bias), floor_v));
-                            if (ch_ok && c0 + 4 * g < n_valid)
-                                *reinterpret_cast<uint2 *>(dst) = make_uint2(*reinterpret_cast<const uint32_t *>(&h0),
-                                                                             *reinterpret_cast<const uint32_t *>(&h1));
-                            s += 4;
-                            const bool wrap = s >= a.hw;          // the next group starts the next image
-                            dst += wrap ? 4 + img_stride - a.hw : 4;
-                            s = wrap ? s - a.hw : s;
+                            for (int i = 0; i < 16; ++i) r[i] = r16[i];
+                            tmem_ld_32x32b_x16(trow + c0 + 16, r16);
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) r[16 + i] = r16[i];
                         }
-                    } else {
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            uint32_t h2[4];
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const __nv_bfloat162 h = __floats2bfloat162_rn(fmaxf(fmaf(__uint_as_float(r[8 * q + 2 * i]), step, bias), floor_v),
+                                                                               fmaxf(fmaf(__uint_as_float(r[8 * q + 2 * i + 1]), step, bias), floor_v));
+                                h2[i] = *reinterpret_cast<const uint32_t *>(&h);
+                            }
+                            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(tb_wr + q * 16), "r"(h2[0]), "r"(h2[1]),
+                                         "r"(h2[2]), "r"(h2[3]) : "memory");
+                        }
+                        __syncwarp();
+                        const bool px_ok = c0 + 4 * pgrp < n_valid;
+                        __nv_bfloat16 *row_ptr = out + img * img_stride + (long long)(ch_base + r_sub) * a.hw + sp;
+#pragma unroll
+                        for (int it = 0; it < 8; ++it) {
+                            uint32_t lo2, hi2;
+                            asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(lo2), "=r"(hi2) : "r"(tb_rd + it * 4 * kTrRowBytes));
+                            if (px_ok && ch_base + 4 * it + r_sub < a.c)
+                                *reinterpret_cast<uint2 *>(row_ptr + (long long)(4 * it) * a.hw) = make_uint2(lo2, hi2);
+                        }
+                        sp += 32;
+                        while (sp >= a.hw) { sp -= a.hw; ++img; }
+                        __syncwarp();                                   // the block may be overwritten
+                    }
+                } else {
+                    int s = s0;
+                    __nv_bfloat16 *dst = out + img0 * img_stride + (long long)(ch_ok ? ch : 0) * a.hw + s;
+                    for (int c0 = 0; c0 < NP; c0 += 16) {
+                        uint32_t r[16];
+                        tmem_ld_32x32b_x16(trow + c0, r);
+                        tmem_ld_wait();
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
                             const __nv_bfloat16 hv = __float2bfloat16_rn(fmaxf(fmaf(__uint_as_float(r[i]), step, bias), floor_v));

@@ -281,7 +281,7 @@ void tc_destroy(tc_ctx *ctx)
 
 void tc_force_exact_path(tc_ctx *ctx, int on)
 {
-    if (ctx) ctx->force_exact = on ? 1 : 0;
+    if (ctx) ctx->force_exact = on == 2 ? 2 : (on ? 1 : 0);
 }
 
 int tc_last_path(const tc_ctx *ctx, int decode)
@@ -754,11 +754,11 @@ tc_status tc_encode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
         ctx->last_encode_path = 1;
         return tc_launch_encode_tc(ctx, a, s);
     }
-    if (!ctx->force_exact && x->dtype == TC_BF16 && tc_encode_wide_supported(ctx, a)) {   // wide layers, unaligned rows
+    if (ctx->force_exact != 1 && x->dtype == TC_BF16 && tc_encode_wide_supported(ctx, a)) {   // wide layers, unaligned rows
         ctx->last_encode_path = 3;
         return tc_launch_encode_wide(ctx, a, s);
     }
-    if (!ctx->force_exact && x->dtype == TC_BF16 && x->c % 2 == 0) {      // shapes the tensor-core kernel does not take
+    if (ctx->force_exact != 1 && x->dtype == TC_BF16 && x->c % 2 == 0) {      // shapes the tensor-core kernel does not take
         ctx->last_encode_path = 2;
         return tc_launch_encode_simt_fp32(ctx, a, s);
     }
@@ -795,11 +795,11 @@ tc_status tc_decode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
         ctx->last_decode_path = 1;
         return tc_launch_decode_tc(ctx, a, (cudaStream_t)cuda_stream);
     }
-    if (!ctx->force_exact && x_hat->dtype == TC_BF16 && tc_decode_wide_supported(ctx, a)) {   // wide layers
+    if (ctx->force_exact != 1 && x_hat->dtype == TC_BF16 && tc_decode_wide_supported(ctx, a)) {   // wide layers
         ctx->last_decode_path = 3;
         return tc_launch_decode_wide(ctx, a, (cudaStream_t)cuda_stream);
     }
-    if (!ctx->force_exact && x_hat->dtype == TC_BF16 && x_hat->c % 2 == 0) {  // shapes the tensor-core kernel does not take
+    if (ctx->force_exact != 1 && x_hat->dtype == TC_BF16 && x_hat->c % 2 == 0) {  // shapes the tensor-core kernel does not take
         ctx->last_decode_path = 2;
         return tc_launch_decode_simt_fp32(ctx, a, (cudaStream_t)cuda_stream);
     }

@@ -29,7 +29,7 @@ struct tc_ctx {
     size_t scratch_bytes = 0;
     void *host_arena = nullptr;           // device staging of tc_roundtrip_host (grown on demand)
     size_t host_arena_bytes = 0;
-    int force_exact = 0;                  // route every tensor through the fp64 kernels
+    int force_exact = 0;                  // 1: route every tensor through the fp64 kernels; 2: skip the resident-basis kernels
     int last_encode_path = 0;             // 0 = fp64 kernels, 1 = tensor-core kernels (resident basis), 2 = fp32 kernels, 3 = tensor-core kernels (streamed basis)
     int last_decode_path = 0;
 };
