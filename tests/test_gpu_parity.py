@@ -332,3 +332,22 @@ def test_tensor_core_path_high_rate_tile_overflows_staging(ctx_tc):
     # staging buffer holds, which exercises the direct-to-global packing route
     spec = fm.LayerSpec(256, 14, 14, 0.999, None, 5200)
     run_case(ctx_tc, spec, 8, 6, 3, torch.bfloat16, False, exact=False)
+
+
+# ---- the streaming kernels on shapes the resident-basis kernels would take ----------------------
+
+@pytest.fixture(scope="module")
+def ctx_stream():
+    """Context whose bf16 tensors skip the resident-basis kernels."""
+    c = tc.tc_create(0)
+    tc.tc_force_exact_path(c, 2)
+    yield c
+    c.close()
+
+
+@pytest.mark.parametrize("c,s,n,bits,splits", [(256, 14, 5, 4, 0), (64, 28, 2, 4, 0), (192, 28, 2, 5, 2), (128, 14, 7, 8, 1),
+                                               (256, 14, 3, 6, 4)])
+def test_streaming_kernels_on_narrow_layers(ctx_stream, c, s, n, bits, splits):
+    spec = fm.LayerSpec(c, s, s, 0.9, None, 6400 + c + s)
+    run_case(ctx_stream, spec, bits, 6, n, torch.bfloat16, False, exact=False, pixel_splits=splits,
+             chunk_pixels=1 if splits else 0, routes=(3, 3))
