@@ -659,6 +659,15 @@ bool tc_decode_tc_supported(const tc_ctx *ctx, const DecodeArgs &a)
     return l.slots > 0;
 }
 
+// Bytes of a tile's stream segment this kernel can stage in shared memory (a segment of up to
+// two stream buffers); longer segments are read from global memory, word by word.
+size_t tc_decode_tc_staging_bytes(const tc_ctx *ctx, const DecodeArgs &a)
+{
+    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, a.chunk_pixels,
+                                     a.splits, ctx->max_smem_optin - 512);
+    return l.slots > 0 ? 2u * (size_t)l.stream_buf : 0u;
+}
+
 tc_status tc_launch_decode_tc(const tc_ctx *ctx, const DecodeArgs &a, cudaStream_t s)
 {
     if (a.n_tiles <= 0) return TC_OK;

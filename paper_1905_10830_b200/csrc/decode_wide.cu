@@ -42,12 +42,14 @@ constexpr int kMaxTileChunks = 512;
 // of padding, which keeps both the 16-byte row writes and the 8-byte reads spread over the banks.
 constexpr int kTrRowBytes = 80;
 constexpr int kTrWarpBytes = 32 * kTrRowBytes;
-constexpr int kSegBytes = 16384;                              // staged stream segment of one work item
+constexpr int kSegBytes = 16384;                              // staged stream segment of one work item: at least this,
+constexpr int kSegBytesMax = 32768;                           // up to this where four ring stages still fit
 constexpr int kSegSlack = 32;                                 // the reader's window may look two words past the end
 
 struct SmemLayout {
     uint32_t ring, bop, lut, start, tbuf, seg, total;
     int stages, np;
+    uint32_t seg_bytes;                                       // size of the segment buffer (0: none)
     bool staged;                                              // room for the segment buffer beside at least three stages
 };
 
@@ -57,9 +59,17 @@ __host__ __device__ inline SmemLayout smem_layout(int c, int k, int lut_entries,
     l.np = ((c + 127) / 128 <= 4) ? 128 : 64;
     const uint32_t bop_bytes = 2u * (uint32_t)k * (uint32_t)l.np;
     const uint32_t fixed = bop_bytes + (uint32_t)lut_entries * 4u + (kMaxTileChunks + 8) * 4u + 16u + 8u * kTrWarpBytes;
-    int stages = ((long long)budget - (long long)fixed - (kSegBytes + kSegSlack)) / kStageBytes;
+    l.seg_bytes = kSegBytesMax;
+    int stages = ((long long)budget - (long long)fixed - (kSegBytesMax + kSegSlack)) / kStageBytes;
+    if (stages < 4) {
+        l.seg_bytes = kSegBytes;
+        stages = ((long long)budget - (long long)fixed - (kSegBytes + kSegSlack)) / kStageBytes;
+    }
     l.staged = stages >= 3;
-    if (!l.staged) stages = ((long long)budget - (long long)fixed) / kStageBytes;
+    if (!l.staged) {
+        l.seg_bytes = 0;
+        stages = ((long long)budget - (long long)fixed) / kStageBytes;
+    }
     if (stages > kMaxStages) stages = kMaxStages;
     l.stages = stages < 2 ? 0 : stages;
     l.ring = 0;
@@ -68,7 +78,7 @@ __host__ __device__ inline SmemLayout smem_layout(int c, int k, int lut_entries,
     l.start = l.lut + (uint32_t)lut_entries * 4u;
     l.tbuf = (l.start + (kMaxTileChunks + 8) * 4u + 15u) & ~15u;      // eight warp-private transpose blocks (epilogue)
     l.seg = l.tbuf + 8u * kTrWarpBytes;
-    l.total = l.seg + (l.staged ? (uint32_t)(kSegBytes + kSegSlack) : 0u);
+    l.total = l.seg + (l.staged ? l.seg_bytes + (uint32_t)kSegSlack : 0u);
     return l;
 }
 
@@ -172,7 +182,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a, 
             const unsigned int seg_lo = s_start[ci_first];
             const unsigned int seg_hi = ci_end < chunks_per_tile ? s_start[ci_end] : tile_total;
             const unsigned int byte_lo = (seg_lo >> 3) & ~15u, byte_hi = ((seg_hi + 127u) >> 7) << 4;
-            const bool staged = L.staged && !bad && byte_hi - byte_lo <= (unsigned int)kSegBytes;
+            const bool staged = L.staged && !bad && byte_hi - byte_lo <= L.seg_bytes;
             if (staged) {
                 const unsigned char *src = reinterpret_cast<const unsigned char *>(a.stream) + (base >> 3) + byte_lo;
                 const uint32_t dst = smem_u32(smem + L.seg);
@@ -447,6 +457,13 @@ bool tc_decode_wide_supported(const tc_ctx *ctx, const DecodeArgs &a)
     const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, ctx->max_smem_optin - 2048);
     if (l.stages < 2) return false;
     return a.chunk_pixels <= l.np;                            // a chunk lies inside one work item
+}
+
+// Bytes of a work item's stream segment this kernel can stage in shared memory (0: none).
+size_t tc_decode_wide_staging_bytes(const tc_ctx *ctx, const DecodeArgs &a)
+{
+    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, ctx->max_smem_optin - 2048);
+    return (l.stages >= 2 && l.staged) ? (size_t)l.seg_bytes * (TC_TILE_PIXELS / l.np) : 0u;
 }
 
 tc_status tc_launch_decode_wide(const tc_ctx *ctx, const DecodeArgs &a, cudaStream_t s)

@@ -791,7 +791,20 @@ tc_status tc_decode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
     a.lut32 = cb->d_lut32; a.basis_t_bf16 = m->d_basis_t_bf16; a.dec_bias = m->d_dec_bias; a.center = m->center;
     a.relu = (params && params->relu) ? 1 : 0;
     a.basis_t_map = m->has_basis_t_map ? &m->basis_t_map : nullptr;
-    if (!ctx->force_exact && x_hat->dtype == TC_BF16 && tc_decode_tc_supported(ctx, a)) {
+    bool resident = !ctx->force_exact && x_hat->dtype == TC_BF16 && tc_decode_tc_supported(ctx, a);
+    if (resident && tc_decode_wide_supported(ctx, a)) {
+        // High-rate streams: when the average tile's segment no longer fits the shared-memory
+        // staging of the resident-basis decoder but still fits that of the streaming decoder,
+        // the latter is faster (it would otherwise read the stream from global memory word by word).
+        // (Only when `stream_bytes` is a length: a caller that passes the capacity of a worst-case
+        // buffer says nothing about the rate.)
+        const size_t worst = (size_t)a.n_tiles * TC_TILE_PIXELS * (size_t)a.k * (size_t)cb->max_len / 8;
+        const size_t avg_tile_bytes = (stream_bytes + (size_t)a.n_tiles - 1) / (size_t)a.n_tiles;
+        if (stream_bytes < worst && avg_tile_bytes > tc_decode_tc_staging_bytes(ctx, a) &&
+            avg_tile_bytes <= tc_decode_wide_staging_bytes(ctx, a))
+            resident = false;
+    }
+    if (resident) {
         ctx->last_decode_path = 1;
         return tc_launch_decode_tc(ctx, a, (cudaStream_t)cuda_stream);
     }

@@ -136,6 +136,8 @@ bool tc_encode_wide_supported(const tc_ctx *ctx, const EncodeArgs &a);
 tc_status tc_launch_encode_wide(const tc_ctx *ctx, const EncodeArgs &a, cudaStream_t s);
 bool tc_decode_wide_supported(const tc_ctx *ctx, const DecodeArgs &a);
 tc_status tc_launch_decode_wide(const tc_ctx *ctx, const DecodeArgs &a, cudaStream_t s);
+size_t tc_decode_tc_staging_bytes(const tc_ctx *ctx, const DecodeArgs &a);     // per tile
+size_t tc_decode_wide_staging_bytes(const tc_ctx *ctx, const DecodeArgs &a);   // per tile
 
 tc_status tc_launch_channel_sums(const void *x, int dtype, int n, int c, int hw, double *sums,
                                  cudaStream_t s);

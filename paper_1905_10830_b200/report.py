@@ -96,6 +96,8 @@ def run(cfgs, reps, with_oracle, max_batch):
                 nbytes = enc.total_bits() // 8
                 t_enc = _time(lambda: tc.tc_encode(ctx, model, cb, x, out=enc), reps)
                 t_dec = _time(lambda: tc.tc_decode(ctx, model, cb, enc, x.shape, x.dtype, out=xhat, stream_bytes=nbytes), reps)
+                q_enc = _time_back_to_back(lambda: tc.tc_encode(ctx, model, cb, x, out=enc))
+                q_dec = _time_back_to_back(lambda: tc.tc_decode(ctx, model, cb, enc, x.shape, x.dtype, out=xhat, stream_bytes=nbytes))
                 assert tc.tc_get_status(ctx) == 0
                 side = enc.layout.chunk_len_bytes + enc.layout.tile_off_bytes
                 algo = raw + nbytes + side
@@ -104,7 +106,7 @@ def run(cfgs, reps, with_oracle, max_batch):
                            b=bits, entropy=tst.entropy, huffman=tst.mean_length, stream=8 * nbytes / values,
                            total=8 * (nbytes + side) / values, mse=tst.mse,
                            enc_gbs=raw / t_enc / 1e6, dec_gbs=raw / t_dec / 1e6, rt_gbs=raw / (t_enc + t_dec) / 1e6,
-                           enc_ms=t_enc, dec_ms=t_dec, enc_frac=algo / t_enc / 1e6 / peak, dec_frac=algo / t_dec / 1e6 / peak,
+                           enc_ms=t_enc, dec_ms=t_dec, q_enc_ms=q_enc, q_dec_ms=q_dec, enc_frac=algo / t_enc / 1e6 / peak, dec_frac=algo / t_dec / 1e6 / peak,
                            enc_frac8=algo / t_enc / 1e6 / 8000, dec_frac8=algo / t_dec / 1e6 / 8000,
                            kernels=["fp64", "tcgen05", "fp32", "tcgen05-stream"][tc.tc_last_path(ctx, False)] + "/" + ["fp64", "tcgen05", "fp32", "tcgen05-stream"][tc.tc_last_path(ctx, True)])
                 if with_oracle:
@@ -117,15 +119,29 @@ def run(cfgs, reps, with_oracle, max_batch):
     return rows, peak
 
 
+def _time_back_to_back(fn, calls=20):
+    """Milliseconds per call when `calls` calls are queued one after the other (one event pair
+    around all of them): what a layer costs inside a pipeline that does not wait between layers."""
+    fn()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(calls):
+        fn()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / calls
+
+
 def to_markdown(rows, peak, with_oracle):
-    head = ["cfg", "layer", "N", "dtype", "b", "entropy", "Huffman", "stream+pad", "+offsets", "MSE", "enc ms", "dec ms", "enc GB/s", "dec GB/s",
+    head = ["cfg", "layer", "N", "dtype", "b", "entropy", "Huffman", "stream+pad", "+offsets", "MSE", "enc ms", "dec ms", "enc / dec ms queued x20", "enc GB/s", "dec GB/s",
             "round trip GB/s", f"HBM frac enc/dec (of {peak:.0f} GB/s measured)", "(of 8000 GB/s)", "kernels enc/dec"]
     if with_oracle:
         head += ["stream bit-exact", "coef max rel err", "symbol mismatch", "only at ties", "x_hat bit-equal"]
     out = ["| " + " | ".join(head) + " |", "|" + "---|" * len(head)]
     for r in rows:
         cells = [r["cfg"], r["layer"], r["batch"], r["dtype"], r["b"], f"{r['entropy']:.3f}", f"{r['huffman']:.3f}", f"{r['stream']:.3f}",
-                 f"{r['total']:.3f}", f"{r['mse']:.3g}", f"{r['enc_ms']:.3f}", f"{r['dec_ms']:.3f}", f"{r['enc_gbs']:.1f}", f"{r['dec_gbs']:.1f}",
+                 f"{r['total']:.3f}", f"{r['mse']:.3g}", f"{r['enc_ms']:.3f}", f"{r['dec_ms']:.3f}", f"{r['q_enc_ms']:.3f} / {r['q_dec_ms']:.3f}", f"{r['enc_gbs']:.1f}", f"{r['dec_gbs']:.1f}",
                  f"{r['rt_gbs']:.1f}", f"{r['enc_frac']:.3f} / {r['dec_frac']:.3f}", f"{r['enc_frac8']:.3f} / {r['dec_frac8']:.3f}", r["kernels"]]
         if with_oracle:
             cells += ["yes" if r["stream_exact"] else "NO", f"{r['coef_err']:.1e}", f"{r['mismatch']:.1e}", "yes" if r["ties_only"] else "NO",
