@@ -271,7 +271,7 @@ typedef struct {
  *               word records TC_ERR_BUFFER_TOO_SMALL.  tc_encode_bound() never fails.
  *   chunk_len   DEVICE uint16[n_chunks], 4-byte aligned;  tile_off  DEVICE uint64[n_tiles + 1]
  *               (tile_off[n_tiles] = total stream length in bits).
- * Errors: INVALID_ARG, UNSUPPORTED (C > 1024, K != C with the tensor-core path, dtype /
+ * Errors: INVALID_ARG, UNSUPPORTED (C > 1024, dtype /
  * basis_dtype mismatch), CUDA. */
 tc_status tc_encode(tc_ctx *ctx, const tc_model *model, const tc_codebook *cb,
                     const tc_tensor *x, const tc_encode_params *params, void *stream_out,

@@ -4,7 +4,7 @@
 // also the validation path and the statistics mode.
 //
 // The same kernels have an fp32 mode (kFp32) for bf16 tensors whose shape the tensor-core
-// kernels do not take (more than 256 channels, odd map sizes): bf16 x bf16 products are exact
+// kernels do not take (channel or coefficient counts that are not multiples of 16): bf16 x bf16 products are exact
 // in fp32, accumulation is fp32 with fused multiply-adds, and the quantiser / dequantiser use
 // the same folded constants as the tensor-core kernels (acc / step + bias, step * acc + bias
 // around the centre symbol), so that the two bf16 routes take their decisions alike.
