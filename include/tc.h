@@ -316,10 +316,15 @@ tc_status tc_decode(tc_ctx *ctx, const tc_model *model, const tc_codebook *cb, c
 
 /* Whole chain on HOST tensors (Section 3: encoder, memory, decoder): copies `x_host` (dense
  * NCHW, `dtype`, pinned memory recommended) to the device, encodes, decodes and copies the
- * reconstruction to `x_hat_host`, all on `cuda_stream`, then synchronises it.  The device
- * buffers (tensor, reconstruction, worst-case stream, offsets) live in a context-owned arena
- * that grows with cudaMalloc when a larger tensor arrives.  `stream_bits` (HOST, may be NULL)
- * receives the length of the coded stream.  Returns the first host- or device-side error. */
+ * reconstruction to `x_hat_host`, then synchronises `cuda_stream`.  Larger batches are worked
+ * through in chunks of whole tiles (about 24 MB of images each, at most 64 chunks), two in
+ * flight: the kernels run on `cuda_stream` while the next chunk is copied in and the previous
+ * one is copied out on two streams the context creates at the first call, so that both
+ * directions of the host link are busy at once; the result and the stream length are those of
+ * one pass over the whole tensor.  The device buffers (two slots of tensor, reconstruction,
+ * worst-case stream, lengths and offsets) live in a context-owned arena that grows with
+ * cudaMalloc when a larger chunk arrives.  `stream_bits` (HOST, may be NULL) receives the
+ * length of the coded stream.  Returns the first host- or device-side error. */
 tc_status tc_roundtrip_host(tc_ctx *ctx, const tc_model *model, const tc_codebook *cb,
                             const void *x_host, void *x_hat_host, int32_t n, int32_t c, int32_t h,
                             int32_t w, int32_t dtype, const tc_encode_params *params,

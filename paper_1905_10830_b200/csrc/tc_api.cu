@@ -275,6 +275,14 @@ void tc_destroy(tc_ctx *ctx)
     cudaDeviceSynchronize();
     if (ctx->scratch) cudaFree(ctx->scratch);
     if (ctx->host_arena) cudaFree(ctx->host_arena);
+    if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
+    if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
+    for (int i = 0; i < 2; ++i) {
+        if (ctx->ev_in[i]) cudaEventDestroy(ctx->ev_in[i]);
+        if (ctx->ev_done[i]) cudaEventDestroy(ctx->ev_done[i]);
+        if (ctx->ev_out[i]) cudaEventDestroy(ctx->ev_out[i]);
+    }
+    if (ctx->chunk_bits) cudaFreeHost(ctx->chunk_bits);
     if (ctx->d_status) cudaFree(ctx->d_status);
     delete ctx;
 }
@@ -834,28 +842,83 @@ tc_status tc_roundtrip_host(tc_ctx *ctx, const tc_model *m, const tc_codebook *c
     DeviceGuard guard(ctx->device);
     cudaStream_t s = (cudaStream_t)cuda_stream;
     const size_t elem = dtype == TC_F32 ? 4 : 2;
-    const size_t bytes = (size_t)n * c * h * w * elem;
+    const size_t image_bytes = (size_t)c * h * w * elem;
+    // The batch is cut into chunks of whole tiles (so that the stream is the one a single call
+    // would write) of about 24 MB, and two chunks are in flight: while one is encoded and decoded
+    // on the caller's stream, the next one is copied in and the previous one is copied out on
+    // two streams of the context -- the link to the host carries both directions at once.
+    const int hw = h * w;
+    int unit = 1;                                   // images per chunk must be a multiple of this
+    while (((long long)unit * hw) % TC_TILE_PIXELS != 0) unit <<= 1;      // at most 128
+    long long chunk_n = (long long)((24ull << 20) / image_bytes);
+    chunk_n = std::max<long long>(chunk_n, ((long long)n + kMaxRoundtripChunks - 1) / kMaxRoundtripChunks);
+    chunk_n = std::max<long long>(unit, (chunk_n + unit - 1) / unit * unit);
+    if (chunk_n >= n) chunk_n = n;
+    const int n_chunks = (int)(((long long)n + chunk_n - 1) / chunk_n);
+    if (n_chunks > kMaxRoundtripChunks) return TC_ERR_UNSUPPORTED;
+    if (!ctx->copy_in) {
+        TC_CUDA(cudaStreamCreateWithFlags(&ctx->copy_in, cudaStreamNonBlocking));
+        TC_CUDA(cudaStreamCreateWithFlags(&ctx->copy_out, cudaStreamNonBlocking));
+        for (int i = 0; i < 2; ++i) {
+            TC_CUDA(cudaEventCreateWithFlags(&ctx->ev_in[i], cudaEventDisableTiming));
+            TC_CUDA(cudaEventCreateWithFlags(&ctx->ev_done[i], cudaEventDisableTiming));
+            TC_CUDA(cudaEventCreateWithFlags(&ctx->ev_out[i], cudaEventDisableTiming));
+        }
+        TC_CUDA(cudaMallocHost((void **)&ctx->chunk_bits, sizeof(unsigned long long) * kMaxRoundtripChunks));
+    }
+    tc_tensor xc{nullptr, (int32_t)chunk_n, c, h, w, dtype};
+    xc.data = (void *)x_host;
+    tc_stream_layout clay;
+    if ((st = tc_encode_bound(m, cb, &xc, params, &clay)) != TC_OK) return st;
+    const size_t chunk_bytes = (size_t)chunk_n * image_bytes;
     auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
-    const size_t off_xhat = up(bytes), off_stream = off_xhat + up(bytes), off_chunk = off_stream + up(lay.stream_bytes),
-                 off_tile = off_chunk + up(lay.chunk_len_bytes), total = off_tile + up(lay.tile_off_bytes);
+    const size_t off_xhat = up(chunk_bytes), off_stream = off_xhat + up(chunk_bytes), off_chunk = off_stream + up(clay.stream_bytes),
+                 off_tile = off_chunk + up(clay.chunk_len_bytes), slot_bytes = off_tile + up(clay.tile_off_bytes);
+    const int n_slots = n_chunks > 1 ? 2 : 1;
+    const size_t total = slot_bytes * n_slots;
     if (total > ctx->host_arena_bytes) {
         if (ctx->host_arena) { TC_CUDA(cudaDeviceSynchronize()); cudaFree(ctx->host_arena); ctx->host_arena = nullptr; ctx->host_arena_bytes = 0; }
         TC_CUDA(cudaMalloc(&ctx->host_arena, total));
         ctx->host_arena_bytes = total;
     }
-    char *base = (char *)ctx->host_arena;
-    tc_tensor xd{base, n, c, h, w, dtype}, xh{base + off_xhat, n, c, h, w, dtype};
-    TC_CUDA(cudaMemcpyAsync(xd.data, x_host, bytes, cudaMemcpyHostToDevice, s));
-    st = tc_encode(ctx, m, cb, &xd, params, base + off_stream, lay.stream_bytes, (uint16_t *)(base + off_chunk),
-                   (uint64_t *)(base + off_tile), nullptr, s);
-    if (st != TC_OK) return st;
-    st = tc_decode(ctx, m, cb, base + off_stream, lay.stream_bytes, (const uint16_t *)(base + off_chunk),
-                   (const uint64_t *)(base + off_tile), params, &xh, s);
-    if (st != TC_OK) return st;
-    TC_CUDA(cudaMemcpyAsync(x_hat_host, xh.data, bytes, cudaMemcpyDeviceToHost, s));
-    uint64_t bits = 0;
-    TC_CUDA(cudaMemcpyAsync(&bits, base + off_tile + (size_t)lay.n_tiles * 8, 8, cudaMemcpyDeviceToHost, s));
+    // the copy-in stream starts after whatever the caller queued before this call
+    TC_CUDA(cudaEventRecord(ctx->ev_done[0], s));
+    TC_CUDA(cudaStreamWaitEvent(ctx->copy_in, ctx->ev_done[0], 0));
+    for (int i = 0; i < n_chunks; ++i) {
+        const int slot = i % n_slots;
+        char *base = (char *)ctx->host_arena + slot_bytes * slot;
+        const long long first = (long long)i * chunk_n;
+        const int32_t cn = (int32_t)std::min<long long>(chunk_n, n - first);
+        const size_t cbytes = (size_t)cn * image_bytes;
+        tc_tensor xd{base, cn, c, h, w, dtype}, xh{base + off_xhat, cn, c, h, w, dtype};
+        tc_stream_layout l;
+        if ((st = tc_encode_bound(m, cb, &xd, params, &l)) != TC_OK) return st;
+        // copy in: the slot's tensor was last read by the encode of chunk i - 2
+        if (i >= n_slots) TC_CUDA(cudaStreamWaitEvent(ctx->copy_in, ctx->ev_done[slot], 0));
+        TC_CUDA(cudaMemcpyAsync(xd.data, (const char *)x_host + (size_t)first * image_bytes, cbytes, cudaMemcpyHostToDevice, ctx->copy_in));
+        TC_CUDA(cudaEventRecord(ctx->ev_in[slot], ctx->copy_in));
+        // encode + decode: after the copy, and after chunk i - 2 has left the slot's reconstruction
+        TC_CUDA(cudaStreamWaitEvent(s, ctx->ev_in[slot], 0));
+        if (i >= n_slots) TC_CUDA(cudaStreamWaitEvent(s, ctx->ev_out[slot], 0));
+        st = tc_encode(ctx, m, cb, &xd, params, base + off_stream, clay.stream_bytes, (uint16_t *)(base + off_chunk),
+                       (uint64_t *)(base + off_tile), nullptr, s);
+        if (st != TC_OK) return st;
+        st = tc_decode(ctx, m, cb, base + off_stream, clay.stream_bytes, (const uint16_t *)(base + off_chunk),
+                       (const uint64_t *)(base + off_tile), params, &xh, s);
+        if (st != TC_OK) return st;
+        TC_CUDA(cudaEventRecord(ctx->ev_done[slot], s));
+        // copy out
+        TC_CUDA(cudaStreamWaitEvent(ctx->copy_out, ctx->ev_done[slot], 0));
+        TC_CUDA(cudaMemcpyAsync((char *)x_hat_host + (size_t)first * image_bytes, xh.data, cbytes, cudaMemcpyDeviceToHost, ctx->copy_out));
+        TC_CUDA(cudaMemcpyAsync(&ctx->chunk_bits[i], base + off_tile + (size_t)l.n_tiles * 8, 8, cudaMemcpyDeviceToHost, ctx->copy_out));
+        TC_CUDA(cudaEventRecord(ctx->ev_out[slot], ctx->copy_out));
+    }
+    // the caller's stream ends after the last copy out, as the one-stream version did
+    TC_CUDA(cudaStreamWaitEvent(s, ctx->ev_out[(n_chunks - 1) % n_slots], 0));
+    if (n_slots > 1 && n_chunks > 1) TC_CUDA(cudaStreamWaitEvent(s, ctx->ev_out[(n_chunks - 2) % n_slots], 0));
     TC_CUDA(cudaStreamSynchronize(s));
+    uint64_t bits = 0;
+    for (int i = 0; i < n_chunks; ++i) bits += ctx->chunk_bits[i];
     if (stream_bits) *stream_bits = bits;
     return tc_get_status(ctx, s);
 }

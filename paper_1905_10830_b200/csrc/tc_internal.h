@@ -12,7 +12,8 @@
 
 constexpr int TC_TILE_PIXELS = 128;   // pixels per tile = threads per epilogue group
 constexpr int TC_MAX_C = 1024;
-constexpr int TC_MAX_CODE_LEN = 12;   // longest code the decode lookup table covers
+constexpr int TC_MAX_CODE_LEN = 12;
+constexpr int kMaxRoundtripChunks = 64;   // longest code the decode lookup table covers
 
 // Device status word: first error wins.
 __device__ __forceinline__ void tc_dev_set_status(unsigned int *status, unsigned int code)
@@ -29,6 +30,12 @@ struct tc_ctx {
     size_t scratch_bytes = 0;
     void *host_arena = nullptr;           // device staging of tc_roundtrip_host (grown on demand)
     size_t host_arena_bytes = 0;
+    // tc_roundtrip_host works through the batch in chunks, two in flight: copy-in and copy-out
+    // streams beside the caller's, events that hand a chunk from one to the next, and a small
+    // pinned array for the chunks' stream lengths (created at first use)
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
+    unsigned long long *chunk_bits = nullptr;   // pinned HOST [kMaxRoundtripChunks]
     int force_exact = 0;                  // 1: route every tensor through the fp64 kernels; 2: skip the resident-basis kernels
     int last_encode_path = 0;             // 0 = fp64 kernels, 1 = tensor-core kernels (resident basis), 2 = fp32 kernels, 3 = tensor-core kernels (streamed basis)
     int last_decode_path = 0;

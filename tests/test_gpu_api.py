@@ -230,6 +230,28 @@ def test_roundtrip_host_matches_the_device_path(ctx, dtype):
     m.close(); cb.close()
 
 
+def test_roundtrip_host_in_several_chunks_matches_one_device_pass(ctx):
+    # 150 maps of 64x56x56 bf16 are 60 MB: the call works through them in two chunks of whole
+    # tiles, two in flight; reconstruction and stream length must equal those of one device pass
+    params = fm.layer_params(fm.LayerSpec(64, 56, 56, 0.9, None, 509))
+    cal = fm.make_maps(params, 8, calib=True, dtype=torch.bfloat16, device="cuda")
+    x = fm.make_maps(params, 150, dtype=torch.bfloat16, device="cuda")
+    model = tc.tc_fit_pca(ctx, cal, 4)
+    st = tc.tc_stats(ctx, model, None, cal)
+    cb = tc.tc_build_codebook(ctx, model, st.hist)
+    host_in = x.cpu().pin_memory()
+    host_out = torch.empty_like(host_in).pin_memory()
+    for _ in range(2):                                         # the second call reuses slots, streams and events
+        host_out.zero_()
+        bits = tc.tc_roundtrip_host(ctx, model, cb, host_in, host_out)
+        enc = tc.tc_encode(ctx, model, cb, x)
+        dev = tc.tc_decode(ctx, model, cb, enc, x.shape, torch.bfloat16)
+        assert tc.tc_get_status(ctx) == 0
+        assert bits == enc.total_bits()
+        assert torch.equal(host_out, dev.cpu())
+    model.close(); cb.close()
+
+
 # ---- the same robustness checks on the tensor-core routes (1: basis resident, 3: basis streamed) ----
 
 @pytest.mark.parametrize("c,s,n,route", [(64, 16, 3, 1), (320, 8, 5, 3), (576, 7, 6, 3)])
