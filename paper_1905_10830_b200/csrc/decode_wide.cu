@@ -2,7 +2,8 @@
 // quantiser, inverse transform), where neither the transposed basis nor a double-buffered
 // accumulator for every channel fits on chip.
 //
-// One persistent block per SM walks work items of NP pixels: a whole tile of 128 pixels up to
+// One persistent block per SM walks work items of NP pixels (two at a time, on two VLD groups,
+// up to 256 channels, where the accumulators of two items fit tensor memory): a whole tile of 128 pixels up to
 // 512 channels, half a tile beyond (the accumulators of all channels, NP columns per block of
 // 128 channels, fill tensor memory exactly).  Per item:
 //   warps 0-7     VLD: one thread per chunk walks the bit stream (the item's segment staged in
@@ -28,8 +29,18 @@ using namespace tcdev;
 using namespace sm100;
 
 constexpr int kVldThreads = 256;
-constexpr int kEpiWarp0 = 8, kLoaderWarp0 = 16, kMmaWarp = 20;
-constexpr int kThreads = 21 * 32;
+// Warp roles for G VLD groups (G = 1: wide layers; G = 2: layers of up to 256 channels, where two
+// work items are in flight, each group with its own B operand and accumulator): VLD warps
+// 0 .. 8G-1, eight epilogue warps, loader warps (four; one when only TMA copies are issued), one
+// MMA warp.
+template <int G>
+struct Roles {
+    static constexpr int kEpiWarp0 = 8 * G;
+    static constexpr int kLoaderWarp0 = kEpiWarp0 + 8;
+    static constexpr int kLoaderWarps = G == 2 ? 1 : 4;
+    static constexpr int kMmaWarp = kLoaderWarp0 + kLoaderWarps;
+    static constexpr int kThreads = (kMmaWarp + 1) * 32;
+};
 constexpr int kTmemCols = 512;
 constexpr int kPanelK = 64;                                   // coefficients per ring stage
 constexpr int kStageBytes = 128 * kPanelK * 2;                // 16 KB: 128 channels x 64 coefficients
@@ -47,62 +58,66 @@ constexpr int kSegBytesMax = 32768;                           // up to this wher
 constexpr int kSegSlack = 32;                                 // the reader's window may look two words past the end
 
 struct SmemLayout {
-    uint32_t ring, bop, lut, start, tbuf, seg, total;
+    uint32_t ring, bop, bop_bytes, lut, start, start_bytes, tbuf, seg, seg_stride, total;
     int stages, np;
     uint32_t seg_bytes;                                       // size of the segment buffer (0: none)
     bool staged;                                              // room for the segment buffer beside at least three stages
 };
 
-__host__ __device__ inline SmemLayout smem_layout(int c, int k, int lut_entries, int budget)
+__host__ __device__ inline SmemLayout smem_layout(int c, int k, int lut_entries, int budget, int groups = 1)
 {
     SmemLayout l;
     l.np = ((c + 127) / 128 <= 4) ? 128 : 64;
-    const uint32_t bop_bytes = 2u * (uint32_t)k * (uint32_t)l.np;
-    const uint32_t fixed = bop_bytes + (uint32_t)lut_entries * 4u + (kMaxTileChunks + 8) * 4u + 16u + 8u * kTrWarpBytes;
-    l.seg_bytes = kSegBytesMax;
-    int stages = ((long long)budget - (long long)fixed - (kSegBytesMax + kSegSlack)) / kStageBytes;
-    if (stages < 4) {
-        l.seg_bytes = kSegBytes;
-        stages = ((long long)budget - (long long)fixed - (kSegBytes + kSegSlack)) / kStageBytes;
+    l.bop_bytes = 2u * (uint32_t)k * (uint32_t)l.np;
+    l.start_bytes = (kMaxTileChunks + 8) * 4u;
+    const uint32_t fixed = (uint32_t)groups * (l.bop_bytes + l.start_bytes) + (uint32_t)lut_entries * 4u + 16u + 8u * kTrWarpBytes;
+    // the largest segment buffer (per group) that leaves enough ring stages: 32 KB beside four
+    // stages, else 16 KB or 8 KB beside three (two with two groups)
+    l.seg_bytes = 0;
+    int stages = 0;
+    const int cands[3] = {kSegBytesMax, kSegBytes, kSegBytes / 2};
+    for (int i = 0; i < 3; ++i) {
+        const int st = (int)(((long long)budget - (long long)fixed - (long long)groups * (cands[i] + kSegSlack)) / kStageBytes);
+        const int need = i == 0 ? 4 : (groups == 2 ? 2 : 3);
+        if (st >= need) { l.seg_bytes = (uint32_t)cands[i]; stages = st; break; }
     }
-    l.staged = stages >= 3;
-    if (!l.staged) {
-        l.seg_bytes = 0;
-        stages = ((long long)budget - (long long)fixed) / kStageBytes;
-    }
+    l.staged = l.seg_bytes != 0;
+    if (!l.staged) stages = (int)(((long long)budget - (long long)fixed) / kStageBytes);
     if (stages > kMaxStages) stages = kMaxStages;
     l.stages = stages < 2 ? 0 : stages;
     l.ring = 0;
     l.bop = (uint32_t)(l.stages * kStageBytes);
-    l.lut = l.bop + bop_bytes;
+    l.lut = l.bop + (uint32_t)groups * l.bop_bytes;
     l.start = l.lut + (uint32_t)lut_entries * 4u;
-    l.tbuf = (l.start + (kMaxTileChunks + 8) * 4u + 15u) & ~15u;      // eight warp-private transpose blocks (epilogue)
+    l.tbuf = (l.start + (uint32_t)groups * l.start_bytes + 15u) & ~15u;      // eight warp-private transpose blocks (epilogue)
     l.seg = l.tbuf + 8u * kTrWarpBytes;
-    l.total = l.seg + (l.staged ? l.seg_bytes + (uint32_t)kSegSlack : 0u);
+    l.seg_stride = l.seg_bytes + (uint32_t)kSegSlack;
+    l.total = l.seg + (l.staged ? (uint32_t)groups * l.seg_stride : 0u);
     return l;
 }
 
 // kTma: the panels of the transposed basis arrive by tiled TMA copies (one instruction per stage,
 // 128-byte swizzle) instead of 1024 cp.async copies; `tmap` is then its tensor map.
-template <bool kPerChannel, bool kTma>
-__global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap tmap)
+template <bool kPerChannel, bool kTma, int G>
+__global__ void __launch_bounds__(Roles<G>::kThreads, 1) decode_wide_kernel(DecodeArgs a, const __grid_constant__ CUtensorMap tmap)
 {
+    constexpr int kEpiWarp0 = Roles<G>::kEpiWarp0, kLoaderWarp0 = Roles<G>::kLoaderWarp0, kMmaWarp = Roles<G>::kMmaWarp;
+    constexpr int kThreads = Roles<G>::kThreads;
+    static_assert(G == 1 || kTma, "two groups leave one loader warp: the basis must come by TMA");
     extern __shared__ __align__(128) unsigned char smem_raw[];
     // the swizzled panels want their 1 KB atoms aligned; the ring starts the buffer
     unsigned char *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     __shared__ __align__(8) unsigned long long s_full[kMaxStages], s_empty[kMaxStages];
-    __shared__ __align__(8) unsigned long long s_bfull, s_bfree, s_tfull, s_tempty;
+    __shared__ __align__(8) unsigned long long s_bfull[2], s_bfree[2], s_tfull[2], s_tempty[2];   // per group
     __shared__ uint32_t s_tmem_base;
-    __shared__ unsigned int s_wsum[8];
+    __shared__ unsigned int s_wsum[2][8];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int lut_size = 1 << a.lut_bits;
-    const SmemLayout L = smem_layout(a.c, a.k, kPerChannel ? 0 : lut_size, a.smem_budget);
+    const SmemLayout L = smem_layout(a.c, a.k, kPerChannel ? 0 : lut_size, a.smem_budget, G);
     const int stages = L.stages, NP = L.np;
     const uint32_t ring_addr = smem_u32(smem + L.ring);
-    const uint32_t bop_addr = smem_u32(smem + L.bop);
     uint32_t *s_lut = reinterpret_cast<uint32_t *>(smem + L.lut);
-    unsigned int *s_start = reinterpret_cast<unsigned int *>(smem + L.start);     // start of every chunk of the tile, then the tile's bits
     const int n_cblocks = (a.c + 127) / 128;                  // blocks of 128 channels
     const int n_kpanels = (a.k + kPanelK - 1) / kPanelK;
     const int items_per_tile = TC_TILE_PIXELS / NP;
@@ -112,10 +127,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a, 
     // ---- set-up ---------------------------------------------------------------------
     if (tid == 0) {
         for (int s = 0; s < kMaxStages; ++s) { mbar_init(smem_u32(&s_full[s]), kTma ? 1 : 128); mbar_init(smem_u32(&s_empty[s]), 1); }
-        mbar_init(smem_u32(&s_bfull), kVldThreads);
-        mbar_init(smem_u32(&s_bfree), 1);
-        mbar_init(smem_u32(&s_tfull), 1);
-        mbar_init(smem_u32(&s_tempty), 256);
+        for (int g = 0; g < 2; ++g) {
+            mbar_init(smem_u32(&s_bfull[g]), kVldThreads);
+            mbar_init(smem_u32(&s_bfree[g]), 1);
+            mbar_init(smem_u32(&s_tfull[g]), 1);
+            mbar_init(smem_u32(&s_tempty[g]), 256);
+        }
         mbar_fence_init();
     }
     if (warp == kMmaWarp) { tmem_alloc(smem_u32(&s_tmem_base), kTmemCols); tmem_relinquish(); }
@@ -133,7 +150,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a, 
 
     if (warp < kEpiWarp0) {
         // ================= VLD =================
-        const int t = tid;                                    // 0..255
+        const int grp = warp >> 3, vw = warp & 7;            // group, warp within the group
+        const int t = tid & 255;
+        const uint32_t bop_addr = smem_u32(smem + L.bop) + (uint32_t)grp * L.bop_bytes;
+        unsigned int *s_start = reinterpret_cast<unsigned int *>(smem + L.start + grp * L.start_bytes);   // start of every chunk of the tile
+        unsigned char *seg_ptr = smem + L.seg + grp * L.seg_stride;
+        const int vld_bar = kVldBar + grp;
         const int S = a.splits, cp = a.chunk_pixels;
         const int chunks_per_tile = S * TC_TILE_PIXELS / cp;  // at most 512
         const int k_sub = a.k / S;
@@ -141,7 +163,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a, 
         const int pix_chunks = NP / cp;                       // chunks of one run of coefficients in an item
         const uint32_t row_bytes = (uint32_t)NP * 16u;        // one group of 8 coefficients of all the item's pixels
         bool alive = true;
-        for (long long n = 0; n < my_items && alive; ++n) {
+        for (long long n = grp; n < my_items && alive; n += G) {
+            const long long li = n / G;                       // items this group has taken before
             const long long item = blockIdx.x + n * gridDim.x;
             const long long tile = item / items_per_tile;
             const int h = (int)(item - tile * items_per_tile);
@@ -161,19 +184,19 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a, 
                 if (lane >= d) inc += up;
             }
             // the B operand and the start positions are free once the previous item's MMAs are done
-            if (!mbar_wait(smem_u32(&s_bfree), (uint32_t)((n & 1) ^ 1))) { alive = false; break; }
-            if (lane == 31) s_wsum[warp] = inc;
-            named_bar_sync(kVldBar, kVldThreads);
+            if (!mbar_wait(smem_u32(&s_bfree[grp]), (uint32_t)((li & 1) ^ 1))) { alive = false; break; }
+            if (lane == 31) s_wsum[grp][vw] = inc;
+            named_bar_sync(vld_bar, kVldThreads);
             unsigned int before = 0, tile_total = 0;
 #pragma unroll
             for (int w = 0; w < 8; ++w) {
-                const unsigned int sw = s_wsum[w];
-                if (w < warp) before += sw;
+                const unsigned int sw = s_wsum[grp][w];
+                if (w < vw) before += sw;
                 tile_total += sw;
             }
             const unsigned int excl = before + inc - (l0 + l1);
             if (2 * t < kMaxTileChunks) { s_start[2 * t] = excl; s_start[2 * t + 1] = excl + l0; }
-            named_bar_sync(kVldBar, kVldThreads);
+            named_bar_sync(vld_bar, kVldThreads);
             bool bad = !tile_ok || (unsigned long long)tile_total > end - base;
 
             // the item's part of the tile's segment, staged in shared memory when it fits: the
@@ -185,14 +208,14 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a, 
             const bool staged = L.staged && !bad && byte_hi - byte_lo <= L.seg_bytes;
             if (staged) {
                 const unsigned char *src = reinterpret_cast<const unsigned char *>(a.stream) + (base >> 3) + byte_lo;
-                const uint32_t dst = smem_u32(smem + L.seg);
+                const uint32_t dst = smem_u32(seg_ptr);
                 for (unsigned int i = (unsigned int)t; i < ((byte_hi - byte_lo) >> 4); i += kVldThreads)
                     cp_async_16(dst + i * 16u, src + (size_t)i * 16u, 16u);
             }
             cp_async_commit();
             cp_async_wait<0>();
-            named_bar_sync(kVldBar, kVldThreads);       // every thread's part of the segment has landed
-            const uint32_t *seg_words = reinterpret_cast<const uint32_t *>(smem + L.seg);
+            named_bar_sync(vld_bar, kVldThreads);       // every thread's part of the segment has landed
+            const uint32_t *seg_words = reinterpret_cast<const uint32_t *>(seg_ptr);
 
             auto decode_chunks = [&](auto &r) {
             for (int u = t; u < item_chunks && !bad; u += kVldThreads) {
@@ -250,7 +273,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a, 
             if (bad) tc_dev_set_status(a.status, TC_ERR_CORRUPT_STREAM);
             // the writes become visible to the tensor core's proxy, then the operand is handed over
             fence_proxy_async_smem();
-            mbar_arrive(smem_u32(&s_bfull));
+            mbar_arrive(smem_u32(&s_bfull[grp]));
         }
         if (!alive && t == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
     } else if (warp < kLoaderWarp0) {
@@ -273,13 +296,14 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a, 
             const int n_valid = (int)(left < (long long)NP ? (left < 0 ? 0 : left) : (long long)NP);
             const long long img0 = left > 0 ? p_first / a.hw : 0;
             const int s0 = left > 0 ? (int)(p_first - img0 * a.hw) : 0;
-            if (!mbar_wait(smem_u32(&s_tfull), (uint32_t)(n & 1))) { alive = false; break; }
+            const int grp = (int)(n % G);
+            if (!mbar_wait(smem_u32(&s_tfull[grp]), (uint32_t)((n / G) & 1))) { alive = false; break; }
             tc_fence_after_sync();
             for (int blk = set; blk < n_cblocks; blk += 2) {
                 const int ch = blk * 128 + wq * 32 + lane;
                 const bool ch_ok = ch < a.c;
                 const float bias = ch_ok ? __ldg(a.dec_bias + ch) : 0.f;
-                const uint32_t trow = tmem_base + (uint32_t)(blk * NP) + ((uint32_t)(wq * 32) << 16);
+                const uint32_t trow = tmem_base + (uint32_t)(grp * 256 + blk * NP) + ((uint32_t)(wq * 32) << 16);
                 if (vec) {
                     // 32 pixels at a time: the thread rounds its channel's values and writes them as one
                     // 64-byte row of the warp's block; the warp then reads the block back four rows per
@@ -347,7 +371,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a, 
                 }
             }
             tc_fence_before_sync();
-            mbar_arrive(smem_u32(&s_tempty));
+            mbar_arrive(smem_u32(&s_tempty[grp]));
         }
         if (!alive && lane == 0 && ew == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
     } else if (warp < kMmaWarp) {
@@ -407,8 +431,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a, 
             int it = 0;
             bool alive = true;
             for (long long n = 0; n < my_items && alive; ++n) {
-                if (!mbar_wait(smem_u32(&s_bfull), (uint32_t)(n & 1))) { alive = false; break; }
-                if (!mbar_wait(smem_u32(&s_tempty), (uint32_t)((n & 1) ^ 1))) { alive = false; break; }
+                const int grp = (int)(n % G);
+                const uint32_t par = (uint32_t)((n / G) & 1);
+                const uint32_t bop_addr = smem_u32(smem + L.bop) + (uint32_t)grp * L.bop_bytes;
+                if (!mbar_wait(smem_u32(&s_bfull[grp]), par)) { alive = false; break; }
+                if (!mbar_wait(smem_u32(&s_tempty[grp]), par ^ 1u)) { alive = false; break; }
                 fence_proxy_async_smem();
                 tc_fence_after_sync();
                 for (int jp = 0; jp < n_kpanels && alive; ++jp) {
@@ -422,14 +449,14 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a, 
                         for (int q = 0; q < nk16; ++q) {
                             const uint64_t adesc = kTma ? make_smem_desc_sw128(stage + q * 32, 1024) : make_smem_desc(stage + q * 256, 128, 1024);
                             const uint64_t bdesc = make_smem_desc(bop_addr + (uint32_t)((j0 + 16 * q) >> 3) * b_lbo, b_lbo, 128);
-                            mma_bf16_ss(tmem_base + (uint32_t)(blk * NP), adesc, bdesc, idesc, (jp | q) != 0 ? 1u : 0u);
+                            mma_bf16_ss(tmem_base + (uint32_t)(grp * 256 + blk * NP), adesc, bdesc, idesc, (jp | q) != 0 ? 1u : 0u);
                         }
                         mma_commit(smem_u32(&s_empty[s]));
                     }
                 }
                 if (alive) {
-                    mma_commit(smem_u32(&s_tfull));
-                    mma_commit(smem_u32(&s_bfree));
+                    mma_commit(smem_u32(&s_tfull[grp]));
+                    mma_commit(smem_u32(&s_bfree[grp]));
                 }
             }
             if (!alive) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
@@ -447,6 +474,23 @@ __global__ void __launch_bounds__(kThreads, 1) decode_wide_kernel(DecodeArgs a, 
 
 }  // namespace
 
+// Two VLD groups (two work items in flight, each with its own B operand and accumulator) where
+// the accumulators of two items fit tensor memory, i.e. up to 256 channels, the basis comes by
+// TMA, and shared memory holds both operands beside two ring stages and the segment buffers.
+static int decode_wide_groups(const tc_ctx *ctx, const DecodeArgs &a)
+{
+    if (!a.basis_t_map || a.c > 256) return 1;
+    const SmemLayout l2 = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, ctx->max_smem_optin - 2048, 2);
+    if (!(l2.stages >= 2 && l2.staged)) return 1;
+    // A stream known to be dense (the caller gave its length, not the capacity of a worst-case
+    // buffer, and the average tile exceeds the two-group segment buffers) is better served by one
+    // group with a large segment buffer than by two that read it from global memory.
+    const unsigned long long worst_bits = (unsigned long long)a.n_tiles * TC_TILE_PIXELS * (unsigned long long)a.k * (unsigned long long)a.lut_bits;
+    const unsigned long long avg_tile_bytes = a.stream_bits / 8ull / (unsigned long long)a.n_tiles;
+    if (a.stream_bits < worst_bits && avg_tile_bytes > l2.seg_bytes) return 1;
+    return 2;
+}
+
 bool tc_decode_wide_supported(const tc_ctx *ctx, const DecodeArgs &a)
 {
     if (a.c % 16 != 0 || a.k % 16 != 0 || a.k < 16 || a.k > a.c || a.c > TC_MAX_C) return false;
@@ -454,15 +498,17 @@ bool tc_decode_wide_supported(const tc_ctx *ctx, const DecodeArgs &a)
     if (a.splits > 1 && (a.chunk_pixels != 1 || a.k % a.splits != 0 || (a.k / a.splits) % 8 != 0)) return false;
     if (a.groups != 1 && a.groups != a.k) return false;
     if (a.lut_bits > TC_MAX_CODE_LEN) return false;
-    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, ctx->max_smem_optin - 2048);
+    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, ctx->max_smem_optin - 2048,
+                                     decode_wide_groups(ctx, a));
     if (l.stages < 2) return false;
     return a.chunk_pixels <= l.np;                            // a chunk lies inside one work item
 }
 
-// Bytes of a work item's stream segment this kernel can stage in shared memory (0: none).
+// Bytes of a tile's stream segment this kernel can stage in shared memory (0: none).
 size_t tc_decode_wide_staging_bytes(const tc_ctx *ctx, const DecodeArgs &a)
 {
-    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, ctx->max_smem_optin - 2048);
+    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, ctx->max_smem_optin - 2048,
+                                     decode_wide_groups(ctx, a));
     return (l.stages >= 2 && l.staged) ? (size_t)l.seg_bytes * (TC_TILE_PIXELS / l.np) : 0u;
 }
 
@@ -470,13 +516,16 @@ tc_status tc_launch_decode_wide(const tc_ctx *ctx, const DecodeArgs &a, cudaStre
 {
     if (a.n_tiles <= 0) return TC_OK;
     DecodeArgs args = a;
-    args.smem_budget = ctx->max_smem_optin - 2048;            // leaves room for the static shared variables
-    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, args.smem_budget);
+    args.smem_budget = ctx->max_smem_optin - 2048;            // leaves room for the static shared variables and the alignment
+    const int groups = decode_wide_groups(ctx, a);
+    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, args.smem_budget, groups);
     if (l.stages < 2) return TC_ERR_UNSUPPORTED;
-    const bool tma = a.basis_t_map != nullptr;
+    const bool tma = a.basis_t_map != nullptr, pc = a.groups != 1;
     void (*kernel)(DecodeArgs, const CUtensorMap) =
-        tma ? (a.groups != 1 ? decode_wide_kernel<true, true> : decode_wide_kernel<false, true>)
-            : (a.groups != 1 ? decode_wide_kernel<true, false> : decode_wide_kernel<false, false>);
+        groups == 2 ? (pc ? decode_wide_kernel<true, true, 2> : decode_wide_kernel<false, true, 2>)
+        : tma       ? (pc ? decode_wide_kernel<true, true, 1> : decode_wide_kernel<false, true, 1>)
+                    : (pc ? decode_wide_kernel<true, false, 1> : decode_wide_kernel<false, false, 1>);
+    const int threads = groups == 2 ? Roles<2>::kThreads : Roles<1>::kThreads;
     const size_t smem_bytes = (size_t)l.total + 1024;         // room to align the buffer to 1 KB
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
         return TC_ERR_CUDA;
@@ -485,6 +534,6 @@ tc_status tc_launch_decode_wide(const tc_ctx *ctx, const DecodeArgs &a, cudaStre
     CUtensorMap map_arg;
     if (tma) map_arg = *a.basis_t_map;
     else memset(&map_arg, 0, sizeof(map_arg));
-    kernel<<<grid, kThreads, smem_bytes, s>>>(args, map_arg);
+    kernel<<<grid, threads, smem_bytes, s>>>(args, map_arg);
     return cudaGetLastError() == cudaSuccess ? TC_OK : TC_ERR_CUDA;
 }
