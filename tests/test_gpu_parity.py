@@ -5,7 +5,8 @@ Bars: the entropy-coded stream is bit-exact given identical symbols and decode r
 exactly; projected coefficients agree within 1e-3 * max(|y|, step); at most 1e-4 of the
 symbols differ, only by +-1 and only where the oracle's position (y - lo)/step lies within
 1e-3 of a half-integer; x_hat agrees within max(1e-3 * max(|x_hat|, step), one output ulp)
-and is bit-identical for at least 99.9 % of the values."""
+and is bit-identical for at least 99.9 % of the values (all but one for tensors of fewer than a
+thousand)."""
 import numpy as np
 import pytest
 import torch
@@ -101,7 +102,7 @@ def run_case(ctx, spec, bits, n_cal, n_test, dtype, per_channel, *, exact, chunk
         mant = 7 if dtype == torch.bfloat16 else 23
         ulp = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(want), 1e-30))) - mant)
         assert np.all(np.abs(got - want) <= np.maximum(1e-3 * np.maximum(np.abs(want), m.step), ulp))
-        assert (got == want).mean() >= 0.999
+        assert (got != want).sum() <= np.ceil(1e-3 * got.size)      # (one value, for tensors of fewer than a thousand)
     model_h.close()
     cb.close()
     return o, enc
@@ -375,3 +376,10 @@ def test_high_rate_stream_is_decoded_by_the_streaming_kernel(ctx_tc):
         assert np.all(np.abs(got - want) <= np.maximum(1e-3 * np.maximum(np.abs(want), o["model"].step), ulp))
         assert (got == want).mean() >= 0.999
     model.close(); cb.close()
+
+
+@pytest.mark.parametrize("c,s,n,routes", [(320, 1, 1, (3, 3)), (1024, 2, 1, (3, 3)), (64, 1, 3, (3, 1))])
+def test_single_pixels_and_tiny_maps(ctx_tc, c, s, n, routes):
+    # one to four pixels: a single, mostly empty tile; 1 x 1 maps have unaligned rows
+    spec = fm.LayerSpec(c, s, s, 0.9, None, 6600 + c)
+    run_case(ctx_tc, spec, 4, 40 if c > 512 else 24, n, torch.bfloat16, False, exact=False, routes=routes)
