@@ -15,6 +15,12 @@
  *     library owns only the opaque handles it returns and a small scratch arena per context.
  *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls that
  *     take one are asynchronous on it unless stated otherwise.
+ *   - A context serves one stream at a time: its scratch arena (the cross-tile bookkeeping of
+ *     tc_encode, the buffers of tc_stats and tc_roundtrip_host) and its status word are shared by
+ *     all calls made on it, so two calls on the same context that could overlap on the GPU --
+ *     different streams, no dependency between them -- corrupt each other's output.  Use one
+ *     context per concurrent stream; models and codebooks may be shared between contexts of the
+ *     same device.
  *   - Errors are return codes.  Argument errors are found on the host before any launch.
  *     Conditions only the device can see (corrupt stream, output capacity exceeded at run
  *     time, a bounded wait that ran out) are recorded in a per-context status word and
@@ -48,7 +54,9 @@ typedef enum {
 /* Element types.  TC_INT8 is not a tensor type: it only names the 8-bit basis of a model. */
 typedef enum { TC_F32 = 0, TC_BF16 = 1, TC_INT8 = 2 } tc_dtype;
 
-/* Dense NCHW tensor in DEVICE memory. `data` must be aligned to its element size. */
+/* Dense NCHW tensor in DEVICE memory.  `data` must be aligned to its element size; bf16 tensors
+ * that start on an 8-byte boundary (any allocation does; a view at an odd element offset may
+ * not) and have H*W % 4 == 0 are moved four pixels at a time, others element by element. */
 typedef struct {
     void *data;
     int32_t n, c, h, w;

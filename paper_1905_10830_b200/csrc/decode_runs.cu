@@ -1,0 +1,592 @@
+// Fused tensor-core decode for bf16 tensors with a per-layer code table (Section 3: VLD, inverse
+// quantiser, inverse transform) whose work follows the information in the stream.
+//
+// After the PCA most coefficients of a pixel quantise to one symbol -- the level nearest zero --
+// and the Huffman code gives that symbol the one-bit code 0 (Section 3.1, "Variable length
+// coding"; Appendix E: the tail channels collapse to a single value).  A run of such symbols is
+// a run of zero bits, so a decoder thread counts leading zeros and jumps over the whole run at
+// once; only the other symbols cost a table lookup and a store.  The operand of the inverse
+// projection is therefore filled first with the value of the modal symbol (16-byte stores) and
+// the decoded symbols are then written into it one by one.
+//
+// One persistent block per SM.  Warp roles:
+//   warps 0-7, 8-15    two VLD groups, each with its own operand buffer (all K coefficients of a
+//                      tile of 128 pixels, K-major); where shared memory holds only one buffer
+//                      (C = K = 256) only group 0 works.  One or two threads per pixel walk the
+//                      pixel's chunks.
+//   warps 16-23        epilogue, all eight warps on every tile: TMEM -> registers,
+//                      x_hat = step * acc + bias, round to bf16, NCHW stores through warp-private
+//                      transpose blocks (the accumulator is held transposed: lane = channel)
+//   warp 24            one thread issues the tcgen05.mma of every tile:
+//                      D[c][pixel] = T[j][c] * (Q[pixel][j] - center)
+// The operand is handed over in panels of 32 coefficients: the MMA thread commits a barrier per
+// panel, and a VLD thread of the next tile that shares the buffer waits only for the panel it is
+// about to touch, so that the VLD of tile t + 1 follows the MMAs of tile t panel by panel.  The
+// accumulators are double-buffered in tensor memory, so the epilogue of tile t overlaps both.
+//
+// A tile whose stream is dense (more than kDenseBits128 / 128 bits per symbol) gains nothing
+// from run skipping; its threads then decode symbol by symbol, eight symbols per 16-byte store.
+#include "device_utils.cuh"
+#include "sm100_ptx.cuh"
+
+namespace {
+
+using namespace tcdev;
+using namespace sm100;
+
+constexpr int kGroupWarps = 8, kEpiWarp0 = 16, kMmaWarp = 24;
+constexpr int kThreads = 25 * 32;
+constexpr int kTmemCols = 512;
+constexpr int kAccCols = 256;
+constexpr int kPanelK = 32;                                   // coefficients per hand-over panel
+constexpr int kMaxPanels = 8;                                 // K <= 256
+constexpr int kRunCap = 20;                                   // zero bits skipped per step (20 + 12 <= 32: one refill per step)
+constexpr int kDenseBits128 = 224;                            // tiles above 1.75 bits per symbol are decoded symbol by symbol
+// A chunk that starts inside a staged segment is read for at most (symbols of the chunk) x 12
+// bits, whatever the bits say; the slack after the last buffer keeps those reads inside the
+// block's shared memory even for a corrupt stream (the buffers lie back to back).
+constexpr int kStreamSlack = 1024;
+constexpr int kTrWarpBytes = 1024;                            // epilogue transpose block of one warp: 32 channel rows x 16 pixels
+
+struct SmemLayout {
+    uint32_t basis, lut, vtab, opnd, tbuf, sbuf, total;
+    uint32_t opnd_bytes;                                      // one operand buffer
+    uint32_t stream_buf;                                      // bytes per staged stream buffer (two per group)
+    int nbuf;                                                 // operand buffers = working VLD groups (0: does not fit)
+};
+
+__host__ __device__ inline SmemLayout smem_layout(int c, int k, int lut_entries, int budget)
+{
+    SmemLayout l;
+    l.basis = 0;
+    const int c_pad = ((c + 127) / 128) * 128;                // the MMA takes 128 channels at a time
+    l.lut = (uint32_t)(((size_t)c_pad * k * 2 + 1023) & ~(size_t)1023);
+    l.vtab = l.lut + (uint32_t)lut_entries * 2;               // 16-bit entries: symbol << 8 | length
+    l.opnd = (l.vtab + 512 + 1023) & ~1023u;                  // 256 bf16 values: symbol - center
+    l.opnd_bytes = (uint32_t)k * TC_TILE_PIXELS * 2;
+    l.nbuf = 0;
+    l.stream_buf = 0;
+    l.tbuf = l.sbuf = l.total = 0;
+    for (int nb = 2; nb >= 1 && l.nbuf == 0; --nb) {
+        const uint32_t tbuf = l.opnd + (uint32_t)nb * l.opnd_bytes;
+        const uint32_t sbuf = tbuf + 8u * kTrWarpBytes;
+        for (uint32_t kb = 16; kb >= 4; --kb)
+            if ((long long)sbuf + 2ll * nb * kb * 1024 + kStreamSlack <= (long long)budget) {
+                l.nbuf = nb; l.tbuf = tbuf; l.sbuf = sbuf; l.stream_buf = kb * 1024;
+                l.total = sbuf + 2u * nb * l.stream_buf + kStreamSlack;
+                break;
+            }
+    }
+    return l;
+}
+
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds_u16(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void sts_u16(uint32_t addr, uint32_t v)
+{
+    asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ void sts_v4(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+
+// MSB-first reader with a 64-bit window hi:lo (left-aligned) and one word of look-ahead.  `used`
+// counts, in its low byte, the bits taken since the window was last moved on by a word; table
+// entries (symbol << 8 | length) are added to it and fed to the funnel shifts as they are (the
+// shifts take their amount modulo 32, lengths are at most 12).  refill() moves the window on by
+// one word when 32 bits or more have been taken; a caller that takes at most 32 bits between two
+// refills always sees at least 32 valid bits after one.
+// kShared: the words lie in shared memory (a staged segment, with readable slack behind it);
+// otherwise in global memory, where words at or past `end` read as zero.
+template <bool kShared>
+struct BitReader {
+    uint32_t hi, lo, ahead, used;
+    uint32_t next_addr;               // shared: address of the word after `ahead`
+    const uint32_t *next, *end;       // global
+    uint32_t start_bits;              // position init() was given, modulo 32, and the words fetched since
+    uint32_t words;
+
+    __device__ __forceinline__ uint32_t fetch()
+    {
+        uint32_t w;
+        if constexpr (kShared) { w = lds_u32(next_addr); next_addr += 4; }
+        else { w = next < end ? __ldg(next) : 0u; ++next; }
+        return w;
+    }
+    // kShared: `base_addr` is the shared address of the segment; else `base` / `end_word` delimit it
+    __device__ __forceinline__ void init(uint32_t base_addr, const uint32_t *base, const uint32_t *end_word, uint32_t bitpos)
+    {
+        if constexpr (kShared) next_addr = base_addr + (bitpos >> 5) * 4u;
+        else { next = base + (bitpos >> 5); end = end_word; }
+        const uint32_t w0 = fetch(), w1 = fetch();
+        ahead = fetch();
+        const uint32_t sh = bitpos & 31u;
+        hi = __funnelshift_l(w1, w0, sh);
+        lo = w1 << sh;
+        used = sh;
+        start_bits = sh;
+        words = 0;
+    }
+    __device__ __forceinline__ void idle()
+    {
+        hi = lo = ahead = used = start_bits = words = 0;
+        next_addr = 0; next = end = nullptr;
+    }
+    __device__ __forceinline__ void take(uint32_t entry)      // entry & 31 bits
+    {
+        hi = __funnelshift_l(lo, hi, entry);
+        lo = __funnelshift_l(0u, lo, entry);
+        used += entry;
+    }
+    __device__ __forceinline__ void refill()
+    {
+        if (used & 32u) {
+            // c = used - 32 bits of the new word's position are already consumed: the window gains
+            // `ahead` behind its 64 - used valid bits
+            hi |= __funnelshift_l(ahead, 0u, used);           // ahead >> (32 - c), zero when c == 0
+            lo |= __funnelshift_l(0u, ahead, used);           // ahead << c
+            used -= 32u;
+            ahead = fetch();
+            ++words;
+        }
+    }
+    __device__ __forceinline__ uint32_t consumed() const { return words * 32u + (used & 0xffu) - start_bits; }
+};
+
+template <bool kRelu>
+__global__ void __launch_bounds__(kThreads, 1) decode_runs_kernel(DecodeArgs a)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ __align__(8) unsigned long long s_full[2], s_empty[2][kMaxPanels], s_tfull[2], s_tempty[2];
+    __shared__ uint32_t s_tmem_base;
+    __shared__ unsigned int s_wsum[2][2][4];   // [group][thread set][warp]: bits per warp, for the start positions
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int lut_size = 1 << a.lut_bits;
+    const SmemLayout L = smem_layout(a.c, a.k, lut_size, a.smem_budget);
+    const int nbuf = L.nbuf;
+    const uint32_t basis_addr = smem_u32(smem + L.basis);
+    const uint32_t lut_addr = smem_u32(smem + L.lut);
+    const uint32_t vtab_addr = smem_u32(smem + L.vtab);
+    const uint32_t opnd_addr = smem_u32(smem + L.opnd);
+    const int n_panels = (a.k + kPanelK - 1) / kPanelK;
+    const int S = a.splits, cp = a.chunk_pixels;
+    const int tpp = S >= 2 ? 2 : 1;                            // threads per pixel
+    const int chunks_per_thread = S / tpp;                     // 1, or 2 with four chunks per pixel
+    const int n_work = cp > 1 ? TC_TILE_PIXELS / cp : TC_TILE_PIXELS * tpp;   // threads of a group that own chunks
+    const int n_thr = ((n_work + 31) / 32) * 32;               // whole warps take part in the group's barriers
+
+    // ---- set-up ---------------------------------------------------------------------
+    if (tid == 0) {
+        for (int g = 0; g < 2; ++g) {
+            mbar_init(smem_u32(&s_full[g]), (uint32_t)n_thr);
+            for (int p = 0; p < kMaxPanels; ++p) mbar_init(smem_u32(&s_empty[g][p]), 1);
+            mbar_init(smem_u32(&s_tfull[g]), 1);
+            mbar_init(smem_u32(&s_tempty[g]), 256);
+        }
+        mbar_fence_init();
+    }
+    if (warp == kMmaWarp) { tmem_alloc(smem_u32(&s_tmem_base), kTmemCols); tmem_relinquish(); }
+    {
+        // transposed basis [c][j] -> K-major core matrices: (c/8)*sbo + (j/8)*128 + (c%8)*16 + (j%8)*2
+        const uint32_t sbo = (uint32_t)(a.k / 8) * 128u;
+        const int chunks_per_row = a.k / 8;
+        const uint4 *src = reinterpret_cast<const uint4 *>(a.basis_t_bf16);
+        const int c_pad = ((a.c + 127) / 128) * 128;         // rows past C are zero: their outputs are never stored
+        for (int i = tid; i < c_pad * chunks_per_row; i += kThreads) {
+            const int ch = i / chunks_per_row, j8 = i - ch * chunks_per_row;
+            cp_async_16(basis_addr + (ch >> 3) * sbo + j8 * 128 + (ch & 7) * 16, ch < a.c ? src + i : src, ch < a.c ? 16u : 0u);
+        }
+        cp_async_commit();
+        unsigned short *s_lut = reinterpret_cast<unsigned short *>(smem + L.lut);
+        for (int i = tid; i < lut_size; i += kThreads) s_lut[i] = a.lut[i];
+        unsigned short *s_vtab = reinterpret_cast<unsigned short *>(smem + L.vtab);
+        for (int i = tid; i < 256; i += kThreads) s_vtab[i] = (unsigned short)(__float_as_uint((float)(i - a.center)) >> 16);
+    }
+    cp_async_wait<0>();
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = s_tmem_base;
+
+    const long long my_tiles = (a.n_tiles > blockIdx.x) ? (a.n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+
+    if (warp < 2 * kGroupWarps) {
+        // ================= VLD groups =================
+        const int grp = warp >> 3;
+        const int tg = tid & 255;                // thread within the group
+        if (grp < nbuf && tg < n_thr) {
+            const int set = cp > 1 ? 0 : tg >> 7;    // which thread of the pixel (warp-uniform)
+            const int t = cp > 1 ? tg : (tg & 127);  // pixel within the tile, or chunk within the tile (cp > 1)
+            const int wq = (t >> 5) & 3;
+            const bool owner = tg < n_work;          // this thread has chunks to decode
+            const int k_sub = a.k / S;               // coefficients per chunk of one pixel
+            const int k_first = set * chunks_per_thread * k_sub;           // this thread's coefficients of a pixel
+            const int k_last = cp > 1 ? a.k : k_first + chunks_per_thread * k_sub;
+            const int p_first = k_first / kPanelK, p_last = (k_last + kPanelK - 1) / kPanelK;     // panels it touches
+            const int chunks_per_tile = S * TC_TILE_PIXELS / cp;
+            const uint32_t opnd_g = opnd_addr + (uint32_t)grp * L.opnd_bytes;
+            const uint32_t sbuf_bytes = L.stream_buf;
+            const uint32_t sbuf_g = smem_u32(smem + L.sbuf) + (uint32_t)grp * 2u * sbuf_bytes;
+            const int bar_id = 1 + grp;
+            const int lb = a.lut_bits;
+            const uint32_t modal2 = lds_u16(vtab_addr + (uint32_t)(a.modal < 0 ? a.center : a.modal) * 2u) * 0x00010001u;
+            bool alive = true;
+
+            // offsets of a tile, validated; a tile that cannot be valid decodes nothing.  `lens`
+            // holds the chunk lengths of this thread's pixel (up to four), or of its chunk.
+            struct TileInfo { unsigned long long base, bits; bool ok, staged; unsigned int l01, l23; };
+            auto tile_info = [&](long long tl) {
+                TileInfo ti{0, 0, false, false, 0, 0};
+                if (tl >= my_tiles) return ti;
+                const long long tile = blockIdx.x + tl * gridDim.x;
+                const unsigned long long base = a.tile_off[tile], end = a.tile_off[tile + 1];
+                ti.ok = (base & 127ull) == 0 && (end & 127ull) == 0 && base <= end && end <= a.stream_bits;
+                if (!ti.ok) return ti;
+                ti.base = base;
+                ti.bits = end - base;
+                ti.staged = ti.bits <= (unsigned long long)sbuf_bytes * 8ull &&
+                            (cp * (k_last - k_first) * TC_MAX_CODE_LEN) / 8 + 16 <= kStreamSlack;
+                if (owner) {
+                    const long long ch = tile * chunks_per_tile + (long long)t * (cp > 1 ? 1 : S);
+                    if (cp > 1 || S == 1) { if (ch < a.n_chunks) ti.l01 = a.chunk_len[ch]; }
+                    else if (ch < a.n_chunks) {      // S chunks of one pixel: an aligned word holds two lengths
+                        ti.l01 = *reinterpret_cast<const unsigned int *>(a.chunk_len + ch);
+                        if (S == 4) ti.l23 = *reinterpret_cast<const unsigned int *>(a.chunk_len + ch + 2);
+                    }
+                }
+                return ti;
+            };
+            // start the copy of a tile's segment into stream buffer `which` (16 bytes per cp.async)
+            auto stage_tile = [&](const TileInfo &ti, int which) {
+                if (ti.ok && ti.staged) {
+                    const uint32_t dst = sbuf_g + (uint32_t)which * sbuf_bytes;
+                    const unsigned char *src = reinterpret_cast<const unsigned char *>(a.stream) + (ti.base >> 3);
+                    const uint32_t n16 = (uint32_t)(ti.bits >> 7);
+                    for (uint32_t i = tg; i < n16; i += n_thr) cp_async_16(dst + i * 16u, src + (size_t)i * 16u, 16u);
+                }
+                cp_async_commit();
+            };
+
+            TileInfo cur = tile_info(grp), nxt = tile_info(grp + nbuf);
+            stage_tile(cur, 0);
+            int li = 0;
+            for (long long tl = grp; tl < my_tiles && alive; tl += nbuf, ++li) {
+                const long long tile = blockIdx.x + tl * gridDim.x;
+                // start of every chunk = sum of the lengths before it in the tile (chunk order: pixel,
+                // then part of the pixel): scan over the pixels' totals
+                const unsigned int len0 = cur.l01 & 0xffffu, len1 = cur.l01 >> 16, len2 = cur.l23 & 0xffffu, len3 = cur.l23 >> 16;
+                const unsigned int tot = len0 + len1 + len2 + len3;
+                unsigned int inc = tot;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const unsigned int up = __shfl_up_sync(0xffffffffu, inc, d);
+                    if (lane >= d) inc += up;
+                }
+                if (lane == 31) s_wsum[grp][set][wq] = inc;
+                cp_async_wait<0>();
+                // every thread's part of this tile's segment has landed, and every thread is done
+                // with the tile before: its stream buffer may take the next tile's segment
+                named_bar_sync(bar_id, n_thr);
+                stage_tile(nxt, (li + 1) & 1);
+                const TileInfo after = tile_info(tl + 2 * nbuf);   // offsets two tiles ahead: their latency hides behind the decode
+                unsigned int before = 0, tile_total = 0;
+                const int n_wq = (n_work / tpp + 31) / 32;          // warps of one thread set
+#pragma unroll
+                for (int w = 0; w < 4; ++w) {
+                    const unsigned int sw = w < n_wq ? s_wsum[grp][set][w] : 0u;
+                    if (w < wq) before += sw;
+                    tile_total += sw;
+                }
+                // this thread's first chunk: after the pixels before it and the chunks of the pixel before its own
+                unsigned int chunk_start = before + inc - tot;
+                unsigned int my_len[2] = {len0, len1};
+                if (cp == 1 && set == 1) {
+                    if (S == 2) { chunk_start += len0; my_len[0] = len1; }
+                    else { chunk_start += len0 + len1; my_len[0] = len2; my_len[1] = len3; }
+                }
+
+                const long long ch = tile * chunks_per_tile + (long long)t * (cp > 1 ? 1 : S);
+                bool active = cur.ok && owner && ch < a.n_chunks;
+                bool bad = !cur.ok || (unsigned long long)tile_total > cur.bits;
+                if (bad) active = false;
+                const long long px0 = tile * TC_TILE_PIXELS + (long long)t * cp;
+                const int n_pix = active ? (int)min((long long)cp, a.pixels - px0) : 0;
+                const uint32_t seg_addr = sbuf_g + (uint32_t)(li & 1) * sbuf_bytes;
+                // dense tiles are decoded symbol by symbol
+                const bool runs = a.modal >= 0 &&
+                                  cur.bits * 128ull <= (unsigned long long)kDenseBits128 * (unsigned long long)a.k * TC_TILE_PIXELS;
+                const uint32_t wait_parity = (uint32_t)((li & 1) ^ 1);   // the buffer's hand-back by the tile before this one
+
+                // walks this thread's chunks; kSh: the segment is staged in shared memory
+                auto decode_tile = [&](auto &r) {
+                    uint32_t expect = 0;               // bits the chunks decoded so far should have taken
+                    for (int pp = 0; pp < cp && alive; ++pp) {
+                        const bool decode = pp < n_pix;
+                        const uint32_t row = (uint32_t)(t * cp + pp);
+                        const uint32_t row_addr = opnd_g + (row >> 3) * 128u + (row & 7u) * 16u;
+                        int ready = p_first;           // panels [p_first, ready) of this row are handed back and filled
+                        // waits for panel p to be handed back by the MMAs of the tile before, then fills this
+                        // thread's coefficients of it with the modal symbol (run mode)
+                        auto prepare = [&](int p) {
+                            if (pp == 0 && !mbar_wait(smem_u32(&s_empty[grp][p]), wait_parity, 200u)) { alive = false; return; }
+                            if (runs && owner) {
+                                const int g0 = max(p * (kPanelK / 8), k_first >> 3), g1 = min((p + 1) * (kPanelK / 8), k_last >> 3);
+                                for (int g = g0; g < g1; ++g) sts_v4(row_addr + (uint32_t)g * 2048u, modal2, modal2, modal2, modal2);
+                            }
+                        };
+                        for (int ci = 0; ci < (cp > 1 ? 1 : chunks_per_thread) && alive; ++ci) {
+                            const int kf = cp > 1 ? 0 : k_first + ci * k_sub, ke = cp > 1 ? a.k : kf + k_sub;
+                            if (runs) {
+                                int pos = kf;
+                                while (pos < ke && alive) {
+                                    uint32_t v = 0;
+                                    if (decode) {
+                                        r.refill();
+                                        const uint32_t n = min((uint32_t)__clz((int)(r.hi | 0x800u)), (uint32_t)(ke - pos));   // <= kRunCap
+                                        r.take(n);
+                                        pos += (int)n;
+                                        if (pos >= ke) break;
+                                        const uint32_t e = lds_u16(lut_addr + (r.hi >> (32 - lb)) * 2u);
+                                        r.take(e);
+                                        v = lds_u16(vtab_addr + (e >> 8) * 2u);
+                                    } else {
+                                        pos = ke - 1;      // nothing to decode: only hand the panels on
+                                    }
+                                    while (ready * kPanelK <= pos && alive) prepare(ready++);
+                                    if (decode && alive) sts_u16(row_addr + ((uint32_t)pos >> 3) * 2048u + ((uint32_t)pos & 7u) * 2u, v);
+                                    ++pos;
+                                }
+                            } else {
+                                for (int k0 = kf; k0 < ke && alive; k0 += 8) {
+                                    while (ready * kPanelK <= k0 && alive) prepare(ready++);
+                                    uint32_t pk[4] = {0u, 0u, 0u, 0u};
+                                    if (decode) {
+#pragma unroll
+                                        for (int i = 0; i < 4; ++i) {
+                                            r.refill();
+                                            const uint32_t e0 = lds_u16(lut_addr + (r.hi >> (32 - lb)) * 2u);
+                                            r.take(e0);
+                                            const uint32_t e1 = lds_u16(lut_addr + (r.hi >> (32 - lb)) * 2u);
+                                            r.take(e1);
+                                            pk[i] = lds_u16(vtab_addr + (e0 >> 8) * 2u) | (lds_u16(vtab_addr + (e1 >> 8) * 2u) << 16);
+                                        }
+                                    }
+                                    if (alive) sts_v4(row_addr + (uint32_t)(k0 >> 3) * 2048u, pk[0], pk[1], pk[2], pk[3]);
+                                }
+                            }
+                            // a chunk of one pixel (or part of it) must end exactly where its length says
+                            if (cp == 1) {
+                                expect += my_len[ci];
+                                if (active && r.consumed() != expect) bad = true;
+                            }
+                        }
+                        while (ready < p_last && alive) prepare(ready++);
+                    }
+                    if (cp > 1 && active && r.consumed() != len0) bad = true;
+                };
+                if (cur.ok && cur.staged) {
+                    BitReader<true> r;
+                    if (active) r.init(seg_addr, nullptr, nullptr, chunk_start);
+                    else r.idle();
+                    decode_tile(r);
+                } else {
+                    BitReader<false> r;
+                    if (active) {
+                        const uint32_t *seg = a.stream + (cur.base >> 5);
+                        r.init(0u, seg, seg + (cur.bits >> 5), chunk_start);
+                    } else r.idle();
+                    decode_tile(r);
+                }
+                // (the issuing thread makes the operand visible to the tensor core's proxy)
+                if (alive) mbar_arrive(smem_u32(&s_full[grp]));
+                if (bad) tc_dev_set_status(a.status, TC_ERR_CORRUPT_STREAM);
+                cur = nxt;
+                nxt = after;
+            }
+            cp_async_wait<0>();
+            if (!alive && tg == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
+        }
+    } else if (warp < kMmaWarp) {
+        // ================= epilogue: all eight warps work on every tile =================
+        // A thread owns one channel (its TMEM lane) of one block of 128 channels.  With two
+        // channel blocks warps 16-19 take the first and warps 20-23 the second; with one block
+        // the two warp sets split the tile's pixels (TMEM columns) in halves.
+        const int set = (warp - kEpiWarp0) >> 2;
+        const int wq = warp & 3;                            // TMEM lane quarter of this warp
+        const int n_blocks = (a.c + 127) / 128;
+        const int blk = n_blocks == 2 ? set : 0;
+        const int col_first = n_blocks == 2 ? 0 : 64 * set, col_count = n_blocks == 2 ? 128 : 64;
+        const int ch = blk * 128 + wq * 32 + lane;
+        const bool ch_ok = ch < a.c;
+        const float step = (float)(a.step * a.basis_scale);        // the operand holds basis / basis_scale
+        const float bias = ch_ok ? a.dec_bias[ch] : 0.f;
+        __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(a.xhat);
+        // With H*W a multiple of 4 every aligned group of four pixels lies inside one image and is
+        // 8-byte aligned (given an 8-byte aligned tensor); otherwise pixels are stored one by one.
+        const bool vec = (a.hw & 3) == 0 && ((uintptr_t)a.xhat & 7u) == 0;
+        const long long img_stride = (long long)a.c * a.hw;
+        const int ch_base = blk * 128 + wq * 32;            // first channel of this warp
+        // transpose block: row = channel (32 bytes = 16 pixels); the two 16-byte halves of a row are
+        // swapped in rows 4-7, 12-15, ... so that neither the row writes nor the reads below collide
+        const uint32_t tb = smem_u32(smem + L.tbuf) + (uint32_t)(warp - kEpiWarp0) * kTrWarpBytes;
+        const uint32_t sw_wr = (uint32_t)((lane >> 2) & 1);
+        const uint32_t tb_wr = tb + (uint32_t)lane * 32u;
+        const int r_sub = lane >> 2, piece = lane & 3;      // read phase: channel row r_sub (+ 8, 16, 24), pixels 4 * piece ...
+        const uint32_t tb_rd = tb + (uint32_t)r_sub * 32u + ((((uint32_t)piece >> 1) ^ ((uint32_t)(r_sub >> 2) & 1u)) << 4) + ((uint32_t)piece & 1u) * 8u;
+        auto convert = [&](uint32_t x0, uint32_t x1) {
+            float f0 = fmaf(__uint_as_float(x0), step, bias), f1 = fmaf(__uint_as_float(x1), step, bias);
+            if constexpr (kRelu) { f0 = fmaxf(f0, 0.f); f1 = fmaxf(f1, 0.f); }   // the layer's non-linearity, when it follows the decoder
+            const __nv_bfloat162 h = __floats2bfloat162_rn(f0, f1);
+            return *reinterpret_cast<const uint32_t *>(&h);
+        };
+        bool alive = true;
+        for (long long tl = 0; tl < my_tiles && alive; ++tl) {
+            const int acc = (int)(tl & 1);
+            const long long tile = blockIdx.x + tl * gridDim.x;
+            const long long p_first = tile * TC_TILE_PIXELS + col_first;
+            const long long left = a.pixels - p_first;                       // pixels from this thread's first column on
+            const int n_valid = (int)(left < (long long)col_count ? (left < 0 ? 0 : left) : (long long)col_count);
+            if (!mbar_wait(smem_u32(&s_tfull[acc]), (uint32_t)((tl >> 1) & 1), 1000u)) { alive = false; break; }
+            tc_fence_after_sync();
+            const uint32_t trow = tmem_base + acc * kAccCols + blk * 128 + ((uint32_t)(wq * 32) << 16) + col_first;
+            if (vec) {
+                // position of this lane's pixel group (4 pixels) in the first pass
+                const long long pg = p_first + 4 * piece;
+                long long img = pg < a.pixels ? pg / a.hw : 0;
+                int sp = pg < a.pixels ? (int)(pg - img * a.hw) : 0;
+                for (int c0 = 0; c0 < col_count; c0 += 16) {
+                    uint32_t r[16];
+                    tmem_ld_32x32b_x16(trow + c0, r);
+                    tmem_ld_wait();
+                    sts_v4(tb_wr + (sw_wr << 4), convert(r[0], r[1]), convert(r[2], r[3]), convert(r[4], r[5]), convert(r[6], r[7]));
+                    sts_v4(tb_wr + ((sw_wr ^ 1u) << 4), convert(r[8], r[9]), convert(r[10], r[11]), convert(r[12], r[13]), convert(r[14], r[15]));
+                    __syncwarp();
+                    const bool px_ok = c0 + 4 * piece < n_valid;
+                    __nv_bfloat16 *row_ptr = out + img * img_stride + (long long)(ch_base + r_sub) * a.hw + sp;
+#pragma unroll
+                    for (int it = 0; it < 4; ++it) {
+                        uint32_t lo2, hi2;
+                        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(lo2), "=r"(hi2) : "r"(tb_rd + it * 256));
+                        if (px_ok && ch_base + 8 * it + r_sub < a.c)
+                            *reinterpret_cast<uint2 *>(row_ptr + (long long)(8 * it) * a.hw) = make_uint2(lo2, hi2);
+                    }
+                    sp += 16;
+                    while (sp >= a.hw) { sp -= a.hw; ++img; }
+                    __syncwarp();                                   // the block may be overwritten
+                }
+            } else {
+                // position of the first pixel; from there on it moves incrementally
+                const long long img0 = left > 0 ? p_first / a.hw : 0;
+                int s = left > 0 ? (int)(p_first - img0 * a.hw) : 0;
+                __nv_bfloat16 *dst = out + img0 * img_stride + (long long)(ch_ok ? ch : 0) * a.hw + s;
+                for (int c0 = 0; c0 < col_count; c0 += 16) {
+                    uint32_t r[16];
+                    tmem_ld_32x32b_x16(trow + c0, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        float f = fmaf(__uint_as_float(r[i]), step, bias);
+                        if constexpr (kRelu) f = fmaxf(f, 0.f);
+                        if (ch_ok && c0 + i < n_valid) *dst = __float2bfloat16_rn(f);
+                        s += 1;
+                        const bool wrap = s == a.hw;            // the next pixel starts the next image
+                        dst += wrap ? 1 + img_stride - a.hw : 1;
+                        s = wrap ? 0 : s;
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            mbar_arrive(smem_u32(&s_tempty[acc]));
+        }
+        if (!alive && lane == 0 && wq == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
+    } else {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            // A = transposed basis (128 channels per instruction), B = the decoded symbols of 128 pixels
+            const uint32_t idesc = make_idesc_bf16(128, TC_TILE_PIXELS, /*A K-major*/ false, /*B K-major*/ false);
+            const uint32_t a_sbo = (uint32_t)(a.k / 8) * 128u;
+            const int n_blocks = (a.c + 127) / 128;
+            bool alive = true;
+            for (long long tl = 0; tl < my_tiles && alive; ++tl) {
+                const int acc = (int)(tl & 1);
+                const int buf = nbuf == 2 ? (int)(tl & 1) : 0;
+                const long long use = nbuf == 2 ? (tl >> 1) : tl;     // how often the buffer was filled before
+                if (!mbar_wait(smem_u32(&s_tempty[acc]), (uint32_t)(((tl >> 1) & 1) ^ 1), 500u)) { alive = false; break; }
+                if (!mbar_wait(smem_u32(&s_full[buf]), (uint32_t)(use & 1), 200u)) { alive = false; break; }
+                // the operand was written with ordinary stores by threads that have arrived on the
+                // barrier: one proxy fence here, between that synchronisation and the MMA's
+                // operand reads, orders them for all writers
+                fence_proxy_async_smem();
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + acc * kAccCols;
+                const uint32_t opnd_b = opnd_addr + (uint32_t)buf * L.opnd_bytes;
+                uint32_t accumulate = 0;
+                for (int p = 0; p < n_panels; ++p) {
+                    const int k0 = p * kPanelK;
+                    const int nk16 = min(kPanelK, a.k - k0) >> 4;
+                    for (int q = 0; q < nk16; ++q) {
+                        const uint64_t bdesc = make_smem_desc(opnd_b + (uint32_t)((k0 + 16 * q) >> 3) * 2048u, 2048, 128);
+                        for (int blk = 0; blk < n_blocks; ++blk) {
+                            const uint64_t adesc = make_smem_desc(basis_addr + blk * 16 * a_sbo + ((k0 + 16 * q) >> 3) * 128, 128, a_sbo);
+                            mma_bf16_ss(d_tmem + blk * 128, adesc, bdesc, idesc, accumulate);
+                        }
+                        accumulate = 1u;
+                    }
+                    mma_commit(smem_u32(&s_empty[buf][p]));      // the panel goes back to the VLD threads
+                }
+                mma_commit(smem_u32(&s_tfull[acc]));
+            }
+            if (!alive) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
+        }
+    }
+
+    // ---- teardown ---------------------------------------------------------------------
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == kMmaWarp) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+}  // namespace
+
+bool tc_decode_runs_supported(const tc_ctx *ctx, const DecodeArgs &a)
+{
+    // K <= C leading components (PCA truncation): K is the reduction dimension of the MMA
+    if (a.c % 16 != 0 || a.k % 16 != 0 || a.k < 16 || a.k > a.c || a.c > 256) return false;
+    if (a.groups != 1) return false;                           // per-channel tables do not fit shared memory
+    if (a.lut_bits > TC_MAX_CODE_LEN) return false;
+    if (a.chunk_pixels > 1 ? a.splits != 1 : (a.splits != 1 && a.splits != 2 && a.splits != 4)) return false;
+    if (a.splits > 1 && (a.k % a.splits != 0 || (a.k / a.splits) % 8 != 0)) return false;
+    const SmemLayout l = smem_layout(a.c, a.k, 1 << a.lut_bits, ctx->max_smem_optin - 512);
+    return l.nbuf > 0;
+}
+
+tc_status tc_launch_decode_runs(const tc_ctx *ctx, const DecodeArgs &a, cudaStream_t s)
+{
+    if (a.n_tiles <= 0) return TC_OK;
+    const SmemLayout l = smem_layout(a.c, a.k, 1 << a.lut_bits, ctx->max_smem_optin - 512);
+    if (l.nbuf == 0) return TC_ERR_UNSUPPORTED;
+    void (*kernel)(DecodeArgs) = a.relu ? decode_runs_kernel<true> : decode_runs_kernel<false>;
+    DecodeArgs args = a;
+    args.smem_budget = ctx->max_smem_optin - 512;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.total) != cudaSuccess)
+        return TC_ERR_CUDA;
+    const unsigned int grid = (unsigned int)((a.n_tiles < ctx->sm_count) ? a.n_tiles : ctx->sm_count);
+    kernel<<<grid, kThreads, l.total, s>>>(args);
+    return cudaGetLastError() == cudaSuccess ? TC_OK : TC_ERR_CUDA;
+}

@@ -503,8 +503,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
         const float floor_v = a.relu ? 0.f : __int_as_float((int)0xff800000u);        // the layer's non-linearity, when it follows the decoder
         __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(a.xhat);
         // With H*W a multiple of 4 every aligned group of four pixels lies inside one image and is
-        // 8-byte aligned; otherwise pixels are stored one by one.
-        const bool vec = (a.hw & 3) == 0;
+        // 8-byte aligned (given an 8-byte aligned tensor); otherwise pixels are stored one by one.
+        const bool vec = (a.hw & 3) == 0 && ((uintptr_t)a.xhat & 7u) == 0;
         const long long img_stride = (long long)a.c * a.hw;
         const int ch_base = blk * 128 + wq * 32;            // first channel of this warp
         const int pgrp = lane & 7, r_sub = lane >> 3;

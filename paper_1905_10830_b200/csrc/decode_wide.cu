@@ -283,7 +283,7 @@ __global__ void __launch_bounds__(Roles<G>::kThreads, 1) decode_wide_kernel(Deco
         const float step = (float)(a.step * a.basis_scale);  // the operand holds basis / basis_scale
         const float floor_v = a.relu ? 0.f : __int_as_float((int)0xff800000u);      // the layer's non-linearity, when it follows the decoder
         __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(a.xhat);
-        const bool vec = (a.hw & 3) == 0;                    // four aligned pixels lie inside one image, 8-byte aligned
+        const bool vec = (a.hw & 3) == 0 && ((uintptr_t)a.xhat & 7u) == 0;                    // four aligned pixels lie inside one image, 8-byte aligned
         const long long img_stride = (long long)a.c * a.hw;
         const uint32_t tb = smem_u32(smem + L.tbuf) + (uint32_t)ew * kTrWarpBytes;
         const uint32_t tb_wr = tb + (uint32_t)lane * kTrRowBytes;                              // this thread's channel row

@@ -14,8 +14,7 @@
 
 namespace {
 
-constexpr size_t kScratchHeader = 64;   // ticket counter, padded
-constexpr size_t kScratchBytes = kScratchHeader + (size_t)TC_NOALLOC_MAX_TILES * sizeof(unsigned long long);
+constexpr size_t kScratchBytes = kEncodeScratchHeader + (size_t)TC_NOALLOC_MAX_TILES * sizeof(unsigned long long);
 
 // Lives in every device that loads the library, from load until the process exits (about 0.5 MB).
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kScratchBytes];
@@ -76,31 +75,9 @@ extern "C" tc_status tc_encode_noalloc(tc_ctx *ctx, const tc_model *m, const tc_
     }
     void *scratch = nullptr;
     if ((st = scratch_address(ctx->device, &scratch)) != TC_OK) return st;
-    // The array still holds the previous call's tickets and tile states: everything this call
-    // will read has to start at zero.
-    const size_t used = kScratchHeader + (size_t)lay.n_tiles * sizeof(unsigned long long);
-    if (cudaMemsetAsync(scratch, 0, used, s) != cudaSuccess) { cudaGetLastError(); return TC_ERR_CUDA; }
-
-    EncodeArgs a{};
-    a.x = x->data; a.n = x->n; a.c = x->c; a.hw = x->h * x->w; a.k = m->k; a.bits = m->bits; a.groups = cb->groups;
-    a.pixels = pixels; a.n_tiles = lay.n_tiles; a.chunk_pixels = lay.chunk_pixels; a.splits = lay.pixel_splits;
-    a.basis64 = m->d_basis64; a.mean64 = m->d_mean64; a.lo = m->lo; a.step = m->step;
-    a.enc = cb->d_enc; a.stream = (uint32_t *)stream_out;
-    a.capacity_bits = (unsigned long long)(capacity & ~(size_t)15) * 8ull;
-    a.chunk_len = chunk_len; a.tile_off = (unsigned long long *)tile_off; a.basis_scale = m->basis_scale;
-    a.dbg_coef = nullptr; a.dbg_sym = nullptr;
-    a.ticket = (unsigned int *)scratch;
-    a.tile_state = (unsigned long long *)((char *)scratch + kScratchHeader);
-    a.status = ctx->d_status; a.clamped = nullptr; a.emit = 1;
-    a.basis_bf16 = m->d_basis_bf16; a.enc_bias = m->d_enc_bias; a.tmu32 = m->d_tmu32;
-    if (!ctx->force_exact && x->dtype == TC_BF16 && tc_encode_tc_supported(ctx, a)) {
-        ctx->last_encode_path = 1;
-        return tc_launch_encode_tc(ctx, a, s);
-    }
-    if (!ctx->force_exact && x->dtype == TC_BF16 && x->c % 2 == 0) {      // shapes the tensor-core kernel does not take
-        ctx->last_encode_path = 2;
-        return tc_launch_encode_simt_fp32(ctx, a, s);
-    }
-    ctx->last_encode_path = 0;
-    return tc_launch_encode_simt(ctx, a, x->dtype, s);
+    // The array still holds the previous call's tickets and tile states; the shared dispatch
+    // clears, on the stream, everything this call will read, then picks the same kernels as
+    // tc_encode (tensor-core kernels with the basis resident or streamed, fp32, fp64).
+    return tc_encode_with_scratch(ctx, m, cb, x, lay.chunk_pixels, lay.pixel_splits, stream_out, capacity, chunk_len, tile_off,
+                                  nullptr, scratch, s);
 }

@@ -591,6 +591,8 @@ bool tc_encode_tc_supported(const tc_ctx *ctx, const EncodeArgs &a)
 {
     // K <= C leading components (PCA truncation): K is the N dimension of the MMA
     if (a.c % 16 != 0 || a.k % 16 != 0 || a.k < 16 || a.k > a.c || a.c > 256 || a.hw % 4 != 0) return false;
+    // the loaders copy groups of four pixels with 8-byte cp.async: the tensor must start on an 8-byte boundary
+    if (((uintptr_t)a.x & 7u) != 0) return false;
     // two chunks per pixel must coincide with the two halves the epilogue threads work on
     // (four chunks: each half splits once more in its middle)
     if (a.splits != 1 && !(a.splits == 2 && a.k % 32 == 0) && !(a.splits == 4 && a.k % 64 == 0 && a.chunk_pixels == 1)) return false;

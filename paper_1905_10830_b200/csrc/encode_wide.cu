@@ -128,7 +128,7 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
         // element loads) of the pixels and little arithmetic besides.
         const int lt = tid - kLoaderWarp0 * 32;               // 0..255
         const __nv_bfloat16 *xin = reinterpret_cast<const __nv_bfloat16 *>(a.x);
-        const bool aligned = (a.hw & 3) == 0;                 // groups of four pixels are 8-byte aligned and inside one image
+        const bool aligned = (a.hw & 3) == 0 && ((uintptr_t)a.x & 7u) == 0;                 // groups of four pixels are 8-byte aligned and inside one image
         const int lag = stages - 1;                           // 1..3 cp.async groups pending behind the one handed over
         // basis piece of a stage: coefficient rows j0 .. j0 + ncols, channels k0 .. k0 + 32, K-major core
         // matrices (j / 8) * 512 + (ch / 8) * 128 + (j % 8) * 16; this thread copies 16-byte piece

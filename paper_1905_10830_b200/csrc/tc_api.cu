@@ -691,6 +691,52 @@ void tc_codebook_free(tc_codebook *cb)
 
 // ---- encode / decode ----------------------------------------------------------------------
 
+}  // extern "C"
+
+// Argument block and kernel choice shared by tc_encode and tc_encode_noalloc.  `scratch` is
+// kEncodeScratchHeader bytes (ticket counter) followed by one 64-bit look-back word per tile;
+// it is cleared on the stream here, whoever owns it.
+tc_status tc_encode_with_scratch(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const tc_tensor *x, int chunk_pixels,
+                                 int splits, void *stream_out, size_t capacity, uint16_t *chunk_len, uint64_t *tile_off,
+                                 const tc_debug_out *debug, void *scratch, cudaStream_t s)
+{
+    const long long pixels = (long long)x->n * x->h * x->w;
+    const long long n_tiles = (pixels + TC_TILE_PIXELS - 1) / TC_TILE_PIXELS;
+    TC_CUDA(cudaMemsetAsync(scratch, 0, kEncodeScratchHeader + (size_t)n_tiles * sizeof(unsigned long long), s));
+
+    EncodeArgs a{};
+    a.x = x->data; a.n = x->n; a.c = x->c; a.hw = x->h * x->w; a.k = m->k; a.bits = m->bits; a.groups = cb->groups;
+    a.pixels = pixels; a.n_tiles = n_tiles; a.chunk_pixels = chunk_pixels; a.splits = splits;
+    a.basis64 = m->d_basis64; a.mean64 = m->d_mean64; a.lo = m->lo; a.step = m->step;
+    a.enc = cb->d_enc; a.stream = (uint32_t *)stream_out;
+    a.capacity_bits = (unsigned long long)(capacity & ~(size_t)15) * 8ull;
+    a.chunk_len = chunk_len; a.tile_off = (unsigned long long *)tile_off; a.basis_scale = m->basis_scale;
+    a.dbg_coef = debug ? debug->coefficients : nullptr;
+    a.dbg_sym = debug ? debug->symbols : nullptr;
+    a.ticket = (unsigned int *)scratch;
+    a.tile_state = (unsigned long long *)((char *)scratch + kEncodeScratchHeader);
+    a.status = ctx->d_status; a.clamped = nullptr; a.emit = 1;
+    a.basis_bf16 = m->d_basis_bf16; a.enc_bias = m->d_enc_bias; a.tmu32 = m->d_tmu32;
+    a.basis_map = m->has_basis_map ? &m->basis_map : nullptr;
+    if (!ctx->force_exact && x->dtype == TC_BF16 && tc_encode_tc_supported(ctx, a)) {
+        ctx->last_encode_path = 1;
+        return tc_launch_encode_tc(ctx, a, s);
+    }
+    if (ctx->force_exact != 1 && x->dtype == TC_BF16 && tc_encode_wide_supported(ctx, a)) {   // wide layers, unaligned rows
+        ctx->last_encode_path = 3;
+        return tc_launch_encode_wide(ctx, a, s);
+    }
+    if (ctx->force_exact != 1 && x->dtype == TC_BF16 && x->c % 2 == 0) {      // shapes the tensor-core kernel does not take
+        ctx->last_encode_path = 2;
+        return tc_launch_encode_simt_fp32(ctx, a, s);
+    }
+    ctx->last_encode_path = 0;
+    return tc_launch_encode_simt(ctx, a, x->dtype, s);
+}
+
+extern "C" {
+
+
 static tc_status check_codec_args(const tc_model *m, const tc_codebook *cb, const tc_tensor *x)
 {
     if (!m || !cb || !valid_tensor(x)) return TC_ERR_INVALID_ARG;
@@ -740,38 +786,10 @@ tc_status tc_encode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
         TC_CUDA(cudaMemsetAsync(tile_off, 0, sizeof(uint64_t), s));
         return TC_OK;
     }
-    const size_t scratch = 64 + (size_t)n_tiles * sizeof(unsigned long long);
+    const size_t scratch = kEncodeScratchHeader + (size_t)n_tiles * sizeof(unsigned long long);
     if ((st = ensure_scratch(ctx, scratch)) != TC_OK) return st;
-    TC_CUDA(cudaMemsetAsync(ctx->scratch, 0, scratch, s));
-
-    EncodeArgs a{};
-    a.x = x->data; a.n = x->n; a.c = x->c; a.hw = x->h * x->w; a.k = m->k; a.bits = m->bits; a.groups = cb->groups;
-    a.pixels = pixels; a.n_tiles = n_tiles; a.chunk_pixels = cs.cp; a.splits = cs.splits;
-    a.basis64 = m->d_basis64; a.mean64 = m->d_mean64; a.lo = m->lo; a.step = m->step;
-    a.enc = cb->d_enc; a.stream = (uint32_t *)stream_out;
-    a.capacity_bits = (unsigned long long)(capacity & ~(size_t)15) * 8ull;
-    a.chunk_len = chunk_len; a.tile_off = (unsigned long long *)tile_off; a.basis_scale = m->basis_scale;
-    a.dbg_coef = debug ? debug->coefficients : nullptr;
-    a.dbg_sym = debug ? debug->symbols : nullptr;
-    a.ticket = (unsigned int *)ctx->scratch;
-    a.tile_state = (unsigned long long *)((char *)ctx->scratch + 64);
-    a.status = ctx->d_status; a.clamped = nullptr; a.emit = 1;
-    a.basis_bf16 = m->d_basis_bf16; a.enc_bias = m->d_enc_bias; a.tmu32 = m->d_tmu32;
-    a.basis_map = m->has_basis_map ? &m->basis_map : nullptr;
-    if (!ctx->force_exact && x->dtype == TC_BF16 && tc_encode_tc_supported(ctx, a)) {
-        ctx->last_encode_path = 1;
-        return tc_launch_encode_tc(ctx, a, s);
-    }
-    if (ctx->force_exact != 1 && x->dtype == TC_BF16 && tc_encode_wide_supported(ctx, a)) {   // wide layers, unaligned rows
-        ctx->last_encode_path = 3;
-        return tc_launch_encode_wide(ctx, a, s);
-    }
-    if (ctx->force_exact != 1 && x->dtype == TC_BF16 && x->c % 2 == 0) {      // shapes the tensor-core kernel does not take
-        ctx->last_encode_path = 2;
-        return tc_launch_encode_simt_fp32(ctx, a, s);
-    }
-    ctx->last_encode_path = 0;
-    return tc_launch_encode_simt(ctx, a, x->dtype, s);
+    return tc_encode_with_scratch(ctx, m, cb, x, cs.cp, cs.splits, stream_out, capacity, chunk_len, tile_off, debug,
+                                  ctx->scratch, s);
 }
 
 tc_status tc_decode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const void *stream, size_t stream_bytes,

@@ -130,6 +130,12 @@ struct DecodeArgs {
     unsigned int *status;
 };
 
+// ---- encode dispatch shared by tc_encode and tc_encode_noalloc (tc_api.cu) --------------------
+constexpr size_t kEncodeScratchHeader = 64;   // ticket counter, padded; the per-tile look-back words follow
+tc_status tc_encode_with_scratch(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const tc_tensor *x, int chunk_pixels,
+                                 int splits, void *stream_out, size_t capacity, uint16_t *chunk_len, uint64_t *tile_off,
+                                 const tc_debug_out *debug, void *scratch, cudaStream_t s);
+
 // ---- launchers (defined in the .cu files) ----------------------------------------------
 tc_status tc_launch_encode_simt(const tc_ctx *ctx, const EncodeArgs &a, int dtype, cudaStream_t s);
 tc_status tc_launch_decode_simt(const tc_ctx *ctx, const DecodeArgs &a, int dtype, cudaStream_t s);

@@ -52,3 +52,45 @@ def chunk_len(enc) -> np.ndarray:
 
 def tile_off(enc) -> np.ndarray:
     return enc.tile_off.cpu().numpy().view(np.uint64)
+
+
+def expected_output_flips(m: oracle.Model, q: np.ndarray, *, out_bf16: bool = True) -> float:
+    """Expected number of reconstructed values that an fp32 tensor-core decoder rounds to the
+    neighbouring output value, for symbols `q` ([P][K]).
+
+    The decoder computes v = fl32(step * acc + bias_c) with acc = sum_j T[j][c] (q_j - center)
+    accumulated in fp32, one rounding per tensor-core step of 16 coefficients (products of a bf16
+    and a small integer are exact), then rounds v once to the output type; the oracle rounds the
+    exact value once.  The two differ only where an output rounding boundary lies between the
+    exact value and v.  A rounding to fp32 errs by at most h = 2^-24 |x|, uniformly; n such errors
+    add like a random walk to a mean magnitude of 0.46 sqrt(sum h_i^2), so with s_i the partial
+    sums after each step
+        E|delta| = 0.46 * 2^-24 * sqrt(sum_i (step s_i)^2 + v^2).
+    Output rounding boundaries are one output ulp u apart, so a value flips with probability
+    E|delta| / u.  Outputs near zero (a bias cancelled by the sum) have a small ulp and carry most
+    of the expectation; it grows with the bit width because more coefficients are non-zero and
+    the cancelled terms grow."""
+    k = m.k
+    t = np.asarray(m.basis[:k], dtype=np.float64)
+    top = (1 << m.bits) - 1
+    center = min(top, max(0.0, float(np.rint(-m.lo / m.step))))
+    d = q.astype(np.float64) - center
+    bias = m.mean + (m.lo + center * m.step) * t.sum(axis=0)
+    run = np.zeros((q.shape[0], t.shape[1]))
+    sum_sq = np.zeros_like(run)
+    for j0 in range(0, k, 16):
+        run = run + m.step * (d[:, j0:j0 + 16] @ t[j0:j0 + 16])
+        sum_sq += run * run
+    v = run + bias
+    mant = 7 if out_bf16 else 23
+    ulp = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(v), 2.0 ** -126))) - mant)
+    delta = 0.46 * 2.0 ** -24 * np.sqrt(sum_sq + v * v)
+    return float(np.minimum(1.0, delta / ulp).sum())
+
+
+def flip_allowance(expected: float) -> int:
+    """Upper bound on the observed count given the model's expectation: twice the expectation
+    (an accumulator that truncates instead of rounding doubles every error) plus 4.5 standard
+    deviations of a Poisson count of that mean, plus one."""
+    lam = 2.0 * expected
+    return int(np.ceil(lam + 4.5 * np.sqrt(lam) + 1.0))

@@ -4,9 +4,9 @@ oracle's model and codebook imported into the library (identical T, mu, lo, step
 Bars: the entropy-coded stream is bit-exact given identical symbols and decode round-trips
 exactly; projected coefficients agree within 1e-3 * max(|y|, step); at most 1e-4 of the
 symbols differ, only by +-1 and only where the oracle's position (y - lo)/step lies within
-1e-3 of a half-integer; x_hat agrees within max(1e-3 * max(|x_hat|, step), one output ulp)
-and is bit-identical for at least 99.9 % of the values (all but one for tensors of fewer than a
-thousand)."""
+1e-3 of a half-integer; x_hat agrees within max(1e-3 * max(|x_hat|, step), one output ulp),
+and the number of values that are not bit-identical stays within what the fp32 arithmetic of
+the decoder explains (tests/helpers.py: expected_output_flips, flip_allowance)."""
 import numpy as np
 import pytest
 import torch
@@ -64,6 +64,10 @@ def check_stream_against_oracle(enc, q_gpu, lengths, bits):
     return ref
 
 
+def _as_set(route):
+    return route if isinstance(route, (set, frozenset, tuple, list)) else (route,)
+
+
 def run_case(ctx, spec, bits, n_cal, n_test, dtype, per_channel, *, exact, chunk_pixels=0, pixel_splits=0, model=None,
              routes=None, k=None, basis_round=None):
     """`routes`: the kernels expected for (encode, decode): 0 fp64, 1 tensor core (basis resident
@@ -77,7 +81,7 @@ def run_case(ctx, spec, bits, n_cal, n_test, dtype, per_channel, *, exact, chunk
     x = o["x"].cuda()
     enc = tc.tc_encode(ctx, model_h, cb, x, chunk_pixels=chunk_pixels, pixel_splits=pixel_splits, debug=True, k=m.k)
     assert tc.tc_get_status(ctx) == 0
-    assert tc.tc_last_path(ctx) == routes[0], "unexpected kernel route"
+    assert tc.tc_last_path(ctx) in _as_set(routes[0]), "unexpected kernel route"
     # coefficients
     y_gpu = enc.coefficients.cpu().numpy().astype(np.float64)
     tol = 1e-3 * np.maximum(np.abs(o["y"]), m.step)
@@ -91,7 +95,7 @@ def run_case(ctx, spec, bits, n_cal, n_test, dtype, per_channel, *, exact, chunk
     # decode: reconstruct what the stream holds
     xhat = tc.tc_decode(ctx, model_h, cb, enc, x.shape, dtype)
     assert tc.tc_get_status(ctx) == 0
-    assert tc.tc_last_path(ctx, True) == routes[1], "unexpected kernel route"
+    assert tc.tc_last_path(ctx, True) in _as_set(routes[1]), "unexpected kernel route"
     want = oracle.reconstruct(m, q_gpu, x.shape, out_bf16=(dtype == torch.bfloat16))
     got = xhat.float().cpu().numpy()
     if exact:
@@ -102,7 +106,9 @@ def run_case(ctx, spec, bits, n_cal, n_test, dtype, per_channel, *, exact, chunk
         mant = 7 if dtype == torch.bfloat16 else 23
         ulp = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(want), 1e-30))) - mant)
         assert np.all(np.abs(got - want) <= np.maximum(1e-3 * np.maximum(np.abs(want), m.step), ulp))
-        assert (got != want).sum() <= np.ceil(1e-3 * got.size)      # (one value, for tensors of fewer than a thousand)
+        # how many values may land on the neighbouring output number follows from the fp32 arithmetic
+        flips, expected = int((got != want).sum()), H.expected_output_flips(m, q_gpu, out_bf16=(dtype == torch.bfloat16))
+        assert flips <= H.flip_allowance(expected), f"{flips} values differ from the oracle's, {expected:.2f} expected"
     model_h.close()
     cb.close()
     return o, enc
