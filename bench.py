@@ -107,7 +107,7 @@ def oracle_setup(spec, bits, calib_maps, sample_images, dtype):
     params = fm.layer_params(spec)
     cal = fm.make_maps(params, calib_maps, calib=True, dtype=dtype)
     x = fm.make_maps(params, sample_images, dtype=dtype)
-    m = oracle.fit_pca(cal, bits, basis_round="bf16" if dtype == torch.bfloat16 else "f32")
+    m = oracle.fit_pca(cal, bits, basis_round="bf16" if dtype == torch.bfloat16 else "f32", zero_level=True)
     q_cal = oracle.quantize(m, oracle.project(m, cal))
     lengths = oracle.huffman_lengths(oracle.histogram(q_cal, bits, False), 12)
     return dict(model=m, lengths=lengths, x=x, bits=bits, dtype=dtype,
@@ -174,6 +174,9 @@ def main():
     ap.add_argument("--workload", type=int, default=5, choices=[3, 4, 5],
                     help="configuration the layer is taken from (default 5: the throughput layer; 3, 4: per-layer profiling)")
     ap.add_argument("--layer", type=int, default=0, help="index of the layer inside --workload")
+    ap.add_argument("--route", type=int, default=0, choices=[0, 2, 3],
+                    help="kernel selection for profiling (tc_force_exact_path): 0 default, 2 the kernels that stream the basis, "
+                         "3 the symbol-by-symbol resident-basis decoder instead of the run-skipping one")
     ap.add_argument("--sample-images", type=int, default=0, help="images per oracle timing sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -219,6 +222,7 @@ def main():
     l2_note = (f"inputs larger than L2 ({raw_bytes / 1e6:.0f} MB per pass), no flush" if raw_bytes > 126e6
                else f"inputs of {raw_bytes / 1e6:.0f} MB fit the 126 MB L2 and are not flushed: profiling only")
     lay = tc.tc_encode_bound(model, cb, x, **chunking)
+    tc.tc_force_exact_path(ctx, args.route)
     enc = tc.tc_encode(ctx, model, cb, x, **chunking)
     xhat = torch.empty_like(x)
     tc.tc_decode(ctx, model, cb, enc, x.shape, x.dtype, out=xhat)
@@ -229,6 +233,7 @@ def main():
     stream_bytes = total_bits // 8
     side_bytes = lay.chunk_len_bytes + lay.tile_off_bytes
     test_stats = tc.tc_stats(ctx, model, cb, x[: min(batch, 256)], groups=1, want_hist=False)
+    tc.tc_force_exact_path(ctx, args.route)
 
     def step():
         tc.tc_encode(ctx, model, cb, x, out=enc, **chunking)

@@ -108,6 +108,13 @@ typedef struct {
                             one scale s = max|T| / 127 for the matrix, every entry becomes
                             s * n with n an integer in [-127, 127]; the decoder uses the
                             transpose of the same matrix.                                   */
+    int32_t zero_level;  /* non-zero: the quantiser grid lo + q * step is shifted by at most half
+                            a step so that y = 0 is one of its levels: lo = -step * n with
+                            n = round(-lo_measured / step), ties to even.  The coefficients are
+                            zero-mean and most of them tiny after the PCA; with zero on a level
+                            a low-variance channel maps to a single value (Appendix E), with zero
+                            between two levels it flips between both, which costs rate and
+                            distortion.  0 keeps lo at the calibration minimum.                */
 } tc_fit_params;
 
 /* Fit on calibration maps (`calib->n` maps).  Mean and covariance (1/(M-1), M = n*h*w pixel

@@ -93,6 +93,9 @@ class Model:
     step: float
     basis_round: str = "f64"   # "f64", "bf16", "f32" or "int8": how the basis was rounded at fit time
     basis_scale: float = 1.0   # "int8": every basis entry is an integer in [-127, 127] times this
+    cal_lo: float | None = None   # range of coefficient 0 on the calibration maps, as measured
+    cal_hi: float | None = None
+    zero_level: bool = False   # the grid was shifted so that y = 0 is a level (zero_level_lo)
 
 
 @dataclass
@@ -146,9 +149,29 @@ def eigh_jacobi(a: np.ndarray):
 JACOBI_MAX_C = 128
 
 
+def zero_level_lo(lo: float, step: float) -> float:
+    """Lowest level of the quantiser grid shifted so that y = 0 is one of its levels.
+
+    Section 3.1 ("Quantization") takes the dynamic range from the highest-variance coefficient and
+    leaves the position of the levels open.  The coefficients are zero-mean (the mean is
+    subtracted before the projection) and, after the PCA, most of them are tiny: Appendix E
+    observes that all values of a low-variance channel map to a single value.  That only happens
+    when zero is a reconstruction level; with zero half-way between two levels such a channel
+    flips between its two neighbours.  So the grid lo + q*step keeps the step the range gives
+    and moves by at most half a step: round(-lo / step) levels (ties to even) lie below zero."""
+    return float(-step * np.rint(-lo / step))
+
+
+def _finish_model(c, k, bits, mean, basis, eig, lo, step, basis_round, scale, zero_level) -> "Model":
+    hi = lo + step * ((1 << bits) - 1)
+    return Model(c, k, bits, mean, basis, eig, zero_level_lo(lo, step) if zero_level else lo, step,
+                 basis_round, scale, lo, hi, zero_level)
+
+
 def fit_pca(x, bits: int, *, k: int | None = None, basis_bf16: bool = False,
-            basis_round: str | None = None, eigensolver: str = "auto") -> Model:
-    """Fit mean, basis and quantiser range on calibration maps.
+            basis_round: str | None = None, eigensolver: str = "auto", zero_level: bool = False) -> Model:
+    """Fit mean, basis and quantiser range on calibration maps.  `zero_level` shifts the quantiser
+    grid so that y = 0 is a level (zero_level_lo).
 
     basis_round: "f64" (keep), "bf16", "f32" or "int8" (8-bit matrix with one scale).  eigensolver: "jacobi" (the in-file solver),
     "lapack" (numpy.linalg.eigh, a library primitive used as one step) or "auto" = Jacobi up
@@ -179,15 +202,16 @@ def fit_pca(x, bits: int, *, k: int | None = None, basis_bf16: bool = False,
                            _p(mean), _p(basis), _p(eig), C.byref(lo), C.byref(step), C.byref(scale))
     if rc != 0:
         raise RuntimeError("oracle eigensolver did not converge")
-    return Model(c, c if k is None else k, bits, mean, basis, eig, lo.value, step.value,
-                 basis_round, scale.value)
+    return _finish_model(c, c if k is None else k, bits, mean, basis, eig, lo.value, step.value,
+                         basis_round, scale.value, zero_level)
 
 
 def with_bits(m: Model, bits: int) -> Model:
     """The same transform with the calibration range divided into 2^bits - 1 steps."""
-    hi = m.lo + m.step * ((1 << m.bits) - 1)
-    return Model(m.c, m.k, bits, m.mean, m.basis, m.eig, m.lo, (hi - m.lo) / ((1 << bits) - 1),
-                 m.basis_round, m.basis_scale)
+    lo = m.lo if m.cal_lo is None else m.cal_lo
+    hi = m.lo + m.step * ((1 << m.bits) - 1) if m.cal_hi is None else m.cal_hi
+    return _finish_model(m.c, m.k, bits, m.mean, m.basis, m.eig, lo, (hi - lo) / ((1 << bits) - 1),
+                         m.basis_round, m.basis_scale, m.zero_level)
 
 
 def project(model: Model, x) -> np.ndarray:
@@ -335,7 +359,7 @@ class Moments:
 
 
 def fit_pca_moments(state: Moments, x_range, bits: int, *, k: int | None = None, basis_round: str = "f64",
-                    eigensolver: str = "auto") -> Model:
+                    eigensolver: str = "auto", zero_level: bool = False) -> Model:
     """fit_pca with mean and covariance from a running state; the range of coefficient 0 is
     measured on `x_range`."""
     x = _f32(x_range)
@@ -359,7 +383,8 @@ def fit_pca_moments(state: Moments, x_range, bits: int, *, k: int | None = None,
                                    _p(mean), _p(basis), _p(eig), C.byref(lo), C.byref(step), C.byref(scale))
     if rc != 0:
         raise RuntimeError("oracle eigensolver did not converge")
-    return Model(c, c if k is None else k, bits, mean, basis, eig, lo.value, step.value, basis_round, scale.value)
+    return _finish_model(c, c if k is None else k, bits, mean, basis, eig, lo.value, step.value, basis_round,
+                         scale.value, zero_level)
 
 
 def fold_forward(model: Model, w: np.ndarray, bias: np.ndarray, scale: np.ndarray, shift: np.ndarray):

@@ -30,7 +30,7 @@ class _Tensor(C.Structure):
 
 
 class _FitParams(C.Structure):
-    _fields_ = [("bits", C.c_int32), ("k", C.c_int32), ("basis_dtype", C.c_int32)]
+    _fields_ = [("bits", C.c_int32), ("k", C.c_int32), ("basis_dtype", C.c_int32), ("zero_level", C.c_int32)]
 
 
 class _ModelDesc(C.Structure):
@@ -244,9 +244,12 @@ def tc_get_status(ctx: Context) -> int:
     return load_library().tc_get_status(ctx.ptr, _stream_ptr(ctx.device))
 
 
-def tc_fit_pca(ctx: Context, calib: torch.Tensor, bits: int, k: int = 0, basis_dtype: int | None = None) -> Model:
+def tc_fit_pca(ctx: Context, calib: torch.Tensor, bits: int, k: int = 0, basis_dtype: int | None = None,
+               zero_level: bool = True) -> Model:
+    """`zero_level` (on by default here; tc_fit_params.zero_level in the C ABI) shifts the quantiser
+    grid so that y = 0 is one of its levels."""
     t = _tensor(calib)
-    params = _FitParams(bits, k, t.dtype if basis_dtype is None else basis_dtype)
+    params = _FitParams(bits, k, t.dtype if basis_dtype is None else basis_dtype, int(zero_level))
     out = C.c_void_p()
     _check(load_library().tc_fit_pca(ctx.ptr, C.byref(t), C.byref(params), C.byref(out),
                                      _stream_ptr(ctx.device)), "tc_fit_pca")
@@ -287,9 +290,9 @@ def tc_fit_state_import(ctx: Context, state: FitState, count: int, s1: np.ndarra
 
 
 def tc_fit_state_finish(ctx: Context, state: FitState, range_maps: torch.Tensor, bits: int, k: int = 0,
-                        basis_dtype: int | None = None) -> Model:
+                        basis_dtype: int | None = None, zero_level: bool = True) -> Model:
     t = _tensor(range_maps)
-    params = _FitParams(bits, k, t.dtype if basis_dtype is None else basis_dtype)
+    params = _FitParams(bits, k, t.dtype if basis_dtype is None else basis_dtype, int(zero_level))
     out = C.c_void_p()
     _check(load_library().tc_fit_state_finish(ctx.ptr, state.ptr, C.byref(t), C.byref(params), C.byref(out),
                                               _stream_ptr(ctx.device)), "tc_fit_state_finish")

@@ -34,13 +34,13 @@ namespace {
 using namespace tcdev;
 using namespace sm100;
 
-constexpr int kGroupWarps = 8, kEpiWarp0 = 16, kMmaWarp = 24;
-constexpr int kThreads = 25 * 32;
+constexpr int kGroupWarps = 8;                                // warps of a VLD group; the epilogue's eight warps and the MMA warp follow
+__host__ __device__ constexpr int block_threads(int nbuf) { return (kGroupWarps * nbuf + 8 + 1) * 32; }
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;
 constexpr int kPanelK = 32;                                   // coefficients per hand-over panel
 constexpr int kMaxPanels = 8;                                 // K <= 256
-constexpr int kRunCap = 20;                                   // zero bits skipped per step (20 + 12 <= 32: one refill per step)
+constexpr uint32_t kRunGuard = 0x800u;                        // bit 11 set: at most 20 zero bits are skipped per step (20 + 12 <= 32: one refill per step)
 constexpr int kDenseBits128 = 224;                            // tiles above 1.75 bits per symbol are decoded symbol by symbol
 // A chunk that starts inside a staged segment is read for at most (symbols of the chunk) x 12
 // bits, whatever the bits say; the slack after the last buffer keeps those reads inside the
@@ -151,11 +151,26 @@ struct BitReader {
     }
     __device__ __forceinline__ void refill()
     {
-        if (used & 32u) {
-            // c = used - 32 bits of the new word's position are already consumed: the window gains
-            // `ahead` behind its 64 - used valid bits
-            hi |= __funnelshift_l(ahead, 0u, used);           // ahead >> (32 - c), zero when c == 0
-            lo |= __funnelshift_l(0u, ahead, used);           // ahead << c
+        // with c = used - 32 bits of the next word's span already taken, the window gains `ahead`
+        // behind its 64 - used valid bits: hi |= ahead >> (32 - c), lo |= ahead << c (the shifts take
+        // their amount modulo 32)
+        if constexpr (kShared) {
+            asm volatile(
+                "{\n\t.reg .pred p;\n\t.reg .b32 t, u;\n\t"
+                "and.b32 t, %3, 32;\n\t"
+                "setp.ne.u32 p, t, 0;\n\t"
+                "shf.l.wrap.b32 t, %2, 0, %3;\n\t"
+                "shf.l.wrap.b32 u, 0, %2, %3;\n\t"
+                "@p or.b32 %0, %0, t;\n\t"
+                "@p or.b32 %1, %1, u;\n\t"
+                "@p add.u32 %3, %3, -32;\n\t"
+                "@p add.u32 %5, %5, 1;\n\t"
+                "@p ld.shared.u32 %2, [%4];\n\t"
+                "@p add.u32 %4, %4, 4;\n\t}"
+                : "+r"(hi), "+r"(lo), "+r"(ahead), "+r"(used), "+r"(next_addr), "+r"(words));
+        } else if (used & 32u) {
+            hi |= __funnelshift_l(ahead, 0u, used);
+            lo |= __funnelshift_l(0u, ahead, used);
             used -= 32u;
             ahead = fetch();
             ++words;
@@ -164,9 +179,12 @@ struct BitReader {
     __device__ __forceinline__ uint32_t consumed() const { return words * 32u + (used & 0xffu) - start_bits; }
 };
 
-template <bool kRelu>
-__global__ void __launch_bounds__(kThreads, 1) decode_runs_kernel(DecodeArgs a)
+// kBufs: operand buffers = working VLD groups (the launch has no warps for a second group when
+// shared memory holds one buffer only, which leaves its threads more registers)
+template <bool kRelu, int kBufs>
+__global__ void __launch_bounds__(block_threads(kBufs), 1) decode_runs_kernel(DecodeArgs a)
 {
+    constexpr int kEpiWarp0 = kGroupWarps * kBufs, kMmaWarp = kEpiWarp0 + 8, kThreads = block_threads(kBufs);
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) unsigned long long s_full[2], s_empty[2][kMaxPanels], s_tfull[2], s_tempty[2];
     __shared__ uint32_t s_tmem_base;
@@ -175,7 +193,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_runs_kernel(DecodeArgs a)
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int lut_size = 1 << a.lut_bits;
     const SmemLayout L = smem_layout(a.c, a.k, lut_size, a.smem_budget);
-    const int nbuf = L.nbuf;
+    constexpr int nbuf = kBufs;
     const uint32_t basis_addr = smem_u32(smem + L.basis);
     const uint32_t lut_addr = smem_u32(smem + L.lut);
     const uint32_t vtab_addr = smem_u32(smem + L.vtab);
@@ -223,11 +241,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_runs_kernel(DecodeArgs a)
 
     const long long my_tiles = (a.n_tiles > blockIdx.x) ? (a.n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
 
-    if (warp < 2 * kGroupWarps) {
+    if (warp < kEpiWarp0) {
         // ================= VLD groups =================
         const int grp = warp >> 3;
         const int tg = tid & 255;                // thread within the group
-        if (grp < nbuf && tg < n_thr) {
+        if (tg < n_thr) {
             const int set = cp > 1 ? 0 : tg >> 7;    // which thread of the pixel (warp-uniform)
             const int t = cp > 1 ? tg : (tg & 127);  // pixel within the tile, or chunk within the tile (cp > 1)
             const int wq = (t >> 5) & 3;
@@ -283,7 +301,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_runs_kernel(DecodeArgs a)
             TileInfo cur = tile_info(grp), nxt = tile_info(grp + nbuf);
             stage_tile(cur, 0);
             int li = 0;
-            for (long long tl = grp; tl < my_tiles && alive; tl += nbuf, ++li) {
+            // (a thread whose wait ran out keeps walking the tiles without decoding: the group's
+            // barriers and the hand-over to the MMA thread need every thread's arrival)
+            for (long long tl = grp; tl < my_tiles; tl += nbuf, ++li) {
                 const long long tile = blockIdx.x + tl * gridDim.x;
                 // start of every chunk = sum of the lengths before it in the tile (chunk order: pixel,
                 // then part of the pixel): scan over the pixels' totals
@@ -312,10 +332,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_runs_kernel(DecodeArgs a)
                 }
                 // this thread's first chunk: after the pixels before it and the chunks of the pixel before its own
                 unsigned int chunk_start = before + inc - tot;
-                unsigned int my_len[2] = {len0, len1};
+                unsigned int my_len0 = len0, my_len1 = len1;
                 if (cp == 1 && set == 1) {
-                    if (S == 2) { chunk_start += len0; my_len[0] = len1; }
-                    else { chunk_start += len0 + len1; my_len[0] = len2; my_len[1] = len3; }
+                    if (S == 2) { chunk_start += len0; my_len0 = len1; }
+                    else { chunk_start += len0 + len1; my_len0 = len2; my_len1 = len3; }
                 }
 
                 const long long ch = tile * chunks_per_tile + (long long)t * (cp > 1 ? 1 : S);
@@ -330,70 +350,68 @@ __global__ void __launch_bounds__(kThreads, 1) decode_runs_kernel(DecodeArgs a)
                                   cur.bits * 128ull <= (unsigned long long)kDenseBits128 * (unsigned long long)a.k * TC_TILE_PIXELS;
                 const uint32_t wait_parity = (uint32_t)((li & 1) ^ 1);   // the buffer's hand-back by the tile before this one
 
-                // walks this thread's chunks; kSh: the segment is staged in shared memory
+                // Walks this thread's chunks.  Control flow is kept uniform across the warp: the lanes
+                // of a warp step together (a lane that has finished its chunk idles until all have),
+                // panels are waited for and filled by all lanes at once when any lane needs the next
+                // one, and a wait that runs out is seen by every lane -- lanes that wander off on
+                // their own would run the rest of the tile one after the other.
                 auto decode_tile = [&](auto &r) {
                     uint32_t expect = 0;               // bits the chunks decoded so far should have taken
-                    for (int pp = 0; pp < cp && alive; ++pp) {
+                    for (int pp = 0; pp < cp; ++pp) {
                         const bool decode = pp < n_pix;
                         const uint32_t row = (uint32_t)(t * cp + pp);
                         const uint32_t row_addr = opnd_g + (row >> 3) * 128u + (row & 7u) * 16u;
-                        int ready = p_first;           // panels [p_first, ready) of this row are handed back and filled
+                        int ready = p_first;           // panels [p_first, ready) of the warp's rows are handed back and filled
                         // waits for panel p to be handed back by the MMAs of the tile before, then fills this
                         // thread's coefficients of it with the modal symbol (run mode)
                         auto prepare = [&](int p) {
-                            if (pp == 0 && !mbar_wait(smem_u32(&s_empty[grp][p]), wait_parity, 200u)) { alive = false; return; }
+                            if (pp == 0 && alive) alive = mbar_wait(smem_u32(&s_empty[grp][p]), wait_parity, 200u);
                             if (runs && owner) {
                                 const int g0 = max(p * (kPanelK / 8), k_first >> 3), g1 = min((p + 1) * (kPanelK / 8), k_last >> 3);
                                 for (int g = g0; g < g1; ++g) sts_v4(row_addr + (uint32_t)g * 2048u, modal2, modal2, modal2, modal2);
                             }
                         };
-                        for (int ci = 0; ci < (cp > 1 ? 1 : chunks_per_thread) && alive; ++ci) {
+                        for (int ci = 0; ci < (cp > 1 ? 1 : chunks_per_thread); ++ci) {
                             const int kf = cp > 1 ? 0 : k_first + ci * k_sub, ke = cp > 1 ? a.k : kf + k_sub;
                             if (runs) {
-                                int pos = kf;
-                                while (pos < ke && alive) {
-                                    uint32_t v = 0;
-                                    if (decode) {
-                                        r.refill();
-                                        const uint32_t n = min((uint32_t)__clz((int)(r.hi | 0x800u)), (uint32_t)(ke - pos));   // <= kRunCap
-                                        r.take(n);
-                                        pos += (int)n;
-                                        if (pos >= ke) break;
-                                        const uint32_t e = lds_u16(lut_addr + (r.hi >> (32 - lb)) * 2u);
-                                        r.take(e);
-                                        v = lds_u16(vtab_addr + (e >> 8) * 2u);
-                                    } else {
-                                        pos = ke - 1;      // nothing to decode: only hand the panels on
-                                    }
-                                    while (ready * kPanelK <= pos && alive) prepare(ready++);
-                                    if (decode && alive) sts_u16(row_addr + ((uint32_t)pos >> 3) * 2048u + ((uint32_t)pos & 7u) * 2u, v);
-                                    ++pos;
+                                int pos = decode ? kf : ke;
+                                while (__any_sync(0xffffffffu, pos < ke)) {
+                                    r.refill();
+                                    // a run of the modal symbol is a run of zero bits: at most 20 per step
+                                    const uint32_t n = pos < ke ? min((uint32_t)__clz((int)(r.hi | kRunGuard)), (uint32_t)(ke - pos)) : 0u;
+                                    r.take(n);
+                                    pos += (int)n;
+                                    const bool sym = pos < ke;             // a symbol follows the run
+                                    const uint32_t e = lds_u16(lut_addr + (r.hi >> (32 - lb)) * 2u);
+                                    r.take(sym ? e : 0u);
+                                    const uint32_t v = lds_u16(vtab_addr + (e >> 8) * 2u);
+                                    while (__any_sync(0xffffffffu, sym && pos >= ready * kPanelK)) prepare(ready++);
+                                    if (sym) sts_u16(row_addr + ((uint32_t)pos >> 3) * 2048u + ((uint32_t)pos & 7u) * 2u, v);
+                                    pos += sym ? 1 : 0;
                                 }
                             } else {
-                                for (int k0 = kf; k0 < ke && alive; k0 += 8) {
-                                    while (ready * kPanelK <= k0 && alive) prepare(ready++);
-                                    uint32_t pk[4] = {0u, 0u, 0u, 0u};
-                                    if (decode) {
+                                for (int k0 = kf; k0 < ke; k0 += 8) {
+                                    while (ready * kPanelK <= k0) prepare(ready++);
+                                    uint32_t pk[4];
 #pragma unroll
-                                        for (int i = 0; i < 4; ++i) {
-                                            r.refill();
-                                            const uint32_t e0 = lds_u16(lut_addr + (r.hi >> (32 - lb)) * 2u);
-                                            r.take(e0);
-                                            const uint32_t e1 = lds_u16(lut_addr + (r.hi >> (32 - lb)) * 2u);
-                                            r.take(e1);
-                                            pk[i] = lds_u16(vtab_addr + (e0 >> 8) * 2u) | (lds_u16(vtab_addr + (e1 >> 8) * 2u) << 16);
-                                        }
+                                    for (int i = 0; i < 4; ++i) {
+                                        r.refill();
+                                        const uint32_t e0 = lds_u16(lut_addr + (r.hi >> (32 - lb)) * 2u);
+                                        r.take(decode ? e0 : 0u);
+                                        const uint32_t e1 = lds_u16(lut_addr + (r.hi >> (32 - lb)) * 2u);
+                                        r.take(decode ? e1 : 0u);
+                                        pk[i] = lds_u16(vtab_addr + (e0 >> 8) * 2u) | (lds_u16(vtab_addr + (e1 >> 8) * 2u) << 16);
                                     }
-                                    if (alive) sts_v4(row_addr + (uint32_t)(k0 >> 3) * 2048u, pk[0], pk[1], pk[2], pk[3]);
+                                    if (decode) sts_v4(row_addr + (uint32_t)(k0 >> 3) * 2048u, pk[0], pk[1], pk[2], pk[3]);
                                 }
                             }
                             // a chunk of one pixel (or part of it) must end exactly where its length says
                             if (cp == 1) {
-                                expect += my_len[ci];
+                                expect += ci == 0 ? my_len0 : my_len1;
                                 if (active && r.consumed() != expect) bad = true;
                             }
                         }
-                        while (ready < p_last && alive) prepare(ready++);
+                        while (ready < p_last) prepare(ready++);
                     }
                     if (cp > 1 && active && r.consumed() != len0) bad = true;
                 };
@@ -411,13 +429,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_runs_kernel(DecodeArgs a)
                     decode_tile(r);
                 }
                 // (the issuing thread makes the operand visible to the tensor core's proxy)
-                if (alive) mbar_arrive(smem_u32(&s_full[grp]));
+                mbar_arrive(smem_u32(&s_full[grp]));
                 if (bad) tc_dev_set_status(a.status, TC_ERR_CORRUPT_STREAM);
                 cur = nxt;
                 nxt = after;
             }
             cp_async_wait<0>();
-            if (!alive && tg == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
+            if (!alive) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
         }
     } else if (warp < kMmaWarp) {
         // ================= epilogue: all eight warps work on every tile =================
@@ -576,17 +594,25 @@ bool tc_decode_runs_supported(const tc_ctx *ctx, const DecodeArgs &a)
     return l.nbuf > 0;
 }
 
+// Bytes of a tile's stream segment this kernel stages in shared memory; longer segments are read
+// from global memory, word by word.
+size_t tc_decode_runs_staging_bytes(const tc_ctx *ctx, const DecodeArgs &a)
+{
+    return smem_layout(a.c, a.k, 1 << a.lut_bits, ctx->max_smem_optin - 512).stream_buf;
+}
+
 tc_status tc_launch_decode_runs(const tc_ctx *ctx, const DecodeArgs &a, cudaStream_t s)
 {
     if (a.n_tiles <= 0) return TC_OK;
     const SmemLayout l = smem_layout(a.c, a.k, 1 << a.lut_bits, ctx->max_smem_optin - 512);
     if (l.nbuf == 0) return TC_ERR_UNSUPPORTED;
-    void (*kernel)(DecodeArgs) = a.relu ? decode_runs_kernel<true> : decode_runs_kernel<false>;
+    void (*kernel)(DecodeArgs) = l.nbuf == 2 ? (a.relu ? decode_runs_kernel<true, 2> : decode_runs_kernel<false, 2>)
+                                             : (a.relu ? decode_runs_kernel<true, 1> : decode_runs_kernel<false, 1>);
     DecodeArgs args = a;
     args.smem_budget = ctx->max_smem_optin - 512;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.total) != cudaSuccess)
         return TC_ERR_CUDA;
     const unsigned int grid = (unsigned int)((a.n_tiles < ctx->sm_count) ? a.n_tiles : ctx->sm_count);
-    kernel<<<grid, kThreads, l.total, s>>>(args);
+    kernel<<<grid, block_threads(l.nbuf), l.total, s>>>(args);
     return cudaGetLastError() == cudaSuccess ? TC_OK : TC_ERR_CUDA;
 }

@@ -185,6 +185,12 @@ tc_status finish_codebook(tc_codebook *cb)
     for (uint8_t l : cb->lengths) mx = std::max<int>(mx, l);
     cb->max_len = mx;
     cb->lut_bits = mx;
+    // canonical codes give the first symbol of the shortest length the all-zero code: with a
+    // one-bit code that is the single bit 0, and a run of that symbol is a run of zero bits
+    cb->modal = -1;
+    if (cb->groups == 1)
+        for (int s = 0; s < nsym && cb->modal < 0; ++s)
+            if (cb->lengths[s] == 1) cb->modal = s;
     std::vector<uint32_t> enc((size_t)cb->groups * nsym);
     std::vector<uint16_t> lut((size_t)cb->groups << cb->lut_bits);
     std::vector<uint32_t> lut32((size_t)cb->groups << cb->lut_bits);
@@ -289,7 +295,7 @@ void tc_destroy(tc_ctx *ctx)
 
 void tc_force_exact_path(tc_ctx *ctx, int on)
 {
-    if (ctx) ctx->force_exact = on == 2 ? 2 : (on ? 1 : 0);
+    if (ctx) ctx->force_exact = (on == 2 || on == 3) ? on : (on ? 1 : 0);
 }
 
 int tc_last_path(const tc_ctx *ctx, int decode)
@@ -452,7 +458,9 @@ static tc_status finish_fit(tc_ctx *ctx, const tc_tensor *range_maps, const tc_f
 
     tc_model_desc d;
     d.c = c; d.k = k; d.bits = params->bits; d.basis_dtype = params->basis_dtype;
-    d.lo = lo; d.step = (hi - lo) / (double)((1 << params->bits) - 1);
+    d.step = (hi - lo) / (double)((1 << params->bits) - 1);
+    // zero_level: shift the grid so that y = 0 is a level (at most half a step; ties to even)
+    d.lo = params->zero_level ? -d.step * std::nearbyint(-lo / d.step) : lo;
     d.basis = basis.data(); d.mean = mean.data(); d.eig = eig.data(); d.basis_scale = basis_scale;
     return tc_model_import(ctx, &d, out);
 }
@@ -718,7 +726,7 @@ tc_status tc_encode_with_scratch(tc_ctx *ctx, const tc_model *m, const tc_codebo
     a.status = ctx->d_status; a.clamped = nullptr; a.emit = 1;
     a.basis_bf16 = m->d_basis_bf16; a.enc_bias = m->d_enc_bias; a.tmu32 = m->d_tmu32;
     a.basis_map = m->has_basis_map ? &m->basis_map : nullptr;
-    if (!ctx->force_exact && x->dtype == TC_BF16 && tc_encode_tc_supported(ctx, a)) {
+    if ((ctx->force_exact == 0 || ctx->force_exact == 3) && x->dtype == TC_BF16 && tc_encode_tc_supported(ctx, a)) {
         ctx->last_encode_path = 1;
         return tc_launch_encode_tc(ctx, a, s);
     }
@@ -817,19 +825,27 @@ tc_status tc_decode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
     a.lut32 = cb->d_lut32; a.basis_t_bf16 = m->d_basis_t_bf16; a.dec_bias = m->d_dec_bias; a.center = m->center;
     a.relu = (params && params->relu) ? 1 : 0;
     a.basis_t_map = m->has_basis_t_map ? &m->basis_t_map : nullptr;
-    bool resident = !ctx->force_exact && x_hat->dtype == TC_BF16 && tc_decode_tc_supported(ctx, a);
-    if (resident && tc_decode_wide_supported(ctx, a)) {
-        // High-rate streams: when the average tile's segment no longer fits the shared-memory
-        // staging of the resident-basis decoder but still fits that of the streaming decoder,
-        // the latter is faster (it would otherwise read the stream from global memory word by word).
-        // (Only when `stream_bytes` is a length: a caller that passes the capacity of a worst-case
-        // buffer says nothing about the rate.)
-        const size_t worst = (size_t)a.n_tiles * TC_TILE_PIXELS * (size_t)a.k * (size_t)cb->max_len / 8;
-        const size_t avg_tile_bytes = (stream_bytes + (size_t)a.n_tiles - 1) / (size_t)a.n_tiles;
-        if (stream_bytes < worst && avg_tile_bytes > tc_decode_tc_staging_bytes(ctx, a) &&
-            avg_tile_bytes <= tc_decode_wide_staging_bytes(ctx, a))
-            resident = false;
+    a.modal = cb->modal;
+    // High-rate streams: a tile's segment that no longer fits the shared-memory staging of a
+    // resident-basis decoder but still fits that of the streaming decoder is better served by the
+    // latter (the former would read the stream from global memory word by word).  Only when
+    // `stream_bytes` is a length: a caller that passes the capacity of a worst-case buffer says
+    // nothing about the rate.
+    const size_t worst = (size_t)a.n_tiles * TC_TILE_PIXELS * (size_t)a.k * (size_t)cb->max_len / 8;
+    const size_t avg_tile_bytes = (stream_bytes + (size_t)a.n_tiles - 1) / (size_t)a.n_tiles;
+    const bool rate_known = stream_bytes < worst;
+    if (ctx->force_exact == 0 && x_hat->dtype == TC_BF16 && tc_decode_runs_supported(ctx, a)) {
+        const bool dense = rate_known && avg_tile_bytes > tc_decode_runs_staging_bytes(ctx, a) &&
+                           tc_decode_wide_supported(ctx, a) && avg_tile_bytes <= tc_decode_wide_staging_bytes(ctx, a);
+        if (!dense) {
+            ctx->last_decode_path = 1;
+            return tc_launch_decode_runs(ctx, a, (cudaStream_t)cuda_stream);
+        }
     }
+    bool resident = (ctx->force_exact == 0 || ctx->force_exact == 3) && x_hat->dtype == TC_BF16 && tc_decode_tc_supported(ctx, a);
+    if (resident && tc_decode_wide_supported(ctx, a) && rate_known && avg_tile_bytes > tc_decode_tc_staging_bytes(ctx, a) &&
+        avg_tile_bytes <= tc_decode_wide_staging_bytes(ctx, a))
+        resident = false;
     if (resident) {
         ctx->last_decode_path = 1;
         return tc_launch_decode_tc(ctx, a, (cudaStream_t)cuda_stream);

@@ -36,7 +36,7 @@ struct tc_ctx {
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
     cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
     unsigned long long *chunk_bits = nullptr;   // pinned HOST [kMaxRoundtripChunks]
-    int force_exact = 0;                  // 1: route every tensor through the fp64 kernels; 2: skip the resident-basis kernels
+    int force_exact = 0;                  // 1: route every tensor through the fp64 kernels; 2: skip the resident-basis kernels; 3: skip the run-skipping decoder
     int last_encode_path = 0;             // 0 = fp64 kernels, 1 = tensor-core kernels (resident basis), 2 = fp32 kernels, 3 = tensor-core kernels (streamed basis)
     int last_decode_path = 0;
 };
@@ -64,6 +64,7 @@ struct tc_model {
 
 struct tc_codebook {
     int bits = 0, groups = 0, max_len = 0, lut_bits = 0;
+    int modal = -1;                         // per-layer table: the symbol coded by the single bit 0 (-1: none)
     std::vector<uint8_t> lengths;           // host [groups][2^bits]
     int device = 0;
     uint32_t *d_enc = nullptr;              // [groups][2^bits]  (code << 8) | length
@@ -120,6 +121,7 @@ struct DecodeArgs {
     const CUtensorMap *basis_t_map;     // HOST pointer to the model's tensor map of basis_t_bf16, or null
     const float *dec_bias;              // [c]
     int center;                         // subtracted from every symbol before the MMA
+    int modal;                          // per-layer table: the symbol whose code is the single bit 0, or -1 if no code has one bit
     int relu;                           // x_hat = max(x_hat, 0) before it is rounded to the tensor type
     int smem_budget;                    // shared memory the tensor-core kernel may lay out (set by its launcher)
     const double *basis64;
@@ -145,11 +147,14 @@ bool tc_encode_tc_supported(const tc_ctx *ctx, const EncodeArgs &a);
 tc_status tc_launch_encode_tc(const tc_ctx *ctx, const EncodeArgs &a, cudaStream_t s);
 bool tc_decode_tc_supported(const tc_ctx *ctx, const DecodeArgs &a);
 tc_status tc_launch_decode_tc(const tc_ctx *ctx, const DecodeArgs &a, cudaStream_t s);
+bool tc_decode_runs_supported(const tc_ctx *ctx, const DecodeArgs &a);
+tc_status tc_launch_decode_runs(const tc_ctx *ctx, const DecodeArgs &a, cudaStream_t s);
 bool tc_encode_wide_supported(const tc_ctx *ctx, const EncodeArgs &a);
 tc_status tc_launch_encode_wide(const tc_ctx *ctx, const EncodeArgs &a, cudaStream_t s);
 bool tc_decode_wide_supported(const tc_ctx *ctx, const DecodeArgs &a);
 tc_status tc_launch_decode_wide(const tc_ctx *ctx, const DecodeArgs &a, cudaStream_t s);
 size_t tc_decode_tc_staging_bytes(const tc_ctx *ctx, const DecodeArgs &a);     // per tile
+size_t tc_decode_runs_staging_bytes(const tc_ctx *ctx, const DecodeArgs &a);   // per tile
 size_t tc_decode_wide_staging_bytes(const tc_ctx *ctx, const DecodeArgs &a);   // per tile
 
 tc_status tc_launch_channel_sums(const void *x, int dtype, int n, int c, int hw, double *sums,

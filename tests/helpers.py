@@ -16,13 +16,13 @@ def basis_round_for(dtype) -> str:
 
 def oracle_side(spec: fm.LayerSpec, bits: int, n_cal: int, n_test: int, dtype, per_channel: bool,
                 lmax: int = 12, model: oracle.Model | None = None, k: int | None = None,
-                basis_round: str | None = None):
+                basis_round: str | None = None, zero_level: bool = True):
     """Returns dict(model, lengths, cal, x, y, q, units) computed by the oracle on CPU maps."""
     params = fm.layer_params(spec)
     cal = fm.make_maps(params, n_cal, calib=True, dtype=dtype)
     x = fm.make_maps(params, n_test, dtype=dtype)
     if model is None:
-        model = oracle.fit_pca(cal, bits, basis_round=basis_round or basis_round_for(dtype), k=k)
+        model = oracle.fit_pca(cal, bits, basis_round=basis_round or basis_round_for(dtype), k=k, zero_level=zero_level)
     elif model.bits != bits:
         model = oracle.with_bits(model, bits)
     q_cal = oracle.quantize(model, oracle.project(model, cal))

@@ -43,7 +43,7 @@ def _expected_routes(d, layout):
     enc_resident = mode == 0 and c <= 256 and hw % 4 == 0 and \
         (splits == 1 or (splits == 2 and k % 32 == 0) or (splits == 4 and k % 64 == 0))
     enc = 1 if enc_resident else 3
-    if mode == 2 or c > 256 or splits == 4:
+    if mode == 2 or c > 256 or (splits == 4 and d["per_channel"]):
         dec = 3
     else:
         dec = (1, 3)          # the resident-basis decoder where its shared-memory plan fits, else the streaming one

@@ -58,7 +58,7 @@ def test_online_fit_matches_the_oracle_and_the_one_shot_fit(ctx, dtype, basis_ro
         tc.tc_fit_state_update(ctx, st, cal[i:i + 2].cuda())
     model = tc.tc_fit_state_finish(ctx, st, cal.cuda(), bits)
     got = tc.tc_model_export(model)
-    want = oracle.fit_pca_moments(oracle.Moments(32).update(cal), cal, bits, basis_round=basis_round)
+    want = oracle.fit_pca_moments(oracle.Moments(32).update(cal), cal, bits, basis_round=basis_round, zero_level=True)
     assert np.allclose(got["mean"], want.mean, rtol=1e-12, atol=1e-14)
     assert np.allclose(got["eig"], want.eig, rtol=1e-6, atol=1e-10 * want.eig[0])
     assert np.isclose(got["lo"], want.lo, rtol=1e-5, atol=1e-6) and np.isclose(got["step"], want.step, rtol=1e-5)
@@ -81,8 +81,12 @@ def test_online_fit_matches_the_oracle_and_the_one_shot_fit(ctx, dtype, basis_ro
     mse_ref = float(((torch.from_numpy(ref_hat) - x.float()) ** 2).mean())
     assert abs(mse_gpu - mse_ref) <= 0.01 * mse_ref + 1e-9
     # range measured on a subset of the maps can only be narrower
-    sub = tc.tc_model_export(tc.tc_fit_state_finish(ctx, st, cal[:1].cuda(), bits))
-    assert sub["lo"] >= got["lo"] - 1e-9
+    sub = tc.tc_model_export(tc.tc_fit_state_finish(ctx, st, cal[:1].cuda(), bits, zero_level=False))
+    whole = tc.tc_model_export(tc.tc_fit_state_finish(ctx, st, cal.cuda(), bits, zero_level=False))
+    assert sub["lo"] >= whole["lo"] - 1e-9
+    # the grid with zero on a level keeps the step and moves by at most half of it
+    assert np.isclose(got["step"], whole["step"], rtol=1e-12) and abs(got["lo"] - whole["lo"]) <= 0.5 * got["step"] * (1 + 1e-9)
+    assert abs(got["lo"] / got["step"] - np.rint(got["lo"] / got["step"])) < 1e-9
     st.close(); model.close(); cb.close()
 
 

@@ -198,9 +198,7 @@ def test_tensor_core_path_per_channel_codebook_and_chunks(ctx_tc):
 @pytest.mark.parametrize("c,splits", [(256, 1), (256, 2), (64, 2), (128, 2), (192, 2), (256, 4), (128, 4), (64, 4), (192, 4)])
 def test_tensor_core_path_pixel_splits(ctx_tc, c, splits):
     spec = fm.LayerSpec(c, 14, 14, 0.9, None, 5300 + c)
-    # four chunks per pixel: the resident-basis encoder takes them, the decoder that streams the basis decodes them
-    _, enc = run_case(ctx_tc, spec, 5, 6, 5, torch.bfloat16, False, exact=False, chunk_pixels=1, pixel_splits=splits,
-                      routes=(1, 3) if splits == 4 else None)
+    _, enc = run_case(ctx_tc, spec, 5, 6, 5, torch.bfloat16, False, exact=False, chunk_pixels=1, pixel_splits=splits)
     assert enc.layout.pixel_splits == splits
 
 
@@ -208,10 +206,10 @@ def test_four_splits_per_channel_codebook_and_high_rate(ctx_tc):
     spec = fm.LayerSpec(64, 14, 14, 0.9, None, 5400)
     run_case(ctx_tc, spec, 4, 6, 3, torch.bfloat16, True, exact=False, chunk_pixels=1, pixel_splits=4, routes=(1, 3))
     run_case(ctx_tc, fm.LayerSpec(256, 14, 14, 0.9, None, 5401), 8, 6, 3, torch.bfloat16, False, exact=False,
-             chunk_pixels=1, pixel_splits=4, routes=(1, 3))
-    # quarters of 24 coefficients: the resident-basis kernels want multiples of 16
+             chunk_pixels=1, pixel_splits=4, routes=(1, 1))
+    # quarters of 24 coefficients: the tensor-core encoders want multiples of 16
     run_case(ctx_tc, fm.LayerSpec(96, 14, 14, 0.9, None, 5402), 4, 6, 3, torch.bfloat16, False, exact=False,
-             chunk_pixels=1, pixel_splits=4, routes=(2, 3))
+             chunk_pixels=1, pixel_splits=4, routes=(2, 1))
 
 
 # ---- PCA truncation: only the K leading components are coded (Section 4, ablation) -----------
@@ -266,7 +264,7 @@ def test_library_fit_with_int8_basis_matches_the_oracle(ctx_tc):
     spec = fm.LayerSpec(64, 14, 14, 0.9, None, 6300)
     params = fm.layer_params(spec)
     cal = fm.make_maps(params, 8, calib=True, dtype=torch.bfloat16)
-    want = oracle.fit_pca(cal, 5, basis_round="int8")
+    want = oracle.fit_pca(cal, 5, basis_round="int8", zero_level=True)
     model = tc.tc_fit_pca(ctx_tc, cal.cuda(), 5, basis_dtype=tc.binding.TC_INT8)
     got = tc.tc_model_export(model)
     assert got["basis_dtype"] == tc.binding.TC_INT8

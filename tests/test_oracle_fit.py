@@ -197,3 +197,64 @@ def test_lapack_step_agrees_with_jacobi_and_f32_rounding():
     assert np.abs(f.basis - a.basis).max() <= 2.0 ** -24
     m4 = oracle.with_bits(a, 4)
     assert m4.lo == a.lo and m4.step == pytest.approx(a.step * 63 / 15, rel=1e-14)
+
+
+# ---- quantiser grid with zero on a level (Section 3.1 "Quantization"; Appendix E) ----------------
+
+def test_zero_level_grid_hand_values():
+    # round(-lo / step) levels below zero, ties to even; the step is kept
+    assert oracle.zero_level_lo(-3.2, 1.0) == -3.0
+    assert oracle.zero_level_lo(-3.7, 1.0) == -4.0
+    assert oracle.zero_level_lo(-2.5, 1.0) == -2.0          # tie: two levels below zero
+    assert oracle.zero_level_lo(-3.5, 1.0) == -4.0          # tie: four
+    assert oracle.zero_level_lo(-0.26, 0.5) == -0.5
+    assert oracle.zero_level_lo(0.2, 1.0) == 0.0            # a range that starts above zero: zero becomes the lowest level
+    for lo, step in ((-1.2345, 0.071), (-17.0, 0.3), (-0.01, 2.0)):
+        got = oracle.zero_level_lo(lo, step)
+        assert abs(got - lo) <= 0.5 * step * (1 + 1e-12)
+        assert abs(got / step - np.rint(got / step)) < 1e-9
+
+
+def test_zero_level_fit_keeps_step_and_puts_zero_on_a_level():
+    spec = fm.LayerSpec(24, 10, 10, 0.8, None, 321)
+    x = fm.make_maps(fm.layer_params(spec), 12, calib=True).numpy()
+    raw = oracle.fit_pca(x, bits=4)
+    m = oracle.fit_pca(x, bits=4, zero_level=True)
+    assert m.zero_level and not raw.zero_level
+    assert m.step == raw.step and np.array_equal(m.basis, raw.basis) and np.array_equal(m.mean, raw.mean)
+    assert m.lo == oracle.zero_level_lo(raw.lo, raw.step)
+    assert m.cal_lo == raw.lo and m.cal_hi == pytest.approx(raw.lo + 15 * raw.step, rel=1e-14)
+    # a zero coefficient vector (the mean map) quantises to the zero level and reconstructs exactly
+    n_below = int(np.rint(-m.lo / m.step))
+    q0 = oracle.quantize(m, np.zeros((1, 24)))
+    assert np.all(q0 == n_below)
+    xhat = oracle.reconstruct(m, q0, (1, 24, 1, 1), out_bf16=False)
+    assert np.allclose(xhat.reshape(-1), m.mean.astype(np.float32), rtol=0, atol=1e-7)
+    # changing the bit width re-divides the measured range, then shifts again
+    m6 = oracle.with_bits(m, 6)
+    assert m6.step == pytest.approx((m.cal_hi - m.cal_lo) / 63, rel=1e-14)
+    assert m6.lo == oracle.zero_level_lo(m.cal_lo, m6.step)
+
+
+def test_zero_level_collapses_low_variance_channels_to_one_value():
+    # Appendix E: after the projection all values of a low-variance channel map to a single value.
+    # With zero between two levels such a channel flips between both; with zero on a level it
+    # does not, and both rate and distortion fall.
+    spec = fm.LayerSpec(48, 12, 12, 0.8, None, 322)
+    p = fm.layer_params(spec)
+    cal = fm.make_maps(p, 24, calib=True).numpy()
+    x = fm.make_maps(p, 6).numpy()
+    raw = oracle.fit_pca(cal, bits=3)
+    # pick a case where zero is clearly between two levels of the measured grid
+    frac = (-raw.lo / raw.step) % 1.0
+    assert 0.1 < frac < 0.9
+    m = oracle.fit_pca(cal, bits=3, zero_level=True)
+    out = {}
+    for name, mod in (("raw", raw), ("zero", m)):
+        q = oracle.quantize(mod, oracle.project(mod, x))
+        tail = q[:, 40:]
+        out[name] = dict(values=len(np.unique(tail)), entropy=oracle.entropy(oracle.histogram(q, 3, False)[0]),
+                         mse=oracle.mse(x, oracle.reconstruct(mod, q, x.shape, out_bf16=False)))
+    assert out["zero"]["values"] == 1
+    assert out["zero"]["entropy"] < out["raw"]["entropy"]
+    assert out["zero"]["mse"] < out["raw"]["mse"]
