@@ -10,19 +10,23 @@
 // the decoded symbols are then written into it one by one.
 //
 // One persistent block per SM.  Warp roles:
-//   warps 0-7, 8-15    two VLD groups, each with its own operand buffer (all K coefficients of a
-//                      tile of 128 pixels, K-major); where shared memory holds only one buffer
-//                      (C = K = 256) only group 0 works.  One or two threads per pixel walk the
-//                      pixel's chunks.
-//   warps 16-23        epilogue, all eight warps on every tile: TMEM -> registers,
+//   warps 0-7, 8-15    two VLD groups on alternating tiles of 128 pixels, each with its own operand
+//                      buffer (all K coefficients of the tile, K-major).  One or two threads per
+//                      pixel walk the pixel's chunks.
+//   warps 16-23        epilogue, all eight warps on every work item: TMEM -> registers,
 //                      x_hat = step * acc + bias, round to bf16, NCHW stores through warp-private
 //                      transpose blocks (the accumulator is held transposed: lane = channel)
 //   warp 24            one thread issues the tcgen05.mma of every tile:
 //                      D[c][pixel] = T[j][c] * (Q[pixel][j] - center)
-// The operand is handed over in panels of 32 coefficients: the MMA thread commits a barrier per
-// panel, and a VLD thread of the next tile that shares the buffer waits only for the panel it is
-// about to touch, so that the VLD of tile t + 1 follows the MMAs of tile t panel by panel.  The
-// accumulators are double-buffered in tensor memory, so the epilogue of tile t overlaps both.
+// The transposed basis is the A operand and lives in TENSOR memory, not in shared memory: each
+// block of 128 channels takes K / 2 columns (two bf16 per column), 256 columns at C = K = 256,
+// loaded once per block with tcgen05.st.  That leaves shared memory to the symbols -- two whole
+// tiles in flight, 128 KB at K = 256 -- and takes the basis off the MMA's shared-memory reads.
+// The other 256 columns hold two accumulators of 128 columns: one tile of 128 pixels up to 128
+// channels; with two channel blocks a work item is half a tile (2 x 64 columns), so that the
+// epilogue of one item overlaps the MMAs of the next.
+// The operand is handed back in panels of 32 coefficients: the MMA thread commits a barrier per
+// panel, and a VLD thread of the group's next tile waits only for the panel it is about to touch.
 //
 // A tile whose stream is dense (more than kDenseBits128 / 128 bits per symbol) gains nothing
 // from run skipping; its threads then decode symbol by symbol, eight symbols per 16-byte store.
@@ -34,10 +38,10 @@ namespace {
 using namespace tcdev;
 using namespace sm100;
 
-constexpr int kGroupWarps = 8;                                // warps of a VLD group; the epilogue's eight warps and the MMA warp follow
-__host__ __device__ constexpr int block_threads(int nbuf) { return (kGroupWarps * nbuf + 8 + 1) * 32; }
+constexpr int kGroupWarps = 8, kEpiWarp0 = 2 * kGroupWarps, kMmaWarp = kEpiWarp0 + 8;
+constexpr int kThreads = (kMmaWarp + 1) * 32;
 constexpr int kTmemCols = 512;
-constexpr int kAccCols = 256;
+constexpr int kAccBase = 256, kAccCols = 128;                 // two accumulators behind the basis columns
 constexpr int kPanelK = 32;                                   // coefficients per hand-over panel
 constexpr int kMaxPanels = 8;                                 // K <= 256
 constexpr uint32_t kRunGuard = 0x800u;                        // bit 11 set: at most 20 zero bits are skipped per step (20 + 12 <= 32: one refill per step)
@@ -47,36 +51,37 @@ constexpr int kDenseBits128 = 224;                            // tiles above 1.7
 // block's shared memory even for a corrupt stream (the buffers lie back to back).
 constexpr int kStreamSlack = 1024;
 constexpr int kTrWarpBytes = 1024;                            // epilogue transpose block of one warp: 32 channel rows x 16 pixels
+// Named barriers.  Hand-overs between warps that both run ordinary instructions use them instead
+// of mbarriers: the waiting side is parked by the hardware, whereas a warp polling an mbarrier
+// keeps issuing and takes issue slots from the warps that work.  (mbarriers remain where the
+// tensor core signals: accumulator ready, operand panel consumed.)
+constexpr int kBarGroup = 1;                                  // + group: the VLD threads of a group, once per tile
+constexpr int kBarFull = 3;                                   // + group: operand complete, VLD threads -> MMA warp
+constexpr int kBarAccFree = 5;                                // + accumulator: drained, epilogue warps -> MMA warp
+constexpr int kBarEpi = 7;                                    // accumulator ready, polling epilogue warp -> the other seven
 
 struct SmemLayout {
-    uint32_t basis, lut, vtab, opnd, tbuf, sbuf, total;
-    uint32_t opnd_bytes;                                      // one operand buffer
-    uint32_t stream_buf;                                      // bytes per staged stream buffer (two per group)
-    int nbuf;                                                 // operand buffers = working VLD groups (0: does not fit)
+    uint32_t lut, opnd, tbuf, sbuf, total;
+    uint32_t opnd_bytes;                                      // one operand buffer (one per VLD group)
+    uint32_t stream_buf;                                      // bytes per staged stream buffer (two per group; 0: does not fit)
 };
 
-__host__ __device__ inline SmemLayout smem_layout(int c, int k, int lut_entries, int budget)
+__host__ __device__ inline SmemLayout smem_layout(int k, int lut_entries, int budget)
 {
     SmemLayout l;
-    l.basis = 0;
-    const int c_pad = ((c + 127) / 128) * 128;                // the MMA takes 128 channels at a time
-    l.lut = (uint32_t)(((size_t)c_pad * k * 2 + 1023) & ~(size_t)1023);
-    l.vtab = l.lut + (uint32_t)lut_entries * 2;               // 16-bit entries: symbol << 8 | length
-    l.opnd = (l.vtab + 512 + 1023) & ~1023u;                  // 256 bf16 values: symbol - center
+    l.lut = 0;                                                // 32-bit entries: bf16(symbol - center) << 16 | length
+    l.opnd = ((uint32_t)lut_entries * 4u + 1023u) & ~1023u;
     l.opnd_bytes = (uint32_t)k * TC_TILE_PIXELS * 2;
-    l.nbuf = 0;
+    l.tbuf = l.opnd + 2u * l.opnd_bytes;
+    l.sbuf = l.tbuf + 8u * kTrWarpBytes;
     l.stream_buf = 0;
-    l.tbuf = l.sbuf = l.total = 0;
-    for (int nb = 2; nb >= 1 && l.nbuf == 0; --nb) {
-        const uint32_t tbuf = l.opnd + (uint32_t)nb * l.opnd_bytes;
-        const uint32_t sbuf = tbuf + 8u * kTrWarpBytes;
-        for (uint32_t kb = 16; kb >= 4; --kb)
-            if ((long long)sbuf + 2ll * nb * kb * 1024 + kStreamSlack <= (long long)budget) {
-                l.nbuf = nb; l.tbuf = tbuf; l.sbuf = sbuf; l.stream_buf = kb * 1024;
-                l.total = sbuf + 2u * nb * l.stream_buf + kStreamSlack;
-                break;
-            }
-    }
+    l.total = 0;
+    for (uint32_t kb = 16; kb >= 4; --kb)
+        if ((long long)l.sbuf + 4ll * kb * 1024 + kStreamSlack <= (long long)budget) {
+            l.stream_buf = kb * 1024;
+            l.total = l.sbuf + 4u * l.stream_buf + kStreamSlack;
+            break;
+        }
     return l;
 }
 
@@ -84,12 +89,6 @@ __device__ __forceinline__ uint32_t lds_u32(uint32_t addr)
 {
     uint32_t v;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
-    return v;
-}
-__device__ __forceinline__ uint32_t lds_u16(uint32_t addr)
-{
-    uint32_t v;
-    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(addr));
     return v;
 }
 __device__ __forceinline__ void sts_u16(uint32_t addr, uint32_t v)
@@ -179,26 +178,22 @@ struct BitReader {
     __device__ __forceinline__ uint32_t consumed() const { return words * 32u + (used & 0xffu) - start_bits; }
 };
 
-// kBufs: operand buffers = working VLD groups (the launch has no warps for a second group when
-// shared memory holds one buffer only, which leaves its threads more registers)
-template <bool kRelu, int kBufs>
-__global__ void __launch_bounds__(block_threads(kBufs), 1) decode_runs_kernel(DecodeArgs a)
+template <bool kRelu>
+__global__ void __launch_bounds__(kThreads, 1) decode_runs_kernel(DecodeArgs a)
 {
-    constexpr int kEpiWarp0 = kGroupWarps * kBufs, kMmaWarp = kEpiWarp0 + 8, kThreads = block_threads(kBufs);
     extern __shared__ __align__(128) unsigned char smem[];
-    __shared__ __align__(8) unsigned long long s_full[2], s_empty[2][kMaxPanels], s_tfull[2], s_tempty[2];
+    __shared__ __align__(8) unsigned long long s_empty[2][kMaxPanels], s_tfull[2];
     __shared__ uint32_t s_tmem_base;
     __shared__ unsigned int s_wsum[2][2][4];   // [group][thread set][warp]: bits per warp, for the start positions
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int lut_size = 1 << a.lut_bits;
-    const SmemLayout L = smem_layout(a.c, a.k, lut_size, a.smem_budget);
-    constexpr int nbuf = kBufs;
-    const uint32_t basis_addr = smem_u32(smem + L.basis);
+    const SmemLayout L = smem_layout(a.k, lut_size, a.smem_budget);
+    constexpr int nbuf = 2;
     const uint32_t lut_addr = smem_u32(smem + L.lut);
-    const uint32_t vtab_addr = smem_u32(smem + L.vtab);
     const uint32_t opnd_addr = smem_u32(smem + L.opnd);
-    const int n_panels = (a.k + kPanelK - 1) / kPanelK;
+    const int n_blocks = (a.c + 127) / 128;                    // blocks of 128 channels
+    const int items = n_blocks;                                // work items per tile: halves of 64 pixels with two channel blocks
     const int S = a.splits, cp = a.chunk_pixels;
     const int tpp = S >= 2 ? 2 : 1;                            // threads per pixel
     const int chunks_per_thread = S / tpp;                     // 1, or 2 with four chunks per pixel
@@ -208,36 +203,61 @@ __global__ void __launch_bounds__(block_threads(kBufs), 1) decode_runs_kernel(De
     // ---- set-up ---------------------------------------------------------------------
     if (tid == 0) {
         for (int g = 0; g < 2; ++g) {
-            mbar_init(smem_u32(&s_full[g]), (uint32_t)n_thr);
             for (int p = 0; p < kMaxPanels; ++p) mbar_init(smem_u32(&s_empty[g][p]), 1);
             mbar_init(smem_u32(&s_tfull[g]), 1);
-            mbar_init(smem_u32(&s_tempty[g]), 256);
         }
         mbar_fence_init();
     }
     if (warp == kMmaWarp) { tmem_alloc(smem_u32(&s_tmem_base), kTmemCols); tmem_relinquish(); }
     {
-        // transposed basis [c][j] -> K-major core matrices: (c/8)*sbo + (j/8)*128 + (c%8)*16 + (j%8)*2
-        const uint32_t sbo = (uint32_t)(a.k / 8) * 128u;
-        const int chunks_per_row = a.k / 8;
-        const uint4 *src = reinterpret_cast<const uint4 *>(a.basis_t_bf16);
-        const int c_pad = ((a.c + 127) / 128) * 128;         // rows past C are zero: their outputs are never stored
-        for (int i = tid; i < c_pad * chunks_per_row; i += kThreads) {
-            const int ch = i / chunks_per_row, j8 = i - ch * chunks_per_row;
-            cp_async_16(basis_addr + (ch >> 3) * sbo + j8 * 128 + (ch & 7) * 16, ch < a.c ? src + i : src, ch < a.c ? 16u : 0u);
+        // per-layer table: bf16(symbol - center) << 16 | code length
+        uint32_t *s_lut = reinterpret_cast<uint32_t *>(smem + L.lut);
+        for (int i = tid; i < lut_size; i += kThreads) {
+            const uint32_t e = a.lut32[i];
+            const float f = (float)((int)((e >> 8) & 0xffu) - a.center);
+            s_lut[i] = (__float_as_uint(f) & 0xffff0000u) | (e & 0xffu);
         }
-        cp_async_commit();
-        unsigned short *s_lut = reinterpret_cast<unsigned short *>(smem + L.lut);
-        for (int i = tid; i < lut_size; i += kThreads) s_lut[i] = a.lut[i];
-        unsigned short *s_vtab = reinterpret_cast<unsigned short *>(smem + L.vtab);
-        for (int i = tid; i < 256; i += kThreads) s_vtab[i] = (unsigned short)(__float_as_uint((float)(i - a.center)) >> 16);
     }
-    cp_async_wait<0>();
-    fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = s_tmem_base;
+    if (warp >= kEpiWarp0 && warp < kMmaWarp) {
+        // Transposed basis -> tensor memory: row c of block b (channel 128 b + c) goes to lane c,
+        // its K coefficients, two per 32-bit column in memory order, to columns b K/2 ... of the A
+        // operand.  A warp reaches the 32 lanes of its quarter; rows past C are zero (their outputs
+        // are never stored).
+        const int wq = warp & 3;
+        const uint32_t *src = reinterpret_cast<const uint32_t *>(a.basis_t_bf16);
+        for (int blk = (warp - kEpiWarp0) >> 2; blk < n_blocks; blk += 2) {
+            const int ch = blk * 128 + wq * 32 + lane;
+            const uint32_t *row = src + (size_t)(ch < a.c ? ch : 0) * (a.k / 2);
+            const uint32_t trow = tmem_base + ((uint32_t)(wq * 32) << 16) + (uint32_t)(blk * (a.k / 2));
+            for (int j = 0; j < a.k / 2; j += 16) {
+                if (a.k / 2 - j >= 16) {
+                    uint32_t r[16];
+#pragma unroll
+                    for (int i = 0; i < 16; i += 4) {
+                        const uint4 v = ch < a.c ? __ldg(reinterpret_cast<const uint4 *>(row + j + i)) : make_uint4(0u, 0u, 0u, 0u);
+                        r[i] = v.x; r[i + 1] = v.y; r[i + 2] = v.z; r[i + 3] = v.w;
+                    }
+                    tmem_st_32x32b_x16(trow + j, r);
+                } else {                                         // K % 32 == 16: eight columns left
+                    uint32_t r[8];
+#pragma unroll
+                    for (int i = 0; i < 8; i += 4) {
+                        const uint4 v = ch < a.c ? __ldg(reinterpret_cast<const uint4 *>(row + j + i)) : make_uint4(0u, 0u, 0u, 0u);
+                        r[i] = v.x; r[i + 1] = v.y; r[i + 2] = v.z; r[i + 3] = v.w;
+                    }
+                    tmem_st_32x32b_x8(trow + j, r);
+                }
+            }
+        }
+        tmem_st_wait();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
 
     const long long my_tiles = (a.n_tiles > blockIdx.x) ? (a.n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
 
@@ -258,9 +278,9 @@ __global__ void __launch_bounds__(block_threads(kBufs), 1) decode_runs_kernel(De
             const uint32_t opnd_g = opnd_addr + (uint32_t)grp * L.opnd_bytes;
             const uint32_t sbuf_bytes = L.stream_buf;
             const uint32_t sbuf_g = smem_u32(smem + L.sbuf) + (uint32_t)grp * 2u * sbuf_bytes;
-            const int bar_id = 1 + grp;
+            const int bar_id = kBarGroup + grp;
             const int lb = a.lut_bits;
-            const uint32_t modal2 = lds_u16(vtab_addr + (uint32_t)(a.modal < 0 ? a.center : a.modal) * 2u) * 0x00010001u;
+            const uint32_t modal2 = (__float_as_uint((float)((a.modal < 0 ? a.center : a.modal) - a.center)) >> 16) * 0x00010001u;   // two bf16 copies of the modal symbol's value
             bool alive = true;
 
             // offsets of a tile, validated; a tile that cannot be valid decodes nothing.  `lens`
@@ -382,9 +402,9 @@ __global__ void __launch_bounds__(block_threads(kBufs), 1) decode_runs_kernel(De
                                     r.take(n);
                                     pos += (int)n;
                                     const bool sym = pos < ke;             // a symbol follows the run
-                                    const uint32_t e = lds_u16(lut_addr + (r.hi >> (32 - lb)) * 2u);
-                                    r.take(sym ? e : 0u);
-                                    const uint32_t v = lds_u16(vtab_addr + (e >> 8) * 2u);
+                                    const uint32_t e = lds_u32(lut_addr + (r.hi >> (32 - lb)) * 4u);
+                                    r.take(sym ? (e & 0xffu) : 0u);
+                                    const uint32_t v = e >> 16;
                                     while (__any_sync(0xffffffffu, sym && pos >= ready * kPanelK)) prepare(ready++);
                                     if (sym) sts_u16(row_addr + ((uint32_t)pos >> 3) * 2048u + ((uint32_t)pos & 7u) * 2u, v);
                                     pos += sym ? 1 : 0;
@@ -396,11 +416,11 @@ __global__ void __launch_bounds__(block_threads(kBufs), 1) decode_runs_kernel(De
 #pragma unroll
                                     for (int i = 0; i < 4; ++i) {
                                         r.refill();
-                                        const uint32_t e0 = lds_u16(lut_addr + (r.hi >> (32 - lb)) * 2u);
-                                        r.take(decode ? e0 : 0u);
-                                        const uint32_t e1 = lds_u16(lut_addr + (r.hi >> (32 - lb)) * 2u);
-                                        r.take(decode ? e1 : 0u);
-                                        pk[i] = lds_u16(vtab_addr + (e0 >> 8) * 2u) | (lds_u16(vtab_addr + (e1 >> 8) * 2u) << 16);
+                                        const uint32_t e0 = lds_u32(lut_addr + (r.hi >> (32 - lb)) * 4u);
+                                        r.take(decode ? (e0 & 0xffu) : 0u);
+                                        const uint32_t e1 = lds_u32(lut_addr + (r.hi >> (32 - lb)) * 4u);
+                                        r.take(decode ? (e1 & 0xffu) : 0u);
+                                        pk[i] = __byte_perm(e0, e1, 0x7632);
                                     }
                                     if (decode) sts_v4(row_addr + (uint32_t)(k0 >> 3) * 2048u, pk[0], pk[1], pk[2], pk[3]);
                                 }
@@ -429,7 +449,7 @@ __global__ void __launch_bounds__(block_threads(kBufs), 1) decode_runs_kernel(De
                     decode_tile(r);
                 }
                 // (the issuing thread makes the operand visible to the tensor core's proxy)
-                mbar_arrive(smem_u32(&s_full[grp]));
+                named_bar_arrive(kBarFull + grp, n_thr + 32);
                 if (bad) tc_dev_set_status(a.status, TC_ERR_CORRUPT_STREAM);
                 cur = nxt;
                 nxt = after;
@@ -438,15 +458,16 @@ __global__ void __launch_bounds__(block_threads(kBufs), 1) decode_runs_kernel(De
             if (!alive) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
         }
     } else if (warp < kMmaWarp) {
-        // ================= epilogue: all eight warps work on every tile =================
-        // A thread owns one channel (its TMEM lane) of one block of 128 channels.  With two
-        // channel blocks warps 16-19 take the first and warps 20-23 the second; with one block
-        // the two warp sets split the tile's pixels (TMEM columns) in halves.
+        // ================= epilogue: all eight warps work on every item =================
+        // A thread owns one channel (its TMEM lane) of one block of 128 channels and 64 pixels of
+        // the item.  With two channel blocks an item is half a tile: warps 16-19 take the first
+        // block and warps 20-23 the second; with one block an item is a tile and the two warp sets
+        // split its pixels (TMEM columns) in halves.
         const int set = (warp - kEpiWarp0) >> 2;
         const int wq = warp & 3;                            // TMEM lane quarter of this warp
-        const int n_blocks = (a.c + 127) / 128;
         const int blk = n_blocks == 2 ? set : 0;
-        const int col_first = n_blocks == 2 ? 0 : 64 * set, col_count = n_blocks == 2 ? 128 : 64;
+        const int col_first = n_blocks == 2 ? 0 : 64 * set;
+        constexpr int col_count = 64;
         const int ch = blk * 128 + wq * 32 + lane;
         const bool ch_ok = ch < a.c;
         const float step = (float)(a.step * a.basis_scale);        // the operand holds basis / basis_scale
@@ -471,15 +492,24 @@ __global__ void __launch_bounds__(block_threads(kBufs), 1) decode_runs_kernel(De
             return *reinterpret_cast<const uint32_t *>(&h);
         };
         bool alive = true;
-        for (long long tl = 0; tl < my_tiles && alive; ++tl) {
-            const int acc = (int)(tl & 1);
+        const long long n_items = my_tiles * items;
+        // (after a wait that ran out the warps keep walking the items: the MMA warp waits for their arrivals)
+        for (long long it = 0; it < n_items; ++it) {
+            const int acc = (int)(it & 1);
+            const long long tl = items == 2 ? (it >> 1) : it;
+            const int item = items == 2 ? (int)(it & 1) : 0;
             const long long tile = blockIdx.x + tl * gridDim.x;
-            const long long p_first = tile * TC_TILE_PIXELS + col_first;
+            const long long p_first = tile * TC_TILE_PIXELS + item * 64 + col_first;
             const long long left = a.pixels - p_first;                       // pixels from this thread's first column on
             const int n_valid = (int)(left < (long long)col_count ? (left < 0 ? 0 : left) : (long long)col_count);
-            if (!mbar_wait(smem_u32(&s_tfull[acc]), (uint32_t)((tl >> 1) & 1), 1000u)) { alive = false; break; }
+            // the first epilogue warp waits for the accumulator and lets the others in
+            if (warp == kEpiWarp0) {
+                if (alive) alive = mbar_wait(smem_u32(&s_tfull[acc]), (uint32_t)((it >> 1) & 1), 100u);
+                tc_fence_before_sync();
+            }
+            named_bar_sync(kBarEpi, 256);
             tc_fence_after_sync();
-            const uint32_t trow = tmem_base + acc * kAccCols + blk * 128 + ((uint32_t)(wq * 32) << 16) + col_first;
+            const uint32_t trow = tmem_base + kAccBase + acc * kAccCols + (n_blocks == 2 ? blk * 64 : 0) + ((uint32_t)(wq * 32) << 16) + col_first;
             if (vec) {
                 // position of this lane's pixel group (4 pixels) in the first pass
                 const long long pg = p_first + 4 * piece;
@@ -527,47 +557,52 @@ __global__ void __launch_bounds__(block_threads(kBufs), 1) decode_runs_kernel(De
                 }
             }
             tc_fence_before_sync();
-            mbar_arrive(smem_u32(&s_tempty[acc]));
+            named_bar_arrive(kBarAccFree + acc, 256 + 32);
         }
-        if (!alive && lane == 0 && wq == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
+        if (!alive && lane == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
     } else {
         // ================= MMA issuer =================
-        if (lane == 0) {
-            // A = transposed basis (128 channels per instruction), B = the decoded symbols of 128 pixels
-            const uint32_t idesc = make_idesc_bf16(128, TC_TILE_PIXELS, /*A K-major*/ false, /*B K-major*/ false);
-            const uint32_t a_sbo = (uint32_t)(a.k / 8) * 128u;
-            const int n_blocks = (a.c + 127) / 128;
-            bool alive = true;
-            for (long long tl = 0; tl < my_tiles && alive; ++tl) {
-                const int acc = (int)(tl & 1);
-                const int buf = nbuf == 2 ? (int)(tl & 1) : 0;
-                const long long use = nbuf == 2 ? (tl >> 1) : tl;     // how often the buffer was filled before
-                if (!mbar_wait(smem_u32(&s_tempty[acc]), (uint32_t)(((tl >> 1) & 1) ^ 1), 500u)) { alive = false; break; }
-                if (!mbar_wait(smem_u32(&s_full[buf]), (uint32_t)(use & 1), 200u)) { alive = false; break; }
-                // the operand was written with ordinary stores by threads that have arrived on the
-                // barrier: one proxy fence here, between that synchronisation and the MMA's
-                // operand reads, orders them for all writers
-                fence_proxy_async_smem();
+        // The whole warp walks the loop and waits on the barriers; lane 0 issues, through
+        // instructions that carry their own guard (no branch around an MMA).
+        // A = transposed basis in tensor memory (128 channels per instruction), B = the decoded
+        // symbols of the item's pixels (rows of the group's operand buffer).
+        const uint32_t issuer = lane == 0 ? 1u : 0u;
+        const int np = items == 2 ? 64 : TC_TILE_PIXELS;          // pixels per work item
+        const uint32_t idesc = make_idesc_bf16(128, np, /*A K-major*/ false, /*B K-major*/ false);
+        const uint32_t a_blk1 = (uint32_t)(a.k / 2);               // columns between the two channel blocks of the basis
+        const int n_k16 = a.k >> 4;
+        long long it = 0;                                         // work items issued so far
+        for (long long tl = 0; tl < my_tiles; ++tl) {
+            const int buf = (int)(tl & 1);
+            __syncwarp();
+            named_bar_sync(kBarFull + buf, n_thr + 32);               // the group's VLD threads have arrived
+            // the operand was written with ordinary stores by threads that have arrived on the
+            // barrier: one proxy fence here, between that synchronisation and the MMA's
+            // operand reads, orders them for all writers
+            fence_proxy_async_smem();
+            const uint64_t b_base = make_smem_desc(opnd_addr + (uint32_t)buf * L.opnd_bytes, 2048, 128);
+            const uint32_t b_hi = (uint32_t)(b_base >> 32);
+            for (int item = 0; item < items; ++item, ++it) {
+                const int acc = (int)(it & 1);
+                __syncwarp();
+                if (it >= 2) named_bar_sync(kBarAccFree + acc, 256 + 32);   // the epilogue has drained the accumulator
                 tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + acc * kAccCols;
-                const uint32_t opnd_b = opnd_addr + (uint32_t)buf * L.opnd_bytes;
-                uint32_t accumulate = 0;
-                for (int p = 0; p < n_panels; ++p) {
-                    const int k0 = p * kPanelK;
-                    const int nk16 = min(kPanelK, a.k - k0) >> 4;
-                    for (int q = 0; q < nk16; ++q) {
-                        const uint64_t bdesc = make_smem_desc(opnd_b + (uint32_t)((k0 + 16 * q) >> 3) * 2048u, 2048, 128);
-                        for (int blk = 0; blk < n_blocks; ++blk) {
-                            const uint64_t adesc = make_smem_desc(basis_addr + blk * 16 * a_sbo + ((k0 + 16 * q) >> 3) * 128, 128, a_sbo);
-                            mma_bf16_ss(d_tmem + blk * 128, adesc, bdesc, idesc, accumulate);
-                        }
-                        accumulate = 1u;
-                    }
-                    mma_commit(smem_u32(&s_empty[buf][p]));      // the panel goes back to the VLD threads
+                const uint32_t d_tmem = tmem_base + kAccBase + acc * kAccCols;
+                // rows 64 item ... of the buffer: eight-row groups are 128 bytes apart; a step of 16
+                // coefficients moves the start address on by two core-matrix columns of 2048 bytes
+                uint32_t b_lo = (uint32_t)b_base + (uint32_t)item * (1024u >> 4);
+                uint32_t a_col = tmem_base;
+                const bool last = item == items - 1;
+                for (int q = 0; q < n_k16; ++q) {
+                    mma_bf16_ts_guarded(d_tmem, a_col, b_lo, b_hi, idesc, q ? 1u : 0u, issuer);
+                    if (n_blocks == 2) mma_bf16_ts_guarded(d_tmem + 64, a_col + a_blk1, b_lo, b_hi, idesc, q ? 1u : 0u, issuer);
+                    // behind the tile's last item a finished panel goes back to the VLD threads
+                    if (last && ((q & 1) || q == n_k16 - 1)) mma_commit_guarded(smem_u32(&s_empty[buf][q >> 1]), issuer);
+                    b_lo += 4096u >> 4;
+                    a_col += 8;
                 }
-                mma_commit(smem_u32(&s_tfull[acc]));
+                mma_commit_guarded(smem_u32(&s_tfull[acc]), issuer);
             }
-            if (!alive) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
         }
     }
 
@@ -590,29 +625,27 @@ bool tc_decode_runs_supported(const tc_ctx *ctx, const DecodeArgs &a)
     if (a.lut_bits > TC_MAX_CODE_LEN) return false;
     if (a.chunk_pixels > 1 ? a.splits != 1 : (a.splits != 1 && a.splits != 2 && a.splits != 4)) return false;
     if (a.splits > 1 && (a.k % a.splits != 0 || (a.k / a.splits) % 8 != 0)) return false;
-    const SmemLayout l = smem_layout(a.c, a.k, 1 << a.lut_bits, ctx->max_smem_optin - 512);
-    return l.nbuf > 0;
+    return smem_layout(a.k, 1 << a.lut_bits, ctx->max_smem_optin - 512).stream_buf > 0;
 }
 
 // Bytes of a tile's stream segment this kernel stages in shared memory; longer segments are read
 // from global memory, word by word.
 size_t tc_decode_runs_staging_bytes(const tc_ctx *ctx, const DecodeArgs &a)
 {
-    return smem_layout(a.c, a.k, 1 << a.lut_bits, ctx->max_smem_optin - 512).stream_buf;
+    return smem_layout(a.k, 1 << a.lut_bits, ctx->max_smem_optin - 512).stream_buf;
 }
 
 tc_status tc_launch_decode_runs(const tc_ctx *ctx, const DecodeArgs &a, cudaStream_t s)
 {
     if (a.n_tiles <= 0) return TC_OK;
-    const SmemLayout l = smem_layout(a.c, a.k, 1 << a.lut_bits, ctx->max_smem_optin - 512);
-    if (l.nbuf == 0) return TC_ERR_UNSUPPORTED;
-    void (*kernel)(DecodeArgs) = l.nbuf == 2 ? (a.relu ? decode_runs_kernel<true, 2> : decode_runs_kernel<false, 2>)
-                                             : (a.relu ? decode_runs_kernel<true, 1> : decode_runs_kernel<false, 1>);
+    const SmemLayout l = smem_layout(a.k, 1 << a.lut_bits, ctx->max_smem_optin - 512);
+    if (l.stream_buf == 0) return TC_ERR_UNSUPPORTED;
+    void (*kernel)(DecodeArgs) = a.relu ? decode_runs_kernel<true> : decode_runs_kernel<false>;
     DecodeArgs args = a;
     args.smem_budget = ctx->max_smem_optin - 512;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.total) != cudaSuccess)
         return TC_ERR_CUDA;
     const unsigned int grid = (unsigned int)((a.n_tiles < ctx->sm_count) ? a.n_tiles : ctx->sm_count);
-    kernel<<<grid, block_threads(l.nbuf), l.total, s>>>(args);
+    kernel<<<grid, kThreads, l.total, s>>>(args);
     return cudaGetLastError() == cudaSuccess ? TC_OK : TC_ERR_CUDA;
 }
