@@ -16,7 +16,7 @@
 //   warps 16-23        epilogue, all eight warps on every work item: TMEM -> registers,
 //                      x_hat = step * acc + bias, round to bf16, NCHW stores through warp-private
 //                      transpose blocks (the accumulator is held transposed: lane = channel)
-//   warp 24            one thread issues the tcgen05.mma of every tile:
+//   warps 24, 25       one thread each issues the tcgen05.mma of its accumulator's work items:
 //                      D[c][pixel] = T[j][c] * (Q[pixel][j] - center)
 // The transposed basis is the A operand and lives in TENSOR memory, not in shared memory: each
 // block of 128 channels takes K / 2 columns (two bf16 per column), 256 columns at C = K = 256,
@@ -39,7 +39,7 @@ using namespace tcdev;
 using namespace sm100;
 
 constexpr int kGroupWarps = 8, kEpiWarp0 = 2 * kGroupWarps, kMmaWarp = kEpiWarp0 + 8;
-constexpr int kThreads = (kMmaWarp + 1) * 32;
+constexpr int kThreads = (kMmaWarp + 2) * 32;                  // two MMA warps, one per accumulator
 constexpr int kTmemCols = 512;
 constexpr int kAccBase = 256, kAccCols = 128;                 // two accumulators behind the basis columns
 constexpr int kPanelK = 32;                                   // coefficients per hand-over panel
@@ -113,8 +113,8 @@ struct BitReader {
     uint32_t hi, lo, ahead, used;
     uint32_t next_addr;               // shared: address of the word after `ahead`
     const uint32_t *next, *end;       // global
-    uint32_t start_bits;              // position init() was given, modulo 32, and the words fetched since
-    uint32_t words;
+    uint32_t origin;                  // shared: bit address (shared address * 8) init() was given; global: that position modulo 32
+    uint32_t words;                   // global: words the window has moved on by
 
     __device__ __forceinline__ uint32_t fetch()
     {
@@ -126,23 +126,24 @@ struct BitReader {
     // kShared: `base_addr` is the shared address of the segment; else `base` / `end_word` delimit it
     __device__ __forceinline__ void init(uint32_t base_addr, const uint32_t *base, const uint32_t *end_word, uint32_t bitpos)
     {
-        if constexpr (kShared) next_addr = base_addr + (bitpos >> 5) * 4u;
-        else { next = base + (bitpos >> 5); end = end_word; }
+        if constexpr (kShared) { next_addr = base_addr + (bitpos >> 5) * 4u; origin = next_addr * 8u + (bitpos & 31u); }
+        else { next = base + (bitpos >> 5); end = end_word; origin = bitpos & 31u; }
         const uint32_t w0 = fetch(), w1 = fetch();
         ahead = fetch();
         const uint32_t sh = bitpos & 31u;
         hi = __funnelshift_l(w1, w0, sh);
         lo = w1 << sh;
         used = sh;
-        start_bits = sh;
         words = 0;
     }
     __device__ __forceinline__ void idle()
     {
-        hi = lo = ahead = used = start_bits = words = 0;
+        hi = lo = ahead = used = origin = words = 0;
         next_addr = 0; next = end = nullptr;
     }
-    __device__ __forceinline__ void take(uint32_t entry)      // entry & 31 bits
+    // `entry`: a bit count below 32, or a table entry with the count in its low byte (what lies
+    // above only reaches bits of `used` that nothing reads)
+    __device__ __forceinline__ void take(uint32_t entry)
     {
         hi = __funnelshift_l(lo, hi, entry);
         lo = __funnelshift_l(0u, lo, entry);
@@ -163,10 +164,9 @@ struct BitReader {
                 "@p or.b32 %0, %0, t;\n\t"
                 "@p or.b32 %1, %1, u;\n\t"
                 "@p add.u32 %3, %3, -32;\n\t"
-                "@p add.u32 %5, %5, 1;\n\t"
                 "@p ld.shared.u32 %2, [%4];\n\t"
                 "@p add.u32 %4, %4, 4;\n\t}"
-                : "+r"(hi), "+r"(lo), "+r"(ahead), "+r"(used), "+r"(next_addr), "+r"(words));
+                : "+r"(hi), "+r"(lo), "+r"(ahead), "+r"(used), "+r"(next_addr));
         } else if (used & 32u) {
             hi |= __funnelshift_l(ahead, 0u, used);
             lo |= __funnelshift_l(0u, ahead, used);
@@ -175,7 +175,12 @@ struct BitReader {
             ++words;
         }
     }
-    __device__ __forceinline__ uint32_t consumed() const { return words * 32u + (used & 0xffu) - start_bits; }
+    // bits taken since init()
+    __device__ __forceinline__ uint32_t consumed() const
+    {
+        if constexpr (kShared) return (next_addr - 12u) * 8u + (used & 0xffu) - origin;   // the window starts three words behind next_addr
+        else return words * 32u + (used & 0xffu) - origin;
+    }
 };
 
 template <bool kRelu>
@@ -203,7 +208,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_runs_kernel(DecodeArgs a)
     // ---- set-up ---------------------------------------------------------------------
     if (tid == 0) {
         for (int g = 0; g < 2; ++g) {
-            for (int p = 0; p < kMaxPanels; ++p) mbar_init(smem_u32(&s_empty[g][p]), 1);
+            for (int p = 0; p < kMaxPanels; ++p) mbar_init(smem_u32(&s_empty[g][p]), (uint32_t)items);   // one commit per item of the tile
             mbar_init(smem_u32(&s_tfull[g]), 1);
         }
         mbar_fence_init();
@@ -280,6 +285,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_runs_kernel(DecodeArgs a)
             const uint32_t sbuf_g = smem_u32(smem + L.sbuf) + (uint32_t)grp * 2u * sbuf_bytes;
             const int bar_id = kBarGroup + grp;
             const int lb = a.lut_bits;
+            const int dense_head = (a.dense_head + 7) & ~7;    // leading coefficients decoded symbol by symbol
             const uint32_t modal2 = (__float_as_uint((float)((a.modal < 0 ? a.center : a.modal) - a.center)) >> 16) * 0x00010001u;   // two bf16 copies of the modal symbol's value
             bool alive = true;
 
@@ -383,47 +389,50 @@ __global__ void __launch_bounds__(kThreads, 1) decode_runs_kernel(DecodeArgs a)
                         const uint32_t row_addr = opnd_g + (row >> 3) * 128u + (row & 7u) * 16u;
                         int ready = p_first;           // panels [p_first, ready) of the warp's rows are handed back and filled
                         // waits for panel p to be handed back by the MMAs of the tile before, then fills this
-                        // thread's coefficients of it with the modal symbol (run mode)
-                        auto prepare = [&](int p) {
+                        // thread's coefficients of it from coefficient `from` on with the modal symbol
+                        auto prepare = [&](int p, int from) {
                             if (pp == 0 && alive) alive = mbar_wait(smem_u32(&s_empty[grp][p]), wait_parity, 200u);
-                            if (runs && owner) {
-                                const int g0 = max(p * (kPanelK / 8), k_first >> 3), g1 = min((p + 1) * (kPanelK / 8), k_last >> 3);
+                            if (owner) {
+                                const int g0 = max(p * (kPanelK / 8), max(k_first, from) >> 3), g1 = min((p + 1) * (kPanelK / 8), k_last >> 3);
                                 for (int g = g0; g < g1; ++g) sts_v4(row_addr + (uint32_t)g * 2048u, modal2, modal2, modal2, modal2);
                             }
                         };
                         for (int ci = 0; ci < (cp > 1 ? 1 : chunks_per_thread); ++ci) {
                             const int kf = cp > 1 ? 0 : k_first + ci * k_sub, ke = cp > 1 ? a.k : kf + k_sub;
-                            if (runs) {
-                                int pos = decode ? kf : ke;
-                                while (__any_sync(0xffffffffu, pos < ke)) {
-                                    r.refill();
-                                    // a run of the modal symbol is a run of zero bits: at most 20 per step
-                                    const uint32_t n = pos < ke ? min((uint32_t)__clz((int)(r.hi | kRunGuard)), (uint32_t)(ke - pos)) : 0u;
-                                    r.take(n);
-                                    pos += (int)n;
-                                    const bool sym = pos < ke;             // a symbol follows the run
-                                    const uint32_t e = lds_u32(lut_addr + (r.hi >> (32 - lb)) * 4u);
-                                    r.take(sym ? (e & 0xffu) : 0u);
-                                    const uint32_t v = e >> 16;
-                                    while (__any_sync(0xffffffffu, sym && pos >= ready * kPanelK)) prepare(ready++);
-                                    if (sym) sts_u16(row_addr + ((uint32_t)pos >> 3) * 2048u + ((uint32_t)pos & 7u) * 2u, v);
-                                    pos += sym ? 1 : 0;
-                                }
-                            } else {
-                                for (int k0 = kf; k0 < ke; k0 += 8) {
-                                    while (ready * kPanelK <= k0) prepare(ready++);
-                                    uint32_t pk[4];
+                            // the leading coefficients (and every coefficient of a dense tile) symbol by symbol,
+                            // eight symbols per 16-byte store; the rest run by run
+                            const int kd = runs ? min(max(dense_head, kf), ke) : ke;
+                            for (int k0 = kf; k0 < kd; k0 += 8) {
+                                while (ready * kPanelK <= k0) prepare(ready++, kd);
+                                uint32_t pk[4];
 #pragma unroll
-                                    for (int i = 0; i < 4; ++i) {
-                                        r.refill();
-                                        const uint32_t e0 = lds_u32(lut_addr + (r.hi >> (32 - lb)) * 4u);
-                                        r.take(decode ? (e0 & 0xffu) : 0u);
-                                        const uint32_t e1 = lds_u32(lut_addr + (r.hi >> (32 - lb)) * 4u);
-                                        r.take(decode ? (e1 & 0xffu) : 0u);
-                                        pk[i] = __byte_perm(e0, e1, 0x7632);
-                                    }
-                                    if (decode) sts_v4(row_addr + (uint32_t)(k0 >> 3) * 2048u, pk[0], pk[1], pk[2], pk[3]);
+                                for (int i = 0; i < 4; ++i) {
+                                    r.refill();
+                                    const uint32_t e0 = lds_u32(lut_addr + (r.hi >> (32 - lb)) * 4u);
+                                    r.take(decode ? e0 : 0u);
+                                    const uint32_t e1 = lds_u32(lut_addr + (r.hi >> (32 - lb)) * 4u);
+                                    r.take(decode ? e1 : 0u);
+                                    pk[i] = __byte_perm(e0, e1, 0x7632);
                                 }
+                                if (decode) sts_v4(row_addr + (uint32_t)(k0 >> 3) * 2048u, pk[0], pk[1], pk[2], pk[3]);
+                            }
+                            uint32_t pos = (uint32_t)kd, rem = decode ? (uint32_t)(ke - kd) : 0u;
+                            uint32_t ready_end = (uint32_t)(ready * kPanelK);
+                            while (__any_sync(0xffffffffu, rem != 0u)) {
+                                r.refill();
+                                // a run of the modal symbol is a run of zero bits: at most 20 per step
+                                const uint32_t n = min((uint32_t)__clz((int)(r.hi | kRunGuard)), rem);
+                                r.take(n);
+                                pos += n;
+                                rem -= n;
+                                const bool sym = rem != 0u;            // a symbol follows the run
+                                const uint32_t e = lds_u32(lut_addr + (r.hi >> (32 - lb)) * 4u);
+                                r.take(sym ? e : 0u);
+                                while (__any_sync(0xffffffffu, sym && pos >= ready_end)) { prepare(ready++, kd); ready_end += kPanelK; }
+                                // coefficient pos of the row: core-matrix column pos / 8 (2048 bytes apart), 2 bytes per coefficient inside
+                                if (sym) sts_u16(row_addr + pos * 2u + (pos >> 3) * 2032u, e >> 16);
+                                pos += sym ? 1u : 0u;
+                                rem -= sym ? 1u : 0u;
                             }
                             // a chunk of one pixel (or part of it) must end exactly where its length says
                             if (cp == 1) {
@@ -431,7 +440,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_runs_kernel(DecodeArgs a)
                                 if (active && r.consumed() != expect) bad = true;
                             }
                         }
-                        while (ready < p_last) prepare(ready++);
+                        while (ready < p_last) prepare(ready++, 0);
                     }
                     if (cp > 1 && active && r.consumed() != len0) bad = true;
                 };
@@ -449,7 +458,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_runs_kernel(DecodeArgs a)
                     decode_tile(r);
                 }
                 // (the issuing thread makes the operand visible to the tensor core's proxy)
-                named_bar_arrive(kBarFull + grp, n_thr + 32);
+                named_bar_arrive(kBarFull + grp, n_thr + 32 * items);
                 if (bad) tc_dev_set_status(a.status, TC_ERR_CORRUPT_STREAM);
                 cur = nxt;
                 nxt = after;
@@ -485,12 +494,28 @@ __global__ void __launch_bounds__(kThreads, 1) decode_runs_kernel(DecodeArgs a)
         const uint32_t tb_wr = tb + (uint32_t)lane * 32u;
         const int r_sub = lane >> 2, piece = lane & 3;      // read phase: channel row r_sub (+ 8, 16, 24), pixels 4 * piece ...
         const uint32_t tb_rd = tb + (uint32_t)r_sub * 32u + ((((uint32_t)piece >> 1) ^ ((uint32_t)(r_sub >> 2) & 1u)) << 4) + ((uint32_t)piece & 1u) * 8u;
+        // two accumulator values -> two bf16: x_hat = step * acc + bias (one packed fused multiply-add)
         auto convert = [&](uint32_t x0, uint32_t x1) {
-            float f0 = fmaf(__uint_as_float(x0), step, bias), f1 = fmaf(__uint_as_float(x1), step, bias);
+            float f0, f1;
+            asm("{\n\t.reg .b64 v, s, b;\n\t"
+                "mov.b64 v, {%2, %3};\n\t"
+                "mov.b64 s, {%4, %4};\n\t"
+                "mov.b64 b, {%5, %5};\n\t"
+                "fma.rn.f32x2 v, v, s, b;\n\t"
+                "mov.b64 {%0, %1}, v;\n\t}"
+                : "=f"(f0), "=f"(f1) : "r"(x0), "r"(x1), "f"(step), "f"(bias));
             if constexpr (kRelu) { f0 = fmaxf(f0, 0.f); f1 = fmaxf(f1, 0.f); }   // the layer's non-linearity, when it follows the decoder
             const __nv_bfloat162 h = __floats2bfloat162_rn(f0, f1);
             return *reinterpret_cast<const uint32_t *>(&h);
         };
+        // the four channel rows this lane stores in the read phase of a pass: offsets inside an image
+        int row_off[4];
+        bool row_ok[4];
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            row_ok[it] = ch_base + 8 * it + r_sub < a.c;
+            row_off[it] = (ch_base + 8 * it + r_sub) * a.hw;
+        }
         bool alive = true;
         const long long n_items = my_tiles * items;
         // (after a wait that ran out the warps keep walking the items: the MMA warp waits for their arrivals)
@@ -523,13 +548,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_runs_kernel(DecodeArgs a)
                     sts_v4(tb_wr + ((sw_wr ^ 1u) << 4), convert(r[8], r[9]), convert(r[10], r[11]), convert(r[12], r[13]), convert(r[14], r[15]));
                     __syncwarp();
                     const bool px_ok = c0 + 4 * piece < n_valid;
-                    __nv_bfloat16 *row_ptr = out + img * img_stride + (long long)(ch_base + r_sub) * a.hw + sp;
+                    __nv_bfloat16 *px_ptr = out + img * img_stride + sp;
 #pragma unroll
                     for (int it = 0; it < 4; ++it) {
                         uint32_t lo2, hi2;
                         asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(lo2), "=r"(hi2) : "r"(tb_rd + it * 256));
-                        if (px_ok && ch_base + 8 * it + r_sub < a.c)
-                            *reinterpret_cast<uint2 *>(row_ptr + (long long)(8 * it) * a.hw) = make_uint2(lo2, hi2);
+                        if (px_ok && row_ok[it]) *reinterpret_cast<uint2 *>(px_ptr + row_off[it]) = make_uint2(lo2, hi2);
                     }
                     sp += 16;
                     while (sp >= a.hw) { sp -= a.hw; ++img; }
@@ -561,48 +585,49 @@ __global__ void __launch_bounds__(kThreads, 1) decode_runs_kernel(DecodeArgs a)
         }
         if (!alive && lane == 0) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
     } else {
-        // ================= MMA issuer =================
-        // The whole warp walks the loop and waits on the barriers; lane 0 issues, through
-        // instructions that carry their own guard (no branch around an MMA).
+        // ================= MMA issuers =================
+        // Two warps, one per accumulator: with two channel blocks warp w issues item w (pixels 64 w ...)
+        // of every tile, with one block the tiles alternate between the warps.  An MMA leaves its
+        // issuing thread about every 64 cycles at best and an item is K / 16 of them per channel block,
+        // so one warp alone would be the slowest stage of the kernel.  The whole warp walks the loop
+        // and waits on the barriers; lane 0 issues, through instructions that carry their own guard
+        // (no branch around an MMA).
         // A = transposed basis in tensor memory (128 channels per instruction), B = the decoded
         // symbols of the item's pixels (rows of the group's operand buffer).
+        const int w = warp - kMmaWarp;
         const uint32_t issuer = lane == 0 ? 1u : 0u;
         const int np = items == 2 ? 64 : TC_TILE_PIXELS;          // pixels per work item
         const uint32_t idesc = make_idesc_bf16(128, np, /*A K-major*/ false, /*B K-major*/ false);
         const uint32_t a_blk1 = (uint32_t)(a.k / 2);               // columns between the two channel blocks of the basis
         const int n_k16 = a.k >> 4;
-        long long it = 0;                                         // work items issued so far
-        for (long long tl = 0; tl < my_tiles; ++tl) {
+        const uint32_t d_tmem = tmem_base + kAccBase + w * kAccCols;
+        for (long long tl = items == 2 ? 0 : w; tl < my_tiles; tl += items == 2 ? 1 : 2) {
             const int buf = (int)(tl & 1);
+            const long long it = items == 2 ? 2 * tl + w : tl;       // index of the work item: item it uses accumulator it % 2 = w
             __syncwarp();
-            named_bar_sync(kBarFull + buf, n_thr + 32);               // the group's VLD threads have arrived
+            named_bar_sync(kBarFull + buf, n_thr + 32 * items);       // the group's VLD threads have arrived
             // the operand was written with ordinary stores by threads that have arrived on the
             // barrier: one proxy fence here, between that synchronisation and the MMA's
             // operand reads, orders them for all writers
             fence_proxy_async_smem();
             const uint64_t b_base = make_smem_desc(opnd_addr + (uint32_t)buf * L.opnd_bytes, 2048, 128);
             const uint32_t b_hi = (uint32_t)(b_base >> 32);
-            for (int item = 0; item < items; ++item, ++it) {
-                const int acc = (int)(it & 1);
-                __syncwarp();
-                if (it >= 2) named_bar_sync(kBarAccFree + acc, 256 + 32);   // the epilogue has drained the accumulator
-                tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + kAccBase + acc * kAccCols;
-                // rows 64 item ... of the buffer: eight-row groups are 128 bytes apart; a step of 16
-                // coefficients moves the start address on by two core-matrix columns of 2048 bytes
-                uint32_t b_lo = (uint32_t)b_base + (uint32_t)item * (1024u >> 4);
-                uint32_t a_col = tmem_base;
-                const bool last = item == items - 1;
-                for (int q = 0; q < n_k16; ++q) {
-                    mma_bf16_ts_guarded(d_tmem, a_col, b_lo, b_hi, idesc, q ? 1u : 0u, issuer);
-                    if (n_blocks == 2) mma_bf16_ts_guarded(d_tmem + 64, a_col + a_blk1, b_lo, b_hi, idesc, q ? 1u : 0u, issuer);
-                    // behind the tile's last item a finished panel goes back to the VLD threads
-                    if (last && ((q & 1) || q == n_k16 - 1)) mma_commit_guarded(smem_u32(&s_empty[buf][q >> 1]), issuer);
-                    b_lo += 4096u >> 4;
-                    a_col += 8;
-                }
-                mma_commit_guarded(smem_u32(&s_tfull[acc]), issuer);
+            __syncwarp();
+            if (it >= 2) named_bar_sync(kBarAccFree + w, 256 + 32);   // the epilogue has drained the accumulator
+            tc_fence_after_sync();
+            // rows 64 w ... of the buffer (two blocks): eight-row groups are 128 bytes apart; a step of 16
+            // coefficients moves the start address on by two core-matrix columns of 2048 bytes
+            uint32_t b_lo = (uint32_t)b_base + (items == 2 ? (uint32_t)w * (1024u >> 4) : 0u);
+            uint32_t a_col = tmem_base;
+            for (int q = 0; q < n_k16; ++q) {
+                mma_bf16_ts_guarded(d_tmem, a_col, b_lo, b_hi, idesc, q ? 1u : 0u, issuer);
+                if (n_blocks == 2) mma_bf16_ts_guarded(d_tmem + 64, a_col + a_blk1, b_lo, b_hi, idesc, q ? 1u : 0u, issuer);
+                // a finished panel goes back to the VLD threads (when every item of the tile has read it)
+                if ((q & 1) || q == n_k16 - 1) mma_commit_guarded(smem_u32(&s_empty[buf][q >> 1]), issuer);
+                b_lo += 4096u >> 4;
+                a_col += 8;
             }
+            mma_commit_guarded(smem_u32(&s_tfull[w]), issuer);
         }
     }
 

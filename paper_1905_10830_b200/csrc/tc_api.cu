@@ -826,6 +826,12 @@ tc_status tc_decode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
     a.relu = (params && params->relu) ? 1 : 0;
     a.basis_t_map = m->has_basis_t_map ? &m->basis_t_map : nullptr;
     a.modal = cb->modal;
+    // Coefficient j has standard deviation sqrt(eig[j]) on the calibration data; where that exceeds
+    // about 0.45 steps more than a quarter of its symbols differ from the zero level and skipping
+    // runs of the zero level no longer pays: those leading coefficients are decoded symbol by symbol.
+    a.dense_head = 0;
+    while (a.dense_head < m->k && a.dense_head < (int)m->eig.size() && std::sqrt(std::max(0.0, m->eig[a.dense_head])) > 0.45 * m->step)
+        ++a.dense_head;
     // High-rate streams: a tile's segment that no longer fits the shared-memory staging of a
     // resident-basis decoder but still fits that of the streaming decoder is better served by the
     // latter (the former would read the stream from global memory word by word).  Only when
