@@ -113,6 +113,25 @@ struct SmemBitWriter {
     }
 };
 
+// Two coefficients at once: the multiply-add and the rounding add are packed (two fp32 lanes per
+// instruction, each lane rounded exactly as the scalar instruction rounds), the clamps are not.
+__device__ __forceinline__ void quantise_bits2(uint32_t acc0, uint32_t acc1, float inv_step, float bias0, float bias1, float vmax,
+                                               uint32_t &q0, uint32_t &q1)
+{
+    float v0, v1;
+    asm("{\n\t.reg .b64 v, s, b, m;\n\t"
+        "mov.b64 v, {%2, %3};\n\t"
+        "mov.b64 s, {%4, %4};\n\t"
+        "mov.b64 b, {%5, %6};\n\t"
+        "mov.b64 m, {%7, %7};\n\t"
+        "fma.rn.f32x2 v, v, s, b;\n\t"
+        "add.rn.f32x2 v, v, m;\n\t"
+        "mov.b64 {%0, %1}, v;\n\t}"
+        : "=f"(v0), "=f"(v1) : "r"(acc0), "r"(acc1), "f"(inv_step), "f"(bias0), "f"(bias1), "f"(kMagic));
+    q0 = __float_as_uint(fminf(fmaxf(v0, kMagic), vmax));
+    q1 = __float_as_uint(fminf(fmaxf(v1, kMagic), vmax));
+}
+
 // kPair (per-layer tables, b <= 4): the code tables are indexed by two neighbouring symbols at
 // once (q0 | q1 << b, at most 256 entries), which halves the lookups of both passes.
 template <bool kPerChannel, bool kDebug, bool kPair>
@@ -242,7 +261,11 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
         }
     } else if (warp == kMmaWarp) {
         // ================= MMA issuer =================
-        if (lane == 0) {
+        // The whole warp walks the loop and waits on the barriers; lane 0 issues, through instructions
+        // that carry their own guard (a branch taken by one lane around every MMA costs about 90
+        // cycles per instruction).
+        {
+            const uint32_t issuer = lane == 0 ? 1u : 0u;
             const uint32_t idesc = make_idesc_bf16(TC_TILE_PIXELS, a.k, /*A MN-major*/ true, /*B K-major*/ false);
             const uint32_t b_sbo = (uint32_t)(a.c / 8) * 128u;
             int it = 0;
@@ -261,13 +284,13 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
                     for (int q = 0; q < nk16; ++q) {
                         const uint64_t adesc = make_smem_desc(ring_addr + s * kStageBytes + q * 4096, 2048, 128);
                         const uint64_t bdesc = make_smem_desc(basis_addr + ((k0 + 16 * q) >> 3) * 128, 128, b_sbo);
-                        mma_bf16_ss(d_tmem, adesc, bdesc, idesc, (kp | q) != 0 ? 1u : 0u);
+                        mma_bf16_ss_guarded(d_tmem, adesc, bdesc, idesc, (kp | q) != 0 ? 1u : 0u, issuer);
                     }
-                    mma_commit(smem_u32(&s_empty[s]));
+                    mma_commit_guarded(smem_u32(&s_empty[s]), issuer);
                 }
-                if (alive) mma_commit(smem_u32(&s_tfull[acc]));
+                if (alive) mma_commit_guarded(smem_u32(&s_tfull[acc]), issuer);
             }
-            if (!alive) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
+            if (!alive && issuer) tc_dev_set_status(a.status, TC_ERR_TIMEOUT);
         }
     } else if (warp >= kStoreWarp0) {
         // ================= store warps =================
@@ -363,10 +386,13 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
                     for (int i = 0; i < 4; ++i) bias4[i] = *reinterpret_cast<const float4 *>(s_bias + col0 + blk * 16 + 4 * i);
                     const float *biasv = reinterpret_cast<const float *>(bias4);
                     tmem_ld_wait();
+                    uint32_t qv[16];
+#pragma unroll
+                    for (int i = 0; i < 16; i += 2) quantise_bits2(r[i], r[i + 1], inv_step, biasv[i], biasv[i + 1], vmax, qv[i], qv[i + 1]);
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
                         const int j = col0 + blk * 16 + i;
-                        const uint32_t vb = quantise_bits(r[i], inv_step, biasv[i], vmax);
+                        const uint32_t vb = qv[i];
                         if constexpr (kPerChannel) my_bits += __ldg(a.enc + j * nsym + (vb & 0xffu)) & 0xffu;
                         else if constexpr (!kPair) {
                             uint32_t l;

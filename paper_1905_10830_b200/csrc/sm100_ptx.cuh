@@ -293,6 +293,17 @@ __device__ __forceinline__ void mma_bf16_ts_guarded(uint32_t d_tmem, uint32_t a_
         ::"r"(d_tmem), "r"(a_tmem), "r"(b_desc_lo), "r"(b_desc_hi), "r"(idesc), "r"(accumulate), "r"(issue)
         : "memory");
 }
+__device__ __forceinline__ void mma_bf16_ss_guarded(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                    uint32_t accumulate, uint32_t issue)
+{
+    asm volatile(
+        "{\n\t.reg .pred p, g;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "setp.ne.b32 g, %5, 0;\n\t"
+        "@g tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(issue)
+        : "memory");
+}
 __device__ __forceinline__ void mma_commit_guarded(uint32_t bar, uint32_t issue)
 {
     asm volatile(
