@@ -34,8 +34,22 @@ from synth import featuremaps as fm
 
 METRIC = "raw_activation_GBps_encode_plus_decode"
 UNIT = "GB/s"
-# dram__bytes_read.sum + dram__bytes_write.sum per tensor value, one ncu capture per kernel
-NCU_DRAM_BYTES_PER_VALUE = {"encode": 2.130, "decode": 1.619}
+PROFILE_SUMMARY = os.path.join("profiles", "encode_decode_tc_kernels_cfg5_batch2048.md")
+
+
+def profiled_dram_bytes_per_value():
+    """DRAM bytes (read + write) per tensor value of the two kernels, read from the committed ncu
+    summary of the benchmark's kernels (row "DRAM bytes per value"); None when the file or the row
+    is missing.  Returns ({"encode": x, "decode": y}, source string)."""
+    path = os.path.join(ROOT, PROFILE_SUMMARY)
+    try:
+        for line in open(path):
+            cells = [c.strip() for c in line.strip().strip("|").split("|")]
+            if len(cells) >= 3 and cells[0].lower().startswith("dram bytes per value"):
+                return {"encode": float(cells[1]), "decode": float(cells[2])}, PROFILE_SUMMARY
+    except (OSError, ValueError):
+        pass
+    return None, None
 
 
 def measured_peaks():
@@ -101,12 +115,12 @@ class ClockSampler:
         return out
 
 
-def oracle_setup(spec, bits, calib_maps, sample_images, dtype):
+def oracle_setup(spec, bits, calib_maps, sample_images, dtype, offset=0):
     """Untimed: the oracle's own model and codebook, and the sample it will code."""
     import oracle
     params = fm.layer_params(spec)
     cal = fm.make_maps(params, calib_maps, calib=True, dtype=dtype)
-    x = fm.make_maps(params, sample_images, dtype=dtype)
+    x = fm.make_maps(params, sample_images, dtype=dtype, offset=offset)
     m = oracle.fit_pca(cal, bits, basis_round="bf16" if dtype == torch.bfloat16 else "f32", zero_level=True)
     q_cal = oracle.quantize(m, oracle.project(m, cal))
     lengths = oracle.huffman_lengths(oracle.histogram(q_cal, bits, False), 12)
@@ -130,29 +144,77 @@ def oracle_timed_pass(o):
                 gbs=raw_bytes / (t2 - t0) / 1e9, bits_per_value=s.total_bits / q.size)
 
 
+def _oracle_worker(conn, job):
+    """One process of the all-cores oracle leg: sets up its own oracle state (untimed), then codes
+    its share of the sample every time it is told to and reports (seconds, raw bytes, bits/value)."""
+    cfg, layer, bits, images, dtype_name, offset = job
+    torch.set_num_threads(1)
+    w = fm.workload(cfg)
+    o = oracle_setup(w.layers[layer], bits, 32, images, getattr(torch, dtype_name), offset=offset)
+    conn.send("ready")
+    while conn.recv() == "run":
+        res = oracle_timed_pass(o)
+        conn.send((res["seconds"], res["raw_bytes"], res["bits_per_value"]))
+
+
+class OracleAllCores:
+    """The oracle on every core this process may use (sched_getaffinity): one spawned process per
+    core, each coding images_total / cores images of the same layer.  A pass takes as long as its
+    slowest worker (set-up excluded, as for the single-core leg)."""
+
+    def __init__(self, cfg, layer, bits, images_total, dtype):
+        import multiprocessing as mp
+        ctx = mp.get_context("spawn")           # never fork a process that has touched the GPU
+        self.cores = len(os.sched_getaffinity(0))
+        self.per = max(1, images_total // self.cores)
+        self.images = self.per * self.cores
+        self.workers = []
+        for i in range(self.cores):
+            parent, child = ctx.Pipe()
+            proc = ctx.Process(target=_oracle_worker, args=(child, (cfg, layer, bits, self.per, str(dtype).split(".")[-1], i)),
+                               daemon=True)
+            proc.start()
+            self.workers.append((proc, parent))
+        for _, conn in self.workers:
+            conn.recv()
+
+    def timed_pass(self):
+        for _, conn in self.workers:
+            conn.send("run")
+        out = [conn.recv() for _, conn in self.workers]
+        seconds, raw = max(o[0] for o in out), sum(o[1] for o in out)
+        return dict(seconds=seconds, raw_bytes=raw, gbs=raw / seconds / 1e9, bits_per_value=out[0][2])
+
+    def close(self):
+        for proc, conn in self.workers:
+            conn.send("stop")
+        for proc, _ in self.workers:
+            proc.join(timeout=10)
+
+
 def run_reference(args, rank):
-    """Reference arm: the CPU oracle, as it stands, on a bounded sample per step."""
+    """Reference arm: the CPU oracle, as it stands, on all host cores, a bounded sample per step."""
     if rank != 0:
         return
     w = fm.workload(5)
     spec = w.layers[0]
-    sample = args.sample_images
+    pool = OracleAllCores(5, 0, args.bits, args.sample_images, w.dtype)
     times = []
     res = None
-    o = oracle_setup(spec, args.bits, 32, sample, w.dtype)
     for i in range(args.warmup + args.steps):
-        res = oracle_timed_pass(o)
+        res = pool.timed_pass()
         if i >= args.warmup:
             times.append(res["seconds"])
+    pool.close()
     total = sum(times)
     value = res["raw_bytes"] * len(times) / total / 1e9
+    sample = f"{pool.images} of {w.batch} images of {spec.name} ({res['raw_bytes'] / 1e6:.1f} MB raw) per step, one process per core"
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "bits": args.bits, "sample": f"{sample} of {w.batch} images per step"},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
-                         "sample": f"{sample} images of {spec.name} ({res['raw_bytes'] / 1e6:.1f} MB raw) per step"},
+        "config": {"workload": w.name, "bits": args.bits, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": pool.cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "bits_per_value": res["bits_per_value"],
     }
@@ -178,11 +240,13 @@ def main():
                     help="kernel selection for profiling (tc_force_exact_path): 0 default, 2 the kernels that stream the basis, "
                          "3 the symbol-by-symbol resident-basis decoder instead of the run-skipping one")
     ap.add_argument("--sample-images", type=int, default=0, help="images per oracle timing sample")
+    ap.add_argument("--sustained-seconds", type=float, default=2.0,
+                    help="length of the back-to-back run behind the `sustained` key (0 = skip)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     if args.sample_images <= 0:      # about 15 s of oracle work in our arm; short steps in the reference arm
-        args.sample_images = 512 if args.impl == "ours" else 128
+        args.sample_images = 2048 if args.impl == "ours" else 128
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     rank = int(os.environ.get("RANK", "0"))
@@ -213,8 +277,21 @@ def main():
     # ---- set-up (untimed): fit, statistics, codebook -- all through the library ---------
     ctx = tc.tc_create(local_rank)
     cal = fm.make_maps(params, w.calib_maps, calib=True, dtype=w.dtype, device=dev)
-    model = tc.tc_fit_pca(ctx, cal, bits=bits, k=args.k,
-                          basis_dtype=tc.binding.TC_INT8 if args.basis == "int8" else None)
+    basis_dtype = tc.binding.TC_INT8 if args.basis == "int8" else None
+    if world > 1:
+        # calibration maps spread over the ranks: every rank accumulates the running fit state of its
+        # own share, one all-reduce (NCCL) sums the states, every rank finishes the same model
+        first, count = sharding.shard_range(w.calib_maps, rank, world)
+        share = cal[first:first + count].contiguous()
+        state = tc.tc_fit_state_create(ctx, spec.c)
+        tc.tc_fit_state_update(ctx, state, share)
+        cnt, s1, s2 = tc.tc_fit_state_export(ctx, state)
+        cnt, s1, s2 = sharding.merge_fit_state(cnt, s1, s2, dev)
+        tc.tc_fit_state_import(ctx, state, cnt, s1, s2)
+        model = tc.tc_fit_state_finish(ctx, state, cal, bits, k=args.k, basis_dtype=basis_dtype)
+        state.close()
+    else:
+        model = tc.tc_fit_pca(ctx, cal, bits=bits, k=args.k, basis_dtype=basis_dtype)
     st = tc.tc_stats(ctx, model, None, cal, groups=1)
     cb = tc.tc_build_codebook(ctx, model, st.hist, groups=1)
     x = fm.make_maps(params, batch, dtype=w.dtype, device=dev, offset=rank)   # each rank its own maps
@@ -265,6 +342,24 @@ def main():
         dist.barrier()
     clocks = sampler.stop()
     total_ms = t_begin.elapsed_time(t_end)
+    # ---- sustained: the same step back to back for at least two seconds, clocks sampled meanwhile ----
+    sustained = None
+    if args.sustained_seconds > 0:
+        n_sus = max(args.steps, int(args.sustained_seconds * 1e3 / max(total_ms / args.steps, 1e-3)) + 1)
+        sus_sampler = ClockSampler(local_rank)
+        torch.cuda.synchronize()
+        sus_sampler.start()
+        s_begin, s_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s_begin.record()
+        for _ in range(n_sus):
+            step()
+        s_end.record()
+        torch.cuda.synchronize()
+        sus_clocks = sus_sampler.stop()
+        sus_ms = s_begin.elapsed_time(s_end)
+        sus_bytes, sus_ms = sharding.aggregate(raw_bytes * n_sus, sus_ms, dev)
+        sustained = {"seconds": sus_ms * 1e-3, "steps": n_sus, "ms_per_step": sus_ms / n_sus,
+                     "value": sus_bytes / (sus_ms * 1e-3) / 1e9, "unit": UNIT, "clocks": sus_clocks}
     enc_ms = [ev[i][0].elapsed_time(ev[i][1]) for i in range(args.steps)]
     dec_ms = [ev[i][1].elapsed_time(ev[i][2]) for i in range(args.steps)]
     if tc.tc_get_status(ctx) != 0:
@@ -313,13 +408,16 @@ def main():
     dom_ms = max(enc_avg, dec_avg)
     achieved = algo_bytes / (dom_ms * 1e-3) / 1e9
     values = x.numel()
-    # DRAM bytes (read + write) of the dominant kernel from the ncu capture of these kernels at
-    # batch 2048 (profiles/encode_decode_tc_kernels_cfg5_batch2048.md), scaled by the values a
-    # launch processes: every tile is read and written once, so traffic grows with the batch.
-    # Only quoted for the configuration the counters were taken on.
-    traffic = None
-    if args.workload == 5 and bits == 4 and args.k == 0 and args.basis == "bf16" and kernels == ("tcgen05", "tcgen05") and lay.pixel_splits == 2:
-        traffic = NCU_DRAM_BYTES_PER_VALUE[dominant] * values
+    # DRAM bytes (read + write) of the dominant kernel from the committed ncu summary of these
+    # kernels (a capture at batch 2048), scaled by the values a launch processes: every tile is read
+    # and written once, so traffic grows with the batch.  Only quoted for the configuration the
+    # counters were taken on.
+    traffic, traffic_source = None, None
+    per_value, src = profiled_dram_bytes_per_value()
+    if per_value and args.workload == 5 and bits == 4 and args.k == 0 and args.basis == "bf16" and args.route == 0 and \
+            kernels == ("tcgen05", "tcgen05") and lay.pixel_splits == 2:
+        traffic = per_value[dominant] * values
+        traffic_source = f"{src}: {per_value[dominant]} DRAM bytes per value at batch 2048, scaled to this launch"
     line = {
         "metric": METRIC,
         "value": job_bytes / (total_ms * 1e-3) / 1e9,
@@ -337,21 +435,31 @@ def main():
         "mse_sample": test_stats.mse,
         "roofline": {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "frac_of_nominal_8TBps": achieved / 8000.0, "peak_source": peak_src,
-                     "algorithmic_bytes_per_launch": algo_bytes, "traffic": traffic,
+                     "algorithmic_bytes_per_launch": algo_bytes, "traffic": traffic, "traffic_source": traffic_source,
+                     "target_frac_of_nominal_8TBps": 0.60,
                      "encode_frac": algo_bytes / (enc_avg * 1e-3) / 1e9 / peak,
                      "decode_frac": algo_bytes / (dec_avg * 1e-3) / 1e9 / peak},
         "gpu_launches": 2 * args.steps,
         "kernels": {"encode": kernels[0], "decode": kernels[1]},
         "clocks": clocks,
     }
+    if sustained is not None:
+        line["sustained"] = sustained
     if e2e is not None:
         line["e2e"] = e2e
     if not args.no_cpu_baseline and world == 1:
-        res = oracle_timed_pass(oracle_setup(spec, bits, 32, args.sample_images, w.dtype))
-        line["cpu_baseline"] = {"value": res["gbs"], "unit": UNIT, "cores": 1, "kind": "oracle",
-                                "sample": f"{args.sample_images} of {batch} images ({res['raw_bytes'] / 1e6:.1f} MB raw), "
-                                          f"{res['seconds']:.1f} s, oracle model fitted on 32 calibration maps",
-                                "bits_per_value": res["bits_per_value"]}
+        # the oracle, as it stands, on all host cores (one process per core) and on one core
+        pool = OracleAllCores(args.workload, args.layer, bits, args.sample_images, w.dtype)
+        allc = pool.timed_pass()
+        allc.update(cores=pool.cores, images=pool.images)
+        pool.close()
+        one = oracle_timed_pass(oracle_setup(spec, bits, 32, max(8, args.sample_images // 16), w.dtype))
+        line["cpu_baseline"] = {"value": allc["gbs"], "unit": UNIT, "cores": allc["cores"], "kind": "oracle",
+                                "sample": f"{allc['images']} of {batch} images ({allc['raw_bytes'] / 1e6:.1f} MB raw) over "
+                                          f"{allc['cores']} processes, {allc['seconds']:.1f} s, oracle model fitted on 32 calibration maps",
+                                "single_core": {"value": one["gbs"], "cores": 1,
+                                                "sample": f"{max(8, args.sample_images // 16)} images, {one['seconds']:.1f} s"},
+                                "bits_per_value": one["bits_per_value"]}
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()

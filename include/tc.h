@@ -256,6 +256,15 @@ typedef struct {
     int32_t relu;         /* tc_decode / tc_roundtrip_host only: non-zero applies the layer's
                              non-linearity after the inverse transform (Section 3.1),
                              x_hat = max(T^T y_hat + mu, 0), before rounding to the tensor type */
+    int32_t mean_tile_bytes; /* tc_decode only, a hint that changes speed, never results: the mean size
+                             of a tile's stream segment in bytes (stream length / n_tiles), 0 = not
+                             known.  It matters for per-channel code tables on layers of up to 256
+                             channels: the decoder that keeps the basis in shared memory stages
+                             segments of up to about 14 KB there and reads longer ones from global
+                             memory word by word, the decoder that streams the basis stages up to
+                             32 KB; told that the segments are long, tc_decode picks the second.
+                             tc_decode never infers the rate from `stream_bytes` (which may be the
+                             length of the stream or the capacity of its buffer).            */
 } tc_encode_params;
 
 typedef struct {

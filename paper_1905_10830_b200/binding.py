@@ -44,7 +44,7 @@ class _CodebookParams(C.Structure):
 
 
 class _EncodeParams(C.Structure):
-    _fields_ = [("chunk_pixels", C.c_int32), ("pixel_splits", C.c_int32), ("relu", C.c_int32)]
+    _fields_ = [("chunk_pixels", C.c_int32), ("pixel_splits", C.c_int32), ("relu", C.c_int32), ("mean_tile_bytes", C.c_int32)]
 
 
 class _StreamLayout(C.Structure):
@@ -458,7 +458,9 @@ def tc_decode(ctx: Context, model: Model, cb: Codebook, enc: EncodedStream, shap
     if out is None:
         out = torch.empty(shape, dtype=dtype, device=enc.words.device)
     t = _tensor(out)
-    p = _EncodeParams(enc.layout.chunk_pixels, enc.layout.pixel_splits, int(relu))
+    # a caller that knows the stream's length also knows the mean tile size: pass it on as the rate hint
+    hint = 0 if stream_bytes is None else min(2**31 - 1, stream_bytes // max(1, enc.layout.n_tiles))
+    p = _EncodeParams(enc.layout.chunk_pixels, enc.layout.pixel_splits, int(relu), int(hint))
     nbytes = enc.words.numel() if stream_bytes is None else stream_bytes
     _check(load_library().tc_decode(ctx.ptr, model.ptr, cb.ptr, enc.words.data_ptr(), nbytes,
                                     enc.chunk_len.data_ptr(), enc.tile_off.data_ptr(), C.byref(p), C.byref(t),

@@ -482,12 +482,9 @@ static int decode_wide_groups(const tc_ctx *ctx, const DecodeArgs &a)
     if (!a.basis_t_map || a.c > 256) return 1;
     const SmemLayout l2 = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, ctx->max_smem_optin - 2048, 2);
     if (!(l2.stages >= 2 && l2.staged)) return 1;
-    // A stream known to be dense (the caller gave its length, not the capacity of a worst-case
-    // buffer, and the average tile exceeds the two-group segment buffers) is better served by one
-    // group with a large segment buffer than by two that read it from global memory.
-    const unsigned long long worst_bits = (unsigned long long)a.n_tiles * TC_TILE_PIXELS * (unsigned long long)a.k * (unsigned long long)a.lut_bits;
-    const unsigned long long avg_tile_bytes = a.stream_bits / 8ull / (unsigned long long)a.n_tiles;
-    if (a.stream_bits < worst_bits && avg_tile_bytes > l2.seg_bytes) return 1;
+    // A stream the caller says is dense (mean tile size above the two-group segment buffers) is better
+    // served by one group with a large segment buffer than by two that read it from global memory.
+    if (a.mean_tile_bytes > 0 && (unsigned long long)a.mean_tile_bytes > l2.seg_bytes) return 1;
     return 2;
 }
 

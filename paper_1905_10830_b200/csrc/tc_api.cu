@@ -826,31 +826,25 @@ tc_status tc_decode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
     a.relu = (params && params->relu) ? 1 : 0;
     a.basis_t_map = m->has_basis_t_map ? &m->basis_t_map : nullptr;
     a.modal = cb->modal;
+    a.mean_tile_bytes = (params && params->mean_tile_bytes > 0) ? params->mean_tile_bytes : 0;
     // Coefficient j has standard deviation sqrt(eig[j]) on the calibration data; where that exceeds
     // about 0.45 steps more than a quarter of its symbols differ from the zero level and skipping
     // runs of the zero level no longer pays: those leading coefficients are decoded symbol by symbol.
     a.dense_head = 0;
     while (a.dense_head < m->k && a.dense_head < (int)m->eig.size() && std::sqrt(std::max(0.0, m->eig[a.dense_head])) > 0.45 * m->step)
         ++a.dense_head;
-    // High-rate streams: a tile's segment that no longer fits the shared-memory staging of a
-    // resident-basis decoder but still fits that of the streaming decoder is better served by the
-    // latter (the former would read the stream from global memory word by word).  Only when
-    // `stream_bytes` is a length: a caller that passes the capacity of a worst-case buffer says
-    // nothing about the rate.
-    const size_t worst = (size_t)a.n_tiles * TC_TILE_PIXELS * (size_t)a.k * (size_t)cb->max_len / 8;
-    const size_t avg_tile_bytes = (stream_bytes + (size_t)a.n_tiles - 1) / (size_t)a.n_tiles;
-    const bool rate_known = stream_bytes < worst;
+    // per-layer code table, up to 256 channels: the run-skipping decoder (it also takes dense tiles)
     if (ctx->force_exact == 0 && x_hat->dtype == TC_BF16 && tc_decode_runs_supported(ctx, a)) {
-        const bool dense = rate_known && avg_tile_bytes > tc_decode_runs_staging_bytes(ctx, a) &&
-                           tc_decode_wide_supported(ctx, a) && avg_tile_bytes <= tc_decode_wide_staging_bytes(ctx, a);
-        if (!dense) {
-            ctx->last_decode_path = 1;
-            return tc_launch_decode_runs(ctx, a, (cudaStream_t)cuda_stream);
-        }
+        ctx->last_decode_path = 1;
+        return tc_launch_decode_runs(ctx, a, (cudaStream_t)cuda_stream);
     }
     bool resident = (ctx->force_exact == 0 || ctx->force_exact == 3) && x_hat->dtype == TC_BF16 && tc_decode_tc_supported(ctx, a);
-    if (resident && tc_decode_wide_supported(ctx, a) && rate_known && avg_tile_bytes > tc_decode_tc_staging_bytes(ctx, a) &&
-        avg_tile_bytes <= tc_decode_wide_staging_bytes(ctx, a))
+    // High-rate streams (params->mean_tile_bytes): a tile's segment that no longer fits the shared-memory
+    // staging of the resident-basis decoder but still fits that of the streaming decoder is better
+    // served by the latter (the former would read the stream from global memory word by word).
+    const size_t hint = (params && params->mean_tile_bytes > 0) ? (size_t)params->mean_tile_bytes : 0;
+    if (resident && hint > tc_decode_tc_staging_bytes(ctx, a) && tc_decode_wide_supported(ctx, a) &&
+        hint <= tc_decode_wide_staging_bytes(ctx, a))
         resident = false;
     if (resident) {
         ctx->last_decode_path = 1;

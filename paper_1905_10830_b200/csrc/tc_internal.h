@@ -122,6 +122,7 @@ struct DecodeArgs {
     const float *dec_bias;              // [c]
     int center;                         // subtracted from every symbol before the MMA
     int modal;                          // per-layer table: the symbol whose code is the single bit 0, or -1 if no code has one bit
+    int mean_tile_bytes;                // caller's hint: mean size of a tile's stream segment, 0 = not known
     int dense_head;                     // run-skipping decoder: leading coefficients that are too often non-modal for run skipping to pay
     int relu;                           // x_hat = max(x_hat, 0) before it is rounded to the tensor type
     int smem_budget;                    // shared memory the tensor-core kernel may lay out (set by its launcher)

@@ -2,7 +2,7 @@
 table: bits/value, encode / decode / round-trip GB/s of raw activations, fraction of the HBM
 roofline, which kernels ran, and parity against the CPU oracle on a sample of each layer.
 
-    python -m paper_1905_10830_b200.report [--cfg 1 2 3 4 5] [--reps 5] [--out FILE]
+    python report.py [--cfg 1 2 3 4 5] [--reps 5] [--out FILE]
 
 The oracle (test infrastructure) is imported only for the parity columns; with --no-oracle the
 table has the throughput columns alone."""
@@ -16,7 +16,7 @@ import sys
 import numpy as np
 import torch
 
-ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 

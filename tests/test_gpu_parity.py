@@ -358,12 +358,13 @@ def test_streaming_kernels_on_narrow_layers(ctx_stream, c, s, n, bits, splits):
              chunk_pixels=1 if splits else 0, routes=(3, 3))
 
 
-def test_high_rate_stream_is_decoded_by_the_streaming_kernel(ctx_tc):
-    # 256 channels at 8 bits: a tile's segment (about 16 KB) exceeds what the resident-basis decoder
-    # stages in shared memory; told the stream's true length, tc_decode picks the streaming kernel,
-    # which stages it.  Both kernels must return the same tensor.
+def test_rate_hint_picks_the_decoder_for_per_channel_tables(ctx_tc):
+    # 256 channels at 8 bits with per-channel code tables: a tile's segment (about 16 KB) exceeds what
+    # the resident-basis decoder stages in shared memory; told the mean tile size (the binding derives
+    # it from the stream's length), tc_decode picks the streaming kernel, which stages it.  Without
+    # the hint the resident-basis decoder runs.  Both must return the same tensor.
     spec = fm.LayerSpec(256, 14, 14, 0.9, None, 6500)
-    o = H.oracle_side(spec, 8, 6, 8, torch.bfloat16, False)
+    o = H.oracle_side(spec, 8, 6, 8, torch.bfloat16, True)
     model = H.import_model(tc, ctx_tc, o["model"], torch.bfloat16)
     cb = tc.tc_codebook_import(ctx_tc, o["lengths"], 8)
     x = o["x"].cuda()
@@ -372,13 +373,14 @@ def test_high_rate_stream_is_decoded_by_the_streaming_kernel(ctx_tc):
     assert nbytes / enc.layout.n_tiles > 14336
     a = tc.tc_decode(ctx_tc, model, cb, enc, x.shape, torch.bfloat16, stream_bytes=nbytes)
     assert tc.tc_get_status(ctx_tc) == 0 and tc.tc_last_path(ctx_tc, True) == 3
-    b = tc.tc_decode(ctx_tc, model, cb, enc, x.shape, torch.bfloat16)            # buffer size as length: resident kernel
+    b = tc.tc_decode(ctx_tc, model, cb, enc, x.shape, torch.bfloat16)            # no hint: resident-basis kernel
     assert tc.tc_get_status(ctx_tc) == 0 and tc.tc_last_path(ctx_tc, True) == 1
     want = oracle.reconstruct(o["model"], enc.symbols.cpu().numpy(), x.shape, out_bf16=True)
+    expected = H.expected_output_flips(o["model"], enc.symbols.cpu().numpy())
     for got in (a.float().cpu().numpy(), b.float().cpu().numpy()):
         ulp = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(want), 1e-30))) - 7)
         assert np.all(np.abs(got - want) <= np.maximum(1e-3 * np.maximum(np.abs(want), o["model"].step), ulp))
-        assert (got == want).mean() >= 0.999
+        assert int((got != want).sum()) <= H.flip_allowance(expected)
     model.close(); cb.close()
 
 
