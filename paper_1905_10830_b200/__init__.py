@@ -10,3 +10,4 @@ from .binding import (  # noqa: F401
     tc_fold_forward, tc_fold_inverse,
     tc_get_status, tc_force_exact_path, tc_last_path, tc_host_huffman_lengths, tc_host_eigh, library_path, load_library,
 )
+from .pipeline import CodedLayer, calibrate_layer_by_layer, run_chain, code_layer  # noqa: F401,E402

@@ -453,13 +453,19 @@ def tc_encode_noalloc(ctx: Context, model: Model, cb: Codebook, x: torch.Tensor,
 
 
 def tc_decode(ctx: Context, model: Model, cb: Codebook, enc: EncodedStream, shape, dtype, *,
-              out: torch.Tensor | None = None, stream_bytes: int | None = None, relu: bool = False) -> torch.Tensor:
-    """Decode `enc`; `relu` applies the layer's non-linearity after the inverse transform."""
+              out: torch.Tensor | None = None, stream_bytes: int | None = None, relu: bool = False,
+              mean_tile_bytes: int | None = None) -> torch.Tensor:
+    """Decode `enc`; `relu` applies the layer's non-linearity after the inverse transform;
+    `mean_tile_bytes` is the rate hint of tc_encode_params (derived from `stream_bytes` when only
+    that is given)."""
     if out is None:
         out = torch.empty(shape, dtype=dtype, device=enc.words.device)
     t = _tensor(out)
     # a caller that knows the stream's length also knows the mean tile size: pass it on as the rate hint
-    hint = 0 if stream_bytes is None else min(2**31 - 1, stream_bytes // max(1, enc.layout.n_tiles))
+    if mean_tile_bytes is not None:
+        hint = mean_tile_bytes
+    else:
+        hint = 0 if stream_bytes is None else min(2**31 - 1, stream_bytes // max(1, enc.layout.n_tiles))
     p = _EncodeParams(enc.layout.chunk_pixels, enc.layout.pixel_splits, int(relu), int(hint))
     nbytes = enc.words.numel() if stream_bytes is None else stream_bytes
     _check(load_library().tc_decode(ctx.ptr, model.ptr, cb.ptr, enc.words.data_ptr(), nbytes,
