@@ -65,6 +65,11 @@ __global__ void __launch_bounds__(kThreads) encode_simt_kernel(EncodeArgs a)
     const double top = (double)(nsym - 1);
     unsigned int clamped = 0;
 
+    if (a.sym_in) {
+        // the symbols were computed by the one-thread-per-value projection kernel
+        if (valid)
+            for (int j = 0; j < a.k; ++j) s_q[j * kThreads + t] = a.sym_in[p * a.k + j];
+    } else
     for (int j0 = 0; j0 < a.k; j0 += RB) {
         __syncthreads();
         if constexpr (kFp32) {
@@ -316,6 +321,12 @@ __global__ void __launch_bounds__(kThreads) decode_simt_kernel(DecodeArgs a)
         }
     }
 
+    if (a.sym_out) {
+        // the reconstruction runs in the one-thread-per-value kernel
+        if (valid)
+            for (int j = 0; j < a.k; ++j) a.sym_out[p * a.k + j] = s_q[j * kThreads + t];
+        return;
+    }
     TOut *out = reinterpret_cast<TOut *>(a.xhat);
     long long obase = 0;
     if (valid) {

@@ -79,5 +79,5 @@ extern "C" tc_status tc_encode_noalloc(tc_ctx *ctx, const tc_model *m, const tc_
     // clears, on the stream, everything this call will read, then picks the same kernels as
     // tc_encode (tensor-core kernels with the basis resident or streamed, fp32, fp64).
     return tc_encode_with_scratch(ctx, m, cb, x, lay.chunk_pixels, lay.pixel_splits, stream_out, capacity, chunk_len, tile_off,
-                                  nullptr, scratch, s);
+                                  nullptr, scratch, /*no arena for symbols: the per-pixel exact kernels*/ nullptr, s);
 }

@@ -706,7 +706,7 @@ void tc_codebook_free(tc_codebook *cb)
 // it is cleared on the stream here, whoever owns it.
 tc_status tc_encode_with_scratch(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const tc_tensor *x, int chunk_pixels,
                                  int splits, void *stream_out, size_t capacity, uint16_t *chunk_len, uint64_t *tile_off,
-                                 const tc_debug_out *debug, void *scratch, cudaStream_t s)
+                                 const tc_debug_out *debug, void *scratch, uint8_t *sym_scratch, cudaStream_t s)
 {
     const long long pixels = (long long)x->n * x->h * x->w;
     const long long n_tiles = (pixels + TC_TILE_PIXELS - 1) / TC_TILE_PIXELS;
@@ -739,6 +739,13 @@ tc_status tc_encode_with_scratch(tc_ctx *ctx, const tc_model *m, const tc_codebo
         return tc_launch_encode_simt_fp32(ctx, a, s);
     }
     ctx->last_encode_path = 0;
+    if (sym_scratch && n_tiles < (long long)kExactParallelTilesPerSm * ctx->sm_count) {
+        // few pixels: projection and quantiser with one thread per (pixel, coefficient), then the
+        // entropy coder of the per-pixel kernel on those symbols -- same arithmetic, same results
+        tc_status st = tc_launch_project_quantise(a, x->dtype, sym_scratch, s);
+        if (st != TC_OK) return st;
+        a.sym_in = sym_scratch;
+    }
     return tc_launch_encode_simt(ctx, a, x->dtype, s);
 }
 
@@ -794,10 +801,13 @@ tc_status tc_encode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
         TC_CUDA(cudaMemsetAsync(tile_off, 0, sizeof(uint64_t), s));
         return TC_OK;
     }
-    const size_t scratch = kEncodeScratchHeader + (size_t)n_tiles * sizeof(unsigned long long);
+    const size_t lookback = (kEncodeScratchHeader + (size_t)n_tiles * sizeof(unsigned long long) + 255) & ~(size_t)255;
+    // small tensors on the exact kernels also park their symbols in the arena (P * K bytes)
+    const bool parallel_exact = n_tiles < (long long)kExactParallelTilesPerSm * ctx->sm_count;
+    const size_t scratch = lookback + (parallel_exact ? (size_t)pixels * m->k : 0);
     if ((st = ensure_scratch(ctx, scratch)) != TC_OK) return st;
     return tc_encode_with_scratch(ctx, m, cb, x, cs.cp, cs.splits, stream_out, capacity, chunk_len, tile_off, debug,
-                                  ctx->scratch, s);
+                                  ctx->scratch, parallel_exact ? (uint8_t *)ctx->scratch + lookback : nullptr, s);
 }
 
 tc_status tc_decode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const void *stream, size_t stream_bytes,
@@ -859,6 +869,14 @@ tc_status tc_decode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
         return tc_launch_decode_simt_fp32(ctx, a, (cudaStream_t)cuda_stream);
     }
     ctx->last_decode_path = 0;
+    if (a.n_tiles < (long long)kExactParallelTilesPerSm * ctx->sm_count) {
+        // few pixels: the per-pixel kernel only decodes the symbols (into the context's arena), the
+        // inverse transform runs with one thread per (pixel, channel) -- same arithmetic, same results
+        if ((st = ensure_scratch(ctx, (size_t)pixels * m->k)) != TC_OK) return st;
+        a.sym_out = (uint8_t *)ctx->scratch;
+        if ((st = tc_launch_decode_simt(ctx, a, x_hat->dtype, (cudaStream_t)cuda_stream)) != TC_OK) return st;
+        return tc_launch_reconstruct(a, x_hat->dtype, a.sym_out, (cudaStream_t)cuda_stream);
+    }
     return tc_launch_decode_simt(ctx, a, x_hat->dtype, (cudaStream_t)cuda_stream);
 }
 

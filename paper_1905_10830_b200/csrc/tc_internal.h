@@ -101,6 +101,7 @@ struct EncodeArgs {
     unsigned int *status;
     unsigned long long *clamped;      // nullable: counts coefficients outside the range
     int emit;                         // 0: symbols only (statistics mode)
+    const uint8_t *sym_in;            // exact kernels: non-null = the symbols [P][K] are given, skip the projection
 };
 
 struct DecodeArgs {
@@ -110,6 +111,7 @@ struct DecodeArgs {
     int splits;                         // chunks per pixel (1, 2 or 4)
     const unsigned long long *tile_off;
     const uint8_t *symbols;     // non-null: take symbols from here instead of the stream
+    uint8_t *sym_out;           // exact kernels: non-null = write the decoded symbols [P][K] there and stop
     int n, c, hw, k, bits, groups;
     long long pixels;
     long long n_tiles, n_chunks;
@@ -138,13 +140,17 @@ struct DecodeArgs {
 constexpr size_t kEncodeScratchHeader = 64;   // ticket counter, padded; the per-tile look-back words follow
 tc_status tc_encode_with_scratch(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const tc_tensor *x, int chunk_pixels,
                                  int splits, void *stream_out, size_t capacity, uint16_t *chunk_len, uint64_t *tile_off,
-                                 const tc_debug_out *debug, void *scratch, cudaStream_t s);
+                                 const tc_debug_out *debug, void *scratch, uint8_t *sym_scratch, cudaStream_t s);
+// tensors of fewer tiles than this many per SM take the one-thread-per-value exact kernels
+constexpr int kExactParallelTilesPerSm = 2;
 
 // ---- launchers (defined in the .cu files) ----------------------------------------------
 tc_status tc_launch_encode_simt(const tc_ctx *ctx, const EncodeArgs &a, int dtype, cudaStream_t s);
 tc_status tc_launch_decode_simt(const tc_ctx *ctx, const DecodeArgs &a, int dtype, cudaStream_t s);
 tc_status tc_launch_encode_simt_fp32(const tc_ctx *ctx, const EncodeArgs &a, cudaStream_t s);
 tc_status tc_launch_decode_simt_fp32(const tc_ctx *ctx, const DecodeArgs &a, cudaStream_t s);
+tc_status tc_launch_project_quantise(const EncodeArgs &a, int dtype, uint8_t *sym, cudaStream_t s);
+tc_status tc_launch_reconstruct(const DecodeArgs &a, int dtype, const uint8_t *sym, cudaStream_t s);
 bool tc_encode_tc_supported(const tc_ctx *ctx, const EncodeArgs &a);
 tc_status tc_launch_encode_tc(const tc_ctx *ctx, const EncodeArgs &a, cudaStream_t s);
 bool tc_decode_tc_supported(const tc_ctx *ctx, const DecodeArgs &a);
