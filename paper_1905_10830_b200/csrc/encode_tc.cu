@@ -134,7 +134,11 @@ __device__ __forceinline__ void quantise_bits2(uint32_t acc0, uint32_t acc1, flo
 
 // kPair (per-layer tables, b <= 4): the code tables are indexed by two neighbouring symbols at
 // once (q0 | q1 << b, at most 256 entries), which halves the lookups of both passes.
-template <bool kPerChannel, bool kDebug, bool kPair>
+// kHist (statistics, Section 3.1 "Variable length coding": the entropy needs the distribution of
+// the symbols): every symbol is also counted, per coefficient channel, into a.hist.  The lanes of
+// a warp hold one coefficient of 32 pixels; the symbol most of them hold (the zero level) is
+// counted once per warp from a ballot, the others one atomic each.
+template <bool kPerChannel, bool kDebug, bool kPair, bool kHist>
 __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -389,6 +393,28 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
                     uint32_t qv[16];
 #pragma unroll
                     for (int i = 0; i < 16; i += 2) quantise_bits2(r[i], r[i + 1], inv_step, biasv[i], biasv[i + 1], vmax, qv[i], qv[i + 1]);
+                    if constexpr (kHist) {
+                        const uint32_t modal_bits = kMagicBits + (uint32_t)a.hist_modal;
+                        unsigned int n_clamped = 0;
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const int j = col0 + blk * 16 + i;
+                            const bool other = valid && qv[i] != modal_bits;
+                            const unsigned int others = __ballot_sync(0xffffffffu, other);
+                            const unsigned int live = __ballot_sync(0xffffffffu, valid);
+                            if (lane == 0 && live != others)
+                                atomicAdd(a.hist + (size_t)j * nsym + a.hist_modal, (unsigned long long)__popc(live & ~others));
+                            if (other) atomicAdd(a.hist + (size_t)j * nsym + (qv[i] & 0xffu), 1ull);
+                            // outside the quantiser's range [lo, lo + (2^b - 1) step]
+                            const float u = fmaf(__uint_as_float(r[i]), inv_step, biasv[i]);
+                            n_clamped += (valid && (u < 0.f || u > (float)(nsym - 1))) ? 1u : 0u;
+                        }
+                        if (a.clamped) {
+#pragma unroll
+                            for (int d = 16; d > 0; d >>= 1) n_clamped += __shfl_xor_sync(0xffffffffu, n_clamped, d);
+                            if (lane == 0 && n_clamped) atomicAdd(a.clamped, (unsigned long long)n_clamped);
+                        }
+                    }
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
                         const int j = col0 + blk * 16 + i;
@@ -632,10 +658,12 @@ tc_status tc_launch_encode_tc(const tc_ctx *ctx, const EncodeArgs &a, cudaStream
     if (a.n_tiles <= 0) return TC_OK;
     const SmemLayout l = smem_layout(a.c, a.k, enc_table_entries(a));
     const bool per_channel = a.groups != 1, debug = a.dbg_coef || a.dbg_sym, pair = !per_channel && a.bits <= kPairMaxBits;
+    if (a.hist && (per_channel || debug)) return TC_ERR_UNSUPPORTED;      // statistics run with a per-layer table
     void (*kernel)(EncodeArgs) =
-        per_channel ? (debug ? encode_tc_kernel<true, true, false> : encode_tc_kernel<true, false, false>)
-        : pair      ? (debug ? encode_tc_kernel<false, true, true> : encode_tc_kernel<false, false, true>)
-                    : (debug ? encode_tc_kernel<false, true, false> : encode_tc_kernel<false, false, false>);
+        a.hist      ? (pair ? encode_tc_kernel<false, false, true, true> : encode_tc_kernel<false, false, false, true>)
+        : per_channel ? (debug ? encode_tc_kernel<true, true, false, false> : encode_tc_kernel<true, false, false, false>)
+        : pair      ? (debug ? encode_tc_kernel<false, true, true, false> : encode_tc_kernel<false, false, true, false>)
+                    : (debug ? encode_tc_kernel<false, true, false, false> : encode_tc_kernel<false, false, false, false>);
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)l.total) != cudaSuccess)
         return TC_ERR_CUDA;
     const unsigned int grid = (unsigned int)((a.n_tiles < ctx->sm_count) ? a.n_tiles : ctx->sm_count);

@@ -289,6 +289,7 @@ void tc_destroy(tc_ctx *ctx)
         if (ctx->ev_out[i]) cudaEventDestroy(ctx->ev_out[i]);
     }
     if (ctx->chunk_bits) cudaFreeHost(ctx->chunk_bits);
+    for (tc_codebook *cb : ctx->stats_cb) tc_codebook_free(cb);
     if (ctx->d_status) cudaFree(ctx->d_status);
     delete ctx;
 }
@@ -706,7 +707,8 @@ void tc_codebook_free(tc_codebook *cb)
 // it is cleared on the stream here, whoever owns it.
 tc_status tc_encode_with_scratch(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const tc_tensor *x, int chunk_pixels,
                                  int splits, void *stream_out, size_t capacity, uint16_t *chunk_len, uint64_t *tile_off,
-                                 const tc_debug_out *debug, void *scratch, uint8_t *sym_scratch, cudaStream_t s)
+                                 const tc_debug_out *debug, void *scratch, uint8_t *sym_scratch, cudaStream_t s,
+                                 unsigned long long *hist, unsigned long long *clamped)
 {
     const long long pixels = (long long)x->n * x->h * x->w;
     const long long n_tiles = (pixels + TC_TILE_PIXELS - 1) / TC_TILE_PIXELS;
@@ -723,9 +725,12 @@ tc_status tc_encode_with_scratch(tc_ctx *ctx, const tc_model *m, const tc_codebo
     a.dbg_sym = debug ? debug->symbols : nullptr;
     a.ticket = (unsigned int *)scratch;
     a.tile_state = (unsigned long long *)((char *)scratch + kEncodeScratchHeader);
-    a.status = ctx->d_status; a.clamped = nullptr; a.emit = 1;
+    a.status = ctx->d_status; a.clamped = clamped; a.emit = 1;
     a.basis_bf16 = m->d_basis_bf16; a.enc_bias = m->d_enc_bias; a.tmu32 = m->d_tmu32;
     a.basis_map = m->has_basis_map ? &m->basis_map : nullptr;
+    a.hist = hist; a.hist_modal = m->center;
+    if (hist && !((ctx->force_exact == 0 || ctx->force_exact == 3) && x->dtype == TC_BF16 && tc_encode_tc_supported(ctx, a)))
+        return TC_ERR_UNSUPPORTED;                      // only the resident-basis tensor-core encoder counts symbols
     if ((ctx->force_exact == 0 || ctx->force_exact == 3) && x->dtype == TC_BF16 && tc_encode_tc_supported(ctx, a)) {
         ctx->last_encode_path = 1;
         return tc_launch_encode_tc(ctx, a, s);
@@ -977,19 +982,88 @@ tc_status tc_roundtrip_host(tc_ctx *ctx, const tc_model *m, const tc_codebook *c
 
 // ---- statistics ---------------------------------------------------------------------------
 
-tc_status tc_stats(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const tc_tensor *x, tc_stats_out *out,
-                   void *cuda_stream)
+// Statistics of a bf16 tensor on the tensor-core kernels: the batch is worked through in chunks of
+// whole tiles; every chunk is encoded (the encoder counts its symbols per coefficient channel and
+// the coefficients outside the quantiser's range while it codes), decoded again, and compared with
+// the input.  The stream is coded with `cb` when that is a per-layer table, else with a
+// fixed-length code of the model's bit width.  Buffers live in the context's arena (grown on
+// demand, kept between calls).  Returns TC_ERR_UNSUPPORTED for shapes those kernels do not take.
+static tc_status stats_tensor_core(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const tc_tensor *x,
+                                   std::vector<unsigned long long> &hist, double &sq, unsigned long long &zeros,
+                                   unsigned long long &clamped, cudaStream_t s)
 {
-    if (!ctx || !m || !out || !valid_tensor(x)) return TC_ERR_INVALID_ARG;
-    if (x->c != m->c) return TC_ERR_INVALID_ARG;
-    if (x->dtype != m->basis_dtype && m->basis_dtype != TC_INT8) return TC_ERR_UNSUPPORTED;   // an 8-bit basis serves both tensor types
-    if (out->groups != 1 && out->groups != m->k) return TC_ERR_INVALID_ARG;
-    if (cb && (cb->bits != m->bits || (cb->groups != 1 && cb->groups != m->k))) return TC_ERR_INVALID_ARG;
+    if (x->dtype != TC_BF16 || ctx->force_exact == 1 || ctx->force_exact == 2) return TC_ERR_UNSUPPORTED;
+    if (m->c % 16 != 0 || m->k % 16 != 0 || m->k < 16 || m->c > 256 || (x->h * x->w) % 4 != 0 || ((uintptr_t)x->data & 7u) != 0)
+        return TC_ERR_UNSUPPORTED;
+    const int nsym = 1 << m->bits;
+    const tc_codebook *code = (cb && cb->groups == 1) ? cb : nullptr;
+    if (!code) {
+        if (!ctx->stats_cb[m->bits]) {
+            std::vector<uint8_t> lengths(nsym, (uint8_t)m->bits);
+            tc_status st = tc_codebook_import(ctx, m->bits, 1, lengths.data(), &ctx->stats_cb[m->bits]);
+            if (st != TC_OK) return st;
+        }
+        code = ctx->stats_cb[m->bits];
+    }
+    const int hw = x->h * x->w;
+    const size_t image_bytes = (size_t)m->c * hw * 2;
+    int unit = 1;                                   // images per chunk: whole tiles
+    while (((long long)unit * hw) % TC_TILE_PIXELS != 0) unit <<= 1;
+    long long chunk_n = std::max<long long>(1, (long long)((32ull << 20) / image_bytes));
+    chunk_n = std::max<long long>(unit, chunk_n / unit * unit);
+    if (chunk_n > x->n) chunk_n = x->n;
+    tc_tensor xc{x->data, (int32_t)chunk_n, x->c, x->h, x->w, x->dtype};
+    tc_stream_layout lay;
+    tc_status st = tc_encode_bound(m, code, &xc, nullptr, &lay);
+    if (st != TC_OK) return st;
+    auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+    const size_t hist_bytes = (size_t)m->k * nsym * sizeof(unsigned long long);
+    const size_t off_stream = up((size_t)chunk_n * image_bytes), off_chunk = off_stream + up(lay.stream_bytes),
+                 off_tile = off_chunk + up(lay.chunk_len_bytes), off_hist = off_tile + up(lay.tile_off_bytes),
+                 off_small = off_hist + up(hist_bytes), total = off_small + 64;
+    if (total > ctx->host_arena_bytes) {
+        if (ctx->host_arena) { TC_CUDA(cudaDeviceSynchronize()); cudaFree(ctx->host_arena); ctx->host_arena = nullptr; ctx->host_arena_bytes = 0; }
+        TC_CUDA(cudaMalloc(&ctx->host_arena, total));
+        ctx->host_arena_bytes = total;
+    }
+    char *base = (char *)ctx->host_arena;
+    unsigned long long *d_hist = (unsigned long long *)(base + off_hist);
+    double *d_sq = (double *)(base + off_small);
+    unsigned long long *d_zeros = (unsigned long long *)(base + off_small + 8), *d_clamped = (unsigned long long *)(base + off_small + 16);
+    TC_CUDA(cudaMemsetAsync(base + off_hist, 0, up(hist_bytes) + 64, s));
+    const long long tiles_max = ((long long)chunk_n * hw + TC_TILE_PIXELS - 1) / TC_TILE_PIXELS;
+    const size_t lookback = kEncodeScratchHeader + (size_t)tiles_max * sizeof(unsigned long long);
+    if ((st = ensure_scratch(ctx, lookback)) != TC_OK) return st;
+    tc_encode_params prm{lay.chunk_pixels, lay.pixel_splits, 0, 0};
+    for (long long first = 0; first < x->n; first += chunk_n) {
+        const int32_t cn = (int32_t)std::min<long long>(chunk_n, x->n - first);
+        tc_tensor xi{(char *)x->data + (size_t)first * image_bytes, cn, x->c, x->h, x->w, x->dtype};
+        tc_tensor xh{base, cn, x->c, x->h, x->w, x->dtype};
+        st = tc_encode_with_scratch(ctx, m, code, &xi, lay.chunk_pixels, lay.pixel_splits, base + off_stream, lay.stream_bytes,
+                                    (uint16_t *)(base + off_chunk), (uint64_t *)(base + off_tile), nullptr, ctx->scratch, nullptr, s,
+                                    d_hist, d_clamped);
+        if (st != TC_OK) return st;
+        st = tc_decode(ctx, m, code, base + off_stream, lay.stream_bytes, (const uint16_t *)(base + off_chunk),
+                       (const uint64_t *)(base + off_tile), &prm, &xh, s);
+        if (st != TC_OK) return st;
+        if ((st = tc_launch_sqerr(xi.data, xh.data, x->dtype, (long long)cn * m->c * hw, d_sq, d_zeros, s)) != TC_OK) return st;
+    }
+    hist.assign((size_t)m->k * nsym, 0ull);
+    TC_CUDA(cudaMemcpyAsync(hist.data(), d_hist, hist_bytes, cudaMemcpyDeviceToHost, s));
+    TC_CUDA(cudaMemcpyAsync(&sq, d_sq, 8, cudaMemcpyDeviceToHost, s));
+    TC_CUDA(cudaMemcpyAsync(&zeros, d_zeros, 8, cudaMemcpyDeviceToHost, s));
+    TC_CUDA(cudaMemcpyAsync(&clamped, d_clamped, 8, cudaMemcpyDeviceToHost, s));
+    TC_CUDA(cudaStreamSynchronize(s));
+    return TC_OK;
+}
+
+// The same on the fp64 kernels: project + quantise (symbols to memory), histogram, reconstruct,
+// squared error; the buffers (P * K + V * element bytes) are allocated for the call.
+static tc_status stats_exact(tc_ctx *ctx, const tc_model *m, const tc_tensor *x, std::vector<unsigned long long> &hist_out,
+                             double &sq, unsigned long long &zeros, unsigned long long &clamped, cudaStream_t s)
+{
     const long long pixels = (long long)x->n * x->h * x->w;
-    if (pixels == 0) return TC_ERR_INVALID_ARG;
-    DeviceGuard guard(ctx->device);
-    cudaStream_t s = (cudaStream_t)cuda_stream;
-    const int nsym = 1 << m->bits, groups = out->groups;
+    const int nsym = 1 << m->bits;
     const size_t elem = (x->dtype == TC_F32) ? 4 : 2;
     const size_t values = (size_t)pixels * m->c, symbols = (size_t)pixels * m->k;
     const size_t hist_bytes = (size_t)m->k * nsym * sizeof(unsigned long long);
@@ -1028,14 +1102,38 @@ tc_status tc_stats(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const 
     if ((st = tc_launch_decode_simt(ctx, d, x->dtype, s)) != TC_OK) return st;
     if ((st = tc_launch_sqerr(x->data, d_xhat, x->dtype, (long long)values, d_sq, d_zeros, s)) != TC_OK) return st;
 
-    std::vector<unsigned long long> hist((size_t)m->k * nsym);
-    double sq = 0.0;
-    unsigned long long zeros = 0, clamped = 0;
-    TC_CUDA(cudaMemcpyAsync(hist.data(), d_hist, hist_bytes, cudaMemcpyDeviceToHost, s));
+    hist_out.assign((size_t)m->k * nsym, 0ull);
+    TC_CUDA(cudaMemcpyAsync(hist_out.data(), d_hist, hist_bytes, cudaMemcpyDeviceToHost, s));
     TC_CUDA(cudaMemcpyAsync(&sq, d_sq, 8, cudaMemcpyDeviceToHost, s));
     TC_CUDA(cudaMemcpyAsync(&zeros, d_zeros, 8, cudaMemcpyDeviceToHost, s));
     TC_CUDA(cudaMemcpyAsync(&clamped, d_clamped, 8, cudaMemcpyDeviceToHost, s));
     TC_CUDA(cudaStreamSynchronize(s));
+    return TC_OK;
+}
+
+tc_status tc_stats(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const tc_tensor *x, tc_stats_out *out,
+                   void *cuda_stream)
+{
+    if (!ctx || !m || !out || !valid_tensor(x)) return TC_ERR_INVALID_ARG;
+    if (x->c != m->c) return TC_ERR_INVALID_ARG;
+    if (x->dtype != m->basis_dtype && m->basis_dtype != TC_INT8) return TC_ERR_UNSUPPORTED;   // an 8-bit basis serves both tensor types
+    if (out->groups != 1 && out->groups != m->k) return TC_ERR_INVALID_ARG;
+    if (cb && (cb->bits != m->bits || (cb->groups != 1 && cb->groups != m->k))) return TC_ERR_INVALID_ARG;
+    const long long pixels = (long long)x->n * x->h * x->w;
+    if (pixels == 0) return TC_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const int nsym = 1 << m->bits, groups = out->groups;
+    const size_t values = (size_t)pixels * m->c, symbols = (size_t)pixels * m->k;
+
+    std::vector<unsigned long long> hist;
+    double sq = 0.0;
+    unsigned long long zeros = 0, clamped = 0;
+    // bf16 tensors of up to 256 channels: the tensor-core kernels, which count while they code;
+    // everything else: the fp64 kernels
+    tc_status st = stats_tensor_core(ctx, m, cb, x, hist, sq, zeros, clamped, s);
+    if (st == TC_ERR_UNSUPPORTED) st = stats_exact(ctx, m, x, hist, sq, zeros, clamped, s);
+    if (st != TC_OK) return st;
 
     // fold the per-channel counts to the requested granularity
     std::vector<unsigned long long> folded((size_t)groups * nsym, 0ull);

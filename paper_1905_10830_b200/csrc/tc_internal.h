@@ -39,6 +39,7 @@ struct tc_ctx {
     int force_exact = 0;                  // 1: route every tensor through the fp64 kernels; 2: skip the resident-basis kernels; 3: skip the run-skipping decoder
     int last_encode_path = 0;             // 0 = fp64 kernels, 1 = tensor-core kernels (resident basis), 2 = fp32 kernels, 3 = tensor-core kernels (streamed basis)
     int last_decode_path = 0;
+    tc_codebook *stats_cb[9] = {};        // tc_stats: fixed-length code tables (one per bit width) for streams coded without a codebook
 };
 
 struct tc_model {
@@ -102,6 +103,8 @@ struct EncodeArgs {
     unsigned long long *clamped;      // nullable: counts coefficients outside the range
     int emit;                         // 0: symbols only (statistics mode)
     const uint8_t *sym_in;            // exact kernels: non-null = the symbols [P][K] are given, skip the projection
+    unsigned long long *hist;         // tensor-core encoder, statistics: non-null = per-coefficient symbol counts [K][2^bits] are added here
+    int hist_modal;                   // the symbol most lanes are expected to hold (counted once per warp): the zero level
 };
 
 struct DecodeArgs {
@@ -140,7 +143,8 @@ struct DecodeArgs {
 constexpr size_t kEncodeScratchHeader = 64;   // ticket counter, padded; the per-tile look-back words follow
 tc_status tc_encode_with_scratch(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const tc_tensor *x, int chunk_pixels,
                                  int splits, void *stream_out, size_t capacity, uint16_t *chunk_len, uint64_t *tile_off,
-                                 const tc_debug_out *debug, void *scratch, uint8_t *sym_scratch, cudaStream_t s);
+                                 const tc_debug_out *debug, void *scratch, uint8_t *sym_scratch, cudaStream_t s,
+                                 unsigned long long *hist = nullptr, unsigned long long *clamped = nullptr);
 // tensors of fewer tiles than this many per SM take the one-thread-per-value exact kernels
 constexpr int kExactParallelTilesPerSm = 2;
 

@@ -306,3 +306,43 @@ def test_tensor_core_routes_overflow_corruption_and_repeatability(ctx, c, s, n, 
     good = tc.tc_decode(ctx, m, cb, enc, x.shape, x.dtype, stream_bytes=nbytes)
     assert tc.tc_get_status(ctx) == 0 and torch.equal(good, ref)
     m.close(); cb.close()
+
+
+@pytest.mark.parametrize("c,s,n,bits,with_cb", [(64, 14, 1400, 4, False), (256, 14, 9, 5, True), (96, 28, 3, 8, True)])
+def test_stats_on_the_tensor_core_kernels(ctx, c, s, n, bits, with_cb):
+    # bf16 tensors of up to 256 channels: the encoder counts the symbols while it codes (Section 3.1,
+    # "Variable length coding": the entropy needs their distribution); 1400 maps of 64 x 14 x 14 are
+    # more than one chunk of the batch
+    spec = fm.LayerSpec(c, s, s, 0.9, None, 520 + c)
+    o = H.oracle_side(spec, bits, 8, n, torch.bfloat16, False)
+    m = H.import_model(tc, ctx, o["model"], torch.bfloat16)
+    cb = tc.tc_codebook_import(ctx, o["lengths"], bits) if with_cb else None
+    x = o["x"].cuda()
+    st = tc.tc_stats(ctx, m, cb, x, groups=c)
+    assert tc.tc_get_status(ctx) == 0
+    hist = st.hist.cpu().numpy().view(np.uint64)
+    # exactly the histogram of the symbols the encoder produces ...
+    cb_any = cb if cb is not None else tc.tc_codebook_import(ctx, o["lengths"], bits)
+    enc = tc.tc_encode(ctx, m, cb_any, x, debug=True)
+    assert tc.tc_last_path(ctx) == 1
+    q_gpu = enc.symbols.cpu().numpy()
+    assert np.array_equal(hist, oracle.histogram(q_gpu, bits, True))
+    # ... which is the oracle's own up to the symbols that may differ at rounding ties
+    ref = oracle.histogram(o["q"], bits, True)
+    assert np.abs(hist.astype(np.int64) - ref.astype(np.int64)).sum() <= 2 * np.ceil(1e-4 * o["q"].size)
+    assert hist.sum() == o["q"].size
+    want_h = np.mean([oracle.entropy(hist[g]) for g in range(c)])
+    assert st.entropy == pytest.approx(want_h, rel=1e-12)
+    if with_cb:
+        assert st.mean_length == pytest.approx(o["lengths"][0][q_gpu].mean(), rel=1e-12)
+    xhat = oracle.reconstruct(o["model"], q_gpu, tuple(x.shape), out_bf16=True)
+    assert st.mse == pytest.approx(oracle.mse(o["x"], xhat), rel=2e-3)
+    assert st.zero_fraction == pytest.approx(float((o["x"] == 0).double().mean()), abs=1e-12)
+    top = (1 << bits) - 1
+    assert st.clamped_fraction == pytest.approx(float(((o["units"] < 0) | (o["units"] > top)).mean()), abs=1e-4)
+    # folded to one table: the sum over the channels
+    st1 = tc.tc_stats(ctx, m, cb, x, groups=1)
+    assert np.array_equal(st1.hist.cpu().numpy().view(np.uint64)[0], hist.sum(axis=0))
+    for h in (m, cb, cb_any):
+        if h is not None:
+            h.close()
