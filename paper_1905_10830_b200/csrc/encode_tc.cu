@@ -113,23 +113,24 @@ struct SmemBitWriter {
     }
 };
 
-// Two coefficients at once: the multiply-add and the rounding add are packed (two fp32 lanes per
-// instruction, each lane rounded exactly as the scalar instruction rounds), the clamps are not.
-__device__ __forceinline__ void quantise_bits2(uint32_t acc0, uint32_t acc1, float inv_step, float bias0, float bias1, float vmax,
+// Two coefficients at once.  The position on the quantiser's grid is computed as a fraction of
+// its range, t = (y - lo) / (step (2^b - 1)), with a saturating multiply-add: the clamp to the
+// first and last level costs nothing.  A second multiply-add (packed: two fp32 lanes per
+// instruction, each rounded exactly as the scalar instruction rounds) scales t back to levels and
+// adds the magic constant, which leaves the level, rounded to nearest even, in the mantissa.
+__device__ __forceinline__ void quantise_bits2(uint32_t acc0, uint32_t acc1, float inv_range, float bias0, float bias1, float top,
                                                uint32_t &q0, uint32_t &q1)
 {
-    float v0, v1;
-    asm("{\n\t.reg .b64 v, s, b, m;\n\t"
+    float t0, t1;
+    asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(t0) : "f"(__uint_as_float(acc0)), "f"(inv_range), "f"(bias0));
+    asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(t1) : "f"(__uint_as_float(acc1)), "f"(inv_range), "f"(bias1));
+    asm("{\n\t.reg .b64 v, s, m;\n\t"
         "mov.b64 v, {%2, %3};\n\t"
         "mov.b64 s, {%4, %4};\n\t"
-        "mov.b64 b, {%5, %6};\n\t"
-        "mov.b64 m, {%7, %7};\n\t"
-        "fma.rn.f32x2 v, v, s, b;\n\t"
-        "add.rn.f32x2 v, v, m;\n\t"
+        "mov.b64 m, {%5, %5};\n\t"
+        "fma.rn.f32x2 v, v, s, m;\n\t"
         "mov.b64 {%0, %1}, v;\n\t}"
-        : "=f"(v0), "=f"(v1) : "r"(acc0), "r"(acc1), "f"(inv_step), "f"(bias0), "f"(bias1), "f"(kMagic));
-    q0 = __float_as_uint(fminf(fmaxf(v0, kMagic), vmax));
-    q1 = __float_as_uint(fminf(fmaxf(v1, kMagic), vmax));
+        : "=r"(q0), "=r"(q1) : "f"(t0), "f"(t1), "f"(top), "f"(kMagic));
 }
 
 // kPair (per-layer tables, b <= 4): the code tables are indexed by two neighbouring symbols at
@@ -186,7 +187,7 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
             cp_async_16(basis_addr + (j >> 3) * sbo + c8 * 128 + (j & 7) * 16, src + i, 16u);
         }
         cp_async_commit();
-        for (int i = tid; i < a.k; i += kThreads) s_bias[i] = a.enc_bias[i];
+        for (int i = tid; i < a.k; i += kThreads) s_bias[i] = a.enc_bias[i] / (float)(nsym - 1);   // as a fraction of the range
         if (enc_in_smem)
             for (int i = tid; i < enc_entries; i += kThreads) {
                 // per-layer table: (1 << length, code) pairs, so that appending a code to a register is
@@ -347,9 +348,9 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
         const uint32_t pair_len_rel = smem_u32(smem + L.len8) - kMagicBits * (1u + (1u << a.bits));   // same for a pair sum
         unsigned short *xch = reinterpret_cast<unsigned short *>(smem + L.xch) + grp * 256;   // [2][128] lengths exchanged between the halves
         long long n_done = 0;                      // tiles this group has handed to its store warp
-        const float inv_step = (float)(a.basis_scale / a.step);   // the operand holds basis / basis_scale
+        const float inv_range = (float)(a.basis_scale / (a.step * (double)(nsym - 1)));   // the operand holds basis / basis_scale
+        const float top = (float)(nsym - 1);
         const float coef_scale = (float)a.basis_scale;
-        const float vmax = kMagic + (float)(nsym - 1);
         const int bar_id = 1 + grp;
         bool alive = true;
 
@@ -392,7 +393,7 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
                     tmem_ld_wait();
                     uint32_t qv[16];
 #pragma unroll
-                    for (int i = 0; i < 16; i += 2) quantise_bits2(r[i], r[i + 1], inv_step, biasv[i], biasv[i + 1], vmax, qv[i], qv[i + 1]);
+                    for (int i = 0; i < 16; i += 2) quantise_bits2(r[i], r[i + 1], inv_range, biasv[i], biasv[i + 1], top, qv[i], qv[i + 1]);
                     if constexpr (kHist) {
                         const uint32_t modal_bits = kMagicBits + (uint32_t)a.hist_modal;
                         unsigned int n_clamped = 0;
@@ -406,8 +407,8 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
                                 atomicAdd(a.hist + (size_t)j * nsym + a.hist_modal, (unsigned long long)__popc(live & ~others));
                             if (other) atomicAdd(a.hist + (size_t)j * nsym + (qv[i] & 0xffu), 1ull);
                             // outside the quantiser's range [lo, lo + (2^b - 1) step]
-                            const float u = fmaf(__uint_as_float(r[i]), inv_step, biasv[i]);
-                            n_clamped += (valid && (u < 0.f || u > (float)(nsym - 1))) ? 1u : 0u;
+                            const float t = fmaf(__uint_as_float(r[i]), inv_range, biasv[i]);
+                            n_clamped += (valid && (t < 0.f || t > 1.f)) ? 1u : 0u;
                         }
                         if (a.clamped) {
 #pragma unroll
