@@ -115,12 +115,19 @@ typedef struct {
                             a low-variance channel maps to a single value (Appendix E), with zero
                             between two levels it flips between both, which costs rate and
                             distortion.  0 keeps lo at the calibration minimum.                */
+    int32_t eigensolver; /* TC_EIG_DEVICE (0): one-sided Jacobi on the device, no C x C matrix
+                            crosses to the host during the fit.  TC_EIG_HOST (1): the
+                            covariance is copied to the host and solved there (Householder
+                            tridiagonalisation + implicit QR, tc_host_eigh).  Both return the
+                            same decomposition up to rounding.                                  */
 } tc_fit_params;
+enum { TC_EIG_DEVICE = 0, TC_EIG_HOST = 1 };
 
 /* Fit on calibration maps (`calib->n` maps).  Mean and covariance (1/(M-1), M = n*h*w pixel
- * vectors) are accumulated on the device in fp64, the eigendecomposition runs on the host,
- * then the range of coefficient 0 is taken on the device.  Synchronous: returns after the
- * model is complete.  Errors: INVALID_ARG, UNSUPPORTED (C > 1024 or C % 8 != 0 ... see
+ * vectors) are accumulated on the device in fp64, the eigendecomposition runs there too
+ * (params->eigensolver), the basis is rounded and the range of coefficient 0 taken on the
+ * device; the model keeps its basis on the device and copies it to the host only when
+ * tc_model_export or a fold asks for it.  Synchronous: returns after the model is complete.  Errors: INVALID_ARG, UNSUPPORTED (C > 1024 or C % 8 != 0 ... see
  * tc_encode), NOT_CONVERGED, CUDA. */
 tc_status tc_fit_pca(tc_ctx *ctx, const tc_tensor *calib, const tc_fit_params *params,
                      tc_model **out, void *cuda_stream);
@@ -138,7 +145,8 @@ tc_status tc_fit_pca(tc_ctx *ctx, const tc_tensor *calib, const tc_fit_params *p
  *                        outer[C][C] (full symmetric matrix) and *count.
  *   tc_fit_state_import  replaces the state by HOST arrays (for example the sum over devices).
  *   tc_fit_state_finish  mean = s / M, covariance = (S - s s^T / M) / (M - 1), then as
- *                        tc_fit_pca: eigendecomposition on the host, basis rounded to
+ *                        tc_fit_pca: eigendecomposition (on the device unless
+ *                        params->eigensolver says otherwise), basis rounded to
  *                        params->basis_dtype, quantiser range from coefficient 0 over
  *                        `range_maps` (DEVICE tensor; the basis is not known while the state
  *                        is being accumulated, so the caller names the maps the range is
@@ -227,7 +235,14 @@ void tc_codebook_free(tc_codebook *cb);
  * from `counts` (weights counts + 1).  HOST pointers.  No device needed. */
 tc_status tc_host_huffman_lengths(const uint64_t *counts, int32_t nsym, int32_t max_length,
                                   uint8_t *lengths);
-/* Host utility behind tc_fit_pca: eigendecomposition of a symmetric n x n matrix `a`
+/* The fit's device eigensolver on its own: `a` is a symmetric n x n matrix in DEVICE memory
+ * (fp64, row-major, left untouched), evals [n] and evecs [n][n] DEVICE arrays, with the same
+ * conventions as tc_host_eigh.  One-sided Jacobi, one launch per round of n / 2 disjoint
+ * column pairs; synchronises the stream once per sweep.  *sweeps (HOST, may be NULL) receives
+ * the number of sweeps.  Errors: INVALID_ARG, NOT_CONVERGED (150 sweeps), CUDA. */
+tc_status tc_device_eigh(tc_ctx *ctx, const double *a, int32_t n, double *evals, double *evecs, int32_t *sweeps,
+                         void *cuda_stream);
+/* Host eigensolver (TC_EIG_HOST): eigendecomposition of a symmetric n x n matrix `a`
  * (HOST, row-major, destroyed).  On return evals[] is descending and row j of `evecs`
  * ([n][n]) is the unit eigenvector of evals[j], signed so that its largest-magnitude entry
  * is positive.  No device needed. */

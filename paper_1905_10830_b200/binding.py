@@ -12,6 +12,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_PKG, "libtc_b200.so")
 
 TC_F32, TC_BF16, TC_INT8 = 0, 1, 2       # TC_INT8 only names the 8-bit basis of a model
+TC_EIG_DEVICE, TC_EIG_HOST = 0, 1
 _STATUS = ["ok", "invalid argument", "unsupported configuration", "output buffer too small",
            "CUDA error", "corrupt stream", "device-side wait timed out",
            "eigensolver did not converge"]
@@ -30,7 +31,8 @@ class _Tensor(C.Structure):
 
 
 class _FitParams(C.Structure):
-    _fields_ = [("bits", C.c_int32), ("k", C.c_int32), ("basis_dtype", C.c_int32), ("zero_level", C.c_int32)]
+    _fields_ = [("bits", C.c_int32), ("k", C.c_int32), ("basis_dtype", C.c_int32), ("zero_level", C.c_int32),
+                ("eigensolver", C.c_int32)]
 
 
 class _ModelDesc(C.Structure):
@@ -66,7 +68,7 @@ class _StatsOut(C.Structure):
 EXPORTS = ["tc_create", "tc_destroy", "tc_status_string", "tc_get_status", "tc_force_exact_path", "tc_last_path", "tc_fit_pca",
            "tc_model_import", "tc_model_export", "tc_model_free", "tc_build_codebook",
            "tc_codebook_import", "tc_codebook_export", "tc_codebook_free",
-           "tc_host_huffman_lengths", "tc_host_eigh", "tc_encode_bound", "tc_encode", "tc_encode_noalloc", "tc_decode", "tc_roundtrip_host",
+           "tc_host_huffman_lengths", "tc_host_eigh", "tc_device_eigh", "tc_encode_bound", "tc_encode", "tc_encode_noalloc", "tc_decode", "tc_roundtrip_host",
            "tc_stats", "tc_fit_state_create", "tc_fit_state_free", "tc_fit_state_update", "tc_fit_state_export",
            "tc_fit_state_import", "tc_fit_state_finish", "tc_fold_forward", "tc_fold_inverse"]
 
@@ -108,6 +110,7 @@ def load_library() -> C.CDLL:
         lib.tc_codebook_free.restype = None
         lib.tc_host_huffman_lengths.argtypes = [vp, i32, i32, vp]
         lib.tc_host_eigh.argtypes = [vp, i32, vp, vp]
+        lib.tc_device_eigh.argtypes = [vp, vp, i32, vp, vp, P(i32), vp]
         lib.tc_encode_bound.argtypes = [vp, vp, P(_Tensor), P(_EncodeParams), P(_StreamLayout)]
         lib.tc_encode.argtypes = [vp, vp, vp, P(_Tensor), P(_EncodeParams), vp, C.c_size_t, vp, vp,
                                   P(_DebugOut), vp]
@@ -245,11 +248,11 @@ def tc_get_status(ctx: Context) -> int:
 
 
 def tc_fit_pca(ctx: Context, calib: torch.Tensor, bits: int, k: int = 0, basis_dtype: int | None = None,
-               zero_level: bool = True) -> Model:
+               zero_level: bool = True, eigensolver: int = TC_EIG_DEVICE) -> Model:
     """`zero_level` (on by default here; tc_fit_params.zero_level in the C ABI) shifts the quantiser
     grid so that y = 0 is one of its levels."""
     t = _tensor(calib)
-    params = _FitParams(bits, k, t.dtype if basis_dtype is None else basis_dtype, int(zero_level))
+    params = _FitParams(bits, k, t.dtype if basis_dtype is None else basis_dtype, int(zero_level), eigensolver)
     out = C.c_void_p()
     _check(load_library().tc_fit_pca(ctx.ptr, C.byref(t), C.byref(params), C.byref(out),
                                      _stream_ptr(ctx.device)), "tc_fit_pca")
@@ -290,9 +293,9 @@ def tc_fit_state_import(ctx: Context, state: FitState, count: int, s1: np.ndarra
 
 
 def tc_fit_state_finish(ctx: Context, state: FitState, range_maps: torch.Tensor, bits: int, k: int = 0,
-                        basis_dtype: int | None = None, zero_level: bool = True) -> Model:
+                        basis_dtype: int | None = None, zero_level: bool = True, eigensolver: int = TC_EIG_DEVICE) -> Model:
     t = _tensor(range_maps)
-    params = _FitParams(bits, k, t.dtype if basis_dtype is None else basis_dtype, int(zero_level))
+    params = _FitParams(bits, k, t.dtype if basis_dtype is None else basis_dtype, int(zero_level), eigensolver)
     out = C.c_void_p()
     _check(load_library().tc_fit_state_finish(ctx.ptr, state.ptr, C.byref(t), C.byref(params), C.byref(out),
                                               _stream_ptr(ctx.device)), "tc_fit_state_finish")
@@ -391,6 +394,21 @@ def tc_host_huffman_lengths(counts: np.ndarray, max_length: int = 12) -> np.ndar
     _check(load_library().tc_host_huffman_lengths(counts.ctypes.data, counts.shape[0], max_length, out.ctypes.data),
            "tc_host_huffman_lengths")
     return out
+
+
+def tc_device_eigh(ctx: Context, a: torch.Tensor):
+    """Eigenvalues (descending), eigenvectors (rows) and the number of Jacobi sweeps for a symmetric
+    float64 CUDA matrix."""
+    if a.dtype != torch.float64 or not a.is_cuda or a.dim() != 2 or a.shape[0] != a.shape[1]:
+        raise ValueError("tc_device_eigh wants a square float64 CUDA tensor")
+    a = a.contiguous()
+    n = a.shape[0]
+    evals = torch.empty(n, dtype=torch.float64, device=a.device)
+    evecs = torch.empty((n, n), dtype=torch.float64, device=a.device)
+    sweeps = C.c_int32(0)
+    _check(load_library().tc_device_eigh(ctx.ptr, a.data_ptr(), n, evals.data_ptr(), evecs.data_ptr(), C.byref(sweeps),
+                                         _stream_ptr(ctx.device)), "tc_device_eigh")
+    return evals, evecs, sweeps.value
 
 
 def tc_host_eigh(a: np.ndarray):

@@ -58,17 +58,11 @@ __host__ __device__ inline SmemLayout smem_layout(int c, int k, int enc_entries)
     return l;
 }
 
-// Quantiser in fp32: v = acc/step - (T mu + lo)/step, rounded to the nearest integer (ties to
-// even) by adding 1.5 * 2^23 -- the integer then sits in the low mantissa bits -- and clamped to
-// [0, 2^b - 1] while still a float.  (A float -> int conversion instruction would do the same
-// but issues at a quarter of the rate.)
+// Quantiser in fp32.  The level is rounded to the nearest integer (ties to even) by adding
+// 1.5 * 2^23 -- the integer then sits in the low mantissa bits.  (A float -> int conversion
+// instruction would do the same but issues at a quarter of the rate.)
 constexpr float kMagic = 12582912.0f;
 constexpr uint32_t kMagicBits = 0x4B400000u;
-// returns kMagicBits + q
-__device__ __forceinline__ uint32_t quantise_bits(uint32_t acc_bits, float inv_step, float bias, float vmax)
-{
-    return __float_as_uint(fminf(fmaxf(fmaf(__uint_as_float(acc_bits), inv_step, bias) + kMagic, kMagic), vmax));
-}
 
 // Bit writer into the shared-memory staging buffer.  A word is stored (plain, predicated
 // store) by the writer that supplies its last bit; bits that other writers own in that word

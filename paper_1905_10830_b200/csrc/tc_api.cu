@@ -110,43 +110,46 @@ tc_status ensure_scratch(tc_ctx *ctx, size_t bytes)
     return TC_OK;
 }
 
+// The host copy of a model's basis, fetched from the device at first use.
+const std::vector<double> *host_basis(const tc_model *m)
+{
+    if (m->basis.empty() && m->d_basis64) {
+        DeviceGuard guard(m->device);
+        m->basis.resize((size_t)m->c * m->c);
+        if (cudaMemcpy(m->basis.data(), m->d_basis64, m->basis.size() * sizeof(double), cudaMemcpyDeviceToHost) != cudaSuccess) {
+            cudaGetLastError();
+            m->basis.clear();
+            return nullptr;
+        }
+    }
+    return &m->basis;
+}
+
+// Completes a model whose basis and mean are on the device (d_basis64, d_mean64) and whose
+// scalars are set: the constants and operand copies the codec kernels read are computed there.
 tc_status finish_model(tc_model *m)
 {
     const int c = m->c, k = m->k;
-    std::vector<double> tmu(k, 0.0), colsum(c, 0.0);
-    for (int j = 0; j < k; ++j) {
-        double s = 0.0;
-        for (int a = 0; a < c; ++a) s += m->basis[(size_t)j * c + a] * m->mean[a];
-        tmu[j] = s;
-        for (int a = 0; a < c; ++a) colsum[a] += m->basis[(size_t)j * c + a];
-    }
-    std::vector<float> enc_bias(k), dec_bias(c), tmu32(k);
-    for (int j = 0; j < k; ++j) { enc_bias[j] = (float)(-(tmu[j] + m->lo) / m->step); tmu32[j] = (float)tmu[j]; }
     // The inverse projection runs on symbols centred on the level nearest to y = 0, so that the
     // accumulators stay small and no large terms cancel in fp32:
     // x_hat = step * sum_j T[j][c] (q_j - center) + mu_c + (lo + center*step) * sum_j T[j][c]
     const double top = (double)((1 << m->bits) - 1);
     m->center = (int)std::min(top, std::max(0.0, std::nearbyint(-m->lo / m->step)));
-    for (int a = 0; a < c; ++a) dec_bias[a] = (float)(m->mean[a] + (m->lo + m->center * m->step) * colsum[a]);
     tc_status st;
-    if ((st = upload(&m->d_basis64, m->basis)) != TC_OK) return st;
-    if ((st = upload(&m->d_mean64, m->mean)) != TC_OK) return st;
-    if ((st = upload(&m->d_enc_bias, enc_bias)) != TC_OK) return st;
-    if ((st = upload(&m->d_dec_bias, dec_bias)) != TC_OK) return st;
-    if ((st = upload(&m->d_tmu32, tmu32)) != TC_OK) return st;
+    if (!m->d_basis64 && (st = upload(&m->d_basis64, m->basis)) != TC_OK) return st;
+    if (!m->d_mean64 && (st = upload(&m->d_mean64, m->mean)) != TC_OK) return st;
+    TC_CUDA(cudaMalloc((void **)&m->d_enc_bias, sizeof(float) * k));
+    TC_CUDA(cudaMalloc((void **)&m->d_tmu32, sizeof(float) * k));
+    TC_CUDA(cudaMalloc((void **)&m->d_dec_bias, sizeof(float) * c));
+    if ((st = tc_launch_model_consts(m->d_basis64, m->d_mean64, c, k, m->lo, m->step, (double)m->center, m->d_enc_bias,
+                                     m->d_tmu32, m->d_dec_bias, nullptr)) != TC_OK) return st;
     if (m->basis_dtype == TC_BF16 || m->basis_dtype == TC_INT8) {
         // an 8-bit basis goes to the bf16 kernels as its integers (exact in bf16); the scale is
         // folded into their quantiser and dequantiser constants
-        std::vector<__nv_bfloat16> b((size_t)k * c), bt((size_t)c * k);
-        for (int j = 0; j < k; ++j)
-            for (int a = 0; a < c; ++a) {
-                const __nv_bfloat16 v = __float2bfloat16((float)(m->basis_dtype == TC_INT8 ? std::nearbyint(m->basis[(size_t)j * c + a] / m->basis_scale)
-                                                                                          : m->basis[(size_t)j * c + a]));
-                b[(size_t)j * c + a] = v;
-                bt[(size_t)a * k + j] = v;
-            }
-        if ((st = upload(&m->d_basis_bf16, b)) != TC_OK) return st;
-        if ((st = upload(&m->d_basis_t_bf16, bt)) != TC_OK) return st;
+        TC_CUDA(cudaMalloc((void **)&m->d_basis_bf16, sizeof(__nv_bfloat16) * (size_t)k * c));
+        TC_CUDA(cudaMalloc((void **)&m->d_basis_t_bf16, sizeof(__nv_bfloat16) * (size_t)k * c));
+        if ((st = tc_launch_basis_bf16(m->d_basis64, c, k, m->basis_scale, m->basis_dtype == TC_INT8, m->d_basis_bf16,
+                                       m->d_basis_t_bf16, nullptr)) != TC_OK) return st;
         // Tensor map for the kernels that stream the basis: boxes of 256 coefficient rows x 32
         // channels (64 bytes), written with the 64-byte swizzle the MMA descriptor names.  Needs
         // rows of a multiple of 16 bytes; without a map those kernels copy the basis with cp.async.
@@ -175,6 +178,7 @@ tc_status finish_model(tc_model *m)
             m->has_basis_t_map = rc == CUDA_SUCCESS;
         }
     }
+    TC_CUDA(cudaStreamSynchronize(nullptr));
     return TC_OK;
 }
 
@@ -360,7 +364,11 @@ tc_status tc_model_export(const tc_model *m, tc_model_desc *d)
     if (!m || !d) return TC_ERR_INVALID_ARG;
     d->c = m->c; d->k = m->k; d->bits = m->bits; d->basis_dtype = m->basis_dtype;
     d->lo = m->lo; d->step = m->step; d->basis_scale = m->basis_scale;
-    if (d->basis) std::copy(m->basis.begin(), m->basis.end(), d->basis);
+    if (d->basis) {
+        const std::vector<double> *b = host_basis(m);
+        if (!b) return TC_ERR_CUDA;
+        std::copy(b->begin(), b->end(), d->basis);
+    }
     if (d->mean) std::copy(m->mean.begin(), m->mean.end(), d->mean);
     if (d->eig) std::copy(m->eig.begin(), m->eig.end(), d->eig);
     return TC_OK;
@@ -376,7 +384,13 @@ void tc_model_free(tc_model *m)
 }
 
 static tc_status finish_fit(tc_ctx *ctx, const tc_tensor *range_maps, const tc_fit_params *params, int k,
-                            std::vector<double> &mean, std::vector<double> &cov, tc_model **out, cudaStream_t s);
+                            const double *d_mean, const double *d_cov, tc_model **out, cudaStream_t s);
+
+static bool valid_fit_params(const tc_fit_params *params)
+{
+    return (params->basis_dtype == TC_F32 || params->basis_dtype == TC_BF16 || params->basis_dtype == TC_INT8) &&
+           (params->eigensolver == TC_EIG_DEVICE || params->eigensolver == TC_EIG_HOST);
+}
 
 tc_status tc_fit_pca(tc_ctx *ctx, const tc_tensor *calib, const tc_fit_params *params, tc_model **out, void *cuda_stream)
 {
@@ -388,7 +402,7 @@ tc_status tc_fit_pca(tc_ctx *ctx, const tc_tensor *calib, const tc_fit_params *p
     if (params->bits < 1 || params->bits > 8 || c > TC_MAX_C) return TC_ERR_UNSUPPORTED;
     const int k = params->k ? params->k : c;
     if (k < 1 || k > c) return TC_ERR_INVALID_ARG;
-    if (params->basis_dtype != TC_F32 && params->basis_dtype != TC_BF16 && params->basis_dtype != TC_INT8) return TC_ERR_INVALID_ARG;
+    if (!valid_fit_params(params)) return TC_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     cudaStream_t s = (cudaStream_t)cuda_stream;
 
@@ -408,62 +422,77 @@ tc_status tc_fit_pca(tc_ctx *ctx, const tc_tensor *calib, const tc_fit_params *p
     TC_CUDA(cudaMemcpyAsync(d_mean, mean.data(), sizeof(double) * c, cudaMemcpyHostToDevice, s));
     st = tc_launch_covariance(calib->data, calib->dtype, n, c, hw, d_mean, d_cov, s);
     if (st != TC_OK) return st;
-    std::vector<double> cov((size_t)c * c);
-    TC_CUDA(cudaMemcpyAsync(cov.data(), d_cov, sizeof(double) * cov.size(), cudaMemcpyDeviceToHost, s));
-    TC_CUDA(cudaStreamSynchronize(s));
-    const double denom = (double)(m_samples - 1);
-    for (int a = 0; a < c; ++a)
-        for (int b = a; b < c; ++b) {
-            const double v = cov[(size_t)a * c + b] / denom;
-            cov[(size_t)a * c + b] = cov[(size_t)b * c + a] = v;
-        }
-    return finish_fit(ctx, calib, params, k, mean, cov, out, s);
+    // centred sums in the upper triangle -> covariance, full symmetric, still on the device
+    if ((st = tc_launch_scale_mirror(d_cov, c, (double)(m_samples - 1), s)) != TC_OK) return st;
+    return finish_fit(ctx, calib, params, k, d_mean, d_cov, out, s);
 }
 
-// Second half of a fit: eigendecomposition of the (symmetric, normalised) covariance on the
-// host, rounding of the basis, range of coefficient 0 over `range_maps` on the device.
+// Second half of a fit, from the mean and the (symmetric, normalised) covariance on the device:
+// eigendecomposition (on the device; on the host if the caller asks for that solver), rounding
+// of the basis, range of coefficient 0 over `range_maps`, the model's constants.  Only vectors of
+// C numbers cross to the host, unless the host solver was asked for.
 static tc_status finish_fit(tc_ctx *ctx, const tc_tensor *range_maps, const tc_fit_params *params, int k,
-                            std::vector<double> &mean, std::vector<double> &cov, tc_model **out, cudaStream_t s)
+                            const double *d_mean, const double *d_cov, tc_model **out, cudaStream_t s)
 {
     const int c = range_maps->c, hw = range_maps->h * range_maps->w, n = range_maps->n;
     const long long m_samples = (long long)n * hw;
     const int range_blocks = tc_range0_max_blocks(m_samples);
-    double *d_buf = nullptr;
-    TC_CUDA(cudaMalloc((void **)&d_buf, (2 * (size_t)c + 2 * (size_t)range_blocks) * sizeof(double)));
-    struct Free { double *p; ~Free() { cudaFree(p); } } freer{d_buf};
-    double *d_mean = d_buf, *d_row0 = d_buf + c, *d_minmax = d_row0 + c;
-    TC_CUDA(cudaMemcpyAsync(d_mean, mean.data(), sizeof(double) * c, cudaMemcpyHostToDevice, s));
+    const size_t cc = (size_t)c * c;
+    // small: eigenvalues [c], scale [1], min / max per block [2 * range_blocks]
+    double *d_small = nullptr, *d_basis = nullptr, *d_mean_copy = nullptr;
+    void *d_work = nullptr;
+    struct Free {
+        double **a, **b, **m; void **w;
+        ~Free() { cudaFree(*a); cudaFree(*b); cudaFree(*m); cudaFree(*w); }
+    } freer{&d_small, &d_basis, &d_mean_copy, &d_work};
+    TC_CUDA(cudaMalloc((void **)&d_small, ((size_t)c + 1 + 2 * (size_t)range_blocks) * sizeof(double)));
+    TC_CUDA(cudaMalloc((void **)&d_basis, cc * sizeof(double)));
+    TC_CUDA(cudaMalloc((void **)&d_mean_copy, (size_t)c * sizeof(double)));
+    double *d_eig = d_small, *d_scale = d_small + c, *d_minmax = d_scale + 1;
+    TC_CUDA(cudaMemcpyAsync(d_mean_copy, d_mean, sizeof(double) * c, cudaMemcpyDeviceToDevice, s));
     tc_status st;
-    std::vector<double> eig(c), basis((size_t)c * c);
-    if (tc_eigh_host(cov.data(), c, eig.data(), basis.data()) != 0) return TC_ERR_NOT_CONVERGED;
-    double basis_scale = 1.0;
-    if (params->basis_dtype == TC_INT8) {
-        double biggest = 0.0;
-        for (double v : basis) biggest = std::max(biggest, std::fabs(v));
-        basis_scale = biggest / 127.0;
-        for (double &v : basis) v = basis_scale * std::nearbyint(v / basis_scale);
+    if (params->eigensolver == TC_EIG_HOST) {
+        std::vector<double> cov(cc), eig(c), basis(cc);
+        TC_CUDA(cudaMemcpyAsync(cov.data(), d_cov, sizeof(double) * cc, cudaMemcpyDeviceToHost, s));
+        TC_CUDA(cudaStreamSynchronize(s));
+        if (tc_eigh_host(cov.data(), c, eig.data(), basis.data()) != 0) return TC_ERR_NOT_CONVERGED;
+        TC_CUDA(cudaMemcpyAsync(d_basis, basis.data(), sizeof(double) * cc, cudaMemcpyHostToDevice, s));
+        TC_CUDA(cudaMemcpyAsync(d_eig, eig.data(), sizeof(double) * c, cudaMemcpyHostToDevice, s));
+        TC_CUDA(cudaStreamSynchronize(s));
     } else {
-        for (double &v : basis) v = round_to_dtype(v, params->basis_dtype);
+        TC_CUDA(cudaMalloc(&d_work, tc_eigh_device_workspace_bytes(c)));
+        if ((st = tc_eigh_device(d_cov, c, d_eig, d_basis, d_work, nullptr, s)) != TC_OK) return st;
     }
+    if ((st = tc_launch_round_basis(d_basis, c, params->basis_dtype, d_scale, s)) != TC_OK) return st;
 
-    TC_CUDA(cudaMemcpyAsync(d_row0, basis.data(), sizeof(double) * c, cudaMemcpyHostToDevice, s));
     int blocks = 0;
-    st = tc_launch_range0(range_maps->data, range_maps->dtype, n, c, hw, d_mean, d_row0, d_minmax, &blocks, s);
+    st = tc_launch_range0(range_maps->data, range_maps->dtype, n, c, hw, d_mean_copy, d_basis, d_minmax, &blocks, s);
     if (st != TC_OK) return st;
-    std::vector<double> mm(2 * (size_t)blocks);
-    TC_CUDA(cudaMemcpyAsync(mm.data(), d_minmax, sizeof(double) * mm.size(), cudaMemcpyDeviceToHost, s));
+    std::vector<double> small((size_t)c + 1 + 2 * (size_t)blocks), mean(c);
+    TC_CUDA(cudaMemcpyAsync(small.data(), d_small, sizeof(double) * small.size(), cudaMemcpyDeviceToHost, s));
+    TC_CUDA(cudaMemcpyAsync(mean.data(), d_mean_copy, sizeof(double) * c, cudaMemcpyDeviceToHost, s));
     TC_CUDA(cudaStreamSynchronize(s));
+    const double *mm = small.data() + c + 1;
     double lo = INFINITY, hi = -INFINITY;
     for (int i = 0; i < blocks; ++i) { lo = std::min(lo, mm[2 * i]); hi = std::max(hi, mm[2 * i + 1]); }
     if (!(hi > lo)) return TC_ERR_INVALID_ARG;    // constant calibration data: no range to quantise
 
-    tc_model_desc d;
-    d.c = c; d.k = k; d.bits = params->bits; d.basis_dtype = params->basis_dtype;
-    d.step = (hi - lo) / (double)((1 << params->bits) - 1);
+    tc_model *m = new (std::nothrow) tc_model();
+    if (!m) return TC_ERR_CUDA;
+    m->c = c; m->k = k; m->bits = params->bits; m->basis_dtype = params->basis_dtype; m->device = ctx->device;
+    m->step = (hi - lo) / (double)((1 << params->bits) - 1);
     // zero_level: shift the grid so that y = 0 is a level (at most half a step; ties to even)
-    d.lo = params->zero_level ? -d.step * std::nearbyint(-lo / d.step) : lo;
-    d.basis = basis.data(); d.mean = mean.data(); d.eig = eig.data(); d.basis_scale = basis_scale;
-    return tc_model_import(ctx, &d, out);
+    m->lo = params->zero_level ? -m->step * std::nearbyint(-lo / m->step) : lo;
+    m->basis_scale = params->basis_dtype == TC_INT8 ? small[c] : 1.0;
+    m->mean = mean;
+    m->eig.assign(small.begin(), small.begin() + c);
+    m->d_basis64 = d_basis; d_basis = nullptr;         // the model owns them from here
+    m->d_mean64 = d_mean_copy; d_mean_copy = nullptr;
+    if (params->basis_dtype == TC_INT8 && !(m->basis_scale > 0.0)) { tc_model_free(m); return TC_ERR_INVALID_ARG; }
+    st = finish_model(m);
+    if (st != TC_OK) { tc_model_free(m); return st; }
+    *out = m;
+    return TC_OK;
 }
 
 // ---- online fit: running sums ---------------------------------------------------------------
@@ -555,23 +584,17 @@ tc_status tc_fit_state_finish(tc_ctx *ctx, const tc_fit_state *st, const tc_tens
     if (params->bits < 1 || params->bits > 8) return TC_ERR_UNSUPPORTED;
     const int k = params->k ? params->k : c;
     if (k < 1 || k > c) return TC_ERR_INVALID_ARG;
-    if (params->basis_dtype != TC_F32 && params->basis_dtype != TC_BF16 && params->basis_dtype != TC_INT8) return TC_ERR_INVALID_ARG;
+    if (!valid_fit_params(params)) return TC_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     cudaStream_t s = (cudaStream_t)cuda_stream;
-    std::vector<double> sum(c), cov((size_t)c * c);
-    int64_t count = 0;
-    tc_status rc = tc_fit_state_export(ctx, st, &count, sum.data(), cov.data(), cuda_stream);
+    // mean = s / M, covariance = (S - s s^T / M) / (M - 1), on the device
+    double *d_buf = nullptr;
+    TC_CUDA(cudaMalloc((void **)&d_buf, ((size_t)c + (size_t)c * c) * sizeof(double)));
+    struct Free { double *p; ~Free() { cudaFree(p); } } freer{d_buf};
+    double *d_mean = d_buf, *d_cov = d_buf + c;
+    tc_status rc = tc_launch_moments_to_cov(st->d_sum, st->d_outer, st->count, c, d_mean, d_cov, s);
     if (rc != TC_OK) return rc;
-    // mean = s / M, covariance = (S - s s^T / M) / (M - 1)
-    const double m = (double)count;
-    std::vector<double> mean(c);
-    for (int a = 0; a < c; ++a) mean[a] = sum[a] / m;
-    for (int a = 0; a < c; ++a)
-        for (int b = a; b < c; ++b) {
-            const double v = (cov[(size_t)a * c + b] - sum[a] * sum[b] / m) / (m - 1.0);
-            cov[(size_t)a * c + b] = cov[(size_t)b * c + a] = v;
-        }
-    return finish_fit(ctx, range_maps, params, k, mean, cov, out, s);
+    return finish_fit(ctx, range_maps, params, k, d_mean, d_cov, out, s);
 }
 
 // ---- folding into the neighbouring convolutions (host arithmetic, fp64) --------------------------
@@ -581,8 +604,10 @@ tc_status tc_fold_forward(const tc_model *m, const double *w, const double *bias
 {
     if (!m || !w || !w_folded || !bias_folded || fan < 1) return TC_ERR_INVALID_ARG;
     const int c = m->c, k = m->k;
+    const std::vector<double> *basis = host_basis(m);
+    if (!basis) return TC_ERR_CUDA;
     for (int j = 0; j < k; ++j) {
-        const double *row = m->basis.data() + (size_t)j * c;
+        const double *row = basis->data() + (size_t)j * c;
         for (int64_t f = 0; f < fan; ++f) {
             double acc = 0.0;
             for (int a = 0; a < c; ++a) acc += row[a] * ((scale ? scale[a] : 1.0) * w[(size_t)a * fan + f]);
@@ -601,9 +626,11 @@ tc_status tc_fold_inverse(const tc_model *m, const double *w_next, const double 
 {
     if (!m || !w_next || !w_folded || !bias_folded || c_out < 1 || taps < 1) return TC_ERR_INVALID_ARG;
     const int c = m->c, k = m->k;
+    const std::vector<double> *basis = host_basis(m);
+    if (!basis) return TC_ERR_CUDA;
     for (int o = 0; o < c_out; ++o) {
         for (int j = 0; j < k; ++j) {
-            const double *row = m->basis.data() + (size_t)j * c;
+            const double *row = basis->data() + (size_t)j * c;
             for (int t = 0; t < taps; ++t) {
                 double acc = 0.0;
                 for (int a = 0; a < c; ++a) acc += w_next[((size_t)o * c + a) * taps + t] * row[a];
@@ -623,6 +650,21 @@ tc_status tc_fold_inverse(const tc_model *m, const double *w_next, const double 
 tc_status tc_host_huffman_lengths(const uint64_t *counts, int32_t nsym, int32_t max_length, uint8_t *lengths)
 {
     return tc_huffman_lengths_host(counts, nsym, max_length, lengths) == 0 ? TC_OK : TC_ERR_INVALID_ARG;
+}
+
+tc_status tc_device_eigh(tc_ctx *ctx, const double *a, int32_t n, double *evals, double *evecs, int32_t *sweeps, void *cuda_stream)
+{
+    if (!ctx || !a || !evals || !evecs || n < 1 || n > TC_MAX_C) return TC_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    void *work = nullptr;
+    TC_CUDA(cudaMalloc(&work, tc_eigh_device_workspace_bytes(n)));
+    int n_sweeps = 0;
+    const tc_status st = tc_eigh_device(a, n, evals, evecs, work, &n_sweeps, s);
+    cudaStreamSynchronize(s);
+    cudaFree(work);
+    if (sweeps) *sweeps = n_sweeps;
+    return st;
 }
 
 tc_status tc_host_eigh(double *a, int32_t n, double *evals, double *evecs)

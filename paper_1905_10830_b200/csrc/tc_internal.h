@@ -47,7 +47,10 @@ struct tc_model {
     double lo = 0, step = 0;
     double basis_scale = 1.0;               // 8-bit basis: entries are integers times this; 1 otherwise
     int center = 0;                         // symbol whose level is nearest to y = 0
-    std::vector<double> basis, mean, eig;   // host copies (basis [c][c])
+    // host copies; a model fitted on the device holds its basis there only, and `basis` is filled
+    // from d_basis64 the first time the host needs it (export, folding)
+    mutable std::vector<double> basis;      // [c][c], or empty
+    std::vector<double> mean, eig;          // [c]
     int device = 0;
     // device copies
     double *d_basis64 = nullptr;            // [c][c] exact values of the (rounded) basis
@@ -186,3 +189,14 @@ tc_status tc_launch_sqerr(const void *x, const void *xhat, int dtype, long long 
 int tc_huffman_lengths_host(const uint64_t *counts, int nsym, int lmax, uint8_t *len);
 void tc_canonical_codes_host(const uint8_t *len, int nsym, uint32_t *code);
 int tc_eigh_host(double *a, int n, double *evals, double *evecs);
+
+// ---- fit on the device (eigh_device.cu) ---------------------------------------------------
+tc_status tc_launch_moments_to_cov(const double *sum, const double *outer, long long count, int c, double *mean, double *cov,
+                                   cudaStream_t s);
+tc_status tc_launch_scale_mirror(double *cov, int c, double denom, cudaStream_t s);
+size_t tc_eigh_device_workspace_bytes(int c);
+tc_status tc_eigh_device(const double *a, int c, double *evals, double *evecs, void *work, int *sweeps_out, cudaStream_t s);
+tc_status tc_launch_round_basis(double *basis, int c, int dtype, double *scale_slot, cudaStream_t s);
+tc_status tc_launch_model_consts(const double *basis, const double *mean, int c, int k, double lo, double step, double center,
+                                 float *enc_bias, float *tmu32, float *dec_bias, cudaStream_t s);
+tc_status tc_launch_basis_bf16(const double *basis, int c, int k, double basis_scale, bool int8, void *b, void *bt, cudaStream_t s);
