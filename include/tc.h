@@ -353,6 +353,40 @@ tc_status tc_decode(tc_ctx *ctx, const tc_model *model, const tc_codebook *cb, c
                     size_t stream_bytes, const uint16_t *chunk_len, const uint64_t *tile_off,
                     const tc_encode_params *params, const tc_tensor *x_hat, void *cuda_stream);
 
+/* Several tensors per call (Section 3.1: every layer has its own encoder and decoder -- its own
+ * PCA matrix, range and code table -- and an inference pass codes them all).  A network's
+ * layers at a small batch are each too small to fill the GPU, and a call per layer pays the
+ * launch and set-up time of its kernels one after the other.  These entry points take the
+ * whole list: the items are checked first (nothing is launched if one is invalid), the
+ * bookkeeping of all of them is cleared at once, and their kernels are spread, largest first,
+ * over four streams of the context so that small layers run beside one another; `cuda_stream`
+ * waits for all of them, so later work on it sees every output.  The results are those of
+ * tc_encode / tc_decode called per item (same arguments, same errors; the first error is
+ * returned after all items that could be launched have been).  Output buffers of different
+ * items must not overlap.  tc_last_path reports the route of the item launched last. */
+typedef struct {
+    const tc_model *model;
+    const tc_codebook *codebook;
+    const tc_tensor *x;
+    const tc_encode_params *params; /* may be NULL */
+    void *stream_out;               /* DEVICE, 16-byte aligned, `capacity` bytes */
+    size_t capacity;
+    uint16_t *chunk_len;            /* DEVICE uint16[n_chunks], 4-byte aligned   */
+    uint64_t *tile_off;             /* DEVICE uint64[n_tiles + 1]                */
+} tc_encode_item;
+typedef struct {
+    const tc_model *model;
+    const tc_codebook *codebook;
+    const void *stream;             /* DEVICE, 16-byte aligned */
+    size_t stream_bytes;
+    const uint16_t *chunk_len;
+    const uint64_t *tile_off;
+    const tc_encode_params *params; /* may be NULL */
+    const tc_tensor *x_hat;
+} tc_decode_item;
+tc_status tc_encode_many(tc_ctx *ctx, const tc_encode_item *items, int32_t n_items, void *cuda_stream);
+tc_status tc_decode_many(tc_ctx *ctx, const tc_decode_item *items, int32_t n_items, void *cuda_stream);
+
 /* Whole chain on HOST tensors (Section 3: encoder, memory, decoder): copies `x_host` (dense
  * NCHW, `dtype`, pinned memory recommended) to the device, encodes, decodes and copies the
  * reconstruction to `x_hat_host`, then synchronises `cuda_stream`.  Larger batches are worked

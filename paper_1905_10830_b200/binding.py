@@ -68,7 +68,7 @@ class _StatsOut(C.Structure):
 EXPORTS = ["tc_create", "tc_destroy", "tc_status_string", "tc_get_status", "tc_force_exact_path", "tc_last_path", "tc_fit_pca",
            "tc_model_import", "tc_model_export", "tc_model_free", "tc_build_codebook",
            "tc_codebook_import", "tc_codebook_export", "tc_codebook_free",
-           "tc_host_huffman_lengths", "tc_host_eigh", "tc_device_eigh", "tc_encode_bound", "tc_encode", "tc_encode_noalloc", "tc_decode", "tc_roundtrip_host",
+           "tc_host_huffman_lengths", "tc_host_eigh", "tc_device_eigh", "tc_encode_bound", "tc_encode", "tc_encode_noalloc", "tc_decode", "tc_encode_many", "tc_decode_many", "tc_roundtrip_host",
            "tc_stats", "tc_fit_state_create", "tc_fit_state_free", "tc_fit_state_update", "tc_fit_state_export",
            "tc_fit_state_import", "tc_fit_state_finish", "tc_fold_forward", "tc_fold_inverse"]
 
@@ -110,6 +110,8 @@ def load_library() -> C.CDLL:
         lib.tc_codebook_free.restype = None
         lib.tc_host_huffman_lengths.argtypes = [vp, i32, i32, vp]
         lib.tc_host_eigh.argtypes = [vp, i32, vp, vp]
+        lib.tc_encode_many.argtypes = [vp, vp, i32, vp]
+        lib.tc_decode_many.argtypes = [vp, vp, i32, vp]
         lib.tc_device_eigh.argtypes = [vp, vp, i32, vp, vp, P(i32), vp]
         lib.tc_encode_bound.argtypes = [vp, vp, P(_Tensor), P(_EncodeParams), P(_StreamLayout)]
         lib.tc_encode.argtypes = [vp, vp, vp, P(_Tensor), P(_EncodeParams), vp, C.c_size_t, vp, vp,
@@ -490,6 +492,55 @@ def tc_decode(ctx: Context, model: Model, cb: Codebook, enc: EncodedStream, shap
                                     enc.chunk_len.data_ptr(), enc.tile_off.data_ptr(), C.byref(p), C.byref(t),
                                     _stream_ptr(ctx.device)), "tc_decode")
     return out
+
+
+class _EncodeItem(C.Structure):
+    _fields_ = [("model", C.c_void_p), ("codebook", C.c_void_p), ("x", C.c_void_p), ("params", C.c_void_p),
+                ("stream_out", C.c_void_p), ("capacity", C.c_size_t), ("chunk_len", C.c_void_p), ("tile_off", C.c_void_p)]
+
+
+class _DecodeItem(C.Structure):
+    _fields_ = [("model", C.c_void_p), ("codebook", C.c_void_p), ("stream", C.c_void_p), ("stream_bytes", C.c_size_t),
+                ("chunk_len", C.c_void_p), ("tile_off", C.c_void_p), ("params", C.c_void_p), ("x_hat", C.c_void_p)]
+
+
+def tc_encode_many(ctx: Context, layers, *, outs=None):
+    """Encode several tensors in one call: `layers` is a list of (model, codebook, x).  Returns the
+    list of EncodedStream; `outs` reuses the buffers of an earlier call."""
+    n = len(layers)
+    tensors, params, items = [], [], (_EncodeItem * max(n, 1))()
+    result = []
+    for i, (model, cb, x) in enumerate(layers):
+        t = _tensor(x)
+        lay = tc_encode_bound(model, cb, x, 0, 0)
+        if outs is not None:
+            out = outs[i]
+        else:
+            out = EncodedStream(torch.empty(max(lay.stream_bytes, 16), dtype=torch.uint8, device=x.device),
+                                torch.empty(max(lay.n_chunks + (lay.n_chunks & 1), 2), dtype=torch.int16, device=x.device),
+                                torch.empty(lay.n_tiles + 1, dtype=torch.int64, device=x.device), lay)
+        p = _EncodeParams(lay.chunk_pixels, lay.pixel_splits)
+        tensors.append(t); params.append(p); result.append(out)
+        items[i] = _EncodeItem(model.ptr, cb.ptr, C.addressof(t), C.addressof(p), out.words.data_ptr(), out.words.numel(),
+                               out.chunk_len.data_ptr(), out.tile_off.data_ptr())
+    _check(load_library().tc_encode_many(ctx.ptr, items, n, _stream_ptr(ctx.device)), "tc_encode_many")
+    return result
+
+
+def tc_decode_many(ctx: Context, layers, *, outs=None, relu: bool = False):
+    """Decode several tensors in one call: `layers` is a list of (model, codebook, enc, shape, dtype)."""
+    n = len(layers)
+    tensors, params, items = [], [], (_DecodeItem * max(n, 1))()
+    result = []
+    for i, (model, cb, enc, shape, dtype) in enumerate(layers):
+        out = outs[i] if outs is not None else torch.empty(shape, dtype=dtype, device=enc.words.device)
+        t = _tensor(out)
+        p = _EncodeParams(enc.layout.chunk_pixels, enc.layout.pixel_splits, int(relu), 0)
+        tensors.append(t); params.append(p); result.append(out)
+        items[i] = _DecodeItem(model.ptr, cb.ptr, enc.words.data_ptr(), enc.words.numel(), enc.chunk_len.data_ptr(),
+                               enc.tile_off.data_ptr(), C.addressof(p), C.addressof(t))
+    _check(load_library().tc_decode_many(ctx.ptr, items, n, _stream_ptr(ctx.device)), "tc_decode_many")
+    return result
 
 
 def tc_roundtrip_host(ctx: Context, model: Model, cb: Codebook, x_host: torch.Tensor, out_host: torch.Tensor, *,

@@ -293,6 +293,11 @@ void tc_destroy(tc_ctx *ctx)
         if (ctx->ev_out[i]) cudaEventDestroy(ctx->ev_out[i]);
     }
     if (ctx->chunk_bits) cudaFreeHost(ctx->chunk_bits);
+    for (int i = 0; i < 4; ++i) {
+        if (ctx->many_streams[i]) cudaStreamDestroy(ctx->many_streams[i]);
+        if (ctx->many_join[i]) cudaEventDestroy(ctx->many_join[i]);
+    }
+    if (ctx->many_fork) cudaEventDestroy(ctx->many_fork);
     for (tc_codebook *cb : ctx->stats_cb) tc_codebook_free(cb);
     if (ctx->d_status) cudaFree(ctx->d_status);
     delete ctx;
@@ -750,11 +755,12 @@ void tc_codebook_free(tc_codebook *cb)
 tc_status tc_encode_with_scratch(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const tc_tensor *x, int chunk_pixels,
                                  int splits, void *stream_out, size_t capacity, uint16_t *chunk_len, uint64_t *tile_off,
                                  const tc_debug_out *debug, void *scratch, uint8_t *sym_scratch, cudaStream_t s,
-                                 unsigned long long *hist, unsigned long long *clamped)
+                                 unsigned long long *hist, unsigned long long *clamped, bool scratch_is_zero)
 {
     const long long pixels = (long long)x->n * x->h * x->w;
     const long long n_tiles = (pixels + TC_TILE_PIXELS - 1) / TC_TILE_PIXELS;
-    TC_CUDA(cudaMemsetAsync(scratch, 0, kEncodeScratchHeader + (size_t)n_tiles * sizeof(unsigned long long), s));
+    if (!scratch_is_zero)
+        TC_CUDA(cudaMemsetAsync(scratch, 0, kEncodeScratchHeader + (size_t)n_tiles * sizeof(unsigned long long), s));
 
     EncodeArgs a{};
     a.x = x->data; a.n = x->n; a.c = x->c; a.hw = x->h * x->w; a.k = m->k; a.bits = m->bits; a.groups = cb->groups;
@@ -857,9 +863,19 @@ tc_status tc_encode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
                                   ctx->scratch, parallel_exact ? (uint8_t *)ctx->scratch + lookback : nullptr, s);
 }
 
-tc_status tc_decode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const void *stream, size_t stream_bytes,
-                    const uint16_t *chunk_len, const uint64_t *tile_off, const tc_encode_params *params,
-                    const tc_tensor *x_hat, void *cuda_stream)
+// Bytes of symbol scratch a decode of `x_hat` may need: small tensors on the exact kernels park
+// their symbols there (whether that route is taken is decided at launch).
+static size_t decode_scratch_bytes(const tc_ctx *ctx, const tc_model *m, const tc_tensor *x_hat)
+{
+    const long long pixels = (long long)x_hat->n * x_hat->h * x_hat->w;
+    const long long n_tiles = (pixels + TC_TILE_PIXELS - 1) / TC_TILE_PIXELS;
+    return n_tiles < (long long)kExactParallelTilesPerSm * ctx->sm_count ? (((size_t)pixels * m->k + 255) & ~(size_t)255) : 0;
+}
+
+// tc_decode with the symbol scratch named by the caller (decode_scratch_bytes of it, or nullptr)
+static tc_status decode_with_scratch(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const void *stream, size_t stream_bytes,
+                                     const uint16_t *chunk_len, const uint64_t *tile_off, const tc_encode_params *params,
+                                     const tc_tensor *x_hat, uint8_t *sym_scratch, void *cuda_stream)
 {
     if (!ctx) return TC_ERR_INVALID_ARG;
     tc_status st = check_codec_args(m, cb, x_hat);
@@ -916,15 +932,161 @@ tc_status tc_decode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const
         return tc_launch_decode_simt_fp32(ctx, a, (cudaStream_t)cuda_stream);
     }
     ctx->last_decode_path = 0;
-    if (a.n_tiles < (long long)kExactParallelTilesPerSm * ctx->sm_count) {
+    if (sym_scratch && a.n_tiles < (long long)kExactParallelTilesPerSm * ctx->sm_count) {
         // few pixels: the per-pixel kernel only decodes the symbols (into the context's arena), the
         // inverse transform runs with one thread per (pixel, channel) -- same arithmetic, same results
-        if ((st = ensure_scratch(ctx, (size_t)pixels * m->k)) != TC_OK) return st;
-        a.sym_out = (uint8_t *)ctx->scratch;
+        a.sym_out = sym_scratch;
         if ((st = tc_launch_decode_simt(ctx, a, x_hat->dtype, (cudaStream_t)cuda_stream)) != TC_OK) return st;
         return tc_launch_reconstruct(a, x_hat->dtype, a.sym_out, (cudaStream_t)cuda_stream);
     }
     return tc_launch_decode_simt(ctx, a, x_hat->dtype, (cudaStream_t)cuda_stream);
+}
+
+tc_status tc_decode(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const void *stream, size_t stream_bytes,
+                    const uint16_t *chunk_len, const uint64_t *tile_off, const tc_encode_params *params,
+                    const tc_tensor *x_hat, void *cuda_stream)
+{
+    if (!ctx || !m || !valid_tensor(x_hat)) return TC_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    const size_t scratch = decode_scratch_bytes(ctx, m, x_hat);
+    if (scratch) {
+        const tc_status st = ensure_scratch(ctx, scratch);
+        if (st != TC_OK) return st;
+    }
+    return decode_with_scratch(ctx, m, cb, stream, stream_bytes, chunk_len, tile_off, params, x_hat,
+                               scratch ? (uint8_t *)ctx->scratch : nullptr, cuda_stream);
+}
+
+// ---- several tensors per call --------------------------------------------------------------------
+
+static tc_status ensure_many_streams(tc_ctx *ctx)
+{
+    if (ctx->many_fork) return TC_OK;
+    for (int i = 0; i < 4; ++i) {
+        TC_CUDA(cudaStreamCreateWithFlags(&ctx->many_streams[i], cudaStreamNonBlocking));
+        TC_CUDA(cudaEventCreateWithFlags(&ctx->many_join[i], cudaEventDisableTiming));
+    }
+    TC_CUDA(cudaEventCreateWithFlags(&ctx->many_fork, cudaEventDisableTiming));
+    return TC_OK;
+}
+
+// Items in descending order of work: the large ones start first, each on its own stream.
+static std::vector<int> by_descending_work(int n, const std::vector<double> &work)
+{
+    std::vector<int> order(n);
+    for (int i = 0; i < n; ++i) order[i] = i;
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return work[a] > work[b]; });
+    return order;
+}
+
+tc_status tc_encode_many(tc_ctx *ctx, const tc_encode_item *items, int32_t n_items, void *cuda_stream)
+{
+    if (!ctx || n_items < 0 || (n_items > 0 && !items)) return TC_ERR_INVALID_ARG;
+    if (n_items == 0) return TC_OK;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    // every item is checked before anything is launched
+    std::vector<ChunkShape> shape(n_items);
+    std::vector<size_t> lookback_at(n_items), symbols_at(n_items, 0);
+    std::vector<double> work(n_items);
+    size_t lookback_total = 0, total = 0;
+    for (int i = 0; i < n_items; ++i) {
+        const tc_encode_item &it = items[i];
+        if (!it.tile_off) return TC_ERR_INVALID_ARG;
+        const tc_status st = check_codec_args(it.model, it.codebook, it.x);
+        if (st != TC_OK) return st;
+        if (!resolve_chunks(it.params, it.model->k, it.codebook->max_len, &shape[i])) return TC_ERR_INVALID_ARG;
+        const long long pixels = (long long)it.x->n * it.x->h * it.x->w;
+        if (pixels > 0 && (!it.stream_out || !it.chunk_len)) return TC_ERR_INVALID_ARG;
+        if (((uintptr_t)it.stream_out & 15u) != 0 || ((uintptr_t)it.chunk_len & 3u) != 0) return TC_ERR_INVALID_ARG;
+        const long long n_tiles = (pixels + TC_TILE_PIXELS - 1) / TC_TILE_PIXELS;
+        lookback_at[i] = lookback_total;
+        lookback_total += (kEncodeScratchHeader + (size_t)n_tiles * sizeof(unsigned long long) + 255) & ~(size_t)255;
+        work[i] = (double)pixels * it.x->c;
+    }
+    total = lookback_total;
+    for (int i = 0; i < n_items; ++i) {
+        const tc_encode_item &it = items[i];
+        const long long pixels = (long long)it.x->n * it.x->h * it.x->w;
+        const long long n_tiles = (pixels + TC_TILE_PIXELS - 1) / TC_TILE_PIXELS;
+        if (n_tiles > 0 && n_tiles < (long long)kExactParallelTilesPerSm * ctx->sm_count) {
+            symbols_at[i] = total;
+            total += ((size_t)pixels * it.model->k + 255) & ~(size_t)255;
+        }
+    }
+    tc_status st = ensure_scratch(ctx, total);
+    if (st != TC_OK) return st;
+    if ((st = ensure_many_streams(ctx)) != TC_OK) return st;
+    // one clear for the look-back state of all items, then the items fan out over the streams
+    TC_CUDA(cudaMemsetAsync(ctx->scratch, 0, lookback_total, s));
+    TC_CUDA(cudaEventRecord(ctx->many_fork, s));
+    const int n_streams = std::min(4, (int)n_items);
+    for (int j = 0; j < n_streams; ++j) TC_CUDA(cudaStreamWaitEvent(ctx->many_streams[j], ctx->many_fork, 0));
+    const std::vector<int> order = by_descending_work(n_items, work);
+    tc_status first_error = TC_OK;
+    for (int r = 0; r < n_items; ++r) {
+        const int i = order[r];
+        const tc_encode_item &it = items[i];
+        cudaStream_t ws = ctx->many_streams[r % n_streams];
+        const long long pixels = (long long)it.x->n * it.x->h * it.x->w;
+        if (pixels == 0) { if (cudaMemsetAsync(it.tile_off, 0, sizeof(uint64_t), ws) != cudaSuccess && first_error == TC_OK) first_error = TC_ERR_CUDA; continue; }
+        st = tc_encode_with_scratch(ctx, it.model, it.codebook, it.x, shape[i].cp, shape[i].splits, it.stream_out, it.capacity,
+                                    it.chunk_len, it.tile_off, nullptr, (char *)ctx->scratch + lookback_at[i],
+                                    symbols_at[i] ? (uint8_t *)ctx->scratch + symbols_at[i] : nullptr, ws, nullptr, nullptr, true);
+        if (st != TC_OK && first_error == TC_OK) first_error = st;
+    }
+    for (int j = 0; j < n_streams; ++j) {
+        TC_CUDA(cudaEventRecord(ctx->many_join[j], ctx->many_streams[j]));
+        TC_CUDA(cudaStreamWaitEvent(s, ctx->many_join[j], 0));
+    }
+    return first_error;
+}
+
+tc_status tc_decode_many(tc_ctx *ctx, const tc_decode_item *items, int32_t n_items, void *cuda_stream)
+{
+    if (!ctx || n_items < 0 || (n_items > 0 && !items)) return TC_ERR_INVALID_ARG;
+    if (n_items == 0) return TC_OK;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    std::vector<size_t> symbols_at(n_items, 0), symbols_bytes(n_items, 0);
+    std::vector<double> work(n_items);
+    size_t total = 0;
+    for (int i = 0; i < n_items; ++i) {
+        const tc_decode_item &it = items[i];
+        const tc_status st = check_codec_args(it.model, it.codebook, it.x_hat);
+        if (st != TC_OK) return st;
+        ChunkShape cs;
+        if (!resolve_chunks(it.params, it.model->k, it.codebook->max_len, &cs)) return TC_ERR_INVALID_ARG;
+        const long long pixels = (long long)it.x_hat->n * it.x_hat->h * it.x_hat->w;
+        if (pixels > 0 && (!it.stream || !it.chunk_len || !it.tile_off || ((uintptr_t)it.stream & 15u) != 0 ||
+                           ((uintptr_t)it.chunk_len & 3u) != 0))
+            return TC_ERR_INVALID_ARG;
+        symbols_bytes[i] = decode_scratch_bytes(ctx, it.model, it.x_hat);
+        symbols_at[i] = total;
+        total += symbols_bytes[i];
+        work[i] = (double)pixels * it.x_hat->c;
+    }
+    tc_status st;
+    if (total && (st = ensure_scratch(ctx, total)) != TC_OK) return st;
+    if ((st = ensure_many_streams(ctx)) != TC_OK) return st;
+    TC_CUDA(cudaEventRecord(ctx->many_fork, s));
+    const int n_streams = std::min(4, (int)n_items);
+    for (int j = 0; j < n_streams; ++j) TC_CUDA(cudaStreamWaitEvent(ctx->many_streams[j], ctx->many_fork, 0));
+    const std::vector<int> order = by_descending_work(n_items, work);
+    tc_status first_error = TC_OK;
+    for (int r = 0; r < n_items; ++r) {
+        const int i = order[r];
+        const tc_decode_item &it = items[i];
+        st = decode_with_scratch(ctx, it.model, it.codebook, it.stream, it.stream_bytes, it.chunk_len, it.tile_off, it.params,
+                                 it.x_hat, symbols_bytes[i] ? (uint8_t *)ctx->scratch + symbols_at[i] : nullptr,
+                                 ctx->many_streams[r % n_streams]);
+        if (st != TC_OK && first_error == TC_OK) first_error = st;
+    }
+    for (int j = 0; j < n_streams; ++j) {
+        TC_CUDA(cudaEventRecord(ctx->many_join[j], ctx->many_streams[j]));
+        TC_CUDA(cudaStreamWaitEvent(s, ctx->many_join[j], 0));
+    }
+    return first_error;
 }
 
 tc_status tc_roundtrip_host(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const void *x_host, void *x_hat_host,

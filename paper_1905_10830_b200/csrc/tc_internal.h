@@ -36,6 +36,9 @@ struct tc_ctx {
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
     cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
     unsigned long long *chunk_bits = nullptr;   // pinned HOST [kMaxRoundtripChunks]
+    // tc_encode_many / tc_decode_many spread their items over these streams (created at first use)
+    cudaStream_t many_streams[4] = {nullptr, nullptr, nullptr, nullptr};
+    cudaEvent_t many_fork = nullptr, many_join[4] = {nullptr, nullptr, nullptr, nullptr};
     int force_exact = 0;                  // 1: route every tensor through the fp64 kernels; 2: skip the resident-basis kernels; 3: skip the run-skipping decoder
     int last_encode_path = 0;             // 0 = fp64 kernels, 1 = tensor-core kernels (resident basis), 2 = fp32 kernels, 3 = tensor-core kernels (streamed basis)
     int last_decode_path = 0;
@@ -147,7 +150,7 @@ constexpr size_t kEncodeScratchHeader = 64;   // ticket counter, padded; the per
 tc_status tc_encode_with_scratch(tc_ctx *ctx, const tc_model *m, const tc_codebook *cb, const tc_tensor *x, int chunk_pixels,
                                  int splits, void *stream_out, size_t capacity, uint16_t *chunk_len, uint64_t *tile_off,
                                  const tc_debug_out *debug, void *scratch, uint8_t *sym_scratch, cudaStream_t s,
-                                 unsigned long long *hist = nullptr, unsigned long long *clamped = nullptr);
+                                 unsigned long long *hist = nullptr, unsigned long long *clamped = nullptr, bool scratch_is_zero = false);
 // tensors of fewer tiles than this many per SM take the one-thread-per-value exact kernels
 constexpr int kExactParallelTilesPerSm = 2;
 

@@ -119,6 +119,61 @@ def run(cfgs, reps, with_oracle, max_batch):
     return rows, peak
 
 
+def layer_sets(cfgs, reps, max_batch):
+    """Configurations with several layers: the whole set coded by one tc_encode_many / tc_decode_many
+    call each, against the same layers coded by one call per layer (queued back to back)."""
+    ctx = tc.tc_create(0)
+    out = []
+    for cfg in cfgs:
+        w = fm.workload(cfg)
+        if sum(w.repeats) < 2 or w.per_channel_codebook:
+            continue
+        bits = w.bits[0]
+        batch = min(w.batch, max_batch)
+        layers = []
+        for spec, repeat in zip(w.layers, w.repeats):
+            params = fm.layer_params(spec)
+            cal = fm.make_maps(params, w.calib_maps, calib=True, dtype=w.dtype, device="cuda")
+            model = tc.tc_fit_pca(ctx, cal, bits=bits)
+            st = tc.tc_stats(ctx, model, None, cal)
+            cb = tc.tc_build_codebook(ctx, model, st.hist)
+            for r in range(repeat):
+                layers.append((model, cb, fm.make_maps(params, batch, dtype=w.dtype, device="cuda", offset=1000 * r)))
+            del cal
+        encs = tc.tc_encode_many(ctx, layers)
+        dec_layers = [(m, cb, e, x.shape, x.dtype) for (m, cb, x), e in zip(layers, encs)]
+        outs = tc.tc_decode_many(ctx, dec_layers)
+
+        def enc_each():
+            for (m, cb, x), e in zip(layers, encs):
+                tc.tc_encode(ctx, m, cb, x, out=e)
+
+        def dec_each():
+            for (m, cb, e, shape, dtype), o in zip(dec_layers, outs):
+                tc.tc_decode(ctx, m, cb, e, shape, dtype, out=o)
+
+        raw = sum(x.numel() * x.element_size() for _, _, x in layers)
+        row = dict(cfg=cfg, name=w.name, layers=len(layers), batch=batch, bits=bits, raw_mb=raw / 1e6,
+                   enc_many=_time(lambda: tc.tc_encode_many(ctx, layers, outs=encs), reps),
+                   dec_many=_time(lambda: tc.tc_decode_many(ctx, dec_layers, outs=outs), reps),
+                   enc_each=_time(enc_each, reps), dec_each=_time(dec_each, reps))
+        assert tc.tc_get_status(ctx) == 0
+        out.append(row)
+        del layers, encs, outs, dec_layers
+        torch.cuda.empty_cache()
+    return out
+
+
+def layer_sets_markdown(rows):
+    out = ["", "Whole layer sets in one call (`tc_encode_many` / `tc_decode_many`) against one call per layer, queued back to back:", "",
+           "| cfg | layers | N | b | raw MB | encode: many ms | per layer ms | decode: many ms | per layer ms | round trip GB/s (many) |",
+           "|---|---|---|---|---|---|---|---|---|---|"]
+    for r in rows:
+        out.append(f"| {r['cfg']} | {r['layers']} | {r['batch']} | {r['bits']} | {r['raw_mb']:.1f} | {r['enc_many']:.3f} | {r['enc_each']:.3f} | "
+                   f"{r['dec_many']:.3f} | {r['dec_each']:.3f} | {r['raw_mb'] / (r['enc_many'] + r['dec_many']) / 1e3 * 1e3:.1f} |")
+    return "\n".join(out)
+
+
 def _time_back_to_back(fn, calls=20):
     """Milliseconds per call when `calls` calls are queued one after the other (one event pair
     around all of them): what a layer costs inside a pipeline that does not wait between layers."""
@@ -160,6 +215,9 @@ def main():
     args = ap.parse_args()
     rows, peak = run(args.cfg, args.reps, not args.no_oracle, args.max_batch)
     md = to_markdown(rows, peak, not args.no_oracle)
+    sets = layer_sets(args.cfg, args.reps, args.max_batch)
+    if sets:
+        md += "\n" + layer_sets_markdown(sets)
     print(md)
     if args.out:
         with open(args.out, "w") as f:
