@@ -797,6 +797,8 @@ tc_status tc_encode_with_scratch(tc_ctx *ctx, const tc_model *m, const tc_codebo
         // entropy coder of the per-pixel kernel on those symbols -- same arithmetic, same results
         tc_status st = tc_launch_project_quantise(a, x->dtype, sym_scratch, s);
         if (st != TC_OK) return st;
+        if (tc_pack_symbols_parts(a) > 0 && ((uintptr_t)sym_scratch & 15u) == 0)
+            return tc_launch_pack_symbols(a, sym_scratch, s);      // several threads per pixel code the symbols
         a.sym_in = sym_scratch;
     }
     return tc_launch_encode_simt(ctx, a, x->dtype, s);
@@ -935,9 +937,8 @@ static tc_status decode_with_scratch(tc_ctx *ctx, const tc_model *m, const tc_co
     if (sym_scratch && a.n_tiles < (long long)kExactParallelTilesPerSm * ctx->sm_count) {
         // few pixels: the per-pixel kernel only decodes the symbols (into the context's arena), the
         // inverse transform runs with one thread per (pixel, channel) -- same arithmetic, same results
-        a.sym_out = sym_scratch;
-        if ((st = tc_launch_decode_simt(ctx, a, x_hat->dtype, (cudaStream_t)cuda_stream)) != TC_OK) return st;
-        return tc_launch_reconstruct(a, x_hat->dtype, a.sym_out, (cudaStream_t)cuda_stream);
+        if ((st = tc_launch_unpack_symbols(a, sym_scratch, (cudaStream_t)cuda_stream)) != TC_OK) return st;
+        return tc_launch_reconstruct(a, x_hat->dtype, sym_scratch, (cudaStream_t)cuda_stream);
     }
     return tc_launch_decode_simt(ctx, a, x_hat->dtype, (cudaStream_t)cuda_stream);
 }

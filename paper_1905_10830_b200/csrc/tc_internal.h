@@ -160,6 +160,9 @@ tc_status tc_launch_decode_simt(const tc_ctx *ctx, const DecodeArgs &a, int dtyp
 tc_status tc_launch_encode_simt_fp32(const tc_ctx *ctx, const EncodeArgs &a, cudaStream_t s);
 tc_status tc_launch_decode_simt_fp32(const tc_ctx *ctx, const DecodeArgs &a, cudaStream_t s);
 tc_status tc_launch_project_quantise(const EncodeArgs &a, int dtype, uint8_t *sym, cudaStream_t s);
+int tc_pack_symbols_parts(const EncodeArgs &a);
+tc_status tc_launch_unpack_symbols(const DecodeArgs &a, uint8_t *sym, cudaStream_t s);
+tc_status tc_launch_pack_symbols(const EncodeArgs &a, const uint8_t *sym, cudaStream_t s);
 tc_status tc_launch_reconstruct(const DecodeArgs &a, int dtype, const uint8_t *sym, cudaStream_t s);
 bool tc_encode_tc_supported(const tc_ctx *ctx, const EncodeArgs &a);
 tc_status tc_launch_encode_tc(const tc_ctx *ctx, const EncodeArgs &a, cudaStream_t s);
