@@ -44,7 +44,8 @@ def check_symbols(q_gpu, o, *, exact: bool):
         assert not bad.any(), f"{bad.sum()} symbols differ on the exact path"
         return 0.0
     rate = bad.mean()
-    assert rate <= 1e-4, f"symbol mismatch rate {rate}"
+    # at most 1e-4 of the symbols; a tensor of fewer than 10 000 symbols may still have one (a tie is a tie)
+    assert bad.sum() <= max(1, int(np.ceil(1e-4 * bad.size))), f"symbol mismatch rate {rate}"
     if bad.any():
         assert np.all(np.abs(diff[bad]) == 1)
         frac = np.abs(units[bad] - np.floor(units[bad]) - 0.5)
