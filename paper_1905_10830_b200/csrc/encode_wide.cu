@@ -74,7 +74,11 @@ __device__ __forceinline__ uint32_t quantise_bits(uint32_t acc_bits, float inv_s
 
 // kTma: the basis pieces arrive by tiled TMA copies (one instruction per stage, 64-byte swizzle)
 // instead of 1024 cp.async copies; `bmap` is then the tensor map of the basis.
-template <bool kPerChannel, bool kDebug, bool kTma>
+// kSymOnly: projection and quantiser only.  A tensor of few tiles leaves most SMs without work,
+// and a tile of a wide layer takes long; in this mode the unit dealt over the blocks is one
+// block of 256 coefficients of one tile, the symbols go to a.sym_park ([P][K] bytes) and the
+// entropy coder runs afterwards as a kernel of its own, several threads per pixel.
+template <bool kPerChannel, bool kDebug, bool kTma, bool kSymOnly>
 __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, int smem_budget,
                                                                   const __grid_constant__ CUtensorMap bmap)
 {
@@ -89,7 +93,7 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nsym = 1 << a.bits;
-    const int enc_entries = kPerChannel ? 0 : nsym;
+    const int enc_entries = (kPerChannel || a.groups != 1) ? 0 : nsym;   // the launcher sizes shared memory by the same rule
     const SmemLayout L = smem_layout(a.k, enc_entries, smem_budget);
     const int stages = L.stages;
     const uint32_t ring_addr = smem_u32(smem + L.ring);
@@ -119,7 +123,9 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
     tc_fence_after_sync();
     const uint32_t tmem_base = s_tmem_base;
 
-    const long long my_tiles = (a.n_tiles > blockIdx.x) ? (a.n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    // units dealt over the blocks: whole tiles, or (tile, coefficient block) pairs
+    const long long n_units = kSymOnly ? a.n_tiles * n_blocks : a.n_tiles;
+    const long long my_tiles = (n_units > blockIdx.x) ? (n_units - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
 
     if (warp >= kLoaderWarp0 && warp < kMmaWarp) {
         // ================= loaders =================
@@ -147,7 +153,9 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
         int it = 0;
         bool alive = true;
         for (long long tl = 0; tl < my_tiles && alive; ++tl) {
-            const long long tile = blockIdx.x + tl * gridDim.x;
+            const long long unit = blockIdx.x + tl * gridDim.x;
+            const long long tile = kSymOnly ? unit / n_blocks : unit;
+            const int nb_lo = kSymOnly ? (int)(unit - tile * n_blocks) : 0, nb_hi = kSymOnly ? nb_lo + 1 : n_blocks;
             const long long p0 = tile * TC_TILE_PIXELS + 4 * mg;
             const bool valid = p0 < a.pixels;
             const long long img = valid ? p0 / a.hw : 0;
@@ -158,7 +166,7 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
             const long long img1 = valid1 ? p1 / a.hw : 0;
             const unsigned short *a_src1 = reinterpret_cast<const unsigned short *>(xin) + img1 * a.c * (long long)a.hw +
                                            (valid1 ? p1 - img1 * a.hw : 0) + (long long)(16 * ch_half) * a.hw;
-            for (int nb = 0; nb < n_blocks && alive; ++nb) {
+            for (int nb = nb_lo; nb < nb_hi && alive; ++nb) {
                 const int j0 = nb * kBlockCoef;
                 const int ncols = min(kBlockCoef, a.k - j0);
                 const __nv_bfloat16 *b_src = b_src0 + (long long)j0 * a.c;
@@ -227,7 +235,9 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
             long long work = 0;                                // (tile, block) pairs issued so far
             bool alive = true;
             for (long long tl = 0; tl < my_tiles && alive; ++tl) {
-                for (int nb = 0; nb < n_blocks && alive; ++nb, ++work) {
+                const long long unit = blockIdx.x + tl * gridDim.x;
+                const int nb_lo = kSymOnly ? (int)(unit % n_blocks) : 0, nb_hi = kSymOnly ? nb_lo + 1 : n_blocks;
+                for (int nb = nb_lo; nb < nb_hi && alive; ++nb, ++work) {
                     const int acc = (int)(work & 1);
                     if (!mbar_wait(smem_u32(&s_tempty[acc]), (uint32_t)(((work >> 1) & 1) ^ 1))) { alive = false; break; }
                     tc_fence_after_sync();
@@ -283,14 +293,18 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
         bool alive = true;
 
         for (long long tl = 0; tl < my_tiles && alive; ++tl) {
-            const long long tile = blockIdx.x + tl * gridDim.x;
+            const long long unit = blockIdx.x + tl * gridDim.x;
+            const long long tile = kSymOnly ? unit / n_blocks : unit;
+            const int nb_lo = kSymOnly ? (int)(unit - tile * n_blocks) : 0, nb_hi = kSymOnly ? nb_lo + 1 : n_blocks;
             const long long p = tile * TC_TILE_PIXELS + m;
             const bool valid = p < a.pixels;
-            s_part[part * TC_TILE_PIXELS + m] = 0u;
-            named_bar_sync(kEpiBar, kEpiThreads);  // the previous tile's symbols have been packed; the sums are zero
+            if constexpr (!kSymOnly) {
+                s_part[part * TC_TILE_PIXELS + m] = 0u;
+                named_bar_sync(kEpiBar, kEpiThreads);  // the previous tile's symbols have been packed; the sums are zero
+            }
 
             // pass 1: quantise block by block, park the symbols, add up the code lengths
-            for (int nb = 0; nb < n_blocks && alive; ++nb, ++work) {
+            for (int nb = nb_lo; nb < nb_hi && alive; ++nb, ++work) {
                 const int acc = (int)(work & 1);
                 if (!mbar_wait(smem_u32(&s_tfull[acc]), (uint32_t)((work >> 1) & 1))) { alive = false; break; }
                 tc_fence_after_sync();
@@ -313,7 +327,8 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
                         const uint32_t vb = quantise_bits(r[i], inv_step, biasv[i], vmax);
-                        if constexpr (kPerChannel) bits16 += __ldg(a.enc + (j0 + i) * nsym + (vb & 0xffu)) & 0xffu;
+                        if constexpr (kSymOnly) {
+                        } else if constexpr (kPerChannel) bits16 += __ldg(a.enc + (j0 + i) * nsym + (vb & 0xffu)) & 0xffu;
                         else {
                             uint32_t l;
                             asm("ld.shared.u8 %0, [%1];" : "=r"(l) : "r"(vb + len8_rel));
@@ -325,18 +340,26 @@ __global__ void __launch_bounds__(kThreads, 1) encode_wide_kernel(EncodeArgs a, 
                         }
                         r[i] = vb;
                     }
+                    uint32_t packed[4];
 #pragma unroll
                     for (int i = 0; i < 16; i += 4)          // low bytes of four values -> one word
-                        s_symq[((j0 + i) >> 2) * TC_TILE_PIXELS + m] =
-                            __byte_perm(__byte_perm(r[i], r[i + 1], 0x0040), __byte_perm(r[i + 2], r[i + 3], 0x0040), 0x5410);
-                    const int run = (j0 >= bnd[1] ? 1 : 0) + (j0 >= bnd[2] ? 1 : 0) + (j0 >= bnd[3] ? 1 : 0);
-                    if (valid) atomicAdd(&s_part[run * TC_TILE_PIXELS + m], bits16);
+                        packed[i >> 2] = __byte_perm(__byte_perm(r[i], r[i + 1], 0x0040), __byte_perm(r[i + 2], r[i + 3], 0x0040), 0x5410);
+                    if constexpr (kSymOnly) {
+                        // sixteen symbols of the pixel's row of [P][K] (K and j0 are multiples of 16)
+                        if (valid) *reinterpret_cast<uint4 *>(a.sym_park + p * a.k + j0) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) s_symq[((j0 >> 2) + i) * TC_TILE_PIXELS + m] = packed[i];
+                        const int run = (j0 >= bnd[1] ? 1 : 0) + (j0 >= bnd[2] ? 1 : 0) + (j0 >= bnd[3] ? 1 : 0);
+                        if (valid) atomicAdd(&s_part[run * TC_TILE_PIXELS + m], bits16);
+                    }
                 }
                 // the accumulator is free for the block after next
                 tc_fence_before_sync();
                 mbar_arrive(smem_u32(&s_tempty[acc]));
             }
             if (!alive) break;
+            if constexpr (kSymOnly) continue;      // offsets and packing belong to the kernel that follows
             named_bar_sync(kEpiBar, kEpiThreads);  // every run's sum is complete
 
             // bit offsets: pixel-major, runs in order inside a pixel
@@ -462,15 +485,19 @@ tc_status tc_launch_encode_wide(const tc_ctx *ctx, const EncodeArgs &a, cudaStre
     if (l.stages < 2) return TC_ERR_UNSUPPORTED;
     const bool per_channel = a.groups != 1, debug = a.dbg_coef || a.dbg_sym;
     const bool tma = a.basis_map != nullptr;
+    const bool sym_only = a.sym_park != nullptr;
     void (*kernel)(EncodeArgs, int, const CUtensorMap) =
-        tma ? (per_channel ? (debug ? encode_wide_kernel<true, true, true> : encode_wide_kernel<true, false, true>)
-                           : (debug ? encode_wide_kernel<false, true, true> : encode_wide_kernel<false, false, true>))
-            : (per_channel ? (debug ? encode_wide_kernel<true, true, false> : encode_wide_kernel<true, false, false>)
-                           : (debug ? encode_wide_kernel<false, true, false> : encode_wide_kernel<false, false, false>));
+        sym_only ? (tma ? (debug ? encode_wide_kernel<false, true, true, true> : encode_wide_kernel<false, false, true, true>)
+                        : (debug ? encode_wide_kernel<false, true, false, true> : encode_wide_kernel<false, false, false, true>))
+        : tma ? (per_channel ? (debug ? encode_wide_kernel<true, true, true, false> : encode_wide_kernel<true, false, true, false>)
+                           : (debug ? encode_wide_kernel<false, true, true, false> : encode_wide_kernel<false, false, true, false>))
+            : (per_channel ? (debug ? encode_wide_kernel<true, true, false, false> : encode_wide_kernel<true, false, false, false>)
+                           : (debug ? encode_wide_kernel<false, true, false, false> : encode_wide_kernel<false, false, false, false>));
     const size_t smem_bytes = (size_t)l.total + 1024;         // room to align the buffer to 1 KB
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
         return TC_ERR_CUDA;
-    const unsigned int grid = (unsigned int)((a.n_tiles < ctx->sm_count) ? a.n_tiles : ctx->sm_count);
+    const long long n_units = sym_only ? a.n_tiles * ((a.k + kBlockCoef - 1) / kBlockCoef) : a.n_tiles;
+    const unsigned int grid = (unsigned int)((n_units < ctx->sm_count) ? n_units : ctx->sm_count);
     EncodeArgs args = a;
     int budget_arg = budget;
     CUtensorMap map_arg;

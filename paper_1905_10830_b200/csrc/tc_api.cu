@@ -785,6 +785,15 @@ tc_status tc_encode_with_scratch(tc_ctx *ctx, const tc_model *m, const tc_codebo
     }
     if (ctx->force_exact != 1 && x->dtype == TC_BF16 && tc_encode_wide_supported(ctx, a)) {   // wide layers, unaligned rows
         ctx->last_encode_path = 3;
+        if (sym_scratch && n_tiles < ctx->sm_count && ((uintptr_t)sym_scratch & 15u) == 0 && tc_pack_symbols_parts(a) > 0) {
+            // fewer tiles than SMs: the projection is dealt over the SMs by blocks of coefficients and leaves
+            // the symbols in the arena, the entropy coder follows as a kernel of its own (same stream)
+            a.sym_park = sym_scratch;
+            const tc_status st = tc_launch_encode_wide(ctx, a, s);
+            if (st != TC_OK) return st;
+            a.sym_park = nullptr;
+            return tc_launch_pack_symbols(a, sym_scratch, s);
+        }
         return tc_launch_encode_wide(ctx, a, s);
     }
     if (ctx->force_exact != 1 && x->dtype == TC_BF16 && x->c % 2 == 0) {      // shapes the tensor-core kernel does not take
