@@ -235,7 +235,8 @@ void tc_codebook_free(tc_codebook *cb);
  * from `counts` (weights counts + 1).  HOST pointers.  No device needed. */
 tc_status tc_host_huffman_lengths(const uint64_t *counts, int32_t nsym, int32_t max_length,
                                   uint8_t *lengths);
-/* The fit's device eigensolver on its own: `a` is a symmetric n x n matrix in DEVICE memory
+/* The fit's device eigensolver on its own (Section 3.1, "Linear transform": the PCA matrix is
+ * the eigenvector matrix of the calibration covariance): `a` is a symmetric n x n matrix in DEVICE memory
  * (fp64, row-major, left untouched), evals [n] and evecs [n][n] DEVICE arrays, with the same
  * conventions as tc_host_eigh.  One-sided Jacobi, one launch per round of n / 2 disjoint
  * column pairs; synchronises the stream once per sweep.  *sweeps (HOST, may be NULL) receives
