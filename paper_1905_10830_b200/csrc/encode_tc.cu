@@ -373,6 +373,7 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
             uint32_t sym[kPair ? kMaxHalfCols / 8 : kMaxHalfCols / 4];   // one byte per symbol, or per pair of symbols
             uint32_t blk_bits[kMaxHalfCols / 64] = {};          // code bits of each block of 16 symbols, one byte each
             unsigned int my_bits = 0, bits_first = 0;          // bits_first: the first half of this thread's coefficients
+            [[maybe_unused]] unsigned int n_clamped = 0;       // statistics mode: coefficients outside the quantiser's range
 #pragma unroll
             for (int blk = 0; blk < kMaxHalfCols / 16; ++blk) {
                 if (blk * 16 < ncols) {
@@ -389,25 +390,16 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
 #pragma unroll
                     for (int i = 0; i < 16; i += 2) quantise_bits2(r[i], r[i + 1], inv_range, biasv[i], biasv[i + 1], top, qv[i], qv[i + 1]);
                     if constexpr (kHist) {
+                        // every symbol other than the zero level is counted; the zero level's count is what
+                        // is left of the pixels, which the caller works out
                         const uint32_t modal_bits = kMagicBits + (uint32_t)a.hist_modal;
-                        unsigned int n_clamped = 0;
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
                             const int j = col0 + blk * 16 + i;
-                            const bool other = valid && qv[i] != modal_bits;
-                            const unsigned int others = __ballot_sync(0xffffffffu, other);
-                            const unsigned int live = __ballot_sync(0xffffffffu, valid);
-                            if (lane == 0 && live != others)
-                                atomicAdd(a.hist + (size_t)j * nsym + a.hist_modal, (unsigned long long)__popc(live & ~others));
-                            if (other) atomicAdd(a.hist + (size_t)j * nsym + (qv[i] & 0xffu), 1ull);
+                            if (valid && qv[i] != modal_bits) atomicAdd(a.hist + (size_t)j * nsym + (qv[i] & 0xffu), 1ull);
                             // outside the quantiser's range [lo, lo + (2^b - 1) step]
                             const float t = fmaf(__uint_as_float(r[i]), inv_range, biasv[i]);
                             n_clamped += (valid && (t < 0.f || t > 1.f)) ? 1u : 0u;
-                        }
-                        if (a.clamped) {
-#pragma unroll
-                            for (int d = 16; d > 0; d >>= 1) n_clamped += __shfl_xor_sync(0xffffffffu, n_clamped, d);
-                            if (lane == 0 && n_clamped) atomicAdd(a.clamped, (unsigned long long)n_clamped);
                         }
                     }
 #pragma unroll
@@ -450,6 +442,13 @@ __global__ void __launch_bounds__(kThreads, 1) encode_tc_kernel(EncodeArgs a)
             // the accumulator buffer is free for the tile after next
             tc_fence_before_sync();
             mbar_arrive(smem_u32(&s_tempty[grp]));
+            if constexpr (kHist) {
+                if (a.clamped) {
+#pragma unroll
+                    for (int d = 16; d > 0; d >>= 1) n_clamped += __shfl_xor_sync(0xffffffffu, n_clamped, d);
+                    if (lane == 0 && n_clamped) atomicAdd(a.clamped, (unsigned long long)n_clamped);
+                }
+            }
             if (!valid) my_bits = 0;
 
             // bit offsets: pixel-major, first half before second half

@@ -1268,6 +1268,14 @@ static tc_status stats_tensor_core(tc_ctx *ctx, const tc_model *m, const tc_code
     TC_CUDA(cudaMemcpyAsync(&zeros, d_zeros, 8, cudaMemcpyDeviceToHost, s));
     TC_CUDA(cudaMemcpyAsync(&clamped, d_clamped, 8, cudaMemcpyDeviceToHost, s));
     TC_CUDA(cudaStreamSynchronize(s));
+    // the encoder counts every symbol but the zero level (m->center): that one takes the rest of the pixels
+    const unsigned long long pixels = (unsigned long long)x->n * hw;
+    for (int j = 0; j < m->k; ++j) {
+        unsigned long long others = 0;
+        for (int q = 0; q < nsym; ++q)
+            if (q != m->center) others += hist[(size_t)j * nsym + q];
+        hist[(size_t)j * nsym + m->center] = pixels - others;
+    }
     return TC_OK;
 }
 

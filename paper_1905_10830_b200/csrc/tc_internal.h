@@ -110,8 +110,8 @@ struct EncodeArgs {
     int emit;                         // 0: symbols only (statistics mode)
     const uint8_t *sym_in;            // exact kernels: non-null = the symbols [P][K] are given, skip the projection
     uint8_t *sym_park;                // streaming encoder: non-null = leave the symbols [P][K] here and stop (the entropy coder runs as a kernel of its own)
-    unsigned long long *hist;         // tensor-core encoder, statistics: non-null = per-coefficient symbol counts [K][2^bits] are added here
-    int hist_modal;                   // the symbol most lanes are expected to hold (counted once per warp): the zero level
+    unsigned long long *hist;         // tensor-core encoder, statistics: non-null = per-coefficient counts [K][2^bits] of every symbol but hist_modal are added here
+    int hist_modal;                   // the symbol of the zero level, which most coefficients hold: statistics mode counts all the others
 };
 
 struct DecodeArgs {
