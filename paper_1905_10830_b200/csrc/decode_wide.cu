@@ -64,10 +64,10 @@ struct SmemLayout {
     bool staged;                                              // room for the segment buffer beside at least three stages
 };
 
-__host__ __device__ inline SmemLayout smem_layout(int c, int k, int lut_entries, int budget, int groups = 1)
+__host__ __device__ inline SmemLayout smem_layout(int c, int k, int lut_entries, int budget, int groups = 1, int item_pixels = 0)
 {
     SmemLayout l;
-    l.np = ((c + 127) / 128 <= 4) ? 128 : 64;
+    l.np = item_pixels ? item_pixels : ((c + 127) / 128 <= 4) ? 128 : 64;
     l.bop_bytes = 2u * (uint32_t)k * (uint32_t)l.np;
     l.start_bytes = (kMaxTileChunks + 8) * 4u;
     const uint32_t fixed = (uint32_t)groups * (l.bop_bytes + l.start_bytes) + (uint32_t)lut_entries * 4u + 16u + 8u * kTrWarpBytes;
@@ -114,7 +114,7 @@ __global__ void __launch_bounds__(Roles<G>::kThreads, 1) decode_wide_kernel(Deco
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int lut_size = 1 << a.lut_bits;
-    const SmemLayout L = smem_layout(a.c, a.k, kPerChannel ? 0 : lut_size, a.smem_budget, G);
+    const SmemLayout L = smem_layout(a.c, a.k, kPerChannel ? 0 : lut_size, a.smem_budget, G, a.item_pixels);
     const int stages = L.stages, NP = L.np;
     const uint32_t ring_addr = smem_u32(smem + L.ring);
     uint32_t *s_lut = reinterpret_cast<uint32_t *>(smem + L.lut);
@@ -515,8 +515,20 @@ tc_status tc_launch_decode_wide(const tc_ctx *ctx, const DecodeArgs &a, cudaStre
     DecodeArgs args = a;
     args.smem_budget = ctx->max_smem_optin - 2048;            // leaves room for the static shared variables and the alignment
     const int groups = decode_wide_groups(ctx, a);
-    const SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, args.smem_budget, groups);
+    SmemLayout l = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, args.smem_budget, groups);
     if (l.stages < 2) return TC_ERR_UNSUPPORTED;
+    // A tensor of few tiles leaves most SMs without a work item: smaller items (64 or 32 pixels, as
+    // long as a chunk still lies inside one) spread it over more of them.  Every item streams the
+    // whole basis, so this only pays while there are fewer items than SMs.
+    args.item_pixels = 0;
+    if (groups == 1) {
+        int np = l.np;
+        while (np > 32 && np / 2 >= a.chunk_pixels && a.n_tiles * (TC_TILE_PIXELS / np) * 2 <= ctx->sm_count) np /= 2;
+        if (np != l.np) {
+            const SmemLayout l2 = smem_layout(a.c, a.k, a.groups == 1 ? (1 << a.lut_bits) : 0, args.smem_budget, groups, np);
+            if (l2.stages >= 2) { l = l2; args.item_pixels = np; }
+        }
+    }
     const bool tma = a.basis_t_map != nullptr, pc = a.groups != 1;
     void (*kernel)(DecodeArgs, const CUtensorMap) =
         groups == 2 ? (pc ? decode_wide_kernel<true, true, 2> : decode_wide_kernel<false, true, 2>)

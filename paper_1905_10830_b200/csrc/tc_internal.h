@@ -138,6 +138,7 @@ struct DecodeArgs {
     int dense_head;                     // run-skipping decoder: leading coefficients that are too often non-modal for run skipping to pay
     int relu;                           // x_hat = max(x_hat, 0) before it is rounded to the tensor type
     int smem_budget;                    // shared memory the tensor-core kernel may lay out (set by its launcher)
+    int item_pixels;                    // streaming decoder: pixels per work item chosen by its launcher (0: the layout's default)
     const double *basis64;
     const double *mean64;
     double lo, step;
