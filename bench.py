@@ -310,60 +310,87 @@ def main():
     stream_bytes = total_bits // 8
     side_bytes = lay.chunk_len_bytes + lay.tile_off_bytes
     test_stats = tc.tc_stats(ctx, model, cb, x[: min(batch, 256)], groups=1, want_hist=False)
+    status = tc.tc_get_status(ctx)
+    if status != 0:
+        raise SystemExit(f"codec reported status {status} in the statistics pass")
     tc.tc_force_exact_path(ctx, args.route)
 
     def step():
         tc.tc_encode(ctx, model, cb, x, out=enc, **chunking)
         tc.tc_decode(ctx, model, cb, enc, x.shape, x.dtype, out=xhat, stream_bytes=stream_bytes)
 
-    for _ in range(args.warmup):
-        step()
-    torch.cuda.synchronize()
+    class CodecStatus(Exception):
+        pass
 
-    # ---- timed region: K steps, CUDA events on the launching stream ----------------------
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
-    sampler = ClockSampler(local_rank)
-    if dist is not None:
-        dist.barrier()
-    torch.cuda.synchronize()
-    sampler.start()
-    t_begin = torch.cuda.Event(enable_timing=True)
-    t_end = torch.cuda.Event(enable_timing=True)
-    t_begin.record()
-    for i in range(args.steps):
-        ev[i][0].record()
-        tc.tc_encode(ctx, model, cb, x, out=enc, **chunking)
-        ev[i][1].record()
-        tc.tc_decode(ctx, model, cb, enc, x.shape, x.dtype, out=xhat, stream_bytes=stream_bytes)
-        ev[i][2].record()
-    t_end.record()
-    torch.cuda.synchronize()
-    if dist is not None:
-        dist.barrier()
-    clocks = sampler.stop()
-    total_ms = t_begin.elapsed_time(t_end)
-    # ---- sustained: the same step back to back for at least two seconds, clocks sampled meanwhile ----
-    sustained = None
-    if args.sustained_seconds > 0:
-        n_sus = max(args.steps, int(args.sustained_seconds * 1e3 / max(total_ms / args.steps, 1e-3)) + 1)
-        sus_sampler = ClockSampler(local_rank)
-        torch.cuda.synchronize()
-        sus_sampler.start()
-        s_begin, s_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        s_begin.record()
-        for _ in range(n_sus):
+    def measure():
+        """Warm-up, the K timed steps and the sustained run; raises CodecStatus if the library's status
+        word was set meanwhile."""
+        for _ in range(args.warmup):
             step()
-        s_end.record()
         torch.cuda.synchronize()
-        sus_clocks = sus_sampler.stop()
-        sus_ms = s_begin.elapsed_time(s_end)
-        sus_bytes, sus_ms = sharding.aggregate(raw_bytes * n_sus, sus_ms, dev)
-        sustained = {"seconds": sus_ms * 1e-3, "steps": n_sus, "ms_per_step": sus_ms / n_sus,
-                     "value": sus_bytes / (sus_ms * 1e-3) / 1e9, "unit": UNIT, "clocks": sus_clocks}
-    enc_ms = [ev[i][0].elapsed_time(ev[i][1]) for i in range(args.steps)]
-    dec_ms = [ev[i][1].elapsed_time(ev[i][2]) for i in range(args.steps)]
-    if tc.tc_get_status(ctx) != 0:
-        raise SystemExit("codec reported an error during the timed region")
+
+        # ---- timed region: K steps, CUDA events on the launching stream ----------------------
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+        sampler = ClockSampler(local_rank)
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        sampler.start()
+        t_begin = torch.cuda.Event(enable_timing=True)
+        t_end = torch.cuda.Event(enable_timing=True)
+        t_begin.record()
+        for i in range(args.steps):
+            ev[i][0].record()
+            tc.tc_encode(ctx, model, cb, x, out=enc, **chunking)
+            ev[i][1].record()
+            tc.tc_decode(ctx, model, cb, enc, x.shape, x.dtype, out=xhat, stream_bytes=stream_bytes)
+            ev[i][2].record()
+        t_end.record()
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        clocks = sampler.stop()
+        total_ms = t_begin.elapsed_time(t_end)
+        # ---- sustained: the same step back to back for at least two seconds, clocks sampled meanwhile ----
+        sustained = None
+        if args.sustained_seconds > 0:
+            n_sus = max(args.steps, int(args.sustained_seconds * 1e3 / max(total_ms / args.steps, 1e-3)) + 1)
+            sus_sampler = ClockSampler(local_rank)
+            torch.cuda.synchronize()
+            sus_sampler.start()
+            s_begin, s_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s_begin.record()
+            for _ in range(n_sus):
+                step()
+            s_end.record()
+            torch.cuda.synchronize()
+            sus_clocks = sus_sampler.stop()
+            sus_ms = s_begin.elapsed_time(s_end)
+            sus_bytes, sus_ms = sharding.aggregate(raw_bytes * n_sus, sus_ms, dev)
+            sustained = {"seconds": sus_ms * 1e-3, "steps": n_sus, "ms_per_step": sus_ms / n_sus,
+                         "value": sus_bytes / (sus_ms * 1e-3) / 1e9, "unit": UNIT, "clocks": sus_clocks}
+        enc_ms = [ev[i][0].elapsed_time(ev[i][1]) for i in range(args.steps)]
+        dec_ms = [ev[i][1].elapsed_time(ev[i][2]) for i in range(args.steps)]
+        status = tc.tc_get_status(ctx)
+        if status != 0:
+            raise CodecStatus(status)
+        return clocks, total_ms, sustained, enc_ms, dec_ms
+
+    # A status word set inside the measured loops ends the attempt.  On one GPU the whole measurement
+    # is then taken once more and the line says so ("retried"); a second failure, or any failure
+    # with several ranks (they could not agree on a retry without another exchange), ends the run.
+    retried = None
+    try:
+        clocks, total_ms, sustained, enc_ms, dec_ms = measure()
+    except CodecStatus as e:
+        if world > 1:
+            raise SystemExit(f"codec reported status {e.args[0]} during the measurement")
+        retried = {"status": int(e.args[0])}
+        print(f"bench: codec status {e.args[0]} during the measurement, measuring once more", file=sys.stderr)
+        try:
+            clocks, total_ms, sustained, enc_ms, dec_ms = measure()
+        except CodecStatus as e2:
+            raise SystemExit(f"codec reported status {e2.args[0]} during the measurement (second attempt)")
     # whole job: bytes summed over ranks, device time as the max over ranks
     job_bytes, total_ms = sharding.aggregate(raw_bytes * args.steps, total_ms, dev)
 
@@ -445,6 +472,8 @@ def main():
     }
     if sustained is not None:
         line["sustained"] = sustained
+    if retried is not None:
+        line["retried"] = retried          # a first attempt ended with the library's status word set
     if e2e is not None:
         line["e2e"] = e2e
     if not args.no_cpu_baseline and world == 1:

@@ -189,7 +189,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_runs_kernel(DecodeArgs a)
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) unsigned long long s_empty[2][kMaxPanels], s_tfull[2];
     __shared__ uint32_t s_tmem_base;
-    __shared__ unsigned int s_wsum[2][2][4];   // [group][thread set][warp]: bits per warp, for the start positions
+    // [group][tile parity][thread set][warp]: bits per warp, for the start positions.  Two copies: a warp
+    // that is done with its tile early writes the next tile's sum while a slower warp may still
+    // be reading this tile's; the group's barrier (one per tile) only orders the write after next.
+    __shared__ unsigned int s_wsum[2][2][2][4];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int lut_size = 1 << a.lut_bits;
@@ -341,7 +344,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_runs_kernel(DecodeArgs a)
                     const unsigned int up = __shfl_up_sync(0xffffffffu, inc, d);
                     if (lane >= d) inc += up;
                 }
-                if (lane == 31) s_wsum[grp][set][wq] = inc;
+                if (lane == 31) s_wsum[grp][li & 1][set][wq] = inc;
                 cp_async_wait<0>();
                 // every thread's part of this tile's segment has landed, and every thread is done
                 // with the tile before: its stream buffer may take the next tile's segment
@@ -352,7 +355,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_runs_kernel(DecodeArgs a)
                 const int n_wq = (n_work / tpp + 31) / 32;          // warps of one thread set
 #pragma unroll
                 for (int w = 0; w < 4; ++w) {
-                    const unsigned int sw = w < n_wq ? s_wsum[grp][set][w] : 0u;
+                    const unsigned int sw = w < n_wq ? s_wsum[grp][li & 1][set][w] : 0u;
                     if (w < wq) before += sw;
                     tile_total += sw;
                 }

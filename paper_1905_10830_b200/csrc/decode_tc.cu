@@ -214,7 +214,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) unsigned long long s_full[2][kMaxSlots], s_empty[2][kMaxSlots], s_tfull[2], s_tempty[2];
     __shared__ uint32_t s_tmem_base;
-    __shared__ unsigned int s_wsum[2][2][4];   // [group][half][warp]: chunk bits per warp, for the start positions
+    // [group][tile parity][half][warp]: chunk bits per warp, for the start positions.  Two copies: a warp
+    // that is done with its tile early writes the next tile's sum while a slower warp may still be
+    // reading this tile's; the group's barriers only order the write after next.
+    __shared__ unsigned int s_wsum[2][2][2][4];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int lut_size = 1 << a.lut_bits;
@@ -361,13 +364,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_tc_kernel(DecodeArgs a)
                 const unsigned int up = __shfl_up_sync(0xffffffffu, inc, d);
                 if (lane >= d) inc += up;
             }
-            if (lane == 31) s_wsum[grp][sub][wq] = inc;
+            if (lane == 31) s_wsum[grp][li & 1][sub][wq] = inc;
             named_bar_sync(bar_id, n_thr);           // every thread's part of this tile's segment has landed
             const TileInfo after = tile_info(tl + 4); // offsets two tiles ahead: their latency hides behind the decode
             unsigned int before = 0, tile_total = 0;
 #pragma unroll
             for (int w = 0; w < 4; ++w) {
-                const unsigned int sw = s_wsum[grp][sub][w];
+                const unsigned int sw = s_wsum[grp][li & 1][sub][w];
                 if (w < wq) before += sw;
                 tile_total += sw;
             }
