@@ -265,6 +265,9 @@ tc_status tc_host_eigh(double *a, int32_t n, double *evals, double *evecs);
  *     inside a tile the chunks follow one another without gaps, so a chunk starts at its
  *     tile's start plus the lengths of the tile's earlier chunks.  A chunk may not exceed
  *     65535 bits: chunk_pixels * K / pixel_splits * (longest code) must stay below that.
+ *   - Defaults (chunk_pixels = pixel_splits = 0): the smallest chunk_pixels that gives a chunk at
+ *     least 96 symbols; from 256 coefficients on two chunks per pixel (K a multiple of 32),
+ *     from 512 on four (K a multiple of 64).  tc_encode_bound reports what will be used.
  * ------------------------------------------------------------------------------------- */
 typedef struct {
     int32_t chunk_pixels; /* power of two in 1..128; 0 = library default for this shape   */

@@ -76,7 +76,8 @@ bool valid_tensor(const tc_tensor *t)
 }
 
 // Chunk shape: `cp` pixels per chunk, or `splits` chunks per pixel when cp == 1.  Defaults
-// keep the side information at 16 bits per 128 to 255 symbols (about 0.1 bit per value).
+// keep the side information at 16 bits per 96 to 255 symbols (0.06 to 0.17 bit per value): a chunk is
+// one decoder thread's work, and a tile of 128 pixels wants as many of them as the rate allows.
 struct ChunkShape {
     int cp, splits;
     long long chunks(long long pixels) const { return splits > 1 ? pixels * splits : (pixels + cp - 1) / cp; }
@@ -86,7 +87,7 @@ bool resolve_chunks(const tc_encode_params *p, int k, int max_len, ChunkShape *o
 {
     int cp = 1;
     if (p && p->chunk_pixels) cp = p->chunk_pixels;
-    else while (cp < TC_TILE_PIXELS && cp * k < 128) cp <<= 1;
+    else while (cp < TC_TILE_PIXELS && cp * k < 96) cp <<= 1;       // at least 96 symbols per chunk: 16 bits of side information per 96 .. 255 symbols
     if (cp < 1 || cp > TC_TILE_PIXELS || (cp & (cp - 1)) != 0) return false;
     // default: a chunk of 128 .. 255 symbols where the shape allows it -- two chunks per pixel
     // from 256 coefficients, four from 512

@@ -160,9 +160,10 @@ def test_pixel_splits_exact_path(ctx, splits):
 
 
 def test_default_chunk_shapes(ctx):
-    # side information stays at 16 bits per 128..255 symbols: K = 16 -> 8 pixels per chunk,
-    # K = 64 -> 2, K = 128 -> 1, K = 256 -> two chunks per pixel, K = 512 -> four
-    for c, want in ((16, (8, 1)), (64, (2, 1)), (128, (1, 1)), (256, (1, 2)), (384, (1, 2)), (512, (1, 4)), (960, (1, 4))):
+    # side information stays at 16 bits per 96..255 symbols: K = 16 -> 8 pixels per chunk, K = 48 and
+    # K = 64 -> 2, K = 96 and K = 128 -> 1, K = 256 -> two chunks per pixel, K = 512 -> four
+    for c, want in ((16, (8, 1)), (48, (2, 1)), (64, (2, 1)), (96, (1, 1)), (128, (1, 1)), (256, (1, 2)), (384, (1, 2)),
+                    (512, (1, 4)), (960, (1, 4))):
         spec = fm.LayerSpec(c, 4, 4, 0.9, None, 90 + c)
         o = H.oracle_side(spec, 4, 4, 1, torch.bfloat16, False)
         model_h = H.import_model(tc, ctx, o["model"], torch.bfloat16)
