@@ -72,7 +72,7 @@ def _parity(ctx, model, cb, x_sample, bits, per_channel):
     flips = "-"
     if dtype == torch.bfloat16:       # how many outputs the fp32 accumulation may round to the neighbouring value (tests/helpers.py)
         from tests import helpers as H
-        flips = f"{int((got != want).sum())} / {H.flip_allowance(H.expected_output_flips(m, q_gpu))}"
+        flips = f"{H.count_output_flips(got, want)} / {H.flip_allowance(H.expected_output_flips(m, q_gpu))}"
     return dict(stream_exact=stream_exact, coef_err=coef_err, mismatch=float(bad.mean()), ties_only=ties_only,
                 xhat_equal=float((got == want).mean()), flips=flips)
 

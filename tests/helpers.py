@@ -94,3 +94,16 @@ def flip_allowance(expected: float) -> int:
     deviations of a Poisson count of that mean, plus one."""
     lam = 2.0 * expected
     return int(np.ceil(lam + 4.5 * np.sqrt(lam) + 1.0))
+
+
+def count_output_flips(got: np.ndarray, want: np.ndarray, channel_axis: int = 1) -> int:
+    """Reconstructed values that differ from the oracle's, counted once per (channel, oracle value):
+    pixels whose symbols agree (at a low bit width: all at the zero level) share one exact value per
+    channel, and if that value sits on an output rounding boundary they all land on the neighbouring
+    number together -- one event of the model above, however many pixels show it."""
+    diff = got != want
+    if not diff.any():
+        return 0
+    idx = np.nonzero(diff)
+    pairs = np.stack([idx[channel_axis].astype(np.float64), want[diff].astype(np.float64)], axis=1)
+    return int(np.unique(pairs, axis=0).shape[0])

@@ -92,7 +92,7 @@ def test_two_layer_chain_calibrated_layer_by_layer():
         got = r_gpu.float().cpu().numpy()
         ulp = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(want), 1e-30))) - 7)
         assert np.all(np.abs(got - want) <= np.maximum(1e-3 * np.maximum(np.abs(want), m.step), ulp))
-        assert int((got != want).sum()) <= H.flip_allowance(H.expected_output_flips(m, q_gpu))
+        assert H.count_output_flips(got, want) <= H.flip_allowance(H.expected_output_flips(m, q_gpu))
 
     # ---- layer 2 was calibrated on layer 1's reconstruction ------------------------------------
     g2 = tc.tc_model_export(layers[1].model)

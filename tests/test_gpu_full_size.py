@@ -66,7 +66,7 @@ def _check_tiles(ctx, model_desc, lengths, bits, x, enc, xhat, tiles):
         got = xhat[i0:i1].float().cpu().numpy().transpose(0, 2, 3, 1).reshape(-1, c)[p0 - i0 * hw: p1 - i0 * hw]
         ulp = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(want), 1e-30))) - 7)
         assert np.all(np.abs(got - want) <= np.maximum(1e-3 * np.maximum(np.abs(want), m.step), ulp))
-        flips += int((got != want).sum())
+        flips += H.count_output_flips(got, want, channel_axis=1)
         expected += H.expected_output_flips(m, q_stream)
     # values that land on the neighbouring bf16 number: no more than the fp32 arithmetic explains
     assert flips <= H.flip_allowance(expected), f"{flips} values differ, {expected:.1f} expected"
