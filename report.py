@@ -31,6 +31,14 @@ def _peak():
     return 6650.0
 
 
+def _tensor_peak():
+    """Measured bf16 matmul rate in TFLOP/s (the burst figure: these kernels are timed alone)."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        return float(json.load(open(path))["bf16_tflops"])
+    return 1590.0
+
+
 def _time(fn, reps):
     fn()
     torch.cuda.synchronize()
@@ -105,6 +113,11 @@ def run(cfgs, reps, with_oracle, max_batch):
                 assert tc.tc_get_status(ctx) == 0
                 side = enc.layout.chunk_len_bytes + enc.layout.tile_off_bytes
                 algo = raw + nbytes + side
+                # which roofline binds the layer: bytes at the copy bandwidth, or the projection's
+                # 2 P C K flops at the matmul rate (the wide layers), and how close each kernel comes
+                flops = 2.0 * (values / spec.c) * spec.c * spec.c                  # K = C in every configuration
+                t_hbm, t_tensor = algo / (peak * 1e9) * 1e3, flops / (_tensor_peak() * 1e12) * 1e3      # ms
+                bound, t_ideal = ("tensor", t_tensor) if t_tensor > t_hbm else ("hbm", t_hbm)
                 tst = tc.tc_stats(ctx, model, cb, x[: min(batch, 64)], groups=groups, want_hist=False)
                 row = dict(cfg=cfg, layer=spec.name + (f" x{repeat}" if repeat > 1 else ""), batch=batch, dtype=str(w.dtype).split(".")[-1],
                            b=bits, entropy=tst.entropy, huffman=tst.mean_length, stream=8 * nbytes / values,
@@ -112,6 +125,7 @@ def run(cfgs, reps, with_oracle, max_batch):
                            enc_gbs=raw / t_enc / 1e6, dec_gbs=raw / t_dec / 1e6, rt_gbs=raw / (t_enc + t_dec) / 1e6,
                            enc_ms=t_enc, dec_ms=t_dec, q_enc_ms=q_enc, q_dec_ms=q_dec, enc_frac=algo / t_enc / 1e6 / peak, dec_frac=algo / t_dec / 1e6 / peak,
                            enc_frac8=algo / t_enc / 1e6 / 8000, dec_frac8=algo / t_dec / 1e6 / 8000,
+                           bound=bound, enc_bound_frac=t_ideal / t_enc, dec_bound_frac=t_ideal / t_dec,
                            kernels=["fp64", "tcgen05", "fp32", "tcgen05-stream"][tc.tc_last_path(ctx, False)] + "/" + ["fp64", "tcgen05", "fp32", "tcgen05-stream"][tc.tc_last_path(ctx, True)])
                 if with_oracle:
                     row.update(_parity(ctx, model, cb, x[: max(1, min(batch, 2))].contiguous(), bits, w.per_channel_codebook))
@@ -194,14 +208,16 @@ def _time_back_to_back(fn, calls=20):
 
 def to_markdown(rows, peak, with_oracle):
     head = ["cfg", "layer", "N", "dtype", "b", "entropy", "Huffman", "stream+pad", "+offsets", "MSE", "enc ms", "dec ms", "enc / dec ms queued x20", "enc GB/s", "dec GB/s",
-            "round trip GB/s", f"HBM frac enc/dec (of {peak:.0f} GB/s measured)", "(of 8000 GB/s)", "kernels enc/dec"]
+            "round trip GB/s", f"HBM frac enc/dec (of {peak:.0f} GB/s measured)", "(of 8000 GB/s)",
+            f"binding roofline (bytes at the copy rate, or 2PCK flops at {_tensor_peak():.0f} TF/s measured)", "frac of it enc/dec", "kernels enc/dec"]
     if with_oracle:
         head += ["stream bit-exact", "coef max rel err", "symbol mismatch", "only at ties", "x_hat bit-equal", "x_hat values off by one / allowed"]
     out = ["| " + " | ".join(head) + " |", "|" + "---|" * len(head)]
     for r in rows:
         cells = [r["cfg"], r["layer"], r["batch"], r["dtype"], r["b"], f"{r['entropy']:.3f}", f"{r['huffman']:.3f}", f"{r['stream']:.3f}",
                  f"{r['total']:.3f}", f"{r['mse']:.3g}", f"{r['enc_ms']:.3f}", f"{r['dec_ms']:.3f}", f"{r['q_enc_ms']:.3f} / {r['q_dec_ms']:.3f}", f"{r['enc_gbs']:.1f}", f"{r['dec_gbs']:.1f}",
-                 f"{r['rt_gbs']:.1f}", f"{r['enc_frac']:.3f} / {r['dec_frac']:.3f}", f"{r['enc_frac8']:.3f} / {r['dec_frac8']:.3f}", r["kernels"]]
+                 f"{r['rt_gbs']:.1f}", f"{r['enc_frac']:.3f} / {r['dec_frac']:.3f}", f"{r['enc_frac8']:.3f} / {r['dec_frac8']:.3f}",
+                 r["bound"], f"{r['enc_bound_frac']:.3f} / {r['dec_bound_frac']:.3f}", r["kernels"]]
         if with_oracle:
             cells += ["yes" if r["stream_exact"] else "NO", f"{r['coef_err']:.1e}", f"{r['mismatch']:.1e}", "yes" if r["ties_only"] else "NO",
                       f"{r['xhat_equal']:.5f}", r["flips"]]
